@@ -1,0 +1,199 @@
+"""CPU oracle of the per-decode-step KVCache retrieval path -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package.  It shares no code with the CUDA library and never imports it.
+
+The arithmetic lives in ``swarm_oracle.cpp`` (plain C++, double accumulation); this
+module compiles it with g++ on first use and exposes thin numpy wrappers.  bf16 tensors
+travel as ``uint16`` arrays holding the raw bits.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "swarm_oracle.cpp")
+_LIB = os.path.join(_HERE, "libswarm_oracle.so")
+
+ORDER_BY_ID = 1
+UNIT_LOAD = 2
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (OpenMP) next to its source; returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["g++", "-O2", "-std=c++17", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra", "-o", tmp, _SRC]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        for name in ("oracle_build_summaries", "oracle_scores", "oracle_topk", "oracle_resolve",
+                     "oracle_gather", "oracle_attention", "oracle_set_threads"):
+            getattr(_lib, name).restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+def _arr(x, dtype):
+    a = np.ascontiguousarray(x, dtype=dtype)
+    return a
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise ValueError(f"{what}: oracle status {rc} (1 bad argument, 2 bad table entry, 3 non-finite)")
+
+
+def set_threads(n: int) -> int:
+    """Set the OpenMP thread count (n <= 0 only queries); returns the count in effect."""
+    return int(_load().oracle_set_threads(ctypes.c_int(n)))
+
+
+def build_summaries(kv_pool, page_base, ctx_len, Hkv, d, S):
+    """kv_pool uint16 [pages][Hkv][2][S][d] -> ksum uint16 [pages][Hkv][2][d] (min, max over valid tokens)."""
+    kv_pool = _arr(kv_pool, np.uint16)
+    page_base = _arr(page_base, np.int64)
+    ctx_len = _arr(ctx_len, np.int32)
+    n_pages = kv_pool.size // (Hkv * 2 * S * d)
+    ksum = np.zeros((n_pages, Hkv, 2, d), dtype=np.uint16)
+    rc = _load().oracle_build_summaries(_p(kv_pool), _p(page_base), _p(ctx_len), ctypes.c_int32(len(ctx_len)),
+                                        ctypes.c_int32(Hkv), ctypes.c_int32(d), ctypes.c_int32(S), _p(ksum))
+    _check(rc, "build_summaries")
+    return ksum
+
+
+def scores(q, ksum, page_base, ctx_len, Hkv, S, Pmax):
+    """q uint16 [B][Hq][d]; returns (score64 [B][Hq][Pmax], score32, cond); entries p >= P_b are -inf / 0."""
+    q = _arr(q, np.uint16)
+    ksum = _arr(ksum, np.uint16)
+    page_base = _arr(page_base, np.int64)
+    ctx_len = _arr(ctx_len, np.int32)
+    B, Hq, d = q.shape
+    s64 = np.full((B, Hq, Pmax), -np.inf, dtype=np.float64)
+    s32 = np.full((B, Hq, Pmax), -np.inf, dtype=np.float32)
+    cond = np.zeros((B, Hq, Pmax), dtype=np.float64)
+    rc = _load().oracle_scores(_p(q), _p(ksum), _p(page_base), _p(ctx_len), ctypes.c_int32(B), ctypes.c_int32(Hq),
+                               ctypes.c_int32(Hkv), ctypes.c_int32(d), ctypes.c_int32(S), ctypes.c_int64(Pmax),
+                               _p(s64), _p(s32), _p(cond))
+    _check(rc, "scores")
+    return s64, s32, cond
+
+
+def topk(score, ctx_len, S, k):
+    """score float32 [B][Hq][Pmax] -> (sel int32 [B][Hq][k] ascending page id, -1 padded; n_sel [B][Hq])."""
+    score = _arr(score, np.float32)
+    ctx_len = _arr(ctx_len, np.int32)
+    B, Hq, Pmax = score.shape
+    sel = np.empty((B, Hq, k), dtype=np.int32)
+    n_sel = np.empty((B, Hq), dtype=np.int32)
+    rc = _load().oracle_topk(_p(score), _p(ctx_len), ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(S),
+                             ctypes.c_int64(Pmax), ctypes.c_int32(k), _p(sel), _p(n_sel))
+    _check(rc, "topk")
+    return sel, n_sel
+
+
+def resolve(sel, n_sel, page_base, page2cluster, cluster_base, replica_mask, cluster_size, D, flags=0):
+    """Returns (uniq int32 [n_uniq] ascending global cluster id, queue_of uint8 [n_uniq], load int32 [D])."""
+    sel = _arr(sel, np.int32)
+    n_sel = _arr(n_sel, np.int32)
+    page_base = _arr(page_base, np.int64)
+    page2cluster = _arr(page2cluster, np.int32)
+    cluster_base = _arr(cluster_base, np.int64)
+    replica_mask = _arr(replica_mask, np.uint32)
+    cluster_size = _arr(cluster_size, np.uint16)
+    B, Hq, k = sel.shape
+    cap = max(int(cluster_base[-1]), 1)
+    uniq = np.empty(cap, dtype=np.int32)
+    queue_of = np.empty(cap, dtype=np.uint8)
+    n_uniq = np.zeros(1, dtype=np.int32)
+    load = np.zeros(D, dtype=np.int32)
+    rc = _load().oracle_resolve(_p(sel), _p(n_sel), _p(page_base), _p(page2cluster), _p(cluster_base),
+                                _p(replica_mask), _p(cluster_size), ctypes.c_int32(B), ctypes.c_int32(Hq),
+                                ctypes.c_int32(k), ctypes.c_int32(D), ctypes.c_uint32(flags), _p(uniq), _p(queue_of),
+                                _p(n_uniq), _p(load))
+    _check(rc, "resolve")
+    n = int(n_uniq[0])
+    return uniq[:n].copy(), queue_of[:n].copy(), load
+
+
+def gather(kv_pool, sel, n_sel, page_base, ctx_len, Hkv, d, S):
+    """Returns (k_g, v_g uint16 [B][Hq][k*S][d] zero padded, n_tok int32 [B][Hq])."""
+    kv_pool = _arr(kv_pool, np.uint16)
+    sel = _arr(sel, np.int32)
+    n_sel = _arr(n_sel, np.int32)
+    page_base = _arr(page_base, np.int64)
+    ctx_len = _arr(ctx_len, np.int32)
+    B, Hq, k = sel.shape
+    k_g = np.empty((B, Hq, k * S, d), dtype=np.uint16)
+    v_g = np.empty((B, Hq, k * S, d), dtype=np.uint16)
+    n_tok = np.empty((B, Hq), dtype=np.int32)
+    rc = _load().oracle_gather(_p(kv_pool), _p(sel), _p(n_sel), _p(page_base), _p(ctx_len), ctypes.c_int32(B),
+                               ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(d), ctypes.c_int32(S),
+                               ctypes.c_int32(k), _p(k_g), _p(v_g), _p(n_tok))
+    _check(rc, "gather")
+    return k_g, v_g, n_tok
+
+
+def attention(q, k_g, v_g, n_tok):
+    """q uint16 [B][Hq][d], k_g/v_g uint16 [B][Hq][rows][d] -> (out float64 [B][Hq][d], lse float64 [B][Hq])."""
+    q = _arr(q, np.uint16)
+    k_g = _arr(k_g, np.uint16)
+    v_g = _arr(v_g, np.uint16)
+    n_tok = _arr(n_tok, np.int32)
+    B, Hq, d = q.shape
+    rows = k_g.shape[2]
+    out = np.empty((B, Hq, d), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    rc = _load().oracle_attention(_p(q), _p(k_g), _p(v_g), _p(n_tok), ctypes.c_int32(B), ctypes.c_int32(Hq),
+                                  ctypes.c_int32(d), ctypes.c_int64(rows), _p(out), _p(lse))
+    _check(rc, "attention")
+    return out, lse
+
+
+@dataclass
+class StepResult:
+    score64: np.ndarray
+    score32: np.ndarray
+    cond: np.ndarray
+    sel: np.ndarray
+    n_sel: np.ndarray
+    uniq: np.ndarray
+    queue_of: np.ndarray
+    load: np.ndarray
+    k_g: np.ndarray
+    v_g: np.ndarray
+    n_tok: np.ndarray
+    out: np.ndarray
+    lse: np.ndarray
+
+
+def step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base, replica_mask, cluster_size, *, Hkv, S, k,
+         D, Pmax, flags=0, sel_override=None) -> StepResult:
+    """The whole path, stage after stage.  ``sel_override=(sel, n_sel)`` replaces the oracle's own selection
+    for the downstream stages (stage-conditional parity)."""
+    d = np.asarray(q).shape[-1]
+    s64, s32, cond = scores(q, ksum, page_base, ctx_len, Hkv, S, Pmax)
+    sel, n_sel = topk(s32, ctx_len, S, k)
+    use_sel, use_n = (sel, n_sel) if sel_override is None else sel_override
+    uniq, queue_of, load = resolve(use_sel, use_n, page_base, page2cluster, cluster_base, replica_mask,
+                                   cluster_size, D, flags)
+    k_g, v_g, n_tok = gather(kv_pool, use_sel, use_n, page_base, ctx_len, Hkv, d, S)
+    out, lse = attention(q, k_g, v_g, n_tok)
+    return StepResult(s64, s32, cond, sel, n_sel, uniq, queue_of, load, k_g, v_g, n_tok, out, lse)
