@@ -1,0 +1,191 @@
+/* swarm.h -- C ABI of the B200 (sm_100a) KVCache retrieval hot path.
+ *
+ * One decode step of one layer, for a batch of requests whose KV cache lives in a paged
+ * pool in device memory:
+ *   (1) score every page of every request against the query (page upper bound over per-page
+ *       min/max key summaries),
+ *   (2) keep the top_k pages per query head,
+ *   (3) map the selected pages to co-activation clusters, merge duplicates and route every
+ *       cluster to the least loaded of the queues that hold a replica of it,
+ *   (4) gather the selected pages' K/V and run single-row attention over them.
+ *
+ * Conventions that hold for every entry point unless stated otherwise:
+ *   - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned.  The library
+ *     allocates no device memory, frees nothing of the caller's and never synchronises the host
+ *     (exceptions are named below: swarm_device_status and swarm_step_host).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it and the call returns at once.  A ctx must be used from one stream at a time.
+ *   - Return value: SWARM_OK or an error code from host-side validation / launch.  Nothing is
+ *     enqueued when an error is returned.
+ *   - Faults seen on the device (table entry out of range, cluster without replica) never trap:
+ *     they set bits in a status word (swarm_device_status), the offending item is skipped or gets
+ *     a sentinel, and the kernel finishes.
+ *   - bf16 tensors are raw 16-bit words.  Layouts are row-major with the last index fastest.
+ *   - head_dim is 128; page_size is 16 or 32 tokens; 1 <= n_queues <= 32; n_q_heads is a multiple
+ *     of n_kv_heads and query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - Inputs must be finite (no NaN / Inf).
+ */
+#ifndef SWARM_H_
+#define SWARM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes (host side) ---------------------------------------------------------- */
+#define SWARM_OK 0
+#define SWARM_ERR_INVALID_ARG 1         /* null / misaligned pointer, dimension out of range        */
+#define SWARM_ERR_UNSUPPORTED 2         /* valid but not implemented (head_dim != 128, ...)        */
+#define SWARM_ERR_WORKSPACE_TOO_SMALL 3 /* swarm_set_workspace not called or too few bytes         */
+#define SWARM_ERR_CUDA 4                /* a CUDA call failed; see swarm_last_cuda_error           */
+
+/* ---- bits of the device status word ---------------------------------------------------- */
+#define SWARM_DEV_BAD_PAGE 1u           /* a selected page id lies outside its request             */
+#define SWARM_DEV_BAD_CLUSTER 2u        /* page2cluster entry outside the request's cluster range  */
+#define SWARM_DEV_BAD_REPLICA 4u        /* replica mask is 0 or names a queue >= n_queues          */
+#define SWARM_DEV_BAD_LENGTH 8u         /* ctx_len < 1 or more pages than the request owns         */
+
+/* ---- flags in swarm_shape.flags --------------------------------------------------------- */
+#define SWARM_ORDER_BY_ID 1u            /* schedule clusters by id only (default: by number of
+                                           replicas ascending, then id; Sec. 5.1)                  */
+#define SWARM_UNIT_LOAD 2u              /* a cluster adds 1 to its queue (default: its page count) */
+
+typedef struct swarm_ctx swarm_ctx;
+
+/* Problem shape; fixed for the lifetime of a ctx. */
+typedef struct swarm_shape {
+  int32_t batch;              /* B  requests                                                     */
+  int32_t n_q_heads;          /* Hq                                                              */
+  int32_t n_kv_heads;         /* Hkv                                                             */
+  int32_t head_dim;           /* d  (128)                                                        */
+  int32_t page_size;          /* S  tokens per page (16 or 32)                                   */
+  int32_t top_k;              /* k  pages kept per query head                                    */
+  int32_t n_queues;           /* D  simulated SSD queues                                         */
+  int32_t max_pages_per_req;  /* Pmax: upper bound on ceil(ctx_len[b] / S); row pitch of scores  */
+  int32_t max_clusters_total; /* upper bound on cluster_base[B]; capacity of uniq / queue_of     */
+  uint32_t flags;
+  int64_t n_pool_pages;       /* pages in the pool (page_base[B] <= n_pool_pages)                */
+} swarm_shape;
+
+/* Read-only device-resident inputs of a step. */
+typedef struct swarm_inputs {
+  const void* q;                        /* bf16 [B][Hq][d]                                       */
+  const void* ksum;                     /* bf16 [n_pool_pages][Hkv][2][d]      0 = min, 1 = max  */
+  const void* kv_pool;                  /* bf16 [n_pool_pages][Hkv][2][S][d]   0 = K,   1 = V    */
+  const int64_t* page_base;             /* [B+1] request b owns pool pages [base[b], base[b+1])  */
+  const int32_t* ctx_len;               /* [B] tokens; 1 <= len <= S * (base[b+1] - base[b])     */
+  const int32_t* page2cluster;          /* [n_pool_pages] cluster id local to the page's request */
+  const int64_t* cluster_base;          /* [B+1] global cluster id = cluster_base[b] + local id  */
+  const uint32_t* cluster_replica_mask; /* [n_clusters] bit j set <=> a replica sits on queue j  */
+  const uint16_t* cluster_size;         /* [n_clusters] pages in the cluster                     */
+} swarm_inputs;
+
+/* Device-resident outputs of a step.  Pointers marked "optional" may be NULL. */
+typedef struct swarm_outputs {
+  float* scores;       /* optional, f32 [B][Hq][Pmax]; entries p >= pages of the request untouched */
+  int32_t* sel;        /* [B][Hq][k] selected page ids (request-local), ascending, -1 padded       */
+  int32_t* n_sel;      /* [B][Hq]    min(k, pages of the request)                                  */
+  int32_t* uniq;       /* [max_clusters_total] global ids of the clusters to fetch, ascending      */
+  uint8_t* queue_of;   /* [max_clusters_total] queue serving uniq[i]; 0xFF if it has no replica    */
+  int32_t* n_uniq;     /* [1]                                                                      */
+  int32_t* queue_load; /* [D] load routed to each queue this step                                  */
+  void* k_out;         /* optional, bf16 [B][Hq][k*S][d] gathered keys, zero beyond n_tok rows     */
+  void* v_out;         /* optional, bf16 [B][Hq][k*S][d] gathered values (given iff k_out is)      */
+  int32_t* n_tok;      /* optional, [B][Hq] valid gathered tokens (only together with k_out)       */
+  float* out;          /* f32 [B][Hq][d] attention output                                          */
+  float* lse;          /* f32 [B][Hq] natural-log sum of exp of the scaled logits                  */
+} swarm_outputs;
+
+/* Lifetime.  swarm_create validates the shape and allocates only host memory plus one auxiliary
+ * CUDA stream and two events (used to run cluster resolution beside attention inside swarm_step).
+ * The CUDA device current at creation must stay current for every later call with this ctx. */
+int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx);
+int32_t swarm_destroy(swarm_ctx* ctx);
+
+/* Scratch memory.  The caller allocates swarm_workspace_bytes(shape) bytes of device memory
+ * (256-byte aligned) and hands them over; they must stay valid while the ctx is used.  Contents
+ * need no initialisation.  Returns < 0 (minus an error code) for an invalid shape. */
+int64_t swarm_workspace_bytes(const swarm_shape* shape);
+int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, void* stream);
+
+/* Number of key-range splits used by the attention kernels (>= 1; 0 restores the default chosen
+ * from the shape).  Results do not depend on it beyond floating-point rounding. */
+int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits);
+
+/* Index build (not part of a decode step): per page and KV head, element-wise min and max of
+ * the valid tokens' keys -- the compact index the scorer reads instead of the keys themselves
+ * (the role the in-memory cluster index plays in Sec. 4.2, Tier 1).
+ * Reads inputs->kv_pool, page_base, ctx_len; writes ksum_out bf16 [n_pool_pages][Hkv][2][d] for
+ * the pages that exist; padding tokens of a partial last page are ignored. */
+int32_t swarm_build_summaries(swarm_ctx* ctx, const swarm_inputs* inputs, void* ksum_out, void* stream);
+
+/* Stages 1-2: activation scoring and top-k selection (Sec. 2.3: relevance scores of the cached
+ * entries against the query, only the highest-scoring entries are activated).
+ *   score[b][h][p] = sum_i max(q[b][h][i] * kmin[p][i], q[b][h][i] * kmax[p][i])   in fp32
+ *   sel[b][h][:]   = the min(k, P_b) pages of largest score, ties to the lower page id,
+ *                    written in ascending page id; remaining slots -1.
+ * Reads inputs->q, ksum, page_base, ctx_len.  `scores` may be NULL (kept in the workspace). */
+int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* inputs, float* scores, int32_t* sel, int32_t* n_sel,
+                     void* stream);
+
+/* Stage 3: global merge of the activated clusters (Eq. 8, without the already-resident term) and
+ * load-balanced bucket scheduling (Sec. 5.1).  Every selected page is mapped through page2cluster;
+ * the union over all heads and requests is deduplicated; clusters are visited by (number of
+ * replicas ascending, global id ascending) -- by id only under SWARM_ORDER_BY_ID -- and each goes
+ * to the replica queue with the smallest load so far (lowest queue id on a tie), adding its
+ * cluster_size (or 1 under SWARM_UNIT_LOAD) to that queue.
+ * Reads inputs->page_base, page2cluster, cluster_base, cluster_replica_mask, cluster_size. */
+int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel,
+                               const int32_t* n_sel, int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq,
+                               int32_t* queue_load, void* stream);
+
+/* Stage 4a: copy the selected pages' K and V blocks, in `sel` order, into contiguous per-head
+ * buffers (the transfer the paper performs across storage tiers, Sec. 6; here within HBM).
+ * Rows beyond the valid tokens are zero.  n_tok may be NULL. */
+int32_t swarm_gather(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel, const int32_t* n_sel,
+                     void* k_out, void* v_out, int32_t* n_tok, void* stream);
+
+/* Stage 4b: Eq. 1 for one query row per head over its own gathered tokens,
+ *   out[b][h] = softmax_t(q . K_t / sqrt(d)) V_t  over t < n_tok[b][h],  lse = log sum exp,
+ * computed as split-K partials (fp32) merged by their log-sum-exp.  k_g / v_g are
+ * bf16 [B][Hq][k*S][d].  n_tok[b][h] must be >= 1. */
+int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
+                          float* out, float* lse, void* stream);
+
+/* Stage 4 without the copy: the same attention, reading the selected pages straight from the pool
+ * (what swarm_step runs).  Reads inputs->q, kv_pool, page_base, ctx_len.  Tokens beyond ctx_len in a
+ * partial last page are masked.  n_sel[b][h] must be >= 1. */
+int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel,
+                                const int32_t* n_sel, float* out, float* lse, void* stream);
+
+/* The fused step: stages 1-4 enqueued back to back with no host round trip.  Attention reads the
+ * selected pages straight from the pool; the gathered copies are written only when k_out / v_out
+ * are given.  Cluster resolution runs on the ctx's auxiliary stream beside attention and is
+ * joined back before the call's work is complete on `stream`.  Integer outputs equal those of the
+ * four separate calls exactly; out / lse agree within rounding.  The call can be captured into a
+ * CUDA graph by the caller (stream capture). */
+int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);
+
+/* End-to-end convenience for callers holding the per-step data in HOST memory (pinned memory
+ * recommended): copies q_host (bf16 [B][Hq][d]) into the ctx's staging area, runs swarm_step with
+ * `inputs` (whose q field is ignored) and `outputs`, copies out, lse, n_uniq, queue_load back into
+ * the given host buffers and WAITS for completion.  Any *_host pointer may be NULL to skip it. */
+int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs,
+                        const void* q_host, float* out_host, float* lse_host, int32_t* n_uniq_host,
+                        int32_t* queue_load_host, void* stream);
+
+/* Reads and clears the device status word.  SYNCHRONISES `stream`. */
+int32_t swarm_device_status(swarm_ctx* ctx, void* stream, uint32_t* bits);
+
+/* Last cudaError_t recorded by this ctx (0 = none). */
+int32_t swarm_last_cuda_error(const swarm_ctx* ctx);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int32_t swarm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWARM_H_ */

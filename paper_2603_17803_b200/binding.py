@@ -1,0 +1,206 @@
+"""ctypes binding of libswarm.so: the same entry points as ``include/swarm.h``, taking torch tensors.
+
+Argument marshalling only -- every step of the path runs in the CUDA kernels of the library.
+There is no CPU fallback: if the library has not been built, or a call fails, an exception is raised.
+torch is used for device memory and streams, nothing else.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libswarm.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 0, 1, 2, 3, 4
+DEV_BAD_PAGE, DEV_BAD_CLUSTER, DEV_BAD_REPLICA, DEV_BAD_LENGTH = 1, 2, 4, 8
+ORDER_BY_ID, UNIT_LOAD = 1, 2
+_ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA"}
+
+EXPORTS = (
+    "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
+    "swarm_set_attn_splits", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
+)
+
+
+class SwarmError(RuntimeError):
+    def __init__(self, code: int, what: str, cuda_error: int = 0):
+        self.code = code
+        self.cuda_error = cuda_error
+        extra = f" (cudaError {cuda_error})" if cuda_error else ""
+        super().__init__(f"{what}: SWARM_ERR_{_ERR_NAMES.get(code, code)}{extra}")
+
+
+class swarm_shape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("batch", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "top_k",
+                                              "n_queues", "max_pages_per_req", "max_clusters_total")] + \
+               [("flags", ctypes.c_uint32), ("n_pool_pages", ctypes.c_int64)]
+
+
+class swarm_inputs(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("q", "ksum", "kv_pool", "page_base", "ctx_len", "page2cluster",
+                                               "cluster_base", "cluster_replica_mask", "cluster_size")]
+
+
+class swarm_outputs(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "sel", "n_sel", "uniq", "queue_of", "n_uniq", "queue_load",
+                                               "k_out", "v_out", "n_tok", "out", "lse")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libswarm.so from the package directory; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_17803_b200.build` "
+                               "(there is no fallback implementation)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(lib, name).restype = ctypes.c_int32
+        lib.swarm_workspace_bytes.restype = ctypes.c_int64
+        _lib = lib
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor], name: str = "tensor", device_check: bool = True):
+    if t is None:
+        return None
+    if device_check and not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(rc: int, what: str, ctx=None):
+    if rc != OK:
+        cuda = load_library().swarm_last_cuda_error(ctx) if (ctx is not None and rc == ERR_CUDA) else 0
+        raise SwarmError(rc, what, cuda)
+
+
+def make_shape(*, batch, n_q_heads, n_kv_heads, page_size, top_k, n_queues, max_pages_per_req, max_clusters_total,
+               n_pool_pages, head_dim=128, flags=0) -> swarm_shape:
+    return swarm_shape(batch, n_q_heads, n_kv_heads, head_dim, page_size, top_k, n_queues, max_pages_per_req,
+                       max_clusters_total, flags, n_pool_pages)
+
+
+def make_inputs(*, q=None, ksum=None, kv_pool=None, page_base=None, ctx_len=None, page2cluster=None,
+                cluster_base=None, cluster_replica_mask=None, cluster_size=None) -> swarm_inputs:
+    """Struct of device pointers.  The caller keeps the tensors alive while the struct is in use."""
+    return swarm_inputs(*[_ptr(t, n) for n, t in (("q", q), ("ksum", ksum), ("kv_pool", kv_pool),
+                                                  ("page_base", page_base), ("ctx_len", ctx_len),
+                                                  ("page2cluster", page2cluster), ("cluster_base", cluster_base),
+                                                  ("cluster_replica_mask", cluster_replica_mask),
+                                                  ("cluster_size", cluster_size))])
+
+
+def make_outputs(*, scores=None, sel=None, n_sel=None, uniq=None, queue_of=None, n_uniq=None, queue_load=None,
+                 k_out=None, v_out=None, n_tok=None, out=None, lse=None) -> swarm_outputs:
+    return swarm_outputs(*[_ptr(t, n) for n, t in (("scores", scores), ("sel", sel), ("n_sel", n_sel),
+                                                   ("uniq", uniq), ("queue_of", queue_of), ("n_uniq", n_uniq),
+                                                   ("queue_load", queue_load), ("k_out", k_out), ("v_out", v_out),
+                                                   ("n_tok", n_tok), ("out", out), ("lse", lse))])
+
+
+def swarm_version() -> int:
+    return int(load_library().swarm_version())
+
+
+def swarm_workspace_bytes(shape: swarm_shape) -> int:
+    n = int(load_library().swarm_workspace_bytes(ctypes.byref(shape)))
+    if n < 0:
+        raise SwarmError(-n, "swarm_workspace_bytes")
+    return n
+
+
+def swarm_create(shape: swarm_shape) -> ctypes.c_void_p:
+    ctx = ctypes.c_void_p()
+    _check(load_library().swarm_create(ctypes.byref(shape), ctypes.byref(ctx)), "swarm_create")
+    return ctx
+
+
+def swarm_destroy(ctx) -> None:
+    _check(load_library().swarm_destroy(ctx), "swarm_destroy")
+
+
+def swarm_set_workspace(ctx, workspace: torch.Tensor, stream=None) -> None:
+    _check(load_library().swarm_set_workspace(ctx, _ptr(workspace, "workspace"),
+                                              ctypes.c_int64(workspace.numel() * workspace.element_size()),
+                                              _stream(stream)), "swarm_set_workspace", ctx)
+
+
+def swarm_set_attn_splits(ctx, n_splits: int) -> None:
+    _check(load_library().swarm_set_attn_splits(ctx, ctypes.c_int32(n_splits)), "swarm_set_attn_splits", ctx)
+
+
+def swarm_build_summaries(ctx, inputs: swarm_inputs, ksum_out: torch.Tensor, stream=None) -> None:
+    _check(load_library().swarm_build_summaries(ctx, ctypes.byref(inputs), _ptr(ksum_out, "ksum_out"),
+                                                _stream(stream)), "swarm_build_summaries", ctx)
+
+
+def swarm_select(ctx, inputs: swarm_inputs, scores, sel, n_sel, stream=None) -> None:
+    _check(load_library().swarm_select(ctx, ctypes.byref(inputs), _ptr(scores, "scores"), _ptr(sel, "sel"),
+                                       _ptr(n_sel, "n_sel"), _stream(stream)), "swarm_select", ctx)
+
+
+def swarm_resolve_clusters(ctx, inputs: swarm_inputs, sel, n_sel, uniq, queue_of, n_uniq, queue_load,
+                           stream=None) -> None:
+    _check(load_library().swarm_resolve_clusters(ctx, ctypes.byref(inputs), _ptr(sel, "sel"), _ptr(n_sel, "n_sel"),
+                                                 _ptr(uniq, "uniq"), _ptr(queue_of, "queue_of"),
+                                                 _ptr(n_uniq, "n_uniq"), _ptr(queue_load, "queue_load"),
+                                                 _stream(stream)), "swarm_resolve_clusters", ctx)
+
+
+def swarm_gather(ctx, inputs: swarm_inputs, sel, n_sel, k_out, v_out, n_tok, stream=None) -> None:
+    _check(load_library().swarm_gather(ctx, ctypes.byref(inputs), _ptr(sel, "sel"), _ptr(n_sel, "n_sel"),
+                                       _ptr(k_out, "k_out"), _ptr(v_out, "v_out"), _ptr(n_tok, "n_tok"),
+                                       _stream(stream)), "swarm_gather", ctx)
+
+
+def swarm_sparse_attn(ctx, q, k_g, v_g, n_tok, out, lse, stream=None) -> None:
+    _check(load_library().swarm_sparse_attn(ctx, _ptr(q, "q"), _ptr(k_g, "k_g"), _ptr(v_g, "v_g"),
+                                            _ptr(n_tok, "n_tok"), _ptr(out, "out"), _ptr(lse, "lse"),
+                                            _stream(stream)), "swarm_sparse_attn", ctx)
+
+
+def swarm_sparse_attn_paged(ctx, inputs: swarm_inputs, sel, n_sel, out, lse, stream=None) -> None:
+    _check(load_library().swarm_sparse_attn_paged(ctx, ctypes.byref(inputs), _ptr(sel, "sel"), _ptr(n_sel, "n_sel"),
+                                                  _ptr(out, "out"), _ptr(lse, "lse"), _stream(stream)),
+           "swarm_sparse_attn_paged", ctx)
+
+
+def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:
+    _check(load_library().swarm_step(ctx, ctypes.byref(inputs), ctypes.byref(outputs), _stream(stream)),
+           "swarm_step", ctx)
+
+
+def swarm_step_host(ctx, inputs: swarm_inputs, outputs: swarm_outputs, q_host, out_host=None, lse_host=None,
+                    n_uniq_host=None, queue_load_host=None, stream=None) -> None:
+    """Host tensors (pinned recommended) for the per-step data; blocks until the step has finished."""
+    _check(load_library().swarm_step_host(ctx, ctypes.byref(inputs), ctypes.byref(outputs),
+                                          _ptr(q_host, "q_host", False), _ptr(out_host, "out_host", False),
+                                          _ptr(lse_host, "lse_host", False), _ptr(n_uniq_host, "n_uniq_host", False),
+                                          _ptr(queue_load_host, "queue_load_host", False), _stream(stream)),
+           "swarm_step_host", ctx)
+
+
+def swarm_device_status(ctx, stream=None) -> int:
+    bits = ctypes.c_uint32(0)
+    _check(load_library().swarm_device_status(ctx, _stream(stream), ctypes.byref(bits)), "swarm_device_status", ctx)
+    return int(bits.value)
+
+
+def swarm_last_cuda_error(ctx) -> int:
+    return int(load_library().swarm_last_cuda_error(ctx))

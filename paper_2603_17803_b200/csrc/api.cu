@@ -1,0 +1,339 @@
+// C-ABI layer of libswarm: argument validation, workspace carving and kernel sequencing.
+// No device memory is allocated here; every scratch byte comes from the caller's workspace.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "swarm_internal.cuh"
+
+using namespace swarm;
+
+struct swarm_ctx {
+  swarm_shape shape;
+  Geometry geo;
+  WorkspaceLayout lay;
+  uint8_t* ws;
+  int64_t ws_bytes;
+  int default_splits;
+  int n_splits;
+  cudaStream_t side;          // cluster resolution runs here beside attention
+  cudaEvent_t ev_fork, ev_join;
+  cudaError_t last_err;
+};
+
+namespace {
+
+inline int64_t align256(int64_t x) { return (x + 255) & ~int64_t(255); }
+
+int32_t check_shape(const swarm_shape* s) {
+  if (s == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (s->batch < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->top_k < 1 || s->max_pages_per_req < 1 ||
+      s->max_clusters_total < 1 || s->n_pool_pages < 1 || s->n_queues < 1 || s->n_queues > 32 ||
+      s->n_q_heads % s->n_kv_heads != 0 || (s->flags & ~(SWARM_ORDER_BY_ID | SWARM_UNIT_LOAD)) != 0u)
+    return SWARM_ERR_INVALID_ARG;
+  if (s->head_dim != kHeadDim || (s->page_size != 16 && s->page_size != 32)) return SWARM_ERR_UNSUPPORTED;
+  // launch-grid and index-width limits
+  const int64_t bh = (int64_t)s->batch * s->n_q_heads;
+  if (bh * s->top_k >= (int64_t(1) << 31) || bh * kMaxSplits >= (int64_t(1) << 31) || s->batch > 65535 ||
+      (int64_t)s->n_kv_heads * (s->n_q_heads / s->n_kv_heads) > 65535 ||
+      (int64_t)s->page_size * s->max_pages_per_req >= (int64_t(1) << 31))
+    return SWARM_ERR_UNSUPPORTED;
+  return SWARM_OK;
+}
+
+WorkspaceLayout make_layout(const swarm_shape& s) {
+  WorkspaceLayout l;
+  const int64_t bh = (int64_t)s.batch * s.n_q_heads;
+  int64_t off = 0;
+  l.status = off;   off = align256(off + 4);
+  l.scores = off;   off = align256(off + bh * s.max_pages_per_req * 4);
+  l.n_tok = off;    off = align256(off + bh * 4);
+  l.q_stage = off;  off = align256(off + bh * kHeadDim * 2);
+  l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);
+  l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
+  l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
+  l.total = off;
+  return l;
+}
+
+int pick_splits(const swarm_shape& s) {
+  // Enough CTAs for ~4 per SM on 148 SMs, at least 4 pages per split, at most kMaxSplits.
+  const int64_t bh = (int64_t)s.batch * s.n_q_heads;
+  int64_t n = (148 * 4 + bh - 1) / bh;
+  n = std::min<int64_t>(n, std::max(1, s.top_k / 4));
+  n = std::min<int64_t>(n, kMaxSplits);
+  return (int)std::max<int64_t>(n, 1);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool bad(const void* p) { return p == nullptr || !aligned16(p); }
+
+int32_t fail(swarm_ctx* ctx, cudaError_t e) {
+  ctx->last_err = e;
+  return SWARM_ERR_CUDA;
+}
+
+#define SWARM_TRY(expr)                              \
+  do {                                               \
+    cudaError_t e_ = (expr);                         \
+    if (e_ != cudaSuccess) return fail(ctx, e_);     \
+  } while (0)
+
+int32_t need_ws(const swarm_ctx* ctx) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (ctx->ws == nullptr) return SWARM_ERR_WORKSPACE_TOO_SMALL;
+  return SWARM_OK;
+}
+
+template <class T>
+T* ws_ptr(const swarm_ctx* ctx, int64_t off) { return reinterpret_cast<T*>(ctx->ws + off); }
+
+bool select_inputs_ok(const swarm_inputs* in) {
+  return in && !bad(in->q) && !bad(in->ksum) && !bad(in->page_base) && !bad(in->ctx_len);
+}
+bool resolve_inputs_ok(const swarm_inputs* in) {
+  return in && !bad(in->page_base) && !bad(in->page2cluster) && !bad(in->cluster_base) &&
+         !bad(in->cluster_replica_mask) && !bad(in->cluster_size);
+}
+bool pool_inputs_ok(const swarm_inputs* in) {
+  return in && !bad(in->kv_pool) && !bad(in->page_base) && !bad(in->ctx_len);
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t swarm_version(void) { return 100; }
+
+int64_t swarm_workspace_bytes(const swarm_shape* shape) {
+  const int32_t rc = check_shape(shape);
+  if (rc != SWARM_OK) return -(int64_t)rc;
+  return make_layout(*shape).total;
+}
+
+int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
+  if (out_ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  const int32_t rc = check_shape(shape);
+  if (rc != SWARM_OK) return rc;
+  swarm_ctx* ctx = new (std::nothrow) swarm_ctx();
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  ctx->shape = *shape;
+  Geometry& g = ctx->geo;
+  g.B = shape->batch; g.Hq = shape->n_q_heads; g.Hkv = shape->n_kv_heads; g.g = g.Hq / g.Hkv;
+  g.S = shape->page_size; g.k = shape->top_k; g.D = shape->n_queues; g.Pmax = shape->max_pages_per_req;
+  g.Cmax = shape->max_clusters_total; g.flags = shape->flags; g.n_pool_pages = shape->n_pool_pages;
+  ctx->lay = make_layout(*shape);
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  ctx->default_splits = ctx->n_splits = pick_splits(*shape);
+  ctx->last_err = cudaSuccess;
+  cudaError_t e = configure_topk();
+  if (e == cudaSuccess) e = configure_resolve();
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return SWARM_ERR_CUDA;
+  }
+  *out_ctx = ctx;
+  return SWARM_OK;
+}
+
+int32_t swarm_destroy(swarm_ctx* ctx) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  cudaEventDestroy(ctx->ev_fork);
+  cudaEventDestroy(ctx->ev_join);
+  cudaStreamDestroy(ctx->side);
+  delete ctx;
+  return SWARM_OK;
+}
+
+int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, void* stream) {
+  if (ctx == nullptr || device_mem == nullptr || (reinterpret_cast<uintptr_t>(device_mem) & 255u))
+    return SWARM_ERR_INVALID_ARG;
+  if (bytes < ctx->lay.total) return SWARM_ERR_WORKSPACE_TOO_SMALL;
+  ctx->ws = static_cast<uint8_t*>(device_mem);
+  ctx->ws_bytes = bytes;
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 256, static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits) {
+  if (ctx == nullptr || n_splits < 0 || n_splits > kMaxSplits) return SWARM_ERR_INVALID_ARG;
+  ctx->n_splits = n_splits == 0 ? ctx->default_splits : n_splits;
+  return SWARM_OK;
+}
+
+int32_t swarm_last_cuda_error(const swarm_ctx* ctx) { return ctx ? (int32_t)ctx->last_err : 0; }
+
+int32_t swarm_device_status(swarm_ctx* ctx, void* stream, uint32_t* bits) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (bits == nullptr) return SWARM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* dev = ws_ptr<uint32_t>(ctx, ctx->lay.status);
+  SWARM_TRY(cudaMemcpyAsync(bits, dev, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+  SWARM_TRY(cudaMemsetAsync(dev, 0, sizeof(uint32_t), st));
+  SWARM_TRY(cudaStreamSynchronize(st));
+  return SWARM_OK;
+}
+
+int32_t swarm_build_summaries(swarm_ctx* ctx, const swarm_inputs* in, void* ksum_out, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!pool_inputs_ok(in) || bad(ksum_out)) return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_build_summaries(ctx->geo, static_cast<const uint16_t*>(in->kv_pool), in->page_base, in->ctx_len,
+                                   static_cast<uint16_t*>(ksum_out), ws_ptr<uint32_t>(ctx, ctx->lay.status),
+                                   static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int32_t* sel, int32_t* n_sel,
+                     void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!select_inputs_ok(in) || bad(sel) || bad(n_sel) || (scores && !aligned16(scores))) return SWARM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* sc = scores ? scores : ws_ptr<float>(ctx, ctx->lay.scores);
+  SWARM_TRY(launch_page_score(ctx->geo, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(in->ksum),
+                              in->page_base, in->ctx_len, sc, ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, st));
+  return SWARM_OK;
+}
+
+int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
+                               int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load,
+                               void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!resolve_inputs_ok(in) || bad(sel) || bad(n_sel) || bad(uniq) || bad(queue_of) || bad(n_uniq) ||
+      bad(queue_load))
+    return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_resolve(ctx->geo, sel, n_sel, in->page_base, in->page2cluster, in->cluster_base,
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags), uniq,
+                           queue_of, n_uniq, queue_load, ws_ptr<uint32_t>(ctx, ctx->lay.status),
+                           static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_gather(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel, void* k_out,
+                     void* v_out, int32_t* n_tok, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!pool_inputs_ok(in) || bad(sel) || bad(n_sel) || bad(k_out) || bad(v_out) || (n_tok && !aligned16(n_tok)))
+    return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_gather(ctx->geo, static_cast<const uint16_t*>(in->kv_pool), sel, n_sel, in->page_base,
+                          in->ctx_len, static_cast<uint16_t*>(k_out), static_cast<uint16_t*>(v_out), n_tok,
+                          ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
+                          float* out, float* lse, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (bad(q) || bad(k_g) || bad(v_g) || bad(n_tok) || bad(out) || bad(lse)) return SWARM_ERR_INVALID_ARG;
+  AttnArgs a{};
+  a.q = static_cast<const uint16_t*>(q);
+  a.k_g = static_cast<const uint16_t*>(k_g);
+  a.v_g = static_cast<const uint16_t*>(v_g);
+  a.n_tok = n_tok;
+  a.part_acc = ws_ptr<float>(ctx, ctx->lay.part_acc);
+  a.part_ml = ws_ptr<float>(ctx, ctx->lay.part_ml);
+  a.out = out;
+  a.lse = lse;
+  a.n_splits = ctx->n_splits;
+  SWARM_TRY(launch_attention(ctx->geo, a, ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+namespace {
+AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
+                    float* out, float* lse) {
+  AttnArgs a{};
+  a.q = static_cast<const uint16_t*>(in->q);
+  a.kv_pool = static_cast<const uint16_t*>(in->kv_pool);
+  a.sel = sel;
+  a.n_sel = n_sel;
+  a.page_base = in->page_base;
+  a.ctx_len = in->ctx_len;
+  a.part_acc = ws_ptr<float>(ctx, ctx->lay.part_acc);
+  a.part_ml = ws_ptr<float>(ctx, ctx->lay.part_ml);
+  a.out = out;
+  a.lse = lse;
+  a.n_splits = ctx->n_splits;
+  return a;
+}
+}  // namespace
+
+int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
+                                float* out, float* lse, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!pool_inputs_ok(in) || bad(in->q) || bad(sel) || bad(n_sel) || bad(out) || bad(lse)) return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, sel, n_sel, out, lse),
+                             ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (!select_inputs_ok(in) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || o == nullptr || bad(o->sel) ||
+      bad(o->n_sel) || bad(o->uniq) || bad(o->queue_of) || bad(o->n_uniq) || bad(o->queue_load) || bad(o->out) ||
+      bad(o->lse) || (o->scores && !aligned16(o->scores)) || (o->n_tok && !aligned16(o->n_tok)) ||
+      ((o->k_out == nullptr) != (o->v_out == nullptr)) || (o->n_tok && !o->k_out) || (o->k_out && (!aligned16(o->k_out) || !aligned16(o->v_out))))
+    return SWARM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* status = ws_ptr<uint32_t>(ctx, ctx->lay.status);
+  const uint16_t* q = static_cast<const uint16_t*>(in->q);
+  const uint16_t* pool = static_cast<const uint16_t*>(in->kv_pool);
+  float* sc = o->scores ? o->scores : ws_ptr<float>(ctx, ctx->lay.scores);
+
+  SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
+                              status, st));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, st));
+
+  // fork: cluster resolution needs only the selection and does not feed attention
+  SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
+  SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+  SWARM_TRY(launch_resolve(ctx->geo, o->sel, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags), o->uniq,
+                           o->queue_of, o->n_uniq, o->queue_load, status, ctx->side));
+  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
+
+  if (o->k_out != nullptr)
+    SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
+                            static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
+  const AttnArgs a = paged_args(ctx, in, o->sel, o->n_sel, o->out, o->lse);
+  SWARM_TRY(launch_attention(ctx->geo, a, status, st));
+  SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  return SWARM_OK;
+}
+
+int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
+                        float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,
+                        void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (in == nullptr || o == nullptr || q_host == nullptr) return SWARM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t bh = (int64_t)ctx->geo.B * ctx->geo.Hq;
+  uint16_t* q_dev = ws_ptr<uint16_t>(ctx, ctx->lay.q_stage);
+  SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
+  swarm_inputs local = *in;
+  local.q = q_dev;
+  rc = swarm_step(ctx, &local, o, stream);
+  if (rc != SWARM_OK) return rc;
+  if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));
+  if (lse_host) SWARM_TRY(cudaMemcpyAsync(lse_host, o->lse, bh * 4, cudaMemcpyDeviceToHost, st));
+  if (n_uniq_host) SWARM_TRY(cudaMemcpyAsync(n_uniq_host, o->n_uniq, 4, cudaMemcpyDeviceToHost, st));
+  if (queue_load_host)
+    SWARM_TRY(cudaMemcpyAsync(queue_load_host, o->queue_load, ctx->geo.D * 4, cudaMemcpyDeviceToHost, st));
+  SWARM_TRY(cudaStreamSynchronize(st));
+  return SWARM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+"""Convenience wrapper: owns a swarm ctx, its workspace and output tensors for one set of device inputs.
+
+Allocation and marshalling only (torch supplies device memory and streams); all computing is done by
+the library's kernels through ``binding``.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import binding as B
+
+
+@dataclass
+class StepOutputs:
+    scores: Optional[torch.Tensor]
+    sel: torch.Tensor
+    n_sel: torch.Tensor
+    uniq: torch.Tensor
+    queue_of: torch.Tensor
+    n_uniq: torch.Tensor
+    queue_load: torch.Tensor
+    k_out: Optional[torch.Tensor]
+    v_out: Optional[torch.Tensor]
+    n_tok: Optional[torch.Tensor]
+    out: torch.Tensor
+    lse: torch.Tensor
+
+
+class Session:
+    """One ctx bound to one resident KV pool (``workload`` tensors must live on a CUDA device)."""
+
+    def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
+                 ksum: Optional[torch.Tensor] = None):
+        cfg = workload.cfg
+        self.cfg = cfg
+        self.w = workload
+        dev = workload.kv_pool.device
+        if dev.type != "cuda":
+            raise ValueError("Session needs the workload on a CUDA device")
+        self.device = dev
+        self.Pmax = cfg.max_pages()
+        self.shape = B.make_shape(batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                                  page_size=cfg.page_size, top_k=cfg.top_k, n_queues=cfg.n_queues,
+                                  max_pages_per_req=self.Pmax, max_clusters_total=max(1, workload.n_clusters),
+                                  n_pool_pages=workload.n_pool_pages, flags=flags)
+        self.ctx = B.swarm_create(self.shape)
+        self.workspace = torch.empty(B.swarm_workspace_bytes(self.shape), dtype=torch.uint8, device=dev)
+        B.swarm_set_workspace(self.ctx, self.workspace)
+        self.ksum = ksum if ksum is not None else torch.empty(
+            (workload.n_pool_pages, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+        self.inputs = self._inputs(workload.q)
+        if ksum is None:
+            B.swarm_build_summaries(self.ctx, self.inputs, self.ksum)
+        Bq, Hq, k, S, d = cfg.batch, cfg.n_q_heads, cfg.top_k, cfg.page_size, cfg.head_dim
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.o = StepOutputs(
+            scores=torch.full((Bq, Hq, self.Pmax), float("-inf"), dtype=torch.float32, device=dev) if keep_scores else None,
+            sel=torch.empty((Bq, Hq, k), **i32), n_sel=torch.empty((Bq, Hq), **i32),
+            uniq=torch.empty(max(1, workload.n_clusters), **i32),
+            queue_of=torch.empty(max(16, workload.n_clusters), dtype=torch.uint8, device=dev),
+            n_uniq=torch.zeros(4, **i32), queue_load=torch.zeros(max(4, cfg.n_queues), **i32),
+            k_out=torch.empty((Bq, Hq, k * S, d), dtype=torch.bfloat16, device=dev) if keep_gathered else None,
+            v_out=torch.empty((Bq, Hq, k * S, d), dtype=torch.bfloat16, device=dev) if keep_gathered else None,
+            n_tok=torch.empty((Bq, Hq), **i32) if keep_gathered else None,
+            out=torch.empty((Bq, Hq, d), dtype=torch.float32, device=dev),
+            lse=torch.empty((Bq, Hq), dtype=torch.float32, device=dev),
+        )
+        self.outputs = B.make_outputs(**{k_: getattr(self.o, k_) for k_ in self.o.__dataclass_fields__})
+
+    def _inputs(self, q):
+        w = self.w
+        return B.make_inputs(q=q, ksum=self.ksum, kv_pool=w.kv_pool, page_base=w.page_base, ctx_len=w.ctx_len,
+                             page2cluster=w.page2cluster, cluster_base=w.cluster_base,
+                             cluster_replica_mask=w.cluster_replica_mask, cluster_size=w.cluster_size)
+
+    def set_query(self, q: torch.Tensor) -> None:
+        self._q = q
+        self.inputs = self._inputs(q)
+
+    # -- the five calls ---------------------------------------------------------------------------
+    def select(self, stream=None):
+        B.swarm_select(self.ctx, self.inputs, self.o.scores, self.o.sel, self.o.n_sel, stream)
+
+    def resolve(self, sel=None, n_sel=None, stream=None):
+        B.swarm_resolve_clusters(self.ctx, self.inputs, self.o.sel if sel is None else sel,
+                                 self.o.n_sel if n_sel is None else n_sel, self.o.uniq, self.o.queue_of,
+                                 self.o.n_uniq, self.o.queue_load, stream)
+
+    def gather(self, sel=None, n_sel=None, stream=None):
+        if self.o.k_out is None:
+            raise ValueError("Session was created with keep_gathered=False")
+        B.swarm_gather(self.ctx, self.inputs, self.o.sel if sel is None else sel,
+                       self.o.n_sel if n_sel is None else n_sel, self.o.k_out, self.o.v_out, self.o.n_tok, stream)
+
+    def sparse_attn(self, stream=None):
+        B.swarm_sparse_attn(self.ctx, self.w.q if not hasattr(self, "_q") else self._q, self.o.k_out, self.o.v_out,
+                            self.o.n_tok, self.o.out, self.o.lse, stream)
+
+    def sparse_attn_paged(self, stream=None):
+        B.swarm_sparse_attn_paged(self.ctx, self.inputs, self.o.sel, self.o.n_sel, self.o.out, self.o.lse, stream)
+
+    def step(self, stream=None):
+        B.swarm_step(self.ctx, self.inputs, self.outputs, stream)
+
+    def step_host(self, q_host, out_host=None, lse_host=None, n_uniq_host=None, queue_load_host=None, stream=None):
+        B.swarm_step_host(self.ctx, self.inputs, self.outputs, q_host, out_host, lse_host, n_uniq_host,
+                          queue_load_host, stream)
+
+    def status(self) -> int:
+        return B.swarm_device_status(self.ctx)
+
+    def close(self):
+        if self.ctx is not None:
+            torch.cuda.synchronize(self.device)
+            B.swarm_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

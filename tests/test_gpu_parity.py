@@ -1,0 +1,306 @@
+"""GPU parity tests: every call goes through the C-ABI library and is compared with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from helpers import to_bf16_bits
+from paper_2603_17803_b200 import binding as B
+from paper_2603_17803_b200 import workloads as W
+from paper_2603_17803_b200.session import Session
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_separate_calls(sess):
+    sess.select()
+    sess.resolve()
+    sess.gather()
+    sess.sparse_attn()
+
+
+def small(name, **kw):
+    return W.scaled(W.CONFIGS[name], **kw)
+
+
+CASES = {
+    # several score tiles, a ragged tail, a partial last page; sized for an oracle run of seconds
+    "c1_small": small("c1_tiny", ctx_len=16 * 700 + 5, top_k=48),
+    "c2_small": small("c2_128k", ctx_len=16 * 1500 + 9, top_k=96, n_topics=12),
+    "c3_small": small("c3_batched", batch=3, ctx_len=16 * 400 + 1, top_k=40, n_topics=8),
+    "c4_small": small("c4_long", batch=2, ctx_len=32 * 900 + 17, top_k=64, n_topics=16),
+    "c5_small": small("c5_skewed", batch=5, ctx_range=(16 * 20, 16 * 900), top_k=32, n_topics=10),
+    "k_exceeds_pages": small("c5_skewed", batch=3, ctx_range=(1, 16 * 12), top_k=24, n_topics=3),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_separate_calls_match_oracle(name):
+    w = W.generate(CASES[name], seed=11, device=DEV)
+    sess = Session(w, keep_scores=True, keep_gathered=True)
+    run_separate_calls(sess)
+    info = parity.check_step(w, sess)
+    assert info["heads"] == w.cfg.batch * w.cfg.n_q_heads
+    sess.close()
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_fused_step_equals_composition(name):
+    w = W.generate(CASES[name], seed=12, device=DEV)
+    a = Session(w, keep_scores=True, keep_gathered=True)
+    run_separate_calls(a)
+    torch.cuda.synchronize()
+    b = Session(w, keep_scores=True, keep_gathered=True, ksum=a.ksum)
+    b.step()
+    info = parity.check_step(w, b)
+    for f in ("sel", "n_sel", "n_tok", "k_out", "v_out", "queue_load"):
+        assert torch.equal(getattr(a.o, f), getattr(b.o, f)), f
+    n = int(a.o.n_uniq[0])
+    assert int(b.o.n_uniq[0]) == n
+    assert torch.equal(a.o.uniq[:n], b.o.uniq[:n]) and torch.equal(a.o.queue_of[:n], b.o.queue_of[:n])
+    assert torch.equal(a.o.scores, b.o.scores)
+    assert (a.o.out - b.o.out).abs().max().item() <= 1e-4
+    assert (a.o.lse - b.o.lse).abs().max().item() <= 1e-4
+    # fused step without the optional outputs gives the same required outputs
+    c = Session(w, ksum=a.ksum)
+    c.step()
+    torch.cuda.synchronize()
+    assert torch.equal(c.o.sel, b.o.sel) and torch.equal(c.o.out, b.o.out) and torch.equal(c.o.queue_load, b.o.queue_load)
+    for s in (a, b, c):
+        s.close()
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_128k"])
+def test_full_size_configs_match_oracle(name):
+    """The two configurations the oracle handles whole, at full size, through the fused step."""
+    w = W.generate(W.CONFIGS[name], seed=0, device=DEV)
+    sess = Session(w, keep_scores=True, keep_gathered=True)
+    sess.step()
+    info = parity.check_step(w, sess)
+    assert info["exact_heads"] >= info["heads"] - 4      # band differences are legal but rare
+    sess.close()
+
+
+@pytest.mark.parametrize("name,reqs,heads", [("c3_batched", [0, 9], [0, 5, 31]), ("c4_long", [1], [0, 17, 63])])
+def test_full_size_sampled(name, reqs, heads):
+    """Full-size launch configuration; stage 3 checked whole, the other stages on sampled requests/heads."""
+    w = W.generate(W.CONFIGS[name], seed=0, device=DEV)
+    sess = Session(w, keep_scores=True)
+    sess.step()
+    parity.check_step(w, sess, requests=reqs, heads=heads)
+    sess.close()
+
+
+def test_c5_full_size_sampled():
+    w = W.generate(W.CONFIGS["c5_skewed"], seed=0, device=DEV)
+    sess = Session(w, keep_scores=True)
+    sess.step()
+    lens = w.ctx_len.cpu().numpy()
+    reqs = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 7})
+    parity.check_step(w, sess, requests=reqs, heads=[0, 13, 31])
+    sess.close()
+
+
+@pytest.mark.parametrize("splits", [1, 2, 7, 64])
+def test_split_count_is_unobservable(splits):
+    w = W.generate(CASES["c2_small"], seed=5, device=DEV)
+    sess = Session(w, keep_gathered=True)
+    B.swarm_set_attn_splits(sess.ctx, splits)
+    run_separate_calls(sess)
+    parity.check_step(w, sess)
+    sess.step()
+    parity.check_step(w, sess)
+    sess.close()
+
+
+@pytest.mark.parametrize("flags", [B.ORDER_BY_ID, B.UNIT_LOAD, B.ORDER_BY_ID | B.UNIT_LOAD])
+@pytest.mark.parametrize("name", ["c3_small", "c5_small"])
+def test_scheduling_flags(name, flags):
+    w = W.generate(CASES[name], seed=6, device=DEV)
+    sess = Session(w, flags=flags)
+    sess.step()
+    parity.check_step(w, sess, flags=flags)
+    sess.close()
+
+
+@pytest.mark.parametrize("replication,D", [("one", 5), ("all", 7), ("all", 32), ("two", 32)])
+def test_replication_extremes(replication, D):
+    cfg = small("c3_batched", batch=2, ctx_len=16 * 300, top_k=50, n_topics=6, replication=replication, n_queues=D)
+    w = W.generate(cfg, seed=7, device=DEV)
+    sess = Session(w, flags=B.UNIT_LOAD if replication == "all" else 0)
+    sess.step()
+    parity.check_step(w, sess, flags=B.UNIT_LOAD if replication == "all" else 0)
+    load = sess.o.queue_load.cpu().numpy()[:D]
+    if replication == "all":
+        assert load.max() - load.min() <= 1
+    sess.close()
+
+
+def test_all_equal_scores_pick_lowest_ids_and_signed_zero_ties():
+    cfg = small("c1_tiny", ctx_len=16 * 300, top_k=20)
+    w = W.generate(cfg, seed=8, device=DEV)
+    w.q.zero_()                                          # every score is exactly 0
+    sess = Session(w, keep_scores=True)
+    sess.step()
+    torch.cuda.synchronize()
+    assert torch.equal(sess.o.sel[0, 3].cpu(), torch.arange(20, dtype=torch.int32))
+    parity.check_step(w, sess)
+    # planted duplicates straddling the k-th place: make the scorer reproduce chosen scores exactly
+    # (q = e_0 and kmin = kmax = the wanted score in coordinate 0), then compare with the oracle's top-k
+    P = cfg.max_pages()
+    sc = torch.zeros((1, 8, P), device=DEV)
+    sc[0, 1] = torch.arange(P, device=DEV) % 7
+    sc[0, 2] = -(torch.arange(P, device=DEV) % 5).float()
+    sc[0, 3] = (torch.arange(P, device=DEV) // 50).float()
+    ref, _ = oracle.topk(sc.cpu().numpy(), w.ctx_len.cpu().numpy(), 16, 20)
+    ksum = torch.zeros_like(sess.ksum)
+    ksum[:, :, :, 0] = sc[0].t()[:, :, None].to(torch.bfloat16)
+    w.q.zero_()
+    w.q[..., 0] = 1.0
+    sess2 = Session(w, keep_scores=True, ksum=ksum)
+    sess2.select()
+    torch.cuda.synchronize()
+    assert torch.equal(sess2.o.scores[0, :, :P], sc[0])
+    assert np.array_equal(sess2.o.sel.cpu().numpy()[0], ref[0])
+    sess.close()
+    sess2.close()
+
+
+def test_structured_attention_outputs_of_order_one():
+    """Dominant key and constant V: outputs of magnitude 1, so the tolerance is meaningful."""
+    cfg = small("c1_tiny", ctx_len=16 * 200, top_k=30)
+    w = W.generate(cfg, seed=9, device=DEV)
+    q = w.q.float()
+    # plant, for head 2, a key in page 77 aligned with q and strong enough to dominate
+    w.kv_pool[77, 2, 0, 5] = (40.0 * q[0, 2] / q[0, 2].norm()).to(torch.bfloat16)
+    w.kv_pool[:, 4, 1] = 1.5                              # head 4: constant V
+    sess = Session(w, keep_gathered=True)
+    sess.step()
+    parity.check_step(w, sess)
+    out = sess.o.out.cpu()
+    assert (out[0, 2] - w.kv_pool[77, 2, 1, 5].float().cpu()).abs().max() < 2e-2
+    assert (out[0, 4] - 1.5).abs().max() < 1e-5
+    sess.close()
+
+
+def test_corrupt_tables_set_status_bits_and_never_trap():
+    cfg = small("c3_batched", batch=2, ctx_len=16 * 100, top_k=16, n_topics=4)
+    w = W.generate(cfg, seed=10, device=DEV)
+    sess = Session(w)
+    sess.step()
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    good_mask = w.cluster_replica_mask.clone()
+    w.cluster_replica_mask.zero_()                        # no replica anywhere
+    sess.step()
+    assert sess.status() & B.DEV_BAD_REPLICA
+    assert int(sess.o.queue_of[0]) == 0xFF
+    w.cluster_replica_mask.copy_(good_mask)
+    good_p2c = w.page2cluster.clone()
+    w.page2cluster.fill_(10 ** 6)                         # cluster ids out of range
+    sess.step()
+    assert sess.status() & B.DEV_BAD_CLUSTER
+    w.page2cluster.copy_(good_p2c)
+    bad_sel = sess.o.sel.clone()
+    bad_sel[0, 0, 0] = 10 ** 6                            # page id out of range, fed to the stage calls
+    sess.resolve(sel=bad_sel)
+    assert sess.status() & B.DEV_BAD_PAGE
+    good_len = w.ctx_len.clone()
+    w.ctx_len[0] = 0
+    sess.select()
+    assert sess.status() & B.DEV_BAD_LENGTH
+    w.ctx_len.copy_(good_len)
+    sess.step()                                           # the ctx is still usable
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    parity.check_step(w, sess)
+    sess.close()
+
+
+def test_invalid_arguments_are_rejected_on_the_host():
+    ok = dict(batch=1, n_q_heads=8, n_kv_heads=2, page_size=16, top_k=4, n_queues=4, max_pages_per_req=8,
+              max_clusters_total=4, n_pool_pages=8)
+    for bad, code in [(dict(head_dim=64), B.ERR_UNSUPPORTED), (dict(page_size=8), B.ERR_UNSUPPORTED),
+                      (dict(n_queues=33), B.ERR_INVALID_ARG), (dict(n_kv_heads=3), B.ERR_INVALID_ARG),
+                      (dict(top_k=0), B.ERR_INVALID_ARG), (dict(flags=64), B.ERR_INVALID_ARG)]:
+        with pytest.raises(B.SwarmError) as e:
+            B.swarm_create(B.make_shape(**{**ok, **bad}))
+        assert e.value.code == code
+    shape = B.make_shape(**ok)
+    ctx = B.swarm_create(shape)
+    t = torch.zeros(1024, dtype=torch.int32, device=DEV)
+    with pytest.raises(B.SwarmError) as e:                # no workspace yet
+        B.swarm_select(ctx, B.make_inputs(q=t, ksum=t, page_base=t, ctx_len=t), None, t, t)
+    assert e.value.code == B.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(B.SwarmError) as e:
+        B.swarm_set_workspace(ctx, torch.empty(16, dtype=torch.uint8, device=DEV))
+    assert e.value.code == B.ERR_WORKSPACE_TOO_SMALL
+    ws = torch.empty(B.swarm_workspace_bytes(shape), dtype=torch.uint8, device=DEV)
+    B.swarm_set_workspace(ctx, ws)
+    with pytest.raises(B.SwarmError) as e:                # null input
+        B.swarm_select(ctx, B.make_inputs(q=t, ksum=None, page_base=t, ctx_len=t), None, t, t)
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.SwarmError) as e:                # misaligned pointer
+        B.swarm_select(ctx, B.make_inputs(q=t[1:], ksum=t, page_base=t, ctx_len=t), None, t, t)
+    assert e.value.code == B.ERR_INVALID_ARG
+    B.swarm_destroy(ctx)
+
+
+def test_step_host_round_trip():
+    w = W.generate(CASES["c2_small"], seed=13, device=DEV)
+    sess = Session(w)
+    sess.step()
+    torch.cuda.synchronize()
+    want_out, want_load = sess.o.out.cpu().clone(), sess.o.queue_load.cpu().clone()
+    q_host = w.q.cpu().pin_memory()
+    out_host = torch.empty_like(want_out).pin_memory()
+    lse_host = torch.empty((1, 32), dtype=torch.float32).pin_memory()
+    n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    load_host = torch.zeros(w.cfg.n_queues, dtype=torch.int32).pin_memory()
+    sess.o.out.zero_()
+    sess.step_host(q_host, out_host, lse_host, n_host, load_host)
+    assert torch.equal(out_host, want_out)
+    assert torch.equal(load_host, want_load[: w.cfg.n_queues])
+    assert int(n_host[0]) == int(sess.o.n_uniq[0])
+    sess.close()
+
+
+def test_step_can_be_captured_in_a_cuda_graph():
+    w = W.generate(CASES["c3_small"], seed=14, device=DEV)
+    sess = Session(w)
+    sess.step()
+    torch.cuda.synchronize()
+    n = int(sess.o.n_uniq[0])
+    sess.o.uniq[n:].zero_()                               # entries beyond n_uniq are not written
+    want = {f: getattr(sess.o, f).clone() for f in ("sel", "out", "lse", "queue_load", "uniq", "n_uniq")}
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        sess.step(stream=s)                               # warm-up on the capture stream
+        s.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            sess.step(stream=s)
+    for f in want:
+        getattr(sess.o, f).zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for f, t in want.items():
+        assert torch.equal(getattr(sess.o, f), t), f
+    sess.close()
+
+
+def test_paged_attention_alone_matches_gathered_attention():
+    w = W.generate(CASES["c4_small"], seed=15, device=DEV)
+    sess = Session(w, keep_gathered=True)
+    run_separate_calls(sess)
+    torch.cuda.synchronize()
+    out, lse = sess.o.out.clone(), sess.o.lse.clone()
+    sess.o.out.zero_()
+    sess.sparse_attn_paged()
+    torch.cuda.synchronize()
+    assert (sess.o.out - out).abs().max().item() <= 1e-5 and (sess.o.lse - lse).abs().max().item() <= 1e-5
+    parity.check_step(w, sess)
+    sess.close()
