@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the fused KVCache retrieval step (select + resolve + gather + attention) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl swarm|reference] [--workload c2_128k]
+
+A step is one swarm_step over one batch of synthetic input (one layer).  The workload is the 128K
+Llama-3-8B-shaped configuration.  Because one step touches less data than the L2 holds, the run
+rotates over several independent data sets (pool, summaries, query) so consecutive steps never
+re-read cached data.  Each step is replayed from a CUDA graph captured from the library call.
+
+Prints ONE JSON line (rank 0).  N > 1 (torchrun) runs N independent replicas -- the path is
+single-GPU by definition, so there is no data-path collective; only the timing barrier and the
+max-over-ranks reduction use torch.distributed.
+
+--impl reference times the CPU oracle (test infrastructure, plain C++) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode steps/sec of fused select+resolve+gather+attn; HBM GB/s (% of peak)"
+UNIT = "steps/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_kernel launch at this workload, from the ncu
+# capture summarised in profiles/ (None until a capture exists for the current kernel).
+ATTN_TRAFFIC_BYTES_NCU = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="swarm", choices=["swarm", "reference"])
+    ap.add_argument("--workload", default="c2_128k")
+    ap.add_argument("--n-rot", type=int, default=8, help="independent data sets rotated through")
+    ap.add_argument("--no-graph", action="store_true", help="call the library directly instead of replaying graphs")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed regions run."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples = []   # (t, sm_mhz, reasons_bitmask)
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self.period = period_s
+
+    def _read(self):
+        nv = self.nv
+        mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        try:
+            reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        except Exception:
+            reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+        return mhz, reasons
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                mhz, reasons = self._read()
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self, windows):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        inside = [s for s in self.samples if any(a <= s[0] <= b for a, b in windows)] or self.samples
+        mhz = sorted(s[1] for s in inside)
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        names = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        reasons = [n for b, n in names.items() if bits & b and n != "gpu_idle"]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples_in_timed_region": len(inside)}
+
+
+# ----------------------------------------------------------------------------------- byte accounting
+
+def step_bytes(w, sel, n_sel):
+    """Algorithmic bytes of one step (what the method must move), from the executed selection.
+    summaries: every existing page's 512 B row per KV head, read once.
+    kv (compulsory): K and V blocks of the distinct (request, kv head, page) triples selected by any head
+    of the group; kv (nominal): one K and V block per selected (head, page) slot."""
+    import numpy as np
+    cfg = w.cfg
+    S, d, Hkv, g = cfg.page_size, cfg.head_dim, cfg.n_kv_heads, cfg.group
+    pages = -(-w.ctx_len.cpu().numpy().astype(np.int64) // S)
+    summaries = int(pages.sum()) * Hkv * 2 * d * 2
+    sel = sel.cpu().numpy()
+    n_sel = n_sel.cpu().numpy()
+    blk = S * d * 2 * 2
+    distinct = 0
+    for b in range(cfg.batch):
+        for kv in range(Hkv):
+            ids = [sel[b, h, : n_sel[b, h]] for h in range(kv * g, (kv + 1) * g)]
+            distinct += len(np.unique(np.concatenate(ids)))
+    nominal = int(n_sel.sum())
+    small = cfg.batch * cfg.n_q_heads * (d * 2 + d * 4 + 4 + cfg.top_k * 4)
+    return dict(summaries=summaries, kv_compulsory=distinct * blk, kv_nominal=nominal * blk, small=small)
+
+
+# ------------------------------------------------------------------------------------------ swarm arm
+
+def run_swarm(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_17803_b200 import workloads as W
+    from paper_2603_17803_b200.session import Session
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    K = args.steps if args.steps is not None else 20000
+    Wm = args.warmup if args.warmup is not None else 50
+    cfg = W.CONFIGS[args.workload]
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    # independent data sets; every rank draws its own (weak scaling: fixed work per GPU)
+    sessions, workloads = [], []
+    for r in range(args.n_rot):
+        w = W.generate(cfg, seed=1000 * rank + r, device=dev, step=r)
+        workloads.append(w)
+        sessions.append(Session(w))
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    graphs = []
+    with torch.cuda.stream(stream):
+        for s in sessions:
+            s.step(stream=stream)
+        stream.synchronize()
+        if not args.no_graph:
+            for s in sessions:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    s.step(stream=stream)
+                graphs.append(g)
+
+        def one_step(i):
+            if graphs:
+                graphs[i % args.n_rot].replay()
+            else:
+                sessions[i % args.n_rot].step(stream=stream)
+
+        for i in range(Wm):
+            one_step(i)
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_a = time.perf_counter()
+        ev0.record(stream)
+        for i in range(K):
+            one_step(i)
+        ev1.record(stream)
+        barrier()
+        t_b = time.perf_counter()
+        ms = ev0.elapsed_time(ev1)
+
+        # the dominant kernel (attention straight from the pool) timed alone, back to back over the rotating sets
+        def time_loop(fn, n):
+            for i in range(min(n, 2 * args.n_rot)):
+                fn(sessions[i % args.n_rot])
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(n):
+                fn(sessions[i % args.n_rot])
+            e1.record(stream)
+            stream.synchronize()
+            return e0.elapsed_time(e1) / n * 1e3    # microseconds per call
+
+        n_loop = max(3 * args.n_rot, min(K, 2000))
+        t_c = time.perf_counter()
+        attn_us = time_loop(lambda s: s.sparse_attn_paged(stream=stream), n_loop)
+        select_us = time_loop(lambda s: s.select(stream=stream), n_loop)
+        resolve_us = time_loop(lambda s: s.resolve(stream=stream), n_loop)
+        t_d = time.perf_counter()
+
+        # end to end: per-step data in pinned host memory, copies inside the timed region
+        B, Hq, d, D = cfg.batch, cfg.n_q_heads, cfg.head_dim, cfg.n_queues
+        q_host = [w.q.cpu().pin_memory() for w in workloads]
+        out_host = torch.empty((B, Hq, d), dtype=torch.float32).pin_memory()
+        lse_host = torch.empty((B, Hq), dtype=torch.float32).pin_memory()
+        n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+        load_host = torch.zeros(D, dtype=torch.int32).pin_memory()
+        K_e2e = min(K, 5000)
+        for i in range(min(Wm, 20)):
+            sessions[i % args.n_rot].step_host(q_host[i % args.n_rot], out_host, lse_host, n_host, load_host, stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_e = time.perf_counter()
+        e0.record(stream)
+        for i in range(K_e2e):
+            sessions[i % args.n_rot].step_host(q_host[i % args.n_rot], out_host, lse_host, n_host, load_host, stream)
+        e1.record(stream)
+        barrier()
+        t_f = time.perf_counter()
+        ms_e2e = e0.elapsed_time(e1)
+    sampler.stop()
+
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+
+    status = max(s.status() for s in sessions)
+    by = step_bytes(workloads[0], sessions[0].o.sel, sessions[0].o.n_sel)
+    peak, peak_kind = measured_peak()
+    step_s = ms / 1e3 / K
+    alg = by["summaries"] + by["kv_compulsory"] + by["small"]
+    nominal = by["summaries"] + by["kv_nominal"] + by["small"]
+    hbm_gbs = alg / step_s / 1e9
+    attn_alg = by["kv_compulsory"]
+    attn_gbs = attn_alg / (attn_us * 1e-6) / 1e9
+
+    result = {
+        "metric": METRIC, "value": world * K / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "context": cfg.max_ctx(), "page_size": cfg.page_size,
+                   "top_k": cfg.top_k, "n_queues": cfg.n_queues, "n_topics": cfg.n_topics,
+                   "parallelism": f"replicas x{world} (no data-path collective)",
+                   "l2_policy": f"rotating {args.n_rot} independent data sets "
+                                f"({args.n_rot * alg / 1e6:.0f} MB touched per rotation > 126 MB L2)",
+                   "launch": "library call" if args.no_graph else "CUDA graph replay of swarm_step"},
+        "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
+        "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
+        "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
+        "roofline": {"kernel": "attn_kernel<16,paged> (+ split combine)", "bound": "hbm", "achieved": attn_gbs,
+                     "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
+                     "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU,
+                     "algorithmic_bytes_per_launch": attn_alg, "avg_launch_us": attn_us,
+                     "nominal_bytes_per_launch": by["kv_nominal"], "nominal_gbs": by["kv_nominal"] / (attn_us * 1e-6) / 1e9},
+        "e2e": {"value": world * K_e2e / (ms_e2e / 1e3), "unit": UNIT, "steps": K_e2e,
+                "h2d_bytes_per_step": B * Hq * d * 2, "d2h_bytes_per_step": B * Hq * d * 4 + B * Hq * 4 + 4 + D * 4,
+                "note": "swarm_step_host: q from pinned host memory, out/lse/n_uniq/queue_load read back; "
+                        "the KV pool and its summaries are resident state, like weights"},
+        "gpu_launches": K * 5,
+        "gpu_launches_per_step": 5,
+        "device_status": status,
+        "clocks": sampler.summary([(t_a, t_b), (t_e, t_f)]),
+    }
+    if rank == 0 and not args.skip_cpu_baseline and world == 1:
+        result["cpu_baseline"] = cpu_baseline(workloads[0], budget_s=12.0)
+    for s in sessions:
+        s.close()
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle
+
+def oracle_inputs(w):
+    import numpy as np
+    from paper_2603_17803_b200.workloads import bits_u16
+    return dict(q=bits_u16(w.q), kv_pool=bits_u16(w.kv_pool), page_base=w.page_base.cpu().numpy(),
+                ctx_len=w.ctx_len.cpu().numpy(), page2cluster=w.page2cluster.cpu().numpy(),
+                cluster_base=w.cluster_base.cpu().numpy(),
+                replica_mask=w.cluster_replica_mask.cpu().numpy().view(np.uint32),
+                cluster_size=w.cluster_size.cpu().numpy().view(np.uint16))
+
+
+def oracle_step_fn(w):
+    import oracle
+    cfg = w.cfg
+    x = oracle_inputs(w)
+    ksum = oracle.build_summaries(x["kv_pool"], x["page_base"], x["ctx_len"], cfg.n_kv_heads, cfg.head_dim,
+                                  cfg.page_size)   # index build: outside the timed step, as on the GPU
+
+    def fn():
+        return oracle.step(x["q"], ksum, x["kv_pool"], x["page_base"], x["ctx_len"], x["page2cluster"],
+                           x["cluster_base"], x["replica_mask"], x["cluster_size"], Hkv=cfg.n_kv_heads,
+                           S=cfg.page_size, k=cfg.top_k, D=cfg.n_queues, Pmax=cfg.max_pages())
+    return fn
+
+
+def cpu_baseline(w, budget_s: float):
+    """The oracle as it stands, on this host's cores, on whole steps of the same workload."""
+    import oracle
+    cores = oracle.set_threads(0)
+    fn = oracle_step_fn(w)
+    fn()
+    n, t0 = 0, time.perf_counter()
+    while True:
+        fn()
+        n += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or n >= 50:
+            break
+    return {"value": n / el, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} whole steps of {w.cfg.name} (all {w.cfg.batch * w.cfg.n_q_heads} heads), "
+                      f"OpenMP over (request, head) units, {el:.1f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same config / metric / unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2603_17803_b200 import workloads as W
+    cfg = W.CONFIGS[args.workload]
+    K = args.steps if args.steps is not None else 5
+    Wm = args.warmup if args.warmup is not None else 1
+    w = W.generate(cfg, seed=0, device="cpu")
+    cores = oracle.set_threads(0)
+    fn = oracle_step_fn(w)
+    t0 = time.perf_counter()
+    fn()
+    t_step = time.perf_counter() - t0
+    # bounded run: if K whole steps would exceed the budget, a step is a sample of the query heads
+    budget = 150.0
+    frac = min(1.0, budget / max(1e-9, (K + Wm) * t_step))
+    heads = max(1, int(cfg.n_q_heads * frac))
+    if heads < cfg.n_q_heads:
+        import dataclasses
+        g = cfg.group
+        heads = max(g, heads // g * g)                # whole KV groups
+        cfg_s = dataclasses.replace(cfg, n_q_heads=heads, n_kv_heads=heads // g)
+        w_s = dataclasses.replace(w, cfg=cfg_s, q=w.q[:, :heads].contiguous(),
+                                  kv_pool=w.kv_pool[:, : heads // g].contiguous())
+        fn = oracle_step_fn(w_s)
+    scale = cfg.n_q_heads / heads
+    for _ in range(Wm):
+        fn()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        fn()
+    el = (time.perf_counter() - t0) * scale
+    value = K / el
+    sample = (f"each step = {heads} of {cfg.n_q_heads} query heads of {cfg.name} "
+              f"(time scaled by {scale:.2f}), {K} steps")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": K, "warmup": Wm, "ms_per_step": el / K * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "context": cfg.max_ctx(), "page_size": cfg.page_size, "top_k": cfg.top_k,
+                   "n_queues": cfg.n_queues, "n_topics": cfg.n_topics},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_swarm(a)
