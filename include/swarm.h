@@ -40,6 +40,7 @@ extern "C" {
 #define SWARM_ERR_UNSUPPORTED 2         /* valid but not implemented (head_dim != 128, ...)        */
 #define SWARM_ERR_WORKSPACE_TOO_SMALL 3 /* swarm_set_workspace not called or too few bytes         */
 #define SWARM_ERR_CUDA 4                /* a CUDA call failed; see swarm_last_cuda_error           */
+#define SWARM_ERR_STATIC_SCRATCH_TOO_SMALL 5 /* problem exceeds the built-in scratch of swarm_sparse_attn_static */
 
 /* ---- bits of the device status word ---------------------------------------------------- */
 #define SWARM_DEV_BAD_PAGE 1u           /* a selected page id lies outside its request             */
@@ -159,6 +160,36 @@ int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const 
  * partial last page are masked.  n_sel[b][h] must be >= 1. */
 int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel,
                                 const int32_t* n_sel, float* out, float* lse, void* stream);
+
+/* swarm_sparse_attn for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for integration reasons only.)
+ *
+ * Some hosts of this library may not call cudaMalloc or hand over a workspace: code running inside
+ * another framework's memory-pool callback or under a fixed, fully pre-reserved memory budget, and
+ * plugins loaded into a process whose allocator they do not own.  For them this variant computes
+ * exactly what swarm_sparse_attn computes, takes no ctx and no workspace, and allocates nothing on
+ * the host or the device: the split-K partial results live in a fixed array compiled into the
+ * library (static __device__ storage, SWARM_STATIC_SCRATCH_BYTES bytes, resident on every GPU
+ * that loads the library until the process exits).
+ *
+ *   q, k_g, v_g, n_tok, out, lse   as for swarm_sparse_attn (device pointers, 16-byte aligned);
+ *                                  k_g / v_g are bf16 [batch][n_q_heads][top_k * page_size][128]
+ *   batch, n_q_heads, top_k, page_size   the shape (page_size 16 or 32)
+ *
+ * Limit: batch * n_q_heads <= SWARM_STATIC_MAX_HEADS; larger problems are rejected with
+ * SWARM_ERR_STATIC_SCRATCH_TOO_SMALL and nothing is enqueued.  The number of key-range splits is
+ * chosen so that the partials fit the array.
+ * Set-up: the first call on each device looks up the array's device address (with that device
+ * current).  Make that first call outside any CUDA stream capture.
+ * Sharing: every call on a device uses the same array, and the array keeps what the last call
+ * wrote.  No part of it has to start at zero -- each call overwrites every slot it later reads --
+ * but two calls whose kernels overlap on the GPU (different streams, or graph branches) race on it;
+ * serialise them. */
+#define SWARM_STATIC_MAX_HEADS 2048
+#define SWARM_STATIC_SCRATCH_BYTES (256 + 4096 * (128 + 2) * 4)
+int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
+                                 int32_t batch, int32_t n_q_heads, int32_t top_k, int32_t page_size, float* out,
+                                 float* lse, void* stream);
 
 /* The fused step: stages 1-4 enqueued back to back with no host round trip.  Attention reads the
  * selected pages straight from the pool; the gathered copies are written only when k_out / v_out

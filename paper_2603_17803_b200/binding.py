@@ -16,14 +16,17 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libswarm.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 0, 1, 2, 3, 4
+ERR_STATIC_SCRATCH_TOO_SMALL = 5
+STATIC_MAX_HEADS = 2048
 DEV_BAD_PAGE, DEV_BAD_CLUSTER, DEV_BAD_REPLICA, DEV_BAD_LENGTH = 1, 2, 4, 8
 ORDER_BY_ID, UNIT_LOAD = 1, 2
-_ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA"}
+_ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA",
+              5: "STATIC_SCRATCH_TOO_SMALL"}
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
     "swarm_set_attn_splits", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
-    "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
+    "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
 )
 
 
@@ -179,6 +182,18 @@ def swarm_sparse_attn_paged(ctx, inputs: swarm_inputs, sel, n_sel, out, lse, str
     _check(load_library().swarm_sparse_attn_paged(ctx, ctypes.byref(inputs), _ptr(sel, "sel"), _ptr(n_sel, "n_sel"),
                                                   _ptr(out, "out"), _ptr(lse, "lse"), _stream(stream)),
            "swarm_sparse_attn_paged", ctx)
+
+
+def swarm_sparse_attn_static(q, k_g, v_g, n_tok, *, batch, n_q_heads, top_k, page_size, out, lse, stream=None) -> None:
+    """swarm_sparse_attn without ctx or workspace, for callers that may not allocate device memory (a plugin
+    inside another framework's allocator, a fixed memory budget): the split-K scratch is a fixed array inside
+    the library.  At most STATIC_MAX_HEADS (batch * n_q_heads) heads; calls that overlap on the GPU race on
+    that array; make the first call on a device outside stream capture."""
+    _check(load_library().swarm_sparse_attn_static(_ptr(q, "q"), _ptr(k_g, "k_g"), _ptr(v_g, "v_g"),
+                                                   _ptr(n_tok, "n_tok"), ctypes.c_int32(batch),
+                                                   ctypes.c_int32(n_q_heads), ctypes.c_int32(top_k),
+                                                   ctypes.c_int32(page_size), _ptr(out, "out"), _ptr(lse, "lse"),
+                                                   _stream(stream)), "swarm_sparse_attn_static")
 
 
 def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:

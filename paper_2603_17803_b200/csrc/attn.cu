@@ -251,3 +251,72 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
 }
 
 }  // namespace swarm
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of swarm_sparse_attn (see swarm.h).  The split-K partials live in a
+// file-scope device array instead of a caller-provided workspace.  Layout of the array:
+//   [0, 256)                       status word (unused by the contiguous-buffer kernel) + padding
+//   [256, 256 + kSlots*128*4)      partial accumulators, one 128-float row per (head, split) slot
+//   [.., .. + kSlots*2*4)          partial (max, sum) pairs
+// Host code must not pass `g_static_scratch` itself to a kernel: on the host that name is only a
+// handle.  Its device address is fetched once per device with cudaGetSymbolAddress.
+namespace {
+constexpr int kStaticSlots = 4096;
+static_assert(SWARM_STATIC_SCRATCH_BYTES == 256 + kStaticSlots * (swarm::kHeadDim + 2) * 4, "header and array size differ");
+static __device__ __align__(256) unsigned char g_static_scratch[SWARM_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+cudaError_t static_scratch_address(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (g_static_ptr[dev] == nullptr) {   // set-up for this device (idempotent if two threads race here)
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
+                                            int32_t batch, int32_t n_q_heads, int32_t top_k, int32_t page_size,
+                                            float* out, float* lse, void* stream) {
+  using namespace swarm;
+  auto bad = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (bad(q) || bad(k_g) || bad(v_g) || bad(n_tok) || bad(out) || bad(lse) || batch < 1 || n_q_heads < 1 || top_k < 1)
+    return SWARM_ERR_INVALID_ARG;
+  if (page_size != 16 && page_size != 32) return SWARM_ERR_UNSUPPORTED;
+  const long long bh = (long long)batch * n_q_heads;
+  if (bh > SWARM_STATIC_MAX_HEADS) return SWARM_ERR_STATIC_SCRATCH_TOO_SMALL;
+  if (bh * top_k >= (1LL << 31)) return SWARM_ERR_UNSUPPORTED;
+  // same split heuristic as the ctx path (about 4 CTAs per SM, >= 4 pages per split), capped by the array
+  long long n = (148 * 4 + bh - 1) / bh;
+  n = n < (top_k / 4 > 1 ? top_k / 4 : 1) ? n : (top_k / 4 > 1 ? top_k / 4 : 1);
+  n = n < kMaxSplits ? n : kMaxSplits;
+  n = n < kStaticSlots / bh ? n : kStaticSlots / bh;
+  n = n < 1 ? 1 : n;
+
+  unsigned char* base = nullptr;
+  if (static_scratch_address(&base) != cudaSuccess) return SWARM_ERR_CUDA;
+  Geometry geo{};
+  geo.B = batch; geo.Hq = n_q_heads; geo.Hkv = n_q_heads; geo.g = 1; geo.S = page_size; geo.k = top_k; geo.D = 1;
+  geo.Pmax = top_k; geo.Cmax = 1; geo.flags = 0; geo.n_pool_pages = 0;
+  AttnArgs a{};
+  a.q = static_cast<const uint16_t*>(q);
+  a.k_g = static_cast<const uint16_t*>(k_g);
+  a.v_g = static_cast<const uint16_t*>(v_g);
+  a.n_tok = n_tok;
+  a.part_acc = reinterpret_cast<float*>(base + 256);
+  a.part_ml = reinterpret_cast<float*>(base + 256 + (size_t)kStaticSlots * kHeadDim * 4);
+  a.out = out;
+  a.lse = lse;
+  a.n_splits = (int)n;
+  return launch_attention(geo, a, reinterpret_cast<uint32_t*>(base), static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? SWARM_OK : SWARM_ERR_CUDA;
+}
