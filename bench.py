@@ -153,19 +153,16 @@ def step_bytes(w, sel, n_sel):
 
 def run_swarm(args):
     import torch
-    import torch.distributed as dist
+    from paper_2603_17803_b200 import replicas
     from paper_2603_17803_b200 import workloads as W
     from paper_2603_17803_b200.session import Session
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = replicas.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
     K = args.steps if args.steps is not None else 20000
     Wm = args.warmup if args.warmup is not None else 50
     cfg = W.CONFIGS[args.workload]
@@ -176,15 +173,14 @@ def run_swarm(args):
     # independent data sets; every rank draws its own (weak scaling: fixed work per GPU)
     sessions, workloads = [], []
     for r in range(args.n_rot):
-        w = W.generate(cfg, seed=1000 * rank + r, device=dev, step=r)
+        w = W.generate(cfg, seed=replicas.replica_seed(rank, r), device=dev, step=r)
         workloads.append(w)
         sessions.append(Session(w))
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     graphs = []
@@ -260,10 +256,7 @@ def run_swarm(args):
         ms_e2e = e0.elapsed_time(e1)
     sampler.stop()
 
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = replicas.max_over_ranks([ms, ms_e2e], device=dev)
 
     status = max(s.status() for s in sessions)
     by = step_bytes(workloads[0], sessions[0].o.sel, sessions[0].o.n_sel)
@@ -276,7 +269,7 @@ def run_swarm(args):
     attn_gbs = attn_alg / (attn_us * 1e-6) / 1e9
 
     result = {
-        "metric": METRIC, "value": world * K / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC, "value": replicas.aggregate_steps_per_s(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": cfg.name, "batch": cfg.batch, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
@@ -294,7 +287,7 @@ def run_swarm(args):
                      "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU,
                      "algorithmic_bytes_per_launch": attn_alg, "avg_launch_us": attn_us,
                      "nominal_bytes_per_launch": by["kv_nominal"], "nominal_gbs": by["kv_nominal"] / (attn_us * 1e-6) / 1e9},
-        "e2e": {"value": world * K_e2e / (ms_e2e / 1e3), "unit": UNIT, "steps": K_e2e,
+        "e2e": {"value": replicas.aggregate_steps_per_s(world, K_e2e, ms_e2e), "unit": UNIT, "steps": K_e2e,
                 "h2d_bytes_per_step": B * Hq * d * 2, "d2h_bytes_per_step": B * Hq * d * 4 + B * Hq * 4 + 4 + D * 4,
                 "note": "swarm_step_host: q from pinned host memory, out/lse/n_uniq/queue_load read back; "
                         "the KV pool and its summaries are resident state, like weights"},
@@ -309,8 +302,7 @@ def run_swarm(args):
         s.close()
     if rank == 0:
         print(json.dumps(result))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle
