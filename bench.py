@@ -294,6 +294,7 @@ def run_swarm(args):
         "gpu_launches": K * 5,
         "gpu_launches_per_step": 5,
         "device_status": status,
+        "n_uniq_clusters": int(sessions[0].o.n_uniq[0]),
         "clocks": sampler.summary([(t_a, t_b), (t_e, t_f)]),
     }
     if rank == 0 and not args.skip_cpu_baseline and world == 1:

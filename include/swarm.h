@@ -47,6 +47,7 @@ extern "C" {
 #define SWARM_DEV_BAD_CLUSTER 2u        /* page2cluster entry outside the request's cluster range  */
 #define SWARM_DEV_BAD_REPLICA 4u        /* replica mask is 0 or names a queue >= n_queues          */
 #define SWARM_DEV_BAD_LENGTH 8u         /* ctx_len < 1 or more pages than the request owns         */
+#define SWARM_DEV_TIMEOUT 16u           /* a bounded wait on an asynchronous copy expired          */
 
 /* ---- flags in swarm_shape.flags --------------------------------------------------------- */
 #define SWARM_ORDER_BY_ID 1u            /* schedule clusters by id only (default: by number of
@@ -106,8 +107,9 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx);
 int32_t swarm_destroy(swarm_ctx* ctx);
 
 /* Scratch memory.  The caller allocates swarm_workspace_bytes(shape) bytes of device memory
- * (256-byte aligned) and hands them over; they must stay valid while the ctx is used.  Contents
- * need no initialisation.  Returns < 0 (minus an error code) for an invalid shape. */
+ * (256-byte aligned) and hands them over; they must stay valid while the ctx is used.  The caller
+ * need not initialise them: swarm_set_workspace enqueues the clearing it needs on `stream`.
+ * swarm_workspace_bytes returns < 0 (minus an error code) for an invalid shape. */
 int64_t swarm_workspace_bytes(const swarm_shape* shape);
 int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, void* stream);
 
@@ -182,11 +184,13 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* inputs, cons
  * Set-up: the first call on each device looks up the array's device address (with that device
  * current).  Make that first call outside any CUDA stream capture.
  * Sharing: every call on a device uses the same array, and the array keeps what the last call
- * wrote.  No part of it has to start at zero -- each call overwrites every slot it later reads --
- * but two calls whose kernels overlap on the GPU (different streams, or graph branches) race on it;
- * serialise them. */
+ * wrote.  The partial results need no clearing (each call overwrites every slot it later reads).
+ * The per-head arrival counters must be zero when a call starts: they are zero when the library is
+ * loaded and the kernel sets each one back to zero after using it, so nothing has to be cleared
+ * between calls.  Two calls whose kernels overlap on the GPU (different streams, or graph
+ * branches) race on the array; serialise them. */
 #define SWARM_STATIC_MAX_HEADS 2048
-#define SWARM_STATIC_SCRATCH_BYTES (256 + 4096 * (128 + 2) * 4)
+#define SWARM_STATIC_SCRATCH_BYTES (256 + 4096 * (128 + 2) * 4 + SWARM_STATIC_MAX_HEADS * 4)
 int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
                                  int32_t batch, int32_t n_q_heads, int32_t top_k, int32_t page_size, float* out,
                                  float* lse, void* stream);

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libswarm.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 0, 1, 2, 3, 4
 ERR_STATIC_SCRATCH_TOO_SMALL = 5
 STATIC_MAX_HEADS = 2048
-DEV_BAD_PAGE, DEV_BAD_CLUSTER, DEV_BAD_REPLICA, DEV_BAD_LENGTH = 1, 2, 4, 8
+DEV_BAD_PAGE, DEV_BAD_CLUSTER, DEV_BAD_REPLICA, DEV_BAD_LENGTH, DEV_TIMEOUT = 1, 2, 4, 8, 16
 ORDER_BY_ID, UNIT_LOAD = 1, 2
 _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA",
               5: "STATIC_SCRATCH_TOO_SMALL"}

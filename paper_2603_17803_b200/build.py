@@ -37,6 +37,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ_DIR, exist_ok=True)
     header_time = _newest(headers)
     extra = ["-Xptxas", "-v"] if verbose else []
+    if os.environ.get("SWARM_TRACE"):          # development-only cycle stamps inside the kernels
+        extra += ["-DSWARM_TRACE"]
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")

@@ -52,14 +52,17 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);
   l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
   l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
+  l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 8);
+  l.tickets = off;  off = align256(off + bh * 4);
   l.total = off;
   return l;
 }
 
 int pick_splits(const swarm_shape& s) {
-  // Enough CTAs for ~4 per SM on 148 SMs, at least 4 pages per split, at most kMaxSplits.
+  // About 2 CTAs per SM on 148 SMs (what the shared-memory rings allow), at least 4 pages per split,
+  // at most kMaxSplits.
   const int64_t bh = (int64_t)s.batch * s.n_q_heads;
-  int64_t n = (148 * 4 + bh - 1) / bh;
+  int64_t n = (148 * 2) / bh;
   n = std::min<int64_t>(n, std::max(1, s.top_k / 4));
   n = std::min<int64_t>(n, kMaxSplits);
   return (int)std::max<int64_t>(n, 1);
@@ -130,6 +133,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->last_err = cudaSuccess;
   cudaError_t e = configure_topk();
   if (e == cudaSuccess) e = configure_resolve();
+  if (e == cudaSuccess) e = configure_attention();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
@@ -156,7 +160,11 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
   if (bytes < ctx->lay.total) return SWARM_ERR_WORKSPACE_TOO_SMALL;
   ctx->ws = static_cast<uint8_t*>(device_mem);
   ctx->ws_bytes = bytes;
-  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 256, static_cast<cudaStream_t>(stream)));
+  // regions that must hold zeros between calls: status word, ticket counters, dedup flags
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 256, st));
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.flags, 0, ctx->lay.part_acc - ctx->lay.flags, st));
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.tickets, 0, ctx->lay.total - ctx->lay.tickets, st));
   return SWARM_OK;
 }
 
@@ -199,7 +207,7 @@ int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int3
   float* sc = scores ? scores : ws_ptr<float>(ctx, ctx->lay.scores);
   SWARM_TRY(launch_page_score(ctx->geo, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(in->ksum),
                               in->page_base, in->ctx_len, sc, ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, st));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, true));
   return SWARM_OK;
 }
 
@@ -212,9 +220,10 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
       bad(queue_load))
     return SWARM_ERR_INVALID_ARG;
   SWARM_TRY(launch_resolve(ctx->geo, sel, n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags), uniq,
-                           queue_of, n_uniq, queue_load, ws_ptr<uint32_t>(ctx, ctx->lay.status),
-                           static_cast<cudaStream_t>(stream)));
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), uniq, queue_of,
+                           n_uniq, queue_load,
+                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
   return SWARM_OK;
 }
 
@@ -242,6 +251,7 @@ int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const 
   a.n_tok = n_tok;
   a.part_acc = ws_ptr<float>(ctx, ctx->lay.part_acc);
   a.part_ml = ws_ptr<float>(ctx, ctx->lay.part_ml);
+  a.tickets = ws_ptr<unsigned>(ctx, ctx->lay.tickets);
   a.out = out;
   a.lse = lse;
   a.n_splits = ctx->n_splits;
@@ -261,6 +271,7 @@ AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, const int32_t*
   a.ctx_len = in->ctx_len;
   a.part_acc = ws_ptr<float>(ctx, ctx->lay.part_acc);
   a.part_ml = ws_ptr<float>(ctx, ctx->lay.part_ml);
+  a.tickets = ws_ptr<unsigned>(ctx, ctx->lay.tickets);
   a.out = out;
   a.lse = lse;
   a.n_splits = ctx->n_splits;
@@ -294,21 +305,23 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
 
   SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
                               status, st));
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, st));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true));
 
   // fork: cluster resolution needs only the selection and does not feed attention
   SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
   SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
   SWARM_TRY(launch_resolve(ctx->geo, o->sel, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags), o->uniq,
-                           o->queue_of, o->n_uniq, o->queue_load, status, ctx->side));
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), o->uniq,
+                           o->queue_of, o->n_uniq,
+                           o->queue_load, status, ctx->side));
   SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
 
   if (o->k_out != nullptr)
     SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
                             static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
   const AttnArgs a = paged_args(ctx, in, o->sel, o->n_sel, o->out, o->lse);
-  SWARM_TRY(launch_attention(ctx->geo, a, status, st));
+  SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/o->k_out == nullptr));
   SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
   return SWARM_OK;
 }

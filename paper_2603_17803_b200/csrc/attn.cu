@@ -1,17 +1,25 @@
 // Stage 4b: single-row attention (Eq. 1) over each head's selected tokens, as split-K flash decoding.
 //
 // Every query head has its own page list, so the contraction is a matrix-vector product: 4*d
-// flops per 2*d*2 bytes of K and V, i.e. bound by HBM bandwidth with arithmetic intensity 1.
-// The kernel therefore streams pages with 16-byte loads straight into registers and keeps the
-// softmax state (running max m, sum l, 128 accumulators) in fp32 registers of the warp that owns
-// the page; nothing is staged through shared memory and no operand is reused.
+// flops per 2*d*2 bytes of K and V, about one flop per byte -- bound by HBM bandwidth, so the
+// arithmetic stays on the fp32 pipes and the design effort goes into keeping bytes in flight.
 //
-// Work split: grid = (request, head, split); the split's pages are dealt round-robin to the 4
-// warps of the CTA.  A warp handles 16 tokens at a time: lane (half, c) loads 16 bytes
-// (coordinates [8c, 8c+8)) of token 2i+half for i = 0..7, so each load instruction of the warp
-// covers two whole 256-byte token rows.  The 8 partial dot products per lane are summed over the
-// 16 lanes of a half with a transposing butterfly (8 shuffles).  Logits are kept in the log2
-// domain (q is pre-scaled by log2(e)/sqrt(d)).  Warps, then splits, are merged by their (m, l).
+// Data movement: each warp owns a ring of kStages shared-memory slots.  A slot holds 16 tokens of K
+// and the same 16 tokens of V (2 x 4 KiB).  Lane 0 fills slots with bulk asynchronous copies
+// (cp.async.bulk, completion counted in bytes on the slot's mbarrier) up to kStages units ahead, so
+// the memory system always has kStages * 8 KiB per warp outstanding while the warp computes on the
+// slot that has landed.  Rings are private to a warp: no CTA-wide barrier in the main loop.
+// Every mbarrier wait is bounded; on expiry the warp records SWARM_DEV_TIMEOUT and stops.
+//
+// Compute on a slot: lane (half, c) reads 16 bytes (coordinates [8c, 8c+8)) of token 2i+half for
+// i = 0..7, conflict-free.  The 8 partial dot products per lane are summed over the 16 lanes of a
+// half with a transposing butterfly (8 shuffles).  Logits live in the log2 domain (q is pre-scaled
+// by log2(e)/sqrt(d)); softmax state (m, l, 128 accumulators) stays in fp32 registers.
+//
+// Work split: grid = (request, head, split); a split's pages are dealt round-robin to the CTA's
+// warps.  Warps are merged through shared memory, splits through fp32 partials in global memory:
+// the CTA that arrives last at the head's ticket counter merges them and writes out / lse, so no
+// second launch is needed.
 //
 // The same kernel serves the contiguous gathered buffers (swarm_sparse_attn) and the paged pool
 // (swarm_step); only the address and valid-token computation differ.
@@ -21,8 +29,40 @@ namespace swarm {
 namespace {
 
 constexpr int kAttnWarps = 4;
+constexpr int kStages = 3;
+constexpr int kUnitTokens = 16;
+constexpr int kHalfSlotBytes = kUnitTokens * kHeadDim * 2;       // 4 KiB of K (or V)
+constexpr int kSlotBytes = 2 * kHalfSlotBytes;
+constexpr int kAttnSmemBytes = kAttnWarps * kStages * kSlotBytes;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr unsigned kWaitLimit = 1u << 22;                         // polls of a try_wait that itself blocks briefly
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_addr(dst)),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
 
 __device__ __forceinline__ float warp_max(float x) {
 #pragma unroll
@@ -42,27 +82,18 @@ struct WarpState {
   float m, l, acc[8];
 };
 
-// 16 tokens (rows of 256 bytes at Kb / Vb), of which the first `valid` exist.
-__device__ __forceinline__ void attend_16(const uint16_t* __restrict__ Kb, const uint16_t* __restrict__ Vb,
-                                          int valid, const float (&qf)[8], int lane, WarpState& st) {
+// 16 tokens in a shared-memory slot (K rows then V rows, 256 bytes each), of which the first `valid` exist.
+__device__ __forceinline__ void attend_16(const unsigned char* __restrict__ slot, int valid, const float (&qf)[8],
+                                          int lane, WarpState& st) {
   const int half = lane >> 4, c = lane & 15;
-  uint4 kr[8], vr[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int t = 2 * i + half;
-    const bool ok = t < valid;
-    kr[i] = ok ? ldg_nc_v4(Kb + t * kHeadDim + c * 8) : make_uint4(0, 0, 0, 0);
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int t = 2 * i + half;
-    const bool ok = t < valid;
-    vr[i] = ok ? ldg_nc_v4(Vb + t * kHeadDim + c * 8) : make_uint4(0, 0, 0, 0);
-  }
+  const uint4* Ks = reinterpret_cast<const uint4*>(slot);
+  const uint4* Vs = reinterpret_cast<const uint4*>(slot + kHalfSlotBytes);
   float s[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const uint32_t w[4] = {kr[i].x, kr[i].y, kr[i].z, kr[i].w};
+    const int t = 2 * i + half;
+    const uint4 kr = Ks[t * 16 + c];
+    const uint32_t w[4] = {kr.x, kr.y, kr.z, kr.w};
     float a = 0.f;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -84,7 +115,7 @@ __device__ __forceinline__ void attend_16(const uint16_t* __restrict__ Kb, const
   }
   float x = s[0] + __shfl_xor_sync(0xFFFFFFFFu, s[0], 1);
   const int my_t = 2 * (c >> 1) + half;
-  if (my_t >= valid) x = -INFINITY;
+  if (my_t >= valid) x = -INFINITY;                     // padding tokens: masked (their bytes may be anything)
   const float m_new = fmaxf(st.m, warp_max(x));
   const float corr = exp2_or_zero(st.m, m_new);
   const float p = exp2_or_zero(x, m_new);
@@ -94,8 +125,11 @@ __device__ __forceinline__ void attend_16(const uint16_t* __restrict__ Kb, const
   for (int e = 0; e < 8; ++e) st.acc[e] *= corr;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
+    const int t = 2 * i + half;
     const float pi = __shfl_sync(0xFFFFFFFFu, p, half * 16 + 2 * i);
-    const uint32_t w[4] = {vr[i].x, vr[i].y, vr[i].z, vr[i].w};
+    uint4 vr = Vs[t * 16 + c];
+    if (t >= valid) vr = make_uint4(0, 0, 0, 0);        // 0 * garbage must stay 0
+    const uint32_t w[4] = {vr.x, vr.y, vr.z, vr.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       st.acc[2 * e] = fmaf(pi, bf16_lo(w[e]), st.acc[2 * e]);
@@ -107,13 +141,27 @@ __device__ __forceinline__ void attend_16(const uint16_t* __restrict__ Kb, const
 template <int S, bool kPaged>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 attn_kernel(Geometry geo, AttnArgs a, uint32_t* __restrict__ status) {
+  constexpr int SB = S / kUnitTokens;                   // 16-token units per page
+  extern __shared__ __align__(128) unsigned char ring[];
+  __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
   __shared__ float s_m[kAttnWarps], s_l[kAttnWarps];
   __shared__ float s_acc[kAttnWarps][kHeadDim];
+  __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int split = blockIdx.x % a.n_splits, bh = blockIdx.x / a.n_splits;
   const int b = bh / geo.Hq, h = bh % geo.Hq, kvh = h / geo.g;
   const int c = lane & 15;
-  const long long blk = (long long)S * kHeadDim;
+  const long long blk = (long long)S * kHeadDim;        // elements per K (or V) block of a page
+
+  if (lane == 0) {
+#pragma unroll
+    for (int sidx = 0; sidx < kStages; ++sidx) mbar_init(&bars[warp][sidx], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  SWARM_STAMP(status, 0);
+  pdl_wait();                                           // the selection comes from the previous kernel
+  SWARM_STAMP(status, 1);
 
   int n_pages, P = 0, tail = S, total_tok = 0;
   long long pool_row0 = 0;
@@ -148,40 +196,83 @@ attn_kernel(Geometry geo, AttnArgs a, uint32_t* __restrict__ status) {
 #pragma unroll
   for (int e = 0; e < 8; ++e) st.acc[e] = 0.f;
 
-  // pages j_begin + warp + 4*i; their ids are fetched 32 at a time (lane i holds the i-th)
-  for (int j0 = j_begin + warp; j0 < j_end; j0 += kAttnWarps * 32) {
+  unsigned char* my_ring = ring + (size_t)warp * kStages * kSlotBytes;
+  unsigned err = 0u;
+  SWARM_STAMP(status, 2);
+
+  // This warp's pages are j_begin + warp + kAttnWarps*i, i = 0 .. n_mine-1, handled 32 at a time
+  // (lane i holds the i-th page id); each page is SB units of 16 tokens.
+  const int n_mine = (j_end - j_begin - warp + kAttnWarps - 1) / kAttnWarps;
+  unsigned fills = 0;                                   // units issued so far (slot = fills % kStages)
+  unsigned drains = 0;                                  // units consumed so far
+  for (int i0 = 0; i0 < n_mine && err == 0u; i0 += 32) {
+    const int n_here = min(32, n_mine - i0);
     int my_p = -1;
-    if (kPaged) {
-      const int j = j0 + kAttnWarps * lane;
-      if (j < j_end) my_p = a.sel[(long long)bh * geo.k + j];
-    }
-    const int n_here = min(32, (j_end - j0 + kAttnWarps - 1) / kAttnWarps);
-    for (int i = 0; i < n_here; ++i) {
-      const int j = j0 + kAttnWarps * i;
-      const uint16_t *Kp, *Vp;
+    if (kPaged && lane < n_here) my_p = a.sel[(long long)bh * geo.k + j_begin + warp + kAttnWarps * (i0 + lane)];
+    const int units = n_here * SB;
+
+    auto unit_valid = [&](int u, int p) -> int {        // valid tokens of unit u (page i0 + u/SB, sub-block u%SB)
+      const int sb = u % SB;
       int valid;
+      if (kPaged) valid = (p == P - 1) ? tail : S;
+      else valid = min(S, total_tok - (j_begin + warp + kAttnWarps * (i0 + u / SB)) * S);
+      return max(0, min(kUnitTokens, valid - sb * kUnitTokens));
+    };
+    auto issue = [&](int u) {                           // all lanes call; lane 0 issues the copies
+      const int p = __shfl_sync(0xFFFFFFFFu, my_p, u / SB);
+      const int sb = u % SB;
+      const uint16_t *Kp, *Vp;
       if (kPaged) {
-        const int p = __shfl_sync(0xFFFFFFFFu, my_p, i);
-        if (p < 0 || p >= P) {                      // corrupt selection: flag it and skip the page
-          if (lane == 0) atomicOr(status, SWARM_DEV_BAD_PAGE);
-          continue;
-        }
-        Kp = a.kv_pool + (((pool_row0 + p) * geo.Hkv + kvh) * 2) * blk;
+        const int pc = (p < 0 || p >= P) ? 0 : p;       // a corrupt id is flagged when consumed; copy something legal
+        Kp = a.kv_pool + (((pool_row0 + pc) * geo.Hkv + kvh) * 2) * blk;
         Vp = Kp + blk;
-        valid = p == P - 1 ? tail : S;
       } else {
+        const long long j = j_begin + warp + kAttnWarps * (i0 + u / SB);
         Kp = a.k_g + ((long long)bh * geo.k + j) * blk;
         Vp = a.v_g + ((long long)bh * geo.k + j) * blk;
-        valid = min(S, total_tok - j * S);
       }
-#pragma unroll
-      for (int sb = 0; sb < S / 16; ++sb) {
-        const int v16 = min(16, valid - sb * 16);
-        if (v16 > 0) attend_16(Kp + sb * 16 * kHeadDim, Vp + sb * 16 * kHeadDim, v16, qf, lane, st);
+      if (lane == 0) {
+        const unsigned slot = fills % kStages;
+        unsigned char* dst = my_ring + slot * kSlotBytes;
+        mbar_expect_tx(&bars[warp][slot], kSlotBytes);
+        bulk_copy_g2s(dst, Kp + sb * kUnitTokens * kHeadDim, kHalfSlotBytes, &bars[warp][slot]);
+        bulk_copy_g2s(dst + kHalfSlotBytes, Vp + sb * kUnitTokens * kHeadDim, kHalfSlotBytes, &bars[warp][slot]);
       }
+      ++fills;
+    };
+
+    int issued = 0;
+    for (; issued < min(units, kStages); ++issued) issue(issued);
+    SWARM_STAMP(status, 3);
+    for (int u = 0; u < units; ++u) {
+      const unsigned slot = drains % kStages, parity = (drains / kStages) & 1u;
+      unsigned polls = 0;
+      while (!mbar_try_wait(&bars[warp][slot], parity) && ++polls < kWaitLimit) {}
+      if (__any_sync(0xFFFFFFFFu, polls >= kWaitLimit)) { err = SWARM_DEV_TIMEOUT; break; }
+      ++drains;
+      const int p = __shfl_sync(0xFFFFFFFFu, my_p, u / SB);
+      if (kPaged && (p < 0 || p >= P)) {
+        if (lane == 0) atomicOr(status, SWARM_DEV_BAD_PAGE);   // corrupt selection: skip the page, keep going
+      } else {
+        const int v16 = unit_valid(u, p);
+        if (v16 > 0) attend_16(my_ring + slot * kSlotBytes, v16, qf, lane, st);
+      }
+      __syncwarp();                                     // every lane is done reading the slot
+      if (issued < units) { issue(issued); ++issued; }
     }
   }
+  if (err) {
+    // a wait expired: give the copies still in flight a bounded chance to land before the CTA's shared
+    // memory is released, then report
+    for (; drains < fills; ++drains) {
+      const unsigned slot = drains % kStages, parity = (drains / kStages) & 1u;
+      unsigned polls = 0;
+      while (!mbar_try_wait(&bars[warp][slot], parity) && ++polls < kWaitLimit) {}
+    }
+    if (lane == 0) atomicOr(status, err);
+  }
 
+  SWARM_STAMP(status, 4);
   // merge the two halves of the warp, then the warps of the CTA
   const float l_warp = warp_sum(st.l);
 #pragma unroll
@@ -203,51 +294,60 @@ attn_kernel(Geometry geo, AttnArgs a, uint32_t* __restrict__ status) {
     L += s_l[w] * sc;
     o += s_acc[w][t] * sc;
   }
-  if (a.n_splits == 1) {
-    a.out[(long long)bh * kHeadDim + t] = L > 0.f ? o / L : 0.f;
-    if (t == 0) a.lse[bh] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-  } else {
+  if (a.n_splits > 1) {
+    // publish this split's partial, then let the last split of the head merge all of them
     const long long slot = (long long)bh * a.n_splits + split;
-    a.part_acc[slot * kHeadDim + t] = o;
-    if (t == 0) { a.part_ml[slot * 2] = M; a.part_ml[slot * 2 + 1] = L; }
+    __stcg(&a.part_acc[slot * kHeadDim + t], o);
+    if (t == 0) { __stcg(&a.part_ml[slot * 2], M); __stcg(&a.part_ml[slot * 2 + 1], L); }
+    __threadfence();
+    __syncthreads();
+    if (t == 0) s_last = (atomicAdd(&a.tickets[bh], 1u) == (unsigned)a.n_splits - 1u);
+    __syncthreads();
+    SWARM_STAMP(status, 5);
+    if (!s_last) return;
+    __threadfence();
+    const float* ml = a.part_ml + (long long)bh * a.n_splits * 2;
+    M = -INFINITY;
+    for (int sp = 0; sp < a.n_splits; ++sp) M = fmaxf(M, __ldcg(&ml[2 * sp]));
+    L = 0.f;
+    o = 0.f;
+    for (int sp = 0; sp < a.n_splits; ++sp) {
+      const float sc = exp2_or_zero(__ldcg(&ml[2 * sp]), M);
+      L += __ldcg(&ml[2 * sp + 1]) * sc;
+      o += __ldcg(&a.part_acc[((long long)bh * a.n_splits + sp) * kHeadDim + t]) * sc;
+    }
+    if (t == 0) a.tickets[bh] = 0u;                     // ready for the next launch
   }
+  a.out[(long long)bh * kHeadDim + t] = L > 0.f ? o / L : 0.f;
+  if (t == 0) a.lse[bh] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  SWARM_STAMP_ANY_CTA(status, 6);
 }
 
-// Merges the split partials of one (request, head): out = sum_s w_s acc_s / sum_s w_s l_s, w_s = 2^(m_s - M).
-__global__ void __launch_bounds__(kHeadDim)
-attn_combine_kernel(int n_splits, const float* __restrict__ part_acc, const float* __restrict__ part_ml,
-                    float* __restrict__ out, float* __restrict__ lse) {
-  const int bh = blockIdx.x, t = threadIdx.x;
-  const float* ml = part_ml + (long long)bh * n_splits * 2;
-  float M = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) M = fmaxf(M, ml[2 * s]);
-  float L = 0.f, o = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float sc = exp2_or_zero(ml[2 * s], M);
-    L += ml[2 * s + 1] * sc;
-    o += part_acc[((long long)bh * n_splits + s) * kHeadDim + t] * sc;
-  }
-  out[(long long)bh * kHeadDim + t] = L > 0.f ? o / L : 0.f;
-  if (t == 0) lse[bh] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+template <int S, bool kPaged>
+cudaError_t launch_variant(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st, bool overlap) {
+  const unsigned grid = (unsigned)geo.B * geo.Hq * a.n_splits;
+  return launch_pdl(attn_kernel<S, kPaged>, dim3(grid), dim3(kAttnWarps * 32), kAttnSmemBytes, st, overlap, geo, a,
+                    status);
 }
 
 }  // namespace
 
-cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st) {
+cudaError_t configure_attention() {
+  cudaError_t e = cudaFuncSetAttribute(attn_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+  return e;
+}
+
+cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
+                             bool overlap) {
   const bool paged = a.kv_pool != nullptr;
-  const unsigned grid = (unsigned)geo.B * geo.Hq * a.n_splits;
-  const int threads = kAttnWarps * 32;
-  if (geo.S == 16) {
-    if (paged) attn_kernel<16, true><<<grid, threads, 0, st>>>(geo, a, status);
-    else attn_kernel<16, false><<<grid, threads, 0, st>>>(geo, a, status);
-  } else {
-    if (paged) attn_kernel<32, true><<<grid, threads, 0, st>>>(geo, a, status);
-    else attn_kernel<32, false><<<grid, threads, 0, st>>>(geo, a, status);
-  }
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || a.n_splits == 1) return e;
-  attn_combine_kernel<<<geo.B * geo.Hq, kHeadDim, 0, st>>>(a.n_splits, a.part_acc, a.part_ml, a.out, a.lse);
-  return cudaGetLastError();
+  if (geo.S == 16)
+    return paged ? launch_variant<16, true>(geo, a, status, st, overlap)
+                 : launch_variant<16, false>(geo, a, status, st, overlap);
+  return paged ? launch_variant<32, true>(geo, a, status, st, overlap)
+               : launch_variant<32, false>(geo, a, status, st, overlap);
 }
 
 }  // namespace swarm
@@ -258,11 +358,14 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
 //   [0, 256)                       status word (unused by the contiguous-buffer kernel) + padding
 //   [256, 256 + kSlots*128*4)      partial accumulators, one 128-float row per (head, split) slot
 //   [.., .. + kSlots*2*4)          partial (max, sum) pairs
+//   [.., .. + kMaxHeads*4)         per-head arrival counters; zero at load (static storage) and set
+//                                  back to zero by the CTA that merges a head, so zero between calls
 // Host code must not pass `g_static_scratch` itself to a kernel: on the host that name is only a
 // handle.  Its device address is fetched once per device with cudaGetSymbolAddress.
 namespace {
 constexpr int kStaticSlots = 4096;
-static_assert(SWARM_STATIC_SCRATCH_BYTES == 256 + kStaticSlots * (swarm::kHeadDim + 2) * 4, "header and array size differ");
+static_assert(SWARM_STATIC_SCRATCH_BYTES == 256 + kStaticSlots * (swarm::kHeadDim + 2) * 4 + SWARM_STATIC_MAX_HEADS * 4,
+              "header and array size differ");
 static __device__ __align__(256) unsigned char g_static_scratch[SWARM_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
@@ -295,8 +398,8 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   const long long bh = (long long)batch * n_q_heads;
   if (bh > SWARM_STATIC_MAX_HEADS) return SWARM_ERR_STATIC_SCRATCH_TOO_SMALL;
   if (bh * top_k >= (1LL << 31)) return SWARM_ERR_UNSUPPORTED;
-  // same split heuristic as the ctx path (about 4 CTAs per SM, >= 4 pages per split), capped by the array
-  long long n = (148 * 4 + bh - 1) / bh;
+  // same split heuristic as the ctx path (about 2 CTAs per SM, >= 4 pages per split), capped by the array
+  long long n = (148 * 2) / bh;
   n = n < (top_k / 4 > 1 ? top_k / 4 : 1) ? n : (top_k / 4 > 1 ? top_k / 4 : 1);
   n = n < kMaxSplits ? n : kMaxSplits;
   n = n < kStaticSlots / bh ? n : kStaticSlots / bh;
@@ -304,6 +407,7 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
 
   unsigned char* base = nullptr;
   if (static_scratch_address(&base) != cudaSuccess) return SWARM_ERR_CUDA;
+  if (configure_attention() != cudaSuccess) return SWARM_ERR_CUDA;   // raises a kernel attribute; allocates nothing
   Geometry geo{};
   geo.B = batch; geo.Hq = n_q_heads; geo.Hkv = n_q_heads; geo.g = 1; geo.S = page_size; geo.k = top_k; geo.D = 1;
   geo.Pmax = top_k; geo.Cmax = 1; geo.flags = 0; geo.n_pool_pages = 0;
@@ -314,6 +418,7 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   a.n_tok = n_tok;
   a.part_acc = reinterpret_cast<float*>(base + 256);
   a.part_ml = reinterpret_cast<float*>(base + 256 + (size_t)kStaticSlots * kHeadDim * 4);
+  a.tickets = reinterpret_cast<unsigned*>(base + 256 + (size_t)kStaticSlots * (kHeadDim + 2) * 4);
   a.out = out;
   a.lse = lse;
   a.n_splits = (int)n;

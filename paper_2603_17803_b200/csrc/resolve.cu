@@ -1,169 +1,243 @@
 // Stage 3: cluster resolution, global merge and load-balanced bucket scheduling (Eq. 8 without the
-// already-resident term; Sec. 5.1).  One CTA: the stage is a few thousand integer operations with a
-// serial tail, and it runs beside the attention kernels, off the critical path.
+// already-resident term; Sec. 5.1).  One launch, off the critical path (it runs beside attention).
 //
-//   mark     every selected (request, page) -> global cluster id; flag[id] = 1.  Idempotent byte
-//            stores: concurrent writers store the same value, so no atomics are needed.
-//   compact  ordered ballot/popc compaction of the flags -> uniq[] ascending by id.
-//   route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
-//            with R >= 2 replicas are visited by (R ascending, id ascending) by one warp: lane j
-//            owns load[j]; one redux.min over (load << 5 | lane) restricted to the replica mask
-//            picks the least-loaded replica with ties to the lowest queue id.
-//            Under SWARM_ORDER_BY_ID the same warp visits every cluster in id order instead.
+//   mark     (all CTAs) every selected (request, page) -> global cluster id; flag[id] = 1.
+//            Idempotent byte stores: concurrent writers store the same value, so the dedup needs no
+//            atomics.  Four independent slots per thread keep the dependent loads overlapped.
+//   tail     (the CTA that finishes marking last, found with one ticket counter)
+//     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 16 flags
+//              with one 16-byte load, a warp scan places them; the flags are cleared on the way
+//              so the next call starts from zeros.
+//     route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
+//              with R >= 2 replicas are visited by (R ascending, id ascending) by one warp: lane j
+//              keeps (load[j] << 5 | j); one redux.min over the lanes named by the replica mask
+//              picks the least-loaded replica with ties to the lowest queue id, and only the lane
+//              whose value equals the minimum adds the cluster's weight.
+//              Under SWARM_ORDER_BY_ID the same warp visits every cluster in id order instead.
 #include "swarm_internal.cuh"
 
 namespace swarm {
 namespace {
 
-constexpr int kResolveThreads = 1024;
-constexpr int kResolveWarps = kResolveThreads / 32;
-constexpr int kSmemFlagBytes = 192 * 1024;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kSlotsPerThread = 4;
 
-template <bool kSmemFlags>
-__global__ void __launch_bounds__(kResolveThreads)
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) {
+  // number of non-zero bytes in w (flags are 0 or 1, but any non-zero byte counts)
+  const uint32_t t = (w | (w >> 1) | (w >> 2) | (w >> 3) | (w >> 4) | (w >> 5) | (w >> 6) | (w >> 7)) & 0x01010101u;
+  return __popc(t);
+}
+
+__global__ void __launch_bounds__(kThreads)
 resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __restrict__ n_sel,
                const int64_t* __restrict__ page_base, const int32_t* __restrict__ page2cluster,
                const int64_t* __restrict__ cluster_base, const uint32_t* __restrict__ replica_mask,
-               const uint16_t* __restrict__ cluster_size, uint8_t* __restrict__ flags_ws,
-               int32_t* __restrict__ uniq, uint8_t* __restrict__ queue_of, int32_t* __restrict__ n_uniq,
-               int32_t* __restrict__ queue_load, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(16) uint8_t sflags[];
-  __shared__ int warp_cnt[kResolveWarps];
+               const uint16_t* __restrict__ cluster_size, uint8_t* __restrict__ flags,
+               unsigned* __restrict__ ticket, uint2* __restrict__ items, int32_t* __restrict__ uniq,
+               uint8_t* __restrict__ queue_of, int32_t* __restrict__ n_uniq, int32_t* __restrict__ queue_load,
+               uint32_t* __restrict__ status) {
+  __shared__ int warp_cnt[kWarps];
   __shared__ int s_load[32];
   __shared__ unsigned s_classes;
-  __shared__ int s_total;
+  __shared__ unsigned s_item_m[32], s_item_w[32];
+  __shared__ bool s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  uint8_t* flags = kSmemFlags ? sflags : flags_ws;
   const long long c_all = cluster_base[geo.B];
   const int C = (int)min((long long)geo.Cmax, c_all);
   unsigned err = (c_all > geo.Cmax) ? SWARM_DEV_BAD_CLUSTER : 0u;
 
-  // clear (the flag array is padded to a multiple of 16 bytes)
+  SWARM_STAMP(status, 0);
+  // ---- mark -------------------------------------------------------------------------------------
   {
-    uint4* f4 = reinterpret_cast<uint4*>(flags);
-    for (int i = tid; i < (C + 15) / 16; i += kResolveThreads) f4[i] = make_uint4(0, 0, 0, 0);
+    const long long slots = (long long)geo.B * geo.Hq * geo.k;
+    const long long base = (long long)blockIdx.x * (kThreads * kSlotsPerThread) + tid;
+    int p[kSlotsPerThread], bh[kSlotsPerThread];
+    bool live[kSlotsPerThread];
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      const long long idx = base + (long long)u * kThreads;
+      live[u] = idx < slots;
+      bh[u] = live[u] ? (int)(idx / geo.k) : 0;
+      p[u] = live[u] ? sel[idx] : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      const long long idx = base + (long long)u * kThreads;
+      live[u] = live[u] && (int)(idx - (long long)bh[u] * geo.k) < n_sel[bh[u]];
+    }
+    long long cid[kSlotsPerThread];
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      cid[u] = -1;
+      if (!live[u]) continue;
+      const int b = bh[u] / geo.Hq;
+      const long long pb = page_base[b];
+      if (p[u] < 0 || p[u] >= page_base[b + 1] - pb) { err |= SWARM_DEV_BAD_PAGE; continue; }
+      const int c = page2cluster[pb + p[u]];
+      const long long cb = cluster_base[b];
+      if (c < 0 || c >= cluster_base[b + 1] - cb || cb + c >= C) { err |= SWARM_DEV_BAD_CLUSTER; continue; }
+      cid[u] = cb + c;
+    }
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u)
+      if (cid[u] >= 0) flags[cid[u]] = 1;
   }
+  if (err) atomicOr(status, err);
+  err = 0u;
+
+  // ---- which CTA is last? -------------------------------------------------------------------------
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  SWARM_STAMP_ANY_CTA(status, 1);
+
+  // ---- compact (flags are read past L1: other CTAs wrote them) -------------------------------------
   if (tid < 32) s_load[tid] = 0;
   if (tid == 0) s_classes = 0u;
-  __syncthreads();
-
-  // mark
-  const long long slots = (long long)geo.B * geo.Hq * geo.k;
-  for (long long idx = tid; idx < slots; idx += kResolveThreads) {
-    const int bh = (int)(idx / geo.k), j = (int)(idx % geo.k);
-    if (j >= n_sel[bh]) continue;
-    const int b = bh / geo.Hq;
-    const int p = sel[idx];
-    const long long pb = page_base[b];
-    if (p < 0 || p >= page_base[b + 1] - pb) { err |= SWARM_DEV_BAD_PAGE; continue; }
-    const int c = page2cluster[pb + p];
-    const long long cb = cluster_base[b];
-    if (c < 0 || c >= cluster_base[b + 1] - cb || cb + c >= C) { err |= SWARM_DEV_BAD_CLUSTER; continue; }
-    flags[cb + c] = 1;
-  }
-  __syncthreads();
-
-  // compact: warp w owns the contiguous span [w*seg, (w+1)*seg)
-  const int seg = (((C + kResolveWarps - 1) / kResolveWarps) + 31) & ~31;
-  const int lo = min(C, warp * seg), hi = min(C, lo + seg);
+  const int n_vec = (C + 15) / 16;                       // the flag array is padded to 16 bytes
+  const int vec_per_warp = (n_vec + kWarps - 1) / kWarps;
+  const int v_lo = min(n_vec, warp * vec_per_warp), v_hi = min(n_vec, v_lo + vec_per_warp);
+  uint4* f4 = reinterpret_cast<uint4*>(flags);
   int cnt = 0;
-  for (int i0 = lo; i0 < hi; i0 += 32) {
-    const int i = i0 + lane;
-    cnt += __popc(__ballot_sync(0xFFFFFFFFu, i < hi && flags[i]));
+  for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
+    const int v = v0 + lane;
+    if (v < v_hi) {
+      const uint4 f = __ldcg(f4 + v);
+      cnt += nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
+    }
   }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
   if (lane == 0) warp_cnt[warp] = cnt;
   __syncthreads();
-  int before = 0;
-  for (int w2 = 0; w2 < warp; ++w2) before += warp_cnt[w2];
-  if (tid == kResolveThreads - 1) s_total = before + cnt;
-  const unsigned lt_mask = (1u << lane) - 1u;
-  for (int i0 = lo; i0 < hi; i0 += 32) {
-    const int i = i0 + lane;
-    const bool f = i < hi && flags[i];
-    const unsigned bal = __ballot_sync(0xFFFFFFFFu, f);
-    if (f) uniq[before + __popc(bal & lt_mask)] = i;
-    before += __popc(bal);
+  int before = 0, n = 0;
+  for (int w2 = 0; w2 < kWarps; ++w2) {
+    if (w2 < warp) before += warp_cnt[w2];
+    n += warp_cnt[w2];
   }
-  __syncthreads();   // uniq[] (global) written by this CTA is visible to it after the barrier
-  const int n = s_total;
+  for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
+    const int v = v0 + lane;
+    uint4 f = make_uint4(0, 0, 0, 0);
+    if (v < v_hi) {
+      f = __ldcg(f4 + v);
+      if (f.x | f.y | f.z | f.w) __stcg(f4 + v, make_uint4(0, 0, 0, 0));   // leave zeros for the next call
+    }
+    const int mine = nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    int pos = before + incl - mine;
+    const uint32_t words[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) uniq[pos++] = v * 16 + j;
+    before += __shfl_sync(0xFFFFFFFFu, incl, 31);
+  }
+  __syncthreads();   // uniq[] written by this CTA is visible to it after the barrier
+  SWARM_STAMP_ANY_CTA(status, 2);
+
   const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
   const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
   const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
 
-  // validate masks, route single-replica clusters, record which replica counts occur
+  // ---- validate masks, route single-replica clusters, record which replica counts occur -----------
   unsigned classes = 0u;
-  for (int i = tid; i < n; i += kResolveThreads) {
+  for (int i = tid; i < n; i += kThreads) {
     const int c = uniq[i];
     const unsigned m = replica_mask[c];
-    if (m == 0u || (m & ~valid_bits)) { err |= SWARM_DEV_BAD_REPLICA; queue_of[i] = 0xFF; continue; }
+    const unsigned wgt = unit ? 1u : (unsigned)cluster_size[c];
+    if (m == 0u || (m & ~valid_bits)) {
+      err |= SWARM_DEV_BAD_REPLICA;
+      queue_of[i] = 0xFF;
+      items[i] = make_uint2(0u, 0u);
+      continue;
+    }
     const int R = __popc(m);
     if (R == 1 && !by_id) {
       const int qd = __ffs(m) - 1;
       queue_of[i] = (uint8_t)qd;
-      atomicAdd(&s_load[qd], unit ? 1 : (int)cluster_size[c]);
+      atomicAdd(&s_load[qd], (int)wgt);
+      items[i] = make_uint2(0u, 0u);                                 // nothing left to do for the serial pass
     } else {
       classes |= 1u << (R - 1);
+      items[i] = make_uint2(m, wgt << 5);                            // what the serial pass needs, in visit order
     }
   }
   if (classes) atomicOr(&s_classes, classes);
   if (err) atomicOr(status, err);
   __syncthreads();
+  SWARM_STAMP_ANY_CTA(status, 3);
 
+  // ---- the ordered greedy, one warp ------------------------------------------------------------------
+  // The visit order is materialised first (32 clusters at a time, in shared memory) so that the serial
+  // loop is a plain counted loop whose operands are fetched one step ahead of the dependent chain
+  // select -> redux.min -> compare -> add.
   if (warp == 0) {
-    unsigned load = (unsigned)s_load[lane];
-    const unsigned todo = by_id ? 1u : (s_classes & ~1u);   // one sweep by id, or one sweep per replica count
+    unsigned L = ((unsigned)s_load[lane] << 5) | (unsigned)lane;     // (load, queue id) in one comparable word
+    const unsigned todo = s_classes & ~1u;
     for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D); ++R) {
       if (!by_id && !((todo >> (R - 1)) & 1u)) continue;
+      // (mask, weight) of 32 clusters per step, fetched two steps ahead of their use
+      uint2 pre0 = lane < n ? items[lane] : make_uint2(0u, 0u);
+      uint2 pre1 = 32 + lane < n ? items[32 + lane] : make_uint2(0u, 0u);
       for (int i0 = 0; i0 < n; i0 += 32) {
         const int i = i0 + lane;
-        unsigned m = 0u, wgt = 0u;
-        if (i < n) {
-          const int c = uniq[i];
-          m = replica_mask[c];
-          if (m == 0u || (m & ~valid_bits)) m = 0u;
-          wgt = unit ? 1u : (unsigned)cluster_size[c];
-        }
+        const unsigned m = pre0.x, wgt = pre0.y;
+        pre0 = pre1;
+        pre1 = i + 64 < n ? items[i + 64] : make_uint2(0u, 0u);
         const bool mine = m != 0u && (by_id || __popc(m) == R);
-        unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
-        int my_q = 0;
-        while (pending) {
-          const int src = __ffs(pending) - 1;
-          pending &= pending - 1;
-          const unsigned mm = __shfl_sync(0xFFFFFFFFu, m, src);
-          const unsigned ww = __shfl_sync(0xFFFFFFFFu, wgt, src);
-          const unsigned key = ((mm >> lane) & 1u) ? ((load << 5) | (unsigned)lane) : 0xFFFFFFFFu;
-          const int qd = (int)(__reduce_min_sync(0xFFFFFFFFu, key) & 31u);
-          if (lane == qd) load += ww;
-          if (lane == src) my_q = qd;
+        const unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
+        const int cnt = __popc(pending);
+        if (cnt == 0) continue;
+        const int rank = __popc(pending & ((1u << lane) - 1u));
+        if (mine) { s_item_m[rank] = m; s_item_w[rank] = wgt; }
+        __syncwarp();
+        unsigned my_q = 0u;
+        unsigned mm = s_item_m[0], ww = s_item_w[0];
+        for (int r = 0; r < cnt; ++r) {
+          const unsigned mm_next = s_item_m[min(r + 1, 31)], ww_next = s_item_w[min(r + 1, 31)];
+          const unsigned key = ((mm >> lane) & 1u) ? L : 0xFFFFFFFFu;
+          const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);
+          if (L == best) L += ww;                                    // lane ids make the values distinct
+          if (rank == r) my_q = best & 31u;
+          mm = mm_next;
+          ww = ww_next;
         }
         if (mine) queue_of[i] = (uint8_t)my_q;
+        __syncwarp();
       }
     }
-    if (lane < geo.D) queue_load[lane] = (int)load;
-    if (lane == 0) *n_uniq = n;
+    SWARM_STAMP_ANY_CTA(status, 4);
+    if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
+    if (lane == 0) {
+      *n_uniq = n;
+      *ticket = 0u;                                                  // ready for the next call
+    }
   }
 }
 
 }  // namespace
 
-cudaError_t configure_resolve() {
-  return cudaFuncSetAttribute(resolve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemFlagBytes);
-}
+cudaError_t configure_resolve() { return cudaSuccess; }
 
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                           const uint16_t* cluster_size, uint8_t* flags_ws, int32_t* uniq, uint8_t* queue_of,
-                           int32_t* n_uniq, int32_t* queue_load, uint32_t* status, cudaStream_t st) {
-  const size_t flag_bytes = ((size_t)geo.Cmax + 15) & ~(size_t)15;
-  if (flag_bytes <= (size_t)kSmemFlagBytes)
-    resolve_kernel<true><<<1, kResolveThreads, flag_bytes, st>>>(geo, sel, n_sel, page_base, page2cluster,
-                                                                 cluster_base, replica_mask, cluster_size, flags_ws,
-                                                                 uniq, queue_of, n_uniq, queue_load, status);
-  else
-    resolve_kernel<false><<<1, kResolveThreads, 0, st>>>(geo, sel, n_sel, page_base, page2cluster, cluster_base,
-                                                         replica_mask, cluster_size, flags_ws, uniq, queue_of,
-                                                         n_uniq, queue_load, status);
+                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
+                           int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
+                           cudaStream_t st) {
+  const long long slots = (long long)geo.B * geo.Hq * geo.k;
+  const unsigned grid = (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
+  resolve_kernel<<<grid, kThreads, 0, st>>>(geo, sel, n_sel, page_base, page2cluster, cluster_base, replica_mask,
+                                            cluster_size, flags_ws, ticket, items, uniq, queue_of, n_uniq, queue_load,
+                                            status);
   return cudaGetLastError();
 }
 

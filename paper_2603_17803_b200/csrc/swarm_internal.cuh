@@ -12,13 +12,15 @@ constexpr int kHeadDim = 128;
 
 // Where each scratch region sits inside the caller-provided workspace (byte offsets, 256-aligned).
 struct WorkspaceLayout {
-  int64_t status;        // uint32 status word
+  int64_t status;        // uint32 status word; +64: ticket counter of the resolve kernel (both start at 0)
   int64_t scores;        // f32 [B][Hq][Pmax]          (used when the caller passes no scores buffer)
   int64_t n_tok;         // i32 [B][Hq]                (used when the caller passes no n_tok buffer)
   int64_t q_stage;       // bf16 [B][Hq][d]            (swarm_step_host)
-  int64_t flags;         // u8  [max_clusters_total]   (cluster dedup when it does not fit in smem)
+  int64_t flags;         // u8  [max_clusters_total]   cluster dedup flags (zero between calls)
   int64_t part_acc;      // f32 [B*Hq][max_splits][d]  split-K partial outputs
   int64_t part_ml;       // f32 [B*Hq][max_splits][2]  split-K partial (max, sum)
+ int64_t items;         // uint2 [max_clusters_total]  (replica mask, weight) of the clusters in visit order
+  int64_t tickets;       // u32 [B*Hq]                 arrival counters of the split merge (zero between calls)
   int64_t total;
 };
 
@@ -33,6 +35,7 @@ struct Geometry {   // plain copy of the shape in kernel-friendly form
 // ---- one-time per-device kernel attribute set-up (dynamic shared-memory limits) ---------------
 cudaError_t configure_topk();
 cudaError_t configure_resolve();
+cudaError_t configure_attention();
 
 // ---- kernel launchers (each returns cudaGetLastError() after the launch) ----------------------
 cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool, const int64_t* page_base,
@@ -40,12 +43,14 @@ cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool,
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st);
+// `overlap`: launch with programmatic dependent launch after the previous kernel of the stream.
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, cudaStream_t st);
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap);
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                           const uint16_t* cluster_size, uint8_t* flags_ws, int32_t* uniq, uint8_t* queue_of,
-                           int32_t* n_uniq, int32_t* queue_load, uint32_t* status, cudaStream_t st);
+                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
+                           int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
+                           cudaStream_t st);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,
                           int32_t* n_tok, uint32_t* status, cudaStream_t st);
@@ -62,11 +67,13 @@ struct AttnArgs {
   const int32_t* ctx_len;
   float* part_acc;
   float* part_ml;
+  unsigned* tickets;   // [B*Hq] arrival counters of the split merge; zero between launches
   float* out;
   float* lse;
   int n_splits;
 };
-cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st);
+cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
+                             bool overlap = false);
 
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -81,5 +88,46 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
 }
 
 __device__ __forceinline__ int pages_of(int ctx_len, int S) { return (ctx_len + S - 1) / S; }
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running; it must call pdl_wait() before it
+// touches anything the predecessor writes.  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+// Launches `kernel` so that it may overlap the tail of the previous kernel in `st` (see pdl_wait).
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap,
+                       Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Development-only cycle stamps (compiled in with -DSWARM_TRACE): thread 0 of CTA 0 records clock64()
+// at up to 16 numbered points of a kernel into bytes [128, 256) of the workspace's status block, where
+// a developer reads them back from the workspace tensor.  Absent from normal builds.
+#ifdef SWARM_TRACE
+#define SWARM_STAMP(status, i)                                                      \
+  do {                                                                              \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
+      reinterpret_cast<unsigned long long*>(status)[16 + (i)] = clock64();          \
+  } while (0)
+#define SWARM_STAMP_ANY_CTA(status, i)                                               \
+  do {                                                                              \
+    if (threadIdx.x == 0) reinterpret_cast<unsigned long long*>(status)[16 + (i)] = clock64(); \
+  } while (0)
+#else
+#define SWARM_STAMP(status, i) do { } while (0)
+#define SWARM_STAMP_ANY_CTA(status, i) do { } while (0)
+#endif
 
 }  // namespace swarm

@@ -2,18 +2,24 @@
 // activated).  One CTA per (request, query head).
 //
 // Scores become order-preserving 32-bit keys (-0 folded onto +0 so the two compare equal).  A
-// most-significant-digit radix select (4 passes of 8 bits, warp-aggregated shared-memory
-// histograms) finds the exact key T of the k-th best page and how many pages tie with it.  The
-// result is then written by an ordered ballot/popc compaction in page-id order: every page with
-// key > T, plus the first (k - #greater) pages with key == T.  That order gives "ties go to the
-// lower page id" and the ascending-id output at once.
+// most-significant-digit radix select finds the exact key T of the k-th best page and how many
+// pages tie with it.  The digits are taken relative to the list's own [min, max] key range, 11
+// bits at a time: page scores of one head sit in a narrow band (often a single binade), and digits
+// cut from the raw bit pattern would throw them all into a handful of histogram bins.  With range-
+// relative digits the shared-memory atomics spread over all 2048 bins and two levels usually finish.
+// The result is then written in page-id order: every page with key > T, plus the first
+// (k - #greater) pages with key == T, placed by a block-wide scan of per-thread counts.  That order
+// gives "ties go to the lower page id" and the ascending-id output at once.
+//
+// topk_regs keeps ITEMS consecutive pages per thread in registers (lists of up to 16384 pages);
+// topk_generic walks lists of any length in shared or global memory with the same algorithm.
 #include "swarm_internal.cuh"
 
 namespace swarm {
 namespace {
 
-constexpr int kTopkThreads = 1024;
-constexpr int kTopkWarps = kTopkThreads / 32;
+constexpr int kBins = 2048;
+constexpr int kDigitBits = 11;
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -21,102 +27,242 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-template <bool kKeysInSmem>
-__global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
-            int32_t* __restrict__ sel, int32_t* __restrict__ n_sel) {
-  extern __shared__ uint32_t skeys[];
-  __shared__ int hist[257];
-  __shared__ int warp_gt[kTopkWarps], warp_eq[kTopkWarps];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_remaining;
+// Shared state of one radix-select run.
+struct SelectState {
+  int hist[kBins];
+  int warp_tot[32];
+  uint32_t red_min[32], red_max[32];
+  uint32_t base;       // keys below `base` are out; candidates satisfy key - base < 2^bits
+  int bits;            // undecided low bits of the candidates
+  int remaining;       // rank still to find among the candidates (counted from the top)
+};
 
+// After the histogram of the current level is complete: locate the bin holding rank `remaining`
+// from the top, narrow (base, bits, remaining), clear the histogram.  All threads call it.
+template <int THREADS>
+__device__ __forceinline__ void narrow(SelectState& st, int tid, int shift) {
+  constexpr int PER = kBins / THREADS;                      // bins per thread, highest bins first
+  const int lane = tid & 31, warp = tid >> 5;
+  int c[PER], sum = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    c[j] = st.hist[kBins - 1 - (tid * PER + j)];
+    sum += c[j];
+  }
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) st.warp_tot[warp] = incl;
+  const uint32_t base = st.base;
+  const int remaining = st.remaining;
+  __syncthreads();
+  int above = incl - sum;
+  for (int w2 = 0; w2 < warp; ++w2) above += st.warp_tot[w2];
+#pragma unroll
+  for (int j = 0; j < PER; ++j) st.hist[kBins - 1 - (tid * PER + j)] = 0;
+  if (above < remaining && remaining <= above + sum) {
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if (above < remaining && remaining <= above + c[j]) {
+        st.base = base + ((uint32_t)(kBins - 1 - (tid * PER + j)) << shift);
+        st.bits = shift;
+        st.remaining = remaining - above;
+        above = remaining;                                   // stop
+      } else {
+        above += c[j];
+      }
+    }
+  }
+  __syncthreads();
+}
+
+template <int THREADS>
+__device__ __forceinline__ void block_minmax(SelectState& st, int tid, uint32_t lo, uint32_t hi) {
+  const int lane = tid & 31, warp = tid >> 5;
+  lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+  hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+  if (lane == 0) { st.red_min[warp] = lo; st.red_max[warp] = hi; }
+  __syncthreads();
+  if (warp == 0) {
+    lo = lane < THREADS / 32 ? st.red_min[lane] : 0xFFFFFFFFu;
+    hi = lane < THREADS / 32 ? st.red_max[lane] : 0u;
+    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    if (lane == 0) {
+      st.base = lo;
+      st.bits = 32 - __clz(hi - lo);                        // 0 when every key is equal
+    }
+  }
+  __syncthreads();
+}
+
+// ---- register-resident variant -------------------------------------------------------------------
+template <int THREADS, int ITEMS>
+__global__ void __launch_bounds__(THREADS)
+topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
+                 int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status) {
+  __shared__ SelectState st;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.x, b = bh / geo.Hq;
+  pdl_launch_dependents();
+  SWARM_STAMP(status, 0);
+  for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
+  pdl_wait();                                               // the scores come from the previous kernel
+  SWARM_STAMP(status, 1);
   const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
 
-  auto key_at = [&](int i) -> uint32_t { return kKeysInSmem ? skeys[i] : score_key(s[i]); };
+  // thread t owns pages [t*ITEMS, (t+1)*ITEMS); keys of pages that do not exist are never used
+  uint32_t key[ITEMS];
+  const int p0 = tid * ITEMS;
+  if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
+#pragma unroll
+    for (int j = 0; j < ITEMS; j += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(s + p0 + j);
+      key[j] = score_key(v.x); key[j + 1] = score_key(v.y); key[j + 2] = score_key(v.z); key[j + 3] = score_key(v.w);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) key[j] = p0 + j < P ? score_key(s[p0 + j]) : 0u;
+  }
+  if (tid == 0) st.remaining = k_eff;
+  SWARM_STAMP(status, 2);
 
-  if (kKeysInSmem)
-    for (int i = tid; i < P; i += kTopkThreads) skeys[i] = score_key(s[i]);
-  if (tid == 0) { s_prefix = 0u; s_remaining = k_eff; }
+  uint32_t T = 0u;
+  int need_eq = P;                                          // k_eff == P keeps everything
+  if (k_eff < P) {
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j)
+      if (p0 + j < P) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+    block_minmax<THREADS>(st, tid, lo, hi);
+    SWARM_STAMP(status, 3);
+    for (int level = 0; level < 4 && st.bits > 0; ++level) {
+      const uint32_t base = st.base;
+      const int bits = st.bits;
+      const int shift = max(bits - kDigitBits, 0);
+      const uint32_t width_m1 = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
+#pragma unroll
+      for (int j = 0; j < ITEMS; ++j) {
+        const uint32_t rel = key[j] - base;
+        if (p0 + j < P && rel <= width_m1) atomicAdd(&st.hist[rel >> shift], 1);
+      }
+      __syncthreads();
+      SWARM_STAMP(status, 4 + 2 * level);
+      narrow<THREADS>(st, tid, shift);
+      SWARM_STAMP(status, 5 + 2 * level);
+    }
+    T = st.base;
+    need_eq = st.remaining;
+  }
+  SWARM_STAMP(status, 12);
+
+  // ordered output: packed (greater, equal) counts per thread, one block-wide exclusive scan
+  int cnt = 0;
+#pragma unroll
+  for (int j = 0; j < ITEMS; ++j)
+    if (p0 + j < P) cnt += (key[j] > T ? 1 : 0) + (key[j] == T ? 0x10000 : 0);
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  __syncthreads();                                          // warp_tot may still be read by narrow()
+  if (lane == 31) st.warp_tot[warp] = incl;
   __syncthreads();
-
-  if (k_eff > 0 && k_eff < P) {
-    const int P_round = (P + 31) & ~31;
-    uint32_t mask = 0u;
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      for (int i = tid; i < 257; i += kTopkThreads) hist[i] = 0;
-      __syncthreads();
-      const uint32_t prefix = s_prefix;
-      for (int i = tid; i < P_round; i += kTopkThreads) {
-        int digit = 256;                                   // bin 256 collects non-candidates
-        if (i < P) {
-          const uint32_t key = key_at(i);
-          if ((key & mask) == prefix) digit = (key >> shift) & 255;
-        }
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
-        if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
-      }
-      __syncthreads();
-      if (warp == 0) {
-        // lane L owns bins [255-8L-7, 255-8L]; find the bin where the count from the top reaches `remaining`
-        int local[8], sum = 0;
+  int before = incl - cnt;
+  for (int w2 = 0; w2 < warp; ++w2) before += st.warp_tot[w2];
+  int gt_before = before & 0xFFFF, eq_before = before >> 16;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { local[j] = hist[255 - 8 * lane - j]; sum += local[j]; }
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += t;
-        }
-        const int remaining = s_remaining;
-        int above = incl - sum;                            // pages in bins above this lane's bins
-        if (above < remaining && remaining <= incl) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (above < remaining && remaining <= above + local[j]) {
-              s_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
-              s_remaining = remaining - above;
-              above = remaining;                           // stop
-            } else {
-              above += local[j];
-            }
-          }
-        }
-      }
-      mask |= 255u << shift;
-      __syncthreads();
+  for (int j = 0; j < ITEMS; ++j) {
+    if (p0 + j < P) {
+      const bool gt = key[j] > T, eq = key[j] == T;
+      if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = p0 + j;
+      gt_before += gt;
+      eq_before += eq;
     }
   }
+  for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
+  if (tid == 0) n_sel[bh] = k_eff;
+  SWARM_STAMP(status, 13);
+}
 
-  // Ordered compaction.  k_eff == P keeps everything (T = 0, every key > T or == T with room).
-  const bool take_all = (k_eff == P);
-  const uint32_t T = take_all ? 0u : s_prefix;
-  const int need_eq = take_all ? P : s_remaining;
-  const int seg = (((P + kTopkWarps - 1) / kTopkWarps) + 31) & ~31;   // per-warp contiguous span
-  const int lo = min(P, warp * seg), hi = min(P, lo + seg);
+// ---- generic variant: any list length, keys in shared memory when they fit, else re-read ----------
+constexpr int kGenericThreads = 1024;
+
+template <bool kKeysInSmem>
+__global__ void __launch_bounds__(kGenericThreads)
+topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
+                    int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status) {
+  extern __shared__ uint32_t skeys[];
+  __shared__ SelectState st;
+  __shared__ int warp_gt[32], warp_eq[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int bh = blockIdx.x, b = bh / geo.Hq;
+  pdl_launch_dependents();
+  for (int i = tid; i < kBins; i += kGenericThreads) st.hist[i] = 0;
+  pdl_wait();
+  const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));
+  const int k_eff = min(geo.k, P);
+  const float* s = scores + (long long)bh * geo.Pmax;
+  int32_t* out = sel + (long long)bh * geo.k;
+  auto key_at = [&](int i) -> uint32_t { return kKeysInSmem ? skeys[i] : score_key(s[i]); };
+
+  uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+  for (int i = tid; i < P; i += kGenericThreads) {
+    const uint32_t key = score_key(s[i]);
+    if (kKeysInSmem) skeys[i] = key;
+    lo = min(lo, key);
+    hi = max(hi, key);
+  }
+  if (tid == 0) st.remaining = k_eff;
+  uint32_t T = 0u;
+  int need_eq = P;
+  if (k_eff < P) {
+    block_minmax<kGenericThreads>(st, tid, lo, hi);
+    for (int level = 0; level < 4 && st.bits > 0; ++level) {
+      const uint32_t base = st.base;
+      const int bits = st.bits;
+      const int shift = max(bits - kDigitBits, 0);
+      const uint32_t width_m1 = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
+      for (int i = tid; i < P; i += kGenericThreads) {
+        const uint32_t rel = key_at(i) - base;
+        if (rel <= width_m1) atomicAdd(&st.hist[rel >> shift], 1);
+      }
+      __syncthreads();
+      narrow<kGenericThreads>(st, tid, shift);
+    }
+    T = st.base;
+    need_eq = st.remaining;
+  } else {
+    __syncthreads();
+  }
+
+  // ordered ballot/popc compaction; warp w owns the contiguous span [w*seg, (w+1)*seg)
+  const int seg = (((P + 31) / 32 + 31) & ~31);
+  const int w_lo = min(P, warp * seg), w_hi = min(P, w_lo + seg);
   int cnt_gt = 0, cnt_eq = 0;
-  for (int i0 = lo; i0 < hi; i0 += 32) {
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
     const int i = i0 + lane;
-    const uint32_t key = i < hi ? key_at(i) : 0u;
-    const bool gt = i < hi && key > T, eq = i < hi && key == T;
-    cnt_gt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
-    cnt_eq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+    const uint32_t key = i < w_hi ? key_at(i) : 0u;
+    cnt_gt += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && key > T));
+    cnt_eq += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && key == T));
   }
   if (lane == 0) { warp_gt[warp] = cnt_gt; warp_eq[warp] = cnt_eq; }
   __syncthreads();
   int gt_before = 0, eq_before = 0;
   for (int w2 = 0; w2 < warp; ++w2) { gt_before += warp_gt[w2]; eq_before += warp_eq[w2]; }
   const unsigned lt_mask = (1u << lane) - 1u;
-  for (int i0 = lo; i0 < hi; i0 += 32) {
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
     const int i = i0 + lane;
-    const uint32_t key = i < hi ? key_at(i) : 0u;
-    const bool gt = i < hi && key > T, eq = i < hi && key == T;
+    const uint32_t key = i < w_hi ? key_at(i) : 0u;
+    const bool gt = i < w_hi && key > T, eq = i < w_hi && key == T;
     const unsigned bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
     const int my_gt = gt_before + __popc(bg & lt_mask);
     const int my_eq = eq_before + __popc(be & lt_mask);
@@ -124,26 +270,37 @@ topk_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __res
     gt_before += __popc(bg);
     eq_before += __popc(be);
   }
-  for (int j = k_eff + tid; j < geo.k; j += kTopkThreads) out[j] = -1;
+  for (int j = k_eff + tid; j < geo.k; j += kGenericThreads) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
 }
+
+constexpr size_t kSmemKeyBytes = 160 * 1024;
 
 }  // namespace
 
 cudaError_t configure_topk() {
-  return cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  return cudaFuncSetAttribute(topk_generic_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)kSmemKeyBytes);
 }
 
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, cudaStream_t st) {
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap) {
+  const dim3 grid(geo.B * geo.Hq);
+#define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                    \
+  return launch_pdl(topk_regs_kernel<THREADS, ITEMS>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
+                    ctx_len, sel, n_sel, status)
+  if (geo.Pmax <= 1024) SWARM_TOPK_REGS(128, 8);
+  if (geo.Pmax <= 2048) SWARM_TOPK_REGS(256, 8);
+  if (geo.Pmax <= 4096) SWARM_TOPK_REGS(512, 8);
+  if (geo.Pmax <= 8192) SWARM_TOPK_REGS(1024, 8);
+  if (geo.Pmax <= 16384) SWARM_TOPK_REGS(1024, 16);
+#undef SWARM_TOPK_REGS
   const size_t key_bytes = (size_t)geo.Pmax * sizeof(uint32_t);
-  const int n_lists = geo.B * geo.Hq;
-  if (key_bytes <= 200 * 1024) {
-    topk_kernel<true><<<n_lists, kTopkThreads, key_bytes, st>>>(geo, scores, ctx_len, sel, n_sel);
-  } else {
-    topk_kernel<false><<<n_lists, kTopkThreads, 0, st>>>(geo, scores, ctx_len, sel, n_sel);
-  }
-  return cudaGetLastError();
+  if (key_bytes <= kSmemKeyBytes)
+    return launch_pdl(topk_generic_kernel<true>, grid, dim3(kGenericThreads), key_bytes, st, overlap, geo, scores,
+                      ctx_len, sel, n_sel, status);
+  return launch_pdl(topk_generic_kernel<false>, grid, dim3(kGenericThreads), 0, st, overlap, geo, scores, ctx_len,
+                    sel, n_sel, status);
 }
 
 }  // namespace swarm
