@@ -38,7 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     header_time = _newest(headers)
     extra = ["-Xptxas", "-v"] if verbose else []
     if os.environ.get("SWARM_TRACE"):          # development-only cycle stamps inside the kernels
-        extra += ["-DSWARM_TRACE"]
+        extra += ["-DSWARM_TRACE=" + os.environ["SWARM_TRACE"]]
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")

@@ -14,8 +14,7 @@ struct swarm_ctx {
   WorkspaceLayout lay;
   uint8_t* ws;
   int64_t ws_bytes;
-  int default_splits;
-  int n_splits;
+  int user_splits;            // 0 = chosen from the shape
   cudaStream_t side;          // cluster resolution runs here beside attention
   cudaEvent_t ev_fork, ev_join;
   cudaError_t last_err;
@@ -53,17 +52,19 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
   l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
   l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 8);
+  l.selmap = off;   off = align256(off + bh * selmap_pitch_bytes(s.max_pages_per_req));
   l.tickets = off;  off = align256(off + bh * 4);
   l.total = off;
   return l;
 }
 
-int pick_splits(const swarm_shape& s) {
-  // About 2 CTAs per SM on 148 SMs (what the shared-memory rings allow), at least 4 pages per split,
-  // at most kMaxSplits.
-  const int64_t bh = (int64_t)s.batch * s.n_q_heads;
-  int64_t n = (148 * 2) / bh;
-  n = std::min<int64_t>(n, std::max(1, s.top_k / 4));
+int pick_splits(const swarm_ctx* ctx, bool paged) {
+  // About 2 CTAs per SM on 148 SMs (what the shared-memory rings allow), at most kMaxSplits; for gathered
+  // buffers at least 4 pages per split.
+  if (ctx->user_splits > 0) return ctx->user_splits;
+  const int64_t groups = attention_groups(ctx->geo, paged);
+  int64_t n = (148 * 2) / groups;
+  if (!paged) n = std::min<int64_t>(n, std::max(1, ctx->geo.k / 4));
   n = std::min<int64_t>(n, kMaxSplits);
   return (int)std::max<int64_t>(n, 1);
 }
@@ -129,9 +130,10 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->lay = make_layout(*shape);
   ctx->ws = nullptr;
   ctx->ws_bytes = 0;
-  ctx->default_splits = ctx->n_splits = pick_splits(*shape);
+  ctx->user_splits = 0;
   ctx->last_err = cudaSuccess;
-  cudaError_t e = configure_topk();
+  cudaError_t e = configure_score();
+  if (e == cudaSuccess) e = configure_topk();
   if (e == cudaSuccess) e = configure_resolve();
   if (e == cudaSuccess) e = configure_attention();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
@@ -170,7 +172,7 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
 
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits) {
   if (ctx == nullptr || n_splits < 0 || n_splits > kMaxSplits) return SWARM_ERR_INVALID_ARG;
-  ctx->n_splits = n_splits == 0 ? ctx->default_splits : n_splits;
+  ctx->user_splits = n_splits;
   return SWARM_OK;
 }
 
@@ -223,7 +225,7 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
                            ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), uniq, queue_of,
                            n_uniq, queue_load,
-                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream), false));
   return SWARM_OK;
 }
 
@@ -254,19 +256,18 @@ int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const 
   a.tickets = ws_ptr<unsigned>(ctx, ctx->lay.tickets);
   a.out = out;
   a.lse = lse;
-  a.n_splits = ctx->n_splits;
+  a.n_splits = pick_splits(ctx, false);
   SWARM_TRY(launch_attention(ctx->geo, a, ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
   return SWARM_OK;
 }
 
 namespace {
-AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
-                    float* out, float* lse) {
+AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, float* out, float* lse) {
   AttnArgs a{};
   a.q = static_cast<const uint16_t*>(in->q);
   a.kv_pool = static_cast<const uint16_t*>(in->kv_pool);
-  a.sel = sel;
-  a.n_sel = n_sel;
+  a.selmap = ws_ptr<uint8_t>(ctx, ctx->lay.selmap);
+  a.selmap_pitch = selmap_pitch_bytes(ctx->geo.Pmax);
   a.page_base = in->page_base;
   a.ctx_len = in->ctx_len;
   a.part_acc = ws_ptr<float>(ctx, ctx->lay.part_acc);
@@ -274,7 +275,7 @@ AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, const int32_t*
   a.tickets = ws_ptr<unsigned>(ctx, ctx->lay.tickets);
   a.out = out;
   a.lse = lse;
-  a.n_splits = ctx->n_splits;
+  a.n_splits = pick_splits(ctx, true);
   return a;
 }
 }  // namespace
@@ -284,8 +285,9 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const in
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!pool_inputs_ok(in) || bad(in->q) || bad(sel) || bad(n_sel) || bad(out) || bad(lse)) return SWARM_ERR_INVALID_ARG;
-  SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, sel, n_sel, out, lse),
-                             ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SWARM_TRY(launch_selmap_from_sel(ctx->geo, sel, n_sel, ws_ptr<uint8_t>(ctx, ctx->lay.selmap), st));
+  SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, out, lse), ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
   return SWARM_OK;
 }
 
@@ -305,23 +307,28 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
 
   SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
                               status, st));
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true));
+  // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true,
+                        ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
+                        ws_ptr<uint8_t>(ctx, ctx->lay.flags)));
 
-  // fork: cluster resolution needs only the selection and does not feed attention
+  // fork: cluster resolution and attention both need only the selection.  Resolution is the longer of
+  // the two (its greedy pass is serial), so it stays on the caller's stream right behind the selection
+  // kernel (programmatic dependent launch) and attention takes the auxiliary stream.
   SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
   SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
-  SWARM_TRY(launch_resolve(ctx->geo, o->sel, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), o->uniq,
-                           o->queue_of, o->n_uniq,
-                           o->queue_load, status, ctx->side));
-  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
-
   if (o->k_out != nullptr)
     SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
-                            static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
-  const AttnArgs a = paged_args(ctx, in, o->sel, o->n_sel, o->out, o->lse);
-  SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/o->k_out == nullptr));
+                            static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status,
+                            ctx->side));
+  const AttnArgs a = paged_args(ctx, in, o->out, o->lse);
+  SWARM_TRY(launch_attention(ctx->geo, a, status, ctx->side, /*overlap=*/false));
+  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
+
+  SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), o->uniq,
+                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true));
   SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
   return SWARM_OK;
 }

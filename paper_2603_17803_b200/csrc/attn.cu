@@ -1,28 +1,33 @@
-// Stage 4b: single-row attention (Eq. 1) over each head's selected tokens, as split-K flash decoding.
+// Stage 4b: single-row attention (Eq. 1) over each head's selected tokens, as split-K flash decoding
+// on the tensor cores.
 //
-// Every query head has its own page list, so the contraction is a matrix-vector product: 4*d
-// flops per 2*d*2 bytes of K and V, about one flop per byte -- bound by HBM bandwidth, so the
-// arithmetic stays on the fp32 pipes and the design effort goes into keeping bytes in flight.
+// Roofline: every selected K/V page has to come out of HBM once; with one query row per head the
+// arithmetic is ~1 flop per byte, so the kernel is bound by HBM bandwidth and everything below is
+// about moving each byte once and spending as few issue slots on it as possible.
 //
-// Data movement: each warp owns a ring of kStages shared-memory slots.  A slot holds 16 tokens of K
-// and the same 16 tokens of V (2 x 4 KiB).  Lane 0 fills slots with bulk asynchronous copies
-// (cp.async.bulk, completion counted in bytes on the slot's mbarrier) up to kStages units ahead, so
-// the memory system always has kStages * 8 KiB per warp outstanding while the warp computes on the
-// slot that has landed.  Rings are private to a warp: no CTA-wide barrier in the main loop.
-// Every mbarrier wait is bounded; on expiry the warp records SWARM_DEV_TIMEOUT and stops.
+//  * Heads of a GQA group share a KV head and, in practice, about half of their pages.  A CTA
+//    therefore serves one (request, KV head, page range): it forms the union of its query heads'
+//    selections from the per-head page bitmaps the selection kernel leaves behind, loads every page
+//    of the union once, and lets each head take part only in the pages it selected (the others are
+//    masked to -inf for that head).  The g <= 8 heads are the M rows of the score MMA.
+//  * Pages travel by TMA: cp.async.bulk.tensor tiles of 16 tokens x 64 coordinates with the 128-byte
+//    swizzle, completion counted on an mbarrier.  Each warp owns a ring of kStages slots (16 tokens of
+//    K and of V = 8 KiB per slot) and keeps it full, so kStages * 8 KiB per warp are always in flight.
+//    Every mbarrier wait is bounded; on expiry the warp records SWARM_DEV_TIMEOUT and stops.
+//  * Arithmetic: mma.sync m16n8k16 bf16 with fp32 accumulation.  S^T[head][token] = Q K^T takes K
+//    tiles with ldmatrix; the probabilities go back in as the B operand of O^T[dim][head] = V^T P^T
+//    (V^T through ldmatrix.trans), so all 16 M rows of that MMA carry useful coordinates.  P is fed as
+//    a bf16 high part plus a bf16 low part (two MMAs), which keeps the result within fp32 rounding of
+//    the exact sum.  About 110 warp instructions per 8 KiB, against ~500 per head on the fp32 pipes.
+//  * Softmax state (m, l per head; 128 x 8 outputs) stays in registers; logits in the log2 domain.
+//    Warps are merged through shared memory, page ranges (splits) through fp32 partials in global
+//    memory: the CTA that arrives last at the group's ticket counter merges them, no second launch.
 //
-// Compute on a slot: lane (half, c) reads 16 bytes (coordinates [8c, 8c+8)) of token 2i+half for
-// i = 0..7, conflict-free.  The 8 partial dot products per lane are summed over the 16 lanes of a
-// half with a transposing butterfly (8 shuffles).  Logits live in the log2 domain (q is pre-scaled
-// by log2(e)/sqrt(d)); softmax state (m, l, 128 accumulators) stays in fp32 registers.
-//
-// Work split: grid = (request, head, split); a split's pages are dealt round-robin to the CTA's
-// warps.  Warps are merged through shared memory, splits through fp32 partials in global memory:
-// the CTA that arrives last at the head's ticket counter merges them and writes out / lse, so no
-// second launch is needed.
-//
-// The same kernel serves the contiguous gathered buffers (swarm_sparse_attn) and the paged pool
-// (swarm_step); only the address and valid-token computation differ.
+// The same kernel serves the contiguous gathered buffers (swarm_sparse_attn: one head per CTA, every
+// page slot of the head) and the paged pool (swarm_step, swarm_sparse_attn_paged).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "swarm_internal.cuh"
 
 namespace swarm {
@@ -31,12 +36,16 @@ namespace {
 constexpr int kAttnWarps = 4;
 constexpr int kStages = 3;
 constexpr int kUnitTokens = 16;
-constexpr int kHalfSlotBytes = kUnitTokens * kHeadDim * 2;       // 4 KiB of K (or V)
-constexpr int kSlotBytes = 2 * kHalfSlotBytes;
-constexpr int kAttnSmemBytes = kAttnWarps * kStages * kSlotBytes;
+constexpr int kBoxBytes = kUnitTokens * 128;                       // 16 token rows x 64 bf16
+constexpr int kSlotBytes = 4 * kBoxBytes;                          // K lo, K hi, V lo, V hi
+constexpr int kRingBytes = kAttnWarps * kStages * kSlotBytes;
+constexpr int kListCap = 1024;                                     // pages per round = 32 bitmap words
+constexpr int kScratchBytes = 8192;   // page list (5 KiB) during the main loop; (max, sum, weight) tables (6 KiB) in the merge
+constexpr int kAttnSmemBytes = 1024 /*alignment slack*/ + kRingBytes + kScratchBytes;
+static_assert(kListCap * 5 <= kScratchBytes && (16 + kAttnWarps) * kMaxSplits * 4 <= kScratchBytes, "scratch too small");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr unsigned kWaitLimit = 1u << 22;                         // polls of a try_wait that itself blocks briefly
+constexpr unsigned kWaitLimit = 1u << 22;                          // polls of a try_wait that itself blocks briefly
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -57,277 +66,487 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_addr(dst)),
-               "l"(src), "r"(bytes), "r"(smem_addr(bar))
-               : "memory");
+// 2-D tiled TMA load: box (64 coordinates, 16 rows) at (x, row) of the tensor behind `map`.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int row, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(row), "r"(smem_addr(bar))
+      : "memory");
 }
-
-__device__ __forceinline__ float warp_max(float x) {
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
-  return x;
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
 }
-__device__ __forceinline__ float warp_sum(float x) {
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-  return x;
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ float exp2_or_zero(float x, float ref) {   // 2^(x-ref), 0 when x = -inf
   return x == -INFINITY ? 0.f : exp2f(x - ref);
 }
-
-struct WarpState {
-  float m, l, acc[8];
-};
-
-// 16 tokens in a shared-memory slot (K rows then V rows, 256 bytes each), of which the first `valid` exist.
-__device__ __forceinline__ void attend_16(const unsigned char* __restrict__ slot, int valid, const float (&qf)[8],
-                                          int lane, WarpState& st) {
-  const int half = lane >> 4, c = lane & 15;
-  const uint4* Ks = reinterpret_cast<const uint4*>(slot);
-  const uint4* Vs = reinterpret_cast<const uint4*>(slot + kHalfSlotBytes);
-  float s[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int t = 2 * i + half;
-    const uint4 kr = Ks[t * 16 + c];
-    const uint32_t w[4] = {kr.x, kr.y, kr.z, kr.w};
-    float a = 0.f;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      a = fmaf(qf[2 * e], bf16_lo(w[e]), a);
-      a = fmaf(qf[2 * e + 1], bf16_hi(w[e]), a);
-    }
-    s[i] = a;
-  }
-  // sum over the 16 lanes of the half; afterwards the lane holds the logit of token 2*(c>>1)+half
-#pragma unroll
-  for (int n = 8, off = 8; n > 1; n >>= 1, off >>= 1) {
-    const bool upper = (c & off) != 0;
-#pragma unroll
-    for (int j = 0; j < n / 2; ++j) {
-      const float keep = upper ? s[j + n / 2] : s[j];
-      const float send = upper ? s[j] : s[j + n / 2];
-      s[j] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
-    }
-  }
-  float x = s[0] + __shfl_xor_sync(0xFFFFFFFFu, s[0], 1);
-  const int my_t = 2 * (c >> 1) + half;
-  if (my_t >= valid) x = -INFINITY;                     // padding tokens: masked (their bytes may be anything)
-  const float m_new = fmaxf(st.m, warp_max(x));
-  const float corr = exp2_or_zero(st.m, m_new);
-  const float p = exp2_or_zero(x, m_new);
-  st.l = st.l * corr + ((c & 1) == 0 ? p : 0.f);
-  st.m = m_new;
-#pragma unroll
-  for (int e = 0; e < 8; ++e) st.acc[e] *= corr;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int t = 2 * i + half;
-    const float pi = __shfl_sync(0xFFFFFFFFu, p, half * 16 + 2 * i);
-    uint4 vr = Vs[t * 16 + c];
-    if (t >= valid) vr = make_uint4(0, 0, 0, 0);        // 0 * garbage must stay 0
-    const uint32_t w[4] = {vr.x, vr.y, vr.z, vr.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      st.acc[2 * e] = fmaf(pi, bf16_lo(w[e]), st.acc[2 * e]);
-      st.acc[2 * e + 1] = fmaf(pi, bf16_hi(w[e]), st.acc[2 * e + 1]);
-    }
-  }
+// p -> (bf16 high part, bf16 low part) of two values, packed for the MMA's B operand
+__device__ __forceinline__ void split_pack(float p0, float p1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(p0), h1 = __float2bfloat16_rn(p1);
+  const __nv_bfloat16 l0 = __float2bfloat16_rn(p0 - __bfloat162float(h0)), l1 = __float2bfloat16_rn(p1 - __bfloat162float(h1));
+  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+// byte offset of 16-byte chunk `chunk` (0..15, 8 coordinates each) of token row `t` inside a K or V tile
+// (two 2 KiB boxes of 64 coordinates, each with the 128-byte swizzle)
+__device__ __forceinline__ uint32_t tile_offset(int t, int chunk) {
+  return (uint32_t)((chunk >> 3) * kBoxBytes + t * 128 + (((chunk & 7) ^ (t & 7)) << 4));
 }
 
 template <int S, bool kPaged>
 __global__ void __launch_bounds__(kAttnWarps * 32)
-attn_kernel(Geometry geo, AttnArgs a, uint32_t* __restrict__ status) {
+attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Geometry geo,
+            AttnArgs a, uint32_t* __restrict__ status) {
   constexpr int SB = S / kUnitTokens;                   // 16-token units per page
-  extern __shared__ __align__(128) unsigned char ring[];
+  extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
-  __shared__ float s_m[kAttnWarps], s_l[kAttnWarps];
-  __shared__ float s_acc[kAttnWarps][kHeadDim];
+  __shared__ __align__(8) uint64_t bar_merge;
+  __shared__ int s_count;
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int split = blockIdx.x % a.n_splits, bh = blockIdx.x / a.n_splits;
-  const int b = bh / geo.Hq, h = bh % geo.Hq, kvh = h / geo.g;
-  const int c = lane & 15;
-  const long long blk = (long long)S * kHeadDim;        // elements per K (or V) block of a page
+  const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
+
+  // ---- which (request, heads, page range) --------------------------------------------------------
+  const int split = blockIdx.x % a.n_splits, grp = blockIdx.x / a.n_splits;
+  int b, kvh = 0, bh0, G;
+  if (kPaged) {
+    const int tiles = (geo.g + 7) / 8;
+    const int tile = grp % tiles, bk = grp / tiles;
+    b = bk / geo.Hkv;
+    kvh = bk % geo.Hkv;
+    bh0 = b * geo.Hq + kvh * geo.g + tile * 8;
+    G = min(8, geo.g - tile * 8);
+  } else {
+    bh0 = grp;
+    b = grp / geo.Hq;
+    G = 1;
+  }
+
+  unsigned char* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);   // TMA swizzle wants 1 KiB alignment
+  uint32_t* list_page = reinterpret_cast<uint32_t*>(ring + kRingBytes);
+  uint8_t* list_mask = reinterpret_cast<uint8_t*>(list_page + kListCap);
 
   if (lane == 0) {
 #pragma unroll
     for (int sidx = 0; sidx < kStages; ++sidx) mbar_init(&bars[warp][sidx], 1);
+    if (warp == 0) mbar_init(&bar_merge, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
   SWARM_STAMP(status, 0);
+  SWARM_KERNEL_BEGIN(status, 2);
   pdl_wait();                                           // the selection comes from the previous kernel
   SWARM_STAMP(status, 1);
 
-  int n_pages, P = 0, tail = S, total_tok = 0;
+  int P = 0, tail = S, total_tok = 0, n_items;          // items: bitmap words (paged) or page slots (gathered)
   long long pool_row0 = 0;
   if (kPaged) {
-    n_pages = a.n_sel[bh];
     const int len = a.ctx_len[b];
     P = pages_of(len, S);
     tail = len - S * (P - 1);
     pool_row0 = a.page_base[b];
+    n_items = (P + 31) / 32;
   } else {
-    total_tok = a.n_tok[bh];
-    n_pages = (total_tok + S - 1) / S;
+    total_tok = a.n_tok[bh0];
+    n_items = (total_tok + S - 1) / S;
   }
-  const int j_begin = (int)((long long)n_pages * split / a.n_splits);
-  const int j_end = (int)((long long)n_pages * (split + 1) / a.n_splits);
+  const int it_begin = (int)((long long)n_items * split / a.n_splits);
+  const int it_end = (int)((long long)n_items * (split + 1) / a.n_splits);
 
-  float qf[8];
+  // ---- Q as the A operand of S^T = Q K^T: row = head (quad), 8 k-steps of 16 coordinates -----------
+  uint32_t qa[8][2];
   {
-    const uint4 qq = *reinterpret_cast<const uint4*>(a.q + (long long)bh * kHeadDim + c * 8);
-    const uint32_t w[4] = {qq.x, qq.y, qq.z, qq.w};
-    const float scale = kLog2e * rsqrtf((float)kHeadDim);
+    const bool row_ok = quad < G;
+    const uint16_t* qrow = a.q + (long long)(bh0 + (row_ok ? quad : 0)) * kHeadDim;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      qf[2 * e] = bf16_lo(w[e]) * scale;
-      qf[2 * e + 1] = bf16_hi(w[e]) * scale;
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + tq * 2) : 0u;
+      qa[ks][1] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + tq * 2) : 0u;
     }
   }
+  const float scale = kLog2e * rsqrtf((float)kHeadDim);
 
-  WarpState st;
-  st.m = -INFINITY;
-  st.l = 0.f;
+  float m_run = -INFINITY, l_run = 0.f;                 // of head `quad`, over this lane's token columns
+  float acc[8][4];                                      // O^T: rows = coordinates 16*mt + quad (+8), cols = heads 2*tq (+1)
 #pragma unroll
-  for (int e = 0; e < 8; ++e) st.acc[e] = 0.f;
+  for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
 
   unsigned char* my_ring = ring + (size_t)warp * kStages * kSlotBytes;
-  unsigned err = 0u;
+  unsigned fills = 0, drains = 0;                       // units issued / consumed so far (slot = count % kStages)
+  bool timed_out = false;
   SWARM_STAMP(status, 2);
 
-  // This warp's pages are j_begin + warp + kAttnWarps*i, i = 0 .. n_mine-1, handled 32 at a time
-  // (lane i holds the i-th page id); each page is SB units of 16 tokens.
-  const int n_mine = (j_end - j_begin - warp + kAttnWarps - 1) / kAttnWarps;
-  unsigned fills = 0;                                   // units issued so far (slot = fills % kStages)
-  unsigned drains = 0;                                  // units consumed so far
-  for (int i0 = 0; i0 < n_mine && err == 0u; i0 += 32) {
-    const int n_here = min(32, n_mine - i0);
-    int my_p = -1;
-    if (kPaged && lane < n_here) my_p = a.sel[(long long)bh * geo.k + j_begin + warp + kAttnWarps * (i0 + lane)];
-    const int units = n_here * SB;
-
-    auto unit_valid = [&](int u, int p) -> int {        // valid tokens of unit u (page i0 + u/SB, sub-block u%SB)
-      const int sb = u % SB;
-      int valid;
-      if (kPaged) valid = (p == P - 1) ? tail : S;
-      else valid = min(S, total_tok - (j_begin + warp + kAttnWarps * (i0 + u / SB)) * S);
-      return max(0, min(kUnitTokens, valid - sb * kUnitTokens));
-    };
-    auto issue = [&](int u) {                           // all lanes call; lane 0 issues the copies
-      const int p = __shfl_sync(0xFFFFFFFFu, my_p, u / SB);
-      const int sb = u % SB;
-      const uint16_t *Kp, *Vp;
-      if (kPaged) {
-        const int pc = (p < 0 || p >= P) ? 0 : p;       // a corrupt id is flagged when consumed; copy something legal
-        Kp = a.kv_pool + (((pool_row0 + pc) * geo.Hkv + kvh) * 2) * blk;
-        Vp = Kp + blk;
-      } else {
-        const long long j = j_begin + warp + kAttnWarps * (i0 + u / SB);
-        Kp = a.k_g + ((long long)bh * geo.k + j) * blk;
-        Vp = a.v_g + ((long long)bh * geo.k + j) * blk;
+  // One round handles up to 32 bitmap words (1024 pages) in paged mode, or all page slots in gathered mode.
+  for (int round0 = it_begin; round0 < it_end; round0 += kPaged ? 32 : (it_end - it_begin)) {
+    int n_list;
+    if (kPaged) {
+      // warp 0: union of the heads' bitmaps -> (page, head mask) list in ascending page order
+      __syncthreads();                                  // the previous round's list is no longer read
+      if (warp == 0) {
+        const int w = round0 + lane;
+        uint32_t hw[8], uni = 0u;
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          hw[hh] = 0u;
+          if (hh < G && w < it_end)
+            hw[hh] = reinterpret_cast<const uint32_t*>(a.selmap + (long long)(bh0 + hh) * a.selmap_pitch)[w];
+          uni |= hw[hh];
+        }
+        if (w * 32 + 32 > P) uni &= (w * 32 >= P) ? 0u : (0xFFFFFFFFu >> (32 - (P - w * 32)));
+        const int cnt = __popc(uni);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        int pos = incl - cnt;
+        while (uni) {
+          const int bit = __ffs(uni) - 1;
+          uni &= uni - 1;
+          uint32_t hm = 0u;
+#pragma unroll
+          for (int hh = 0; hh < 8; ++hh) hm |= ((hw[hh] >> bit) & 1u) << hh;
+          list_page[pos] = (uint32_t)(w * 32 + bit);
+          list_mask[pos] = (uint8_t)hm;
+          ++pos;
+        }
+        if (lane == 31) s_count = incl;
       }
+      __syncthreads();
+      n_list = s_count;
+    } else {
+      n_list = it_end - it_begin;
+    }
+    SWARM_STAMP(status, 3);
+
+    // this warp's entries: warp, warp + 4, ...; each is SB units of 16 tokens
+    const int n_mine = (n_list - warp + kAttnWarps - 1) / kAttnWarps;
+    const int units = (n_mine > 0 && !timed_out) ? n_mine * SB : 0;   // after a timeout only the barriers are kept
+
+    auto entry_page = [&](int i) -> int {               // page id (paged) or page slot (gathered) of entry i
+      return kPaged ? (int)list_page[warp + kAttnWarps * i] : round0 + warp + kAttnWarps * i;
+    };
+    auto issue = [&](int u) {
       if (lane == 0) {
+        const int pg = entry_page(u / SB), sb = u % SB;
+        long long rowK, rowV;
+        if (kPaged) {
+          rowK = ((pool_row0 + pg) * geo.Hkv + kvh) * 2 * S + sb * kUnitTokens;
+          rowV = rowK + S;
+        } else {
+          rowK = rowV = ((long long)bh0 * geo.k + pg) * S + sb * kUnitTokens;
+        }
         const unsigned slot = fills % kStages;
-        unsigned char* dst = my_ring + slot * kSlotBytes;
-        mbar_expect_tx(&bars[warp][slot], kSlotBytes);
-        bulk_copy_g2s(dst, Kp + sb * kUnitTokens * kHeadDim, kHalfSlotBytes, &bars[warp][slot]);
-        bulk_copy_g2s(dst + kHalfSlotBytes, Vp + sb * kUnitTokens * kHeadDim, kHalfSlotBytes, &bars[warp][slot]);
+        const uint32_t dst = smem_addr(my_ring + slot * kSlotBytes);
+        uint64_t* bar = &bars[warp][slot];
+        mbar_expect_tx(bar, kSlotBytes);
+        tma_load_2d(dst, &mapK, 0, (int)rowK, bar);
+        tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar);
+        tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar);
+        tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar);
       }
       ++fills;
     };
 
     int issued = 0;
     for (; issued < min(units, kStages); ++issued) issue(issued);
-    SWARM_STAMP(status, 3);
     for (int u = 0; u < units; ++u) {
       const unsigned slot = drains % kStages, parity = (drains / kStages) & 1u;
       unsigned polls = 0;
       while (!mbar_try_wait(&bars[warp][slot], parity) && ++polls < kWaitLimit) {}
-      if (__any_sync(0xFFFFFFFFu, polls >= kWaitLimit)) { err = SWARM_DEV_TIMEOUT; break; }
+      if (__any_sync(0xFFFFFFFFu, polls >= kWaitLimit)) { timed_out = true; break; }
       ++drains;
-      const int p = __shfl_sync(0xFFFFFFFFu, my_p, u / SB);
-      if (kPaged && (p < 0 || p >= P)) {
-        if (lane == 0) atomicOr(status, SWARM_DEV_BAD_PAGE);   // corrupt selection: skip the page, keep going
-      } else {
-        const int v16 = unit_valid(u, p);
-        if (v16 > 0) attend_16(my_ring + slot * kSlotBytes, v16, qf, lane, st);
+
+      const int ei = u / SB, sb = u % SB;
+      const int pg = entry_page(ei);
+      const unsigned hm = kPaged ? list_mask[warp + kAttnWarps * ei] : 1u;
+      int valid;
+      if (kPaged) valid = (pg == P - 1) ? tail : S;
+      else valid = min(S, total_tok - pg * S);
+      const int v16 = min(kUnitTokens, valid - sb * kUnitTokens);
+      const uint32_t kt = smem_addr(my_ring + slot * kSlotBytes), vt = kt + 2 * kBoxBytes;
+
+      if (v16 > 0) {
+        if (v16 < kUnitTokens) {
+          // padding tokens: their V rows may hold anything, and 0 * NaN must not reach the accumulators
+          unsigned char* vrows = my_ring + slot * kSlotBytes + 2 * kBoxBytes;
+          for (int i = lane; i < (kUnitTokens - v16) * 16; i += 32) {
+            const int t = v16 + (i >> 4), ch = i & 15;
+            *reinterpret_cast<uint4*>(vrows + tile_offset(t, ch)) = make_uint4(0, 0, 0, 0);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordered before the slot's next TMA fill
+          __syncwarp();
+        }
+        // S^T[head][token] = Q K^T : 2 token tiles x 8 k-steps
+        float sacc[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) sacc[nt][e] = 0.f;
+#pragma unroll
+        for (int s4 = 0; s4 < 4; ++s4) {
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            uint32_t r[4];
+            ldmatrix_x4(r, kt + tile_offset(8 * nt + (lane & 7), 4 * s4 + (lane >> 3)));
+            mma_bf16(sacc[nt], qa[2 * s4][0], 0u, qa[2 * s4][1], 0u, r[0], r[1]);
+            mma_bf16(sacc[nt], qa[2 * s4 + 1][0], 0u, qa[2 * s4 + 1][1], 0u, r[2], r[3]);
+          }
+        }
+        // softmax of head `quad` over this lane's tokens 2*tq, 2*tq+1, 8+2*tq, 8+2*tq+1
+        const bool head_on = quad < G && ((hm >> quad) & 1u);
+        float x[4] = {sacc[0][0] * scale, sacc[0][1] * scale, sacc[1][0] * scale, sacc[1][1] * scale};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int t = (e >> 1) * 8 + 2 * tq + (e & 1);
+          if (!head_on || t >= v16) x[e] = -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        const float corr = m_new == -INFINITY ? 1.f : exp2_or_zero(m_run, m_new);
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = exp2_or_zero(x[e], m_new);
+        l_run = l_run * corr + (p[0] + p[1]) + (p[2] + p[3]);
+        m_run = m_new;
+        uint32_t b0h, b0l, b1h, b1l;
+        split_pack(p[0], p[1], b0h, b0l);
+        split_pack(p[2], p[3], b1h, b1l);
+        // rescale the outputs of heads 2*tq and 2*tq+1 (their factors live in quads 2*tq and 2*tq+1)
+        const float c0 = __shfl_sync(0xFFFFFFFFu, corr, 8 * tq), c1 = __shfl_sync(0xFFFFFFFFu, corr, 8 * tq + 4);
+        if (__any_sync(0xFFFFFFFFu, corr != 1.f)) {
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) {
+            acc[mt][0] *= c0; acc[mt][1] *= c1; acc[mt][2] *= c0; acc[mt][3] *= c1;
+          }
+        }
+        // O^T[coordinate][head] += V^T P^T : 8 tiles of 16 coordinates, P as high + low bf16 parts
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          uint32_t r[4];
+          ldmatrix_x4_trans(r, vt + tile_offset(((lane >> 4) & 1) * 8 + (lane & 7), 2 * mt + ((lane >> 3) & 1)));
+          mma_bf16(acc[mt], r[0], r[1], r[2], r[3], b0h, b1h);
+          mma_bf16(acc[mt], r[0], r[1], r[2], r[3], b0l, b1l);
+        }
       }
       __syncwarp();                                     // every lane is done reading the slot
       if (issued < units) { issue(issued); ++issued; }
     }
   }
-  if (err) {
-    // a wait expired: give the copies still in flight a bounded chance to land before the CTA's shared
-    // memory is released, then report
+  if (timed_out) {
+    // give the copies still in flight a bounded chance to land before the shared memory is released
     for (; drains < fills; ++drains) {
       const unsigned slot = drains % kStages, parity = (drains / kStages) & 1u;
       unsigned polls = 0;
       while (!mbar_try_wait(&bars[warp][slot], parity) && ++polls < kWaitLimit) {}
     }
-    if (lane == 0) atomicOr(status, err);
+    if (lane == 0) atomicOr(status, SWARM_DEV_TIMEOUT);
   }
-
   SWARM_STAMP(status, 4);
-  // merge the two halves of the warp, then the warps of the CTA
-  const float l_warp = warp_sum(st.l);
-#pragma unroll
-  for (int e = 0; e < 8; ++e) st.acc[e] += __shfl_xor_sync(0xFFFFFFFFu, st.acc[e], 16);
-  if (lane < 16) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) s_acc[warp][c * 8 + e] = st.acc[e];
-  }
-  if (lane == 0) { s_m[warp] = st.m; s_l[warp] = l_warp; }
+  SWARM_STAMP_ANY_CTA(status, 7);
+
+  // ---- merge the warps of the CTA (the ring is idle now and is reused as scratch) ------------------
   __syncthreads();
-  const int t = threadIdx.x;                          // one output coordinate per thread
-  float M = s_m[0];
+  float* s_acc = reinterpret_cast<float*>(ring);        // [warp][head 8][128]
+  float* s_m = s_acc + kAttnWarps * 8 * kHeadDim;       // [warp][8]
+  float* s_l = s_m + kAttnWarps * 8;                    // [warp][8]
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+  if (tq == 0) { s_m[warp * 8 + quad] = m_run; s_l[warp * 8 + quad] = l_run; }
 #pragma unroll
-  for (int w = 1; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w]);
-  float L = 0.f, o = 0.f;
+  for (int mt = 0; mt < 8; ++mt) {
+    float* base = s_acc + (warp * 8 + 2 * tq) * kHeadDim + 16 * mt + quad;
+    base[0] = acc[mt][0];
+    base[kHeadDim] = acc[mt][1];
+    base[8] = acc[mt][2];
+    base[kHeadDim + 8] = acc[mt][3];
+  }
+  __syncthreads();
+  const int t = threadIdx.x;                            // one output coordinate per thread
+  float M[8], L[8], o[8];
 #pragma unroll
-  for (int w = 0; w < kAttnWarps; ++w) {
-    const float sc = exp2_or_zero(s_m[w], M);
-    L += s_l[w] * sc;
-    o += s_acc[w][t] * sc;
+  for (int hh = 0; hh < 8; ++hh) {
+    M[hh] = -INFINITY; L[hh] = 0.f; o[hh] = 0.f;
+    if (hh < G) {
+#pragma unroll
+      for (int w = 0; w < kAttnWarps; ++w) M[hh] = fmaxf(M[hh], s_m[w * 8 + hh]);
+#pragma unroll
+      for (int w = 0; w < kAttnWarps; ++w) {
+        const float sc = exp2_or_zero(s_m[w * 8 + hh], M[hh]);
+        L[hh] += s_l[w * 8 + hh] * sc;
+        o[hh] += s_acc[(w * 8 + hh) * kHeadDim + t] * sc;
+      }
+    }
   }
   if (a.n_splits > 1) {
-    // publish this split's partial, then let the last split of the head merge all of them
-    const long long slot = (long long)bh * a.n_splits + split;
-    __stcg(&a.part_acc[slot * kHeadDim + t], o);
-    if (t == 0) { __stcg(&a.part_ml[slot * 2], M); __stcg(&a.part_ml[slot * 2 + 1], L); }
-    __threadfence();
-    __syncthreads();
-    if (t == 0) s_last = (atomicAdd(&a.tickets[bh], 1u) == (unsigned)a.n_splits - 1u);
+    // publish this split's partials, then let the last split of the group merge all of them
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) {
+      if (hh < G) {
+        const long long slot = (long long)(bh0 + hh) * a.n_splits + split;
+        __stcg(&a.part_acc[slot * kHeadDim + t], o[hh]);
+        if (t == 0) { __stcg(&a.part_ml[slot * 2], M[hh]); __stcg(&a.part_ml[slot * 2 + 1], L[hh]); }
+      }
+    }
+    __syncthreads();                                    // all of the CTA's partial stores are issued ...
+    if (t == 0) {                                       // ... and published by one release-acquire ticket
+      unsigned prev;
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.tickets + grp) : "memory");
+      s_last = (prev == (unsigned)a.n_splits - 1u);
+    }
     __syncthreads();
     SWARM_STAMP(status, 5);
-    if (!s_last) return;
-    __threadfence();
-    const float* ml = a.part_ml + (long long)bh * a.n_splits * 2;
-    M = -INFINITY;
-    for (int sp = 0; sp < a.n_splits; ++sp) M = fmaxf(M, __ldcg(&ml[2 * sp]));
-    L = 0.f;
-    o = 0.f;
-    for (int sp = 0; sp < a.n_splits; ++sp) {
-      const float sc = exp2_or_zero(__ldcg(&ml[2 * sp]), M);
-      L += __ldcg(&ml[2 * sp + 1]) * sc;
-      o += __ldcg(&a.part_acc[((long long)bh * a.n_splits + sp) * kHeadDim + t]) * sc;
+    SWARM_STAMP_ANY_CTA(status, 8);
+    if (!s_last) { SWARM_KERNEL_END(status, 2); return; }
+    // Fetch the group's partial outputs ([head][split][128] floats, contiguous) with one bulk copy per
+    // batch of heads into the idle ring while the (max, sum) pairs are loaded directly; then reduce from
+    // shared memory.  One memory round trip instead of a chain of dependent loads.
+    float* s_part = reinterpret_cast<float*>(ring);
+    float* s_pm = reinterpret_cast<float*>(list_page);  // [head][kMaxSplits]  (the page list is no longer needed)
+    float* s_pl = s_pm + 8 * kMaxSplits;
+    const int row_bytes = a.n_splits * kHeadDim * 4;
+    const int heads_per_batch = max(1, kRingBytes / row_bytes);
+    unsigned phase = 0;
+    for (int hb = 0; hb < G; hb += heads_per_batch) {
+      const int nb = min(heads_per_batch, G - hb);
+      __syncthreads();                                  // everyone is done with the ring and the scratch
+      if (t == 0) {
+        asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy traffic (shared scratch, the partials) first
+        mbar_expect_tx(&bar_merge, (unsigned)(nb * row_bytes));
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_addr(s_part)),
+                     "l"(a.part_acc + (long long)(bh0 + hb) * a.n_splits * kHeadDim), "r"((unsigned)(nb * row_bytes)),
+                     "r"(smem_addr(&bar_merge))
+                     : "memory");
+      }
+      for (int idx = t; idx < nb * a.n_splits; idx += kAttnWarps * 32) {
+        const int hh = idx / a.n_splits, sp = idx - hh * a.n_splits;
+        const float2 ml =
+            __ldcg(reinterpret_cast<const float2*>(a.part_ml + ((long long)(bh0 + hb + hh) * a.n_splits + sp) * 2));
+        s_pm[hh * kMaxSplits + sp] = ml.x;
+        s_pl[hh * kMaxSplits + sp] = ml.y;
+      }
+      __syncthreads();
+      unsigned polls = 0;
+      while (!mbar_try_wait(&bar_merge, phase) && ++polls < kWaitLimit) {}
+      if (polls >= kWaitLimit) { if (t == 0) atomicOr(status, SWARM_DEV_TIMEOUT); }
+      phase ^= 1u;
+      SWARM_STAMP_ANY_CTA(status, 9);
+      // warp w reduces heads w, w + 4, ...: lanes first turn the (max, sum) pairs into weights, then each
+      // lane sums 4 coordinates over the splits
+      float* s_w = s_pl + 8 * kMaxSplits;               // [kMaxSplits] per warp
+      for (int hh = warp; hh < nb; hh += kAttnWarps) {
+        const float m0 = lane < a.n_splits ? s_pm[hh * kMaxSplits + lane] : -INFINITY;
+        const float m1 = lane + 32 < a.n_splits ? s_pm[hh * kMaxSplits + lane + 32] : -INFINITY;
+        float Mx = fmaxf(m0, m1);
+#pragma unroll
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o2));
+        const float w0 = exp2_or_zero(m0, Mx), w1 = exp2_or_zero(m1, Mx);
+        float Ls = (lane < a.n_splits ? s_pl[hh * kMaxSplits + lane] * w0 : 0.f) +
+                   (lane + 32 < a.n_splits ? s_pl[hh * kMaxSplits + lane + 32] * w1 : 0.f);
+#pragma unroll
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) Ls += __shfl_xor_sync(0xFFFFFFFFu, Ls, o2);
+        s_w[warp * kMaxSplits + lane] = w0;
+        s_w[warp * kMaxSplits + lane + 32] = w1;
+        __syncwarp();
+        const float4* rows = reinterpret_cast<const float4*>(s_part + (long long)hh * a.n_splits * kHeadDim) + lane;
+        float4 os = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int sp = 0; sp < a.n_splits; ++sp) {
+          const float sc = s_w[warp * kMaxSplits + sp];
+          const float4 v = rows[sp * (kHeadDim / 4)];
+          os.x = fmaf(v.x, sc, os.x); os.y = fmaf(v.y, sc, os.y); os.z = fmaf(v.z, sc, os.z); os.w = fmaf(v.w, sc, os.w);
+        }
+        const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
+        reinterpret_cast<float4*>(a.out + (long long)(bh0 + hb + hh) * kHeadDim)[lane] =
+            make_float4(os.x * inv, os.y * inv, os.z * inv, os.w * inv);
+        if (lane == 0) a.lse[bh0 + hb + hh] = Ls > 0.f ? (Mx + log2f(Ls)) * kLn2 : -INFINITY;
+        __syncwarp();
+      }
     }
-    if (t == 0) a.tickets[bh] = 0u;                     // ready for the next launch
+    if (t == 0) a.tickets[grp] = 0u;                    // ready for the next launch
+  } else {
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) {
+      if (hh < G) {
+        a.out[(long long)(bh0 + hh) * kHeadDim + t] = L[hh] > 0.f ? o[hh] / L[hh] : 0.f;
+        if (t == 0) a.lse[bh0 + hh] = L[hh] > 0.f ? (M[hh] + log2f(L[hh])) * kLn2 : -INFINITY;
+      }
+    }
   }
-  a.out[(long long)bh * kHeadDim + t] = L > 0.f ? o / L : 0.f;
-  if (t == 0) a.lse[bh] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
   SWARM_STAMP_ANY_CTA(status, 6);
+  SWARM_KERNEL_END(status, 2);
+}
+
+// Per-head page bitmap from an explicit selection list (for callers that bring their own `sel`).
+__global__ void __launch_bounds__(256)
+selmap_from_sel_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __restrict__ n_sel,
+                       uint8_t* __restrict__ selmap, int pitch) {
+  const int bh = blockIdx.x;
+  uint32_t* row = reinterpret_cast<uint32_t*>(selmap + (long long)bh * pitch);
+  for (int i = threadIdx.x; i < pitch / 4; i += blockDim.x) row[i] = 0u;
+  __syncthreads();
+  const int n = min(n_sel[bh], geo.k);
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    const int p = sel[(long long)bh * geo.k + j];
+    if (p >= 0 && p < geo.Pmax) atomicOr(&row[p >> 5], 1u << (p & 31));
+  }
+}
+
+// ---- host side: tensor maps -----------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor of `rows` token rows x 128 coordinates at `base`; boxes of 16 rows x 64 coordinates, 128-byte swizzle
+cudaError_t make_row_map(CUtensorMap* map, const void* base, long long rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kUnitTokens};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 template <int S, bool kPaged>
-cudaError_t launch_variant(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st, bool overlap) {
-  const unsigned grid = (unsigned)geo.B * geo.Hq * a.n_splits;
-  return launch_pdl(attn_kernel<S, kPaged>, dim3(grid), dim3(kAttnWarps * 32), kAttnSmemBytes, st, overlap, geo, a,
-                    status);
+cudaError_t launch_variant(const CUtensorMap& mk, const CUtensorMap& mv, const Geometry& geo, const AttnArgs& a,
+                           uint32_t* status, unsigned grid, cudaStream_t st, bool overlap) {
+  return launch_pdl(attn_kernel<S, kPaged>, dim3(grid), dim3(kAttnWarps * 32), kAttnSmemBytes, st, overlap, mk, mv, geo,
+                    a, status);
 }
 
 }  // namespace
@@ -340,14 +559,39 @@ cudaError_t configure_attention() {
   return e;
 }
 
+int attention_groups(const Geometry& geo, bool paged) {
+  return paged ? geo.B * geo.Hkv * ((geo.g + 7) / 8) : geo.B * geo.Hq;
+}
+
+cudaError_t launch_selmap_from_sel(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, uint8_t* selmap,
+                                   cudaStream_t st) {
+  selmap_from_sel_kernel<<<geo.B * geo.Hq, 256, 0, st>>>(geo, sel, n_sel, selmap, selmap_pitch_bytes(geo.Pmax));
+  return cudaGetLastError();
+}
+
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
                              bool overlap) {
   const bool paged = a.kv_pool != nullptr;
+  CUtensorMap mk, mv;
+  cudaError_t e;
+  if (paged) {
+    const long long rows = geo.n_pool_pages * geo.Hkv * 2 * geo.S;
+    if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
+    e = make_row_map(&mk, a.kv_pool, rows);
+    mv = mk;
+  } else {
+    const long long rows = (long long)geo.B * geo.Hq * geo.k * geo.S;
+    if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
+    e = make_row_map(&mk, a.k_g, rows);
+    if (e == cudaSuccess) e = make_row_map(&mv, a.v_g, rows);
+  }
+  if (e != cudaSuccess) return e;
+  const unsigned grid = (unsigned)attention_groups(geo, paged) * a.n_splits;
   if (geo.S == 16)
-    return paged ? launch_variant<16, true>(geo, a, status, st, overlap)
-                 : launch_variant<16, false>(geo, a, status, st, overlap);
-  return paged ? launch_variant<32, true>(geo, a, status, st, overlap)
-               : launch_variant<32, false>(geo, a, status, st, overlap);
+    return paged ? launch_variant<16, true>(mk, mv, geo, a, status, grid, st, overlap)
+                 : launch_variant<16, false>(mk, mv, geo, a, status, grid, st, overlap);
+  return paged ? launch_variant<32, true>(mk, mv, geo, a, status, grid, st, overlap)
+               : launch_variant<32, false>(mk, mv, geo, a, status, grid, st, overlap);
 }
 
 }  // namespace swarm

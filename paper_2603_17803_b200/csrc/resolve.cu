@@ -1,7 +1,8 @@
 // Stage 3: cluster resolution, global merge and load-balanced bucket scheduling (Eq. 8 without the
 // already-resident term; Sec. 5.1).  One launch, off the critical path (it runs beside attention).
 //
-//   mark     (all CTAs) every selected (request, page) -> global cluster id; flag[id] = 1.
+//   mark     (all CTAs; inside swarm_step the selection kernel does it instead and this phase is skipped)
+//            every selected (request, page) -> global cluster id; flag[id] = 1.
 //            Idempotent byte stores: concurrent writers store the same value, so the dedup needs no
 //            atomics.  Four independent slots per thread keep the dependent loads overlapped.
 //   tail     (the CTA that finishes marking last, found with one ticket counter)
@@ -44,13 +45,15 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
   __shared__ bool s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();                                            // the flags / the selection come from the previous kernel
   const long long c_all = cluster_base[geo.B];
   const int C = (int)min((long long)geo.Cmax, c_all);
   unsigned err = (c_all > geo.Cmax) ? SWARM_DEV_BAD_CLUSTER : 0u;
 
   SWARM_STAMP(status, 0);
-  // ---- mark -------------------------------------------------------------------------------------
-  {
+  SWARM_KERNEL_BEGIN(status, 3);
+  // ---- mark (skipped when the selection kernel already set the flags: sel == nullptr) -------------
+  if (sel != nullptr) {
     const long long slots = (long long)geo.B * geo.Hq * geo.k;
     const long long base = (long long)blockIdx.x * (kThreads * kSlotsPerThread) + tid;
     int p[kSlotsPerThread], bh[kSlotsPerThread];
@@ -88,12 +91,16 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
   err = 0u;
 
   // ---- which CTA is last? -------------------------------------------------------------------------
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+  if (gridDim.x > 1) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+  } else {
+    __syncthreads();   // one CTA: its own marks are visible to all of its threads after the barrier
+  }
   SWARM_STAMP_ANY_CTA(status, 1);
 
   // ---- compact (flags are read past L1: other CTAs wrote them) -------------------------------------
@@ -205,9 +212,9 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
         for (int r = 0; r < cnt; ++r) {
           const unsigned mm_next = s_item_m[min(r + 1, 31)], ww_next = s_item_w[min(r + 1, 31)];
           const unsigned key = ((mm >> lane) & 1u) ? L : 0xFFFFFFFFu;
-          const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);
-          if (L == best) L += ww;                                    // lane ids make the values distinct
-          if (rank == r) my_q = best & 31u;
+          const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);   // ~60 cycles per cluster end to end;
+          if (L == best) L += ww;                                      // shuffle- and ballot-based variants
+          if (rank == r) my_q = best & 31u;                            // measured slower on sm_100
           mm = mm_next;
           ww = ww_next;
         }
@@ -216,10 +223,11 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
       }
     }
     SWARM_STAMP_ANY_CTA(status, 4);
+    SWARM_KERNEL_END(status, 3);
     if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
     if (lane == 0) {
       *n_uniq = n;
-      *ticket = 0u;                                                  // ready for the next call
+      if (gridDim.x > 1) *ticket = 0u;                               // ready for the next call
     }
   }
 }
@@ -232,13 +240,13 @@ cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                            const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                           cudaStream_t st) {
+                           cudaStream_t st, bool overlap) {
   const long long slots = (long long)geo.B * geo.Hq * geo.k;
-  const unsigned grid = (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
-  resolve_kernel<<<grid, kThreads, 0, st>>>(geo, sel, n_sel, page_base, page2cluster, cluster_base, replica_mask,
-                                            cluster_size, flags_ws, ticket, items, uniq, queue_of, n_uniq, queue_load,
-                                            status);
-  return cudaGetLastError();
+  const unsigned grid =
+      sel == nullptr ? 1u : (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
+  return launch_pdl(resolve_kernel, dim3(grid), dim3(kThreads), 0, st, overlap, geo, sel, n_sel, page_base,
+                    page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq, queue_of,
+                    n_uniq, queue_load, status);
 }
 
 }  // namespace swarm

@@ -19,12 +19,16 @@ struct WorkspaceLayout {
   int64_t flags;         // u8  [max_clusters_total]   cluster dedup flags (zero between calls)
   int64_t part_acc;      // f32 [B*Hq][max_splits][d]  split-K partial outputs
   int64_t part_ml;       // f32 [B*Hq][max_splits][2]  split-K partial (max, sum)
- int64_t items;         // uint2 [max_clusters_total]  (replica mask, weight) of the clusters in visit order
+  int64_t items;         // uint2 [max_clusters_total]  (replica mask, weight) of the clusters in visit order
+  int64_t selmap;        // u8  [B*Hq][pitch]           per-head bitmap of the selected pages
   int64_t tickets;       // u32 [B*Hq]                 arrival counters of the split merge (zero between calls)
   int64_t total;
 };
 
 constexpr int kMaxSplits = 64;
+
+// Row pitch of the per-head selection bitmap: one bit per page, rounded up to 16 bytes.
+__host__ __device__ inline int selmap_pitch_bytes(int Pmax) { return ((Pmax + 7) / 8 + 15) & ~15; }
 
 struct Geometry {   // plain copy of the shape in kernel-friendly form
   int B, Hq, Hkv, g, S, k, D, Pmax, Cmax;
@@ -33,6 +37,7 @@ struct Geometry {   // plain copy of the shape in kernel-friendly form
 };
 
 // ---- one-time per-device kernel attribute set-up (dynamic shared-memory limits) ---------------
+cudaError_t configure_score();
 cudaError_t configure_topk();
 cudaError_t configure_resolve();
 cudaError_t configure_attention();
@@ -44,13 +49,17 @@ cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st);
 // `overlap`: launch with programmatic dependent launch after the previous kernel of the stream.
+// `selmap` (optional): per (request, head) bitmap of the selected pages, rows of selmap_pitch_bytes(Pmax).
+// `flags` with the three tables (optional): also mark the selected pages' clusters (see launch_resolve).
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap);
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap = nullptr,
+                        const int64_t* page_base = nullptr, const int32_t* page2cluster = nullptr,
+                        const int64_t* cluster_base = nullptr, uint8_t* flags = nullptr);
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                            const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                           cudaStream_t st);
+                           cudaStream_t st, bool overlap);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,
                           int32_t* n_tok, uint32_t* status, cudaStream_t st);
@@ -61,8 +70,8 @@ struct AttnArgs {
   const uint16_t* v_g;
   const int32_t* n_tok;
   const uint16_t* kv_pool;
-  const int32_t* sel;
-  const int32_t* n_sel;
+  const uint8_t* selmap;   // paged mode: per (request, head) bitmap of selected pages, rows of selmap_pitch bytes
+  int selmap_pitch;
   const int64_t* page_base;
   const int32_t* ctx_len;
   float* part_acc;
@@ -74,6 +83,11 @@ struct AttnArgs {
 };
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
                              bool overlap = false);
+// (request, head group) units the attention grid is split over: one per KV head (and per 8 heads of the
+// group) in paged mode, one per query head for gathered buffers.
+int attention_groups(const Geometry& geo, bool paged);
+cudaError_t launch_selmap_from_sel(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, uint8_t* selmap,
+                                   cudaStream_t st);
 
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -112,22 +126,34 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Development-only cycle stamps (compiled in with -DSWARM_TRACE): thread 0 of CTA 0 records clock64()
+// Development-only time stamps (compiled in with -DSWARM_TRACE): thread 0 of CTA 0 records %globaltimer (ns)
 // at up to 16 numbered points of a kernel into bytes [128, 256) of the workspace's status block, where
 // a developer reads them back from the workspace tensor.  Absent from normal builds.
 #ifdef SWARM_TRACE
-#define SWARM_STAMP(status, i)                                                      \
-  do {                                                                              \
-    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
-      reinterpret_cast<unsigned long long*>(status)[16 + (i)] = clock64();          \
+__device__ __forceinline__ unsigned long long trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define SWARM_STAMP_RAW(status, i, any_cta)                                                          \
+  do {                                                                                               \
+    if (threadIdx.x == 0 && ((any_cta) || (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)))  \
+      reinterpret_cast<unsigned long long*>(status)[16 + (i)] = trace_now();                         \
   } while (0)
-#define SWARM_STAMP_ANY_CTA(status, i)                                               \
-  do {                                                                              \
-    if (threadIdx.x == 0) reinterpret_cast<unsigned long long*>(status)[16 + (i)] = clock64(); \
-  } while (0)
+#endif
+#if defined(SWARM_TRACE) && SWARM_TRACE == 1      // phases inside one kernel
+#define SWARM_STAMP(status, i) SWARM_STAMP_RAW(status, i, false)
+#define SWARM_STAMP_ANY_CTA(status, i) SWARM_STAMP_RAW(status, i, true)
 #else
 #define SWARM_STAMP(status, i) do { } while (0)
 #define SWARM_STAMP_ANY_CTA(status, i) do { } while (0)
+#endif
+#if defined(SWARM_TRACE) && SWARM_TRACE == 2      // entry of the first CTA / exit of the last CTA of kernel k
+#define SWARM_KERNEL_BEGIN(status, k) SWARM_STAMP_RAW(status, 2 * (k), false)
+#define SWARM_KERNEL_END(status, k) SWARM_STAMP_RAW(status, 2 * (k) + 1, true)
+#else
+#define SWARM_KERNEL_BEGIN(status, k) do { } while (0)
+#define SWARM_KERNEL_END(status, k) do { } while (0)
 #endif
 
 }  // namespace swarm

@@ -3,10 +3,10 @@
 //
 // Scores become order-preserving 32-bit keys (-0 folded onto +0 so the two compare equal).  A
 // most-significant-digit radix select finds the exact key T of the k-th best page and how many
-// pages tie with it.  The digits are taken relative to the list's own [min, max] key range, 11
+// pages tie with it.  The digits are taken relative to the list's own [min, max] key range, 12
 // bits at a time: page scores of one head sit in a narrow band (often a single binade), and digits
 // cut from the raw bit pattern would throw them all into a handful of histogram bins.  With range-
-// relative digits the shared-memory atomics spread over all 2048 bins and two levels usually finish.
+// relative digits the shared-memory atomics spread over all 4096 bins and two levels usually finish.
 // The result is then written in page-id order: every page with key > T, plus the first
 // (k - #greater) pages with key == T, placed by a block-wide scan of per-thread counts.  That order
 // gives "ties go to the lower page id" and the ascending-id output at once.
@@ -18,8 +18,8 @@
 namespace swarm {
 namespace {
 
-constexpr int kBins = 2048;
-constexpr int kDigitBits = 11;
+constexpr int kBins = 4096;
+constexpr int kDigitBits = 12;
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -27,11 +27,34 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Optional by-products of the selection, written while the selected pages are still in registers.
+//   selmap  one bit per page and query head (bit p%8 of byte p/8 of row [b][h], rows of `selmap_pitch`
+//           bytes): lets the attention kernel form, per KV head, the union of its query heads' pages.
+//   flags   cluster dedup flags (see resolve.cu): flag[cluster_base[b] + page2cluster[...]] = 1.
+struct TopkExtras {
+  uint8_t* selmap;
+  int selmap_pitch;
+  const int64_t* page_base;
+  const int32_t* page2cluster;
+  const int64_t* cluster_base;
+  uint8_t* flags;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ void mark_cluster(const Geometry& geo, const TopkExtras& x, int b, int p) {
+  const long long pb = x.page_base[b], cb = x.cluster_base[b];
+  const int c = x.page2cluster[pb + p];
+  if (c < 0 || c >= x.cluster_base[b + 1] - cb || cb + c >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
+  else x.flags[cb + c] = 1;
+}
+
 // Shared state of one radix-select run.
 struct SelectState {
   int hist[kBins];
   int warp_tot[32];
   uint32_t red_min[32], red_max[32];
+  uint32_t cand[1024]; // candidate keys of the chosen bin, when few enough to finish by direct ranking
+  int n_cand;          // number of keys in the chosen bin (set by narrow), then the fill counter of cand[]
   uint32_t base;       // keys below `base` are out; candidates satisfy key - base < 2^bits
   int bits;            // undecided low bits of the candidates
   int remaining;       // rank still to find among the candidates (counted from the top)
@@ -70,6 +93,7 @@ __device__ __forceinline__ void narrow(SelectState& st, int tid, int shift) {
         st.base = base + ((uint32_t)(kBins - 1 - (tid * PER + j)) << shift);
         st.bits = shift;
         st.remaining = remaining - above;
+        st.n_cand = c[j];
         above = remaining;                                   // stop
       } else {
         above += c[j];
@@ -99,16 +123,41 @@ __device__ __forceinline__ void block_minmax(SelectState& st, int tid, uint32_t 
   __syncthreads();
 }
 
+// The chosen bin holds few keys (already gathered in st.cand[0 .. n)): rank them directly.  The key whose
+// rank interval contains `remaining` is the k-th best key; ties share the interval, so every thread that
+// finds it writes the same values.
+template <int THREADS>
+__device__ __forceinline__ void finish_by_ranking(SelectState& st, int tid, int n) {
+  const int remaining = st.remaining;
+  __syncthreads();
+  for (int i = tid; i < n; i += THREADS) {
+    const uint32_t mine = st.cand[i];
+    int gt = 0, eq = 0;
+    for (int j = 0; j < n; ++j) {
+      const uint32_t other = st.cand[j];
+      gt += other > mine;
+      eq += other == mine;
+    }
+    if (gt < remaining && remaining <= gt + eq) {
+      st.base = mine;
+      st.bits = 0;
+      st.remaining = remaining - gt;
+    }
+  }
+  __syncthreads();
+}
+
 // ---- register-resident variant -------------------------------------------------------------------
 template <int THREADS, int ITEMS>
 __global__ void __launch_bounds__(THREADS)
 topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
-                 int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status) {
+                 int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
   __shared__ SelectState st;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.x, b = bh / geo.Hq;
   pdl_launch_dependents();
   SWARM_STAMP(status, 0);
+  SWARM_KERNEL_BEGIN(status, 1);
   for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
   pdl_wait();                                               // the scores come from the previous kernel
   SWARM_STAMP(status, 1);
@@ -156,6 +205,19 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
       SWARM_STAMP(status, 4 + 2 * level);
       narrow<THREADS>(st, tid, shift);
       SWARM_STAMP(status, 5 + 2 * level);
+      const int n_cand = st.n_cand;
+      if (st.bits > 0 && n_cand <= 1024) {
+        // few keys left: gather them and rank directly instead of running more digit levels
+        const uint32_t cbase = st.base;
+        const uint32_t cwidth_m1 = (1u << st.bits) - 1u;
+        __syncthreads();                                    // everyone has read n_cand before it becomes the fill counter
+        if (tid == 0) st.n_cand = 0;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j)
+          if (p0 + j < P && key[j] - cbase <= cwidth_m1) st.cand[atomicAdd(&st.n_cand, 1)] = key[j];
+        finish_by_ranking<THREADS>(st, tid, n_cand);
+      }
     }
     T = st.base;
     need_eq = st.remaining;
@@ -179,18 +241,33 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   int before = incl - cnt;
   for (int w2 = 0; w2 < warp; ++w2) before += st.warp_tot[w2];
   int gt_before = before & 0xFFFF, eq_before = before >> 16;
+  unsigned picked = 0u;                                     // bit j: page p0 + j is selected
 #pragma unroll
   for (int j = 0; j < ITEMS; ++j) {
     if (p0 + j < P) {
       const bool gt = key[j] > T, eq = key[j] == T;
-      if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = p0 + j;
+      if (gt || (eq && eq_before < need_eq)) {
+        out[gt_before + min(eq_before, need_eq)] = p0 + j;
+        picked |= 1u << j;
+      }
       gt_before += gt;
       eq_before += eq;
     }
   }
+  if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
+    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch + p0 / 8;
+    if (ITEMS == 8) *row = (uint8_t)picked;
+    else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
+  }
+  if (x.flags != nullptr) {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j)
+      if ((picked >> j) & 1u) mark_cluster(geo, x, b, p0 + j);
+  }
   for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
   SWARM_STAMP(status, 13);
+  SWARM_KERNEL_END(status, 1);
 }
 
 // ---- generic variant: any list length, keys in shared memory when they fit, else re-read ----------
@@ -199,7 +276,7 @@ constexpr int kGenericThreads = 1024;
 template <bool kKeysInSmem>
 __global__ void __launch_bounds__(kGenericThreads)
 topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
-                    int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status) {
+                    int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
   extern __shared__ uint32_t skeys[];
   __shared__ SelectState st;
   __shared__ int warp_gt[32], warp_eq[32];
@@ -266,9 +343,21 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
     const unsigned bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
     const int my_gt = gt_before + __popc(bg & lt_mask);
     const int my_eq = eq_before + __popc(be & lt_mask);
-    if (gt || (eq && my_eq < need_eq)) out[my_gt + min(my_eq, need_eq)] = i;
+    const bool take = gt || (eq && my_eq < need_eq);
+    if (take) {
+      out[my_gt + min(my_eq, need_eq)] = i;
+      if (x.flags != nullptr) mark_cluster(geo, x, b, i);
+    }
+    const unsigned word = __ballot_sync(0xFFFFFFFFu, take);
+    if (x.selmap != nullptr && lane == 0 && i0 / 8 + 4 <= x.selmap_pitch)
+      *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + i0 / 8) = word;
     gt_before += __popc(bg);
     eq_before += __popc(be);
+  }
+  if (x.selmap != nullptr) {                                // words past the last page of the request
+    const int first = ((P + 31) / 32) * 4;
+    for (int o = first + tid * 4; o + 4 <= x.selmap_pitch; o += kGenericThreads * 4)
+      *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + o) = 0u;
   }
   for (int j = k_eff + tid; j < geo.k; j += kGenericThreads) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
@@ -284,11 +373,21 @@ cudaError_t configure_topk() {
 }
 
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap) {
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap,
+                        const int64_t* page_base, const int32_t* page2cluster, const int64_t* cluster_base,
+                        uint8_t* flags) {
+  TopkExtras x;
+  x.selmap = selmap;
+  x.selmap_pitch = selmap_pitch_bytes(geo.Pmax);
+  x.page_base = page_base;
+  x.page2cluster = page2cluster;
+  x.cluster_base = cluster_base;
+  x.flags = flags;
+  x.status = status;
   const dim3 grid(geo.B * geo.Hq);
 #define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                    \
   return launch_pdl(topk_regs_kernel<THREADS, ITEMS>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
-                    ctx_len, sel, n_sel, status)
+                    ctx_len, sel, n_sel, status, x)
   if (geo.Pmax <= 1024) SWARM_TOPK_REGS(128, 8);
   if (geo.Pmax <= 2048) SWARM_TOPK_REGS(256, 8);
   if (geo.Pmax <= 4096) SWARM_TOPK_REGS(512, 8);
@@ -298,9 +397,9 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   const size_t key_bytes = (size_t)geo.Pmax * sizeof(uint32_t);
   if (key_bytes <= kSmemKeyBytes)
     return launch_pdl(topk_generic_kernel<true>, grid, dim3(kGenericThreads), key_bytes, st, overlap, geo, scores,
-                      ctx_len, sel, n_sel, status);
+                      ctx_len, sel, n_sel, status, x);
   return launch_pdl(topk_generic_kernel<false>, grid, dim3(kGenericThreads), 0, st, overlap, geo, scores, ctx_len,
-                    sel, n_sel, status);
+                    sel, n_sel, status, x);
 }
 
 }  // namespace swarm
