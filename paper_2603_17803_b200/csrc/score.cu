@@ -7,7 +7,7 @@
 // A warp reads a row with one 16-byte load per lane (lanes 0-15 hold minima, 16-31 maxima), so the
 // sign-split form needs one multiply-add per element and query head, with the weights (min(q,0) on
 // the low lanes, max(q,0) on the high lanes) held in registers for all G heads of the KV group.
-// The multiply-adds are issued two at a time (fma.rn.f32x2 on even/odd coordinates).
+// (Packed fma.rn.f32x2 was measured slower than scalar FMAs on sm_100 for the same work and is not used.)
 //
 // R rows are handled together; their R*G partial sums are summed across the 32 lanes with a
 // transposing butterfly: at each level a lane keeps half of its sums and hands the other half to
@@ -19,6 +19,8 @@
 // Every warp requests all of its NB*R rows (8 KiB) before it starts the arithmetic, and 12 warps fit
 // on an SM, so about 96 KiB per SM are in flight.  HBM-bound: 512 B per row against about 40 warp
 // instructions.
+#include <cuda.h>
+
 #include <algorithm>
 
 #include "swarm_internal.cuh"
@@ -28,22 +30,6 @@ namespace {
 
 constexpr int kScoreWarps = 4;
 int g_sm_count = 148;                                      // set by configure_score()
-
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ float sum2(uint64_t v) {
-  float lo, hi;
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-  return lo + hi;
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
 
 __host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
 
@@ -62,6 +48,24 @@ __device__ __forceinline__ float butterfly(float (&v)[NV]) {
 #pragma unroll
   for (int o = 16 >> ilog2(NV); o >= 1; o >>= 1) r += __shfl_xor_sync(0xFFFFFFFFu, r, o);
   return r;
+}
+
+// Weights of this lane's 8 coordinates for the G heads starting at bh0 (= request * Hq + head): min(q,0) on
+// the lanes that hold minima, max(q,0) on the lanes that hold maxima; w[c] belongs to head (c XOR head_sel).
+template <int G>
+__device__ __forceinline__ void load_weights(float (&w)[G][8], const uint16_t* __restrict__ q, long long bh0,
+                                             int head_sel, int lane) {
+#pragma unroll
+  for (int cc = 0; cc < G; ++cc) {
+    const uint4 qq = *reinterpret_cast<const uint4*>(q + (bh0 + (cc ^ head_sel)) * kHeadDim + (lane & 15) * 8);
+    const uint32_t words[4] = {qq.x, qq.y, qq.z, qq.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float lo = bf16_lo(words[e]), hi = bf16_hi(words[e]);
+      w[cc][2 * e] = lane < 16 ? fminf(lo, 0.f) : fmaxf(lo, 0.f);
+      w[cc][2 * e + 1] = lane < 16 ? fminf(hi, 0.f) : fmaxf(hi, 0.f);
+    }
+  }
 }
 
 template <int G, int R, int NB>
@@ -107,20 +111,10 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     }
 
   SWARM_STAMP(status, 1);
-  // Weights of this lane's 8 coordinates, as 4 (even, odd) pairs; w[c] belongs to head (c XOR head_sel).
+  // Weights of this lane's 8 coordinates; w[c] belongs to head (c XOR head_sel).
   const int h0 = kvh * geo.g + tile * G;
-  uint64_t w[G][4];
-#pragma unroll
-  for (int c = 0; c < G; ++c) {
-    const int h = h0 + (c ^ head_sel);
-    const uint4 qq = *reinterpret_cast<const uint4*>(q + ((long long)(b * geo.Hq + h) * kHeadDim + (lane & 15) * 8));
-    const uint32_t words[4] = {qq.x, qq.y, qq.z, qq.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float lo = bf16_lo(words[e]), hi = bf16_hi(words[e]);
-      w[c][e] = lane < 16 ? pack2(fminf(lo, 0.f), fminf(hi, 0.f)) : pack2(fmaxf(lo, 0.f), fmaxf(hi, 0.f));
-    }
-  }
+  float w[G][8];
+  load_weights<G>(w, q, (long long)b * geo.Hq + h0, head_sel, lane);
 
   SWARM_STAMP(status, 2);
 #pragma unroll
@@ -131,15 +125,15 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
     for (int a = 0; a < R; ++a) {
       const uint32_t words[4] = {data[nb][a].x, data[nb][a].y, data[nb][a].z, data[nb][a].w};
-      uint64_t x[4];
+      float x[8];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) x[e] = pack2(bf16_lo(words[e]), bf16_hi(words[e]));
+      for (int e = 0; e < 4; ++e) { x[2 * e] = bf16_lo(words[e]); x[2 * e + 1] = bf16_hi(words[e]); }
 #pragma unroll
       for (int c = 0; c < G; ++c) {
-        uint64_t acc = 0ull;
+        float acc = 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc = ffma2(w[c][e], x[e], acc);
-        v[a * G + c] = sum2(acc);
+        for (int e = 0; e < 8; ++e) acc = fmaf(w[c][e], x[e], acc);
+        v[a * G + c] = acc;
       }
     }
     const float total = butterfly<NV>(v);
@@ -151,25 +145,25 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
   SWARM_KERNEL_END(status, 0);
 }
 
-#if defined(SWARM_TRACE) && SWARM_TRACE == 3     // phases of the streaming scorer only
-#define SCORE_STAMP(status, i) SWARM_STAMP_RAW(status, i, false)
-#define SCORE_STAMP_ANY(status, i) SWARM_STAMP_RAW(status, i, true)
-#else
-#define SCORE_STAMP(status, i) do { } while (0)
-#define SCORE_STAMP_ANY(status, i) do { } while (0)
-#endif
-
-// ---- streaming variant -----------------------------------------------------------------------------
-// One persistent CTA per SM.  The summaries of `ppc` consecutive pages of a request (all KV heads) are one
-// contiguous block of memory, so a producer warp brings them in with one bulk asynchronous copy per block
-// (64 KiB) into a 3-slot shared-memory ring while 16 consumer warps score the block that has landed:
-// the bytes in flight (up to 192 KiB per SM) no longer depend on how many registers the arithmetic needs.
-// The CTAs split the blocks of all requests evenly; each (KV head, 8-row batch) of a block is one warp's item.
-constexpr int kStreamConsumers = 16;
-constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
-constexpr int kStreamStages = 3;
-constexpr int kStreamBlockBytes = 64 * 1024;
-constexpr int kStreamMaxBatch = 1024;                     // requests whose block counts fit the shared prefix table
+// ---- streaming tensor-core variant ---------------------------------------------------------------------
+// score[page][head] is a dense contraction: [pages x 256] (minima | maxima) times [256 x heads]
+// (min(q,0) | max(q,0)), all operands exactly representable in bf16.  On the fp32 pipes it costs ~100 warp
+// instructions per 512-byte row, which was measured to hold a 148-SM streaming kernel at about half of
+// the memory bandwidth; as m16n8k16 MMAs (16 pages x up to 8 heads per tile, fp32 accumulation) it costs
+// ~3, and the kernel runs at the speed of the bulk copies.
+//
+// One persistent CTA per SM.  A block is 16 consecutive pages of one request for a group of up to 8 KV
+// heads: per KV head four TMA boxes of 16 pages x 64 coordinates (128-byte swizzle) = 8 KiB, so a block of
+// 8 KV heads is 64 KiB.  A producer warp keeps a 3-slot ring full; consumer warp j scores KV head j of the
+// block that has landed with ldmatrix + mma and stores the tile of scores.  Waits are bounded.
+constexpr int kMmaConsumers = 8;                           // = KV heads per block
+constexpr int kMmaThreads = (kMmaConsumers + 1) * 32;
+constexpr int kMmaStages = 3;
+constexpr int kMmaPages = 16;                              // pages per block = M of the MMA tile
+constexpr int kMmaHeadBytes = 4 * kMmaPages * 128;         // 4 boxes of 16 pages x 128 B
+constexpr int kMmaStageBytes = kMmaConsumers * kMmaHeadBytes;
+constexpr int kMmaSmemBytes = 1024 + kMmaStages * kMmaStageBytes;
+constexpr int kStreamMaxBatch = 1024;                      // requests whose block counts fit the shared prefix table
 constexpr unsigned kStreamWaitLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t sm_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -185,33 +179,30 @@ __device__ __forceinline__ bool sm_try_wait(uint64_t* bar, unsigned parity) {
   return ok != 0;
 }
 
-template <int G, int R>
-__global__ void __launch_bounds__(kStreamThreads, 1)
-page_score_stream_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ ksum,
-                         const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
-                         float* __restrict__ scores, uint32_t* __restrict__ status, int ppc) {
-  constexpr int NV = G * R;
-  constexpr int LOG_NV = ilog2(NV), LOG_G = ilog2(G);
-  extern __shared__ __align__(128) unsigned char stream_ring[];
-  __shared__ __align__(8) uint64_t full[kStreamStages], empty[kStreamStages];
+__global__ void __launch_bounds__(kMmaThreads, 1)
+page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
+                      const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
+                      float* __restrict__ scores, uint32_t* __restrict__ status) {
+  extern __shared__ unsigned char mma_smem_raw[];
+  __shared__ __align__(8) uint64_t full[kMmaStages], empty[kMmaStages];
   __shared__ int s_cum[kStreamMaxBatch + 1];               // blocks before request b
   __shared__ int s_abort;
   pdl_launch_dependents();
   SWARM_KERNEL_BEGIN(status, 0);
-  SCORE_STAMP(status, 0);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  unsigned char* ring = mma_smem_raw + ((1024u - (sm_addr(mma_smem_raw) & 1023u)) & 1023u);
 
+  const int kv_groups = (geo.Hkv + kMmaConsumers - 1) / kMmaConsumers;   // blocks per page tile
   if (tid == 0) {
-    for (int sidx = 0; sidx < kStreamStages; ++sidx) {
+    for (int sidx = 0; sidx < kMmaStages; ++sidx) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&full[sidx])), "r"(1));
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&empty[sidx])), "r"(kStreamConsumers));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&empty[sidx])), "r"(kMmaConsumers));
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_abort = 0;
     s_cum[0] = 0;
   }
-  // blocks per request (serial prefix by one warp: B is small next to the streaming work)
-  if (warp == 0) {
+  if (warp == 1) {                                         // blocks per request, prefix by one warp
     int running = 0;
     for (int b0 = 0; b0 < geo.B; b0 += 32) {
       const int b = b0 + lane;
@@ -220,7 +211,7 @@ page_score_stream_kernel(Geometry geo, const uint16_t* __restrict__ q, const uin
         const int len = ctx_len[b];
         const int P = pages_of(len, geo.S);
         if (len < 1 || P > page_base[b + 1] - page_base[b] || P > geo.Pmax) atomicOr(status, SWARM_DEV_BAD_LENGTH);
-        else nb = (P + ppc - 1) / ppc;
+        else nb = ((P + kMmaPages - 1) / kMmaPages) * kv_groups;
       }
       int incl = nb;
 #pragma unroll
@@ -233,132 +224,147 @@ page_score_stream_kernel(Geometry geo, const uint16_t* __restrict__ q, const uin
     }
   }
   __syncthreads();
-  SCORE_STAMP(status, 1);
   const int total = s_cum[geo.B];
   const int blk_lo = (int)((long long)total * blockIdx.x / gridDim.x);
   const int blk_hi = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
-  const int row_bytes = geo.Hkv * 512;                     // summaries of one page, all KV heads
+  const int n_blk = blk_hi - blk_lo;
 
-  // request of a block index, found by walking forward (blocks are visited in order)
-  int cur_b = 0;
-  auto locate = [&](int blk) {
-    while (s_cum[cur_b + 1] <= blk) ++cur_b;
-    return blk - s_cum[cur_b];                            // block index inside request cur_b
-  };
-
-  if (warp == kStreamConsumers) {
+  if (warp == kMmaConsumers) {
     // ---- producer ----
     if (lane == 0) {
-      for (int blk = blk_lo; blk < blk_hi; ++blk) {
-        const int k = blk - blk_lo, stage = k % kStreamStages;
-        if (k >= kStreamStages) {
-          const unsigned parity = ((k / kStreamStages) - 1) & 1u;
+      int fb = 0;
+      for (int k = 0; k < n_blk; ++k) {
+        const int stage = k % kMmaStages;
+        if (k >= kMmaStages) {
+          const unsigned parity = ((k / kMmaStages) - 1) & 1u;
           unsigned polls = 0;
           while (!sm_try_wait(&empty[stage], parity) && ++polls < kStreamWaitLimit && !s_abort) {}
           if (polls >= kStreamWaitLimit || s_abort) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; break; }
         }
-        const int c = locate(blk);
-        const int b = cur_b;
-        const int P = pages_of(ctx_len[b], geo.S);
-        const int pages = min(ppc, P - c * ppc);
-        const unsigned bytes = (unsigned)(pages * row_bytes);
-        const uint16_t* src = ksum + (page_base[b] + (long long)c * ppc) * geo.Hkv * 2 * kHeadDim;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])), "r"(bytes)
+        const int blk = blk_lo + k;
+        while (s_cum[fb + 1] <= blk) ++fb;
+        const int c = blk - s_cum[fb];
+        const int tile = c / kv_groups, kvg = c % kv_groups;
+        const int n_kv = min(kMmaConsumers, geo.Hkv - kvg * kMmaConsumers);
+        const int page0 = (int)(page_base[fb] + (long long)tile * kMmaPages);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])),
+                     "r"((unsigned)(n_kv * kMmaHeadBytes))
                      : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                         sm_addr(stream_ring + (size_t)stage * kStreamBlockBytes)),
-                     "l"(src), "r"(bytes), "r"(sm_addr(&full[stage]))
-                     : "memory");
+        for (int j = 0; j < n_kv; ++j) {
+#pragma unroll
+          for (int bx = 0; bx < 4; ++bx) {
+            const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + j * kMmaHeadBytes + bx * (kMmaPages * 128));
+            asm volatile(
+                "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + j), "r"(page0), "r"(sm_addr(&full[stage]))
+                : "memory");
+          }
+        }
       }
     }
     return;
   }
 
-  // ---- consumers ----
-  const int pi = lane >> (5 - LOG_NV);                      // slot permutation, as in page_score_kernel
-  const int row_sel = pi >> LOG_G, head_sel = pi & (G - 1);
-  const int tiles = geo.g / G;
-  const int batches = (ppc + R - 1) / R;
-  const int items_full = geo.Hkv * tiles * batches;
-  uint64_t w[G][4];
-  int w_key = -1;                                           // (request, kv head, tile) the weights belong to
-
-  auto load_weights = [&](int b, int kvh, int tile) {
-    const int key = (b * geo.Hkv + kvh) * tiles + tile;
-    if (key == w_key) return;
-    w_key = key;
-    const int h0 = kvh * geo.g + tile * G;
-#pragma unroll
-    for (int cc = 0; cc < G; ++cc) {
-      const int h = h0 + (cc ^ head_sel);
-      const uint4 qq = *reinterpret_cast<const uint4*>(q + ((long long)(b * geo.Hq + h) * kHeadDim + (lane & 15) * 8));
-      const uint32_t words[4] = {qq.x, qq.y, qq.z, qq.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float lo = bf16_lo(words[e]), hi = bf16_hi(words[e]);
-        w[cc][e] = lane < 16 ? pack2(fminf(lo, 0.f), fminf(hi, 0.f)) : pack2(fmaxf(lo, 0.f), fmaxf(hi, 0.f));
-      }
-    }
-  };
-  if (blk_lo < blk_hi) {                                    // the first item's weights, fetched while the first block is in flight
-    locate(blk_lo);
-    const int kt = warp / batches;
-    if (warp < items_full) load_weights(cur_b, kt / tiles, kt % tiles);
-  }
-
-  for (int blk = blk_lo; blk < blk_hi; ++blk) {
-    const int k = blk - blk_lo, stage = k % kStreamStages;
-    const int c = locate(blk);
+  // ---- consumers: warp j <-> KV head j of the block ----
+  const int quad = lane >> 2, tq = lane & 3;
+  const int tiles = (geo.g + 7) / 8;                        // head tiles of 8 per KV head (N of the MMA)
+  uint32_t wb[16][2];                                       // B operand: weights of head `quad`, 16 k-steps
+  long long w_key = -1;
+  int cur_b = 0;
+  for (int k = 0; k < n_blk; ++k) {
+    const int blk = blk_lo + k, stage = k % kMmaStages;
+    while (s_cum[cur_b + 1] <= blk) ++cur_b;
     const int b = cur_b;
+    const int c = blk - s_cum[b];
+    const int tile_p = c / kv_groups, kvg = c % kv_groups;
+    const int kvh = kvg * kMmaConsumers + warp;
+    const bool active = kvh < geo.Hkv;
     const int P = pages_of(ctx_len[b], geo.S);
-    const int pages = min(ppc, P - c * ppc);
+    const int p0 = tile_p * kMmaPages;
     {
-      const unsigned parity = (k / kStreamStages) & 1u;
+      const unsigned parity = (k / kMmaStages) & 1u;
       unsigned polls = 0;
-      while (!sm_try_wait(&full[stage], parity) && ++polls < kStreamWaitLimit && !s_abort) {}
+      while (!sm_try_wait(&full[stage], parity) && ++polls < kStreamWaitLimit) __nanosleep(32);
       if (__any_sync(0xFFFFFFFFu, polls >= kStreamWaitLimit || s_abort != 0)) {
         if (lane == 0) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; }
         break;
       }
     }
-    SCORE_STAMP(status, 2 + 2 * k);
-    const unsigned char* blkmem = stream_ring + (size_t)stage * kStreamBlockBytes;
-    for (int item = warp; item < items_full; item += kStreamConsumers) {
-      const int rb = item % batches, kt = item / batches;
-      const int tile = kt % tiles, kvh = kt / tiles;
-      if (rb * R >= pages) continue;
-      const int h0 = kvh * geo.g + tile * G;
-      load_weights(b, kvh, tile);
-      float v[NV];
+    if (active) {
+      const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + warp * kMmaHeadBytes);
+      for (int ht = 0; ht < tiles; ++ht) {
+        const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
+        const long long key = ((long long)b * geo.Hq + h0);
+        if (key != w_key) {
+          // weights of head h0 + quad: min(q,0) against the minima (k < 128), max(q,0) against the maxima
+          w_key = key;
+          const uint16_t* qrow = q + (key + (quad < nh ? quad : 0)) * kHeadDim;
 #pragma unroll
-      for (int a = 0; a < R; ++a) {
-        const int pl = rb * R + (a ^ row_sel);              // page inside the block
-        uint4 d = make_uint4(0, 0, 0, 0);
-        if (pl < pages) d = *reinterpret_cast<const uint4*>(blkmem + ((size_t)pl * geo.Hkv + kvh) * 512 + lane * 16);
-        const uint32_t words[4] = {d.x, d.y, d.z, d.w};
-        uint64_t x[4];
+          for (int ks = 0; ks < 16; ++ks) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) x[e] = pack2(bf16_lo(words[e]), bf16_hi(words[e]));
+            for (int half = 0; half < 2; ++half) {
+              const int col = ks * 16 + half * 8 + tq * 2;                // 0..255
+              uint32_t pr = *reinterpret_cast<const uint32_t*>(qrow + (col & 127));
+              // clamp each bf16 by its sign bit: keep negatives for the minima part, positives for the maxima part
+              const bool want_neg = col < 128;
+              uint32_t lo = pr & 0xFFFFu, hi = pr >> 16;
+              if (((lo >> 15) != 0u) != want_neg) lo = 0u;
+              if (((hi >> 15) != 0u) != want_neg) hi = 0u;
+              wb[ks][half] = quad < nh ? (lo | (hi << 16)) : 0u;
+            }
+          }
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int cc = 0; cc < G; ++cc) {
-          uint64_t acc = 0ull;
+        for (int ks = 0; ks < 16; ++ks) {
+          // A tile: 16 pages x 16 coordinates; matrices (rows 0-7 | 8-15) x (chunk 2ks | 2ks+1)
+          const int m = lane >> 3, r = (m & 1) * 8 + (lane & 7), cc = 2 * ks + (m >> 1);
+          uint32_t a[4];
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                       : "r"(base + (uint32_t)((cc >> 3) * (kMmaPages * 128) + r * 128 + (((cc & 7) ^ (r & 7)) << 4))));
+          asm volatile(
+              "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+              : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+              : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(wb[ks][0]), "r"(wb[ks][1]));
+        }
+        // C: (page p0 + quad, heads 2tq, 2tq+1), (page p0 + quad + 8, same heads)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc = ffma2(w[cc][e], x[e], acc);
-          v[a * G + cc] = sum2(acc);
+        for (int e = 0; e < 4; ++e) {
+          const int hh = 2 * tq + (e & 1), p = p0 + quad + (e >> 1) * 8;
+          if (hh < nh && p < P) scores[((long long)b * geo.Hq + h0 + hh) * geo.Pmax + p] = acc[e];
         }
       }
-      const float total_v = butterfly<NV>(v);
-      const int r = pi >> LOG_G, hh = pi & (G - 1);
-      const int p = c * ppc + rb * R + r;
-      if ((lane & ((1 << (5 - LOG_NV)) - 1)) == 0 && rb * R + r < pages)
-        scores[((long long)(b * geo.Hq + h0 + hh)) * geo.Pmax + p] = total_v;
     }
     __syncwarp();
-    SCORE_STAMP(status, 3 + 2 * k);
     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sm_addr(&empty[stage])) : "memory");
   }
-  SCORE_STAMP_ANY(status, 15);
   SWARM_KERNEL_END(status, 0);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// summaries as a 3-D bf16 tensor [page][kv head][256]; boxes of 16 pages x 1 KV head x 64 coordinates
+cudaError_t make_summary_map(CUtensorMap* map, const void* ksum, int Hkv, long long n_pool_pages) {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess)
+      return cudaErrorNotSupported;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  const cuuint64_t dims[3] = {256, (cuuint64_t)Hkv, (cuuint64_t)n_pool_pages};
+  const cuuint64_t strides[2] = {512, (cuuint64_t)Hkv * 512};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)kMmaPages};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ksum), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 template <int G, int R, int NB>
@@ -370,14 +376,15 @@ cudaError_t launch_one(const Geometry& geo, const uint16_t* q, const uint16_t* k
   return cudaGetLastError();
 }
 
-template <int G, int R>
-cudaError_t launch_stream(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
-                          const int32_t* ctx_len, float* scores, uint32_t* status, cudaStream_t st) {
-  const int ppc = kStreamBlockBytes / (geo.Hkv * 512);
-  const long long max_blocks = (long long)geo.B * ((geo.Pmax + ppc - 1) / ppc);
+cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
+                       const int32_t* ctx_len, float* scores, uint32_t* status, cudaStream_t st) {
+  CUtensorMap map;
+  cudaError_t e = make_summary_map(&map, ksum, geo.Hkv, geo.n_pool_pages);
+  if (e != cudaSuccess) return e;
+  const int kv_groups = (geo.Hkv + kMmaConsumers - 1) / kMmaConsumers;
+  const long long max_blocks = (long long)geo.B * ((geo.Pmax + kMmaPages - 1) / kMmaPages) * kv_groups;
   const int grid = (int)std::min<long long>(g_sm_count, std::max<long long>(1, max_blocks));
-  page_score_stream_kernel<G, R><<<grid, kStreamThreads, kStreamStages * kStreamBlockBytes, st>>>(
-      geo, q, ksum, page_base, ctx_len, scores, status, ppc);
+  page_score_mma_kernel<<<grid, kMmaThreads, kMmaSmemBytes, st>>>(map, geo, q, page_base, ctx_len, scores, status);
   return cudaGetLastError();
 }
 
@@ -389,25 +396,16 @@ cudaError_t configure_score() {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   g_sm_count = sms > 0 ? sms : 148;
-  const int bytes = kStreamStages * kStreamBlockBytes;
-  e = cudaFuncSetAttribute(page_score_stream_kernel<8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(page_score_stream_kernel<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(page_score_stream_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(page_score_stream_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  return e;
+  return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaSmemBytes);
 }
 
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st) {
-  // Streaming variant whenever one page's summaries (all KV heads) fit the block size a few times over and
-  // the batch fits its prefix table; otherwise the register-resident grid kernel.
-  if (geo.Hkv * 512 * 2 <= kStreamBlockBytes && geo.B <= kStreamMaxBatch) {
-    if (geo.g % 8 == 0) return launch_stream<8, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);
-    if (geo.g % 4 == 0) return launch_stream<4, 8>(geo, q, ksum, page_base, ctx_len, scores, status, st);
-    if (geo.g % 2 == 0) return launch_stream<2, 8>(geo, q, ksum, page_base, ctx_len, scores, status, st);
-    return launch_stream<1, 8>(geo, q, ksum, page_base, ctx_len, scores, status, st);
-  }
+  // Streaming tensor-core variant whenever the batch fits its prefix table and the pool fits 32-bit TMA
+  // coordinates; otherwise the register-resident grid kernel on the fp32 pipes.
+  if (geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31))
+    return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, st);
   // Heads of a KV group are processed G at a time, G the largest of 8/4/2/1 dividing the group size.
   if (geo.g % 8 == 0) return launch_one<8, 4, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);
   if (geo.g % 4 == 0) return launch_one<4, 8, 2>(geo, q, ksum, page_base, ctx_len, scores, status, st);
