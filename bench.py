@@ -243,7 +243,7 @@ def run_swarm(args):
 
         n_loop = max(3 * args.n_rot, min(K, 2000))
         t_c = time.perf_counter()
-        attn_us = time_loop(lambda s: s.sparse_attn_paged(stream=stream), n_loop)
+        attn_us = time_loop(lambda s: s.sparse_attn_paged(stream=stream, reuse_last_selection=True), n_loop)
         select_us = time_loop(lambda s: s.select(stream=stream), n_loop)
         resolve_us = time_loop(lambda s: s.resolve(stream=stream), n_loop)
         t_d = time.perf_counter()

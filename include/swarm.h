@@ -159,7 +159,9 @@ int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const 
 
 /* Stage 4 without the copy: the same attention, reading the selected pages straight from the pool
  * (what swarm_step runs).  Reads inputs->q, kv_pool, page_base, ctx_len.  Tokens beyond ctx_len in a
- * partial last page are masked.  n_sel[b][h] must be >= 1. */
+ * partial last page are masked.  n_sel[b][h] must be >= 1.
+ * sel and n_sel may both be NULL: the selection made by the last swarm_select or swarm_step on this
+ * ctx is attended (its per-head page bitmaps are kept in the workspace), without rebuilding them. */
 int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel,
                                 const int32_t* n_sel, float* out, float* lse, void* stream);
 

@@ -209,7 +209,8 @@ int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int3
   float* sc = scores ? scores : ws_ptr<float>(ctx, ctx->lay.scores);
   SWARM_TRY(launch_page_score(ctx->geo, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(in->ksum),
                               in->page_base, in->ctx_len, sc, ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, true));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, true,
+                        ws_ptr<uint8_t>(ctx, ctx->lay.selmap)));
   return SWARM_OK;
 }
 
@@ -284,9 +285,12 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const in
                                 float* out, float* lse, void* stream) {
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
-  if (!pool_inputs_ok(in) || bad(in->q) || bad(sel) || bad(n_sel) || bad(out) || bad(lse)) return SWARM_ERR_INVALID_ARG;
+  if (!pool_inputs_ok(in) || bad(in->q) || bad(out) || bad(lse) || ((sel == nullptr) != (n_sel == nullptr)) ||
+      (sel && (bad(sel) || bad(n_sel))))
+    return SWARM_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  SWARM_TRY(launch_selmap_from_sel(ctx->geo, sel, n_sel, ws_ptr<uint8_t>(ctx, ctx->lay.selmap), st));
+  if (sel != nullptr)   // otherwise: the page bitmaps of this ctx's last swarm_select / swarm_step are reused
+    SWARM_TRY(launch_selmap_from_sel(ctx->geo, sel, n_sel, ws_ptr<uint8_t>(ctx, ctx->lay.selmap), st));
   SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, out, lse), ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
   return SWARM_OK;
 }

@@ -20,6 +20,7 @@ namespace {
 
 constexpr int kBins = 4096;
 constexpr int kDigitBits = 12;
+constexpr int kRankMax = 64;                               // finish by direct ranking at or below this many candidates
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t u = __float_as_uint(s);
@@ -53,12 +54,22 @@ struct SelectState {
   int hist[kBins];
   int warp_tot[32];
   uint32_t red_min[32], red_max[32];
-  uint32_t cand[1024]; // candidate keys of the chosen bin, when few enough to finish by direct ranking
+  uint32_t cand[kRankMax]; // candidate keys of the chosen bin, when few enough to finish by direct ranking
   int n_cand;          // number of keys in the chosen bin (set by narrow), then the fill counter of cand[]
   uint32_t base;       // keys below `base` are out; candidates satisfy key - base < 2^bits
   int bits;            // undecided low bits of the candidates
   int remaining;       // rank still to find among the candidates (counted from the top)
 };
+
+// Where digit `bin` is counted.  Thread t owns the PER consecutive digits below (kBins - 1 - t*PER); its
+// j-th digit lives at word j*THREADS + t, so the threads of a warp touch consecutive words when they read
+// or clear their digits (no bank conflicts).
+template <int THREADS>
+__device__ __forceinline__ int hist_slot(uint32_t bin) {
+  constexpr int PER = kBins / THREADS;
+  const uint32_t idx = (uint32_t)(kBins - 1) - bin;         // rank of the digit from the top
+  return (int)((idx % PER) * THREADS + idx / PER);
+}
 
 // After the histogram of the current level is complete: locate the bin holding rank `remaining`
 // from the top, narrow (base, bits, remaining), clear the histogram.  All threads call it.
@@ -69,7 +80,7 @@ __device__ __forceinline__ void narrow(SelectState& st, int tid, int shift) {
   int c[PER], sum = 0;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
-    c[j] = st.hist[kBins - 1 - (tid * PER + j)];
+    c[j] = st.hist[j * THREADS + tid];
     sum += c[j];
   }
   int incl = sum;
@@ -85,7 +96,7 @@ __device__ __forceinline__ void narrow(SelectState& st, int tid, int shift) {
   int above = incl - sum;
   for (int w2 = 0; w2 < warp; ++w2) above += st.warp_tot[w2];
 #pragma unroll
-  for (int j = 0; j < PER; ++j) st.hist[kBins - 1 - (tid * PER + j)] = 0;
+  for (int j = 0; j < PER; ++j) st.hist[j * THREADS + tid] = 0;
   if (above < remaining && remaining <= above + sum) {
 #pragma unroll
     for (int j = 0; j < PER; ++j) {
@@ -199,14 +210,14 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
 #pragma unroll
       for (int j = 0; j < ITEMS; ++j) {
         const uint32_t rel = key[j] - base;
-        if (p0 + j < P && rel <= width_m1) atomicAdd(&st.hist[rel >> shift], 1);
+        if (p0 + j < P && rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
       }
       __syncthreads();
       SWARM_STAMP(status, 4 + 2 * level);
       narrow<THREADS>(st, tid, shift);
       SWARM_STAMP(status, 5 + 2 * level);
       const int n_cand = st.n_cand;
-      if (st.bits > 0 && n_cand <= 1024) {
+      if (st.bits > 0 && n_cand <= kRankMax) {
         // few keys left: gather them and rank directly instead of running more digit levels
         const uint32_t cbase = st.base;
         const uint32_t cwidth_m1 = (1u << st.bits) - 1u;
@@ -310,7 +321,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
       const uint32_t width_m1 = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
       for (int i = tid; i < P; i += kGenericThreads) {
         const uint32_t rel = key_at(i) - base;
-        if (rel <= width_m1) atomicAdd(&st.hist[rel >> shift], 1);
+        if (rel <= width_m1) atomicAdd(&st.hist[hist_slot<kGenericThreads>(rel >> shift)], 1);
       }
       __syncthreads();
       narrow<kGenericThreads>(st, tid, shift);

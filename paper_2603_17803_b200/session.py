@@ -99,8 +99,9 @@ class Session:
         B.swarm_sparse_attn(self.ctx, self.w.q if not hasattr(self, "_q") else self._q, self.o.k_out, self.o.v_out,
                             self.o.n_tok, self.o.out, self.o.lse, stream)
 
-    def sparse_attn_paged(self, stream=None):
-        B.swarm_sparse_attn_paged(self.ctx, self.inputs, self.o.sel, self.o.n_sel, self.o.out, self.o.lse, stream)
+    def sparse_attn_paged(self, stream=None, reuse_last_selection=False):
+        sel, n_sel = (None, None) if reuse_last_selection else (self.o.sel, self.o.n_sel)
+        B.swarm_sparse_attn_paged(self.ctx, self.inputs, sel, n_sel, self.o.out, self.o.lse, stream)
 
     def step(self, stream=None):
         B.swarm_step(self.ctx, self.inputs, self.outputs, stream)

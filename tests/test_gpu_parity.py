@@ -303,4 +303,9 @@ def test_paged_attention_alone_matches_gathered_attention():
     torch.cuda.synchronize()
     assert (sess.o.out - out).abs().max().item() <= 1e-5 and (sess.o.lse - lse).abs().max().item() <= 1e-5
     parity.check_step(w, sess)
+    out2 = sess.o.out.clone()
+    sess.o.out.zero_()
+    sess.sparse_attn_paged(reuse_last_selection=True)     # bitmaps left in the workspace by the calls above
+    torch.cuda.synchronize()
+    assert torch.equal(sess.o.out, out2)
     sess.close()
