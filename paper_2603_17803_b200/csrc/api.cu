@@ -314,7 +314,7 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
   // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
   SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true,
                         ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
-                        ws_ptr<uint8_t>(ctx, ctx->lay.flags)));
+                        ws_ptr<uint8_t>(ctx, ctx->lay.flags), in->cluster_replica_mask, in->cluster_size));
 
   // fork: cluster resolution and attention both need only the selection.  Resolution is the longer of
   // the two (its greedy pass is serial), so it stays on the caller's stream right behind the selection

@@ -110,11 +110,18 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
   const int vec_per_warp = (n_vec + kWarps - 1) / kWarps;
   const int v_lo = min(n_vec, warp * vec_per_warp), v_hi = min(n_vec, v_lo + vec_per_warp);
   uint4* f4 = reinterpret_cast<uint4*>(flags);
+  const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
+  const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
+  const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
+  // pass 1: count (the common case of one 16-flag vector per lane keeps it in registers for pass 2)
+  const bool one_vec = v_hi - v_lo <= 32;
+  uint4 f_keep = make_uint4(0, 0, 0, 0);
   int cnt = 0;
   for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
     const int v = v0 + lane;
     if (v < v_hi) {
       const uint4 f = __ldcg(f4 + v);
+      f_keep = f;
       cnt += nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
     }
   }
@@ -127,11 +134,14 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
     if (w2 < warp) before += warp_cnt[w2];
     n += warp_cnt[w2];
   }
+  // pass 2: place the ids, clear the flags, and in the same go validate each cluster's replica mask, route
+  // the single-replica ones and stash what the serial pass needs
+  unsigned classes = 0u;
   for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
     const int v = v0 + lane;
     uint4 f = make_uint4(0, 0, 0, 0);
     if (v < v_hi) {
-      f = __ldcg(f4 + v);
+      f = one_vec ? f_keep : __ldcg(f4 + v);
       if (f.x | f.y | f.z | f.w) __stcg(f4 + v, make_uint4(0, 0, 0, 0));   // leave zeros for the next call
     }
     const int mine = nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
@@ -144,40 +154,30 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
     int pos = before + incl - mine;
     const uint32_t words[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
-    for (int j = 0; j < 16; ++j)
-      if ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) uniq[pos++] = v * 16 + j;
+    for (int j = 0; j < 16; ++j) {
+      if ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) {
+        const int c = v * 16 + j, i = pos++;
+        uniq[i] = c;
+        const unsigned m = replica_mask[c];
+        const unsigned wgt = unit ? 1u : (unsigned)cluster_size[c];
+        if (m == 0u || (m & ~valid_bits)) {
+          err |= SWARM_DEV_BAD_REPLICA;
+          queue_of[i] = 0xFF;
+          items[i] = make_uint2(0u, 0u);
+        } else if (__popc(m) == 1 && !by_id) {
+          const int qd = __ffs(m) - 1;
+          queue_of[i] = (uint8_t)qd;
+          atomicAdd(&s_load[qd], (int)wgt);
+          items[i] = make_uint2(0u, 0u);                             // nothing left to do for the serial pass
+        } else {
+          classes |= 1u << (__popc(m) - 1);
+          items[i] = make_uint2(m, wgt << 5);                        // what the serial pass needs, in visit order
+        }
+      }
+    }
     before += __shfl_sync(0xFFFFFFFFu, incl, 31);
   }
-  __syncthreads();   // uniq[] written by this CTA is visible to it after the barrier
   SWARM_STAMP_ANY_CTA(status, 2);
-
-  const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
-  const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
-  const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
-
-  // ---- validate masks, route single-replica clusters, record which replica counts occur -----------
-  unsigned classes = 0u;
-  for (int i = tid; i < n; i += kThreads) {
-    const int c = uniq[i];
-    const unsigned m = replica_mask[c];
-    const unsigned wgt = unit ? 1u : (unsigned)cluster_size[c];
-    if (m == 0u || (m & ~valid_bits)) {
-      err |= SWARM_DEV_BAD_REPLICA;
-      queue_of[i] = 0xFF;
-      items[i] = make_uint2(0u, 0u);
-      continue;
-    }
-    const int R = __popc(m);
-    if (R == 1 && !by_id) {
-      const int qd = __ffs(m) - 1;
-      queue_of[i] = (uint8_t)qd;
-      atomicAdd(&s_load[qd], (int)wgt);
-      items[i] = make_uint2(0u, 0u);                                 // nothing left to do for the serial pass
-    } else {
-      classes |= 1u << (R - 1);
-      items[i] = make_uint2(m, wgt << 5);                            // what the serial pass needs, in visit order
-    }
-  }
   if (classes) atomicOr(&s_classes, classes);
   if (err) atomicOr(status, err);
   __syncthreads();

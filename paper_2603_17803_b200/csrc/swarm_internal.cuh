@@ -54,7 +54,8 @@ cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
                         int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap = nullptr,
                         const int64_t* page_base = nullptr, const int32_t* page2cluster = nullptr,
-                        const int64_t* cluster_base = nullptr, uint8_t* flags = nullptr);
+                        const int64_t* cluster_base = nullptr, uint8_t* flags = nullptr,
+                        const uint32_t* replica_mask = nullptr, const uint16_t* cluster_size = nullptr);
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                            const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,

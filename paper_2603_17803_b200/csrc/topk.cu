@@ -40,7 +40,30 @@ struct TopkExtras {
   const int64_t* cluster_base;
   uint8_t* flags;
   uint32_t* status;
+  // tables the next kernels read through dependent loads; pulled into L2 while this kernel waits for the scores
+  const uint32_t* replica_mask;
+  const uint16_t* cluster_size;
+  long long n_pool_pages;
 };
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Spread over the whole grid: one 128-byte line per thread and step, at most ~8 MiB in total.
+__device__ __forceinline__ void prefetch_tables(const Geometry& geo, const TopkExtras& x) {
+  if (x.flags == nullptr) return;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x, nthreads = (long long)gridDim.x * blockDim.x;
+  const long long cap = 8LL << 20;
+  const long long p2c_bytes = min(x.n_pool_pages * 4, cap), mask_bytes = min((long long)geo.Cmax * 4, cap),
+                  size_bytes = min((long long)geo.Cmax * 2, cap);
+  for (long long o = tid * 128; o < p2c_bytes; o += nthreads * 128)
+    prefetch_l2(reinterpret_cast<const char*>(x.page2cluster) + o);
+  if (x.replica_mask != nullptr)
+    for (long long o = tid * 128; o < mask_bytes; o += nthreads * 128)
+      prefetch_l2(reinterpret_cast<const char*>(x.replica_mask) + o);
+  if (x.cluster_size != nullptr)
+    for (long long o = tid * 128; o < size_bytes; o += nthreads * 128)
+      prefetch_l2(reinterpret_cast<const char*>(x.cluster_size) + o);
+}
 
 __device__ __forceinline__ void mark_cluster(const Geometry& geo, const TopkExtras& x, int b, int p) {
   const long long pb = x.page_base[b], cb = x.cluster_base[b];
@@ -170,6 +193,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 1);
   for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
+  prefetch_tables(geo, x);
   pdl_wait();                                               // the scores come from the previous kernel
   SWARM_STAMP(status, 1);
   const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
@@ -295,6 +319,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   const int bh = blockIdx.x, b = bh / geo.Hq;
   pdl_launch_dependents();
   for (int i = tid; i < kBins; i += kGenericThreads) st.hist[i] = 0;
+  prefetch_tables(geo, x);
   pdl_wait();
   const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));
   const int k_eff = min(geo.k, P);
@@ -386,7 +411,7 @@ cudaError_t configure_topk() {
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
                         int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap,
                         const int64_t* page_base, const int32_t* page2cluster, const int64_t* cluster_base,
-                        uint8_t* flags) {
+                        uint8_t* flags, const uint32_t* replica_mask, const uint16_t* cluster_size) {
   TopkExtras x;
   x.selmap = selmap;
   x.selmap_pitch = selmap_pitch_bytes(geo.Pmax);
@@ -395,6 +420,9 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   x.cluster_base = cluster_base;
   x.flags = flags;
   x.status = status;
+  x.replica_mask = replica_mask;
+  x.cluster_size = cluster_size;
+  x.n_pool_pages = geo.n_pool_pages;
   const dim3 grid(geo.B * geo.Hq);
 #define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                    \
   return launch_pdl(topk_regs_kernel<THREADS, ITEMS>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
