@@ -31,9 +31,9 @@ METRIC = "decode steps/sec of fused select+resolve+gather+attn; HBM GB/s (% of p
 UNIT = "steps/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_kernel launch at this workload, from the ncu
-# capture summarised in profiles/ (None until a capture exists for the current kernel).
-ATTN_TRAFFIC_BYTES_NCU = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_kernel launch at the default workload (c2_128k),
+# from the ncu capture summarised in profiles/; reported only for that workload.
+ATTN_TRAFFIC_BYTES_NCU = 33_062_400 + 7_424   # profiles/launch_list_c2_128k.md: dram read + write of attn_kernel<16,paged>
 
 
 def parse_args():
@@ -297,9 +297,9 @@ def run_swarm(args):
         "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
         "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
         "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
-        "roofline": {"kernel": "attn_kernel<16,paged> (+ split combine)", "bound": "hbm", "achieved": attn_gbs,
+        "roofline": {"kernel": "attn_kernel<paged> (tensor-core split-K attention over the union of selected pages, merge included)", "bound": "hbm", "achieved": attn_gbs,
                      "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
-                     "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU,
+                     "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU if cfg.name == "c2_128k" else None,
                      "algorithmic_bytes_per_launch": attn_alg, "avg_launch_us": attn_us,
                      "nominal_bytes_per_launch": by["kv_nominal"], "nominal_gbs": by["kv_nominal"] / (attn_us * 1e-6) / 1e9},
         "e2e": {"value": replicas.aggregate_steps_per_s(world, K_e2e, ms_e2e), "unit": UNIT, "steps": K_e2e,
