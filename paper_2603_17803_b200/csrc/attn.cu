@@ -6,9 +6,9 @@
 // about moving each byte once and spending as few issue slots on it as possible.
 //
 //  * Heads of a GQA group share a KV head and, in practice, about half of their pages.  A CTA
-//    therefore serves one (request, KV head, page range): it forms the union of its query heads'
-//    selections from the per-head page bitmaps the selection kernel leaves behind, loads every page
-//    of the union once, and lets each head take part only in the pages it selected (the others are
+//    therefore serves one (request, KV head, split): it forms the union of its query heads'
+//    selections from the per-head page bitmaps the selection kernel leaves behind, takes an equal
+//    share of the union's pages (by rank, so the splits are balanced), loads every page of it once, and lets each head take part only in the pages it selected (the others are
 //    masked to -inf for that head).  The g <= 8 heads are the M rows of the score MMA.
 //  * Pages travel by TMA: cp.async.bulk.tensor tiles of 16 tokens x 64 coordinates with the 128-byte
 //    swizzle, completion counted on an mbarrier.  Each warp owns a ring of kStages slots (16 tokens of
@@ -33,7 +33,7 @@
 namespace swarm {
 namespace {
 
-constexpr int kAttnWarps = 4;
+constexpr int kAttnWarps = 8;
 constexpr int kStages = 3;
 constexpr int kUnitTokens = 16;
 constexpr int kBoxBytes = kUnitTokens * 128;                       // 16 token rows x 64 bf16
@@ -151,14 +151,48 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   pdl_wait();                                           // the selection comes from the previous kernel
   SWARM_STAMP(status, 1);
 
-  int P = 0, tail = S, total_tok = 0, n_items;          // items: bitmap words (paged) or page slots (gathered)
+  int P = 0, tail = S, total_tok = 0, n_items;          // items: pages of the union (paged) or page slots (gathered)
   long long pool_row0 = 0;
+  int n_words = 0;
+
+  // 4 consecutive bitmap words (128 pages) of every head of the group, and their union with pages >= P cut off
+  auto load_words = [&](int w0, uint4 (&hw)[8], uint4& uni) {
+    uni = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) {
+      hw[hh] = make_uint4(0u, 0u, 0u, 0u);
+      if (hh < G && w0 < n_words)
+        hw[hh] = *reinterpret_cast<const uint4*>(a.selmap + (long long)(bh0 + hh) * a.selmap_pitch + (long long)w0 * 4);
+      uni.x |= hw[hh].x; uni.y |= hw[hh].y; uni.z |= hw[hh].z; uni.w |= hw[hh].w;
+    }
+    uint32_t* u = &uni.x;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int first = (w0 + j) * 32;
+      if (first + 32 > P) u[j] &= first >= P ? 0u : (0xFFFFFFFFu >> (32 - (P - first)));
+    }
+  };
+
   if (kPaged) {
     const int len = a.ctx_len[b];
     P = pages_of(len, S);
     tail = len - S * (P - 1);
     pool_row0 = a.page_base[b];
-    n_items = (P + 31) / 32;
+    n_words = (P + 31) / 32;
+    // number of pages in the union of the group's selections: the splits share them evenly by rank
+    if (warp == 0) {
+      int total = 0;
+      for (int base = 0; base < n_words; base += 128) {
+        uint4 hw[8], uni;
+        load_words(base + lane * 4, hw, uni);
+        total += __popc(uni.x) + __popc(uni.y) + __popc(uni.z) + __popc(uni.w);
+      }
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+      if (lane == 0) s_count = total;
+    }
+    __syncthreads();
+    n_items = s_count;
   } else {
     total_tok = a.n_tok[bh0];
     n_items = (total_tok + S - 1) / S;
@@ -191,45 +225,51 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   bool timed_out = false;
   SWARM_STAMP(status, 2);
 
-  // One round handles up to 32 bitmap words (1024 pages) in paged mode, or all page slots in gathered mode.
-  for (int round0 = it_begin; round0 < it_end; round0 += kPaged ? 32 : (it_end - it_begin)) {
+  // One round handles up to kListCap pages of this split's share of the union (paged), or all its page slots.
+  for (int round0 = it_begin; round0 < it_end; round0 += kPaged ? kListCap : (it_end - it_begin)) {
     int n_list;
     if (kPaged) {
-      // warp 0: union of the heads' bitmaps -> (page, head mask) list in ascending page order
+      // warp 0: pages of the union with rank in [round0, round_end) -> (page, head mask) list, ascending
+      const int round_end = min(it_end, round0 + kListCap);
       __syncthreads();                                  // the previous round's list is no longer read
       if (warp == 0) {
-        const int w = round0 + lane;
-        uint32_t hw[8], uni = 0u;
+        int rank0 = 0;                                  // union pages before the current 128 words
+        for (int base = 0; base < n_words && rank0 < round_end; base += 128) {
+          uint4 hw[8], uni;
+          const int w0 = base + lane * 4;
+          load_words(w0, hw, uni);
+          const int cnt = __popc(uni.x) + __popc(uni.y) + __popc(uni.z) + __popc(uni.w);
+          int incl = cnt;
 #pragma unroll
-        for (int hh = 0; hh < 8; ++hh) {
-          hw[hh] = 0u;
-          if (hh < G && w < it_end)
-            hw[hh] = reinterpret_cast<const uint32_t*>(a.selmap + (long long)(bh0 + hh) * a.selmap_pitch)[w];
-          uni |= hw[hh];
-        }
-        if (w * 32 + 32 > P) uni &= (w * 32 >= P) ? 0u : (0xFFFFFFFFu >> (32 - (P - w * 32)));
-        const int cnt = __popc(uni);
-        int incl = cnt;
+          for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+          }
+          int rank = rank0 + incl - cnt;                // rank of this lane's first union page
+          rank0 += __shfl_sync(0xFFFFFFFFu, incl, 31);
+          if (rank + cnt > round0 && rank < round_end) {
+            const uint32_t* u = &uni.x;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += t;
-        }
-        int pos = incl - cnt;
-        while (uni) {
-          const int bit = __ffs(uni) - 1;
-          uni &= uni - 1;
-          uint32_t hm = 0u;
+            for (int j = 0; j < 4; ++j) {
+              uint32_t bits = u[j];
+              while (bits) {
+                const int bit = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (rank >= round0 && rank < round_end) {
+                  uint32_t hm = 0u;
 #pragma unroll
-          for (int hh = 0; hh < 8; ++hh) hm |= ((hw[hh] >> bit) & 1u) << hh;
-          list_page[pos] = (uint32_t)(w * 32 + bit);
-          list_mask[pos] = (uint8_t)hm;
-          ++pos;
+                  for (int hh = 0; hh < 8; ++hh) hm |= (((&hw[hh].x)[j] >> bit) & 1u) << hh;
+                  list_page[rank - round0] = (uint32_t)((w0 + j) * 32 + bit);
+                  list_mask[rank - round0] = (uint8_t)hm;
+                }
+                ++rank;
+              }
+            }
+          }
         }
-        if (lane == 31) s_count = incl;
       }
       __syncthreads();
-      n_list = s_count;
+      n_list = round_end - round0;
     } else {
       n_list = it_end - it_begin;
     }
@@ -380,12 +420,13 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     base[kHeadDim + 8] = acc[mt][3];
   }
   __syncthreads();
-  const int t = threadIdx.x;                            // one output coordinate per thread
+  const int t = threadIdx.x;                            // threads 0..127: one output coordinate each
+  const bool has_dim = t < kHeadDim;
   float M[8], L[8], o[8];
 #pragma unroll
   for (int hh = 0; hh < 8; ++hh) {
     M[hh] = -INFINITY; L[hh] = 0.f; o[hh] = 0.f;
-    if (hh < G) {
+    if (hh < G && has_dim) {
 #pragma unroll
       for (int w = 0; w < kAttnWarps; ++w) M[hh] = fmaxf(M[hh], s_m[w * 8 + hh]);
 #pragma unroll
@@ -400,7 +441,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     // publish this split's partials, then let the last split of the group merge all of them
 #pragma unroll
     for (int hh = 0; hh < 8; ++hh) {
-      if (hh < G) {
+      if (hh < G && has_dim) {
         const long long slot = (long long)(bh0 + hh) * a.n_splits + split;
         __stcg(&a.part_acc[slot * kHeadDim + t], o[hh]);
         if (t == 0) { __stcg(&a.part_ml[slot * 2], M[hh]); __stcg(&a.part_ml[slot * 2 + 1], L[hh]); }
@@ -486,7 +527,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   } else {
 #pragma unroll
     for (int hh = 0; hh < 8; ++hh) {
-      if (hh < G) {
+      if (hh < G && has_dim) {
         a.out[(long long)(bh0 + hh) * kHeadDim + t] = L[hh] > 0.f ? o[hh] / L[hh] : 0.f;
         if (t == 0) a.lse[bh0 + hh] = L[hh] > 0.f ? (M[hh] + log2f(L[hh])) * kLn2 : -INFINITY;
       }
@@ -643,7 +684,7 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   if (bh > SWARM_STATIC_MAX_HEADS) return SWARM_ERR_STATIC_SCRATCH_TOO_SMALL;
   if (bh * top_k >= (1LL << 31)) return SWARM_ERR_UNSUPPORTED;
   // same split heuristic as the ctx path (about 2 CTAs per SM, >= 4 pages per split), capped by the array
-  long long n = (148 * 2) / bh;
+  long long n = 148 / bh;
   n = n < (top_k / 4 > 1 ? top_k / 4 : 1) ? n : (top_k / 4 > 1 ? top_k / 4 : 1);
   n = n < kMaxSplits ? n : kMaxSplits;
   n = n < kStaticSlots / bh ? n : kStaticSlots / bh;
