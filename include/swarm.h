@@ -208,7 +208,10 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outpu
 /* End-to-end convenience for callers holding the per-step data in HOST memory (pinned memory
  * recommended): copies q_host (bf16 [B][Hq][d]) into the ctx's staging area, runs swarm_step with
  * `inputs` (whose q field is ignored) and `outputs`, copies out, lse, n_uniq, queue_load back into
- * the given host buffers and WAITS for completion.  Any *_host pointer may be NULL to skip it. */
+ * the given host buffers and WAITS for completion.  Any *_host pointer may be NULL to skip it.
+ * With pinned host buffers and a non-default stream the first call with a given set of pointers
+ * records these operations into a CUDA graph (owned by the ctx) and later calls replay it; the
+ * tensor shapes and the device tables must then stay where they are, their contents may change. */
 int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs,
                         const void* q_host, float* out_host, float* lse_host, int32_t* n_uniq_host,
                         int32_t* queue_load_host, void* stream);

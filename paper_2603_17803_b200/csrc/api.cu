@@ -18,6 +18,9 @@ struct swarm_ctx {
   cudaStream_t side;          // cluster resolution runs here beside attention
   cudaEvent_t ev_fork, ev_join;
   cudaError_t last_err;
+  cudaGraphExec_t host_graph;  // swarm_step_host: the recorded step, valid for the arguments in host_key
+  unsigned char host_key[256];
+  bool host_graph_ok;
 };
 
 namespace {
@@ -132,6 +135,9 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->ws_bytes = 0;
   ctx->user_splits = 0;
   ctx->last_err = cudaSuccess;
+  ctx->host_graph = nullptr;
+  ctx->host_graph_ok = true;
+  std::memset(ctx->host_key, 0, sizeof ctx->host_key);
   cudaError_t e = configure_score();
   if (e == cudaSuccess) e = configure_topk();
   if (e == cudaSuccess) e = configure_resolve();
@@ -149,6 +155,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
 
 int32_t swarm_destroy(swarm_ctx* ctx) {
   if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (ctx->host_graph != nullptr) cudaGraphExecDestroy(ctx->host_graph);
   cudaEventDestroy(ctx->ev_fork);
   cudaEventDestroy(ctx->ev_join);
   cudaStreamDestroy(ctx->side);
@@ -337,6 +344,39 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
   return SWARM_OK;
 }
 
+namespace {
+// Everything swarm_step_host enqueues for one step: copy q in, the step, copy the results out.
+int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
+                          float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,
+                          cudaStream_t st) {
+  const int64_t bh = (int64_t)ctx->geo.B * ctx->geo.Hq;
+  uint16_t* q_dev = ws_ptr<uint16_t>(ctx, ctx->lay.q_stage);
+  SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
+  swarm_inputs local = *in;
+  local.q = q_dev;
+  const int32_t rc = swarm_step(ctx, &local, o, st);
+  if (rc != SWARM_OK) return rc;
+  if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));
+  if (lse_host) SWARM_TRY(cudaMemcpyAsync(lse_host, o->lse, bh * 4, cudaMemcpyDeviceToHost, st));
+  if (n_uniq_host) SWARM_TRY(cudaMemcpyAsync(n_uniq_host, o->n_uniq, 4, cudaMemcpyDeviceToHost, st));
+  if (queue_load_host)
+    SWARM_TRY(cudaMemcpyAsync(queue_load_host, o->queue_load, ctx->geo.D * 4, cudaMemcpyDeviceToHost, st));
+  return SWARM_OK;
+}
+
+// The arguments a captured host step depends on; a replay is valid only while none of them changes.
+struct HostStepKey {
+  swarm_inputs in;
+  swarm_outputs out;
+  const void* q_host;
+  void *out_host, *lse_host, *n_uniq_host, *queue_load_host;
+  void* stream;
+  int user_splits;
+};
+}  // namespace
+
+static_assert(sizeof(HostStepKey) <= 256, "host_key too small");
+
 int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
                         float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,
                         void* stream) {
@@ -344,18 +384,51 @@ int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outp
   if (rc != SWARM_OK) return rc;
   if (in == nullptr || o == nullptr || q_host == nullptr) return SWARM_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int64_t bh = (int64_t)ctx->geo.B * ctx->geo.Hq;
-  uint16_t* q_dev = ws_ptr<uint16_t>(ctx, ctx->lay.q_stage);
-  SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
-  swarm_inputs local = *in;
-  local.q = q_dev;
-  rc = swarm_step(ctx, &local, o, stream);
+
+  // A step is seven small operations; issued one by one their launch cost exceeds their run time.  The
+  // first call with a given set of pointers records them into a CUDA graph, later calls replay it.
+  HostStepKey key;
+  std::memset(&key, 0, sizeof key);
+  key.in = *in;
+  key.in.q = nullptr;                                     // ignored by this entry point
+  key.out = *o;
+  key.q_host = q_host;
+  key.out_host = out_host; key.lse_host = lse_host; key.n_uniq_host = n_uniq_host; key.queue_load_host = queue_load_host;
+  key.stream = stream;
+  key.user_splits = ctx->user_splits;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  const bool can_capture = ctx->host_graph_ok && st != nullptr &&
+                           cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  if (can_capture) {
+    if (ctx->host_graph == nullptr || std::memcmp(&key, ctx->host_key, sizeof key) != 0) {
+      if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+        rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st);
+        const cudaError_t e = cudaStreamEndCapture(st, &graph);
+        if (rc == SWARM_OK && e == cudaSuccess && graph != nullptr &&
+            cudaGraphInstantiate(&ctx->host_graph, graph, 0) == cudaSuccess) {
+          std::memcpy(ctx->host_key, &key, sizeof key);
+        } else {
+          ctx->host_graph = nullptr;
+          ctx->host_graph_ok = false;                     // e.g. pageable host memory: use plain launches from now on
+          cudaGetLastError();
+        }
+        if (graph != nullptr) cudaGraphDestroy(graph);
+        if (rc != SWARM_OK) return rc;
+      } else {
+        ctx->host_graph_ok = false;
+        cudaGetLastError();
+      }
+    }
+    if (ctx->host_graph != nullptr) {
+      SWARM_TRY(cudaGraphLaunch(ctx->host_graph, st));
+      SWARM_TRY(cudaStreamSynchronize(st));
+      return SWARM_OK;
+    }
+  }
+  rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st);
   if (rc != SWARM_OK) return rc;
-  if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));
-  if (lse_host) SWARM_TRY(cudaMemcpyAsync(lse_host, o->lse, bh * 4, cudaMemcpyDeviceToHost, st));
-  if (n_uniq_host) SWARM_TRY(cudaMemcpyAsync(n_uniq_host, o->n_uniq, 4, cudaMemcpyDeviceToHost, st));
-  if (queue_load_host)
-    SWARM_TRY(cudaMemcpyAsync(queue_load_host, o->queue_load, ctx->geo.D * 4, cudaMemcpyDeviceToHost, st));
   SWARM_TRY(cudaStreamSynchronize(st));
   return SWARM_OK;
 }

@@ -593,6 +593,7 @@ cudaError_t launch_variant(const CUtensorMap& mk, const CUtensorMap& mv, const G
 }  // namespace
 
 cudaError_t configure_attention() {
+  if (encode_tiled_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
   cudaError_t e = cudaFuncSetAttribute(attn_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);

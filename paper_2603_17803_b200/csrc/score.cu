@@ -346,17 +346,22 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// summaries as a 3-D bf16 tensor [page][kv head][256]; boxes of 16 pages x 1 KV head x 64 coordinates
-cudaError_t make_summary_map(CUtensorMap* map, const void* ksum, int Hkv, long long n_pool_pages) {
+EncodeTiledFn summary_encode_fn() {
   static EncodeTiledFn fn = nullptr;
   if (fn == nullptr) {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
-        qr != cudaDriverEntryPointSuccess)
-      return cudaErrorNotSupported;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
   }
+  return fn;
+}
+
+// summaries as a 3-D bf16 tensor [page][kv head][256]; boxes of 16 pages x 1 KV head x 64 coordinates
+cudaError_t make_summary_map(CUtensorMap* map, const void* ksum, int Hkv, long long n_pool_pages) {
+  EncodeTiledFn fn = summary_encode_fn();
+  if (fn == nullptr) return cudaErrorNotSupported;
   const cuuint64_t dims[3] = {256, (cuuint64_t)Hkv, (cuuint64_t)n_pool_pages};
   const cuuint64_t strides[2] = {512, (cuuint64_t)Hkv * 512};
   const cuuint32_t box[3] = {64, 1, (cuuint32_t)kMmaPages};
@@ -396,6 +401,7 @@ cudaError_t configure_score() {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   g_sm_count = sms > 0 ? sms : 148;
+  if (summary_encode_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
   return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaSmemBytes);
 }
 
