@@ -41,7 +41,7 @@ def _load():
     global _lib
     if _lib is None:
         _lib = ctypes.CDLL(build())
-        for name in ("oracle_build_summaries", "oracle_scores", "oracle_topk", "oracle_resolve",
+        for name in ("oracle_build_summaries", "oracle_scores", "oracle_topk", "oracle_resolve", "oracle_resolve_cached",
                      "oracle_gather", "oracle_attention", "oracle_set_threads"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -131,6 +131,37 @@ def resolve(sel, n_sel, page_base, page2cluster, cluster_base, replica_mask, clu
     _check(rc, "resolve")
     n = int(n_uniq[0])
     return uniq[:n].copy(), queue_of[:n].copy(), load
+
+
+def resolve_cached(sel, n_sel, page_base, page2cluster, cluster_base, replica_mask, cluster_size, resident, freq, D,
+                   t_base, t_transfer, flags=0):
+    """Eq. 8 with the resident term plus cache bookkeeping.  Returns (uniq, queue_of, load, n_hit, freq_new, score);
+    ``freq`` is not modified."""
+    sel = _arr(sel, np.int32)
+    n_sel = _arr(n_sel, np.int32)
+    page_base = _arr(page_base, np.int64)
+    page2cluster = _arr(page2cluster, np.int32)
+    cluster_base = _arr(cluster_base, np.int64)
+    replica_mask = _arr(replica_mask, np.uint32)
+    cluster_size = _arr(cluster_size, np.uint16)
+    resident = _arr(resident, np.uint8)
+    freq_new = np.array(freq, dtype=np.int32, copy=True)
+    B, Hq, k = sel.shape
+    cap = max(int(cluster_base[-1]), 1)
+    uniq = np.empty(cap, dtype=np.int32)
+    queue_of = np.empty(cap, dtype=np.uint8)
+    n_uniq = np.zeros(1, dtype=np.int32)
+    n_hit = np.zeros(1, dtype=np.int32)
+    load = np.zeros(D, dtype=np.int32)
+    score = np.zeros(cap, dtype=np.float64)
+    rc = _load().oracle_resolve_cached(_p(sel), _p(n_sel), _p(page_base), _p(page2cluster), _p(cluster_base),
+                                       _p(replica_mask), _p(cluster_size), _p(resident), _p(freq_new),
+                                       ctypes.c_double(t_base), ctypes.c_double(t_transfer), ctypes.c_int32(B),
+                                       ctypes.c_int32(Hq), ctypes.c_int32(k), ctypes.c_int32(D), ctypes.c_uint32(flags),
+                                       _p(uniq), _p(queue_of), _p(n_uniq), _p(load), _p(n_hit), _p(score))
+    _check(rc, "resolve_cached")
+    n = int(n_uniq[0])
+    return uniq[:n].copy(), queue_of[:n].copy(), load, int(n_hit[0]), freq_new, score[: int(cluster_base[-1])]
 
 
 def gather(kv_pool, sel, n_sel, page_base, ctx_len, Hkv, d, S):

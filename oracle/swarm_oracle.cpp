@@ -20,6 +20,8 @@
 //                           term) and entry-bucket scheduling (Sec. 5.1): sort
 //                           by replication factor ascending, route each item
 //                           to its currently smallest bucket
+//   oracle_resolve_cached   the same with Eq. 8's resident term, the activation-frequency update of
+//                           Sec. 5.2 (cache replacement) and the cost-effectiveness score of Eq. 6
 //   oracle_gather           the transfer of the selected pages (Sec. 6
 //                           "Asynchronous I/O"), here a byte copy
 //   oracle_attention        Eq. 1 over the gathered tokens, one query row
@@ -176,20 +178,11 @@ int oracle_topk(const float* score, const int32_t* ctx_len, int32_t B, int32_t H
   return ORACLE_OK;
 }
 
-// Global merge + bucket scheduling.
-//   G = { cluster_base[b] + page2cluster[page_base[b] + p] : p selected by any head of request b }
-//   order G by (number of replicas ascending, id ascending)   [id ascending only, under ORDER_BY_ID]
-//   for c in that order: q* = the replica queue of c with the smallest (load, queue id);
-//                        queue_of[c] = q*;  load[q*] += cluster_size[c]   [+= 1 under UNIT_LOAD]
-// Output: uniq ascending by id, queue_of parallel to uniq, load[D], n_uniq.
-int oracle_resolve(const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
-                   const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                   const uint16_t* cluster_size, int32_t B, int32_t Hq, int32_t k, int32_t D, uint32_t flags,
-                   int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* load) {
-  if (!sel || !n_sel || !page_base || !page2cluster || !cluster_base || !replica_mask || !cluster_size || !uniq ||
-      !queue_of || !n_uniq || !load || B < 1 || Hq < 1 || k < 1 || D < 1 || D > 32)
-    return ORACLE_BAD_ARG;
-  std::set<int64_t> G;
+namespace {
+
+// The activated clusters: G = { cluster_base[b] + page2cluster[page_base[b] + p] : p selected by any head of b }.
+int collect_activated(const int32_t* sel, const int32_t* n_sel, const int64_t* page_base, const int32_t* page2cluster,
+                      const int64_t* cluster_base, int32_t B, int32_t Hq, int32_t k, std::set<int64_t>& G) {
   for (int32_t b = 0; b < B; ++b) {
     const int64_t n_pages = page_base[b + 1] - page_base[b];
     const int64_t n_clusters = cluster_base[b + 1] - cluster_base[b];
@@ -205,8 +198,17 @@ int oracle_resolve(const int32_t* sel, const int32_t* n_sel, const int64_t* page
       }
     }
   }
+  return ORACLE_OK;
+}
+
+// Bucket scheduling of the clusters in `fetch` (ascending id):
+//   order by (number of replicas ascending, id ascending)   [id ascending only, under ORDER_BY_ID]
+//   for c in that order: q* = the replica queue of c with the smallest (load, queue id);
+//                        queue_of[c] = q*;  load[q*] += cluster_size[c]   [+= 1 under UNIT_LOAD]
+int schedule(const std::vector<int64_t>& fetch, const uint32_t* replica_mask, const uint16_t* cluster_size, int32_t D,
+             uint32_t flags, int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* load) {
   const uint32_t valid_bits = D == 32 ? 0xFFFFFFFFu : ((1u << D) - 1u);
-  std::vector<int64_t> order(G.begin(), G.end());  // ascending id
+  std::vector<int64_t> order(fetch);
   for (int64_t c : order)
     if (replica_mask[c] == 0 || (replica_mask[c] & ~valid_bits)) return ORACLE_BAD_TABLE;
   if (!(flags & ORACLE_ORDER_BY_ID))
@@ -231,6 +233,55 @@ int oracle_resolve(const int32_t* sel, const int32_t* n_sel, const int64_t* page
   *n_uniq = static_cast<int32_t>(placed.size());
   for (int qd = 0; qd < D; ++qd) load[qd] = static_cast<int32_t>(L[static_cast<size_t>(qd)]);
   return ORACLE_OK;
+}
+
+}  // namespace
+
+// Global merge + bucket scheduling: every activated cluster is fetched (Eq. 8 without the resident term).
+// Output: uniq ascending by id, queue_of parallel to uniq, load[D], n_uniq.
+int oracle_resolve(const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
+                   const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
+                   const uint16_t* cluster_size, int32_t B, int32_t Hq, int32_t k, int32_t D, uint32_t flags,
+                   int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* load) {
+  if (!sel || !n_sel || !page_base || !page2cluster || !cluster_base || !replica_mask || !cluster_size || !uniq ||
+      !queue_of || !n_uniq || !load || B < 1 || Hq < 1 || k < 1 || D < 1 || D > 32)
+    return ORACLE_BAD_ARG;
+  std::set<int64_t> G;
+  const int rc = collect_activated(sel, n_sel, page_base, page2cluster, cluster_base, B, Hq, k, G);
+  if (rc != ORACLE_OK) return rc;
+  return schedule(std::vector<int64_t>(G.begin(), G.end()), replica_mask, cluster_size, D, flags, uniq, queue_of,
+                  n_uniq, load);
+}
+
+// Global merge with the resident term (Eq. 8) and the cache bookkeeping of Sec. 5.2 / Eq. 6:
+//   A = activated clusters;  E_IO = A \ resident  is scheduled as above;  n_hit = |A and resident|
+//   freq[c] += 1 for c in A;  freq[c] -= 1 for resident c not in A
+//   score[c] = freq[c] * (t_base + size[c] * t_transfer) / size[c]   for every cluster, after the update
+int oracle_resolve_cached(const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
+                          const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
+                          const uint16_t* cluster_size, const uint8_t* resident, int32_t* freq, double t_base,
+                          double t_transfer, int32_t B, int32_t Hq, int32_t k, int32_t D, uint32_t flags,
+                          int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* load, int32_t* n_hit,
+                          double* score) {
+  if (!sel || !n_sel || !page_base || !page2cluster || !cluster_base || !replica_mask || !cluster_size || !resident ||
+      !freq || !uniq || !queue_of || !n_uniq || !load || !n_hit || !score || B < 1 || Hq < 1 || k < 1 || D < 1 || D > 32)
+    return ORACLE_BAD_ARG;
+  std::set<int64_t> A;
+  const int rc = collect_activated(sel, n_sel, page_base, page2cluster, cluster_base, B, Hq, k, A);
+  if (rc != ORACLE_OK) return rc;
+  const int64_t n_clusters = cluster_base[B];
+  std::vector<int64_t> fetch;
+  int32_t hits = 0;
+  for (int64_t c : A) {
+    freq[c] += 1;
+    if (resident[c]) ++hits; else fetch.push_back(c);
+  }
+  for (int64_t c = 0; c < n_clusters; ++c)
+    if (resident[c] && A.find(c) == A.end()) freq[c] -= 1;
+  for (int64_t c = 0; c < n_clusters; ++c)
+    score[c] = static_cast<double>(freq[c]) * (t_base + cluster_size[c] * t_transfer) / cluster_size[c];
+  *n_hit = hits;
+  return schedule(fetch, replica_mask, cluster_size, D, flags, uniq, queue_of, n_uniq, load);
 }
 
 // Kg/Vg[b][h][j*S + t][:] = pool[page_base[b] + sel[b][h][j]][kv(h)][K/V][t][:] for the valid tokens of the

@@ -456,3 +456,52 @@ def test_step_invariants_on_a_scaled_topic_workload():
         last_sel = (r.sel[b] == P[b] - 1).any(axis=-1)
         tail = cl[b] - cfg.page_size * (P[b] - 1)
         assert np.array_equal(r.n_tok[b], full - last_sel * (cfg.page_size - tail))
+
+
+# ------------------------------------------------------------------ resident filter and cache counters
+
+def test_resolve_cached_is_set_difference_with_counter_updates_and_eq6_scores():
+    rng = np.random.default_rng(13)
+    D = 5
+    for trial in range(40):
+        sel, n_sel, page_base, p2c, cluster_base, mask, size = random_resolve_case(rng, D=D)
+        C = int(cluster_base[-1])
+        resident = (rng.random(C) < 0.3).astype(np.uint8)
+        freq = rng.integers(-3, 10, size=C).astype(np.int32)
+        t_base, t_tr = 80.0, 2.5
+        uniq, qof, load, n_hit, freq_new, score = oracle.resolve_cached(sel, n_sel, page_base, p2c, cluster_base, mask,
+                                                                          size, resident, freq, D, t_base, t_tr)
+        activated = set()
+        B, Hq, _ = sel.shape
+        for b in range(B):
+            for h in range(Hq):
+                for p in sel[b, h, : n_sel[b, h]]:
+                    activated.add(int(cluster_base[b]) + int(p2c[page_base[b] + p]))
+        res = {c for c in range(C) if resident[c]}
+        assert list(uniq) == sorted(activated - res)                       # E_IO = union minus resident (Eq. 8)
+        assert n_hit == len(activated & res)
+        want = freq.copy()
+        for c in range(C):
+            if c in activated:
+                want[c] += 1
+            elif c in res:
+                want[c] -= 1
+        assert np.array_equal(freq_new, want)
+        assert np.allclose(score, want * (t_base + size * t_tr) / size, rtol=1e-14, atol=0)
+        replay_check(uniq, qof, load, mask, size, D, 0)                    # the fetched ones are scheduled as before
+    # nothing resident: identical to the plain merge; everything resident: nothing to fetch
+    none = np.zeros(C, np.uint8)
+    a = oracle.resolve(sel, n_sel, page_base, p2c, cluster_base, mask, size, D)
+    b = oracle.resolve_cached(sel, n_sel, page_base, p2c, cluster_base, mask, size, none, freq, D, 1.0, 1.0)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b[:3])) and b[3] == 0
+    allr = np.ones(C, np.uint8)
+    c = oracle.resolve_cached(sel, n_sel, page_base, p2c, cluster_base, mask, size, allr, freq, D, 1.0, 1.0)
+    assert len(c[0]) == 0 and int(c[2].sum()) == 0 and c[3] == len(a[0])
+
+
+def test_cache_score_hand_case():
+    # Eq. 6 by hand: f = 6 activations, s = 4 entries, T_base = 100, T_transfer = 5 -> 6 * (100 + 20) / 4 = 180
+    sel = np.zeros((1, 1, 1), np.int32)
+    out = oracle.resolve_cached(sel, np.ones((1, 1), np.int32), [0, 1], [0], [0, 1], np.array([1], np.uint32),
+                                np.array([4], np.uint16), np.array([1], np.uint8), np.array([5], np.int32), 2, 100.0, 5.0)
+    assert out[3] == 1 and list(out[4]) == [6] and out[5][0] == 180.0 and len(out[0]) == 0
