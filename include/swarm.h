@@ -100,6 +100,17 @@ typedef struct swarm_outputs {
   float* lse;          /* f32 [B][Hq] natural-log sum of exp of the scaled logits                  */
 } swarm_outputs;
 
+/* Optional DRAM-tier cache state (Sec. 4.2 "hot clusters", Sec. 5.2 "cache replacement").  Device pointers,
+ * indexed by global cluster id.  See swarm_set_cache. */
+typedef struct swarm_cache {
+  const uint8_t* resident; /* [n_clusters] 1 = the cluster is held in the fast tier: activated but not fetched */
+  int32_t* freq;           /* [n_clusters] activation frequency f_i, updated in place every step               */
+  float* score;            /* [n_clusters] cost-effectiveness score of Eq. 6, rewritten every step; may be NULL */
+  int32_t* n_hit;          /* [1] activated clusters found resident this step; may be NULL                     */
+  float t_base;            /* T_base: addressing latency per fetch                                             */
+  float t_transfer;        /* T_transfer: transfer cost per entry (page)                                       */
+} swarm_cache;
+
 /* Lifetime.  swarm_create validates the shape and allocates only host memory plus one auxiliary
  * CUDA stream and two events (used to run cluster resolution beside attention inside swarm_step).
  * The CUDA device current at creation must stay current for every later call with this ctx. */
@@ -112,6 +123,13 @@ int32_t swarm_destroy(swarm_ctx* ctx);
  * swarm_workspace_bytes returns < 0 (minus an error code) for an invalid shape. */
 int64_t swarm_workspace_bytes(const swarm_shape* shape);
 int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, void* stream);
+
+/* Attaches (or, with NULL, detaches) cache state to the ctx; the struct is copied.  While attached,
+ * swarm_resolve_clusters and swarm_step compute the full Eq. 8: the clusters to fetch are the activated
+ * ones minus the resident ones (only those appear in uniq / queue_of / queue_load), and the bookkeeping of
+ * Sec. 5.2 runs in the same kernel: freq += 1 for every activated cluster, freq -= 1 for every resident
+ * cluster that was not activated, score = freq * (t_base + size * t_transfer) / size for every cluster. */
+int32_t swarm_set_cache(swarm_ctx* ctx, const swarm_cache* cache);
 
 /* Number of key-range splits used by the attention kernels (>= 1; 0 restores the default chosen
  * from the shape).  Results do not depend on it beyond floating-point rounding. */

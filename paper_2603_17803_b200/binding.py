@@ -25,7 +25,7 @@ _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
-    "swarm_set_attn_splits", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_set_attn_splits", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
 )
 
@@ -52,6 +52,11 @@ class swarm_inputs(ctypes.Structure):
 class swarm_outputs(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("scores", "sel", "n_sel", "uniq", "queue_of", "n_uniq", "queue_load",
                                                "k_out", "v_out", "n_tok", "out", "lse")]
+
+
+class swarm_cache(ctypes.Structure):
+    _fields_ = [("resident", ctypes.c_void_p), ("freq", ctypes.c_void_p), ("score", ctypes.c_void_p),
+                ("n_hit", ctypes.c_void_p), ("t_base", ctypes.c_float), ("t_transfer", ctypes.c_float)]
 
 
 _lib = None
@@ -146,6 +151,17 @@ def swarm_set_workspace(ctx, workspace: torch.Tensor, stream=None) -> None:
 
 def swarm_set_attn_splits(ctx, n_splits: int) -> None:
     _check(load_library().swarm_set_attn_splits(ctx, ctypes.c_int32(n_splits)), "swarm_set_attn_splits", ctx)
+
+
+def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_base=0.0, t_transfer=0.0) -> None:
+    """Attach cache state (uint8 resident, int32 freq, optional float32 score, optional int32 n_hit), or detach it
+    when ``resident`` is None.  The caller keeps the tensors alive while they are attached."""
+    if resident is None:
+        _check(load_library().swarm_set_cache(ctx, None), "swarm_set_cache", ctx)
+        return
+    c = swarm_cache(_ptr(resident, "resident"), _ptr(freq, "freq"), _ptr(score, "score"), _ptr(n_hit, "n_hit"),
+                    float(t_base), float(t_transfer))
+    _check(load_library().swarm_set_cache(ctx, ctypes.byref(c)), "swarm_set_cache", ctx)
 
 
 def swarm_build_summaries(ctx, inputs: swarm_inputs, ksum_out: torch.Tensor, stream=None) -> None:

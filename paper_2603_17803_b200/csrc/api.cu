@@ -21,6 +21,8 @@ struct swarm_ctx {
   cudaGraphExec_t host_graph;  // swarm_step_host: the recorded step, valid for the arguments in host_key
   unsigned char host_key[256];
   bool host_graph_ok;
+  bool has_cache;
+  swarm_cache cache;
 };
 
 namespace {
@@ -137,6 +139,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->last_err = cudaSuccess;
   ctx->host_graph = nullptr;
   ctx->host_graph_ok = true;
+  ctx->has_cache = false;
   std::memset(ctx->host_key, 0, sizeof ctx->host_key);
   cudaError_t e = configure_score();
   if (e == cudaSuccess) e = configure_topk();
@@ -180,6 +183,17 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits) {
   if (ctx == nullptr || n_splits < 0 || n_splits > kMaxSplits) return SWARM_ERR_INVALID_ARG;
   ctx->user_splits = n_splits;
+  return SWARM_OK;
+}
+
+int32_t swarm_set_cache(swarm_ctx* ctx, const swarm_cache* cache) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (cache != nullptr && (cache->resident == nullptr || cache->freq == nullptr || !(cache->t_base >= 0.f) ||
+                           !(cache->t_transfer >= 0.f)))
+    return SWARM_ERR_INVALID_ARG;
+  ctx->has_cache = cache != nullptr;
+  if (cache != nullptr) ctx->cache = *cache;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
   return SWARM_OK;
 }
 
@@ -233,7 +247,8 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
                            ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), uniq, queue_of,
                            n_uniq, queue_load,
-                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream), false));
+                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream), false,
+                           ctx->has_cache ? &ctx->cache : nullptr));
   return SWARM_OK;
 }
 
@@ -339,7 +354,8 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
   SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
                            ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), o->uniq,
-                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true));
+                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true,
+                           ctx->has_cache ? &ctx->cache : nullptr));
   SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
   return SWARM_OK;
 }

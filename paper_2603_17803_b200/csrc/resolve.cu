@@ -9,6 +9,8 @@
 //     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 16 flags
 //              with one 16-byte load, a warp scan places them; the flags are cleared on the way
 //              so the next call starts from zeros.
+//              With cache state attached (swarm_set_cache) the same pass drops the activated clusters
+//              that are resident (Eq. 8) and updates the activation frequencies and Eq. 6 scores.
 //     route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
 //              with R >= 2 replicas are visited by (R ascending, id ascending) by one warp: lane j
 //              keeps (load[j] << 5 | j); one redux.min over the lanes named by the replica mask
@@ -30,8 +32,9 @@ __device__ __forceinline__ int nonzero_bytes(uint32_t w) {
   return __popc(t);
 }
 
+template <bool kCached>
 __global__ void __launch_bounds__(kThreads)
-resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __restrict__ n_sel,
+resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel, const int32_t* __restrict__ n_sel,
                const int64_t* __restrict__ page_base, const int32_t* __restrict__ page2cluster,
                const int64_t* __restrict__ cluster_base, const uint32_t* __restrict__ replica_mask,
                const uint16_t* __restrict__ cluster_size, uint8_t* __restrict__ flags,
@@ -43,8 +46,10 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
   __shared__ unsigned s_classes;
   __shared__ unsigned s_item_m[32], s_item_w[32];
   __shared__ bool s_last;
+  __shared__ int s_hits;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_hits = 0;
   pdl_wait();                                            // the flags / the selection come from the previous kernel
   const long long c_all = cluster_base[geo.B];
   const int C = (int)min((long long)geo.Cmax, c_all);
@@ -123,6 +128,12 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
       const uint4 f = __ldcg(f4 + v);
       f_keep = f;
       cnt += nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
+      if (kCached) {                                       // activated but resident: not fetched (Eq. 8)
+        const uint32_t words[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) && cache.resident[v * 16 + j]) --cnt;
+      }
     }
   }
 #pragma unroll
@@ -144,7 +155,30 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
       f = one_vec ? f_keep : __ldcg(f4 + v);
       if (f.x | f.y | f.z | f.w) __stcg(f4 + v, make_uint4(0, 0, 0, 0));   // leave zeros for the next call
     }
-    const int mine = nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
+    const uint32_t words[4] = {f.x, f.y, f.z, f.w};
+    unsigned fetch_bits = 0u;                              // bit j: cluster v*16+j is activated and has to be fetched
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const bool on = ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) != 0u;
+      bool fetch = on;
+      if (kCached) {
+        // cache bookkeeping of Sec. 5.2 for every cluster, activated or not
+        const int c = v * 16 + j;
+        if (v < v_hi && c < C) {
+          const bool res = cache.resident[c] != 0;
+          int fr = cache.freq[c];
+          if (on) ++fr; else if (res) --fr;
+          if (on || res) cache.freq[c] = fr;
+          if (cache.score != nullptr) {
+            const float sz = (float)cluster_size[c];
+            cache.score[c] = (float)fr * (cache.t_base + sz * cache.t_transfer) / sz;
+          }
+          if (on && res) { fetch = false; atomicAdd(&s_hits, 1); }
+        }
+      }
+      fetch_bits |= (fetch ? 1u : 0u) << j;
+    }
+    const int mine = __popc(fetch_bits);
     int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -152,10 +186,9 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
       if (lane >= o) incl += t;
     }
     int pos = before + incl - mine;
-    const uint32_t words[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      if ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) {
+      if ((fetch_bits >> j) & 1u) {
         const int c = v * 16 + j, i = pos++;
         uniq[i] = c;
         const unsigned m = replica_mask[c];
@@ -227,6 +260,7 @@ resolve_kernel(Geometry geo, const int32_t* __restrict__ sel, const int32_t* __r
     if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
     if (lane == 0) {
       *n_uniq = n;
+      if (kCached && cache.n_hit != nullptr) *cache.n_hit = s_hits;
       if (gridDim.x > 1) *ticket = 0u;                               // ready for the next call
     }
   }
@@ -240,13 +274,17 @@ cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                            const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                           cudaStream_t st, bool overlap) {
+                           cudaStream_t st, bool overlap, const swarm_cache* cache) {
   const long long slots = (long long)geo.B * geo.Hq * geo.k;
   const unsigned grid =
       sel == nullptr ? 1u : (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
-  return launch_pdl(resolve_kernel, dim3(grid), dim3(kThreads), 0, st, overlap, geo, sel, n_sel, page_base,
-                    page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq, queue_of,
-                    n_uniq, queue_load, status);
+  if (cache != nullptr)
+    return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), 0, st, overlap, geo, *cache, sel, n_sel,
+                      page_base, page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq,
+                      queue_of, n_uniq, queue_load, status);
+  return launch_pdl(resolve_kernel<false>, dim3(grid), dim3(kThreads), 0, st, overlap, geo, swarm_cache{}, sel, n_sel,
+                    page_base, page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq,
+                    queue_of, n_uniq, queue_load, status);
 }
 
 }  // namespace swarm

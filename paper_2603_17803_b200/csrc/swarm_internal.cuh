@@ -60,7 +60,7 @@ cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                            const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                           cudaStream_t st, bool overlap);
+                           cudaStream_t st, bool overlap, const swarm_cache* cache = nullptr);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,
                           int32_t* n_tok, uint32_t* status, cudaStream_t st);

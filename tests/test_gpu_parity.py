@@ -309,3 +309,46 @@ def test_paged_attention_alone_matches_gathered_attention():
     torch.cuda.synchronize()
     assert torch.equal(sess.o.out, out2)
     sess.close()
+
+
+@pytest.mark.parametrize("name", ["c3_small", "c5_small"])
+def test_resident_filter_and_cache_counters(name):
+    """Eq. 8 with the resident term, activation frequencies and Eq. 6 scores, against the oracle on the GPU's
+    own selection; two steps in a row so the counters accumulate; then detached again."""
+    w = W.generate(CASES[name], seed=16, device=DEV)
+    sess = Session(w)
+    C = w.n_clusters
+    g = torch.Generator(device="cpu").manual_seed(5)
+    resident = (torch.rand(C, generator=g) < 0.3).to(torch.uint8).to(DEV)
+    freq0 = torch.randint(-3, 10, (C,), generator=g, dtype=torch.int32)
+    freq = freq0.to(DEV)
+    score = torch.zeros(C, dtype=torch.float32, device=DEV)
+    n_hit = torch.zeros(4, dtype=torch.int32, device=DEV)
+    t_base, t_tr = 80.0, 2.5
+    B.swarm_set_cache(sess.ctx, resident=resident, freq=freq, score=score, n_hit=n_hit, t_base=t_base, t_transfer=t_tr)
+    tabs = parity.host_tables(w)
+    want_freq = freq0.numpy().copy()
+    for step_no in range(2):
+        if step_no == 0:
+            sess.step()
+        else:                                             # the separate call takes the same path
+            sess.resolve()
+        torch.cuda.synchronize()
+        assert sess.status() == 0
+        uniq, qof, load, hits, want_freq, want_score = oracle.resolve_cached(
+            sess.o.sel.cpu().numpy(), sess.o.n_sel.cpu().numpy(), tabs["page_base"], tabs["page2cluster"],
+            tabs["cluster_base"], tabs["replica_mask"], tabs["cluster_size"], resident.cpu().numpy(), want_freq,
+            w.cfg.n_queues, t_base, t_tr)
+        n = int(sess.o.n_uniq[0])
+        assert n == len(uniq) and hits > 0
+        assert np.array_equal(sess.o.uniq[:n].cpu().numpy(), uniq)
+        assert np.array_equal(sess.o.queue_of[:n].cpu().numpy(), qof)
+        assert np.array_equal(sess.o.queue_load.cpu().numpy()[: w.cfg.n_queues], load)
+        assert int(n_hit[0]) == hits
+        assert np.array_equal(freq.cpu().numpy(), want_freq)
+        assert np.allclose(score.cpu().numpy(), want_score, rtol=1e-6, atol=1e-6)
+    B.swarm_set_cache(sess.ctx)                           # detached: plain merge again
+    sess.step()
+    parity.check_step(w, sess)
+    assert np.array_equal(freq.cpu().numpy(), want_freq)
+    sess.close()
