@@ -352,3 +352,31 @@ def test_resident_filter_and_cache_counters(name):
     parity.check_step(w, sess)
     assert np.array_equal(freq.cpu().numpy(), want_freq)
     sess.close()
+
+
+EDGE_SHAPES = {
+    # group of 16 heads per KV head (two head tiles in the scorer and in attention), 32-token pages
+    "g16_s32": small("c4_long", batch=2, n_q_heads=32, n_kv_heads=2, ctx_len=32 * 300 + 5, top_k=24, n_topics=6),
+    # odd number of KV heads, group of 2
+    "hkv3_g2": small("c2_128k", batch=2, n_q_heads=6, n_kv_heads=3, ctx_len=16 * 500 + 3, top_k=33, n_topics=5),
+    # more KV heads than one scorer block holds (two KV groups), MHA
+    "hkv16_g1": small("c1_tiny", batch=1, n_q_heads=16, n_kv_heads=16, ctx_len=16 * 260, top_k=17),
+    # a single page per head, a single queue
+    "k1_d1": small("c3_batched", batch=3, ctx_len=16 * 150 + 1, top_k=1, n_topics=4, n_queues=1, replication="one"),
+    # group of 12 heads: a full head tile of 8 plus a partial one of 4
+    "g12": small("c2_128k", batch=1, n_q_heads=24, n_kv_heads=2, ctx_len=16 * 400, top_k=40, n_topics=6),
+}
+
+
+@pytest.mark.parametrize("name", list(EDGE_SHAPES))
+def test_unusual_shapes(name):
+    w = W.generate(EDGE_SHAPES[name], seed=17, device=DEV)
+    a = Session(w, keep_scores=True, keep_gathered=True)
+    run_separate_calls(a)
+    parity.check_step(w, a)
+    b = Session(w, keep_scores=True, keep_gathered=True, ksum=a.ksum)
+    b.step()
+    parity.check_step(w, b)
+    assert torch.equal(a.o.sel, b.o.sel) and (a.o.out - b.o.out).abs().max().item() <= 1e-4
+    a.close()
+    b.close()
