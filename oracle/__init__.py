@@ -96,15 +96,16 @@ def scores(q, ksum, page_base, ctx_len, Hkv, S, Pmax):
     return s64, s32, cond
 
 
-def topk(score, ctx_len, S, k):
-    """score float32 [B][Hq][Pmax] -> (sel int32 [B][Hq][k] ascending page id, -1 padded; n_sel [B][Hq])."""
+def topk(score, ctx_len, S, k, window=0):
+    """score float32 [B][Hq][Pmax] -> (sel int32 [B][Hq][k] ascending page id, -1 padded; n_sel [B][Hq]).
+    The last ``window`` pages of every request are always selected."""
     score = _arr(score, np.float32)
     ctx_len = _arr(ctx_len, np.int32)
     B, Hq, Pmax = score.shape
     sel = np.empty((B, Hq, k), dtype=np.int32)
     n_sel = np.empty((B, Hq), dtype=np.int32)
     rc = _load().oracle_topk(_p(score), _p(ctx_len), ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(S),
-                             ctypes.c_int64(Pmax), ctypes.c_int32(k), _p(sel), _p(n_sel))
+                             ctypes.c_int64(Pmax), ctypes.c_int32(k), ctypes.c_int32(window), _p(sel), _p(n_sel))
     _check(rc, "topk")
     return sel, n_sel
 
@@ -216,12 +217,12 @@ class StepResult:
 
 
 def step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base, replica_mask, cluster_size, *, Hkv, S, k,
-         D, Pmax, flags=0, sel_override=None) -> StepResult:
+         D, Pmax, flags=0, window=0, sel_override=None) -> StepResult:
     """The whole path, stage after stage.  ``sel_override=(sel, n_sel)`` replaces the oracle's own selection
     for the downstream stages (stage-conditional parity)."""
     d = np.asarray(q).shape[-1]
     s64, s32, cond = scores(q, ksum, page_base, ctx_len, Hkv, S, Pmax)
-    sel, n_sel = topk(s32, ctx_len, S, k)
+    sel, n_sel = topk(s32, ctx_len, S, k, window)
     use_sel, use_n = (sel, n_sel) if sel_override is None else sel_override
     uniq, queue_of, load = resolve(use_sel, use_n, page_base, page2cluster, cluster_base, replica_mask,
                                    cluster_size, D, flags)

@@ -156,9 +156,12 @@ int oracle_scores(const uint16_t* q, const uint16_t* ksum, const int64_t* page_b
 // Per (b,h): order the P_b pages by (score descending, page id ascending), keep the first
 // k_eff = min(k, P_b), and emit them in ascending page id.  Unused slots are -1.
 // Scores compare as real numbers (so -0 == +0).
+// Local window (Sec. 4.2, Tier 1 (2)): the last `window` pages of a request are always kept -- they rank
+// above every score -- and the remaining k - window places go to the best of the other pages.
 int oracle_topk(const float* score, const int32_t* ctx_len, int32_t B, int32_t Hq, int32_t S, int64_t Pmax,
-                int32_t k, int32_t* sel, int32_t* n_sel) {
-  if (!score || !ctx_len || !sel || !n_sel || B < 1 || Hq < 1 || S < 1 || k < 1) return ORACLE_BAD_ARG;
+                int32_t k, int32_t window, int32_t* sel, int32_t* n_sel) {
+  if (!score || !ctx_len || !sel || !n_sel || B < 1 || Hq < 1 || S < 1 || k < 1 || window < 0 || window > k)
+    return ORACLE_BAD_ARG;
 #pragma omp parallel for collapse(2) schedule(dynamic, 1)
   for (int32_t b = 0; b < B; ++b) {
     for (int32_t h = 0; h < Hq; ++h) {
@@ -166,7 +169,13 @@ int oracle_topk(const float* score, const int32_t* ctx_len, int32_t B, int32_t H
       const float* s = score + (static_cast<int64_t>(b) * Hq + h) * Pmax;
       std::vector<int32_t> ids(static_cast<size_t>(P));
       for (int64_t p = 0; p < P; ++p) ids[static_cast<size_t>(p)] = static_cast<int32_t>(p);
-      std::stable_sort(ids.begin(), ids.end(), [s](int32_t a, int32_t c) { return s[a] > s[c]; });
+      const int64_t first_window = P - window;              // pages >= this are in the local window
+      std::stable_sort(ids.begin(), ids.end(), [s, first_window](int32_t a, int32_t c) {
+        const bool wa = a >= first_window, wc = c >= first_window;
+        if (wa != wc) return wa;                            // window pages first
+        if (wa) return false;                               // among themselves: keep id order
+        return s[a] > s[c];
+      });
       const int64_t k_eff = std::min<int64_t>(k, P);
       std::vector<int32_t> best(ids.begin(), ids.begin() + k_eff);
       std::sort(best.begin(), best.end());

@@ -505,3 +505,22 @@ def test_cache_score_hand_case():
     out = oracle.resolve_cached(sel, np.ones((1, 1), np.int32), [0, 1], [0], [0, 1], np.array([1], np.uint32),
                                 np.array([4], np.uint16), np.array([1], np.uint8), np.array([5], np.int32), 2, 100.0, 5.0)
     assert out[3] == 1 and list(out[4]) == [6] and out[5][0] == 180.0 and len(out[0]) == 0
+
+
+def test_topk_local_window_is_the_last_pages_plus_the_best_of_the_rest():
+    rng = np.random.default_rng(14)
+    for _ in range(100):
+        P = int(rng.integers(1, 30))
+        k = int(rng.integers(1, 12))
+        w = int(rng.integers(0, k + 1))
+        vals = rng.integers(-4, 5, size=P).astype(np.float32)
+        sc = np.full((1, 1, 32), np.nan, dtype=np.float32)
+        sc[0, 0, :P] = vals
+        sel, n = oracle.topk(sc, [P], 1, k, window=w)
+        k_eff = min(k, P)
+        window_pages = list(range(max(0, P - w), P))
+        rest = brute_topk(vals[: max(0, P - w)], k_eff - len(window_pages)) if k_eff > len(window_pages) else []
+        want = sorted(set(window_pages[-k_eff:] if len(window_pages) > k_eff else window_pages) | set(rest))
+        assert n[0, 0] == k_eff and list(sel[0, 0, :k_eff]) == want
+    with pytest.raises(ValueError):
+        oracle.topk(sc, [P], 1, 3, window=4)
