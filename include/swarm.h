@@ -69,6 +69,10 @@ typedef struct swarm_shape {
   int32_t max_clusters_total; /* upper bound on cluster_base[B]; capacity of uniq / queue_of     */
   uint32_t flags;
   int64_t n_pool_pages;       /* pages in the pool (page_base[B] <= n_pool_pages)                */
+  int32_t local_window_pages; /* W: the last W pages of every request are always selected and    */
+                              /* take W of the k places (local window of Sec. 4.2, Tier 1 (2));  */
+                              /* 0 <= W <= top_k; 0 = plain top-k                                */
+  int32_t reserved;           /* must be 0                                                       */
 } swarm_shape;
 
 /* Read-only device-resident inputs of a step. */

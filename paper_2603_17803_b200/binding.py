@@ -41,7 +41,8 @@ class SwarmError(RuntimeError):
 class swarm_shape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("batch", "n_q_heads", "n_kv_heads", "head_dim", "page_size", "top_k",
                                               "n_queues", "max_pages_per_req", "max_clusters_total")] + \
-               [("flags", ctypes.c_uint32), ("n_pool_pages", ctypes.c_int64)]
+               [("flags", ctypes.c_uint32), ("n_pool_pages", ctypes.c_int64),
+                ("local_window_pages", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class swarm_inputs(ctypes.Structure):
@@ -99,9 +100,9 @@ def _check(rc: int, what: str, ctx=None):
 
 
 def make_shape(*, batch, n_q_heads, n_kv_heads, page_size, top_k, n_queues, max_pages_per_req, max_clusters_total,
-               n_pool_pages, head_dim=128, flags=0) -> swarm_shape:
+               n_pool_pages, head_dim=128, flags=0, local_window_pages=0) -> swarm_shape:
     return swarm_shape(batch, n_q_heads, n_kv_heads, head_dim, page_size, top_k, n_queues, max_pages_per_req,
-                       max_clusters_total, flags, n_pool_pages)
+                       max_clusters_total, flags, n_pool_pages, local_window_pages, 0)
 
 
 def make_inputs(*, q=None, ksum=None, kv_pool=None, page_base=None, ctx_len=None, page2cluster=None,

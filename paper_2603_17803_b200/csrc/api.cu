@@ -33,7 +33,8 @@ int32_t check_shape(const swarm_shape* s) {
   if (s == nullptr) return SWARM_ERR_INVALID_ARG;
   if (s->batch < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->top_k < 1 || s->max_pages_per_req < 1 ||
       s->max_clusters_total < 1 || s->n_pool_pages < 1 || s->n_queues < 1 || s->n_queues > 32 ||
-      s->n_q_heads % s->n_kv_heads != 0 || (s->flags & ~(SWARM_ORDER_BY_ID | SWARM_UNIT_LOAD)) != 0u)
+      s->n_q_heads % s->n_kv_heads != 0 || (s->flags & ~(SWARM_ORDER_BY_ID | SWARM_UNIT_LOAD)) != 0u ||
+      s->local_window_pages < 0 || s->local_window_pages > s->top_k || s->reserved != 0)
     return SWARM_ERR_INVALID_ARG;
   if (s->head_dim != kHeadDim || (s->page_size != 16 && s->page_size != 32)) return SWARM_ERR_UNSUPPORTED;
   // launch-grid and index-width limits
@@ -132,6 +133,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   g.B = shape->batch; g.Hq = shape->n_q_heads; g.Hkv = shape->n_kv_heads; g.g = g.Hq / g.Hkv;
   g.S = shape->page_size; g.k = shape->top_k; g.D = shape->n_queues; g.Pmax = shape->max_pages_per_req;
   g.Cmax = shape->max_clusters_total; g.flags = shape->flags; g.n_pool_pages = shape->n_pool_pages;
+  g.W = shape->local_window_pages;
   ctx->lay = make_layout(*shape);
   ctx->ws = nullptr;
   ctx->ws_bytes = 0;

@@ -696,7 +696,7 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   if (configure_attention() != cudaSuccess) return SWARM_ERR_CUDA;   // raises a kernel attribute; allocates nothing
   Geometry geo{};
   geo.B = batch; geo.Hq = n_q_heads; geo.Hkv = n_q_heads; geo.g = 1; geo.S = page_size; geo.k = top_k; geo.D = 1;
-  geo.Pmax = top_k; geo.Cmax = 1; geo.flags = 0; geo.n_pool_pages = 0;
+  geo.Pmax = top_k; geo.Cmax = 1; geo.flags = 0; geo.n_pool_pages = 0; geo.W = 0;
   AttnArgs a{};
   a.q = static_cast<const uint16_t*>(q);
   a.k_g = static_cast<const uint16_t*>(k_g);

@@ -32,6 +32,7 @@ __host__ __device__ inline int selmap_pitch_bytes(int Pmax) { return ((Pmax + 7)
 
 struct Geometry {   // plain copy of the shape in kernel-friendly form
   int B, Hq, Hkv, g, S, k, D, Pmax, Cmax;
+  int W;                // local window in pages: the last W pages of a request are always selected
   unsigned flags;
   long long n_pool_pages;
 };

@@ -198,6 +198,8 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   SWARM_STAMP(status, 1);
   const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
+  const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
+  const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
 
@@ -214,16 +216,19 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) key[j] = p0 + j < P ? score_key(s[p0 + j]) : 0u;
   }
-  if (tid == 0) st.remaining = k_eff;
+  if (tid == 0) st.remaining = k_sel;
   SWARM_STAMP(status, 2);
 
   uint32_t T = 0u;
-  int need_eq = P;                                          // k_eff == P keeps everything
-  if (k_eff < P) {
+  int need_eq = P;                                          // k_sel == Pw keeps everything
+  if (k_sel == 0) {
+    T = 0xFFFFFFFFu;                                        // nothing but the window
+    need_eq = 0;
+  } else if (k_sel < Pw) {
     uint32_t lo = 0xFFFFFFFFu, hi = 0u;
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j)
-      if (p0 + j < P) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+      if (p0 + j < Pw) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
     block_minmax<THREADS>(st, tid, lo, hi);
     SWARM_STAMP(status, 3);
     for (int level = 0; level < 4 && st.bits > 0; ++level) {
@@ -234,7 +239,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
 #pragma unroll
       for (int j = 0; j < ITEMS; ++j) {
         const uint32_t rel = key[j] - base;
-        if (p0 + j < P && rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
+        if (p0 + j < Pw && rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
       }
       __syncthreads();
       SWARM_STAMP(status, 4 + 2 * level);
@@ -250,7 +255,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j)
-          if (p0 + j < P && key[j] - cbase <= cwidth_m1) st.cand[atomicAdd(&st.n_cand, 1)] = key[j];
+          if (p0 + j < Pw && key[j] - cbase <= cwidth_m1) st.cand[atomicAdd(&st.n_cand, 1)] = key[j];
         finish_by_ranking<THREADS>(st, tid, n_cand);
       }
     }
@@ -262,8 +267,10 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   // ordered output: packed (greater, equal) counts per thread, one block-wide exclusive scan
   int cnt = 0;
 #pragma unroll
-  for (int j = 0; j < ITEMS; ++j)
-    if (p0 + j < P) cnt += (key[j] > T ? 1 : 0) + (key[j] == T ? 0x10000 : 0);
+  for (int j = 0; j < ITEMS; ++j) {
+    if (p0 + j >= Pw) key[j] = p0 + j < P ? 0xFFFFFFFFu : 0u;   // window pages rank above every score
+    if (p0 + j < P) cnt += ((key[j] > T || p0 + j >= Pw) ? 1 : 0) + ((key[j] == T && p0 + j < Pw) ? 0x10000 : 0);
+  }
   int incl = cnt;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -280,7 +287,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
 #pragma unroll
   for (int j = 0; j < ITEMS; ++j) {
     if (p0 + j < P) {
-      const bool gt = key[j] > T, eq = key[j] == T;
+      const bool gt = key[j] > T || p0 + j >= Pw, eq = key[j] == T && p0 + j < Pw;
       if (gt || (eq && eq_before < need_eq)) {
         out[gt_before + min(eq_before, need_eq)] = p0 + j;
         picked |= 1u << j;
@@ -323,6 +330,8 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   pdl_wait();
   const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));
   const int k_eff = min(geo.k, P);
+  const int Pw = P - min(geo.W, P);                         // see topk_regs_kernel
+  const int k_sel = k_eff - (P - Pw);
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
   auto key_at = [&](int i) -> uint32_t { return kKeysInSmem ? skeys[i] : score_key(s[i]); };
@@ -331,20 +340,26 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   for (int i = tid; i < P; i += kGenericThreads) {
     const uint32_t key = score_key(s[i]);
     if (kKeysInSmem) skeys[i] = key;
-    lo = min(lo, key);
-    hi = max(hi, key);
+    if (i < Pw) {
+      lo = min(lo, key);
+      hi = max(hi, key);
+    }
   }
-  if (tid == 0) st.remaining = k_eff;
+  if (tid == 0) st.remaining = k_sel;
   uint32_t T = 0u;
   int need_eq = P;
-  if (k_eff < P) {
+  if (k_sel == 0) {
+    T = 0xFFFFFFFFu;
+    need_eq = 0;
+    __syncthreads();
+  } else if (k_sel < Pw) {
     block_minmax<kGenericThreads>(st, tid, lo, hi);
     for (int level = 0; level < 4 && st.bits > 0; ++level) {
       const uint32_t base = st.base;
       const int bits = st.bits;
       const int shift = max(bits - kDigitBits, 0);
       const uint32_t width_m1 = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
-      for (int i = tid; i < P; i += kGenericThreads) {
+      for (int i = tid; i < Pw; i += kGenericThreads) {
         const uint32_t rel = key_at(i) - base;
         if (rel <= width_m1) atomicAdd(&st.hist[hist_slot<kGenericThreads>(rel >> shift)], 1);
       }
@@ -364,8 +379,8 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
     const int i = i0 + lane;
     const uint32_t key = i < w_hi ? key_at(i) : 0u;
-    cnt_gt += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && key > T));
-    cnt_eq += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && key == T));
+    cnt_gt += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && (key > T || i >= Pw)));
+    cnt_eq += __popc(__ballot_sync(0xFFFFFFFFu, i < w_hi && key == T && i < Pw));
   }
   if (lane == 0) { warp_gt[warp] = cnt_gt; warp_eq[warp] = cnt_eq; }
   __syncthreads();
@@ -375,7 +390,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
     const int i = i0 + lane;
     const uint32_t key = i < w_hi ? key_at(i) : 0u;
-    const bool gt = i < w_hi && key > T, eq = i < w_hi && key == T;
+    const bool gt = i < w_hi && (key > T || i >= Pw), eq = i < w_hi && key == T && i < Pw;
     const unsigned bg = __ballot_sync(0xFFFFFFFFu, gt), be = __ballot_sync(0xFFFFFFFFu, eq);
     const int my_gt = gt_before + __popc(bg & lt_mask);
     const int my_eq = eq_before + __popc(be & lt_mask);

@@ -33,7 +33,7 @@ class Session:
     """One ctx bound to one resident KV pool (``workload`` tensors must live on a CUDA device)."""
 
     def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
-                 ksum: Optional[torch.Tensor] = None):
+                 ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0):
         cfg = workload.cfg
         self.cfg = cfg
         self.w = workload
@@ -45,7 +45,8 @@ class Session:
         self.shape = B.make_shape(batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                                   page_size=cfg.page_size, top_k=cfg.top_k, n_queues=cfg.n_queues,
                                   max_pages_per_req=self.Pmax, max_clusters_total=max(1, workload.n_clusters),
-                                  n_pool_pages=workload.n_pool_pages, flags=flags)
+                                  n_pool_pages=workload.n_pool_pages, flags=flags,
+                                  local_window_pages=local_window_pages)
         self.ctx = B.swarm_create(self.shape)
         self.workspace = torch.empty(B.swarm_workspace_bytes(self.shape), dtype=torch.uint8, device=dev)
         B.swarm_set_workspace(self.ctx, self.workspace)

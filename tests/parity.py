@@ -44,14 +44,21 @@ def check_scores(gpu_scores, s64, cond, P):
     return float((err / np.maximum(np.abs(ref), 1e-30)).max())
 
 
-def check_selection(sel_row, n_sel, s64_row, P, k):
-    """Band rule for one (request, head).  Returns the number of band pages that differ from the exact top-k."""
+def check_selection(sel_row, n_sel, s64_row, P, k, window=0):
+    """Band rule for one (request, head).  Returns the number of band pages that differ from the exact top-k.
+    With a local window the last `window` pages must all be there and the rule applies to the others."""
     k_eff = min(k, P)
     assert n_sel == k_eff
     chosen = sel_row[:k_eff]
     assert np.all(sel_row[k_eff:] == -1)
     assert np.all(chosen >= 0) and np.all(chosen < P)
     assert np.all(np.diff(chosen) > 0), "selection must be strictly ascending (no duplicates)"
+    w_eff = min(window, P)
+    if w_eff:
+        assert np.array_equal(chosen[k_eff - w_eff:], np.arange(P - w_eff, P)), "local window pages missing"
+        P, k_eff, chosen = P - w_eff, k_eff - w_eff, chosen[:k_eff - w_eff]
+        if k_eff == 0:
+            return 0
     s = s64_row[:P]
     order = np.lexsort((np.arange(P), -s))
     tau = s[order[k_eff - 1]]
@@ -104,6 +111,7 @@ def check_request(w, sess, b, tabs, *, heads=None, check_gathered=True):
     q_b = bits_u16(w.q[b:b + 1])
     s64, s32, cond = oracle.scores(q_b, ksum_ref, pb, cl, Hkv, S, P)
     o = sess.o
+    W = int(sess.shape.local_window_pages)
     hs = range(Hq) if heads is None else heads
     info = dict(band_diffs=0, exact_heads=0, heads=0)
     sel_gpu = o.sel[b].cpu().numpy()
@@ -113,12 +121,12 @@ def check_request(w, sess, b, tabs, *, heads=None, check_gathered=True):
         info["score_rel_err"] = check_scores(sc_gpu[list(hs)], s64[0][list(hs)], cond[0][list(hs)], P)
         if P < sc_gpu.shape[-1]:
             assert np.all(np.isneginf(sc_gpu[:, P:])), "scores beyond the request's pages were written"
-        sel_on_gpu_scores, _ = oracle.topk(sc_gpu[None, :, :P], cl, S, k)
+        sel_on_gpu_scores, _ = oracle.topk(sc_gpu[None, :, :P], cl, S, k, W)
         assert np.array_equal(sel_on_gpu_scores[0][list(hs)], sel_gpu[list(hs)]), \
             "selection is not the exact top-k of the GPU's own scores"
-    sel_ref, nsel_ref = oracle.topk(s32, cl, S, k)
+    sel_ref, nsel_ref = oracle.topk(s32, cl, S, k, W)
     for h in hs:
-        info["band_diffs"] += check_selection(sel_gpu[h], int(nsel_gpu[h]), s64[0, h], P, k)
+        info["band_diffs"] += check_selection(sel_gpu[h], int(nsel_gpu[h]), s64[0, h], P, k, W)
         info["exact_heads"] += int(np.array_equal(sel_gpu[h], sel_ref[0, h]))
         info["heads"] += 1
 

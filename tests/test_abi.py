@@ -57,6 +57,6 @@ def test_shape_validation_runs_without_a_gpu(lib_path):
 
 def test_struct_layouts_match_the_header():
     from paper_2603_17803_b200 import binding as B
-    assert ctypes.sizeof(B.swarm_shape) == 48          # 9 x int32 + uint32 + int64
+    assert ctypes.sizeof(B.swarm_shape) == 56          # 9 x int32 + uint32 + int64 + 2 x int32
     assert ctypes.sizeof(B.swarm_inputs) == 9 * 8
     assert ctypes.sizeof(B.swarm_outputs) == 12 * 8

@@ -380,3 +380,65 @@ def test_unusual_shapes(name):
     assert torch.equal(a.o.sel, b.o.sel) and (a.o.out - b.o.out).abs().max().item() <= 1e-4
     a.close()
     b.close()
+
+
+# ---- local window (Sec. 4.2, Tier 1 (2)): the last W pages of every request are always selected ------------
+@pytest.mark.parametrize("name,window", [("c1_small", 1), ("c2_small", 16), ("c3_small", 2), ("c4_small", 8), ("c5_small", 3),
+                                         ("k_exceeds_pages", 8), ("k_exceeds_pages", 24)])
+def test_local_window(name, window):
+    cfg = CASES[name]
+    window = min(window, cfg.top_k)
+    w = W.generate(cfg, seed=23, device=DEV)
+    a = Session(w, keep_scores=True, keep_gathered=True, local_window_pages=window)
+    a.step()
+    parity.check_step(w, a)
+    sel, n_sel = a.o.sel.cpu().numpy(), a.o.n_sel.cpu().numpy()
+    ctx = w.ctx_len.cpu().numpy()
+    for b in range(cfg.batch):
+        P = -(-int(ctx[b]) // cfg.page_size)
+        w_eff = min(window, P)
+        for h in range(cfg.n_q_heads):
+            n = int(n_sel[b, h])
+            assert list(sel[b, h, n - w_eff:n]) == list(range(P - w_eff, P))
+    b_ = Session(w, keep_scores=True, keep_gathered=True, ksum=a.ksum, local_window_pages=window)
+    run_separate_calls(b_)
+    parity.check_step(w, b_)
+    assert torch.equal(a.o.sel, b_.o.sel)
+    a.close()
+    b_.close()
+
+
+def test_local_window_covering_all_of_k_and_longer_than_a_request():
+    cfg = small("c3_batched", batch=3, ctx_len=16 * 40, top_k=12, n_topics=4)
+    w = W.generate(cfg, seed=29, device=DEV)
+    w.ctx_len[1] = 16 * 5 + 3                               # 6 pages < window
+    a = Session(w, keep_scores=True, keep_gathered=True, local_window_pages=12)
+    a.step()
+    parity.check_step(w, a)
+    a.close()
+    with pytest.raises(B.SwarmError):
+        Session(w, local_window_pages=13)
+
+
+# ---- every list-length variant of the selection kernel, with and without a local window --------------------
+@pytest.mark.parametrize("pages", [900, 2000, 4000, 8000, 16000, 30000, 45000])
+@pytest.mark.parametrize("window", [0, 5])
+def test_selection_at_every_list_length(pages, window):
+    cfg = small("c1_tiny", batch=2, n_q_heads=2, n_kv_heads=1, ctx_len=16 * pages - 7, top_k=100, n_topics=8)
+    w = W.generate(cfg, seed=31, device=DEV)
+    w.ctx_len[1] = 16 * (pages // 3) + 1                    # a shorter request beside the long one
+    sess = Session(w, keep_scores=True, local_window_pages=window)
+    sess.select()
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    sc = sess.o.scores.cpu().numpy()
+    sel, n_sel = sess.o.sel.cpu().numpy(), sess.o.n_sel.cpu().numpy()
+    ctx = w.ctx_len.cpu().numpy()
+    want, n_want = oracle.topk(sc, ctx, cfg.page_size, cfg.top_k, window)
+    assert np.array_equal(n_sel, n_want) and np.array_equal(sel, want)
+    # the fused step marks the same pages and attends to them
+    sess.step()
+    torch.cuda.synchronize()
+    assert np.array_equal(sess.o.sel.cpu().numpy(), want)
+    parity.check_step(w, sess, requests=[1], heads=[1])
+    sess.close()
