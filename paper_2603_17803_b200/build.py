@@ -37,13 +37,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ_DIR, exist_ok=True)
     header_time = _newest(headers)
     extra = ["-Xptxas", "-v"] if verbose else []
-    if os.environ.get("SWARM_TRACE"):          # development-only cycle stamps inside the kernels
-        extra += ["-DSWARM_TRACE=" + os.environ["SWARM_TRACE"]]
+    trace = ["-DSWARM_TRACE=" + os.environ["SWARM_TRACE"]] if os.environ.get("SWARM_TRACE") else []
+    trace += os.environ.get("SWARM_DEFINES", "").split()   # development-only extra -D flags
+    trace_only = os.environ.get("SWARM_TRACE_ONLY")      # development-only time stamps, optionally in one file
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), header_time):
-            cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
+            mine = trace if not trace_only or os.path.basename(src) == trace_only else []
+            cmd = [_nvcc(), *NVCC_FLAGS, *extra, *mine, "-c", src, "-o", obj]
             res = subprocess.run(cmd, capture_output=True, text=True)
             if verbose or res.returncode != 0:
                 sys.stderr.write(res.stdout + res.stderr)

@@ -107,14 +107,14 @@ __device__ __forceinline__ uint32_t tile_offset(int t, int chunk) {
 }
 
 template <int S, bool kPaged>
-__global__ void __launch_bounds__(kAttnWarps * 32)
+__global__ void __launch_bounds__(kAttnWarps * 32, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Geometry geo,
             AttnArgs a, uint32_t* __restrict__ status) {
   constexpr int SB = S / kUnitTokens;                   // 16-token units per page
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
   __shared__ __align__(8) uint64_t bar_merge;
-  __shared__ int s_count;
+  __shared__ int s_wcnt[kAttnWarps];
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
@@ -155,44 +155,52 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   long long pool_row0 = 0;
   int n_words = 0;
 
-  // 4 consecutive bitmap words (128 pages) of every head of the group, and their union with pages >= P cut off
-  auto load_words = [&](int w0, uint4 (&hw)[8], uint4& uni) {
-    uni = make_uint4(0u, 0u, 0u, 0u);
+  // one bitmap word (32 pages) of every head of the group; the row pitch bounds the loads, so they do not
+  // have to wait for the request's length
+  const int pitch_words = a.selmap_pitch / 4;
+  struct HeadWords { uint32_t v[8]; };
+  auto load_raw = [&](int w) -> HeadWords {
+    HeadWords hw;
 #pragma unroll
     for (int hh = 0; hh < 8; ++hh) {
-      hw[hh] = make_uint4(0u, 0u, 0u, 0u);
-      if (hh < G && w0 < n_words)
-        hw[hh] = *reinterpret_cast<const uint4*>(a.selmap + (long long)(bh0 + hh) * a.selmap_pitch + (long long)w0 * 4);
-      uni.x |= hw[hh].x; uni.y |= hw[hh].y; uni.z |= hw[hh].z; uni.w |= hw[hh].w;
+      hw.v[hh] = 0u;
+      if (hh < G && w < pitch_words)
+        hw.v[hh] = *reinterpret_cast<const uint32_t*>(a.selmap + (long long)(bh0 + hh) * a.selmap_pitch + (long long)w * 4);
     }
-    uint32_t* u = &uni.x;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int first = (w0 + j) * 32;
-      if (first + 32 > P) u[j] &= first >= P ? 0u : (0xFFFFFFFFu >> (32 - (P - first)));
-    }
+    return hw;
   };
+  // their union, with the pages >= P cut off
+  auto union_of = [&](int w, const HeadWords& hw) -> uint32_t {
+    uint32_t uni = 0u;
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) uni |= hw.v[hh];
+    const int first = w * 32;
+    if (first + 32 > P) uni &= first >= P ? 0u : (0xFFFFFFFFu >> (32 - (P - first)));
+    return uni;
+  };
+  constexpr int kChunkWords = kAttnWarps * 32;          // bitmap words one pass of the CTA covers
 
   if (kPaged) {
+    // number of pages in the union of the group's selections: the splits share them evenly by rank
+    HeadWords hw = load_raw((int)threadIdx.x);          // in flight together with the two loads below
     const int len = a.ctx_len[b];
+    pool_row0 = a.page_base[b];
     P = pages_of(len, S);
     tail = len - S * (P - 1);
-    pool_row0 = a.page_base[b];
-    n_words = (P + 31) / 32;
-    // number of pages in the union of the group's selections: the splits share them evenly by rank
-    if (warp == 0) {
-      int total = 0;
-      for (int base = 0; base < n_words; base += 128) {
-        uint4 hw[8], uni;
-        load_words(base + lane * 4, hw, uni);
-        total += __popc(uni.x) + __popc(uni.y) + __popc(uni.z) + __popc(uni.w);
-      }
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-      if (lane == 0) s_count = total;
+    n_words = min((P + 31) / 32, pitch_words);
+    int total = 0;
+    for (int base = 0; base < n_words; base += kChunkWords) {
+      const int w = base + (int)threadIdx.x;
+      if (base > 0) hw = load_raw(w);
+      total += __popc(union_of(w, hw));
     }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+    if (lane == 0) s_wcnt[warp] = total;
     __syncthreads();
-    n_items = s_count;
+    n_items = 0;
+#pragma unroll
+    for (int w2 = 0; w2 < kAttnWarps; ++w2) n_items += s_wcnt[w2];
   } else {
     total_tok = a.n_tok[bh0];
     n_items = (total_tok + S - 1) / S;
@@ -229,42 +237,42 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   for (int round0 = it_begin; round0 < it_end; round0 += kPaged ? kListCap : (it_end - it_begin)) {
     int n_list;
     if (kPaged) {
-      // warp 0: pages of the union with rank in [round0, round_end) -> (page, head mask) list, ascending
+      // pages of the union with rank in [round0, round_end) -> (page, head mask) list, ascending; every
+      // thread ranks the pages of its own word with a CTA-wide scan of the per-thread counts
       const int round_end = min(it_end, round0 + kListCap);
-      __syncthreads();                                  // the previous round's list is no longer read
-      if (warp == 0) {
-        int rank0 = 0;                                  // union pages before the current 128 words
-        for (int base = 0; base < n_words && rank0 < round_end; base += 128) {
-          uint4 hw[8], uni;
-          const int w0 = base + lane * 4;
-          load_words(w0, hw, uni);
-          const int cnt = __popc(uni.x) + __popc(uni.y) + __popc(uni.z) + __popc(uni.w);
-          int incl = cnt;
+      int rank0 = 0;                                    // union pages before the current chunk of words
+      for (int base = 0; base < n_words && rank0 < round_end; base += kChunkWords) {
+        const int w = base + (int)threadIdx.x;
+        const HeadWords hw = load_raw(w);
+        uint32_t bits = union_of(w, hw);
+        const int cnt = __popc(bits);
+        int incl = cnt;
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if (lane >= o) incl += t;
-          }
-          int rank = rank0 + incl - cnt;                // rank of this lane's first union page
-          rank0 += __shfl_sync(0xFFFFFFFFu, incl, 31);
-          if (rank + cnt > round0 && rank < round_end) {
-            const uint32_t* u = &uni.x;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        __syncthreads();                                // the counts of the previous pass, and the previous
+        if (lane == 31) s_wcnt[warp] = incl;            // round's list, are no longer read
+        __syncthreads();
+        int rank = rank0 + incl - cnt;                  // rank of this thread's first union page
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t bits = u[j];
-              while (bits) {
-                const int bit = __ffs(bits) - 1;
-                bits &= bits - 1;
-                if (rank >= round0 && rank < round_end) {
-                  uint32_t hm = 0u;
+        for (int w2 = 0; w2 < kAttnWarps; ++w2) {
+          if (w2 < warp) rank += s_wcnt[w2];
+          rank0 += s_wcnt[w2];
+        }
+        if (rank + cnt > round0 && rank < round_end) {
+          while (bits) {
+            const int bit = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (rank >= round0 && rank < round_end) {
+              uint32_t hm = 0u;
 #pragma unroll
-                  for (int hh = 0; hh < 8; ++hh) hm |= (((&hw[hh].x)[j] >> bit) & 1u) << hh;
-                  list_page[rank - round0] = (uint32_t)((w0 + j) * 32 + bit);
-                  list_mask[rank - round0] = (uint8_t)hm;
-                }
-                ++rank;
-              }
+              for (int hh = 0; hh < 8; ++hh) hm |= ((hw.v[hh] >> bit) & 1u) << hh;
+              list_page[rank - round0] = (uint32_t)(w * 32 + bit);
+              list_mask[rank - round0] = (uint8_t)hm;
             }
+            ++rank;
           }
         }
       }

@@ -6,9 +6,10 @@
 //            Idempotent byte stores: concurrent writers store the same value, so the dedup needs no
 //            atomics.  Four independent slots per thread keep the dependent loads overlapped.
 //   tail     (the CTA that finishes marking last, found with one ticket counter)
-//     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 16 flags
-//              with one 16-byte load, a warp scan places them; the flags are cleared on the way
-//              so the next call starts from zeros.
+//     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 4 flags
+//              with one load (the replica masks and sizes of those clusters are requested in the same
+//              round trip), a warp scan places them; the flags are cleared on the way so the next call
+//              starts from zeros.
 //              With cache state attached (swarm_set_cache) the same pass drops the activated clusters
 //              that are resident (Eq. 8) and updates the activation frequencies and Eq. 6 scores.
 //     route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
@@ -40,7 +41,8 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
                const uint16_t* __restrict__ cluster_size, uint8_t* __restrict__ flags,
                unsigned* __restrict__ ticket, uint2* __restrict__ items, int32_t* __restrict__ uniq,
                uint8_t* __restrict__ queue_of, int32_t* __restrict__ n_uniq, int32_t* __restrict__ queue_load,
-               uint32_t* __restrict__ status) {
+               uint32_t* __restrict__ status, int items_cap) {
+  extern __shared__ uint2 s_items[];                     // (mask, weight << 5) in visit order, when they fit
   __shared__ int warp_cnt[kWarps];
   __shared__ int s_load[32];
   __shared__ unsigned s_classes;
@@ -50,8 +52,8 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) s_hits = 0;
+  const long long c_all = cluster_base[geo.B];           // an input table: not written by the previous kernel
   pdl_wait();                                            // the flags / the selection come from the previous kernel
-  const long long c_all = cluster_base[geo.B];
   const int C = (int)min((long long)geo.Cmax, c_all);
   unsigned err = (c_all > geo.Cmax) ? SWARM_DEV_BAD_CLUSTER : 0u;
 
@@ -109,37 +111,51 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
   SWARM_STAMP_ANY_CTA(status, 1);
 
   // ---- compact (flags are read past L1: other CTAs wrote them) -------------------------------------
+  // Every lane takes 4 flags (one word) at a time, so that up to 1024 clusters keep all 256 threads busy in a
+  // single pass; warp w owns a contiguous range of words, which keeps the ids in ascending order.
   if (tid < 32) s_load[tid] = 0;
   if (tid == 0) s_classes = 0u;
-  const int n_vec = (C + 15) / 16;                       // the flag array is padded to 16 bytes
+  const int n_vec = (C + 3) / 4;                         // the flag array is padded to 16 bytes
   const int vec_per_warp = (n_vec + kWarps - 1) / kWarps;
   const int v_lo = min(n_vec, warp * vec_per_warp), v_hi = min(n_vec, v_lo + vec_per_warp);
-  uint4* f4 = reinterpret_cast<uint4*>(flags);
+  uint32_t* f1 = reinterpret_cast<uint32_t*>(flags);
   const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
   const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
   const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
-  // pass 1: count (the common case of one 16-flag vector per lane keeps it in registers for pass 2)
+  // pass 1: count (the common case of one word per lane keeps it in registers for pass 2)
   const bool one_vec = v_hi - v_lo <= 32;
-  uint4 f_keep = make_uint4(0, 0, 0, 0);
+  uint32_t f_keep = 0u;
+  // With one word per lane the replica masks and sizes of its 4 clusters are requested together with the
+  // flags (one memory round trip instead of two dependent ones); a row that would cross the end of the
+  // tables is read entry by entry later.
+  const int v_mine = v_lo + lane;
+  const bool tables_ahead = one_vec && v_mine < v_hi && v_mine * 4 + 4 <= C;
+  uint4 mk = make_uint4(0u, 0u, 0u, 0u);
+  uint2 sz = make_uint2(0u, 0u);
+  if (tables_ahead) {
+    mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v_mine * 4));
+    sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v_mine * 4));
+  }
   int cnt = 0;
   for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
     const int v = v0 + lane;
     if (v < v_hi) {
-      const uint4 f = __ldcg(f4 + v);
+      const uint32_t f = __ldcg(f1 + v);
       f_keep = f;
-      cnt += nonzero_bytes(f.x) + nonzero_bytes(f.y) + nonzero_bytes(f.z) + nonzero_bytes(f.w);
+      cnt += nonzero_bytes(f);
       if (kCached) {                                       // activated but resident: not fetched (Eq. 8)
-        const uint32_t words[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) && cache.resident[v * 16 + j]) --cnt;
+        for (int j = 0; j < 4; ++j)
+          if (((f >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
       }
     }
   }
+  SWARM_STAMP_ANY_CTA(status, 5);
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
   if (lane == 0) warp_cnt[warp] = cnt;
   __syncthreads();
+  SWARM_STAMP_ANY_CTA(status, 6);
   int before = 0, n = 0;
   for (int w2 = 0; w2 < kWarps; ++w2) {
     if (w2 < warp) before += warp_cnt[w2];
@@ -150,28 +166,27 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
   unsigned classes = 0u;
   for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
     const int v = v0 + lane;
-    uint4 f = make_uint4(0, 0, 0, 0);
+    uint32_t f = 0u;
     if (v < v_hi) {
-      f = one_vec ? f_keep : __ldcg(f4 + v);
-      if (f.x | f.y | f.z | f.w) __stcg(f4 + v, make_uint4(0, 0, 0, 0));   // leave zeros for the next call
+      f = one_vec ? f_keep : __ldcg(f1 + v);
+      if (f) __stcg(f1 + v, 0u);                           // leave zeros for the next call
     }
-    const uint32_t words[4] = {f.x, f.y, f.z, f.w};
-    unsigned fetch_bits = 0u;                              // bit j: cluster v*16+j is activated and has to be fetched
+    unsigned fetch_bits = 0u;                              // bit j: cluster v*4+j is activated and has to be fetched
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const bool on = ((words[j >> 2] >> (8 * (j & 3))) & 0xFFu) != 0u;
+    for (int j = 0; j < 4; ++j) {
+      const bool on = ((f >> (8 * j)) & 0xFFu) != 0u;
       bool fetch = on;
       if (kCached) {
         // cache bookkeeping of Sec. 5.2 for every cluster, activated or not
-        const int c = v * 16 + j;
+        const int c = v * 4 + j;
         if (v < v_hi && c < C) {
           const bool res = cache.resident[c] != 0;
           int fr = cache.freq[c];
           if (on) ++fr; else if (res) --fr;
           if (on || res) cache.freq[c] = fr;
           if (cache.score != nullptr) {
-            const float sz = (float)cluster_size[c];
-            cache.score[c] = (float)fr * (cache.t_base + sz * cache.t_transfer) / sz;
+            const float size_f = (float)cluster_size[c];
+            cache.score[c] = (float)fr * (cache.t_base + size_f * cache.t_transfer) / size_f;
           }
           if (on && res) { fetch = false; atomicAdd(&s_hits, 1); }
         }
@@ -186,26 +201,35 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
       if (lane >= o) incl += t;
     }
     int pos = before + incl - mine;
+    SWARM_STAMP_ANY_CTA(status, 7);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
+    for (int j = 0; j < 4; ++j) {
       if ((fetch_bits >> j) & 1u) {
-        const int c = v * 16 + j, i = pos++;
+        const int c = v * 4 + j, i = pos++;
         uniq[i] = c;
-        const unsigned m = replica_mask[c];
-        const unsigned wgt = unit ? 1u : (unsigned)cluster_size[c];
+        unsigned m, size;
+        if (tables_ahead) {
+          m = (&mk.x)[j];
+          size = ((&sz.x)[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+        } else {
+          m = replica_mask[c];
+          size = cluster_size[c];
+        }
+        const unsigned wgt = unit ? 1u : size;
+        uint2 item = make_uint2(0u, 0u);                             // (0, 0): nothing left to do for the serial pass
         if (m == 0u || (m & ~valid_bits)) {
           err |= SWARM_DEV_BAD_REPLICA;
           queue_of[i] = 0xFF;
-          items[i] = make_uint2(0u, 0u);
         } else if (__popc(m) == 1 && !by_id) {
           const int qd = __ffs(m) - 1;
           queue_of[i] = (uint8_t)qd;
           atomicAdd(&s_load[qd], (int)wgt);
-          items[i] = make_uint2(0u, 0u);                             // nothing left to do for the serial pass
         } else {
           classes |= 1u << (__popc(m) - 1);
-          items[i] = make_uint2(m, wgt << 5);                        // what the serial pass needs, in visit order
+          item = make_uint2(m, wgt << 5);                            // what the serial pass needs, in visit order
         }
+        if (n <= items_cap) s_items[i] = item;                       // the serial pass then never waits on global memory
+        else items[i] = item;
       }
     }
     before += __shfl_sync(0xFFFFFFFFu, incl, 31);
@@ -226,13 +250,15 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
     for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D); ++R) {
       if (!by_id && !((todo >> (R - 1)) & 1u)) continue;
       // (mask, weight) of 32 clusters per step, fetched two steps ahead of their use
-      uint2 pre0 = lane < n ? items[lane] : make_uint2(0u, 0u);
-      uint2 pre1 = 32 + lane < n ? items[32 + lane] : make_uint2(0u, 0u);
+      const bool staged = n <= items_cap;
+      auto item_at = [&](int i) -> uint2 { return i >= n ? make_uint2(0u, 0u) : (staged ? s_items[i] : items[i]); };
+      uint2 pre0 = item_at(lane);
+      uint2 pre1 = item_at(32 + lane);
       for (int i0 = 0; i0 < n; i0 += 32) {
         const int i = i0 + lane;
         const unsigned m = pre0.x, wgt = pre0.y;
         pre0 = pre1;
-        pre1 = i + 64 < n ? items[i + 64] : make_uint2(0u, 0u);
+        pre1 = item_at(i + 64);
         const bool mine = m != 0u && (by_id || __popc(m) == R);
         const unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
         const int cnt = __popc(pending);
@@ -268,7 +294,16 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
 
 }  // namespace
 
-cudaError_t configure_resolve() { return cudaSuccess; }
+constexpr size_t kItemStageBytes = 32 * 1024;
+
+cudaError_t configure_resolve() {
+  // static + dynamic shared memory exceed the 48 KiB that needs no opt-in
+  cudaError_t e = cudaFuncSetAttribute(resolve_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kItemStageBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(resolve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kItemStageBytes);
+  return e;
+}
 
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
@@ -278,13 +313,17 @@ cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_
   const long long slots = (long long)geo.B * geo.Hq * geo.k;
   const unsigned grid =
       sel == nullptr ? 1u : (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
+  // Shared-memory stage for the serial pass's operands.  Its size also keeps the attention CTAs of the fused
+  // step (which take most of an SM's shared memory) off this CTA's SM, so the serial pass keeps the issue slots.
+  const size_t own_sm_bytes = kItemStageBytes;
+  const int items_cap = (int)(own_sm_bytes / sizeof(uint2));
   if (cache != nullptr)
-    return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), 0, st, overlap, geo, *cache, sel, n_sel,
+    return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), own_sm_bytes, st, overlap, geo, *cache, sel, n_sel,
                       page_base, page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq,
-                      queue_of, n_uniq, queue_load, status);
-  return launch_pdl(resolve_kernel<false>, dim3(grid), dim3(kThreads), 0, st, overlap, geo, swarm_cache{}, sel, n_sel,
+                      queue_of, n_uniq, queue_load, status, items_cap);
+  return launch_pdl(resolve_kernel<false>, dim3(grid), dim3(kThreads), own_sm_bytes, st, overlap, geo, swarm_cache{}, sel, n_sel,
                     page_base, page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq,
-                    queue_of, n_uniq, queue_load, status);
+                    queue_of, n_uniq, queue_load, status, items_cap);
 }
 
 }  // namespace swarm
