@@ -66,12 +66,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-// 2-D tiled TMA load: box (64 coordinates, 16 rows) at (x, row) of the tensor behind `map`.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int row, uint64_t* bar) {
+// 2-D tiled TMA load: box (64 coordinates, 16 rows) at (x, row) of the tensor behind `map`.  The pages are
+// read once per step: `policy` (evict-first) keeps them from pushing the small tables, the workspace and the
+// kernels' own instructions out of L2.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int row, uint64_t* bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(row), "r"(smem_addr(bar))
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+      "l"(map), "r"(x), "r"(row), "r"(smem_addr(bar)), "l"(policy)
       : "memory");
+}
+__device__ __forceinline__ uint64_t evict_first_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -228,6 +236,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
 
+  const uint64_t stream_policy = evict_first_policy();
   unsigned char* my_ring = ring + (size_t)warp * kStages * kSlotBytes;
   unsigned fills = 0, drains = 0;                       // units issued / consumed so far (slot = count % kStages)
   bool timed_out = false;
@@ -304,10 +313,10 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         const uint32_t dst = smem_addr(my_ring + slot * kSlotBytes);
         uint64_t* bar = &bars[warp][slot];
         mbar_expect_tx(bar, kSlotBytes);
-        tma_load_2d(dst, &mapK, 0, (int)rowK, bar);
-        tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar);
-        tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar);
-        tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar);
+        tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
+        tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar, stream_policy);
+        tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar, stream_policy);
+        tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar, stream_policy);
       }
       ++fills;
     };

@@ -224,14 +224,23 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     }
   }
   __syncthreads();
-  const int total = s_cum[geo.B];
-  const int blk_lo = (int)((long long)total * blockIdx.x / gridDim.x);
-  const int blk_hi = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
+  // The CTAs share the work in units of one KV head of one block (8 KiB), so that their byte counts differ by
+  // one unit at most; a CTA's first and last block may therefore cover only some of the block's KV heads.
+  const long long total_units = (long long)s_cum[geo.B] * kMmaConsumers;
+  const long long u_lo = total_units * blockIdx.x / gridDim.x, u_hi = total_units * (blockIdx.x + 1) / gridDim.x;
+  const int blk_lo = (int)(u_lo / kMmaConsumers);
+  const int blk_hi = u_hi > u_lo ? (int)((u_hi - 1) / kMmaConsumers) + 1 : blk_lo;
   const int n_blk = blk_hi - blk_lo;
+  const int first_head = (int)(u_lo % kMmaConsumers);                    // of block blk_lo
+  const int last_heads = u_hi > u_lo ? (int)((u_hi - 1) % kMmaConsumers) + 1 : 0;   // heads of block blk_hi - 1
 
   if (warp == kMmaConsumers) {
     // ---- producer ----
     if (lane == 0) {
+      // the summaries are read once per step: evict-first keeps them from displacing the small tables, the
+      // workspace and the kernels' own instructions in L2
+      uint64_t stream_policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
       int fb = 0;
       for (int k = 0; k < n_blk; ++k) {
         const int stage = k % kMmaStages;
@@ -245,18 +254,19 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
         while (s_cum[fb + 1] <= blk) ++fb;
         const int c = blk - s_cum[fb];
         const int tile = c / kv_groups, kvg = c % kv_groups;
-        const int n_kv = min(kMmaConsumers, geo.Hkv - kvg * kMmaConsumers);
+        const int j_lo = k == 0 ? first_head : 0;
+        const int j_hi = min(k == n_blk - 1 ? last_heads : kMmaConsumers, geo.Hkv - kvg * kMmaConsumers);
         const int page0 = (int)(page_base[fb] + (long long)tile * kMmaPages);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])),
-                     "r"((unsigned)(n_kv * kMmaHeadBytes))
+                     "r"((unsigned)(max(j_hi - j_lo, 0) * kMmaHeadBytes))
                      : "memory");
-        for (int j = 0; j < n_kv; ++j) {
+        for (int j = j_lo; j < j_hi; ++j) {
 #pragma unroll
           for (int bx = 0; bx < 4; ++bx) {
             const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + j * kMmaHeadBytes + bx * (kMmaPages * 128));
             asm volatile(
-                "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + j), "r"(page0), "r"(sm_addr(&full[stage]))
+                "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + j), "r"(page0), "r"(sm_addr(&full[stage])), "l"(stream_policy)
                 : "memory");
           }
         }
@@ -278,7 +288,8 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     const int c = blk - s_cum[b];
     const int tile_p = c / kv_groups, kvg = c % kv_groups;
     const int kvh = kvg * kMmaConsumers + warp;
-    const bool active = kvh < geo.Hkv;
+    const bool active = kvh < geo.Hkv && warp >= (k == 0 ? first_head : 0) &&
+                        warp < (k == n_blk - 1 ? last_heads : kMmaConsumers);
     const int P = pages_of(ctx_len[b], geo.S);
     const int p0 = tile_p * kMmaPages;
     {
