@@ -65,11 +65,24 @@ __device__ __forceinline__ void prefetch_tables(const Geometry& geo, const TopkE
       prefetch_l2(reinterpret_cast<const char*>(x.cluster_size) + o);
 }
 
-__device__ __forceinline__ void mark_cluster(const Geometry& geo, const TopkExtras& x, int b, int p) {
-  const long long pb = x.page_base[b], cb = x.cluster_base[b];
-  const int c = x.page2cluster[pb + p];
-  if (c < 0 || c >= x.cluster_base[b + 1] - cb || cb + c >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
-  else x.flags[cb + c] = 1;
+// Bases of request b in the page and cluster tables.  They are inputs, not results of the previous kernel, so
+// they are read before the wait on it.
+struct RequestBases {
+  long long pb, cb, cn;
+};
+__device__ __forceinline__ RequestBases load_bases(const TopkExtras& x, int b) {
+  RequestBases r{0, 0, 0};
+  if (x.flags != nullptr) {
+    r.pb = x.page_base[b];
+    r.cb = x.cluster_base[b];
+    r.cn = x.cluster_base[b + 1];
+  }
+  return r;
+}
+__device__ __forceinline__ void mark_cluster(const Geometry& geo, const TopkExtras& x, const RequestBases& rb, int p) {
+  const int c = x.page2cluster[rb.pb + p];
+  if (c < 0 || c >= rb.cn - rb.cb || rb.cb + c >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
+  else x.flags[rb.cb + c] = 1;
 }
 
 // Shared state of one radix-select run.
@@ -194,9 +207,11 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   SWARM_KERNEL_BEGIN(status, 1);
   for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
   prefetch_tables(geo, x);
+  const RequestBases rb = load_bases(x, b);
+  const int len_b = ctx_len[b];
   pdl_wait();                                               // the scores come from the previous kernel
   SWARM_STAMP(status, 1);
-  const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
+  const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
   const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
@@ -304,7 +319,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   if (x.flags != nullptr) {
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j)
-      if ((picked >> j) & 1u) mark_cluster(geo, x, b, p0 + j);
+      if ((picked >> j) & 1u) mark_cluster(geo, x, rb, p0 + j);
   }
   for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
@@ -327,8 +342,10 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   pdl_launch_dependents();
   for (int i = tid; i < kBins; i += kGenericThreads) st.hist[i] = 0;
   prefetch_tables(geo, x);
+  const RequestBases rb = load_bases(x, b);
+  const int len_b = ctx_len[b];
   pdl_wait();
-  const int P = max(0, min(pages_of(ctx_len[b], geo.S), geo.Pmax));
+  const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // see topk_regs_kernel
   const int k_sel = k_eff - (P - Pw);
@@ -397,7 +414,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
     const bool take = gt || (eq && my_eq < need_eq);
     if (take) {
       out[my_gt + min(my_eq, need_eq)] = i;
-      if (x.flags != nullptr) mark_cluster(geo, x, b, i);
+      if (x.flags != nullptr) mark_cluster(geo, x, rb, i);
     }
     const unsigned word = __ballot_sync(0xFFFFFFFFu, take);
     if (x.selmap != nullptr && lane == 0 && i0 / 8 + 4 <= x.selmap_pitch)
