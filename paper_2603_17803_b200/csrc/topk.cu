@@ -317,9 +317,18 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
     else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
   }
   if (x.flags != nullptr) {
+    // all the table reads first, then the flag stores: a byte store may alias anything, so interleaving them
+    // would make every read wait for the store before it
+    int c[ITEMS];
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j)
-      if ((picked >> j) & 1u) mark_cluster(geo, x, rb, p0 + j);
+    for (int j = 0; j < ITEMS; ++j) c[j] = ((picked >> j) & 1u) ? x.page2cluster[rb.pb + p0 + j] : 0;
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) {
+      if ((picked >> j) & 1u) {
+        if (c[j] < 0 || c[j] >= rb.cn - rb.cb || rb.cb + c[j] >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
+        else x.flags[rb.cb + c[j]] = 1;
+      }
+    }
   }
   for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
