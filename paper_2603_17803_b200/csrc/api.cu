@@ -57,7 +57,7 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);
   l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
   l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
-  l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 8);
+  l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 16);
   l.selmap = off;   off = align256(off + bh * selmap_pitch_bytes(s.max_pages_per_req));
   l.tickets = off;  off = align256(off + bh * 4);
   l.total = off;
@@ -247,7 +247,7 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
     return SWARM_ERR_INVALID_ARG;
   SWARM_TRY(launch_resolve(ctx->geo, sel, n_sel, in->page_base, in->page2cluster, in->cluster_base,
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), uniq, queue_of,
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), uniq, queue_of,
                            n_uniq, queue_load,
                            ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream), false,
                            ctx->has_cache ? &ctx->cache : nullptr));
@@ -355,7 +355,7 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
 
   SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint2>(ctx, ctx->lay.items), o->uniq,
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), o->uniq,
                            o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true,
                            ctx->has_cache ? &ctx->cache : nullptr));
   SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));

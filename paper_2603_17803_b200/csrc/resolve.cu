@@ -39,10 +39,11 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
                const int64_t* __restrict__ page_base, const int32_t* __restrict__ page2cluster,
                const int64_t* __restrict__ cluster_base, const uint32_t* __restrict__ replica_mask,
                const uint16_t* __restrict__ cluster_size, uint8_t* __restrict__ flags,
-               unsigned* __restrict__ ticket, uint2* __restrict__ items, int32_t* __restrict__ uniq,
+               unsigned* __restrict__ ticket, uint4* __restrict__ items, int32_t* __restrict__ uniq,
                uint8_t* __restrict__ queue_of, int32_t* __restrict__ n_uniq, int32_t* __restrict__ queue_load,
                uint32_t* __restrict__ status, int items_cap) {
-  extern __shared__ uint2 s_items[];                     // (mask, weight << 5) in visit order, when they fit
+  extern __shared__ uint4 s_items[];                     // (mask, weight << 5, output slot, -) of the serial pass, when they fit
+  __shared__ int2 s_seg[kWarps];                         // (start, length) of each warp's segment of the item list
   __shared__ int warp_cnt[kWarps];
   __shared__ int s_load[32];
   __shared__ unsigned s_classes;
@@ -122,56 +123,94 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
   const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
   const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
   const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
-  // pass 1: count (the common case of one word per lane keeps it in registers for pass 2)
-  const bool one_vec = v_hi - v_lo <= 32;
-  uint32_t f_keep = 0u;
-  // With one word per lane the replica masks and sizes of its 4 clusters are requested together with the
-  // flags (one memory round trip instead of two dependent ones); a row that would cross the end of the
-  // tables is read entry by entry later.
-  const int v_mine = v_lo + lane;
-  const bool tables_ahead = one_vec && v_mine < v_hi && v_mine * 4 + 4 <= C;
-  uint4 mk = make_uint4(0u, 0u, 0u, 0u);
-  uint2 sz = make_uint2(0u, 0u);
-  if (tables_ahead) {
-    mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v_mine * 4));
-    sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v_mine * 4));
-  }
-  int cnt = 0;
-  for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
-    const int v = v0 + lane;
+
+  // One word of flags with the replica masks and sizes of its 4 clusters, all requested in the same memory
+  // round trip; a row that would cross the end of the tables is read entry by entry.
+  struct Row {
+    uint32_t f;
+    uint4 mk;
+    uint2 sz;
+  };
+  auto load_row = [&](int v, bool with_flags) -> Row {
+    Row r;
+    r.f = 0u;
+    r.mk = make_uint4(0u, 0u, 0u, 0u);
+    r.sz = make_uint2(0u, 0u);
     if (v < v_hi) {
-      const uint32_t f = __ldcg(f1 + v);
-      f_keep = f;
-      cnt += nonzero_bytes(f);
-      if (kCached) {                                       // activated but resident: not fetched (Eq. 8)
+      if (with_flags) r.f = __ldcg(f1 + v);
+      if (v * 4 + 4 <= C) {
+        r.mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v * 4));
+        r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));
+      } else {
+        uint32_t* mk = &r.mk.x;
+        uint32_t* sz = &r.sz.x;
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (((f >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+        for (int j = 0; j < 4; ++j) {
+          if (v * 4 + j < C) {
+            mk[j] = replica_mask[v * 4 + j];
+            sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
+          }
+        }
+      }
+    }
+    return r;
+  };
+
+  // pass 1: count.  With one word per lane (up to 1024 clusters) the row stays in registers for pass 2.
+  const bool one_vec = v_hi - v_lo <= 32;
+  Row keep = load_row(v_lo + lane, true);
+  int cnt = 0;
+  if (one_vec) {
+    cnt = nonzero_bytes(keep.f);
+    if (kCached) {                                         // activated but resident: not fetched (Eq. 8)
+      const int v = v_lo + lane;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (((keep.f >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+    }
+  } else {
+    for (int v0 = v_lo; v0 < v_hi; v0 += 128) {            // four independent loads in flight per lane
+      uint32_t f[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u + lane;
+        f[u] = v < v_hi ? __ldcg(f1 + v) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        cnt += nonzero_bytes(f[u]);
+        if (kCached) {
+          const int v = v0 + 32 * u + lane;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (((f[u] >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+        }
       }
     }
   }
-  SWARM_STAMP_ANY_CTA(status, 5);
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
   if (lane == 0) warp_cnt[warp] = cnt;
   __syncthreads();
-  SWARM_STAMP_ANY_CTA(status, 6);
   int before = 0, n = 0;
   for (int w2 = 0; w2 < kWarps; ++w2) {
     if (w2 < warp) before += warp_cnt[w2];
     n += warp_cnt[w2];
   }
-  // pass 2: place the ids, clear the flags, and in the same go validate each cluster's replica mask, route
-  // the single-replica ones and stash what the serial pass needs
+  // pass 2: place the ids, clear the flags, validate each cluster's replica mask and route the single-replica
+  // ones.  The clusters that need the serial pass are packed, in id order, into this warp's segment of the
+  // item list, which starts at the warp's first output position (a segment cannot outgrow the warp's ids).
+  const bool staged = n <= items_cap;
+  const int seg_base = before;
+  int seg_len = 0;
   unsigned classes = 0u;
+  Row cur = keep;
   for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
     const int v = v0 + lane;
-    uint32_t f = 0u;
-    if (v < v_hi) {
-      f = one_vec ? f_keep : __ldcg(f1 + v);
-      if (f) __stcg(f1 + v, 0u);                           // leave zeros for the next call
-    }
-    unsigned fetch_bits = 0u;                              // bit j: cluster v*4+j is activated and has to be fetched
+    const Row nxt = load_row(v + 32, true);                // the next row travels while this one is processed
+    const uint32_t f = cur.f;
+    if (f) __stcg(f1 + v, 0u);                             // leave zeros for the next call
+    unsigned fetch_bits = 0u, serial_bits = 0u;            // bit j: cluster v*4+j is fetched / needs the serial pass
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const bool on = ((f >> (8 * j)) & 0xFFu) != 0u;
@@ -191,49 +230,54 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
           if (on && res) { fetch = false; atomicAdd(&s_hits, 1); }
         }
       }
+      const unsigned m = (&cur.mk.x)[j];
+      const bool valid = m != 0u && !(m & ~valid_bits);
       fetch_bits |= (fetch ? 1u : 0u) << j;
+      serial_bits |= (fetch && valid && (by_id || __popc(m) > 1) ? 1u : 0u) << j;
     }
-    const int mine = __popc(fetch_bits);
+    // one scan for both output positions: ids in the low half, serial items in the high half
+    const int mine = __popc(fetch_bits) | (__popc(serial_bits) << 16);
     int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
       if (lane >= o) incl += t;
     }
-    int pos = before + incl - mine;
-    SWARM_STAMP_ANY_CTA(status, 7);
+    int pos = before + ((incl - mine) & 0xFFFF);
+    int spos = seg_base + seg_len + ((incl - mine) >> 16);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if ((fetch_bits >> j) & 1u) {
         const int c = v * 4 + j, i = pos++;
         uniq[i] = c;
-        unsigned m, size;
-        if (tables_ahead) {
-          m = (&mk.x)[j];
-          size = ((&sz.x)[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
-        } else {
-          m = replica_mask[c];
-          size = cluster_size[c];
-        }
+        const unsigned m = (&cur.mk.x)[j];
+        const unsigned size = ((&cur.sz.x)[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
         const unsigned wgt = unit ? 1u : size;
-        uint2 item = make_uint2(0u, 0u);                             // (0, 0): nothing left to do for the serial pass
-        if (m == 0u || (m & ~valid_bits)) {
+        if ((serial_bits >> j) & 1u) {
+          classes |= 1u << (__popc(m) - 1);
+          const uint4 item = make_uint4(m, wgt << 5, (unsigned)i, 0u);   // what the serial pass needs
+          if (staged) s_items[spos] = item;                // the serial pass then never waits on global memory
+          else items[spos] = item;
+          ++spos;
+        } else if (m == 0u || (m & ~valid_bits)) {
           err |= SWARM_DEV_BAD_REPLICA;
           queue_of[i] = 0xFF;
-        } else if (__popc(m) == 1 && !by_id) {
-          const int qd = __ffs(m) - 1;
+        } else {
+          const int qd = __ffs(m) - 1;                     // a single replica: nothing to decide
           queue_of[i] = (uint8_t)qd;
           atomicAdd(&s_load[qd], (int)wgt);
-        } else {
-          classes |= 1u << (__popc(m) - 1);
-          item = make_uint2(m, wgt << 5);                            // what the serial pass needs, in visit order
         }
-        if (n <= items_cap) s_items[i] = item;                       // the serial pass then never waits on global memory
-        else items[i] = item;
       }
     }
-    before += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    before += tot & 0xFFFF;
+    seg_len += tot >> 16;
+    cur = nxt;
   }
+  if (lane == 0) s_seg[warp] = make_int2(seg_base, seg_len);
+  if (staged)                                              // in shared memory the serial pass walks one flat list:
+    for (int k = seg_base + seg_len + lane; k < before; k += 32)   // blank the rest of this warp's slots
+      s_items[k] = make_uint4(0u, 0u, 0u, 0u);
   SWARM_STAMP_ANY_CTA(status, 2);
   if (classes) atomicOr(&s_classes, classes);
   if (err) atomicOr(status, err);
@@ -241,44 +285,48 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
   SWARM_STAMP_ANY_CTA(status, 3);
 
   // ---- the ordered greedy, one warp ------------------------------------------------------------------
-  // The visit order is materialised first (32 clusters at a time, in shared memory) so that the serial
-  // loop is a plain counted loop whose operands are fetched one step ahead of the dependent chain
-  // select -> redux.min -> compare -> add.
+  // It walks the warps' segments in order, which is id order (from shared memory: all of them as one list,
+  // the unused slots blank).  32 clusters at a time are staged in shared
+  // memory so that the serial loop is a plain counted loop whose operands are fetched one step ahead of
+  // the dependent chain select -> redux.min -> compare -> add.
   if (warp == 0) {
     unsigned L = ((unsigned)s_load[lane] << 5) | (unsigned)lane;     // (load, queue id) in one comparable word
-    const unsigned todo = s_classes & ~1u;
+    const unsigned todo = by_id ? 1u : (s_classes & ~1u);
     for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D); ++R) {
       if (!by_id && !((todo >> (R - 1)) & 1u)) continue;
-      // (mask, weight) of 32 clusters per step, fetched two steps ahead of their use
-      const bool staged = n <= items_cap;
-      auto item_at = [&](int i) -> uint2 { return i >= n ? make_uint2(0u, 0u) : (staged ? s_items[i] : items[i]); };
-      uint2 pre0 = item_at(lane);
-      uint2 pre1 = item_at(32 + lane);
-      for (int i0 = 0; i0 < n; i0 += 32) {
-        const int i = i0 + lane;
-        const unsigned m = pre0.x, wgt = pre0.y;
-        pre0 = pre1;
-        pre1 = item_at(i + 64);
-        const bool mine = m != 0u && (by_id || __popc(m) == R);
-        const unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
-        const int cnt = __popc(pending);
-        if (cnt == 0) continue;
-        const int rank = __popc(pending & ((1u << lane) - 1u));
-        if (mine) { s_item_m[rank] = m; s_item_w[rank] = wgt; }
-        __syncwarp();
-        unsigned my_q = 0u;
-        unsigned mm = s_item_m[0], ww = s_item_w[0];
-        for (int r = 0; r < cnt; ++r) {
-          const unsigned mm_next = s_item_m[min(r + 1, 31)], ww_next = s_item_w[min(r + 1, 31)];
-          const unsigned key = ((mm >> lane) & 1u) ? L : 0xFFFFFFFFu;
-          const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);   // ~60 cycles per cluster end to end;
-          if (L == best) L += ww;                                      // shuffle- and ballot-based variants
-          if (rank == r) my_q = best & 31u;                            // measured slower on sm_100
-          mm = mm_next;
-          ww = ww_next;
+      for (int w2 = 0; w2 < (staged ? 1 : kWarps); ++w2) {
+        const int base = staged ? 0 : s_seg[w2].x, len = staged ? n : s_seg[w2].y;
+        // (mask, weight, output slot) of 32 clusters per step, fetched two steps ahead of their use
+        auto item_at = [&](int k) -> uint4 {
+          return k >= len ? make_uint4(0u, 0u, 0u, 0u) : (staged ? s_items[base + k] : items[base + k]);
+        };
+        uint4 pre0 = item_at(lane);
+        uint4 pre1 = item_at(32 + lane);
+        for (int k0 = 0; k0 < len; k0 += 32) {
+          const unsigned m = pre0.x, wgt = pre0.y, slot = pre0.z;
+          pre0 = pre1;
+          pre1 = item_at(k0 + 64 + lane);
+          const bool mine = m != 0u && (by_id || __popc(m) == R);
+          const unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
+          const int cnt_p = __popc(pending);
+          if (cnt_p == 0) continue;
+          const int rank = __popc(pending & ((1u << lane) - 1u));
+          if (mine) { s_item_m[rank] = m; s_item_w[rank] = wgt; }
+          __syncwarp();
+          unsigned my_q = 0u;
+          unsigned mm = s_item_m[0], ww = s_item_w[0];
+          for (int r = 0; r < cnt_p; ++r) {
+            const unsigned mm_next = s_item_m[min(r + 1, 31)], ww_next = s_item_w[min(r + 1, 31)];
+            const unsigned key = ((mm >> lane) & 1u) ? L : 0xFFFFFFFFu;
+            const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);   // ~55 cycles per cluster end to end;
+            if (L == best) L += ww;                                      // shuffle-, ballot- and register-based
+            if (rank == r) my_q = best & 31u;                            // variants measured slower on sm_100
+            mm = mm_next;
+            ww = ww_next;
+          }
+          if (mine) queue_of[slot] = (uint8_t)my_q;
+          __syncwarp();
         }
-        if (mine) queue_of[i] = (uint8_t)my_q;
-        __syncwarp();
       }
     }
     SWARM_STAMP_ANY_CTA(status, 4);
@@ -294,7 +342,7 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
 
 }  // namespace
 
-constexpr size_t kItemStageBytes = 32 * 1024;
+constexpr size_t kItemStageBytes = 96 * 1024;
 
 cudaError_t configure_resolve() {
   // static + dynamic shared memory exceed the 48 KiB that needs no opt-in
@@ -307,7 +355,7 @@ cudaError_t configure_resolve() {
 
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
+                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
                            cudaStream_t st, bool overlap, const swarm_cache* cache) {
   const long long slots = (long long)geo.B * geo.Hq * geo.k;
@@ -316,7 +364,7 @@ cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_
   // Shared-memory stage for the serial pass's operands.  Its size also keeps the attention CTAs of the fused
   // step (which take most of an SM's shared memory) off this CTA's SM, so the serial pass keeps the issue slots.
   const size_t own_sm_bytes = kItemStageBytes;
-  const int items_cap = (int)(own_sm_bytes / sizeof(uint2));
+  const int items_cap = (int)(own_sm_bytes / sizeof(uint4));
   if (cache != nullptr)
     return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), own_sm_bytes, st, overlap, geo, *cache, sel, n_sel,
                       page_base, page2cluster, cluster_base, replica_mask, cluster_size, flags_ws, ticket, items, uniq,

@@ -19,7 +19,7 @@ struct WorkspaceLayout {
   int64_t flags;         // u8  [max_clusters_total]   cluster dedup flags (zero between calls)
   int64_t part_acc;      // f32 [B*Hq][max_splits][d]  split-K partial outputs
   int64_t part_ml;       // f32 [B*Hq][max_splits][2]  split-K partial (max, sum)
-  int64_t items;         // uint2 [max_clusters_total]  (replica mask, weight) of the clusters in visit order
+  int64_t items;         // uint4 [max_clusters_total]  (replica mask, weight, output slot, -) of the serial pass
   int64_t selmap;        // u8  [B*Hq][pitch]           per-head bitmap of the selected pages
   int64_t tickets;       // u32 [B*Hq]                 arrival counters of the split merge (zero between calls)
   int64_t total;
@@ -59,7 +59,7 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
                         const uint32_t* replica_mask = nullptr, const uint16_t* cluster_size = nullptr);
 cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                            const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint2* items,
+                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
                            int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
                            cudaStream_t st, bool overlap, const swarm_cache* cache = nullptr);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
