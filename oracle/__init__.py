@@ -229,3 +229,77 @@ def step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base, repli
     k_g, v_g, n_tok = gather(kv_pool, use_sel, use_n, page_base, ctx_len, Hkv, d, S)
     out, lse = attention(q, k_g, v_g, n_tok)
     return StepResult(s64, s32, cond, sel, n_sel, uniq, queue_of, load, k_g, v_g, n_tok, out, lse)
+
+
+# ---- cluster-granular selection through the medoid index (Sec. 4.2, Tier 1 (1); Sec. 4.1) -------------------
+def medoid_rows(ksum, page_base, cluster_base, medoid_page):
+    """Index build: row c = the key summary of cluster c's medoid page (c a global cluster id)."""
+    ksum = np.asarray(ksum)
+    page_base, cluster_base = np.asarray(page_base), np.asarray(cluster_base)
+    medoid_page = np.asarray(medoid_page)
+    rows = np.zeros((int(cluster_base[-1]),) + ksum.shape[1:], dtype=ksum.dtype)
+    for b in range(len(cluster_base) - 1):
+        for c in range(int(cluster_base[b]), int(cluster_base[b + 1])):
+            rows[c] = ksum[int(page_base[b]) + int(medoid_page[c])]
+    return rows
+
+
+def expand_clusters(sel_c, n_sel_c, cluster_base, cluster_page_ptr, cluster_pages):
+    """Pages of the selected clusters of every (request, head): ascending page id, -1 padded, and their number."""
+    sel_c, n_sel_c = np.asarray(sel_c), np.asarray(n_sel_c)
+    B, Hq, _ = sel_c.shape
+    lists = [[None] * Hq for _ in range(B)]
+    width = 1
+    for b in range(B):
+        for h in range(Hq):
+            pages = set()
+            for j in range(int(n_sel_c[b, h])):
+                c = int(cluster_base[b]) + int(sel_c[b, h, j])
+                pages.update(int(p) for p in cluster_pages[int(cluster_page_ptr[c]):int(cluster_page_ptr[c + 1])])
+            lists[b][h] = sorted(pages)
+            width = max(width, len(pages))
+    sel_p = np.full((B, Hq, width), -1, dtype=np.int32)
+    n_sel_p = np.zeros((B, Hq), dtype=np.int32)
+    for b in range(B):
+        for h in range(Hq):
+            n_sel_p[b, h] = len(lists[b][h])
+            sel_p[b, h, :len(lists[b][h])] = lists[b][h]
+    return sel_p, n_sel_p
+
+
+@dataclass
+class MedoidStepResult:
+    score64: np.ndarray
+    score32: np.ndarray
+    cond: np.ndarray
+    sel_clusters: np.ndarray
+    n_sel_clusters: np.ndarray
+    sel_pages: np.ndarray
+    n_sel_pages: np.ndarray
+    uniq: np.ndarray
+    queue_of: np.ndarray
+    load: np.ndarray
+    out: np.ndarray
+    lse: np.ndarray
+
+
+def medoid_step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base, replica_mask, cluster_size,
+                cluster_page_ptr, cluster_pages, medoid_page, *, Hkv, S, k_c, D, flags=0,
+                sel_override=None) -> MedoidStepResult:
+    """The step with the medoid index: each cluster is scored by the page upper bound of its medoid page, the k_c
+    best clusters of every head are retrieved whole, and the head attends to all of their pages.  The index is a
+    context of its own whose "pages" are the clusters, so stages 1-2 are the page routines run on it."""
+    d = np.asarray(q).shape[-1]
+    cluster_base = np.asarray(cluster_base)
+    n_c = (cluster_base[1:] - cluster_base[:-1]).astype(np.int64)
+    rows = medoid_rows(ksum, page_base, cluster_base, medoid_page)
+    len_c = (n_c * S).astype(np.int32)
+    s64, s32, cond = scores(q, rows, cluster_base, len_c, Hkv, S, int(max(1, n_c.max())))
+    sel_c, n_sel_c = topk(s32, len_c, S, k_c)
+    use_c, use_n = (sel_c, n_sel_c) if sel_override is None else sel_override
+    sel_p, n_sel_p = expand_clusters(use_c, use_n, cluster_base, cluster_page_ptr, cluster_pages)
+    uniq, queue_of, load = resolve(sel_p, n_sel_p, page_base, page2cluster, cluster_base, replica_mask, cluster_size,
+                                   D, flags)
+    k_g, v_g, n_tok = gather(kv_pool, sel_p, n_sel_p, page_base, ctx_len, Hkv, d, S)
+    out, lse = attention(q, k_g, v_g, n_tok)
+    return MedoidStepResult(s64, s32, cond, sel_c, n_sel_c, sel_p, n_sel_p, uniq, queue_of, load, out, lse)

@@ -288,3 +288,31 @@ def generate(cfg: WorkloadConfig, seed: int = 0, device="cpu", layer: int = 0, s
 def bits_u16(t: torch.Tensor) -> np.ndarray:
     """Raw bits of a bf16 (or 16-bit integer) tensor as a host uint16 array (the form the oracle takes)."""
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def cluster_members(w: "Workload"):
+    """Member lists of the clusters, derived from the page -> cluster table, and one medoid page per cluster.
+
+    Returns (cluster_page_ptr int64 [C + 1], cluster_pages int32 [pages], medoid_page int32 [C]) on the workload's
+    device: members in ascending page id (local to the request), clusters by global id.  The medoid is the middle
+    member -- which member represents a cluster is decided by the offline clustering, which is not modelled here.
+    """
+    p2c = w.page2cluster.cpu().numpy()
+    page_base = w.page_base.cpu().numpy()
+    cluster_base = w.cluster_base.cpu().numpy()
+    ctx = w.ctx_len.cpu().numpy()
+    C = int(cluster_base[-1])
+    S = w.cfg.page_size
+    counts = np.zeros(C, dtype=np.int64)
+    members = []
+    for b in range(len(ctx)):
+        P = -(-int(ctx[b]) // S)
+        local = p2c[page_base[b]:page_base[b] + P].astype(np.int64)
+        order = np.argsort(local, kind="stable")            # pages grouped by cluster, ascending page id inside
+        members.append(order.astype(np.int32))
+        counts[cluster_base[b]:cluster_base[b + 1]] = np.bincount(local, minlength=int(cluster_base[b + 1] - cluster_base[b]))
+    ptr = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    pages = np.concatenate(members) if members else np.zeros(0, np.int32)
+    medoid = np.where(counts > 0, pages[np.minimum(ptr[:-1] + counts // 2, max(len(pages) - 1, 0))], 0).astype(np.int32)
+    dev = w.page2cluster.device
+    return (torch.from_numpy(ptr).to(dev), torch.from_numpy(pages).to(dev), torch.from_numpy(medoid).to(dev))

@@ -524,3 +524,87 @@ def test_topk_local_window_is_the_last_pages_plus_the_best_of_the_rest():
         assert n[0, 0] == k_eff and list(sel[0, 0, :k_eff]) == want
     with pytest.raises(ValueError):
         oracle.topk(sc, [P], 1, 3, window=4)
+
+
+# ------------------------------------------------------------------------------- medoid index (cluster mode)
+
+def test_medoid_step_with_one_page_clusters_is_the_page_step():
+    """Clusters of one page each, each its own medoid: cluster-granular selection must reduce to page selection."""
+    rng = np.random.default_rng(21)
+    pages = (9, 6)
+    q, pool, ksum, page_base, ctx_len = rand_case(rng, pages=pages, ctx=[9 * 4 - 1, 6 * 4])
+    n = int(page_base[-1])
+    page2cluster = np.concatenate([np.arange(p) for p in pages]).astype(np.int32)
+    cluster_base = page_base.copy()
+    mask = rng.integers(1, 8, size=n).astype(np.uint32)
+    size = np.ones(n, dtype=np.uint16)
+    ptr = np.arange(n + 1, dtype=np.int64)
+    r_page = oracle.step(q, ksum, pool, page_base, ctx_len, page2cluster, cluster_base, mask, size, Hkv=2, S=4, k=3,
+                         D=3, Pmax=9)
+    r_med = oracle.medoid_step(q, ksum, pool, page_base, ctx_len, page2cluster, cluster_base, mask, size, ptr,
+                               page2cluster, page2cluster, Hkv=2, S=4, k_c=3, D=3)
+    assert np.array_equal(r_med.sel_clusters, r_page.sel) and np.array_equal(r_med.n_sel_clusters, r_page.n_sel)
+    assert np.array_equal(r_med.sel_pages[..., :3], r_page.sel)
+    assert np.array_equal(r_med.uniq, r_page.uniq) and np.array_equal(r_med.queue_of, r_page.queue_of)
+    assert np.array_equal(r_med.load, r_page.load)
+    assert np.array_equal(r_med.out, r_page.out) and np.array_equal(r_med.lse, r_page.lse)
+
+
+def test_medoid_step_scores_medoids_and_attends_whole_clusters():
+    from paper_2603_17803_b200 import workloads as W
+    cfg = W.scaled(W.CONFIGS["c5_skewed"], batch=3, ctx_range=(300, 900), top_k=8, n_topics=6)
+    w = W.generate(cfg, seed=5)
+    ptr, members, medoid = (t.numpy() for t in W.cluster_members(w))
+    u = W.bits_u16
+    pb, cl, cb = w.page_base.numpy(), w.ctx_len.numpy(), w.cluster_base.numpy()
+    p2c = w.page2cluster.numpy()
+    mask = w.cluster_replica_mask.numpy().view(np.uint32)
+    size = w.cluster_size.numpy().view(np.uint16)
+    S, Hq = cfg.page_size, cfg.n_q_heads
+    # the member lists are the inverse of the page -> cluster table, and each medoid is a member
+    for b in range(cfg.batch):
+        P = -(-int(cl[b]) // S)
+        seen = []
+        for c in range(int(cb[b]), int(cb[b + 1])):
+            mem = members[ptr[c]:ptr[c + 1]]
+            assert np.all(np.diff(mem) > 0) and np.all(p2c[pb[b] + mem] == c - cb[b])
+            assert len(mem) == 0 or medoid[c] in mem
+            seen += mem.tolist()
+        assert sorted(seen) == list(range(P))
+    ksum = oracle.build_summaries(u(w.kv_pool), pb, cl, cfg.n_kv_heads, cfg.head_dim, S)
+    k_c = 3
+    r = oracle.medoid_step(u(w.q), ksum, u(w.kv_pool), pb, cl, p2c, cb, mask, size, ptr, members, medoid,
+                           Hkv=cfg.n_kv_heads, S=S, k_c=k_c, D=cfg.n_queues)
+    page_s64, page_s32, _ = oracle.scores(u(w.q), ksum, pb, cl, cfg.n_kv_heads, S, cfg.max_pages())
+    need = set()
+    for b in range(cfg.batch):
+        n_c = int(cb[b + 1] - cb[b])
+        for h in range(Hq):
+            # a cluster's score is the page score of its medoid; the selection is the exhaustive top-k of those
+            want_scores = page_s32[b, h, medoid[cb[b]:cb[b + 1]]]
+            assert np.array_equal(r.score32[b, h, :n_c], want_scores)
+            want = brute_topk(want_scores, k_c)
+            n = int(r.n_sel_clusters[b, h])
+            assert n == min(k_c, n_c) and list(r.sel_clusters[b, h, :n]) == want
+            # all pages of the selected clusters, nothing else
+            pages = sorted(p for c in want for p in members[ptr[cb[b] + c]:ptr[cb[b] + c + 1]].tolist())
+            assert list(r.sel_pages[b, h, :r.n_sel_pages[b, h]]) == pages
+            assert r.n_sel_pages[b, h] == int(size[cb[b] + np.array(want)].sum())
+            need.update(int(cb[b]) + c for c in want)
+    assert sorted(need) == list(r.uniq)
+    replay_check(r.uniq, r.queue_of, r.load, mask, size, cfg.n_queues, 0)
+    # attention is Eq. 1 over exactly those pages: recompute one head from the pool in numpy
+    b, h = 1, 5
+    kvh = h // (Hq // cfg.n_kv_heads)
+    pool = W.bits_u16(w.kv_pool)
+    f = lambda bits: (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    ks, vs = [], []
+    P = -(-int(cl[b]) // S)
+    for p in r.sel_pages[b, h, :r.n_sel_pages[b, h]]:
+        valid = S if p < P - 1 else int(cl[b]) - S * (P - 1)
+        ks.append(f(pool[pb[b] + p, kvh, 0, :valid]))
+        vs.append(f(pool[pb[b] + p, kvh, 1, :valid]))
+    K, V = np.concatenate(ks), np.concatenate(vs)
+    logits = K @ f(u(w.q)[b, h]) / np.sqrt(cfg.head_dim)
+    pr = np.exp(logits - logits.max())
+    assert np.allclose(r.out[b, h], (pr / pr.sum()) @ V, rtol=1e-9, atol=1e-9)
