@@ -115,6 +115,19 @@ typedef struct swarm_cache {
   float t_transfer;        /* T_transfer: transfer cost per entry (page)                                       */
 } swarm_cache;
 
+/* Medoid index for cluster-granular selection (Sec. 4.2, Tier 1 (1): the medoid of each cluster is its index
+ * entry and is scored against the query to decide whether the cluster is retrieved).  Device pointers.
+ * Clusters carry their global id (cluster_base[b] + local id), as in the other cluster tables. */
+typedef struct swarm_medoid_index {
+  const void* medoid_ksum;          /* bf16 [max_clusters_total][Hkv][2][d]: key summary (min, max) of each cluster's */
+                                    /* medoid page, written by swarm_build_medoid_index                               */
+  const int64_t* cluster_page_ptr;  /* [n_clusters + 1] start of each cluster's members in cluster_pages               */
+  const int32_t* cluster_pages;     /* member pages of the clusters, ids local to the request                          */
+  int32_t top_k_clusters;           /* k_c clusters kept per query head                                                */
+  int32_t max_clusters_per_req;     /* upper bound on the clusters of one request (<= max_pages_per_req); row pitch    */
+                                    /* of the cluster scores                                                           */
+} swarm_medoid_index;
+
 /* Lifetime.  swarm_create validates the shape and allocates only host memory plus one auxiliary
  * CUDA stream and two events (used to run cluster resolution beside attention inside swarm_step).
  * The CUDA device current at creation must stay current for every later call with this ctx. */
@@ -226,6 +239,26 @@ int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g
  * four separate calls exactly; out / lse agree within rounding.  The call can be captured into a
  * CUDA graph by the caller (stream capture). */
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);
+
+/* Index build for swarm_step_medoid (not part of a decode step): copies, for every cluster, the key summary of
+ * its medoid page medoid_page[cluster] (page id local to the request) into row `cluster` of medoid_ksum_out
+ * (bf16 [max_clusters_total][Hkv][2][d]).  Reads inputs->ksum, page_base, cluster_base.  Which member is the
+ * medoid is decided offline (Algorithm 1) and is an input here. */
+int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* medoid_page,
+                                 void* medoid_ksum_out, void* stream);
+
+/* The decode step with the paper's own selector (Sec. 4.2 Tier 1 (1), Sec. 4.1): clusters, not pages, are
+ * scored and retrieved.
+ *   score[b][h][c] = the page upper bound of swarm_select evaluated on the medoid page of cluster c
+ *   sel[b][h][:]   = the min(k_c, C_b) clusters of largest score (ties to the lower id), ascending, ids local
+ *                    to the request, -1 padded; n_sel their number           (outputs->sel is [B][Hq][k_c])
+ *   uniq, queue_of, n_uniq, queue_load: as in swarm_step for the union of the selected clusters
+ *   out, lse: Eq. 1 of every head over ALL pages of its selected clusters (clusters are the retrieval unit)
+ * outputs->scores (optional) is [B][Hq][max_clusters_per_req]; k_out, v_out and n_tok must be NULL.
+ * A member page outside the request sets SWARM_DEV_BAD_PAGE and is skipped.  The local window of the shape
+ * is not applied.  Page bitmaps longer than 160 KiB per head (1.3 M pages) are SWARM_ERR_UNSUPPORTED. */
+int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_medoid_index* index,
+                          const swarm_outputs* outputs, void* stream);
 
 /* End-to-end convenience for callers holding the per-step data in HOST memory (pinned memory
  * recommended): copies q_host (bf16 [B][Hq][d]) into the ctx's staging area, runs swarm_step with

@@ -27,6 +27,7 @@ EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
     "swarm_set_attn_splits", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
+    "swarm_build_medoid_index", "swarm_step_medoid",
 )
 
 
@@ -97,6 +98,12 @@ def _check(rc: int, what: str, ctx=None):
     if rc != OK:
         cuda = load_library().swarm_last_cuda_error(ctx) if (ctx is not None and rc == ERR_CUDA) else 0
         raise SwarmError(rc, what, cuda)
+
+
+class swarm_medoid_index(ctypes.Structure):
+    _fields_ = [("medoid_ksum", ctypes.c_void_p), ("cluster_page_ptr", ctypes.c_void_p),
+                ("cluster_pages", ctypes.c_void_p), ("top_k_clusters", ctypes.c_int32),
+                ("max_clusters_per_req", ctypes.c_int32)]
 
 
 def make_shape(*, batch, n_q_heads, n_kv_heads, page_size, top_k, n_queues, max_pages_per_req, max_clusters_total,
@@ -216,6 +223,25 @@ def swarm_sparse_attn_static(q, k_g, v_g, n_tok, *, batch, n_q_heads, top_k, pag
 def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:
     _check(load_library().swarm_step(ctx, ctypes.byref(inputs), ctypes.byref(outputs), _stream(stream)),
            "swarm_step", ctx)
+
+
+def make_medoid_index(*, medoid_ksum, cluster_page_ptr, cluster_pages, top_k_clusters,
+                      max_clusters_per_req) -> swarm_medoid_index:
+    return swarm_medoid_index(_ptr(medoid_ksum, "medoid_ksum"), _ptr(cluster_page_ptr, "cluster_page_ptr"),
+                              _ptr(cluster_pages, "cluster_pages"), top_k_clusters, max_clusters_per_req)
+
+
+def swarm_build_medoid_index(ctx, inputs: swarm_inputs, medoid_page: torch.Tensor, medoid_ksum_out: torch.Tensor,
+                             stream=None) -> None:
+    _check(load_library().swarm_build_medoid_index(ctx, ctypes.byref(inputs), _ptr(medoid_page, "medoid_page"),
+                                                   _ptr(medoid_ksum_out, "medoid_ksum_out"), _stream(stream)),
+           "swarm_build_medoid_index", ctx)
+
+
+def swarm_step_medoid(ctx, inputs: swarm_inputs, index: swarm_medoid_index, outputs: swarm_outputs,
+                      stream=None) -> None:
+    _check(load_library().swarm_step_medoid(ctx, ctypes.byref(inputs), ctypes.byref(index), ctypes.byref(outputs),
+                                            _stream(stream)), "swarm_step_medoid", ctx)
 
 
 def swarm_step_host(ctx, inputs: swarm_inputs, outputs: swarm_outputs, q_host, out_host=None, lse_host=None,

@@ -147,6 +147,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   if (e == cudaSuccess) e = configure_topk();
   if (e == cudaSuccess) e = configure_resolve();
   if (e == cudaSuccess) e = configure_attention();
+  if (e == cudaSuccess) e = configure_medoid();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
@@ -394,6 +395,67 @@ struct HostStepKey {
 }  // namespace
 
 static_assert(sizeof(HostStepKey) <= 256, "host_key too small");
+
+int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* medoid_page,
+                                 void* medoid_ksum_out, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (in == nullptr || bad(in->ksum) || bad(in->page_base) || bad(in->cluster_base) || bad(medoid_page) ||
+      bad(medoid_ksum_out))
+    return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_medoid_rows(ctx->geo, static_cast<const uint16_t*>(in->ksum), in->page_base, in->cluster_base,
+                               medoid_page, static_cast<uint16_t*>(medoid_ksum_out),
+                               ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  return SWARM_OK;
+}
+
+int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_medoid_index* idx,
+                          const swarm_outputs* o, void* stream) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (in == nullptr || bad(in->q) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || idx == nullptr ||
+      bad(idx->medoid_ksum) || bad(idx->cluster_page_ptr) || bad(idx->cluster_pages) || o == nullptr || bad(o->sel) ||
+      bad(o->n_sel) || bad(o->uniq) || bad(o->queue_of) || bad(o->n_uniq) || bad(o->queue_load) || bad(o->out) ||
+      bad(o->lse) || (o->scores && !aligned16(o->scores)) || o->k_out != nullptr || o->v_out != nullptr ||
+      o->n_tok != nullptr || idx->top_k_clusters < 1 || idx->max_clusters_per_req < 1 ||
+      idx->max_clusters_per_req > ctx->geo.Pmax)
+    return SWARM_ERR_INVALID_ARG;
+  if (selmap_pitch_bytes(ctx->geo.Pmax) > kMaxExpandRowBytes ||
+      (int64_t)ctx->geo.B * ctx->geo.Hq * idx->top_k_clusters >= (int64_t(1) << 31))
+    return SWARM_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* status = ws_ptr<uint32_t>(ctx, ctx->lay.status);
+  float* sc = o->scores ? o->scores : ws_ptr<float>(ctx, ctx->lay.scores);
+  int32_t* len_c = ws_ptr<int32_t>(ctx, ctx->lay.n_tok);   // clusters of each request x page size
+
+  // the page kernels, run over the index: one "page" per cluster, requests laid out like cluster_base
+  Geometry gc = ctx->geo;
+  gc.Pmax = idx->max_clusters_per_req;
+  gc.k = idx->top_k_clusters;
+  gc.W = 0;
+  gc.n_pool_pages = ctx->geo.Cmax;
+  SWARM_TRY(launch_cluster_len(ctx->geo, in->cluster_base, len_c, st));
+  SWARM_TRY(launch_page_score(gc, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(idx->medoid_ksum),
+                              in->cluster_base, len_c, sc, status, st));
+  SWARM_TRY(launch_topk(gc, sc, len_c, o->sel, o->n_sel, status, st, true));
+  // selected clusters -> page bitmaps per head (for attention) and cluster flags (for the resolve kernel)
+  SWARM_TRY(launch_expand_clusters(ctx->geo, idx->top_k_clusters, o->sel, o->n_sel, in->cluster_base,
+                                   idx->cluster_page_ptr, idx->cluster_pages, in->ctx_len,
+                                   ws_ptr<uint8_t>(ctx, ctx->lay.selmap), ws_ptr<uint8_t>(ctx, ctx->lay.flags), status, st,
+                                   true));
+  SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
+  SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+  const AttnArgs a = paged_args(ctx, in, o->out, o->lse);
+  SWARM_TRY(launch_attention(ctx->geo, a, status, ctx->side, /*overlap=*/false));
+  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
+  SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), o->uniq,
+                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true,
+                           ctx->has_cache ? &ctx->cache : nullptr));
+  SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  return SWARM_OK;
+}
 
 int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
                         float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,

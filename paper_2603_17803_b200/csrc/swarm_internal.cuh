@@ -42,6 +42,7 @@ cudaError_t configure_score();
 cudaError_t configure_topk();
 cudaError_t configure_resolve();
 cudaError_t configure_attention();
+cudaError_t configure_medoid();
 
 // ---- kernel launchers (each returns cudaGetLastError() after the launch) ----------------------
 cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool, const int64_t* page_base,
@@ -90,6 +91,17 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
 int attention_groups(const Geometry& geo, bool paged);
 cudaError_t launch_selmap_from_sel(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, uint8_t* selmap,
                                    cudaStream_t st);
+
+// Medoid index (cluster-granular selection): see medoid.cu.
+constexpr int kMaxExpandRowBytes = 160 * 1024;            // longest per-head page bitmap the expansion assembles in shared memory
+cudaError_t launch_medoid_rows(const Geometry& geo, const uint16_t* ksum, const int64_t* page_base,
+                               const int64_t* cluster_base, const int32_t* medoid_page, uint16_t* medoid_ksum,
+                               uint32_t* status, cudaStream_t st);
+cudaError_t launch_cluster_len(const Geometry& geo, const int64_t* cluster_base, int32_t* len, cudaStream_t st);
+cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* sel_c, const int32_t* n_sel_c,
+                                   const int64_t* cluster_base, const int64_t* cluster_page_ptr,
+                                   const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
+                                   uint32_t* status, cudaStream_t st, bool overlap);
 
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -111,6 +111,33 @@ class Session:
         B.swarm_step_host(self.ctx, self.inputs, self.outputs, q_host, out_host, lse_host, n_uniq_host,
                           queue_load_host, stream)
 
+    def enable_medoid_index(self, top_k_clusters: int, keep_scores: bool = False) -> None:
+        """Builds the medoid index of the workload's clusters and the outputs of step_medoid()."""
+        from .workloads import cluster_members
+        w, cfg, dev = self.w, self.cfg, self.device
+        self.cluster_page_ptr, self.cluster_pages, self.medoid_page = cluster_members(w)
+        n_c = max(1, w.n_clusters)
+        per_req = (w.cluster_base[1:] - w.cluster_base[:-1]).max().item()
+        self.max_clusters_per_req = max(1, int(per_req))
+        self.medoid_ksum = torch.empty((n_c, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+        B.swarm_build_medoid_index(self.ctx, self.inputs, self.medoid_page, self.medoid_ksum)
+        self.medoid_index = B.make_medoid_index(medoid_ksum=self.medoid_ksum, cluster_page_ptr=self.cluster_page_ptr,
+                                                cluster_pages=self.cluster_pages, top_k_clusters=top_k_clusters,
+                                                max_clusters_per_req=self.max_clusters_per_req)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.top_k_clusters = top_k_clusters
+        self.sel_clusters = torch.empty((cfg.batch, cfg.n_q_heads, top_k_clusters), **i32)
+        self.n_sel_clusters = torch.empty((cfg.batch, cfg.n_q_heads), **i32)
+        self.cluster_scores = torch.full((cfg.batch, cfg.n_q_heads, self.max_clusters_per_req), float("-inf"),
+                                         dtype=torch.float32, device=dev) if keep_scores else None
+        o = self.o
+        self.medoid_outputs = B.make_outputs(scores=self.cluster_scores, sel=self.sel_clusters,
+                                             n_sel=self.n_sel_clusters, uniq=o.uniq, queue_of=o.queue_of,
+                                             n_uniq=o.n_uniq, queue_load=o.queue_load, out=o.out, lse=o.lse)
+
+    def step_medoid(self, stream=None):
+        B.swarm_step_medoid(self.ctx, self.inputs, self.medoid_index, self.medoid_outputs, stream)
+
     def status(self) -> int:
         return B.swarm_device_status(self.ctx)
 

@@ -442,3 +442,88 @@ def test_selection_at_every_list_length(pages, window):
     assert np.array_equal(sess.o.sel.cpu().numpy(), want)
     parity.check_step(w, sess, requests=[1], heads=[1])
     sess.close()
+
+
+# ---- medoid index (Sec. 4.2 Tier 1 (1)): clusters are scored by their medoid page and retrieved whole -------
+def check_medoid_step(w, sess, k_c, flags=0):
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    cfg = w.cfg
+    tabs = parity.host_tables(w)
+    ptr, members, medoid = (t.cpu().numpy() for t in (sess.cluster_page_ptr, sess.cluster_pages, sess.medoid_page))
+    ksum = W.bits_u16(sess.ksum)
+    rows_gpu = W.bits_u16(sess.medoid_ksum)
+    rows_ref = oracle.medoid_rows(ksum, tabs["page_base"], tabs["cluster_base"], medoid)
+    assert np.array_equal(rows_gpu[: len(rows_ref)], rows_ref), "medoid index rows differ"
+    sel_c, n_sel_c = sess.sel_clusters.cpu().numpy(), sess.n_sel_clusters.cpu().numpy()
+    r = oracle.medoid_step(W.bits_u16(w.q), ksum, W.bits_u16(w.kv_pool), tabs["page_base"], tabs["ctx_len"],
+                           tabs["page2cluster"], tabs["cluster_base"], tabs["replica_mask"], tabs["cluster_size"],
+                           ptr, members, medoid, Hkv=cfg.n_kv_heads, S=cfg.page_size, k_c=k_c, D=cfg.n_queues,
+                           flags=flags, sel_override=(sel_c, n_sel_c))
+    cb = tabs["cluster_base"]
+    exact = 0
+    for b in range(cfg.batch):
+        n_c = int(cb[b + 1] - cb[b])
+        if sess.cluster_scores is not None:
+            sc = sess.cluster_scores[b].cpu().numpy()
+            parity.check_scores(sc, r.score64[b], r.cond[b], n_c)
+            on_gpu_scores, _ = oracle.topk(sc[None, :, :n_c], np.array([n_c * cfg.page_size], np.int32),
+                                           cfg.page_size, k_c)
+            assert np.array_equal(on_gpu_scores[0], sel_c[b]), "not the exact top-k of the GPU's own cluster scores"
+        for h in range(cfg.n_q_heads):
+            parity.check_selection(sel_c[b, h], int(n_sel_c[b, h]), r.score64[b, h], n_c, k_c)
+            exact += int(np.array_equal(sel_c[b, h], r.sel_clusters[b, h]))
+    o = sess.o
+    n = int(o.n_uniq.cpu().numpy()[0])
+    assert n == len(r.uniq) and np.array_equal(o.uniq.cpu().numpy()[:n], r.uniq)
+    assert np.array_equal(o.queue_of.cpu().numpy()[:n], r.queue_of)
+    assert np.array_equal(o.queue_load.cpu().numpy()[: cfg.n_queues], r.load)
+    parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), r.out, r.lse)
+    return exact
+
+
+@pytest.mark.parametrize("name,k_c", [("c1_small", 6), ("c2_small", 12), ("c3_small", 5), ("c4_small", 9),
+                                      ("c5_small", 4), ("k_exceeds_pages", 7)])
+def test_medoid_step_matches_oracle(name, k_c):
+    w = W.generate(CASES[name], seed=37, device=DEV)
+    sess = Session(w)
+    sess.enable_medoid_index(k_c, keep_scores=True)
+    sess.step_medoid()
+    exact = check_medoid_step(w, sess, k_c)
+    assert exact >= 0.9 * w.cfg.batch * w.cfg.n_q_heads
+    # the page step still works on the same session afterwards, and the medoid step again after it
+    sess.step()
+    torch.cuda.synchronize()
+    first = sess.sel_clusters.clone()
+    sess.step_medoid()
+    torch.cuda.synchronize()
+    assert torch.equal(first, sess.sel_clusters)
+    check_medoid_step(w, sess, k_c)
+    sess.close()
+
+
+def test_medoid_step_rejects_bad_arguments_and_flags_bad_members():
+    w = W.generate(CASES["c3_small"], seed=41, device=DEV)
+    sess = Session(w, keep_gathered=True)
+    sess.enable_medoid_index(4)
+    with pytest.raises(B.SwarmError):                       # gathered outputs are not part of this step
+        B.swarm_step_medoid(sess.ctx, sess.inputs, sess.medoid_index, sess.outputs)
+    bad = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=sess.cluster_page_ptr,
+                              cluster_pages=sess.cluster_pages, top_k_clusters=0,
+                              max_clusters_per_req=sess.max_clusters_per_req)
+    with pytest.raises(B.SwarmError):
+        B.swarm_step_medoid(sess.ctx, sess.inputs, bad, sess.medoid_outputs)
+    sess.cluster_pages.fill_(1 << 20)                       # members outside every request: flagged, never followed
+    sess.step_medoid()
+    torch.cuda.synchronize()
+    assert sess.status() & B.DEV_BAD_PAGE
+    sess.close()
+
+
+def test_medoid_step_full_size_c2():
+    w = W.generate(W.CONFIGS["c2_128k"], seed=43, device=DEV)
+    sess = Session(w)
+    sess.enable_medoid_index(32, keep_scores=True)          # 32 clusters of 8 pages: the page step's 256 pages per head
+    sess.step_medoid()
+    check_medoid_step(w, sess, 32)
+    sess.close()
