@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_kernel launch at the default workload (c2_128k),
 # from the ncu capture summarised in profiles/; reported only for that workload.
-ATTN_TRAFFIC_BYTES_NCU = 33_062_400 + 7_424   # profiles/launch_list_c2_128k.md: dram read + write of attn_kernel<16,paged>
+ATTN_TRAFFIC_BYTES_NCU = 33_072_128 + 12_544   # profiles/launch_list_c2_128k.md: dram read + write of attn_kernel<16,paged>
 
 
 def parse_args():
