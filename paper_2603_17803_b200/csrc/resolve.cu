@@ -324,13 +324,25 @@ resolve_kernel(Geometry geo, swarm_cache cache, const int32_t* __restrict__ sel,
             mm = mm_next;
             ww = ww_next;
           }
-          if (mine) queue_of[slot] = (uint8_t)my_q;
+          // From shared memory the choice goes back into the item and is written out after the pass: a global
+          // store issued while the attention kernel starts or retires was measured to hold this warp for 2 us.
+          if (mine) {
+            if (staged) s_items[base + k0 + lane].w = my_q;
+            else queue_of[slot] = (uint8_t)my_q;
+          }
           __syncwarp();
         }
       }
     }
     SWARM_STAMP_ANY_CTA(status, 4);
     SWARM_KERNEL_END(status, 3);
+    if (staged) {
+      __syncwarp();
+      for (int k = lane; k < n; k += 32) {
+        const uint4 item = s_items[k];
+        if (item.x != 0u) queue_of[item.z] = (uint8_t)item.w;
+      }
+    }
     if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
     if (lane == 0) {
       *n_uniq = n;
