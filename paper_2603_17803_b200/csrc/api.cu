@@ -64,12 +64,12 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   return l;
 }
 
-int pick_splits(const swarm_ctx* ctx, bool paged) {
+int pick_splits(const swarm_ctx* ctx, bool paged, bool fused = false) {
   // About 1 CTA of 8 warps per SM on 148 SMs (what the shared-memory rings allow), at most kMaxSplits; for gathered
-  // buffers at least 4 pages per split.
+  // buffers at least 4 pages per split.  Inside the fused step one SM is left for the resolution CTA.
   if (ctx->user_splits > 0) return ctx->user_splits;
   const int64_t groups = attention_groups(ctx->geo, paged);
-  int64_t n = 148 / groups;
+  int64_t n = (fused ? 147 : 148) / groups;
   if (!paged) n = std::min<int64_t>(n, std::max(1, ctx->geo.k / 4));
   n = std::min<int64_t>(n, kMaxSplits);
   return (int)std::max<int64_t>(n, 1);
@@ -107,6 +107,16 @@ bool resolve_inputs_ok(const swarm_inputs* in) {
 }
 bool pool_inputs_ok(const swarm_inputs* in) {
   return in && !bad(in->kv_pool) && !bad(in->page_base) && !bad(in->ctx_len);
+}
+
+// Arguments of the cluster-resolution body; sel == nullptr when the flags were set by the selection kernel.
+ResolveArgs step_resolve_args(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
+                              int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load) {
+  return make_resolve_args(ctx->geo, sel, n_sel, in->page_base, in->page2cluster, in->cluster_base,
+                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
+                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), uniq, queue_of,
+                           n_uniq, queue_load, ws_ptr<uint32_t>(ctx, ctx->lay.status),
+                           ctx->has_cache ? &ctx->cache : nullptr);
 }
 
 }  // namespace
@@ -246,12 +256,7 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
   if (!resolve_inputs_ok(in) || bad(sel) || bad(n_sel) || bad(uniq) || bad(queue_of) || bad(n_uniq) ||
       bad(queue_load))
     return SWARM_ERR_INVALID_ARG;
-  SWARM_TRY(launch_resolve(ctx->geo, sel, n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), uniq, queue_of,
-                           n_uniq, queue_load,
-                           ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream), false,
-                           ctx->has_cache ? &ctx->cache : nullptr));
+  SWARM_TRY(launch_resolve(step_resolve_args(ctx, in, sel, n_sel, uniq, queue_of, n_uniq, queue_load), static_cast<cudaStream_t>(stream), false));
   return SWARM_OK;
 }
 
@@ -341,25 +346,15 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
                         ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
                         ws_ptr<uint8_t>(ctx, ctx->lay.flags), in->cluster_replica_mask, in->cluster_size));
 
-  // fork: cluster resolution and attention both need only the selection.  Resolution is the longer of
-  // the two (its greedy pass is serial), so it stays on the caller's stream right behind the selection
-  // kernel (programmatic dependent launch) and attention takes the auxiliary stream.
-  SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
-  SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+  // Cluster resolution and attention both need only the selection: one launch runs them side by side, the
+  // attention CTAs plus one CTA for the resolution (whose serial pass is the longest item of the step).
   if (o->k_out != nullptr)
     SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
-                            static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status,
-                            ctx->side));
-  const AttnArgs a = paged_args(ctx, in, o->out, o->lse);
-  SWARM_TRY(launch_attention(ctx->geo, a, status, ctx->side, /*overlap=*/false));
-  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
-
-  SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), o->uniq,
-                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true,
-                           ctx->has_cache ? &ctx->cache : nullptr));
-  SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
+                            static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
+  AttnArgs a = paged_args(ctx, in, o->out, o->lse);
+  a.n_splits = pick_splits(ctx, true, /*fused=*/true);
+  const ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, &rs));
   return SWARM_OK;
 }
 
@@ -443,17 +438,10 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
                                    idx->cluster_page_ptr, idx->cluster_pages, in->ctx_len,
                                    ws_ptr<uint8_t>(ctx, ctx->lay.selmap), ws_ptr<uint8_t>(ctx, ctx->lay.flags), status, st,
                                    true));
-  SWARM_TRY(cudaEventRecord(ctx->ev_fork, st));
-  SWARM_TRY(cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
-  const AttnArgs a = paged_args(ctx, in, o->out, o->lse);
-  SWARM_TRY(launch_attention(ctx->geo, a, status, ctx->side, /*overlap=*/false));
-  SWARM_TRY(cudaEventRecord(ctx->ev_join, ctx->side));
-  SWARM_TRY(launch_resolve(ctx->geo, /*sel=*/nullptr, o->n_sel, in->page_base, in->page2cluster, in->cluster_base,
-                           in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
-                           ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), o->uniq,
-                           o->queue_of, o->n_uniq, o->queue_load, status, st, /*overlap=*/true,
-                           ctx->has_cache ? &ctx->cache : nullptr));
-  SWARM_TRY(cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  AttnArgs a = paged_args(ctx, in, o->out, o->lse);
+  a.n_splits = pick_splits(ctx, true, /*fused=*/true);
+  const ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, &rs));
   return SWARM_OK;
 }
 

@@ -29,6 +29,7 @@
 #include <cuda_bf16.h>
 
 #include "swarm_internal.cuh"
+#include "resolve_body.cuh"
 
 namespace swarm {
 namespace {
@@ -114,10 +115,21 @@ __device__ __forceinline__ uint32_t tile_offset(int t, int chunk) {
   return (uint32_t)((chunk >> 3) * kBoxBytes + t * 128 + (((chunk & 7) ^ (t & 7)) << 4));
 }
 
-template <int S, bool kPaged>
+// kFused != 0 (fused step only): CTA 0 of the grid does not attend; it runs cluster resolution (stage 3) beside
+// the attention CTAs -- 1: plain, 2: with cache state.  As a kernel of its own on a second stream the serial
+// pass stalled for about 2 us each time the attention kernel started or retired; as one more CTA of the same
+// grid it does not, and the step needs neither the second stream nor its two events.
+template <int S, bool kPaged, int kFused>
 __global__ void __launch_bounds__(kAttnWarps * 32, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Geometry geo,
-            AttnArgs a, uint32_t* __restrict__ status) {
+            AttnArgs a, uint32_t* __restrict__ status, const __grid_constant__ ResolveArgs rs) {
+  static_assert(kFused == 0 || kPaged, "cluster resolution rides with the paged kernel only");
+  static_assert(resolve_detail::kThreads == kAttnWarps * 32, "the resolution body runs in a CTA of this kernel");
+  if (kFused != 0 && blockIdx.x == 0) {
+    resolve_detail::resolve_body<kFused == 2>(rs, 0, 1);
+    return;
+  }
+  const int cta = (int)blockIdx.x - (kFused != 0 ? 1 : 0);
   constexpr int SB = S / kUnitTokens;                   // 16-token units per page
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
@@ -128,7 +140,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
 
   // ---- which (request, heads, page range) --------------------------------------------------------
-  const int split = blockIdx.x % a.n_splits, grp = blockIdx.x / a.n_splits;
+  const int split = cta % a.n_splits, grp = cta / a.n_splits;
   int b, kvh = 0, bh0, G;
   if (kPaged) {
     const int tiles = (geo.g + 7) / 8;
@@ -602,19 +614,36 @@ cudaError_t make_row_map(CUtensorMap* map, const void* base, long long rows) {
 
 template <int S, bool kPaged>
 cudaError_t launch_variant(const CUtensorMap& mk, const CUtensorMap& mv, const Geometry& geo, const AttnArgs& a,
-                           uint32_t* status, unsigned grid, cudaStream_t st, bool overlap) {
-  return launch_pdl(attn_kernel<S, kPaged>, dim3(grid), dim3(kAttnWarps * 32), kAttnSmemBytes, st, overlap, mk, mv, geo,
-                    a, status);
+                           uint32_t* status, unsigned grid, cudaStream_t st, bool overlap, const ResolveArgs* rs) {
+  const dim3 block(kAttnWarps * 32);
+  if constexpr (kPaged) {
+    if (rs != nullptr && rs->has_cache)
+      return launch_pdl(attn_kernel<S, true, 2>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
+    if (rs != nullptr)
+      return launch_pdl(attn_kernel<S, true, 1>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
+  }
+  return launch_pdl(attn_kernel<S, kPaged, 0>, dim3(grid), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status,
+                    ResolveArgs{});
+}
+
+template <class K>
+cudaError_t allow_smem(K kernel) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
 }
 
 }  // namespace
 
 cudaError_t configure_attention() {
   if (encode_tiled_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
-  cudaError_t e = cudaFuncSetAttribute(attn_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+  static_assert(kAttnSmemBytes >= (int)resolve_detail::kItemStageBytes, "the resolution CTA stages its items here");
+  cudaError_t e = allow_smem(attn_kernel<16, true, 0>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 1>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 2>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, false, 0>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 0>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 1>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 2>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, false, 0>);
   return e;
 }
 
@@ -629,7 +658,7 @@ cudaError_t launch_selmap_from_sel(const Geometry& geo, const int32_t* sel, cons
 }
 
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
-                             bool overlap) {
+                             bool overlap, const ResolveArgs* fused_resolve) {
   const bool paged = a.kv_pool != nullptr;
   CUtensorMap mk, mv;
   cudaError_t e;
@@ -647,10 +676,10 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
   if (e != cudaSuccess) return e;
   const unsigned grid = (unsigned)attention_groups(geo, paged) * a.n_splits;
   if (geo.S == 16)
-    return paged ? launch_variant<16, true>(mk, mv, geo, a, status, grid, st, overlap)
-                 : launch_variant<16, false>(mk, mv, geo, a, status, grid, st, overlap);
-  return paged ? launch_variant<32, true>(mk, mv, geo, a, status, grid, st, overlap)
-               : launch_variant<32, false>(mk, mv, geo, a, status, grid, st, overlap);
+    return paged ? launch_variant<16, true>(mk, mv, geo, a, status, grid, st, overlap, fused_resolve)
+                 : launch_variant<16, false>(mk, mv, geo, a, status, grid, st, overlap, nullptr);
+  return paged ? launch_variant<32, true>(mk, mv, geo, a, status, grid, st, overlap, fused_resolve)
+               : launch_variant<32, false>(mk, mv, geo, a, status, grid, st, overlap, nullptr);
 }
 
 }  // namespace swarm

@@ -1,0 +1,376 @@
+// Stage 3: cluster resolution, global merge and load-balanced bucket scheduling (Eq. 8 without the
+// already-resident term; Sec. 5.1).  One launch, off the critical path (it runs beside attention).
+//
+//   mark     (all CTAs; inside swarm_step the selection kernel does it instead and this phase is skipped)
+//            every selected (request, page) -> global cluster id; flag[id] = 1.
+//            Idempotent byte stores: concurrent writers store the same value, so the dedup needs no
+//            atomics.  Four independent slots per thread keep the dependent loads overlapped.
+//   tail     (the CTA that finishes marking last, found with one ticket counter)
+//     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 4 flags
+//              with one load (the replica masks and sizes of those clusters are requested in the same
+//              round trip), a warp scan places them; the flags are cleared on the way so the next call
+//              starts from zeros.
+//              With cache state attached (swarm_set_cache) the same pass drops the activated clusters
+//              that are resident (Eq. 8) and updates the activation frequencies and Eq. 6 scores.
+//     route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
+//              with R >= 2 replicas are visited by (R ascending, id ascending) by one warp: lane j
+//              keeps (load[j] << 5 | j); one redux.min over the lanes named by the replica mask
+//              picks the least-loaded replica with ties to the lowest queue id, and only the lane
+//              whose value equals the minimum adds the cluster's weight.
+//              Under SWARM_ORDER_BY_ID the same warp visits every cluster in id order instead.
+//
+// The body is a device function so that two kernels can run it: resolve_kernel (swarm_resolve_clusters) and,
+// inside the fused step, one extra CTA of the attention kernel (a kernel of its own beside attention was
+// measured to stall for about 2 us whenever the attention kernel started or retired).
+#pragma once
+#include "swarm_internal.cuh"
+
+namespace swarm {
+namespace resolve_detail {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kSlotsPerThread = 4;
+constexpr size_t kItemStageBytes = 96 * 1024;            // shared-memory stage of the serial pass's operands
+
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) {
+  // number of non-zero bytes in w (flags are 0 or 1, but any non-zero byte counts)
+  const uint32_t t = (w | (w >> 1) | (w >> 2) | (w >> 3) | (w >> 4) | (w >> 5) | (w >> 6) | (w >> 7)) & 0x01010101u;
+  return __popc(t);
+}
+
+// `cta` of `n_ctas` CTAs of kThreads threads run the body; dynamic shared memory holds at least
+// items_cap * 16 bytes.
+template <bool kCached>
+__device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int n_ctas) {
+  const Geometry& geo = r.geo;
+  const swarm_cache& cache = r.cache;
+  const int32_t* __restrict__ sel = r.sel;
+  const int32_t* __restrict__ n_sel = r.n_sel;
+  const int64_t* __restrict__ page_base = r.page_base;
+  const int32_t* __restrict__ page2cluster = r.page2cluster;
+  const int64_t* __restrict__ cluster_base = r.cluster_base;
+  const uint32_t* __restrict__ replica_mask = r.replica_mask;
+  const uint16_t* __restrict__ cluster_size = r.cluster_size;
+  uint8_t* __restrict__ flags = r.flags;
+  unsigned* __restrict__ ticket = r.ticket;
+  uint4* __restrict__ items = r.items;
+  int32_t* __restrict__ uniq = r.uniq;
+  uint8_t* __restrict__ queue_of = r.queue_of;
+  int32_t* __restrict__ n_uniq = r.n_uniq;
+  int32_t* __restrict__ queue_load = r.queue_load;
+  uint32_t* __restrict__ status = r.status;
+  const int items_cap = r.items_cap;
+  (void)n_sel;
+  extern __shared__ uint4 s_items[];                     // (mask, weight << 5, output slot, -) of the serial pass, when they fit
+  __shared__ int2 s_seg[kWarps];                         // (start, length) of each warp's segment of the item list
+  __shared__ int warp_cnt[kWarps];
+  __shared__ int s_load[32];
+  __shared__ unsigned s_classes;
+  __shared__ unsigned s_item_m[32], s_item_w[32];
+  __shared__ bool s_last;
+  __shared__ int s_hits;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_hits = 0;
+  const long long c_all = cluster_base[geo.B];           // an input table: not written by the previous kernel
+  pdl_wait();                                            // the flags / the selection come from the previous kernel
+  const int C = (int)min((long long)geo.Cmax, c_all);
+  unsigned err = (c_all > geo.Cmax) ? SWARM_DEV_BAD_CLUSTER : 0u;
+
+  SWARM_STAMP(status, 0);
+  SWARM_KERNEL_BEGIN(status, 3);
+  // ---- mark (skipped when the selection kernel already set the flags: sel == nullptr) -------------
+  if (sel != nullptr) {
+    const long long slots = (long long)geo.B * geo.Hq * geo.k;
+    const long long base = (long long)cta * (kThreads * kSlotsPerThread) + tid;
+    int p[kSlotsPerThread], bh[kSlotsPerThread];
+    bool live[kSlotsPerThread];
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      const long long idx = base + (long long)u * kThreads;
+      live[u] = idx < slots;
+      bh[u] = live[u] ? (int)(idx / geo.k) : 0;
+      p[u] = live[u] ? sel[idx] : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      const long long idx = base + (long long)u * kThreads;
+      live[u] = live[u] && (int)(idx - (long long)bh[u] * geo.k) < n_sel[bh[u]];
+    }
+    long long cid[kSlotsPerThread];
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u) {
+      cid[u] = -1;
+      if (!live[u]) continue;
+      const int b = bh[u] / geo.Hq;
+      const long long pb = page_base[b];
+      if (p[u] < 0 || p[u] >= page_base[b + 1] - pb) { err |= SWARM_DEV_BAD_PAGE; continue; }
+      const int c = page2cluster[pb + p[u]];
+      const long long cb = cluster_base[b];
+      if (c < 0 || c >= cluster_base[b + 1] - cb || cb + c >= C) { err |= SWARM_DEV_BAD_CLUSTER; continue; }
+      cid[u] = cb + c;
+    }
+#pragma unroll
+    for (int u = 0; u < kSlotsPerThread; ++u)
+      if (cid[u] >= 0) flags[cid[u]] = 1;
+  }
+  if (err) atomicOr(status, err);
+  err = 0u;
+
+  // ---- which CTA is last? -------------------------------------------------------------------------
+  if (n_ctas > 1) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(ticket, 1u) == (unsigned)n_ctas - 1u);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+  } else {
+    __syncthreads();   // one CTA: its own marks are visible to all of its threads after the barrier
+  }
+  SWARM_STAMP_ANY_CTA(status, 1);
+
+  // ---- compact (flags are read past L1: other CTAs wrote them) -------------------------------------
+  // Every lane takes 4 flags (one word) at a time, so that up to 1024 clusters keep all 256 threads busy in a
+  // single pass; warp w owns a contiguous range of words, which keeps the ids in ascending order.
+  if (tid < 32) s_load[tid] = 0;
+  if (tid == 0) s_classes = 0u;
+  const int n_vec = (C + 3) / 4;                         // the flag array is padded to 16 bytes
+  const int vec_per_warp = (n_vec + kWarps - 1) / kWarps;
+  const int v_lo = min(n_vec, warp * vec_per_warp), v_hi = min(n_vec, v_lo + vec_per_warp);
+  uint32_t* f1 = reinterpret_cast<uint32_t*>(flags);
+  const unsigned valid_bits = geo.D == 32 ? 0xFFFFFFFFu : ((1u << geo.D) - 1u);
+  const bool by_id = (geo.flags & SWARM_ORDER_BY_ID) != 0;
+  const bool unit = (geo.flags & SWARM_UNIT_LOAD) != 0;
+
+  // One word of flags with the replica masks and sizes of its 4 clusters, all requested in the same memory
+  // round trip; a row that would cross the end of the tables is read entry by entry.
+  struct Row {
+    uint32_t f;
+    uint4 mk;
+    uint2 sz;
+  };
+  auto load_row = [&](int v, bool with_flags) -> Row {
+    Row r;
+    r.f = 0u;
+    r.mk = make_uint4(0u, 0u, 0u, 0u);
+    r.sz = make_uint2(0u, 0u);
+    if (v < v_hi) {
+      if (with_flags) r.f = __ldcg(f1 + v);
+      if (v * 4 + 4 <= C) {
+        r.mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v * 4));
+        r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));
+      } else {
+        uint32_t* mk = &r.mk.x;
+        uint32_t* sz = &r.sz.x;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (v * 4 + j < C) {
+            mk[j] = replica_mask[v * 4 + j];
+            sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
+          }
+        }
+      }
+    }
+    return r;
+  };
+
+  // pass 1: count.  With one word per lane (up to 1024 clusters) the row stays in registers for pass 2.
+  const bool one_vec = v_hi - v_lo <= 32;
+  Row keep = load_row(v_lo + lane, true);
+  int cnt = 0;
+  if (one_vec) {
+    cnt = nonzero_bytes(keep.f);
+    if (kCached) {                                         // activated but resident: not fetched (Eq. 8)
+      const int v = v_lo + lane;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (((keep.f >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+    }
+  } else {
+    for (int v0 = v_lo; v0 < v_hi; v0 += 128) {            // four independent loads in flight per lane
+      uint32_t f[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u + lane;
+        f[u] = v < v_hi ? __ldcg(f1 + v) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        cnt += nonzero_bytes(f[u]);
+        if (kCached) {
+          const int v = v0 + 32 * u + lane;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (((f[u] >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+  if (lane == 0) warp_cnt[warp] = cnt;
+  __syncthreads();
+  int before = 0, n = 0;
+  for (int w2 = 0; w2 < kWarps; ++w2) {
+    if (w2 < warp) before += warp_cnt[w2];
+    n += warp_cnt[w2];
+  }
+  // pass 2: place the ids, clear the flags, validate each cluster's replica mask and route the single-replica
+  // ones.  The clusters that need the serial pass are packed, in id order, into this warp's segment of the
+  // item list, which starts at the warp's first output position (a segment cannot outgrow the warp's ids).
+  const bool staged = n <= items_cap;
+  const int seg_base = before;
+  int seg_len = 0;
+  unsigned classes = 0u;
+  Row cur = keep;
+  for (int v0 = v_lo; v0 < v_hi; v0 += 32) {
+    const int v = v0 + lane;
+    const Row nxt = load_row(v + 32, true);                // the next row travels while this one is processed
+    const uint32_t f = cur.f;
+    if (f) __stcg(f1 + v, 0u);                             // leave zeros for the next call
+    unsigned fetch_bits = 0u, serial_bits = 0u;            // bit j: cluster v*4+j is fetched / needs the serial pass
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool on = ((f >> (8 * j)) & 0xFFu) != 0u;
+      bool fetch = on;
+      if (kCached) {
+        // cache bookkeeping of Sec. 5.2 for every cluster, activated or not
+        const int c = v * 4 + j;
+        if (v < v_hi && c < C) {
+          const bool res = cache.resident[c] != 0;
+          int fr = cache.freq[c];
+          if (on) ++fr; else if (res) --fr;
+          if (on || res) cache.freq[c] = fr;
+          if (cache.score != nullptr) {
+            const float size_f = (float)cluster_size[c];
+            cache.score[c] = (float)fr * (cache.t_base + size_f * cache.t_transfer) / size_f;
+          }
+          if (on && res) { fetch = false; atomicAdd(&s_hits, 1); }
+        }
+      }
+      const unsigned m = (&cur.mk.x)[j];
+      const bool valid = m != 0u && !(m & ~valid_bits);
+      fetch_bits |= (fetch ? 1u : 0u) << j;
+      serial_bits |= (fetch && valid && (by_id || __popc(m) > 1) ? 1u : 0u) << j;
+    }
+    // one scan for both output positions: ids in the low half, serial items in the high half
+    const int mine = __popc(fetch_bits) | (__popc(serial_bits) << 16);
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    int pos = before + ((incl - mine) & 0xFFFF);
+    int spos = seg_base + seg_len + ((incl - mine) >> 16);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if ((fetch_bits >> j) & 1u) {
+        const int c = v * 4 + j, i = pos++;
+        uniq[i] = c;
+        const unsigned m = (&cur.mk.x)[j];
+        const unsigned size = ((&cur.sz.x)[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+        const unsigned wgt = unit ? 1u : size;
+        if ((serial_bits >> j) & 1u) {
+          classes |= 1u << (__popc(m) - 1);
+          const uint4 item = make_uint4(m, wgt << 5, (unsigned)i, 0u);   // what the serial pass needs
+          if (staged) s_items[spos] = item;                // the serial pass then never waits on global memory
+          else items[spos] = item;
+          ++spos;
+        } else if (m == 0u || (m & ~valid_bits)) {
+          err |= SWARM_DEV_BAD_REPLICA;
+          queue_of[i] = 0xFF;
+        } else {
+          const int qd = __ffs(m) - 1;                     // a single replica: nothing to decide
+          queue_of[i] = (uint8_t)qd;
+          atomicAdd(&s_load[qd], (int)wgt);
+        }
+      }
+    }
+    const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    before += tot & 0xFFFF;
+    seg_len += tot >> 16;
+    cur = nxt;
+  }
+  if (lane == 0) s_seg[warp] = make_int2(seg_base, seg_len);
+  if (staged)                                              // in shared memory the serial pass walks one flat list:
+    for (int k = seg_base + seg_len + lane; k < before; k += 32)   // blank the rest of this warp's slots
+      s_items[k] = make_uint4(0u, 0u, 0u, 0u);
+  SWARM_STAMP_ANY_CTA(status, 2);
+  if (classes) atomicOr(&s_classes, classes);
+  if (err) atomicOr(status, err);
+  __syncthreads();
+  SWARM_STAMP_ANY_CTA(status, 3);
+
+  // ---- the ordered greedy, one warp ------------------------------------------------------------------
+  // It walks the warps' segments in order, which is id order (from shared memory: all of them as one list,
+  // the unused slots blank).  32 clusters at a time are staged in shared
+  // memory so that the serial loop is a plain counted loop whose operands are fetched one step ahead of
+  // the dependent chain select -> redux.min -> compare -> add.
+  if (warp == 0) {
+    unsigned L = ((unsigned)s_load[lane] << 5) | (unsigned)lane;     // (load, queue id) in one comparable word
+    const unsigned todo = by_id ? 1u : (s_classes & ~1u);
+    for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D); ++R) {
+      if (!by_id && !((todo >> (R - 1)) & 1u)) continue;
+      for (int w2 = 0; w2 < (staged ? 1 : kWarps); ++w2) {
+        const int base = staged ? 0 : s_seg[w2].x, len = staged ? n : s_seg[w2].y;
+        // (mask, weight, output slot) of 32 clusters per step, fetched two steps ahead of their use
+        auto item_at = [&](int k) -> uint4 {
+          return k >= len ? make_uint4(0u, 0u, 0u, 0u) : (staged ? s_items[base + k] : items[base + k]);
+        };
+        uint4 pre0 = item_at(lane);
+        uint4 pre1 = item_at(32 + lane);
+        for (int k0 = 0; k0 < len; k0 += 32) {
+          const unsigned m = pre0.x, wgt = pre0.y, slot = pre0.z;
+          pre0 = pre1;
+          pre1 = item_at(k0 + 64 + lane);
+          const bool mine = m != 0u && (by_id || __popc(m) == R);
+          const unsigned pending = __ballot_sync(0xFFFFFFFFu, mine);
+          const int cnt_p = __popc(pending);
+          if (cnt_p == 0) continue;
+          const int rank = __popc(pending & ((1u << lane) - 1u));
+          if (mine) { s_item_m[rank] = m; s_item_w[rank] = wgt; }
+          __syncwarp();
+          unsigned my_q = 0u;
+          unsigned mm = s_item_m[0], ww = s_item_w[0];
+          for (int r = 0; r < cnt_p; ++r) {
+            const unsigned mm_next = s_item_m[min(r + 1, 31)], ww_next = s_item_w[min(r + 1, 31)];
+            const unsigned key = ((mm >> lane) & 1u) ? L : 0xFFFFFFFFu;
+            const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);   // ~55 cycles per cluster end to end;
+            if (L == best) L += ww;                                      // shuffle-, ballot- and register-based
+            if (rank == r) my_q = best & 31u;                            // variants measured slower on sm_100
+            mm = mm_next;
+            ww = ww_next;
+          }
+          // From shared memory the choice goes back into the item and is written out after the pass: a global
+          // store issued while the attention kernel starts or retires was measured to hold this warp for 2 us.
+          if (mine) {
+            if (staged) s_items[base + k0 + lane].w = my_q;
+            else queue_of[slot] = (uint8_t)my_q;
+          }
+          __syncwarp();
+        }
+      }
+    }
+    SWARM_STAMP_ANY_CTA(status, 4);
+    SWARM_KERNEL_END(status, 3);
+    if (staged) {
+      __syncwarp();
+      for (int k = lane; k < n; k += 32) {
+        const uint4 item = s_items[k];
+        if (item.x != 0u) queue_of[item.z] = (uint8_t)item.w;
+      }
+    }
+    if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
+    if (lane == 0) {
+      *n_uniq = n;
+      if (kCached && cache.n_hit != nullptr) *cache.n_hit = s_hits;
+      if (n_ctas > 1) *ticket = 0u;                               // ready for the next call
+    }
+  }
+}
+
+}  // namespace resolve_detail
+}  // namespace swarm

@@ -58,11 +58,35 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
                         const int64_t* page_base = nullptr, const int32_t* page2cluster = nullptr,
                         const int64_t* cluster_base = nullptr, uint8_t* flags = nullptr,
                         const uint32_t* replica_mask = nullptr, const uint16_t* cluster_size = nullptr);
-cudaError_t launch_resolve(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
-                           const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
-                           const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
-                           int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                           cudaStream_t st, bool overlap, const swarm_cache* cache = nullptr);
+// Everything the cluster-resolution body needs (see resolve_body.cuh).  sel == nullptr: the flags are already
+// set (by the selection or the expansion kernel) and a single CTA runs the tail.
+struct ResolveArgs {
+  Geometry geo;
+  swarm_cache cache;
+  bool has_cache;
+  const int32_t* sel;
+  const int32_t* n_sel;
+  const int64_t* page_base;
+  const int32_t* page2cluster;
+  const int64_t* cluster_base;
+  const uint32_t* replica_mask;
+  const uint16_t* cluster_size;
+  uint8_t* flags;
+  unsigned* ticket;
+  uint4* items;
+  int32_t* uniq;
+  uint8_t* queue_of;
+  int32_t* n_uniq;
+  int32_t* queue_load;
+  uint32_t* status;
+  int items_cap;
+};
+ResolveArgs make_resolve_args(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
+                              const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
+                              const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
+                              int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
+                              const swarm_cache* cache = nullptr);
+cudaError_t launch_resolve(const ResolveArgs& r, cudaStream_t st, bool overlap);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,
                           int32_t* n_tok, uint32_t* status, cudaStream_t st);
@@ -84,8 +108,9 @@ struct AttnArgs {
   float* lse;
   int n_splits;
 };
+// `fused_resolve` (paged mode only): one extra CTA of the grid runs cluster resolution with these arguments.
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
-                             bool overlap = false);
+                             bool overlap = false, const ResolveArgs* fused_resolve = nullptr);
 // (request, head group) units the attention grid is split over: one per KV head (and per 8 heads of the
 // group) in paged mode, one per query head for gathered buffers.
 int attention_groups(const Geometry& geo, bool paged);
