@@ -320,8 +320,8 @@ def run_swarm(args):
                 "h2d_bytes_per_step": B * Hq * d * 2, "d2h_bytes_per_step": B * Hq * d * 4 + B * Hq * 4 + 4 + D * 4,
                 "note": "swarm_step_host: q from pinned host memory, out/lse/n_uniq/queue_load read back; "
                         "the KV pool and its summaries are resident state, like weights"},
-        "gpu_launches": K * 5,
-        "gpu_launches_per_step": 5,
+        "gpu_launches": K * 3,   # scorer, selection, attention + cluster resolution
+        "gpu_launches_per_step": 3,
         "device_status": status,
         "n_uniq_clusters": int(sessions[0].o.n_uniq[0]),
         "clocks": sampler.summary([(t_a, t_b), (t_e, t_f)]),

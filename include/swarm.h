@@ -128,8 +128,7 @@ typedef struct swarm_medoid_index {
                                     /* of the cluster scores                                                           */
 } swarm_medoid_index;
 
-/* Lifetime.  swarm_create validates the shape and allocates only host memory plus one auxiliary
- * CUDA stream and two events (used to run cluster resolution beside attention inside swarm_step).
+/* Lifetime.  swarm_create validates the shape and allocates only host memory.
  * The CUDA device current at creation must stay current for every later call with this ctx. */
 int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx);
 int32_t swarm_destroy(swarm_ctx* ctx);
@@ -234,8 +233,8 @@ int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g
 
 /* The fused step: stages 1-4 enqueued back to back with no host round trip.  Attention reads the
  * selected pages straight from the pool; the gathered copies are written only when k_out / v_out
- * are given.  Cluster resolution runs on the ctx's auxiliary stream beside attention and is
- * joined back before the call's work is complete on `stream`.  Integer outputs equal those of the
+ * are given.  Three launches on `stream`: scoring, selection, and one kernel in which cluster resolution
+ * runs as one extra CTA beside the attention CTAs.  Integer outputs equal those of the
  * four separate calls exactly; out / lse agree within rounding.  The call can be captured into a
  * CUDA graph by the caller (stream capture). */
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);

@@ -15,8 +15,6 @@ struct swarm_ctx {
   uint8_t* ws;
   int64_t ws_bytes;
   int user_splits;            // 0 = chosen from the shape
-  cudaStream_t side;          // cluster resolution runs here beside attention
-  cudaEvent_t ev_fork, ev_join;
   cudaError_t last_err;
   cudaGraphExec_t host_graph;  // swarm_step_host: the recorded step, valid for the arguments in host_key
   unsigned char host_key[256];
@@ -158,9 +156,6 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   if (e == cudaSuccess) e = configure_resolve();
   if (e == cudaSuccess) e = configure_attention();
   if (e == cudaSuccess) e = configure_medoid();
-  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     delete ctx;
     return SWARM_ERR_CUDA;
@@ -172,9 +167,6 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
 int32_t swarm_destroy(swarm_ctx* ctx) {
   if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
   if (ctx->host_graph != nullptr) cudaGraphExecDestroy(ctx->host_graph);
-  cudaEventDestroy(ctx->ev_fork);
-  cudaEventDestroy(ctx->ev_join);
-  cudaStreamDestroy(ctx->side);
   delete ctx;
   return SWARM_OK;
 }
