@@ -263,6 +263,8 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swar
  * recommended): copies q_host (bf16 [B][Hq][d]) into the ctx's staging area, runs swarm_step with
  * `inputs` (whose q field is ignored) and `outputs`, copies out, lse, n_uniq, queue_load back into
  * the given host buffers and WAITS for completion.  Any *_host pointer may be NULL to skip it.
+ * Result buffers that are pinned and addressable by the device (unified addressing; out_host 16-byte aligned)
+ * are filled by one small kernel storing straight into them, otherwise by one copy operation each.
  * With pinned host buffers and a non-default stream the first call with a given set of pointers
  * records these operations into a CUDA graph (owned by the ctx) and later calls replay it; the
  * tensor shapes and the device tables must then stay where they are, their contents may change. */

@@ -107,6 +107,20 @@ bool pool_inputs_ok(const swarm_inputs* in) {
   return in && !bad(in->kv_pool) && !bad(in->page_base) && !bad(in->ctx_len);
 }
 
+// The device's address of a pinned host buffer (unified addressing), or null when the device cannot store to it
+// directly (pageable memory, no mapping, misaligned) or when the pointer itself is null.
+template <class T>
+T* device_view(T* host, size_t align) {
+  if (host == nullptr || (reinterpret_cast<uintptr_t>(host) & (align - 1)) != 0) return nullptr;
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return nullptr;
+  return static_cast<T*>(attr.devicePointer);
+}
+
 // Arguments of the cluster-resolution body; sel == nullptr when the flags were set by the selection kernel.
 ResolveArgs step_resolve_args(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
                               int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load) {
@@ -362,6 +376,17 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   local.q = q_dev;
   const int32_t rc = swarm_step(ctx, &local, o, st);
   if (rc != SWARM_OK) return rc;
+  // Results: when every destination is pinned host memory the device can address (and 16-byte aligned for
+  // out), one small kernel stores them there; otherwise one copy operation per buffer.
+  float* out_d = device_view<float>(out_host, 16);
+  float* lse_d = device_view<float>(lse_host, 4);
+  int32_t* n_uniq_d = device_view<int32_t>(n_uniq_host, 4);
+  int32_t* queue_load_d = device_view<int32_t>(queue_load_host, 4);
+  if ((out_host == nullptr || out_d) && (lse_host == nullptr || lse_d) && (n_uniq_host == nullptr || n_uniq_d) &&
+      (queue_load_host == nullptr || queue_load_d)) {
+    SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d, st));
+    return SWARM_OK;
+  }
   if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));
   if (lse_host) SWARM_TRY(cudaMemcpyAsync(lse_host, o->lse, bh * 4, cudaMemcpyDeviceToHost, st));
   if (n_uniq_host) SWARM_TRY(cudaMemcpyAsync(n_uniq_host, o->n_uniq, 4, cudaMemcpyDeviceToHost, st));

@@ -116,4 +116,33 @@ cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool,
   return cudaGetLastError();
 }
 
+// Results of a step written straight into host memory the device can address (pinned, unified addressing):
+// one small kernel instead of four copy operations.  16-byte vectors for out, words for the rest.
+namespace {
+__global__ void __launch_bounds__(256)
+publish_kernel(const float* __restrict__ out, const float* __restrict__ lse, const int32_t* __restrict__ n_uniq,
+               const int32_t* __restrict__ queue_load, float* out_h, float* lse_h, int32_t* n_uniq_h,
+               int32_t* queue_load_h, int n_out4, int n_lse, int n_queues) {
+  pdl_wait();                                               // the results come from the previous kernel
+  const int t = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
+  if (out_h != nullptr)
+    for (int i = t; i < n_out4; i += stride)
+      reinterpret_cast<float4*>(out_h)[i] = __ldcg(reinterpret_cast<const float4*>(out) + i);
+  if (lse_h != nullptr)
+    for (int i = t; i < n_lse; i += stride) lse_h[i] = __ldcg(lse + i);
+  if (queue_load_h != nullptr)
+    for (int i = t; i < n_queues; i += stride) queue_load_h[i] = __ldcg(queue_load + i);
+  if (n_uniq_h != nullptr && t == 0) *n_uniq_h = __ldcg(n_uniq);
+}
+}  // namespace
+
+cudaError_t launch_publish(const Geometry& geo, const float* out, const float* lse, const int32_t* n_uniq,
+                           const int32_t* queue_load, float* out_h, float* lse_h, int32_t* n_uniq_h,
+                           int32_t* queue_load_h, cudaStream_t st) {
+  const int n_out4 = geo.B * geo.Hq * kHeadDim / 4;
+  const int grid = max(1, min(32, (n_out4 + 255) / 256));
+  return launch_pdl(publish_kernel, dim3(grid), dim3(256), 0, st, true, out, lse, n_uniq, queue_load, out_h, lse_h,
+                    n_uniq_h, queue_load_h, n_out4, geo.B * geo.Hq, geo.D);
+}
+
 }  // namespace swarm
