@@ -264,6 +264,24 @@ def test_step_host_round_trip():
     assert torch.equal(out_host, want_out)
     assert torch.equal(load_host, want_load[: w.cfg.n_queues])
     assert int(n_host[0]) == int(sess.o.n_uniq[0])
+    # on a stream of its own the call records a graph and replays it; repeated calls give the same bytes
+    stream = torch.cuda.Stream()
+    for _ in range(3):
+        out_host.zero_(); lse_host.zero_(); n_host.zero_(); load_host.zero_()
+        sess.step_host(q_host, out_host, lse_host, n_host, load_host, stream=stream)
+        assert torch.equal(out_host, want_out) and torch.equal(load_host, want_load[: w.cfg.n_queues])
+        assert torch.equal(lse_host.view(-1), sess.o.lse.cpu().view(-1)) and int(n_host[0]) == int(sess.o.n_uniq[0])
+    # pageable (and odd-offset) destinations take the copy path and give the same bytes
+    out_page = torch.empty(want_out.numel() + 1, dtype=torch.float32)[1:].view_as(want_out)
+    lse_page = torch.empty((1, 32), dtype=torch.float32)
+    n_page, load_page = torch.zeros(1, dtype=torch.int32), torch.zeros(w.cfg.n_queues, dtype=torch.int32)
+    sess.step_host(q_host, out_page, lse_page, n_page, load_page)
+    assert torch.equal(out_page, want_out) and torch.equal(load_page, want_load[: w.cfg.n_queues])
+    assert int(n_page[0]) == int(sess.o.n_uniq[0])
+    # a mix: pinned out, no lse, pageable counters
+    out_host.zero_()
+    sess.step_host(q_host, out_host, None, n_page, None)
+    assert torch.equal(out_host, want_out)
     sess.close()
 
 
