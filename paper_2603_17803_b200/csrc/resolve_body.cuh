@@ -73,6 +73,7 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) s_hits = 0;
+  pdl_launch_dependents();                               // the next kernel in the stream may be scheduled while this one runs
   const long long c_all = cluster_base[geo.B];           // an input table: not written by the previous kernel
   pdl_wait();                                            // the flags / the selection come from the previous kernel
   const int C = (int)min((long long)geo.Cmax, c_all);

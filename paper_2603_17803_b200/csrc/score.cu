@@ -77,6 +77,7 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
   constexpr int LOG_NV = ilog2(NV), LOG_G = ilog2(G);
   static_assert(NV <= 32 && (1 << LOG_NV) == NV && (1 << LOG_G) == G, "R and G must be powers of two, R*G <= 32");
   pdl_launch_dependents();   // the next kernel may be scheduled as soon as every CTA of this one runs
+  pdl_wait();                // launched behind whatever precedes it in the stream (see launch_mma)
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 0);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -202,6 +203,11 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     s_abort = 0;
     s_cum[0] = 0;
   }
+  // Launched with programmatic serialization behind whatever precedes it in the stream -- inside a chain of
+  // steps the previous step's attention + resolution kernel -- so that this kernel's launch and set-up
+  // overlap that kernel's tail.  Nothing a predecessor may have written (q, lengths, tables, summaries) is
+  // read before this point.
+  pdl_wait();
   if (warp == 1) {                                         // blocks per request, prefix by one warp
     int running = 0;
     for (int b0 = 0; b0 < geo.B; b0 += 32) {
@@ -388,8 +394,8 @@ cudaError_t launch_one(const Geometry& geo, const uint16_t* q, const uint16_t* k
                        const int32_t* ctx_len, float* scores, uint32_t* status, cudaStream_t st) {
   const int pages_per_cta = kScoreWarps * R * NB;
   dim3 grid((geo.Pmax + pages_per_cta - 1) / pages_per_cta, geo.Hkv * (geo.g / G), geo.B);
-  page_score_kernel<G, R, NB><<<grid, kScoreWarps * 32, 0, st>>>(geo, q, ksum, page_base, ctx_len, scores, status);
-  return cudaGetLastError();
+  return launch_pdl(page_score_kernel<G, R, NB>, grid, dim3(kScoreWarps * 32), 0, st, true, geo, q, ksum, page_base,
+                    ctx_len, scores, status);
 }
 
 cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
@@ -400,8 +406,8 @@ cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* k
   const int kv_groups = (geo.Hkv + kMmaConsumers - 1) / kMmaConsumers;
   const long long max_blocks = (long long)geo.B * ((geo.Pmax + kMmaPages - 1) / kMmaPages) * kv_groups;
   const int grid = (int)std::min<long long>(g_sm_count, std::max<long long>(1, max_blocks));
-  page_score_mma_kernel<<<grid, kMmaThreads, kMmaSmemBytes, st>>>(map, geo, q, page_base, ctx_len, scores, status);
-  return cudaGetLastError();
+  return launch_pdl(page_score_mma_kernel, dim3(grid), dim3(kMmaThreads), kMmaSmemBytes, st, true, map, geo, q, page_base,
+                    ctx_len, scores, status);
 }
 
 }  // namespace
