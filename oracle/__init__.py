@@ -303,3 +303,31 @@ def medoid_step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base
     k_g, v_g, n_tok = gather(kv_pool, sel_p, n_sel_p, page_base, ctx_len, Hkv, d, S)
     out, lse = attention(q, k_g, v_g, n_tok)
     return MedoidStepResult(s64, s32, cond, sel_c, n_sel_c, sel_p, n_sel_p, uniq, queue_of, load, out, lse)
+
+
+# ---- batched submission order (Sec. 5.1, last paragraph) ------------------------------------------------------
+def submit_order(queue_of, replica_mask_of_uniq, D, flags=0):
+    """Order in which the fetched clusters are submitted: the head of every bucket (queue) is taken, queue after
+    queue, into one batch; then the next heads; and so on until the buckets are empty.  A bucket holds its
+    clusters in the order the scheduling pass assigned them: by (number of replicas ascending, position in uniq
+    ascending), or by position alone under ORDER_BY_ID.
+    queue_of[i] / replica_mask_of_uniq[i] belong to uniq[i].  Returns (order, n_rounds): order[j] is the index
+    into uniq of the j-th submitted cluster."""
+    queue_of = np.asarray(queue_of)
+    masks = np.asarray(replica_mask_of_uniq, dtype=np.uint32)
+    n = len(queue_of)
+    visit = list(range(n))
+    if not (flags & ORDER_BY_ID):
+        visit.sort(key=lambda i: (bin(int(masks[i])).count("1"), i))
+    buckets = [[] for _ in range(D)]
+    for i in visit:
+        q = int(queue_of[i])
+        if q < D:                                            # clusters with a bad replica mask (0xFF) are never submitted
+            buckets[q].append(i)
+    order = []
+    rounds = max((len(b) for b in buckets), default=0)
+    for r in range(rounds):
+        for q in range(D):
+            if r < len(buckets[q]):
+                order.append(buckets[q][r])
+    return np.asarray(order, dtype=np.int32), rounds

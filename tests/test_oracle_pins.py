@@ -608,3 +608,46 @@ def test_medoid_step_scores_medoids_and_attends_whole_clusters():
     logits = K @ f(u(w.q)[b, h]) / np.sqrt(cfg.head_dim)
     pr = np.exp(logits - logits.max())
     assert np.allclose(r.out[b, h], (pr / pr.sum()) @ V, rtol=1e-9, atol=1e-9)
+
+
+# --------------------------------------------------------------------------------- batched submission order
+
+def test_submit_order_hand_case():
+    # uniq index:        0     1     2     3     4     5
+    masks = np.array([0b011, 0b100, 0b110, 0b001, 0b111, 0b010], dtype=np.uint32)   # replicas: 2 1 2 1 3 1
+    queue = np.array([1, 2, 2, 0, 0, 1], dtype=np.uint8)
+    # visit order by (replicas, index): 1 3 5 | 0 2 | 4 -> buckets: q0 [3, 4], q1 [5, 0], q2 [1, 2]
+    order, rounds = oracle.submit_order(queue, masks, 3)
+    assert rounds == 2 and list(order) == [3, 5, 1, 4, 0, 2]
+    # by position alone: buckets q0 [3, 4], q1 [0, 5], q2 [1, 2]
+    order, rounds = oracle.submit_order(queue, masks, 3, oracle.ORDER_BY_ID)
+    assert rounds == 2 and list(order) == [3, 0, 1, 4, 5, 2]
+
+
+@pytest.mark.parametrize("flags", [0, oracle.ORDER_BY_ID])
+def test_submit_order_is_a_round_robin_over_the_buckets(flags):
+    rng = np.random.default_rng(31)
+    for _ in range(20):
+        D = 5
+        sel, n_sel, page_base, p2c, cbase, mask, size = random_resolve_case(rng, D=D)
+        uniq, queue_of, load = oracle.resolve(sel, n_sel, page_base, p2c, cbase, mask, size, D, flags)
+        order, rounds = oracle.submit_order(queue_of, mask[uniq], D, flags)
+        n = len(uniq)
+        assert sorted(order.tolist()) == list(range(n))                       # every cluster exactly once
+        counts = np.bincount(queue_of, minlength=D)
+        assert rounds == counts.max(initial=0)
+        # batch r holds one cluster of every queue that still has one, in queue order
+        pos = 0
+        taken = np.zeros(D, dtype=np.int64)
+        for r in range(rounds):
+            qs = [q for q in range(D) if counts[q] > r]
+            batch = order[pos:pos + len(qs)]
+            assert [int(queue_of[i]) for i in batch] == qs
+            pos += len(qs)
+            taken[qs] += 1
+        assert pos == n
+        # inside a bucket: assignment order, i.e. the order in which a replay of the scheduling pass meets them
+        key = (lambda i: i) if flags & oracle.ORDER_BY_ID else (lambda i: (bin(int(mask[uniq[i]])).count("1"), i))
+        for q in range(D):
+            mine = [int(i) for i in order if queue_of[i] == q]
+            assert mine == sorted(mine, key=key)
