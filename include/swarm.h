@@ -147,6 +147,18 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
  * cluster that was not activated, score = freq * (t_base + size * t_transfer) / size for every cluster. */
 int32_t swarm_set_cache(swarm_ctx* ctx, const swarm_cache* cache);
 
+/* Attaches (or, with NULL, detaches) the optional output of the batched submission (Sec. 5.1: the head of
+ * every SSD bucket is taken into one submission batch, then the next heads, and so on).  While attached,
+ * swarm_resolve_clusters, swarm_step and swarm_step_medoid also write
+ *   submit_order[j]  int32 [max_clusters_total]: index into uniq of the j-th submitted cluster.  Bucket q
+ *                    holds the clusters assigned to queue q in assignment order (replica count ascending, then
+ *                    position in uniq; position alone under SWARM_ORDER_BY_ID); batch r is the r-th cluster of
+ *                    every bucket that has one, in queue order; batches follow one another.
+ *   submit_info[0]   number of batches (the largest bucket), submit_info[1] clusters submitted (those with a
+ *                    bad replica mask are left out).  submit_info may be NULL.
+ * Device pointers, 16-byte aligned; the caller keeps them valid while attached. */
+int32_t swarm_set_submit_order(swarm_ctx* ctx, int32_t* submit_order, int32_t* submit_info);
+
 /* Number of key-range splits used by the attention kernels (>= 1; 0 restores the default chosen
  * from the shape).  Results do not depend on it beyond floating-point rounding. */
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits);

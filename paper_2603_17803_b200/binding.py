@@ -27,7 +27,7 @@ EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
     "swarm_set_attn_splits", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
-    "swarm_build_medoid_index", "swarm_step_medoid",
+    "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
 )
 
 
@@ -170,6 +170,12 @@ def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_
     c = swarm_cache(_ptr(resident, "resident"), _ptr(freq, "freq"), _ptr(score, "score"), _ptr(n_hit, "n_hit"),
                     float(t_base), float(t_transfer))
     _check(load_library().swarm_set_cache(ctx, ctypes.byref(c)), "swarm_set_cache", ctx)
+
+
+def swarm_set_submit_order(ctx, submit_order=None, submit_info=None) -> None:
+    """Attach int32 device tensors for the batched submission order (or detach with None)."""
+    _check(load_library().swarm_set_submit_order(ctx, _ptr(submit_order, "submit_order"),
+                                                 _ptr(submit_info, "submit_info")), "swarm_set_submit_order", ctx)
 
 
 def swarm_build_summaries(ctx, inputs: swarm_inputs, ksum_out: torch.Tensor, stream=None) -> None:

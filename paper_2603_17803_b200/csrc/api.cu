@@ -21,6 +21,8 @@ struct swarm_ctx {
   bool host_graph_ok;
   bool has_cache;
   swarm_cache cache;
+  int32_t* submit_order;      // optional outputs of the resolution (swarm_set_submit_order)
+  int32_t* submit_info;
 };
 
 namespace {
@@ -128,7 +130,7 @@ ResolveArgs step_resolve_args(swarm_ctx* ctx, const swarm_inputs* in, const int3
                            in->cluster_replica_mask, in->cluster_size, ws_ptr<uint8_t>(ctx, ctx->lay.flags),
                            ws_ptr<unsigned>(ctx, ctx->lay.status + 64), ws_ptr<uint4>(ctx, ctx->lay.items), uniq, queue_of,
                            n_uniq, queue_load, ws_ptr<uint32_t>(ctx, ctx->lay.status),
-                           ctx->has_cache ? &ctx->cache : nullptr);
+                           ctx->has_cache ? &ctx->cache : nullptr, ctx->submit_order, ctx->submit_info);
 }
 
 }  // namespace
@@ -164,6 +166,8 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->host_graph = nullptr;
   ctx->host_graph_ok = true;
   ctx->has_cache = false;
+  ctx->submit_order = nullptr;
+  ctx->submit_info = nullptr;
   std::memset(ctx->host_key, 0, sizeof ctx->host_key);
   cudaError_t e = configure_score();
   if (e == cudaSuccess) e = configure_topk();
@@ -212,6 +216,16 @@ int32_t swarm_set_cache(swarm_ctx* ctx, const swarm_cache* cache) {
     return SWARM_ERR_INVALID_ARG;
   ctx->has_cache = cache != nullptr;
   if (cache != nullptr) ctx->cache = *cache;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
+  return SWARM_OK;
+}
+
+int32_t swarm_set_submit_order(swarm_ctx* ctx, int32_t* submit_order, int32_t* submit_info) {
+  if (ctx == nullptr || (submit_order == nullptr && submit_info != nullptr) || !aligned16(submit_order) ||
+      !aligned16(submit_info))
+    return SWARM_ERR_INVALID_ARG;
+  ctx->submit_order = submit_order;
+  ctx->submit_info = submit_info;
   if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
   return SWARM_OK;
 }

@@ -635,7 +635,7 @@ cudaError_t allow_smem(K kernel) {
 
 cudaError_t configure_attention() {
   if (encode_tiled_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
-  static_assert(kAttnSmemBytes >= (int)resolve_detail::kItemStageBytes, "the resolution CTA stages its items here");
+  static_assert(kAttnSmemBytes >= (int)resolve_detail::kResolveSmemBytes, "the resolution CTA stages its items here");
   cudaError_t e = allow_smem(attn_kernel<16, true, 0>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 1>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 2>);

@@ -16,9 +16,9 @@ __global__ void __launch_bounds__(kThreads) resolve_kernel(ResolveArgs r) {
 cudaError_t configure_resolve() {
   // static + dynamic shared memory exceed the 48 KiB that needs no opt-in
   cudaError_t e = cudaFuncSetAttribute(resolve_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)kItemStageBytes);
+                                       (int)kResolveSmemBytes);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(resolve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kItemStageBytes);
+    e = cudaFuncSetAttribute(resolve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResolveSmemBytes);
   return e;
 }
 
@@ -26,8 +26,10 @@ ResolveArgs make_resolve_args(const Geometry& geo, const int32_t* sel, const int
                               const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                               const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
                               int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                              const swarm_cache* cache) {
+                              const swarm_cache* cache, int32_t* submit_order, int32_t* submit_info) {
   ResolveArgs r{};
+  r.submit_order = submit_order;
+  r.submit_info = submit_info;
   r.geo = geo;
   r.has_cache = cache != nullptr;
   if (cache != nullptr) r.cache = *cache;
@@ -44,8 +46,8 @@ cudaError_t launch_resolve(const ResolveArgs& r, cudaStream_t st, bool overlap) 
       r.sel == nullptr ? 1u : (unsigned)((slots + kThreads * kSlotsPerThread - 1) / (kThreads * kSlotsPerThread));
   // The dynamic shared memory stages the serial pass's operands.
   if (r.has_cache)
-    return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), kItemStageBytes, st, overlap, r);
-  return launch_pdl(resolve_kernel<false>, dim3(grid), dim3(kThreads), kItemStageBytes, st, overlap, r);
+    return launch_pdl(resolve_kernel<true>, dim3(grid), dim3(kThreads), kResolveSmemBytes, st, overlap, r);
+  return launch_pdl(resolve_kernel<false>, dim3(grid), dim3(kThreads), kResolveSmemBytes, st, overlap, r);
 }
 
 }  // namespace swarm

@@ -32,6 +32,7 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kSlotsPerThread = 4;
 constexpr size_t kItemStageBytes = 96 * 1024;            // shared-memory stage of the serial pass's operands
+constexpr size_t kResolveSmemBytes = kItemStageBytes + kItemStageBytes / 2;   // + key and rank of the submission order
 
 __device__ __forceinline__ int nonzero_bytes(uint32_t w) {
   // number of non-zero bytes in w (flags are 0 or 1, but any non-zero byte counts)
@@ -369,6 +370,70 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       *n_uniq = n;
       if (kCached && cache.n_hit != nullptr) *cache.n_hit = s_hits;
       if (n_ctas > 1) *ticket = 0u;                               // ready for the next call
+    }
+  }
+
+  // ---- batched submission order (Sec. 5.1, last paragraph; only when the caller attached the output) ------
+  // Bucket q holds its clusters in assignment order: (replica count ascending, position in uniq ascending), or
+  // position alone under SWARM_ORDER_BY_ID.  Batch r takes the r-th cluster of every bucket that has one, in
+  // queue order.  Three steps: every thread forms the (class, queue) key of its clusters; one warp walks the
+  // keys in position order and ranks each cluster inside its (class, queue) group; every thread then turns
+  // (class, queue, rank) into the cluster's place in the submission order with the bucket sizes alone.
+  if (r.submit_order != nullptr) {
+    __shared__ int s_group[33 * 32];                       // clusters per (class, queue); then the start of each group in its bucket
+    __shared__ int s_bucket[32];                           // clusters per queue
+    uint32_t* key_of = staged ? reinterpret_cast<uint32_t*>(s_items + items_cap) : reinterpret_cast<uint32_t*>(items);
+    uint32_t* rank_of = key_of + (staged ? items_cap : n);
+    for (int i = tid; i < 33 * 32; i += kThreads) s_group[i] = 0;
+    __syncthreads();                                       // also: every queue_of entry is written
+    for (int i = tid; i < n; i += kThreads) {
+      const unsigned q = __ldcg(queue_of + i);
+      const unsigned cls = by_id ? 0u : (unsigned)__popc(replica_mask[__ldcg(uniq + i)]);
+      key_of[i] = q >= 32u ? 0xFFFFFFFFu : (cls * 32u + q);   // clusters with a bad replica mask are not submitted
+    }
+    __syncthreads();
+    if (warp == 0) {
+      const unsigned lt = (1u << lane) - 1u;
+      for (int i0 = 0; i0 < n; i0 += 32) {
+        const int i = i0 + lane;
+        const uint32_t key = i < n ? key_of[i] : 0xFFFFFFFFu;
+        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+        if (key != 0xFFFFFFFFu) {
+          rank_of[i] = (uint32_t)(s_group[key] + __popc(same & lt));
+        }
+        __syncwarp();
+        if (key != 0xFFFFFFFFu && (same & lt) == 0u) s_group[key] += __popc(same);   // the group's first lane
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    if (tid < 32) {                                        // bucket sizes; group counts -> group starts
+      int run = 0;
+      for (int c = 0; c <= 32; ++c) {
+        const int t = s_group[c * 32 + tid];
+        s_group[c * 32 + tid] = run;
+        run += t;
+      }
+      s_bucket[tid] = run;
+    }
+    __syncthreads();
+    int submitted = 0, rounds = 0;
+    for (int q = 0; q < geo.D; ++q) {
+      submitted += s_bucket[q];
+      rounds = max(rounds, s_bucket[q]);
+    }
+    for (int i = tid; i < n; i += kThreads) {
+      const uint32_t key = key_of[i];
+      if (key == 0xFFFFFFFFu) continue;
+      const int q = (int)(key & 31u);
+      const int depth = s_group[key] + (int)rank_of[i];    // position inside bucket q
+      int pos = 0;
+      for (int q2 = 0; q2 < geo.D; ++q2) pos += min(s_bucket[q2], depth) + ((q2 < q && s_bucket[q2] > depth) ? 1 : 0);
+      r.submit_order[pos] = i;
+    }
+    if (tid == 0 && r.submit_info != nullptr) {
+      r.submit_info[0] = rounds;
+      r.submit_info[1] = submitted;
     }
   }
 }

@@ -80,12 +80,15 @@ struct ResolveArgs {
   int32_t* queue_load;
   uint32_t* status;
   int items_cap;
+  int32_t* submit_order;   // optional: submission order (indices into uniq), see resolve_body.cuh
+  int32_t* submit_info;    // optional: [0] batches, [1] clusters submitted
 };
 ResolveArgs make_resolve_args(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                               const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
                               const uint16_t* cluster_size, uint8_t* flags_ws, unsigned* ticket, uint4* items,
                               int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load, uint32_t* status,
-                              const swarm_cache* cache = nullptr);
+                              const swarm_cache* cache = nullptr, int32_t* submit_order = nullptr,
+                              int32_t* submit_info = nullptr);
 cudaError_t launch_resolve(const ResolveArgs& r, cudaStream_t st, bool overlap);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,

@@ -135,6 +135,13 @@ class Session:
                                              n_sel=self.n_sel_clusters, uniq=o.uniq, queue_of=o.queue_of,
                                              n_uniq=o.n_uniq, queue_load=o.queue_load, out=o.out, lse=o.lse)
 
+    def enable_submit_order(self) -> None:
+        """Attaches the outputs of the batched submission order (indices into uniq, and [batches, submitted])."""
+        i32 = dict(dtype=torch.int32, device=self.device)
+        self.submit_order = torch.full((max(4, self.w.n_clusters),), -1, **i32)
+        self.submit_info = torch.zeros(4, **i32)
+        B.swarm_set_submit_order(self.ctx, self.submit_order, self.submit_info)
+
     def step_medoid(self, stream=None):
         B.swarm_step_medoid(self.ctx, self.inputs, self.medoid_index, self.medoid_outputs, stream)
 

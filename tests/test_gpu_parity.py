@@ -100,6 +100,10 @@ def test_c5_full_size_sampled():
     lens = w.ctx_len.cpu().numpy()
     reqs = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 7})
     parity.check_step(w, sess, requests=reqs, heads=[0, 13, 31])
+    # more fetched clusters than the resolution kernel stages in shared memory: the submission order too
+    sess.enable_submit_order()
+    sess.step()
+    assert check_submit_order(w, sess) > 20000
     sess.close()
 
 
@@ -544,4 +548,56 @@ def test_medoid_step_full_size_c2():
     sess.enable_medoid_index(32, keep_scores=True)          # 32 clusters of 8 pages: the page step's 256 pages per head
     sess.step_medoid()
     check_medoid_step(w, sess, 32)
+    sess.close()
+
+
+# ---- batched submission order (Sec. 5.1): heads of all buckets per batch -----------------------------------
+def check_submit_order(w, sess, flags=0):
+    torch.cuda.synchronize()
+    tabs = parity.host_tables(w)
+    n = int(sess.o.n_uniq.cpu().numpy()[0])
+    uniq = sess.o.uniq.cpu().numpy()[:n]
+    queue_of = sess.o.queue_of.cpu().numpy()[:n]
+    want, rounds = oracle.submit_order(queue_of, tabs["replica_mask"][uniq], w.cfg.n_queues, flags)
+    info = sess.submit_info.cpu().numpy()
+    assert info[0] == rounds and info[1] == len(want)
+    assert np.array_equal(sess.submit_order.cpu().numpy()[: len(want)], want)
+    return len(want)
+
+
+@pytest.mark.parametrize("flags", [0, B.ORDER_BY_ID])
+@pytest.mark.parametrize("name", ["c2_small", "c3_small", "c5_small"])
+def test_submit_order_matches_oracle(name, flags):
+    w = W.generate(CASES[name], seed=47, device=DEV)
+    sess = Session(w, flags=flags)
+    sess.enable_submit_order()
+    sess.step()
+    parity.check_step(w, sess, flags=flags)
+    assert check_submit_order(w, sess, flags) > 0
+    sess.submit_order.fill_(-1)
+    sess.select()
+    sess.resolve()                                          # the separate call writes it too
+    check_submit_order(w, sess, flags)
+    sess.enable_medoid_index(5)
+    sess.step_medoid()
+    check_submit_order(w, sess, flags)
+    B.swarm_set_submit_order(sess.ctx, None, None)          # detached: nothing is written any more
+    sess.submit_order.fill_(-7)
+    sess.step()
+    torch.cuda.synchronize()
+    assert int(sess.submit_order.max()) == -7
+    sess.close()
+
+
+def test_submit_order_full_size_and_bad_masks():
+    w = W.generate(W.CONFIGS["c3_batched"], seed=53, device=DEV)     # 3071 clusters, half of them with two replicas
+    sess = Session(w)
+    sess.enable_submit_order()
+    sess.step()
+    assert check_submit_order(w, sess) > 2000
+    w.cluster_replica_mask[::7] = 0                         # no replica anywhere: never submitted
+    sess.step()
+    torch.cuda.synchronize()
+    assert sess.status() & B.DEV_BAD_REPLICA
+    check_submit_order(w, sess)
     sess.close()
