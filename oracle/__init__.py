@@ -331,3 +331,22 @@ def submit_order(queue_of, replica_mask_of_uniq, D, flags=0):
             if r < len(buckets[q]):
                 order.append(buckets[q][r])
     return np.asarray(order, dtype=np.int32), rounds
+
+
+# ---- Algorithm 1: offline co-activation clustering ------------------------------------------------------------
+def build_clusters(dist, tau, members_cap=None):
+    """dist float32 [n][n], tau -> (rho int32 [n], ptr int32 [C + 1], members int32, medoid int32 [C]).
+    Clusters in creation order; members in joining order, medoid first; an entry may sit in several clusters."""
+    dist = np.ascontiguousarray(dist, dtype=np.float32)
+    n = dist.shape[0]
+    assert dist.shape == (n, n)
+    cap = int(members_cap if members_cap is not None else max(1, n) * 64)
+    rho = np.zeros(n, dtype=np.int32)
+    ptr = np.zeros(n + 1, dtype=np.int32)
+    members = np.zeros(cap, dtype=np.int32)
+    medoid = np.zeros(n, dtype=np.int32)
+    n_c = np.zeros(1, dtype=np.int32)
+    _check(_load().oracle_build_clusters(_p(dist), ctypes.c_int32(n), ctypes.c_float(tau), _p(rho), _p(ptr),
+                                         _p(members), ctypes.c_int64(cap), _p(medoid), _p(n_c)), "build_clusters")
+    C = int(n_c[0])
+    return rho, ptr[:C + 1].copy(), members[:int(ptr[C])].copy(), medoid[:C].copy()

@@ -25,6 +25,8 @@
 //   oracle_gather           the transfer of the selected pages (Sec. 6
 //                           "Asynchronous I/O"), here a byte copy
 //   oracle_attention        Eq. 1 over the gathered tokens, one query row
+//   oracle_build_clusters   Algorithm 1 (offline co-activation clustering): density of Eq. 4, medoid queue,
+//                           expansion by the average distance of Eq. 5; decisions in fp32 (see the function)
 //
 // Parity status: nothing numeric in the paper pins this path (it prints no
 // worked example for it), so against the authors' system every function here
@@ -362,6 +364,66 @@ int oracle_attention(const uint16_t* q, const uint16_t* k_g, const uint16_t* v_g
     }
     lse[bh] = m + std::log(l);
   }
+  return ORACLE_OK;
+}
+
+// Algorithm 1 (co-activation clustering) on a given distance matrix D [n][n] (fp32, row-major) and radius tau.
+// Decisions depend on floating-point comparisons, so they are taken in fp32, the precision of the matrix:
+//   density   rho[i] = #{ j != i : D[i][j] <= tau }                                   (Step 3; the listing's <=)
+//   medoids   entries by (rho descending, index ascending); a covered entry is skipped
+//   expansion C = {m}; candidates { e != m : D[m][e] <= tau } by (D[m][e] ascending, index ascending); every
+//             candidate is visited once, in that order, and joins when the average of its distances to the
+//             current members is <= tau.  The sum runs in fp32 in the order the members joined, reads
+//             D[member][candidate], and is compared against tau * |C| (fp32 product).  Covered entries stay
+//             candidates: that is how an entry comes to sit in several clusters.
+//   stop      when every entry is covered.
+// Output: clusters in creation order as CSR (ptr [n + 1] sized by the caller, members in joining order with the
+// medoid first), medoid[c], rho[i].  Returns ORACLE_BAD_ARG if members_cap is too small.
+int oracle_build_clusters(const float* D, int32_t n, float tau, int32_t* rho, int32_t* ptr, int32_t* members,
+                          int64_t members_cap, int32_t* medoid, int32_t* n_clusters) {
+  if (!D || !rho || !ptr || !members || !medoid || !n_clusters || n < 1) return ORACLE_BAD_ARG;
+  for (int32_t i = 0; i < n; ++i) {
+    int32_t c = 0;
+    for (int32_t j = 0; j < n; ++j)
+      if (j != i && D[static_cast<int64_t>(i) * n + j] <= tau) ++c;
+    rho[i] = c;
+  }
+  std::vector<int32_t> queue(static_cast<size_t>(n));
+  for (int32_t i = 0; i < n; ++i) queue[static_cast<size_t>(i)] = i;
+  std::stable_sort(queue.begin(), queue.end(), [rho](int32_t a, int32_t b) { return rho[a] > rho[b]; });
+  std::vector<char> covered(static_cast<size_t>(n), 0);
+  int32_t n_cov = 0, nc = 0;
+  int64_t fill = 0;
+  ptr[0] = 0;
+  for (int32_t qi = 0; qi < n && n_cov < n; ++qi) {
+    const int32_t m = queue[static_cast<size_t>(qi)];
+    if (covered[static_cast<size_t>(m)]) continue;
+    const float* row_m = D + static_cast<int64_t>(m) * n;
+    std::vector<int32_t> cand;
+    for (int32_t e = 0; e < n; ++e)
+      if (e != m && row_m[e] <= tau) cand.push_back(e);
+    std::stable_sort(cand.begin(), cand.end(), [row_m](int32_t a, int32_t b) { return row_m[a] < row_m[b]; });
+    std::vector<int32_t> mem{m};
+    std::vector<float> sum(cand.size());
+    for (size_t ci = 0; ci < cand.size(); ++ci) sum[ci] = row_m[cand[ci]];      // distance to the only member so far
+    for (size_t ci = 0; ci < cand.size(); ++ci) {
+      const float bound = tau * static_cast<float>(mem.size());
+      if (sum[ci] <= bound) {
+        const int32_t e = cand[ci];
+        mem.push_back(e);
+        const float* row_e = D + static_cast<int64_t>(e) * n;
+        for (size_t cj = ci + 1; cj < cand.size(); ++cj) sum[cj] = sum[cj] + row_e[cand[cj]];
+      }
+    }
+    if (fill + static_cast<int64_t>(mem.size()) > members_cap) return ORACLE_BAD_ARG;
+    for (int32_t e : mem) {
+      members[fill++] = e;
+      if (!covered[static_cast<size_t>(e)]) { covered[static_cast<size_t>(e)] = 1; ++n_cov; }
+    }
+    medoid[nc] = m;
+    ptr[++nc] = static_cast<int32_t>(fill);
+  }
+  *n_clusters = nc;
   return ORACLE_OK;
 }
 

@@ -651,3 +651,83 @@ def test_submit_order_is_a_round_robin_over_the_buckets(flags):
         for q in range(D):
             mine = [int(i) for i in order if queue_of[i] == q]
             assert mine == sorted(mine, key=key)
+
+
+# ------------------------------------------------------------------------ Algorithm 1 (offline clustering)
+
+def sym(n, fill, pairs):
+    d = np.full((n, n), fill, dtype=np.float32)
+    np.fill_diagonal(d, 0.0)
+    for (i, j), v in pairs.items():
+        d[i, j] = d[j, i] = v
+    return d
+
+
+def test_algorithm1_hand_case():
+    g = read_golden("algorithm1_hand_case.txt")
+    d = sym(5, 0.9, {(0, 1): 0.1, (0, 2): 0.2, (1, 2): 0.3, (3, 4): 0.1, (2, 3): 0.4, (2, 4): 0.5})
+    rho, ptr, members, medoid = oracle.build_clusters(d, 0.5)
+    assert list(rho) == g["rho"] and list(ptr) == g["ptr"] and list(members) == g["members"]
+    assert list(medoid) == g["medoid"]
+
+
+def test_algorithm1_extreme_radii_and_blocks():
+    rng = np.random.default_rng(41)
+    n = 12
+    d = rng.uniform(0.2, 0.8, size=(n, n)).astype(np.float32)
+    d = np.minimum(d, d.T)
+    np.fill_diagonal(d, 0.0)
+    # a radius below every distance: every entry is its own cluster, in index order
+    rho, ptr, members, medoid = oracle.build_clusters(d, 0.1)
+    assert not rho.any() and list(ptr) == list(range(n + 1)) and list(members) == list(range(n))
+    assert list(medoid) == list(range(n))
+    # a radius above every distance: one cluster, the others in order of their distance to entry 0
+    rho, ptr, members, medoid = oracle.build_clusters(d, 0.9)
+    assert np.all(rho == n - 1) and list(ptr) == [0, n] and list(medoid) == [0]
+    assert list(members) == [0] + sorted(range(1, n), key=lambda e: (d[0, e], e))
+    # well separated blocks of different sizes: the clusters are the blocks, the largest first
+    blocks = [[0, 5, 7], [1, 2, 3, 4, 6], [8, 9], [10], [11]]
+    d = np.full((n, n), 0.9, dtype=np.float32)
+    for blk in blocks:
+        for i in blk:
+            for j in blk:
+                d[i, j] = 0.25
+    np.fill_diagonal(d, 0.0)
+    rho, ptr, members, medoid = oracle.build_clusters(d, 0.5)
+    got = [list(members[ptr[c]:ptr[c + 1]]) for c in range(len(medoid))]
+    assert got == [[1, 2, 3, 4, 6], [0, 5, 7], [8, 9], [10], [11]]
+    assert list(medoid) == [1, 0, 8, 10, 11]
+
+
+def test_algorithm1_replay_in_exact_arithmetic():
+    """Distances on a grid of 1/64: fp32 sums are exact, so an exact-arithmetic replay must agree everywhere."""
+    from fractions import Fraction
+    rng = np.random.default_rng(43)
+    for n, tau64 in [(30, 20), (64, 28), (90, 16)]:
+        g = rng.integers(1, 64, size=(n, n))
+        g = np.minimum(g, g.T)
+        np.fill_diagonal(g, 0)
+        d = (g / 64.0).astype(np.float32)
+        tau = tau64 / 64.0
+        rho, ptr, members, medoid = oracle.build_clusters(d, tau)
+        want_rho = [(g[i] <= tau64).sum() - 1 for i in range(n)]
+        assert list(rho) == want_rho
+        queue = sorted(range(n), key=lambda i: (-want_rho[i], i))
+        covered, clusters, meds = set(), [], []
+        for m in queue:
+            if len(covered) == n:
+                break
+            if m in covered:
+                continue
+            cand = sorted((e for e in range(n) if e != m and g[m, e] <= tau64), key=lambda e: (g[m, e], e))
+            mem = [m]
+            for c in cand:
+                if Fraction(int(sum(g[e, c] for e in mem)), len(mem)) <= tau64:
+                    mem.append(c)
+            clusters.append(mem)
+            meds.append(m)
+            covered.update(mem)
+        got = [list(members[ptr[c]:ptr[c + 1]]) for c in range(len(medoid))]
+        assert got == clusters and list(medoid) == meds
+        assert set(members.tolist()) == set(range(n))                       # every entry is covered
+        assert any(members.tolist().count(e) > 1 for e in range(n))         # and some sit in several clusters
