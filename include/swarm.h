@@ -271,6 +271,25 @@ int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, con
 int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_medoid_index* index,
                           const swarm_outputs* outputs, void* stream);
 
+/* Offline index build (no ctx; not part of a decode step): Algorithm 1, co-activation clustering of n entries
+ * from their distance matrix dist (fp32 [n][n] row-major, d = 1 - co-activation probability) and the cluster
+ * radius tau.  All pointers are device pointers, 16-byte aligned.
+ *   density[i]  = #{ j != i : dist[i][j] <= tau }                                   (Step 3, Eq. 4)
+ *   medoids     entries by (density descending, index ascending); an entry already covered is skipped
+ *   expansion   C = {m}; the candidates { e != m : dist[m][e] <= tau } are visited once by (dist[m][e] ascending,
+ *               index ascending); a candidate joins when the average of its distances to the current members is
+ *               <= tau (Step 4, Eq. 5): fp32 sum in joining order over dist[member][candidate], compared against
+ *               tau * |C|.  Covered entries stay candidates, so an entry may join several clusters (replicas).
+ *   stop        when every entry is covered.
+ * Outputs: clusters in creation order as cluster_ptr [n + 1] (only n_clusters + 1 entries are written) and
+ * cluster_members (joining order, medoid first), medoid [n] (n_clusters written), n_clusters [1],
+ * dev_status [1] = 0, or 1 if cluster_members (members_cap entries, at least n) was too small -- the output is
+ * then incomplete.  n <= 32768.  workspace: swarm_build_clusters_workspace_bytes(n) bytes (< 0: minus an error code). */
+int64_t swarm_build_clusters_workspace_bytes(int32_t n_entries);
+int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, void* workspace, int64_t workspace_bytes,
+                             int32_t* density, int32_t* cluster_ptr, int32_t* cluster_members, int64_t members_cap,
+                             int32_t* medoid, int32_t* n_clusters, int32_t* dev_status, void* stream);
+
 /* End-to-end convenience for callers holding the per-step data in HOST memory (pinned memory
  * recommended): copies q_host (bf16 [B][Hq][d]) into the ctx's staging area, runs swarm_step with
  * `inputs` (whose q field is ignored) and `outputs`, copies out, lse, n_uniq, queue_load back into

@@ -28,6 +28,7 @@ EXPORTS = (
     "swarm_set_attn_splits", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
+    "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
 )
 
 
@@ -75,6 +76,7 @@ def load_library() -> ctypes.CDLL:
         for name in EXPORTS:
             getattr(lib, name).restype = ctypes.c_int32
         lib.swarm_workspace_bytes.restype = ctypes.c_int64
+        lib.swarm_build_clusters_workspace_bytes.restype = ctypes.c_int64
         _lib = lib
     return _lib
 
@@ -170,6 +172,37 @@ def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_
     c = swarm_cache(_ptr(resident, "resident"), _ptr(freq, "freq"), _ptr(score, "score"), _ptr(n_hit, "n_hit"),
                     float(t_base), float(t_transfer))
     _check(load_library().swarm_set_cache(ctx, ctypes.byref(c)), "swarm_set_cache", ctx)
+
+
+def swarm_build_clusters_workspace_bytes(n_entries: int) -> int:
+    n = int(load_library().swarm_build_clusters_workspace_bytes(ctypes.c_int32(n_entries)))
+    if n < 0:
+        raise SwarmError(-n, "swarm_build_clusters_workspace_bytes")
+    return n
+
+
+def swarm_build_clusters(dist: torch.Tensor, tau: float, members_cap: Optional[int] = None, stream=None):
+    """Algorithm 1 on a float32 [n][n] CUDA distance matrix.  Returns (density, cluster_ptr, cluster_members,
+    medoid) as int32 CUDA tensors trimmed to the clusters found; raises if members_cap was too small."""
+    n = int(dist.shape[0])
+    if dist.dtype != torch.float32 or dist.dim() != 2 or dist.shape[1] != n:
+        raise ValueError("dist must be a float32 [n][n] tensor")
+    lib = load_library()
+    ws_bytes = swarm_build_clusters_workspace_bytes(n)
+    dev = dist.device
+    cap = int(members_cap if members_cap is not None else 16 * n)
+    i32 = dict(dtype=torch.int32, device=dev)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    density, ptr, medoid = torch.empty(n, **i32), torch.empty(n + 4, **i32), torch.empty(n, **i32)
+    members, info = torch.empty(max(cap, 4), **i32), torch.zeros(8, **i32)
+    _check(lib.swarm_build_clusters(_ptr(dist, "dist"), ctypes.c_int32(n), ctypes.c_float(tau), _ptr(ws),
+                                    ctypes.c_int64(ws_bytes), _ptr(density), _ptr(ptr), _ptr(members),
+                                    ctypes.c_int64(cap), _ptr(medoid), _ptr(info[0:4]), _ptr(info[4:8]),
+                                    _stream(stream)), "swarm_build_clusters")
+    n_clusters, status = int(info[0]), int(info[4])
+    if status != 0:
+        raise SwarmError(ERR_WORKSPACE_TOO_SMALL, "swarm_build_clusters (members_cap)")
+    return density, ptr[: n_clusters + 1], members[: int(ptr[n_clusters])], medoid[:n_clusters]
 
 
 def swarm_set_submit_order(ctx, submit_order=None, submit_info=None) -> None:

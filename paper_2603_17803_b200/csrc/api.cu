@@ -230,6 +230,25 @@ int32_t swarm_set_submit_order(swarm_ctx* ctx, int32_t* submit_order, int32_t* s
   return SWARM_OK;
 }
 
+int64_t swarm_build_clusters_workspace_bytes(int32_t n_entries) {
+  if (n_entries < 1 || n_entries > 32768) return -(int64_t)SWARM_ERR_UNSUPPORTED;
+  return build_clusters_workspace_bytes(n_entries);
+}
+
+int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, void* workspace, int64_t workspace_bytes,
+                             int32_t* density, int32_t* cluster_ptr, int32_t* cluster_members, int64_t members_cap,
+                             int32_t* medoid, int32_t* n_clusters, int32_t* dev_status, void* stream) {
+  if (n_entries < 1 || !(tau >= 0.f) || bad(dist) || bad(workspace) || bad(density) || bad(cluster_ptr) ||
+      bad(cluster_members) || bad(medoid) || bad(n_clusters) || bad(dev_status) || members_cap < n_entries)
+    return SWARM_ERR_INVALID_ARG;
+  if (n_entries > 32768) return SWARM_ERR_UNSUPPORTED;
+  if (workspace_bytes < build_clusters_workspace_bytes(n_entries)) return SWARM_ERR_WORKSPACE_TOO_SMALL;
+  const cudaError_t e = launch_build_clusters(dist, n_entries, tau, workspace, density, cluster_ptr, cluster_members,
+                                              members_cap, medoid, n_clusters, dev_status,
+                                              static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SWARM_OK : SWARM_ERR_CUDA;
+}
+
 int32_t swarm_last_cuda_error(const swarm_ctx* ctx) { return ctx ? (int32_t)ctx->last_err : 0; }
 
 int32_t swarm_device_status(swarm_ctx* ctx, void* stream, uint32_t* bits) {

@@ -135,6 +135,12 @@ cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* 
                                    const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
                                    uint32_t* status, cudaStream_t st, bool overlap);
 
+// Algorithm 1 (offline co-activation clustering): see cluster.cu.
+long long build_clusters_workspace_bytes(int n);
+cudaError_t launch_build_clusters(const float* dist, int n, float tau, void* workspace, int32_t* rho, int32_t* ptr,
+                                  int32_t* members, long long members_cap, int32_t* medoid, int32_t* n_clusters,
+                                  int32_t* dev_status, cudaStream_t st);
+
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

@@ -316,3 +316,21 @@ def cluster_members(w: "Workload"):
     medoid = np.where(counts > 0, pages[np.minimum(ptr[:-1] + counts // 2, max(len(pages) - 1, 0))], 0).astype(np.int32)
     dev = w.page2cluster.device
     return (torch.from_numpy(ptr).to(dev), torch.from_numpy(pages).to(dev), torch.from_numpy(medoid).to(dev))
+
+
+def coactivation_distances(n: int, n_topics: int, seed: int, device="cpu", noise: float = 0.15,
+                           bridge_frac: float = 0.1) -> torch.Tensor:
+    """Synthetic distance matrix d = 1 - P for Algorithm 1: entries of one latent topic are co-activated with high
+    probability (small distance), entries of different topics rarely; a fraction of "bridge" entries is also close
+    to a second topic, which is what makes an entry join several clusters.  Symmetric, zero diagonal, float32 in
+    [0, 1].  Stands in for the co-activation profile the paper measures on real models."""
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    topic = torch.randint(0, n_topics, (n,), generator=g)
+    second = torch.where(torch.rand(n, generator=g) < bridge_frac, torch.randint(0, n_topics, (n,), generator=g), topic)
+    same = (topic[:, None] == topic[None, :]) | (second[:, None] == topic[None, :]) | (topic[:, None] == second[None, :])
+    base = torch.where(same, torch.tensor(0.25), torch.tensor(0.85))
+    jitter = (torch.rand((n, n), generator=g) - 0.5) * 2.0 * noise
+    d = (base + jitter).clamp_(0.0, 1.0)
+    d = torch.minimum(d, d.T).contiguous()
+    d.fill_diagonal_(0.0)
+    return d.to(torch.float32).to(device)

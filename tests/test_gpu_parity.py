@@ -601,3 +601,102 @@ def test_submit_order_full_size_and_bad_masks():
     assert sess.status() & B.DEV_BAD_REPLICA
     check_submit_order(w, sess)
     sess.close()
+
+
+# ---- Algorithm 1 (offline co-activation clustering) ---------------------------------------------------------
+def check_clusters(dist, tau, cap=None):
+    density, ptr, members, medoid = B.swarm_build_clusters(dist, tau, members_cap=cap)
+    torch.cuda.synchronize()
+    rho, ptr_ref, members_ref, medoid_ref = oracle.build_clusters(dist.cpu().numpy(), tau, members_cap=cap)
+    assert np.array_equal(density.cpu().numpy(), rho)
+    assert np.array_equal(medoid.cpu().numpy(), medoid_ref)
+    assert np.array_equal(ptr.cpu().numpy(), ptr_ref)
+    assert np.array_equal(members.cpu().numpy(), members_ref)
+    return len(medoid_ref), len(members_ref)
+
+
+@pytest.mark.parametrize("n,topics,tau", [(5, 1, 0.5), (37, 3, 0.4), (256, 8, 0.38), (1000, 20, 0.4),
+                                          (1027, 12, 0.33), (2048, 64, 0.45), (3000, 30, 0.05), (600, 4, 1.0)])
+def test_algorithm1_matches_oracle(n, topics, tau):
+    dist = W.coactivation_distances(n, topics, seed=n, device=DEV)
+    n_clusters, n_members = check_clusters(dist, tau, cap=64 * n if tau < 1.0 else None)
+    assert n_members >= n and n_clusters >= 1
+    if tau == 0.05:
+        assert n_clusters == n                              # radius below every distance: singletons
+    if tau == 1.0:
+        assert n_clusters == 1 and n_members == n           # radius above every distance: one cluster
+
+
+def test_algorithm1_hand_case_and_capacity():
+    d = np.full((5, 5), 0.9, dtype=np.float32)
+    np.fill_diagonal(d, 0.0)
+    for (i, j), v in {(0, 1): 0.1, (0, 2): 0.2, (1, 2): 0.3, (3, 4): 0.1, (2, 3): 0.4, (2, 4): 0.5}.items():
+        d[i, j] = d[j, i] = v
+    dist = torch.from_numpy(d).to(DEV)
+    density, ptr, members, medoid = B.swarm_build_clusters(dist, 0.5)
+    assert density.tolist() == [2, 2, 4, 2, 2] and ptr.tolist() == [0, 3, 6]
+    assert members.tolist() == [2, 0, 1, 3, 4, 2] and medoid.tolist() == [2, 3]
+    with pytest.raises(B.SwarmError):                       # six memberships do not fit five slots
+        B.swarm_build_clusters(dist, 0.5, members_cap=5)
+    with pytest.raises(B.SwarmError):
+        B.swarm_build_clusters(dist, -1.0)
+
+
+def test_algorithm1_clusters_drive_the_medoid_step():
+    """Clusters with replicas built on the GPU from a distance matrix, then used as the index of the medoid step."""
+    cfg = small("c2_128k", ctx_len=16 * 640, top_k=32, n_topics=8)
+    w = W.generate(cfg, seed=59, device=DEV)
+    P = cfg.max_pages()
+    dist = W.coactivation_distances(P, 16, seed=61, device=DEV)
+    density, ptr, members, medoid = B.swarm_build_clusters(dist, 0.4, members_cap=64 * P)
+    C = len(medoid)
+    assert len(members) > P                                 # some pages sit in several clusters
+    # cluster tables of the workload replaced by the ones just built (one request)
+    sizes = (ptr[1:] - ptr[:-1]).to(torch.int16)
+    rng = np.random.default_rng(3)
+    mask = torch.from_numpy(np.array([(1 << int(a)) | (1 << int(b)) for a, b in
+                                      zip(rng.integers(0, 8, C), rng.integers(0, 8, C))], dtype=np.int32)).to(DEV)
+    w.cluster_base = torch.tensor([0, C], dtype=torch.int64, device=DEV)
+    w.cluster_replica_mask, w.cluster_size = mask, sizes
+    w.page2cluster = torch.zeros(P, dtype=torch.int32, device=DEV)      # not read by the medoid step
+    sess = Session(w)
+    k_c = 6
+    sess.cluster_page_ptr, sess.cluster_pages, sess.medoid_page = ptr.to(torch.int64), members, medoid
+    sess.max_clusters_per_req = C
+    sess.medoid_ksum = torch.empty((C, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=DEV)
+    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum)
+    sess.medoid_index = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=sess.cluster_page_ptr,
+                                            cluster_pages=members, top_k_clusters=k_c, max_clusters_per_req=C)
+    i32 = dict(dtype=torch.int32, device=DEV)
+    sess.sel_clusters = torch.empty((1, cfg.n_q_heads, k_c), **i32)
+    sess.n_sel_clusters = torch.empty((1, cfg.n_q_heads), **i32)
+    sess.cluster_scores = None
+    o = sess.o
+    sess.medoid_outputs = B.make_outputs(sel=sess.sel_clusters, n_sel=sess.n_sel_clusters, uniq=o.uniq,
+                                         queue_of=o.queue_of, n_uniq=o.n_uniq, queue_load=o.queue_load, out=o.out,
+                                         lse=o.lse)
+    sess.step_medoid()
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    # oracle: scores/top-k over the medoids, union of the members, scheduling of the selected clusters
+    tabs = parity.host_tables(w)
+    ksum = W.bits_u16(sess.ksum)
+    rows = oracle.medoid_rows(ksum, tabs["page_base"], tabs["cluster_base"], medoid.cpu().numpy())
+    len_c = np.array([C * cfg.page_size], np.int32)
+    s64, s32, cond = oracle.scores(W.bits_u16(w.q), rows, tabs["cluster_base"], len_c, cfg.n_kv_heads, cfg.page_size, C)
+    sel_c, n_sel_c = sess.sel_clusters.cpu().numpy(), sess.n_sel_clusters.cpu().numpy()
+    for h in range(cfg.n_q_heads):
+        parity.check_selection(sel_c[0, h], int(n_sel_c[0, h]), s64[0, h], C, k_c)
+    sel_p, n_sel_p = oracle.expand_clusters(sel_c, n_sel_c, tabs["cluster_base"], ptr.cpu().numpy(), members.cpu().numpy())
+    ident = np.arange(C, dtype=np.int32)                     # scheduling sees the selected clusters themselves
+    uniq, queue_of, load = oracle.resolve(sel_c, n_sel_c, tabs["cluster_base"], ident, tabs["cluster_base"],
+                                          tabs["replica_mask"], tabs["cluster_size"], cfg.n_queues, 0)
+    n = int(o.n_uniq.cpu().numpy()[0])
+    assert n == len(uniq) and np.array_equal(o.uniq.cpu().numpy()[:n], uniq)
+    assert np.array_equal(o.queue_of.cpu().numpy()[:n], queue_of)
+    assert np.array_equal(o.queue_load.cpu().numpy()[: cfg.n_queues], load)
+    k_g, v_g, n_tok = oracle.gather(W.bits_u16(w.kv_pool), sel_p, n_sel_p, tabs["page_base"], tabs["ctx_len"],
+                                    cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
+    out, lse = oracle.attention(W.bits_u16(w.q), k_g, v_g, n_tok)
+    parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
+    sess.close()
