@@ -616,7 +616,8 @@ def check_clusters(dist, tau, cap=None):
 
 
 @pytest.mark.parametrize("n,topics,tau", [(5, 1, 0.5), (37, 3, 0.4), (256, 8, 0.38), (1000, 20, 0.4),
-                                          (1027, 12, 0.33), (2048, 64, 0.45), (3000, 30, 0.05), (600, 4, 1.0)])
+                                          (1027, 12, 0.33), (2048, 64, 0.45), (3000, 30, 0.05), (600, 4, 1.0),
+                                          (8192, 64, 0.4)])
 def test_algorithm1_matches_oracle(n, topics, tau):
     dist = W.coactivation_distances(n, topics, seed=n, device=DEV)
     n_clusters, n_members = check_clusters(dist, tau, cap=64 * n if tau < 1.0 else None)
