@@ -1,7 +1,9 @@
-// Stage 3: cluster resolution, global merge and load-balanced bucket scheduling (Eq. 8 without the
-// already-resident term; Sec. 5.1).  One launch, off the critical path (it runs beside attention).
+// Stage 3: cluster resolution, global merge and load-balanced bucket scheduling (Eq. 8; Sec. 5.1), written as
+// a device function that two kernels run: resolve_kernel (swarm_resolve_clusters) and, inside the fused step,
+// block 0 of the attention kernel (beside the attention CTAs; as a kernel of its own on a second stream it
+// lost about 2 us whenever the attention kernel started).
 //
-//   mark     (all CTAs; inside swarm_step the selection kernel does it instead and this phase is skipped)
+//   mark     (all CTAs; inside the fused step the selection kernel has done it and this phase is skipped)
 //            every selected (request, page) -> global cluster id; flag[id] = 1.
 //            Idempotent byte stores: concurrent writers store the same value, so the dedup needs no
 //            atomics.  Four independent slots per thread keep the dependent loads overlapped.
@@ -9,7 +11,8 @@
 //     compact  ordered compaction of the flags -> uniq[] ascending by id: each lane takes 4 flags
 //              with one load (the replica masks and sizes of those clusters are requested in the same
 //              round trip), a warp scan places them; the flags are cleared on the way so the next call
-//              starts from zeros.
+//              starts from zeros.  The clusters that need the serial pass are packed, with their output
+//              slots, into per-warp segments of an item list (shared memory when it fits).
 //              With cache state attached (swarm_set_cache) the same pass drops the activated clusters
 //              that are resident (Eq. 8) and updates the activation frequencies and Eq. 6 scores.
 //     route    single-replica clusters go to their queue (integer histogram, order-free).  Clusters
@@ -18,10 +21,7 @@
 //              picks the least-loaded replica with ties to the lowest queue id, and only the lane
 //              whose value equals the minimum adds the cluster's weight.
 //              Under SWARM_ORDER_BY_ID the same warp visits every cluster in id order instead.
-//
-// The body is a device function so that two kernels can run it: resolve_kernel (swarm_resolve_clusters) and,
-// inside the fused step, one extra CTA of the attention kernel (a kernel of its own beside attention was
-// measured to stall for about 2 us whenever the attention kernel started or retired).
+//     submit   (optional output) the batched submission order of Sec. 5.1, see the end of the body.
 #pragma once
 #include "swarm_internal.cuh"
 
