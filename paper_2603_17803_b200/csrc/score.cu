@@ -162,6 +162,7 @@ constexpr int kMmaThreads = (kMmaConsumers + 1) * 32;
 constexpr int kMmaStages = 3;
 constexpr int kMmaPages = 16;                              // pages per block = M of the MMA tile
 constexpr int kMmaHeadBytes = 4 * kMmaPages * 128;         // 4 boxes of 16 pages x 128 B
+constexpr int kBoxHeads = 2;                               // KV heads per TMA box (rows of a box: page-major, head-minor)
 constexpr int kMmaStageBytes = kMmaConsumers * kMmaHeadBytes;
 constexpr int kMmaSmemBytes = 1024 + kMmaStages * kMmaStageBytes;
 constexpr int kStreamMaxBatch = 1024;                      // requests whose block counts fit the shared prefix table
@@ -263,16 +264,19 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
         const int j_lo = k == 0 ? first_head : 0;
         const int j_hi = min(k == n_blk - 1 ? last_heads : kMmaConsumers, geo.Hkv - kvg * kMmaConsumers);
         const int page0 = (int)(page_base[fb] + (long long)tile * kMmaPages);
+        // one box carries kBoxHeads KV heads: the copy engine's rate per box, not the memory, bounds small boxes
+        const int p_lo = j_lo / kBoxHeads, p_hi = j_hi > j_lo ? (j_hi + kBoxHeads - 1) / kBoxHeads : p_lo;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])),
-                     "r"((unsigned)(max(j_hi - j_lo, 0) * kMmaHeadBytes))
+                     "r"((unsigned)((p_hi - p_lo) * kBoxHeads * kMmaHeadBytes))
                      : "memory");
-        for (int j = j_lo; j < j_hi; ++j) {
+        for (int pj = p_lo; pj < p_hi; ++pj) {
 #pragma unroll
           for (int bx = 0; bx < 4; ++bx) {
-            const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + j * kMmaHeadBytes + bx * (kMmaPages * 128));
+            const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + pj * (kBoxHeads * kMmaHeadBytes) +
+                                         bx * (kBoxHeads * kMmaPages * 128));
             asm volatile(
                 "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
-                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + j), "r"(page0), "r"(sm_addr(&full[stage])), "l"(stream_policy)
+                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + pj * kBoxHeads), "r"(page0), "r"(sm_addr(&full[stage])), "l"(stream_policy)
                 : "memory");
           }
         }
@@ -308,7 +312,9 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       }
     }
     if (active) {
-      const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + warp * kMmaHeadBytes);
+      // rows of a box: (page, head of the box) pairs, page-major; 128-byte swizzle over the row index
+      const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + (warp / kBoxHeads) * (kBoxHeads * kMmaHeadBytes));
+      const int hl = warp % kBoxHeads;
       for (int ht = 0; ht < tiles; ++ht) {
         const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
         const long long key = ((long long)b * geo.Hq + h0);
@@ -339,7 +345,8 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           uint32_t a[4];
           asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                        : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
-                       : "r"(base + (uint32_t)((cc >> 3) * (kMmaPages * 128) + r * 128 + (((cc & 7) ^ (r & 7)) << 4))));
+                       : "r"(base + (uint32_t)((cc >> 3) * (kBoxHeads * kMmaPages * 128) + (r * kBoxHeads + hl) * 128 +
+                                               (((cc & 7) ^ ((r * kBoxHeads + hl) & 7)) << 4))));
           asm volatile(
               "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
               : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
@@ -381,7 +388,7 @@ cudaError_t make_summary_map(CUtensorMap* map, const void* ksum, int Hkv, long l
   if (fn == nullptr) return cudaErrorNotSupported;
   const cuuint64_t dims[3] = {256, (cuuint64_t)Hkv, (cuuint64_t)n_pool_pages};
   const cuuint64_t strides[2] = {512, (cuuint64_t)Hkv * 512};
-  const cuuint32_t box[3] = {64, 1, (cuuint32_t)kMmaPages};
+  const cuuint32_t box[3] = {64, (cuuint32_t)kBoxHeads, (cuuint32_t)kMmaPages};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ksum), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
