@@ -111,8 +111,9 @@ __device__ __forceinline__ void split_pack(float p0, float p1, uint32_t& hi, uin
 }
 // byte offset of 16-byte chunk `chunk` (0..15, 8 coordinates each) of token row `t` inside a K or V tile
 // (two 2 KiB boxes of 64 coordinates, each with the 128-byte swizzle)
-__device__ __forceinline__ uint32_t tile_offset(int t, int chunk) {
-  return (uint32_t)((chunk >> 3) * kBoxBytes + t * 128 + (((chunk & 7) ^ (t & 7)) << 4));
+// `half` = bytes between the box of coordinates 0-63 and the box of coordinates 64-127
+__device__ __forceinline__ uint32_t tile_offset(int t, int chunk, int half) {
+  return (uint32_t)((chunk >> 3) * half + t * 128 + (((chunk & 7) ^ (t & 7)) << 4));
 }
 
 // kFused != 0 (fused step only): CTA 0 of the grid does not attend; it runs cluster resolution (stage 3) beside
@@ -131,6 +132,12 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   }
   const int cta = (int)blockIdx.x - (kFused != 0 ? 1 : 0);
   constexpr int SB = S / kUnitTokens;                   // 16-token units per page
+  // With 16-token pages read from the pool, the K rows and the V rows of a (page, KV head) are adjacent, and one
+  // box of 32 rows brings both: two copies of 4 KiB per unit instead of four of 2 KiB (the copy engine's rate per
+  // box, not the memory, bounds small boxes).  Slot layout then: [K | V] x coordinates 0-63, [K | V] x 64-127.
+  constexpr bool kWide = kPaged && S == kUnitTokens;
+  constexpr int kHalf = kWide ? 2 * kBoxBytes : kBoxBytes;   // bytes between the two coordinate halves
+  constexpr int kVOff = kWide ? kBoxBytes : 2 * kBoxBytes;   // V tile relative to the K tile
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
   __shared__ __align__(8) uint64_t bar_merge;
@@ -325,10 +332,15 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         const uint32_t dst = smem_addr(my_ring + slot * kSlotBytes);
         uint64_t* bar = &bars[warp][slot];
         mbar_expect_tx(bar, kSlotBytes);
-        tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
-        tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar, stream_policy);
-        tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar, stream_policy);
-        tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar, stream_policy);
+        if (kWide) {                                   // mapK's box is 32 rows here: K then V
+          tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
+          tma_load_2d(dst + kHalf, &mapK, 64, (int)rowK, bar, stream_policy);
+        } else {
+          tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
+          tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar, stream_policy);
+          tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar, stream_policy);
+          tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar, stream_policy);
+        }
       }
       ++fills;
     };
@@ -349,15 +361,15 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       if (kPaged) valid = (pg == P - 1) ? tail : S;
       else valid = min(S, total_tok - pg * S);
       const int v16 = min(kUnitTokens, valid - sb * kUnitTokens);
-      const uint32_t kt = smem_addr(my_ring + slot * kSlotBytes), vt = kt + 2 * kBoxBytes;
+      const uint32_t kt = smem_addr(my_ring + slot * kSlotBytes), vt = kt + kVOff;
 
       if (v16 > 0) {
         if (v16 < kUnitTokens) {
           // padding tokens: their V rows may hold anything, and 0 * NaN must not reach the accumulators
-          unsigned char* vrows = my_ring + slot * kSlotBytes + 2 * kBoxBytes;
+          unsigned char* vrows = my_ring + slot * kSlotBytes + kVOff;
           for (int i = lane; i < (kUnitTokens - v16) * 16; i += 32) {
             const int t = v16 + (i >> 4), ch = i & 15;
-            *reinterpret_cast<uint4*>(vrows + tile_offset(t, ch)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(vrows + tile_offset(t, ch, kHalf)) = make_uint4(0, 0, 0, 0);
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordered before the slot's next TMA fill
           __syncwarp();
@@ -373,7 +385,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt) {
             uint32_t r[4];
-            ldmatrix_x4(r, kt + tile_offset(8 * nt + (lane & 7), 4 * s4 + (lane >> 3)));
+            ldmatrix_x4(r, kt + tile_offset(8 * nt + (lane & 7), 4 * s4 + (lane >> 3), kHalf));
             mma_bf16(sacc[nt], qa[2 * s4][0], 0u, qa[2 * s4][1], 0u, r[0], r[1]);
             mma_bf16(sacc[nt], qa[2 * s4 + 1][0], 0u, qa[2 * s4 + 1][1], 0u, r[2], r[3]);
           }
@@ -411,7 +423,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
           uint32_t r[4];
-          ldmatrix_x4_trans(r, vt + tile_offset(((lane >> 4) & 1) * 8 + (lane & 7), 2 * mt + ((lane >> 3) & 1)));
+          ldmatrix_x4_trans(r, vt + tile_offset(((lane >> 4) & 1) * 8 + (lane & 7), 2 * mt + ((lane >> 3) & 1), kHalf));
           mma_bf16(acc[mt], r[0], r[1], r[2], r[3], b0h, b1h);
           mma_bf16(acc[mt], r[0], r[1], r[2], r[3], b0l, b1l);
         }
@@ -598,13 +610,14 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 tensor of `rows` token rows x 128 coordinates at `base`; boxes of 16 rows x 64 coordinates, 128-byte swizzle
-cudaError_t make_row_map(CUtensorMap* map, const void* base, long long rows) {
+// bf16 tensor of `rows` token rows x 128 coordinates at `base`; boxes of `box_rows` rows x 64 coordinates,
+// 128-byte swizzle
+cudaError_t make_row_map(CUtensorMap* map, const void* base, long long rows, int box_rows = kUnitTokens) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
   const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)kUnitTokens};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -665,7 +678,7 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
   if (paged) {
     const long long rows = geo.n_pool_pages * geo.Hkv * 2 * geo.S;
     if (rows >= (1LL << 31)) return cudaErrorInvalidValue;
-    e = make_row_map(&mk, a.kv_pool, rows);
+    e = make_row_map(&mk, a.kv_pool, rows, geo.S == kUnitTokens ? 2 * kUnitTokens : kUnitTokens);   // 16-token pages: K and V in one box
     mv = mk;
   } else {
     const long long rows = (long long)geo.B * geo.Hq * geo.k * geo.S;
