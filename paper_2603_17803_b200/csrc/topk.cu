@@ -107,6 +107,16 @@ __device__ __forceinline__ int hist_slot(uint32_t bin) {
   return (int)((idx % PER) * THREADS + idx / PER);
 }
 
+// Sum of the totals of the warps before `warp` (THREADS / 32 <= 32 totals in shared memory): every warp reduces
+// the masked totals with shuffles instead of each thread adding them up one by one.
+template <int THREADS>
+__device__ __forceinline__ int totals_before(const int* warp_tot, int warp, int lane) {
+  int v = (lane < THREADS / 32 && lane < warp) ? warp_tot[lane] : 0;
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
 // After the histogram of the current level is complete: locate the bin holding rank `remaining`
 // from the top, narrow (base, bits, remaining), clear the histogram.  All threads call it.
 template <int THREADS>
@@ -129,8 +139,7 @@ __device__ __forceinline__ void narrow(SelectState& st, int tid, int shift) {
   const uint32_t base = st.base;
   const int remaining = st.remaining;
   __syncthreads();
-  int above = incl - sum;
-  for (int w2 = 0; w2 < warp; ++w2) above += st.warp_tot[w2];
+  int above = incl - sum + totals_before<THREADS>(st.warp_tot, warp, lane);
 #pragma unroll
   for (int j = 0; j < PER; ++j) st.hist[j * THREADS + tid] = 0;
   if (above < remaining && remaining <= above + sum) {
@@ -295,8 +304,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   __syncthreads();                                          // warp_tot may still be read by narrow()
   if (lane == 31) st.warp_tot[warp] = incl;
   __syncthreads();
-  int before = incl - cnt;
-  for (int w2 = 0; w2 < warp; ++w2) before += st.warp_tot[w2];
+  const int before = incl - cnt + totals_before<THREADS>(st.warp_tot, warp, lane);
   int gt_before = before & 0xFFFF, eq_before = before >> 16;
   unsigned picked = 0u;                                     // bit j: page p0 + j is selected
 #pragma unroll
