@@ -65,11 +65,11 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
 }
 
 int pick_splits(const swarm_ctx* ctx, bool paged, bool fused = false) {
-  // About 1 CTA of 8 warps per SM on 148 SMs (what the shared-memory rings allow), at most kMaxSplits; for gathered
+  // About 1 CTA of 8 warps per SM (what the shared-memory rings allow), at most kMaxSplits; for gathered
   // buffers at least 4 pages per split.  Inside the fused step one SM is left for the resolution CTA.
   if (ctx->user_splits > 0) return ctx->user_splits;
   const int64_t groups = attention_groups(ctx->geo, paged);
-  int64_t n = (fused ? 147 : 148) / groups;
+  int64_t n = (sm_count() - (fused ? 1 : 0)) / groups;
   if (!paged) n = std::min<int64_t>(n, std::max(1, ctx->geo.k / 4));
   n = std::min<int64_t>(n, kMaxSplits);
   return (int)std::max<int64_t>(n, 1);

@@ -30,6 +30,9 @@ namespace {
 
 constexpr int kScoreWarps = 4;
 int g_sm_count = 148;                                      // set by configure_score()
+}  // namespace
+int sm_count() { return g_sm_count; }
+namespace {
 
 __host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
 

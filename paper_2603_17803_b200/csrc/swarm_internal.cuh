@@ -39,6 +39,7 @@ struct Geometry {   // plain copy of the shape in kernel-friendly form
 
 // ---- one-time per-device kernel attribute set-up (dynamic shared-memory limits) ---------------
 cudaError_t configure_score();
+int sm_count();         // SMs of the device current at configure_score() (148 on B200)
 cudaError_t configure_topk();
 cudaError_t configure_resolve();
 cudaError_t configure_attention();
