@@ -260,6 +260,15 @@ def run_swarm(args):
         attn_us = time_loop(lambda s: s.sparse_attn_paged(stream=stream, reuse_last_selection=True), n_loop)
         select_us = time_loop(lambda s: s.select(stream=stream), n_loop)
         resolve_us = time_loop(lambda s: s.resolve(stream=stream), n_loop)
+        # the same step with the paper's own selector (medoid index, whole clusters retrieved): k_c clusters of
+        # ~8 pages stand for the page step's top_k pages
+        k_c = max(1, cfg.top_k // 8)
+        for s_ in sessions:
+            s_.enable_medoid_index(k_c)
+        medoid_us = time_loop(lambda s: s.step_medoid(stream=stream), n_loop)
+        for s_ in sessions:
+            s_.step(stream=stream)                       # leave the page step's outputs in place for the checks below
+        stream.synchronize()
         t_d = time.perf_counter()
 
         # end to end: per-step data in pinned host memory, copies inside the timed region
@@ -311,6 +320,8 @@ def run_swarm(args):
         "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
         "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
         "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
+        "medoid_step": {"us_per_step": medoid_us, "top_k_clusters": k_c,
+                        "note": "swarm_step_medoid on the same data sets: clusters scored by their medoid page, whole clusters attended"},
         "roofline": {"kernel": "attn_kernel<paged> (tensor-core split-K attention over the union of selected pages, merge included)", "bound": "hbm", "achieved": attn_gbs,
                      "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
                      "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU if cfg.name == "c2_128k" else None,
