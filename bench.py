@@ -46,6 +46,7 @@ def parse_args():
     ap.add_argument("--n-rot", type=int, default=8, help="independent data sets rotated through")
     ap.add_argument("--no-graph", action="store_true", help="call the library directly instead of replaying graphs")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--attn-splits", type=int, default=0, help="key-range splits of the attention kernel (0: chosen from the shape)")
     return ap.parse_args()
 
 
@@ -156,6 +157,7 @@ def run_swarm(args):
     from paper_2603_17803_b200 import replicas
     from paper_2603_17803_b200 import workloads as W
     from paper_2603_17803_b200.session import Session
+    from paper_2603_17803_b200 import binding as B
 
     world, rank, local_rank = replicas.env_world()
     if not torch.cuda.is_available():
@@ -176,6 +178,8 @@ def run_swarm(args):
         w = W.generate(cfg, seed=replicas.replica_seed(rank, r), device=dev, step=r)
         workloads.append(w)
         sessions.append(Session(w))
+        if args.attn_splits > 0:
+            B.swarm_set_attn_splits(sessions[-1].ctx, args.attn_splits)
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()
 
