@@ -283,7 +283,7 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swar
  *   stop        when every entry is covered.
  * Outputs: clusters in creation order as cluster_ptr [n + 1] (only n_clusters + 1 entries are written) and
  * cluster_members (joining order, medoid first), medoid [n] (n_clusters written), n_clusters [1],
- * dev_status [1] = 0, or 1 if cluster_members (members_cap entries, at least n) was too small -- the output is
+ * dev_status [1] = 0, or 1 if cluster_members (members_cap entries, at least n, below 2^31) was too small -- the output is
  * then incomplete.  n <= 32768.  workspace: swarm_build_clusters_workspace_bytes(n) bytes (< 0: minus an error code). */
 int64_t swarm_build_clusters_workspace_bytes(int32_t n_entries);
 int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, void* workspace, int64_t workspace_bytes,

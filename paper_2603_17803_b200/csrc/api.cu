@@ -254,7 +254,8 @@ int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, vo
                              int32_t* density, int32_t* cluster_ptr, int32_t* cluster_members, int64_t members_cap,
                              int32_t* medoid, int32_t* n_clusters, int32_t* dev_status, void* stream) {
   if (n_entries < 1 || !(tau >= 0.f) || bad(dist) || bad(workspace) || bad(density) || bad(cluster_ptr) ||
-      bad(cluster_members) || bad(medoid) || bad(n_clusters) || bad(dev_status) || members_cap < n_entries)
+      bad(cluster_members) || bad(medoid) || bad(n_clusters) || bad(dev_status) || members_cap < n_entries ||
+      members_cap > 0x7FFFFFFFLL)                            // cluster_ptr holds 32-bit offsets
     return SWARM_ERR_INVALID_ARG;
   if (n_entries > 32768) return SWARM_ERR_UNSUPPORTED;
   if (workspace_bytes < build_clusters_workspace_bytes(n_entries)) return SWARM_ERR_WORKSPACE_TOO_SMALL;
