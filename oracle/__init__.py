@@ -350,3 +350,20 @@ def build_clusters(dist, tau, members_cap=None):
                                          _p(members), ctypes.c_int64(cap), _p(medoid), _p(n_c)), "build_clusters")
     C = int(n_c[0])
     return rho, ptr[:C + 1].copy(), members[:int(ptr[C])].copy(), medoid[:C].copy()
+
+
+# ---- placement of the clusters' entries across the SSDs (Eq. 7) and entry-level scheduling --------------------
+def entry_replica_masks(cluster_ptr, cluster_members, n_entries, D):
+    """Round-robin placement of Eq. 7: clusters are laid out one after another, a global pointer advances by one
+    disk per stored entry, so the j-th entry of cluster i lands on disk (|C_0| + ... + |C_{i-1}| + j) mod D.
+    An entry stored with several clusters has one copy per cluster; returns, per entry, the set of disks holding
+    a copy as a bit mask (uint32 [n_entries])."""
+    cluster_ptr, cluster_members = np.asarray(cluster_ptr), np.asarray(cluster_members)
+    masks = np.zeros(n_entries, dtype=np.uint32)
+    p_global = 0
+    for c in range(len(cluster_ptr) - 1):
+        disk = p_global % D                                  # id_i of Eq. 7
+        for j in range(int(cluster_ptr[c]), int(cluster_ptr[c + 1])):
+            masks[int(cluster_members[j])] |= np.uint32(1 << ((disk + (j - int(cluster_ptr[c]))) % D))
+        p_global += int(cluster_ptr[c + 1] - cluster_ptr[c])
+    return masks

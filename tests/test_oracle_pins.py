@@ -731,3 +731,25 @@ def test_algorithm1_replay_in_exact_arithmetic():
         assert got == clusters and list(medoid) == meds
         assert set(members.tolist()) == set(range(n))                       # every entry is covered
         assert any(members.tolist().count(e) > 1 for e in range(n))         # and some sit in several clusters
+
+
+# ------------------------------------------------------------------------------- Eq. 7 placement of entries
+
+def test_entry_placement_hand_case_and_round_robin():
+    # clusters [2 0 1] and [3 4 2] on 4 disks: entries land on disks 0 1 2 | 3 0 1; entry 2 has copies on 0 and 1
+    masks = oracle.entry_replica_masks([0, 3, 6], [2, 0, 1, 3, 4, 2], 5, 4)
+    assert list(masks) == [0b0010, 0b0100, 0b0011, 0b1000, 0b0001]
+    # without replicas every entry has one copy and the disks fill evenly
+    rng = np.random.default_rng(51)
+    sizes = rng.integers(1, 9, size=40)
+    ptr = np.concatenate([[0], np.cumsum(sizes)])
+    members = rng.permutation(int(ptr[-1]))
+    D = 6
+    masks = oracle.entry_replica_masks(ptr, members, int(ptr[-1]), D)
+    assert all(bin(int(m)).count("1") == 1 for m in masks)
+    per_disk = np.bincount([int(m).bit_length() - 1 for m in masks], minlength=D)
+    assert per_disk.max() - per_disk.min() <= 1
+    # each cluster's entries sit on consecutive disks (wrap-around), starting where the previous cluster stopped
+    for c in range(len(sizes)):
+        disks = [int(masks[e]).bit_length() - 1 for e in members[ptr[c]:ptr[c + 1]]]
+        assert disks == [(int(ptr[c]) + j) % D for j in range(int(sizes[c]))]
