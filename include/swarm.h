@@ -123,6 +123,12 @@ typedef struct swarm_medoid_index {
                                     /* medoid page, written by swarm_build_medoid_index                               */
   const int64_t* cluster_page_ptr;  /* [n_clusters + 1] start of each cluster's members in cluster_pages               */
   const int32_t* cluster_pages;     /* member pages of the clusters, ids local to the request                          */
+  const uint32_t* entry_replica_mask; /* NULL: the selected clusters are scheduled as units (cluster tables of the     */
+                                    /* inputs).  Otherwise entry-level scheduling, the paper's exact model (Sec. 5.1    */
+                                    /* with the placement of Eq. 7): [n_pool_pages] queues holding a copy of each page; */
+                                    /* see swarm_step_medoid                                                            */
+  int64_t n_member_entries;         /* length of cluster_pages: offsets in cluster_page_ptr beyond it set               */
+                                    /* SWARM_DEV_BAD_CLUSTER and the cluster is skipped                                 */
   int32_t top_k_clusters;           /* k_c clusters kept per query head                                                */
   int32_t max_clusters_per_req;     /* upper bound on the clusters of one request (<= max_pages_per_req); row pitch    */
                                     /* of the cluster scores                                                           */
@@ -266,6 +272,12 @@ int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, con
  *   uniq, queue_of, n_uniq, queue_load: as in swarm_step for the union of the selected clusters
  *   out, lse: Eq. 1 of every head over ALL pages of its selected clusters (clusters are the retrieval unit)
  * outputs->scores (optional) is [B][Hq][max_clusters_per_req]; k_out, v_out and n_tok must be NULL.
+ * Entry-level scheduling (index->entry_replica_mask given): the I/O set of Eq. 8 is the union of the member
+ * PAGES of all selected clusters; each page is one unit of weight 1 with replica set entry_replica_mask[pool
+ * page] (a page stored with several clusters has several copies).  uniq then holds pool page ids
+ * (page_base[b] + page), queue_of / queue_load / the submission order refer to pages, the cluster tables of the
+ * inputs and the cache state are not used by the scheduling, and the ctx must have been created with
+ * max_clusters_total >= n_pool_pages (SWARM_ERR_INVALID_ARG otherwise; uniq and queue_of sized accordingly).
  * A member page outside the request sets SWARM_DEV_BAD_PAGE and is skipped.  The local window of the shape
  * is not applied.  Page bitmaps longer than 160 KiB per head (1.3 M pages) are SWARM_ERR_UNSUPPORTED. */
 int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_medoid_index* index,

@@ -478,8 +478,9 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
       bad(idx->medoid_ksum) || bad(idx->cluster_page_ptr) || bad(idx->cluster_pages) || o == nullptr || bad(o->sel) ||
       bad(o->n_sel) || bad(o->uniq) || bad(o->queue_of) || bad(o->n_uniq) || bad(o->queue_load) || bad(o->out) ||
       bad(o->lse) || (o->scores && !aligned16(o->scores)) || o->k_out != nullptr || o->v_out != nullptr ||
-      o->n_tok != nullptr || idx->top_k_clusters < 1 || idx->max_clusters_per_req < 1 ||
-      idx->max_clusters_per_req > ctx->geo.Pmax)
+      o->n_tok != nullptr || idx->top_k_clusters < 1 || idx->n_member_entries < 0 || idx->max_clusters_per_req < 1 ||
+      idx->max_clusters_per_req > ctx->geo.Pmax ||
+      (idx->entry_replica_mask != nullptr && (!aligned16(idx->entry_replica_mask) || ctx->geo.Cmax < ctx->geo.n_pool_pages)))
     return SWARM_ERR_INVALID_ARG;
   if (selmap_pitch_bytes(ctx->geo.Pmax) > kMaxExpandRowBytes ||
       (int64_t)ctx->geo.B * ctx->geo.Hq * idx->top_k_clusters >= (int64_t(1) << 31))
@@ -503,10 +504,19 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
   SWARM_TRY(launch_expand_clusters(ctx->geo, idx->top_k_clusters, o->sel, o->n_sel, in->cluster_base,
                                    idx->cluster_page_ptr, idx->cluster_pages, in->ctx_len,
                                    ws_ptr<uint8_t>(ctx, ctx->lay.selmap), ws_ptr<uint8_t>(ctx, ctx->lay.flags), status, st,
-                                   true));
+                                   true, idx->entry_replica_mask != nullptr ? in->page_base : nullptr,
+                                   idx->n_member_entries));
   AttnArgs a = paged_args(ctx, in, o->out, o->lse);
   a.n_splits = pick_splits(ctx, true, /*fused=*/true);
-  const ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  if (idx->entry_replica_mask != nullptr) {
+    // entry-level scheduling: the units are the pool pages, every one of weight 1, each with its own replica set
+    rs.cluster_base = in->page_base;
+    rs.replica_mask = idx->entry_replica_mask;
+    rs.cluster_size = nullptr;
+    rs.geo.flags |= SWARM_UNIT_LOAD;
+    rs.has_cache = false;
+  }
   SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, &rs));
   return SWARM_OK;
 }

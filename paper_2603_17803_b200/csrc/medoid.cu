@@ -55,7 +55,7 @@ expand_clusters_kernel(Geometry geo, int k_c, int pitch, const int32_t* __restri
                        const int32_t* __restrict__ n_sel_c, const int64_t* __restrict__ cluster_base,
                        const int64_t* __restrict__ cluster_page_ptr, const int32_t* __restrict__ cluster_pages,
                        const int32_t* __restrict__ ctx_len, uint8_t* __restrict__ selmap, uint8_t* __restrict__ flags,
-                       uint32_t* __restrict__ status) {
+                       uint32_t* __restrict__ status, const int64_t* __restrict__ entry_base, long long n_member_entries) {
   extern __shared__ uint32_t s_row[];
   const int bh = blockIdx.x, b = bh / geo.Hq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -69,12 +69,22 @@ expand_clusters_kernel(Geometry geo, int k_c, int pitch, const int32_t* __restri
   for (int j = warp; j < n; j += blockDim.x / 32) {         // one warp per selected cluster
     const int c = sel_c[(long long)bh * k_c + j];
     if (c < 0 || c >= cn - cb || cb + c >= geo.Cmax) { err |= SWARM_DEV_BAD_CLUSTER; continue; }
-    if (lane == 0) flags[cb + c] = 1;
     const long long e0 = cluster_page_ptr[cb + c], e1 = cluster_page_ptr[cb + c + 1];
+    if (e0 < 0 || e1 < e0 || e1 > n_member_entries) { err |= SWARM_DEV_BAD_CLUSTER; continue; }   // corrupt member offsets
+    // what gets scheduled: the cluster as a whole, or (entry level) each of its pages on its own
+    if (lane == 0 && entry_base == nullptr) flags[cb + c] = 1;
     for (long long e = e0 + lane; e < e1; e += 32) {
       const int p = cluster_pages[e];
-      if (p < 0 || p >= P || p >= pitch * 8) err |= SWARM_DEV_BAD_PAGE;
-      else atomicOr(&s_row[p >> 5], 1u << (p & 31));
+      if (p < 0 || p >= P || p >= pitch * 8) {
+        err |= SWARM_DEV_BAD_PAGE;
+      } else {
+        atomicOr(&s_row[p >> 5], 1u << (p & 31));
+        if (entry_base != nullptr) {
+          const long long unit = entry_base[b] + p;
+          if (unit < geo.Cmax) flags[unit] = 1;
+          else err |= SWARM_DEV_BAD_CLUSTER;
+        }
+      }
     }
   }
   if (err) atomicOr(status, err);
@@ -105,11 +115,12 @@ cudaError_t launch_cluster_len(const Geometry& geo, const int64_t* cluster_base,
 cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* sel_c, const int32_t* n_sel_c,
                                    const int64_t* cluster_base, const int64_t* cluster_page_ptr,
                                    const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
-                                   uint32_t* status, cudaStream_t st, bool overlap) {
+                                   uint32_t* status, cudaStream_t st, bool overlap, const int64_t* entry_base,
+                                   long long n_member_entries) {
   const int pitch = selmap_pitch_bytes(geo.Pmax);
   return launch_pdl(expand_clusters_kernel, dim3((unsigned)(geo.B * geo.Hq)), dim3(256), (size_t)pitch, st, overlap, geo,
                     k_c, pitch, sel_c, n_sel_c, cluster_base, cluster_page_ptr, cluster_pages, ctx_len, selmap, flags,
-                    status);
+                    status, entry_base, n_member_entries);
 }
 
 }  // namespace swarm

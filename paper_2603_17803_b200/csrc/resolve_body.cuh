@@ -162,7 +162,7 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       if (with_flags) r.f = __ldcg(f1 + v);
       if (v * 4 + 4 <= C) {
         r.mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v * 4));
-        r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));
+        if (!unit) r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));   // no size table needed for unit loads
       } else {
         uint32_t* mk = &r.mk.x;
         uint32_t* sz = &r.sz.x;
@@ -170,7 +170,7 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
         for (int j = 0; j < 4; ++j) {
           if (v * 4 + j < C) {
             mk[j] = replica_mask[v * 4 + j];
-            sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
+            if (!unit) sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
           }
         }
       }

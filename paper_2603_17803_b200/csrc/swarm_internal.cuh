@@ -134,7 +134,8 @@ cudaError_t launch_cluster_len(const Geometry& geo, const int64_t* cluster_base,
 cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* sel_c, const int32_t* n_sel_c,
                                    const int64_t* cluster_base, const int64_t* cluster_page_ptr,
                                    const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
-                                   uint32_t* status, cudaStream_t st, bool overlap);
+                                   uint32_t* status, cudaStream_t st, bool overlap, const int64_t* entry_base,
+                                   long long n_member_entries);
 
 // Algorithm 1 (offline co-activation clustering): see cluster.cu.
 long long build_clusters_workspace_bytes(int n);

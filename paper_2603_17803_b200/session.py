@@ -33,7 +33,8 @@ class Session:
     """One ctx bound to one resident KV pool (``workload`` tensors must live on a CUDA device)."""
 
     def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
-                 ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0):
+                 ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0,
+                 max_clusters_total: Optional[int] = None):
         cfg = workload.cfg
         self.cfg = cfg
         self.w = workload
@@ -44,7 +45,7 @@ class Session:
         self.Pmax = cfg.max_pages()
         self.shape = B.make_shape(batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                                   page_size=cfg.page_size, top_k=cfg.top_k, n_queues=cfg.n_queues,
-                                  max_pages_per_req=self.Pmax, max_clusters_total=max(1, workload.n_clusters),
+                                  max_pages_per_req=self.Pmax, max_clusters_total=max(1, workload.n_clusters, max_clusters_total or 0),
                                   n_pool_pages=workload.n_pool_pages, flags=flags,
                                   local_window_pages=local_window_pages)
         self.ctx = B.swarm_create(self.shape)
@@ -60,8 +61,8 @@ class Session:
         self.o = StepOutputs(
             scores=torch.full((Bq, Hq, self.Pmax), float("-inf"), dtype=torch.float32, device=dev) if keep_scores else None,
             sel=torch.empty((Bq, Hq, k), **i32), n_sel=torch.empty((Bq, Hq), **i32),
-            uniq=torch.empty(max(1, workload.n_clusters), **i32),
-            queue_of=torch.empty(max(16, workload.n_clusters), dtype=torch.uint8, device=dev),
+            uniq=torch.empty(max(1, workload.n_clusters, max_clusters_total or 0), **i32),
+            queue_of=torch.empty(max(16, workload.n_clusters, max_clusters_total or 0), dtype=torch.uint8, device=dev),
             n_uniq=torch.zeros(4, **i32), queue_load=torch.zeros(max(4, cfg.n_queues), **i32),
             k_out=torch.empty((Bq, Hq, k * S, d), dtype=torch.bfloat16, device=dev) if keep_gathered else None,
             v_out=torch.empty((Bq, Hq, k * S, d), dtype=torch.bfloat16, device=dev) if keep_gathered else None,
@@ -138,7 +139,7 @@ class Session:
     def enable_submit_order(self) -> None:
         """Attaches the outputs of the batched submission order (indices into uniq, and [batches, submitted])."""
         i32 = dict(dtype=torch.int32, device=self.device)
-        self.submit_order = torch.full((max(4, self.w.n_clusters),), -1, **i32)
+        self.submit_order = torch.full((max(4, self.o.uniq.numel()),), -1, **i32)
         self.submit_info = torch.zeros(4, **i32)
         B.swarm_set_submit_order(self.ctx, self.submit_order, self.submit_info)
 

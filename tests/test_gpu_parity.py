@@ -539,6 +539,10 @@ def test_medoid_step_rejects_bad_arguments_and_flags_bad_members():
     sess.step_medoid()
     torch.cuda.synchronize()
     assert sess.status() & B.DEV_BAD_PAGE
+    sess.cluster_page_ptr.fill_(1 << 40)                    # member offsets beyond the member array: skipped
+    sess.step_medoid()
+    torch.cuda.synchronize()
+    assert sess.status() & B.DEV_BAD_CLUSTER
     sess.close()
 
 
@@ -699,5 +703,39 @@ def test_algorithm1_clusters_drive_the_medoid_step():
     k_g, v_g, n_tok = oracle.gather(W.bits_u16(w.kv_pool), sel_p, n_sel_p, tabs["page_base"], tabs["ctx_len"],
                                     cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
     out, lse = oracle.attention(W.bits_u16(w.q), k_g, v_g, n_tok)
+    parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
+    sess.close()
+
+    # entry-level scheduling (the paper's exact model): every page of the selected clusters is a unit of its own,
+    # with the copies Eq. 7 gives it -- one per cluster that stores it
+    entry_masks = oracle.entry_replica_masks(ptr.cpu().numpy(), members.cpu().numpy(), P, cfg.n_queues)
+    assert (np.array([bin(int(x)).count("1") for x in entry_masks]) > 1).any()
+    sess = Session(w, max_clusters_total=P)
+    sess.medoid_ksum = torch.empty((C, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=DEV)
+    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum)
+    masks_dev = torch.from_numpy(entry_masks.view(np.int32)).to(DEV)
+    ptr64 = ptr.to(torch.int64)                               # kept alive: the index holds its address
+    index = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=ptr64, cluster_pages=members,
+                                top_k_clusters=k_c, max_clusters_per_req=C, entry_replica_mask=masks_dev)
+    sel_c2 = torch.empty((1, cfg.n_q_heads, k_c), **i32)
+    n_sel_c2 = torch.empty((1, cfg.n_q_heads), **i32)
+    o = sess.o
+    outs = B.make_outputs(sel=sel_c2, n_sel=n_sel_c2, uniq=o.uniq, queue_of=o.queue_of, n_uniq=o.n_uniq,
+                          queue_load=o.queue_load, out=o.out, lse=o.lse)
+    sess.enable_submit_order()
+    B.swarm_step_medoid(sess.ctx, sess.inputs, index, outs)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    assert np.array_equal(sel_c2.cpu().numpy(), sel_c)        # same selection as before
+    ones = np.ones(P, dtype=np.uint16)
+    ident_p = np.arange(P, dtype=np.int32)
+    uniq, queue_of, load = oracle.resolve(sel_p, n_sel_p, tabs["page_base"], ident_p, tabs["page_base"], entry_masks, ones,
+                                          cfg.n_queues, oracle.UNIT_LOAD)
+    n = int(o.n_uniq.cpu().numpy()[0])
+    assert n == len(uniq) and np.array_equal(o.uniq.cpu().numpy()[:n], uniq)
+    assert np.array_equal(o.queue_of.cpu().numpy()[:n], queue_of)
+    assert np.array_equal(o.queue_load.cpu().numpy()[: cfg.n_queues], load) and int(load.sum()) == n
+    want_order, rounds = oracle.submit_order(queue_of, entry_masks[uniq], cfg.n_queues)
+    assert np.array_equal(sess.submit_order.cpu().numpy()[:n], want_order)
     parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
     sess.close()
