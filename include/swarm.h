@@ -127,6 +127,8 @@ typedef struct swarm_medoid_index {
                                     /* inputs).  Otherwise entry-level scheduling, the paper's exact model (Sec. 5.1    */
                                     /* with the placement of Eq. 7): [n_pool_pages] queues holding a copy of each page; */
                                     /* see swarm_step_medoid                                                            */
+  const int32_t* cluster_ctx_len;   /* [B] clusters of request b x page_size (the index seen as a context of its own), */
+                                    /* written by swarm_build_medoid_index                                              */
   int64_t n_member_entries;         /* length of cluster_pages: offsets in cluster_page_ptr beyond it set               */
                                     /* SWARM_DEV_BAD_CLUSTER and the cluster is skipped                                 */
   int32_t top_k_clusters;           /* k_c clusters kept per query head                                                */
@@ -259,10 +261,10 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outpu
 
 /* Index build for swarm_step_medoid (not part of a decode step): copies, for every cluster, the key summary of
  * its medoid page medoid_page[cluster] (page id local to the request) into row `cluster` of medoid_ksum_out
- * (bf16 [max_clusters_total][Hkv][2][d]).  Reads inputs->ksum, page_base, cluster_base.  Which member is the
- * medoid is decided offline (Algorithm 1) and is an input here. */
+ * (bf16 [max_clusters_total][Hkv][2][d]), and writes cluster_ctx_len_out [B] (int32).  Reads inputs->ksum,
+ * page_base, cluster_base.  Which member is the medoid is decided offline (Algorithm 1) and is an input here. */
 int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* medoid_page,
-                                 void* medoid_ksum_out, void* stream);
+                                 void* medoid_ksum_out, int32_t* cluster_ctx_len_out, void* stream);
 
 /* The decode step with the paper's own selector (Sec. 4.2 Tier 1 (1), Sec. 4.1): clusters, not pages, are
  * scored and retrieved.

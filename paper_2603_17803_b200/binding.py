@@ -105,7 +105,7 @@ def _check(rc: int, what: str, ctx=None):
 class swarm_medoid_index(ctypes.Structure):
     _fields_ = [("medoid_ksum", ctypes.c_void_p), ("cluster_page_ptr", ctypes.c_void_p),
                 ("cluster_pages", ctypes.c_void_p), ("entry_replica_mask", ctypes.c_void_p),
-                ("n_member_entries", ctypes.c_int64), ("top_k_clusters", ctypes.c_int32),
+                ("cluster_ctx_len", ctypes.c_void_p), ("n_member_entries", ctypes.c_int64), ("top_k_clusters", ctypes.c_int32),
                 ("max_clusters_per_req", ctypes.c_int32)]
 
 
@@ -265,17 +265,18 @@ def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -
            "swarm_step", ctx)
 
 
-def make_medoid_index(*, medoid_ksum, cluster_page_ptr, cluster_pages, top_k_clusters,
+def make_medoid_index(*, medoid_ksum, cluster_page_ptr, cluster_pages, cluster_ctx_len, top_k_clusters,
                       max_clusters_per_req, entry_replica_mask=None) -> swarm_medoid_index:
     return swarm_medoid_index(_ptr(medoid_ksum, "medoid_ksum"), _ptr(cluster_page_ptr, "cluster_page_ptr"),
                               _ptr(cluster_pages, "cluster_pages"), _ptr(entry_replica_mask, "entry_replica_mask"),
-                              int(cluster_pages.numel()), top_k_clusters, max_clusters_per_req)
+                              _ptr(cluster_ctx_len, "cluster_ctx_len"), int(cluster_pages.numel()), top_k_clusters, max_clusters_per_req)
 
 
 def swarm_build_medoid_index(ctx, inputs: swarm_inputs, medoid_page: torch.Tensor, medoid_ksum_out: torch.Tensor,
-                             stream=None) -> None:
+                             cluster_ctx_len_out: torch.Tensor, stream=None) -> None:
     _check(load_library().swarm_build_medoid_index(ctx, ctypes.byref(inputs), _ptr(medoid_page, "medoid_page"),
-                                                   _ptr(medoid_ksum_out, "medoid_ksum_out"), _stream(stream)),
+                                                   _ptr(medoid_ksum_out, "medoid_ksum_out"),
+                                                   _ptr(cluster_ctx_len_out, "cluster_ctx_len_out"), _stream(stream)),
            "swarm_build_medoid_index", ctx)
 
 

@@ -458,12 +458,13 @@ struct HostStepKey {
 static_assert(sizeof(HostStepKey) <= 256, "host_key too small");
 
 int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* medoid_page,
-                                 void* medoid_ksum_out, void* stream) {
+                                 void* medoid_ksum_out, int32_t* cluster_ctx_len_out, void* stream) {
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (in == nullptr || bad(in->ksum) || bad(in->page_base) || bad(in->cluster_base) || bad(medoid_page) ||
-      bad(medoid_ksum_out))
+      bad(medoid_ksum_out) || bad(cluster_ctx_len_out))
     return SWARM_ERR_INVALID_ARG;
+  SWARM_TRY(launch_cluster_len(ctx->geo, in->cluster_base, cluster_ctx_len_out, static_cast<cudaStream_t>(stream)));
   SWARM_TRY(launch_medoid_rows(ctx->geo, static_cast<const uint16_t*>(in->ksum), in->page_base, in->cluster_base,
                                medoid_page, static_cast<uint16_t*>(medoid_ksum_out),
                                ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
@@ -475,7 +476,8 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (in == nullptr || bad(in->q) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || idx == nullptr ||
-      bad(idx->medoid_ksum) || bad(idx->cluster_page_ptr) || bad(idx->cluster_pages) || o == nullptr || bad(o->sel) ||
+      bad(idx->medoid_ksum) || bad(idx->cluster_page_ptr) || bad(idx->cluster_pages) || bad(idx->cluster_ctx_len) ||
+      o == nullptr || bad(o->sel) ||
       bad(o->n_sel) || bad(o->uniq) || bad(o->queue_of) || bad(o->n_uniq) || bad(o->queue_load) || bad(o->out) ||
       bad(o->lse) || (o->scores && !aligned16(o->scores)) || o->k_out != nullptr || o->v_out != nullptr ||
       o->n_tok != nullptr || idx->top_k_clusters < 1 || idx->n_member_entries < 0 || idx->max_clusters_per_req < 1 ||
@@ -488,7 +490,7 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint32_t* status = ws_ptr<uint32_t>(ctx, ctx->lay.status);
   float* sc = o->scores ? o->scores : ws_ptr<float>(ctx, ctx->lay.scores);
-  int32_t* len_c = ws_ptr<int32_t>(ctx, ctx->lay.n_tok);   // clusters of each request x page size
+  const int32_t* len_c = idx->cluster_ctx_len;             // clusters of each request x page size
 
   // the page kernels, run over the index: one "page" per cluster, requests laid out like cluster_base
   Geometry gc = ctx->geo;
@@ -496,7 +498,6 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
   gc.k = idx->top_k_clusters;
   gc.W = 0;
   gc.n_pool_pages = ctx->geo.Cmax;
-  SWARM_TRY(launch_cluster_len(ctx->geo, in->cluster_base, len_c, st));
   SWARM_TRY(launch_page_score(gc, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(idx->medoid_ksum),
                               in->cluster_base, len_c, sc, status, st));
   SWARM_TRY(launch_topk(gc, sc, len_c, o->sel, o->n_sel, status, st, true));

@@ -121,9 +121,11 @@ class Session:
         per_req = (w.cluster_base[1:] - w.cluster_base[:-1]).max().item()
         self.max_clusters_per_req = max(1, int(per_req))
         self.medoid_ksum = torch.empty((n_c, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
-        B.swarm_build_medoid_index(self.ctx, self.inputs, self.medoid_page, self.medoid_ksum)
+        self.cluster_ctx_len = torch.empty(max(4, cfg.batch), dtype=torch.int32, device=dev)
+        B.swarm_build_medoid_index(self.ctx, self.inputs, self.medoid_page, self.medoid_ksum, self.cluster_ctx_len)
         self.medoid_index = B.make_medoid_index(medoid_ksum=self.medoid_ksum, cluster_page_ptr=self.cluster_page_ptr,
-                                                cluster_pages=self.cluster_pages, top_k_clusters=top_k_clusters,
+                                                cluster_pages=self.cluster_pages, cluster_ctx_len=self.cluster_ctx_len,
+                                                top_k_clusters=top_k_clusters,
                                                 max_clusters_per_req=self.max_clusters_per_req)
         i32 = dict(dtype=torch.int32, device=dev)
         self.top_k_clusters = top_k_clusters

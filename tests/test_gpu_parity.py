@@ -531,7 +531,7 @@ def test_medoid_step_rejects_bad_arguments_and_flags_bad_members():
     with pytest.raises(B.SwarmError):                       # gathered outputs are not part of this step
         B.swarm_step_medoid(sess.ctx, sess.inputs, sess.medoid_index, sess.outputs)
     bad = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=sess.cluster_page_ptr,
-                              cluster_pages=sess.cluster_pages, top_k_clusters=0,
+                              cluster_pages=sess.cluster_pages, cluster_ctx_len=sess.cluster_ctx_len, top_k_clusters=0,
                               max_clusters_per_req=sess.max_clusters_per_req)
     with pytest.raises(B.SwarmError):
         B.swarm_step_medoid(sess.ctx, sess.inputs, bad, sess.medoid_outputs)
@@ -669,9 +669,11 @@ def test_algorithm1_clusters_drive_the_medoid_step():
     sess.cluster_page_ptr, sess.cluster_pages, sess.medoid_page = ptr.to(torch.int64), members, medoid
     sess.max_clusters_per_req = C
     sess.medoid_ksum = torch.empty((C, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=DEV)
-    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum)
+    sess.cluster_ctx_len = torch.empty(4, dtype=torch.int32, device=DEV)
+    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum, sess.cluster_ctx_len)
     sess.medoid_index = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=sess.cluster_page_ptr,
-                                            cluster_pages=members, top_k_clusters=k_c, max_clusters_per_req=C)
+                                            cluster_pages=members, cluster_ctx_len=sess.cluster_ctx_len,
+                                            top_k_clusters=k_c, max_clusters_per_req=C)
     i32 = dict(dtype=torch.int32, device=DEV)
     sess.sel_clusters = torch.empty((1, cfg.n_q_heads, k_c), **i32)
     sess.n_sel_clusters = torch.empty((1, cfg.n_q_heads), **i32)
@@ -712,10 +714,12 @@ def test_algorithm1_clusters_drive_the_medoid_step():
     assert (np.array([bin(int(x)).count("1") for x in entry_masks]) > 1).any()
     sess = Session(w, max_clusters_total=P)
     sess.medoid_ksum = torch.empty((C, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=DEV)
-    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum)
+    len_dev = torch.empty(4, dtype=torch.int32, device=DEV)
+    B.swarm_build_medoid_index(sess.ctx, sess.inputs, medoid, sess.medoid_ksum, len_dev)
     masks_dev = torch.from_numpy(entry_masks.view(np.int32)).to(DEV)
     ptr64 = ptr.to(torch.int64)                               # kept alive: the index holds its address
     index = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=ptr64, cluster_pages=members,
+                                cluster_ctx_len=len_dev,
                                 top_k_clusters=k_c, max_clusters_per_req=C, entry_replica_mask=masks_dev)
     sel_c2 = torch.empty((1, cfg.n_q_heads, k_c), **i32)
     n_sel_c2 = torch.empty((1, cfg.n_q_heads), **i32)
