@@ -743,3 +743,19 @@ def test_algorithm1_clusters_drive_the_medoid_step():
     assert np.array_equal(sess.submit_order.cpu().numpy()[:n], want_order)
     parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
     sess.close()
+
+
+def test_medoid_step_full_size_c3_and_wide_groups():
+    w = W.generate(W.CONFIGS["c3_batched"], seed=67, device=DEV)      # 16 requests, 256 clusters each
+    sess = Session(w)
+    sess.enable_medoid_index(16, keep_scores=True)
+    sess.step_medoid()
+    check_medoid_step(w, sess, 16)
+    sess.close()
+    for name in ("g16_s32", "hkv3_g2", "k1_d1"):                      # 16-head groups on 32-token pages, odd KV heads, one queue
+        w = W.generate(EDGE_SHAPES[name], seed=71, device=DEV)
+        sess = Session(w)
+        sess.enable_medoid_index(3, keep_scores=True)
+        sess.step_medoid()
+        check_medoid_step(w, sess, 3)
+        sess.close()
