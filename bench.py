@@ -270,8 +270,24 @@ def run_swarm(args):
         for s_ in sessions:
             s_.enable_medoid_index(k_c)
         medoid_us = time_loop(lambda s: s.step_medoid(stream=stream), n_loop)
+        # the page step with the optional parts of cluster resolution switched on, one at a time
+        cache_state = []
         for s_ in sessions:
-            s_.step(stream=stream)                       # leave the page step's outputs in place for the checks below
+            n_c = s_.w.n_clusters
+            g_ = torch.Generator(device="cpu").manual_seed(7)
+            cache_state.append(dict(resident=(torch.rand(n_c, generator=g_) < 0.25).to(torch.uint8).to(dev),
+                                    freq=torch.zeros(n_c, dtype=torch.int32, device=dev),
+                                    score=torch.zeros(n_c, dtype=torch.float32, device=dev),
+                                    n_hit=torch.zeros(4, dtype=torch.int32, device=dev)))
+            B.swarm_set_cache(s_.ctx, t_base=80.0, t_transfer=2.5, **cache_state[-1])
+        cached_us = time_loop(lambda s: s.step(stream=stream), n_loop)
+        for s_ in sessions:
+            B.swarm_set_cache(s_.ctx)
+            s_.enable_submit_order()
+        submit_us = time_loop(lambda s: s.step(stream=stream), n_loop)
+        for s_ in sessions:
+            B.swarm_set_submit_order(s_.ctx, None, None)
+            s_.step(stream=stream)                       # leave the plain page step's outputs in place for the checks below
         stream.synchronize()
         t_d = time.perf_counter()
 
@@ -324,6 +340,8 @@ def run_swarm(args):
         "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
         "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
         "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
+        "step_variants_us": {"with_cache_state(25% resident: Eq. 8 filter, counters, Eq. 6)": cached_us,
+                             "with_submission_order(Sec. 5.1 batches)": submit_us},
         "medoid_step": {"us_per_step": medoid_us, "top_k_clusters": k_c,
                         "note": "swarm_step_medoid on the same data sets: clusters scored by their medoid page, whole clusters attended"},
         "roofline": {"kernel": "attn_kernel<paged> (tensor-core split-K attention over the union of selected pages, merge included)", "bound": "hbm", "achieved": attn_gbs,
