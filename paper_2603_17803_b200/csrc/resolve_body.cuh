@@ -223,6 +223,10 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   // ones.  The clusters that need the serial pass are packed, in id order, into this warp's segment of the
   // item list, which starts at the warp's first output position (a segment cannot outgrow the warp's ids).
   const bool staged = n <= items_cap;
+  // submission order (optional): (replica class, queue) keys, kept in shared memory next to the items so that
+  // the ordering pass at the end does not have to read the results back from global memory
+  uint32_t* order_key = reinterpret_cast<uint32_t*>(s_items + items_cap);
+  const bool order_keys_early = r.submit_order != nullptr && staged;
   const int seg_base = before;
   int seg_len = 0;
   unsigned classes = 0u;
@@ -284,10 +288,12 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
         } else if (m == 0u || (m & ~valid_bits)) {
           err |= SWARM_DEV_BAD_REPLICA;
           queue_of[i] = 0xFF;
+          if (order_keys_early) order_key[i] = 0xFFFFFFFFu;
         } else {
           const int qd = __ffs(m) - 1;                     // a single replica: nothing to decide
           queue_of[i] = (uint8_t)qd;
           atomicAdd(&s_load[qd], (int)wgt);
+          if (order_keys_early) order_key[i] = 32u + (unsigned)qd;
         }
       }
     }
@@ -362,7 +368,10 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       __syncwarp();
       for (int k = lane; k < n; k += 32) {
         const uint4 item = s_items[k];
-        if (item.x != 0u) queue_of[item.z] = (uint8_t)item.w;
+        if (item.x != 0u) {
+          queue_of[item.z] = (uint8_t)item.w;
+          if (order_keys_early) order_key[item.z] = (by_id ? 0u : (unsigned)__popc(item.x) * 32u) + item.w;
+        }
       }
     }
     if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
@@ -386,10 +395,12 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
     uint32_t* rank_of = key_of + (staged ? items_cap : n);
     for (int i = tid; i < 33 * 32; i += kThreads) s_group[i] = 0;
     __syncthreads();                                       // also: every queue_of entry is written
-    for (int i = tid; i < n; i += kThreads) {
-      const unsigned q = __ldcg(queue_of + i);
-      const unsigned cls = by_id ? 0u : (unsigned)__popc(replica_mask[__ldcg(uniq + i)]);
-      key_of[i] = q >= 32u ? 0xFFFFFFFFu : (cls * 32u + q);   // clusters with a bad replica mask are not submitted
+    if (!order_keys_early) {
+      for (int i = tid; i < n; i += kThreads) {
+        const unsigned q = __ldcg(queue_of + i);
+        const unsigned cls = by_id ? 0u : (unsigned)__popc(replica_mask[__ldcg(uniq + i)]);
+        key_of[i] = q >= 32u ? 0xFFFFFFFFu : (cls * 32u + q);   // clusters with a bad replica mask are not submitted
+      }
     }
     __syncthreads();
     if (warp == 0) {
