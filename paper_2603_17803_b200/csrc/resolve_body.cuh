@@ -320,7 +320,31 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   if (warp == 0) {
     unsigned L = ((unsigned)s_load[lane] << 5) | (unsigned)lane;     // (load, queue id) in one comparable word
     const unsigned todo = by_id ? 1u : (s_classes & ~1u);
-    for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D); ++R) {
+    // Common case: everything the serial pass has to visit is of one replica class (or the order is by id) and
+    // sits in shared memory.  The warps' segments then hold exactly the visit order, densely, and the pass is a
+    // flat loop over each segment: no per-batch staging, the next item fetched while the current one is decided;
+    // lane r of every group of 32 keeps the queue of the group's r-th cluster.
+    const bool flat = staged && __popc(todo) <= 1;
+    if (flat && todo != 0u) {
+      for (int w2 = 0; w2 < kWarps; ++w2) {
+        const int base = s_seg[w2].x, len = s_seg[w2].y;
+        for (int g0 = 0; g0 < len; g0 += 32) {
+          const int cnt_g = min(32, len - g0);
+          unsigned my_q = 0u;
+          uint4 it = s_items[base + g0];
+          for (int rr = 0; rr < cnt_g; ++rr) {
+            const uint4 nx = s_items[min(base + g0 + rr + 1, items_cap - 1)];
+            const unsigned key = ((it.x >> lane) & 1u) ? L : 0xFFFFFFFFu;
+            const unsigned best = __reduce_min_sync(0xFFFFFFFFu, key);
+            if (L == best) L += it.y;
+            if (lane == rr) my_q = best & 31u;
+            it = nx;
+          }
+          if (lane < cnt_g) s_items[base + g0 + lane].w = my_q;
+        }
+      }
+    }
+    for (int R = by_id ? 0 : 2; R <= (by_id ? 0 : geo.D) && !flat; ++R) {
       if (!by_id && !((todo >> (R - 1)) & 1u)) continue;
       for (int w2 = 0; w2 < (staged ? 1 : kWarps); ++w2) {
         const int base = staged ? 0 : s_seg[w2].x, len = staged ? n : s_seg[w2].y;
