@@ -367,3 +367,23 @@ def entry_replica_masks(cluster_ptr, cluster_members, n_entries, D):
             masks[int(cluster_members[j])] |= np.uint32(1 << ((disk + (j - int(cluster_ptr[c]))) % D))
         p_global += int(cluster_ptr[c + 1] - cluster_ptr[c])
     return masks
+
+
+# ---- which clusters the fast tier holds (Sec. 4.2, Tier 1 (3): cached in descending order of the Eq. 6 score) ----
+def cache_admit(score, cluster_size, capacity_pages):
+    """Clusters are taken in descending score (ties to the lower id) while they still fit into the capacity,
+    counted in pages; the first one that does not fit ends the admission.  Returns (resident uint8 [C],
+    clusters admitted, pages used)."""
+    score = np.asarray(score, dtype=np.float32)
+    size = np.asarray(cluster_size).astype(np.int64)
+    order = sorted(range(len(score)), key=lambda c: (-float(score[c]), c))
+    resident = np.zeros(len(score), dtype=np.uint8)
+    used = 0
+    n = 0
+    for c in order:
+        if used + int(size[c]) > capacity_pages:
+            break
+        resident[c] = 1
+        used += int(size[c])
+        n += 1
+    return resident, n, used

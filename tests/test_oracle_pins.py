@@ -753,3 +753,30 @@ def test_entry_placement_hand_case_and_round_robin():
     for c in range(len(sizes)):
         disks = [int(masks[e]).bit_length() - 1 for e in members[ptr[c]:ptr[c + 1]]]
         assert disks == [(int(ptr[c]) + j) % D for j in range(int(sizes[c]))]
+
+
+# ------------------------------------------------------------------------------------ cache admission (Eq. 6)
+
+def test_cache_admission_hand_case_and_limits():
+    score = np.array([3.0, 9.0, 9.0, 1.0, 5.0], dtype=np.float32)
+    size = np.array([4, 2, 3, 1, 6], dtype=np.uint16)
+    # order by score: 1, 2 (tie, lower id first), 4, 0, 3 with sizes 2, 3, 6, 4, 1
+    res, n, used = oracle.cache_admit(score, size, 11)
+    assert list(res) == [0, 1, 1, 0, 1] and n == 3 and used == 11
+    res, n, used = oracle.cache_admit(score, size, 10)      # cluster 4 (6 pages) does not fit after 5: admission ends
+    assert list(res) == [0, 1, 1, 0, 0] and n == 2 and used == 5
+    assert oracle.cache_admit(score, size, 0)[1] == 0
+    res, n, used = oracle.cache_admit(score, size, 1000)
+    assert res.all() and n == 5 and used == 16
+    # growing the capacity never evicts
+    rng = np.random.default_rng(61)
+    score = rng.integers(0, 20, size=200).astype(np.float32)
+    size = rng.integers(1, 17, size=200).astype(np.uint16)
+    prev = np.zeros(200, dtype=np.uint8)
+    for cap in range(0, 1800, 37):
+        res, n, used = oracle.cache_admit(score, size, cap)
+        assert np.all(res >= prev) and used <= cap and used == int(size[res == 1].sum())
+        if n < 200:                                          # the best cluster left out really does not fit
+            nxt = min((c for c in range(200) if not res[c]), key=lambda c: (-score[c], c))
+            assert used + int(size[nxt]) > cap
+        prev = res
