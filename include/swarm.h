@@ -285,6 +285,17 @@ int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, con
 int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_medoid_index* index,
                           const swarm_outputs* outputs, void* stream);
 
+/* Which clusters the fast tier holds (no ctx; Sec. 4.2 Tier 1 (3): "clusters are cached in descending order of
+ * this score" under a fixed capacity; Sec. 5.2: the cached set follows the updated scores).  Clusters are taken in
+ * descending score (the Eq. 6 values swarm_set_cache maintains; ties to the lower id) while their sizes
+ * (cluster_size, pages) still fit into capacity_pages; the first cluster that does not fit ends the admission.
+ * Writes resident[c] = 1 or 0 for every cluster -- the table swarm_set_cache reads -- and, if info is not NULL,
+ * info[0] = clusters admitted, info[1] = pages used.  Device pointers, 16-byte aligned; n_clusters <= 65536;
+ * workspace: swarm_cache_admit_workspace_bytes(n_clusters) bytes (< 0: minus an error code). */
+int64_t swarm_cache_admit_workspace_bytes(int32_t n_clusters);
+int32_t swarm_cache_admit(const float* score, const uint16_t* cluster_size, int32_t n_clusters, int64_t capacity_pages,
+                          void* workspace, int64_t workspace_bytes, uint8_t* resident, int32_t* info, void* stream);
+
 /* Offline index build (no ctx; not part of a decode step): Algorithm 1, co-activation clustering of n entries
  * from their distance matrix dist (fp32 [n][n] row-major, d = 1 - co-activation probability) and the cluster
  * radius tau.  All pointers are device pointers, 16-byte aligned.

@@ -29,6 +29,7 @@ EXPORTS = (
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
+    "swarm_cache_admit_workspace_bytes", "swarm_cache_admit",
 )
 
 
@@ -77,6 +78,7 @@ def load_library() -> ctypes.CDLL:
             getattr(lib, name).restype = ctypes.c_int32
         lib.swarm_workspace_bytes.restype = ctypes.c_int64
         lib.swarm_build_clusters_workspace_bytes.restype = ctypes.c_int64
+        lib.swarm_cache_admit_workspace_bytes.restype = ctypes.c_int64
         _lib = lib
     return _lib
 
@@ -173,6 +175,26 @@ def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_
     c = swarm_cache(_ptr(resident, "resident"), _ptr(freq, "freq"), _ptr(score, "score"), _ptr(n_hit, "n_hit"),
                     float(t_base), float(t_transfer))
     _check(load_library().swarm_set_cache(ctx, ctypes.byref(c)), "swarm_set_cache", ctx)
+
+
+def swarm_cache_admit_workspace_bytes(n_clusters: int) -> int:
+    n = int(load_library().swarm_cache_admit_workspace_bytes(ctypes.c_int32(n_clusters)))
+    if n < 0:
+        raise SwarmError(-n, "swarm_cache_admit_workspace_bytes")
+    return n
+
+
+def swarm_cache_admit(score: torch.Tensor, cluster_size: torch.Tensor, capacity_pages: int, resident: torch.Tensor,
+                      info: Optional[torch.Tensor] = None, stream=None) -> None:
+    """resident[c] = 1 for the clusters the fast tier holds: descending score while their sizes fit the capacity."""
+    n = int(score.numel())
+    ws = torch.empty(swarm_cache_admit_workspace_bytes(n), dtype=torch.uint8, device=score.device)
+    _check(load_library().swarm_cache_admit(_ptr(score, "score"), _ptr(cluster_size, "cluster_size"), ctypes.c_int32(n),
+                                            ctypes.c_int64(capacity_pages), _ptr(ws), ctypes.c_int64(ws.numel()),
+                                            _ptr(resident, "resident"), _ptr(info, "info"), _stream(stream)),
+           "swarm_cache_admit")
+    if stream is None:
+        torch.cuda.current_stream(score.device).synchronize()     # the scratch is freed when this returns
 
 
 def swarm_build_clusters_workspace_bytes(n_entries: int) -> int:

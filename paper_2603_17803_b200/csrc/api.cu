@@ -265,6 +265,23 @@ int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, vo
   return e == cudaSuccess ? SWARM_OK : SWARM_ERR_CUDA;
 }
 
+int64_t swarm_cache_admit_workspace_bytes(int32_t n_clusters) {
+  if (n_clusters < 1 || n_clusters > 65536) return -(int64_t)SWARM_ERR_UNSUPPORTED;
+  return cache_admit_workspace_bytes(n_clusters);
+}
+
+int32_t swarm_cache_admit(const float* score, const uint16_t* cluster_size, int32_t n_clusters, int64_t capacity_pages,
+                          void* workspace, int64_t workspace_bytes, uint8_t* resident, int32_t* info, void* stream) {
+  if (n_clusters < 1 || capacity_pages < 0 || bad(score) || bad(cluster_size) || bad(workspace) || bad(resident) ||
+      !aligned16(info))
+    return SWARM_ERR_INVALID_ARG;
+  if (n_clusters > 65536) return SWARM_ERR_UNSUPPORTED;
+  if (workspace_bytes < cache_admit_workspace_bytes(n_clusters)) return SWARM_ERR_WORKSPACE_TOO_SMALL;
+  const cudaError_t e = launch_cache_admit(score, cluster_size, n_clusters, capacity_pages, workspace, resident, info,
+                                           static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? SWARM_OK : SWARM_ERR_CUDA;
+}
+
 int32_t swarm_last_cuda_error(const swarm_ctx* ctx) { return ctx ? (int32_t)ctx->last_err : 0; }
 
 int32_t swarm_device_status(swarm_ctx* ctx, void* stream, uint32_t* bits) {

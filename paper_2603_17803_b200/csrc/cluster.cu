@@ -187,6 +187,97 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
 
 }  // namespace
 
+// ---- admission to the fast tier (Sec. 4.2, Tier 1 (3)): clusters in descending Eq. 6 score while they fit -------
+namespace {
+
+// order[place] = c with place = #{ j : score[j] > score[c] or (score[j] == score[c] and j < c) }
+__global__ void __launch_bounds__(256)
+score_order_kernel(const float* __restrict__ score, int n, int32_t* __restrict__ order) {
+  __shared__ float s_sc[2048];
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const float mine = i < n ? score[i] : 0.f;
+  int place = 0;
+  for (int base = 0; base < n; base += 2048) {
+    __syncthreads();
+    for (int t = threadIdx.x; t < 2048 && base + t < n; t += blockDim.x) s_sc[t] = score[base + t];
+    __syncthreads();
+    const int lim = min(2048, n - base);
+    for (int t = 0; t < lim; ++t) {
+      const float other = s_sc[t];
+      place += (other > mine) || (other == mine && base + t < i);
+    }
+  }
+  if (i < n) order[place] = i;
+}
+
+// One CTA walks the order: running page count by a block scan per chunk; a cluster is admitted while the count
+// stays within the capacity, and the first one that does not fit ends the admission (everything after it is out).
+__global__ void __launch_bounds__(1024)
+admit_kernel(const int32_t* __restrict__ order, const uint16_t* __restrict__ size, int n, long long capacity,
+             uint8_t* __restrict__ resident, int32_t* __restrict__ info) {
+  __shared__ long long s_warp[32];
+  __shared__ long long s_used_final;
+  __shared__ int s_first_out;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
+  long long used = 0;                                      // pages of the clusters before the current chunk
+  int admitted = 0;
+  bool closed = false;
+  for (int base = 0; base < n; base += 1024) {
+    const int r = base + tid;
+    const int c = r < n ? order[r] : -1;
+    const long long mine = c >= 0 ? (long long)size[c] : 0;
+    long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (tid == 0) s_first_out = 1 << 30;
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    long long before = used;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+    const bool fits = !closed && c >= 0 && before + incl <= capacity;
+    if (c >= 0 && !fits) atomicMin(&s_first_out, r);
+    __syncthreads();
+    const int first_out = s_first_out;                     // rank of the first cluster that does not fit (if any)
+    const bool in = c >= 0 && !closed && r < first_out;
+    if (c >= 0) resident[c] = in ? 1 : 0;
+    if (!closed) {
+      if (first_out < (1 << 30)) {
+        if (r == first_out) s_used_final = before + incl - mine;   // pages used when the admission ended
+        admitted += first_out - base;
+      } else {
+        for (int w = 0; w < 32; ++w) used += s_warp[w];
+        admitted += min(1024, n - base);
+      }
+    }
+    __syncthreads();
+    if (!closed && first_out < (1 << 30)) {
+      used = s_used_final;
+      closed = true;
+    }
+  }
+  if (tid == 0 && info != nullptr) {
+    info[0] = admitted;
+    info[1] = (int32_t)min(used, 0x7FFFFFFFLL);
+  }
+}
+
+}  // namespace
+
+long long cache_admit_workspace_bytes(int n) { return ((long long)n * 4 + 255) / 256 * 256; }
+
+cudaError_t launch_cache_admit(const float* score, const uint16_t* size, int n, long long capacity, void* workspace,
+                               uint8_t* resident, int32_t* info, cudaStream_t st) {
+  int32_t* order = static_cast<int32_t*>(workspace);
+  score_order_kernel<<<dim3((n + 255) / 256), dim3(256), 0, st>>>(score, n, order);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_pdl(admit_kernel, dim3(1), dim3(1024), 0, st, true, order, size, n, capacity, resident, info);
+}
+
 long long build_clusters_workspace_bytes(int n) {
   // queue, cand_raw, cand (int32), sum (float), covered (bytes), each padded to 256 bytes
   const long long words = ((long long)n * 4 + 255) / 256 * 256;

@@ -143,6 +143,11 @@ cudaError_t launch_build_clusters(const float* dist, int n, float tau, void* wor
                                   int32_t* members, long long members_cap, int32_t* medoid, int32_t* n_clusters,
                                   int32_t* dev_status, cudaStream_t st);
 
+// Admission of clusters to the fast tier by Eq. 6 score (cluster.cu).
+long long cache_admit_workspace_bytes(int n);
+cudaError_t launch_cache_admit(const float* score, const uint16_t* size, int n, long long capacity, void* workspace,
+                               uint8_t* resident, int32_t* info, cudaStream_t st);
+
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

@@ -759,3 +759,42 @@ def test_medoid_step_full_size_c3_and_wide_groups():
         sess.step_medoid()
         check_medoid_step(w, sess, 3)
         sess.close()
+
+
+# ---- admission of clusters to the fast tier by their Eq. 6 score -------------------------------------------
+@pytest.mark.parametrize("n,cap_frac", [(5, 0.7), (200, 0.3), (1024, 0.5), (3000, 0.25), (5000, 0.0), (5000, 2.0)])
+def test_cache_admission_matches_oracle(n, cap_frac):
+    g = torch.Generator(device="cpu").manual_seed(n)
+    score = torch.randint(0, 40, (n,), generator=g).to(torch.float32) * 0.25      # many ties
+    size = torch.randint(1, 17, (n,), generator=g, dtype=torch.int16)
+    cap = int(cap_frac * int(size.sum()))
+    resident = torch.full((n + 16,), 7, dtype=torch.uint8, device=DEV)
+    info = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.swarm_cache_admit(score.to(DEV), size.to(DEV), cap, resident, info)
+    torch.cuda.synchronize()
+    want, n_in, used = oracle.cache_admit(score.numpy(), size.numpy().view(np.uint16), cap)
+    assert np.array_equal(resident.cpu().numpy()[:n], want) and int(resident[n:].min()) == 7
+    assert info.cpu().numpy()[:2].tolist() == [n_in, used]
+
+
+def test_cache_admission_feeds_the_resident_filter():
+    """Scores maintained by the step (Eq. 6) -> admission -> the next step fetches only what is not resident."""
+    w = W.generate(CASES["c3_small"], seed=73, device=DEV)
+    sess = Session(w)
+    C = w.n_clusters
+    resident = torch.zeros(C + 16, dtype=torch.uint8, device=DEV)
+    freq = torch.zeros(C, dtype=torch.int32, device=DEV)
+    score = torch.zeros(C, dtype=torch.float32, device=DEV)
+    n_hit = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.swarm_set_cache(sess.ctx, resident=resident, freq=freq, score=score, n_hit=n_hit, t_base=80.0, t_transfer=2.5)
+    sess.step()                                             # nothing resident yet: every activated cluster scores
+    torch.cuda.synchronize()
+    n_first = int(sess.o.n_uniq[0])
+    assert int(n_hit[0]) == 0 and int((freq > 0).sum()) == n_first
+    B.swarm_cache_admit(score, w.cluster_size, 10_000_000, resident)       # room for everything with a score
+    want, _, _ = oracle.cache_admit(score.cpu().numpy(), w.cluster_size.cpu().numpy().view(np.uint16), 10_000_000)
+    assert np.array_equal(resident.cpu().numpy()[:C], want) and want.all()
+    sess.step()                                             # same query: everything activated is resident now
+    torch.cuda.synchronize()
+    assert int(sess.o.n_uniq[0]) == 0 and int(n_hit[0]) == n_first
+    sess.close()
