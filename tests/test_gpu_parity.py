@@ -798,3 +798,49 @@ def test_cache_admission_feeds_the_resident_filter():
     torch.cuda.synchronize()
     assert int(sess.o.n_uniq[0]) == 0 and int(n_hit[0]) == n_first
     sess.close()
+
+
+# ---- the selector report: its figures recomputed on the host in fp64 from the selectors' own lists -------------
+@pytest.mark.parametrize("name,k_c", [("c2_small", 12), ("c5_small", 4)])
+def test_selector_report_figures(name, k_c):
+    from helpers import from_bf16_bits
+    from paper_2603_17803_b200 import selector_report as R
+    w = W.generate(CASES[name], seed=79, device=DEV)
+    rep = R.compare(w, k_c, keep_lists=True)
+    cfg, tabs = w.cfg, parity.host_tables(w)
+    S, d, g = cfg.page_size, cfg.head_dim, cfg.n_q_heads // cfg.n_kv_heads
+    q = from_bf16_bits(W.bits_u16(w.q)).astype(np.float64)
+    pool = W.bits_u16(w.kv_pool)
+    ptr, members, _ = (t.cpu().numpy() for t in W.cluster_members(w))
+    for sel_name in ("pages", "medoids"):
+        lists, n_lists = rep[sel_name]["lists"]
+        if sel_name == "medoids":                           # the pages those clusters hold
+            sel_p, n_p = oracle.expand_clusters(lists, n_lists, tabs["cluster_base"], ptr, members)
+        else:
+            sel_p, n_p = lists, n_lists
+        att_n, mass_r, top_r = [], [], []
+        for b in range(cfg.batch):
+            ctx = int(tabs["ctx_len"][b])
+            P = -(-ctx // S)
+            pb = int(tabs["page_base"][b])
+            for h in range(cfg.n_q_heads):
+                keys = from_bf16_bits(pool[pb:pb + P, h // g, 0]).astype(np.float64).reshape(P * S, d)
+                logit = keys @ q[b, h] / np.sqrt(d)
+                logit[ctx:] = -np.inf
+                prob = np.exp(logit - logit.max())
+                mass = (prob / prob.sum()).reshape(P, S).sum(1)
+                pages = sel_p[b, h, : n_p[b, h]]
+                att_n.append(len(pages))
+                mass_r.append(mass[pages].sum())
+                best = np.argsort(-mass, kind="stable")[: min(cfg.top_k, P)]
+                top_r.append(np.isin(best, pages).mean())
+        got = rep[sel_name]
+        assert got["attended_pages"] == pytest.approx(np.mean(att_n), rel=1e-6)
+        assert got["mass_recall"] == pytest.approx(np.mean(mass_r), abs=2e-4)
+        assert got["topk_recall"] == pytest.approx(np.mean(top_r), abs=5e-3)     # near-ties of mass order differently in fp32
+        uniq, _, load = oracle.resolve(sel_p, n_p, tabs["page_base"], tabs["page2cluster"], tabs["cluster_base"],
+                                       tabs["replica_mask"], tabs["cluster_size"], cfg.n_queues)
+        assert got["io_clusters"] == len(uniq) and got["io_pages"] == int(tabs["cluster_size"][uniq].sum())
+        assert got["io_pages"] == int(load.sum()) and got["max_queue_load"] == int(load.max())
+    # whole clusters attended: the medoid selector's I/O is exactly what its heads attend, no partial clusters
+    assert rep["medoids"]["io_pages"] >= rep["medoids"]["attended_pages"]
