@@ -1,5 +1,8 @@
 // C-ABI layer of libswarm: argument validation, workspace carving and kernel sequencing.
-// No device memory is allocated here; every scratch byte comes from the caller's workspace.
+// No device memory is allocated here; every scratch byte comes from the caller's workspace.  (swarm_create
+// allocates one 64-byte word of pinned host memory, the completion word of swarm_step_host.)
+#include <atomic>
+#include <chrono>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -19,10 +22,13 @@ struct swarm_ctx {
   cudaGraphExec_t host_graph;  // swarm_step_host: the recorded step, valid for the arguments in host_key
   unsigned char host_key[256];
   bool host_graph_ok;
+  bool host_graph_signals;    // the recorded step ends by raising *done_h
   bool has_cache;
   swarm_cache cache;
   int32_t* submit_order;      // optional outputs of the resolution (swarm_set_submit_order)
   int32_t* submit_info;
+  unsigned* done_h;           // one word of pinned host memory the publish kernel raises when a host step is complete,
+  unsigned* done_d;           // and the address the device writes it through (both null if the allocation failed)
 };
 
 namespace {
@@ -180,16 +186,32 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->last_err = cudaSuccess;
   ctx->host_graph = nullptr;
   ctx->host_graph_ok = true;
+  ctx->host_graph_signals = false;
   ctx->has_cache = false;
   ctx->submit_order = nullptr;
   ctx->submit_info = nullptr;
   std::memset(ctx->host_key, 0, sizeof ctx->host_key);
+  ctx->done_h = nullptr;
+  ctx->done_d = nullptr;
+  void* flag = nullptr;
+  if (cudaHostAlloc(&flag, 64, cudaHostAllocMapped) == cudaSuccess) {
+    void* flag_d = nullptr;
+    if (cudaHostGetDevicePointer(&flag_d, flag, 0) == cudaSuccess) {
+      ctx->done_h = static_cast<unsigned*>(flag);
+      ctx->done_d = static_cast<unsigned*>(flag_d);
+      *ctx->done_h = 0u;
+    } else {
+      cudaFreeHost(flag);
+    }
+  }
+  cudaGetLastError();                                     // without the word, host steps wait on the stream
   cudaError_t e = configure_score();
   if (e == cudaSuccess) e = configure_topk();
   if (e == cudaSuccess) e = configure_resolve();
   if (e == cudaSuccess) e = configure_attention();
   if (e == cudaSuccess) e = configure_medoid();
   if (e != cudaSuccess) {
+    if (ctx->done_h != nullptr) cudaFreeHost(ctx->done_h);
     delete ctx;
     return SWARM_ERR_CUDA;
   }
@@ -200,6 +222,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
 int32_t swarm_destroy(swarm_ctx* ctx) {
   if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
   if (ctx->host_graph != nullptr) cudaGraphExecDestroy(ctx->host_graph);
+  if (ctx->done_h != nullptr) cudaFreeHost(ctx->done_h);
   delete ctx;
   return SWARM_OK;
 }
@@ -431,13 +454,18 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
 }
 
 namespace {
-// Everything swarm_step_host enqueues for one step: copy q in, the step, copy the results out.
+// Everything swarm_step_host enqueues for one step: q in, the step, the results out.  *signals is set when the
+// last operation raises ctx->done_h on completion.
 int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
                           float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool* signals) {
+  *signals = false;
   const int64_t bh = (int64_t)ctx->geo.B * ctx->geo.Hq;
   uint16_t* q_dev = ws_ptr<uint16_t>(ctx, ctx->lay.q_stage);
-  SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
+  // q: read over the bus by a kernel when the device can address the buffer, else one copy operation
+  const void* q_view = device_view<const void>(q_host, 16);
+  if (q_view != nullptr) SWARM_TRY(launch_fetch(q_view, q_dev, bh * kHeadDim * 2, st));
+  else SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
   swarm_inputs local = *in;
   local.q = q_dev;
   const int32_t rc = swarm_step(ctx, &local, o, st);
@@ -450,7 +478,9 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   int32_t* queue_load_d = device_view<int32_t>(queue_load_host, 4);
   if ((out_host == nullptr || out_d) && (lse_host == nullptr || lse_d) && (n_uniq_host == nullptr || n_uniq_d) &&
       (queue_load_host == nullptr || queue_load_d)) {
-    SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d, st));
+    SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d,
+                             ws_ptr<unsigned>(ctx, ctx->lay.status + 96), ctx->done_d, st));
+    *signals = ctx->done_d != nullptr;
     return SWARM_OK;
   }
   if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));
@@ -459,6 +489,21 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   if (queue_load_host)
     SWARM_TRY(cudaMemcpyAsync(queue_load_host, o->queue_load, ctx->geo.D * 4, cudaMemcpyDeviceToHost, st));
   return SWARM_OK;
+}
+
+// Waits for the word the publish kernel raises; gives up after ~50 ms (a failed launch never raises it) and lets
+// the caller fall back to the stream, which also reports the error.
+bool wait_done_word(swarm_ctx* ctx) {
+  volatile unsigned* done = ctx->done_h;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (;;) {
+    for (int i = 0; i < 2048; ++i)
+      if (*done != 0u) {
+        std::atomic_thread_fence(std::memory_order_acquire);
+        return true;
+      }
+    if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(50)) return false;
+  }
 }
 
 // The arguments a captured host step depends on; a replay is valid only while none of them changes.
@@ -566,7 +611,8 @@ int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outp
       if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
       cudaGraph_t graph = nullptr;
       if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
-        rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st);
+        rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st,
+                               &ctx->host_graph_signals);
         const cudaError_t e = cudaStreamEndCapture(st, &graph);
         if (rc == SWARM_OK && e == cudaSuccess && graph != nullptr &&
             cudaGraphInstantiate(&ctx->host_graph, graph, 0) == cudaSuccess) {
@@ -584,12 +630,17 @@ int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outp
       }
     }
     if (ctx->host_graph != nullptr) {
+      // The results land in host memory through the publish kernel, which raises a word there when all of them
+      // are visible: waiting on that word returns a few microseconds before the stream reports completion.
+      if (ctx->host_graph_signals) *static_cast<volatile unsigned*>(ctx->done_h) = 0u;
       SWARM_TRY(cudaGraphLaunch(ctx->host_graph, st));
+      if (ctx->host_graph_signals && wait_done_word(ctx)) return SWARM_OK;
       SWARM_TRY(cudaStreamSynchronize(st));
       return SWARM_OK;
     }
   }
-  rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st);
+  bool signals = false;
+  rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st, &signals);
   if (rc != SWARM_OK) return rc;
   SWARM_TRY(cudaStreamSynchronize(st));
   return SWARM_OK;
