@@ -185,16 +185,16 @@ __device__ __forceinline__ void block_minmax(SelectState& st, int tid, uint32_t 
 template <int THREADS>
 __device__ __forceinline__ void finish_by_ranking(SelectState& st, int tid, int n) {
   const int remaining = st.remaining;
+  const int lane = tid & 31, warp = tid >> 5;
   __syncthreads();
-  for (int i = tid; i < n; i += THREADS) {
+  // one warp per candidate: the lanes hold all (at most 64) candidates, two ballots count those above and equal
+  const bool v0 = lane < n, v1 = lane + 32 < n;
+  const uint32_t o0 = v0 ? st.cand[lane] : 0u, o1 = v1 ? st.cand[lane + 32] : 0u;
+  for (int i = warp; i < n; i += THREADS / 32) {
     const uint32_t mine = st.cand[i];
-    int gt = 0, eq = 0;
-    for (int j = 0; j < n; ++j) {
-      const uint32_t other = st.cand[j];
-      gt += other > mine;
-      eq += other == mine;
-    }
-    if (gt < remaining && remaining <= gt + eq) {
+    const int gt = __popc(__ballot_sync(0xFFFFFFFFu, v0 && o0 > mine)) + __popc(__ballot_sync(0xFFFFFFFFu, v1 && o1 > mine));
+    const int eq = __popc(__ballot_sync(0xFFFFFFFFu, v0 && o0 == mine)) + __popc(__ballot_sync(0xFFFFFFFFu, v1 && o1 == mine));
+    if (lane == 0 && gt < remaining && remaining <= gt + eq) {
       st.base = mine;
       st.bits = 0;
       st.remaining = remaining - gt;
@@ -288,13 +288,19 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   }
   SWARM_STAMP(status, 12);
 
-  // ordered output: packed (greater, equal) counts per thread, one block-wide exclusive scan
-  int cnt = 0;
+  // ordered output: packed (greater, equal) counts per thread, one block-wide exclusive scan.  A thread keeps
+  // its pages above the threshold (window pages rank above every score) and at it as two bit masks: about one
+  // page in P / k is selected, so everything after the scan walks the set bits instead of all ITEMS pages.
+  unsigned gt_mask = 0u, eq_mask = 0u;
 #pragma unroll
   for (int j = 0; j < ITEMS; ++j) {
-    if (p0 + j >= Pw) key[j] = p0 + j < P ? 0xFFFFFFFFu : 0u;   // window pages rank above every score
-    if (p0 + j < P) cnt += ((key[j] > T || p0 + j >= Pw) ? 1 : 0) + ((key[j] == T && p0 + j < Pw) ? 0x10000 : 0);
+    if (p0 + j < P) {
+      const bool win = p0 + j >= Pw;
+      gt_mask |= (unsigned)(win || key[j] > T) << j;
+      eq_mask |= (unsigned)(!win && key[j] == T) << j;
+    }
   }
+  const int cnt = __popc(gt_mask) | (__popc(eq_mask) << 16);
   int incl = cnt;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -305,18 +311,14 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   if (lane == 31) st.warp_tot[warp] = incl;
   __syncthreads();
   const int before = incl - cnt + totals_before<THREADS>(st.warp_tot, warp, lane);
-  int gt_before = before & 0xFFFF, eq_before = before >> 16;
+  const int gt_before = before & 0xFFFF, eq_before = before >> 16;
   unsigned picked = 0u;                                     // bit j: page p0 + j is selected
-#pragma unroll
-  for (int j = 0; j < ITEMS; ++j) {
-    if (p0 + j < P) {
-      const bool gt = key[j] > T || p0 + j >= Pw, eq = key[j] == T && p0 + j < Pw;
-      if (gt || (eq && eq_before < need_eq)) {
-        out[gt_before + min(eq_before, need_eq)] = p0 + j;
-        picked |= 1u << j;
-      }
-      gt_before += gt;
-      eq_before += eq;
+  for (unsigned todo = gt_mask | eq_mask; todo != 0u; todo &= todo - 1u) {
+    const unsigned bit = todo & (0u - todo), below = bit - 1u;
+    const int eq_b = eq_before + __popc(eq_mask & below);
+    if ((gt_mask & bit) || eq_b < need_eq) {
+      out[gt_before + __popc(gt_mask & below) + min(eq_b, need_eq)] = p0 + (__ffs(bit) - 1);
+      picked |= bit;
     }
   }
   if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
@@ -325,16 +327,24 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
     else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
   }
   if (x.flags != nullptr) {
-    // all the table reads first, then the flag stores: a byte store may alias anything, so interleaving them
-    // would make every read wait for the store before it
-    int c[ITEMS];
+    // four selected pages at a time: all the table reads first, then the flag stores -- a byte store may alias
+    // anything, so interleaving them would make every read wait for the store before it
+    for (unsigned todo = picked; todo != 0u;) {
+      int c[4];
+      bool have[4];
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j) c[j] = ((picked >> j) & 1u) ? x.page2cluster[rb.pb + p0 + j] : 0;
+      for (int i = 0; i < 4; ++i) {
+        have[i] = todo != 0u;
+        const int j = __ffs(todo) - 1;
+        todo &= todo - 1u;                                  // 0 stays 0
+        c[i] = have[i] ? x.page2cluster[rb.pb + p0 + j] : 0;
+      }
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j) {
-      if ((picked >> j) & 1u) {
-        if (c[j] < 0 || c[j] >= rb.cn - rb.cb || rb.cb + c[j] >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
-        else x.flags[rb.cb + c[j]] = 1;
+      for (int i = 0; i < 4; ++i) {
+        if (have[i]) {
+          if (c[i] < 0 || c[i] >= rb.cn - rb.cb || rb.cb + c[i] >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
+          else x.flags[rb.cb + c[i]] = 1;
+        }
       }
     }
   }
