@@ -230,6 +230,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   // thread t owns pages [t*ITEMS, (t+1)*ITEMS); keys of pages that do not exist are never used
   uint32_t key[ITEMS];
   const int p0 = tid * ITEMS;
+  const bool full = p0 + ITEMS <= Pw;                       // all of this thread's pages exist and are scored: no per-page checks
   if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
 #pragma unroll
     for (int j = 0; j < ITEMS; j += 4) {
@@ -250,9 +251,14 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
     need_eq = 0;
   } else if (k_sel < Pw) {
     uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+    if (full) {
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j)
-      if (p0 + j < Pw) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+      for (int j = 0; j < ITEMS; ++j) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+    } else {
+#pragma unroll
+      for (int j = 0; j < ITEMS; ++j)
+        if (p0 + j < Pw) { lo = min(lo, key[j]); hi = max(hi, key[j]); }
+    }
     block_minmax<THREADS>(st, tid, lo, hi);
     SWARM_STAMP(status, 3);
     for (int level = 0; level < 4 && st.bits > 0; ++level) {
@@ -260,10 +266,18 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
       const int bits = st.bits;
       const int shift = max(bits - kDigitBits, 0);
       const uint32_t width_m1 = bits >= 32 ? 0xFFFFFFFFu : ((1u << bits) - 1u);
+      if (full) {
 #pragma unroll
-      for (int j = 0; j < ITEMS; ++j) {
-        const uint32_t rel = key[j] - base;
-        if (p0 + j < Pw && rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
+        for (int j = 0; j < ITEMS; ++j) {
+          const uint32_t rel = key[j] - base;
+          if (rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) {
+          const uint32_t rel = key[j] - base;
+          if (p0 + j < Pw && rel <= width_m1) atomicAdd(&st.hist[hist_slot<THREADS>(rel >> shift)], 1);
+        }
       }
       __syncthreads();
       SWARM_STAMP(status, 4 + 2 * level);
@@ -279,7 +293,7 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j)
-          if (p0 + j < Pw && key[j] - cbase <= cwidth_m1) st.cand[atomicAdd(&st.n_cand, 1)] = key[j];
+          if ((full || p0 + j < Pw) && key[j] - cbase <= cwidth_m1) st.cand[atomicAdd(&st.n_cand, 1)] = key[j];
         finish_by_ranking<THREADS>(st, tid, n_cand);
       }
     }
@@ -292,12 +306,20 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   // its pages above the threshold (window pages rank above every score) and at it as two bit masks: about one
   // page in P / k is selected, so everything after the scan walks the set bits instead of all ITEMS pages.
   unsigned gt_mask = 0u, eq_mask = 0u;
+  if (full) {
 #pragma unroll
-  for (int j = 0; j < ITEMS; ++j) {
-    if (p0 + j < P) {
-      const bool win = p0 + j >= Pw;
-      gt_mask |= (unsigned)(win || key[j] > T) << j;
-      eq_mask |= (unsigned)(!win && key[j] == T) << j;
+    for (int j = 0; j < ITEMS; ++j) {
+      gt_mask |= (unsigned)(key[j] > T) << j;
+      eq_mask |= (unsigned)(key[j] == T) << j;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) {
+      if (p0 + j < P) {
+        const bool win = p0 + j >= Pw;
+        gt_mask |= (unsigned)(win || key[j] > T) << j;
+        eq_mask |= (unsigned)(!win && key[j] == T) << j;
+      }
     }
   }
   const int cnt = __popc(gt_mask) | (__popc(eq_mask) << 16);
