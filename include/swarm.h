@@ -320,11 +320,13 @@ int32_t swarm_build_clusters(const float* dist, int32_t n_entries, float tau, vo
  * `inputs` (whose q field is ignored) and `outputs`, copies out, lse, n_uniq, queue_load back into
  * the given host buffers and WAITS for completion.  Any *_host pointer may be NULL to skip it.
  * Result buffers that are pinned and addressable by the device (unified addressing; out_host 16-byte aligned)
- * are filled by one small kernel storing straight into them, otherwise by one copy operation each; q_host,
- * likewise, is read over the bus by a kernel when the device can address it (16-byte aligned), else copied.
- * When the results are stored by that kernel the call returns as soon as they are visible in host memory (the
- * kernel raises a word of pinned memory owned by the ctx after a system-wide fence), which is a few
- * microseconds before the stream itself reports completion; later work on the stream is ordered as usual.
+ * are written by the step's last kernel itself, which stores each result there as it produces it; otherwise by
+ * one copy operation each.  q_host, likewise, is read over the bus by a kernel when the device can address it
+ * (16-byte aligned), else copied.  When the results are stored by the kernel the call returns as soon as they
+ * are visible in host memory (the last part of the kernel to finish raises a word of pinned memory owned by the
+ * ctx after a system-wide fence), which is a few microseconds before the stream itself reports completion;
+ * later work on the stream is ordered as usual.  Device-side outputs that have no host buffer (sel, uniq,
+ * queue_of, the submission order) are complete when the stream is.
  * With pinned host buffers and a non-default stream the first call with a given set of pointers
  * records these operations into a CUDA graph (owned by the ctx) and later calls replay it; the
  * tensor shapes and the device tables must then stay where they are, their contents may change. */

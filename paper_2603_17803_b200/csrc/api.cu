@@ -420,7 +420,17 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const in
   return SWARM_OK;
 }
 
+namespace {
+int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host);
+}
+
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream) {
+  return step_impl(ctx, in, o, stream, nullptr);
+}
+
+namespace {
+// The fused step; `host` (swarm_step_host only) makes the last kernel store the small results into host memory too.
+int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host) {
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!select_inputs_ok(in) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || o == nullptr || bad(o->sel) ||
@@ -448,12 +458,15 @@ int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* 
                             static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
   AttnArgs a = paged_args(ctx, in, o->out, o->lse);
   a.n_splits = pick_splits(ctx, true, /*fused=*/true);
-  const ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
+  if (host != nullptr) {
+    a.host = *host;
+    rs.host = *host;
+  }
   SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, &rs));
   return SWARM_OK;
 }
 
-namespace {
 // Everything swarm_step_host enqueues for one step: q in, the step, the results out.  *signals is set when the
 // last operation raises ctx->done_h on completion.
 int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
@@ -468,19 +481,27 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   else SWARM_TRY(cudaMemcpyAsync(q_dev, q_host, bh * kHeadDim * 2, cudaMemcpyHostToDevice, st));
   swarm_inputs local = *in;
   local.q = q_dev;
-  const int32_t rc = swarm_step(ctx, &local, o, st);
-  if (rc != SWARM_OK) return rc;
   // Results: when every destination is pinned host memory the device can address (and 16-byte aligned for
-  // out), one small kernel stores them there; otherwise one copy operation per buffer.
+  // out), the step's last kernel stores them there as it produces them and raises the completion word (or,
+  // without that word, one small kernel stores them after the step); otherwise one copy operation per buffer.
   float* out_d = device_view<float>(out_host, 16);
   float* lse_d = device_view<float>(lse_host, 4);
   int32_t* n_uniq_d = device_view<int32_t>(n_uniq_host, 4);
   int32_t* queue_load_d = device_view<int32_t>(queue_load_host, 4);
-  if ((out_host == nullptr || out_d) && (lse_host == nullptr || lse_d) && (n_uniq_host == nullptr || n_uniq_d) &&
-      (queue_load_host == nullptr || queue_load_d)) {
+  const bool direct = (out_host == nullptr || out_d) && (lse_host == nullptr || lse_d) &&
+                      (n_uniq_host == nullptr || n_uniq_d) && (queue_load_host == nullptr || queue_load_d);
+  if (direct && ctx->done_d != nullptr) {
+    const HostMirror host{out_d, lse_d, n_uniq_d, queue_load_d, ws_ptr<unsigned>(ctx, ctx->lay.status + 96), ctx->done_d,
+                          (unsigned)attention_groups(ctx->geo, true) + 1u};
+    const int32_t rc = step_impl(ctx, &local, o, st, &host);
+    *signals = rc == SWARM_OK;
+    return rc;
+  }
+  const int32_t rc = swarm_step(ctx, &local, o, st);
+  if (rc != SWARM_OK) return rc;
+  if (direct) {
     SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d,
-                             ws_ptr<unsigned>(ctx, ctx->lay.status + 96), ctx->done_d, st));
-    *signals = ctx->done_d != nullptr;
+                             ws_ptr<unsigned>(ctx, ctx->lay.status + 96), nullptr, st));
     return SWARM_OK;
   }
   if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));

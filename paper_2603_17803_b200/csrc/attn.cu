@@ -558,9 +558,12 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
           os.x = fmaf(v.x, sc, os.x); os.y = fmaf(v.y, sc, os.y); os.z = fmaf(v.z, sc, os.z); os.w = fmaf(v.w, sc, os.w);
         }
         const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
-        reinterpret_cast<float4*>(a.out + (long long)(bh0 + hb + hh) * kHeadDim)[lane] =
-            make_float4(os.x * inv, os.y * inv, os.z * inv, os.w * inv);
-        if (lane == 0) a.lse[bh0 + hb + hh] = Ls > 0.f ? (Mx + log2f(Ls)) * kLn2 : -INFINITY;
+        const float4 res = make_float4(os.x * inv, os.y * inv, os.z * inv, os.w * inv);
+        const float lse_h = Ls > 0.f ? (Mx + log2f(Ls)) * kLn2 : -INFINITY;
+        reinterpret_cast<float4*>(a.out + (long long)(bh0 + hb + hh) * kHeadDim)[lane] = res;
+        if (lane == 0) a.lse[bh0 + hb + hh] = lse_h;
+        if (a.host.out_h != nullptr) reinterpret_cast<float4*>(a.host.out_h + (long long)(bh0 + hb + hh) * kHeadDim)[lane] = res;
+        if (a.host.lse_h != nullptr && lane == 0) a.host.lse_h[bh0 + hb + hh] = lse_h;
         __syncwarp();
       }
     }
@@ -569,10 +572,18 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
     for (int hh = 0; hh < 8; ++hh) {
       if (hh < G && has_dim) {
-        a.out[(long long)(bh0 + hh) * kHeadDim + t] = L[hh] > 0.f ? o[hh] / L[hh] : 0.f;
-        if (t == 0) a.lse[bh0 + hh] = L[hh] > 0.f ? (M[hh] + log2f(L[hh])) * kLn2 : -INFINITY;
+        const float res = L[hh] > 0.f ? o[hh] / L[hh] : 0.f;
+        const float lse_h = L[hh] > 0.f ? (M[hh] + log2f(L[hh])) * kLn2 : -INFINITY;
+        a.out[(long long)(bh0 + hh) * kHeadDim + t] = res;
+        if (t == 0) a.lse[bh0 + hh] = lse_h;
+        if (a.host.out_h != nullptr) a.host.out_h[(long long)(bh0 + hh) * kHeadDim + t] = res;
+        if (a.host.lse_h != nullptr && t == 0) a.host.lse_h[bh0 + hh] = lse_h;
       }
     }
+  }
+  if (a.host.done_h != nullptr) {                         // host step: this group's results are in host memory
+    __syncthreads();
+    if (t == 0) host_arrive(a.host);
   }
   SWARM_STAMP_ANY_CTA(status, 6);
   SWARM_KERNEL_END(status, 2);

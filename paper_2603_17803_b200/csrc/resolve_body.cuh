@@ -399,6 +399,8 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       }
     }
     if (lane < geo.D) queue_load[lane] = (int)(L >> 5);
+    if (lane < geo.D && r.host.queue_load_h != nullptr) r.host.queue_load_h[lane] = (int)(L >> 5);
+    if (lane == 0 && r.host.n_uniq_h != nullptr) *r.host.n_uniq_h = n;
     if (lane == 0) {
       *n_uniq = n;
       if (kCached && cache.n_hit != nullptr) *cache.n_hit = s_hits;
@@ -470,6 +472,10 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       r.submit_info[0] = rounds;
       r.submit_info[1] = submitted;
     }
+  }
+  if (r.host.done_h != nullptr) {                          // host step: the resolution's results are in host memory
+    __syncthreads();
+    if (tid == 0) host_arrive(r.host);
   }
 }
 

@@ -61,6 +61,19 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
                         const uint32_t* replica_mask = nullptr, const uint16_t* cluster_size = nullptr);
 // Everything the cluster-resolution body needs (see resolve_body.cuh).  sel == nullptr: the flags are already
 // set (by the selection or the expansion kernel) and a single CTA runs the tail.
+// Host-step extension of the fused attention + resolution kernel: the step's small results are also stored
+// into host memory the device can address, and the last of `arrivals` finishing parts (one per attention group,
+// one for the resolution CTA) raises *done_h after a system-wide fence.  All null / zero when unused.
+struct HostMirror {
+  float* out_h;
+  float* lse_h;
+  int32_t* n_uniq_h;
+  int32_t* queue_load_h;
+  unsigned* ticket;        // arrival counter in the workspace; zero between launches
+  unsigned* done_h;
+  unsigned arrivals;
+};
+
 struct ResolveArgs {
   Geometry geo;
   swarm_cache cache;
@@ -83,6 +96,7 @@ struct ResolveArgs {
   int items_cap;
   int32_t* submit_order;   // optional: submission order (indices into uniq), see resolve_body.cuh
   int32_t* submit_info;    // optional: [0] batches, [1] clusters submitted
+  HostMirror host{};
 };
 ResolveArgs make_resolve_args(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                               const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
@@ -118,6 +132,7 @@ struct AttnArgs {
   float* out;
   float* lse;
   int n_splits;
+  HostMirror host{};
 };
 // `fused_resolve` (paged mode only): one extra CTA of the grid runs cluster resolution with these arguments.
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,
@@ -154,6 +169,19 @@ cudaError_t launch_cache_admit(const float* score, const uint16_t* size, int n, 
 // ---- device helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// One part of a host step is complete.  Called by one thread of the CTA after a CTA-wide barrier that every
+// thread reached past its stores: the barrier orders those before this thread's system-wide fence, which is
+// cumulative over them.
+__device__ __forceinline__ void host_arrive(const HostMirror& h) {
+  __threadfence_system();
+  const unsigned arrived = atomicAdd(h.ticket, 1u);
+  if (arrived == h.arrivals - 1u) {
+    *h.ticket = 0u;                                         // ready for the next launch
+    __threadfence_system();
+    *reinterpret_cast<volatile unsigned*>(h.done_h) = 1u;
+  }
+}
 
 __device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
   uint4 r;

@@ -289,6 +289,40 @@ def test_step_host_round_trip():
     sess.close()
 
 
+@pytest.mark.parametrize("name", ["c3_small", "c5_small", "k_exceeds_pages"])
+def test_step_host_follows_a_query_buffer_rewritten_between_calls(name):
+    """The same pinned buffers, new contents every call: every call's results are those of its own query and are
+    complete in host memory when the call returns (the recorded graph, the fetch of q and the completion word
+    are all reused from call to call)."""
+    w = W.generate(CASES[name], seed=17, device=DEV)
+    cfg = w.cfg
+    sess = Session(w)
+    ref = Session(w, ksum=sess.ksum)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    q_host = torch.empty_like(w.q, device="cpu").pin_memory()
+    out_host = torch.empty((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.float32).pin_memory()
+    lse_host = torch.empty((cfg.batch, cfg.n_q_heads), dtype=torch.float32).pin_memory()
+    n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    load_host = torch.zeros(cfg.n_queues, dtype=torch.int32).pin_memory()
+    stream = torch.cuda.Stream()
+    for it in range(40):
+        q = (w.q.cpu().float() + 0.5 * torch.randn(w.q.shape, generator=g)).to(torch.bfloat16)
+        q_host.copy_(q)
+        out_host.fill_(float("nan")); lse_host.fill_(float("nan")); n_host.fill_(-1); load_host.fill_(-1)
+        sess.step_host(q_host, out_host, lse_host, n_host, load_host, stream=stream)
+        got = (out_host.clone(), lse_host.clone(), int(n_host[0]), load_host.clone())   # read at once, no synchronize
+        ref.set_query(q.to(DEV))
+        ref.step()
+        torch.cuda.synchronize()
+        assert torch.equal(got[0], ref.o.out.cpu()), f"call {it}"
+        assert torch.equal(got[1], ref.o.lse.cpu()) and got[2] == int(ref.o.n_uniq[0])
+        assert torch.equal(got[3], ref.o.queue_load.cpu()[: cfg.n_queues])
+        assert torch.equal(sess.o.sel, ref.o.sel) and torch.equal(sess.o.uniq[: got[2]], ref.o.uniq[: got[2]])
+    assert sess.status() == 0
+    sess.close()
+    ref.close()
+
+
 def test_step_can_be_captured_in_a_cuda_graph():
     w = W.generate(CASES["c3_small"], seed=14, device=DEV)
     sess = Session(w)
