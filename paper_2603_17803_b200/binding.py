@@ -318,6 +318,32 @@ def swarm_step_host(ctx, inputs: swarm_inputs, outputs: swarm_outputs, q_host, o
            "swarm_step_host", ctx)
 
 
+def marshal_step_host(ctx, inputs: swarm_inputs, outputs: swarm_outputs, q_host, out_host=None, lse_host=None,
+                      n_uniq_host=None, queue_load_host=None, stream=None) -> tuple:
+    """The C arguments of swarm_step_host for these tensors, for callers that repeat the call with the same ones
+    (the structures and tensors must stay alive and in place while the tuple is used)."""
+    return (ctx, ctypes.byref(inputs), ctypes.byref(outputs), _ptr(q_host, "q_host", False),
+            _ptr(out_host, "out_host", False), _ptr(lse_host, "lse_host", False),
+            _ptr(n_uniq_host, "n_uniq_host", False), _ptr(queue_load_host, "queue_load_host", False), _stream(stream))
+
+
+def swarm_step_host_marshalled(ctx, args: tuple) -> None:
+    """swarm_step_host with arguments prepared by marshal_step_host."""
+    rc = _step_host_fn()(*args)
+    if rc != OK:
+        _check(rc, "swarm_step_host", ctx)
+
+
+_STEP_HOST_FN = None
+
+
+def _step_host_fn():
+    global _STEP_HOST_FN
+    if _STEP_HOST_FN is None:
+        _STEP_HOST_FN = load_library().swarm_step_host
+    return _STEP_HOST_FN
+
+
 def swarm_device_status(ctx, stream=None) -> int:
     bits = ctypes.c_uint32(0)
     _check(load_library().swarm_device_status(ctx, _stream(stream), ctypes.byref(bits)), "swarm_device_status", ctx)

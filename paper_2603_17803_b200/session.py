@@ -109,8 +109,17 @@ class Session:
         B.swarm_step(self.ctx, self.inputs, self.outputs, stream)
 
     def step_host(self, q_host, out_host=None, lse_host=None, n_uniq_host=None, queue_load_host=None, stream=None):
-        B.swarm_step_host(self.ctx, self.inputs, self.outputs, q_host, out_host, lse_host, n_uniq_host,
-                          queue_load_host, stream)
+        """swarm_step_host.  The call is synchronous and tens of microseconds long, so the marshalled arguments of
+        the last call are kept and reused while the same tensor objects (and stream) are passed again; buffers
+        must not be resized in place between calls."""
+        key = (id(q_host), id(out_host), id(lse_host), id(n_uniq_host), id(queue_load_host), id(stream), id(self.inputs))
+        call = getattr(self, "_host_call", None)
+        if call is None or call[0] != key:
+            keep = (q_host, out_host, lse_host, n_uniq_host, queue_load_host, stream, self.inputs)   # ids stay unique while held
+            call = (key, B.marshal_step_host(self.ctx, self.inputs, self.outputs, q_host, out_host, lse_host,
+                                             n_uniq_host, queue_load_host, stream), keep)
+            self._host_call = call
+        B.swarm_step_host_marshalled(self.ctx, call[1])
 
     def enable_medoid_index(self, top_k_clusters: int, keep_scores: bool = False) -> None:
         """Builds the medoid index of the workload's clusters and the outputs of step_medoid()."""
