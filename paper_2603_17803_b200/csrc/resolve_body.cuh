@@ -152,25 +152,45 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
     uint32_t f;
     uint4 mk;
     uint2 sz;
+    uint32_t res;                                          // with cache state: the 4 clusters' resident bytes ...
+    int4 fr;                                               // ... and their frequency counters
   };
+  // vector loads of the cache state need its arrays aligned like the library's own tables
+  const bool cache_vec = kCached && (reinterpret_cast<uintptr_t>(cache.resident) & 3u) == 0 &&
+                         (reinterpret_cast<uintptr_t>(cache.freq) & 15u) == 0;
+  const bool need_sz = !unit || (kCached && cache.score != nullptr);   // unit loads need no size table, Eq. 6 does
   auto load_row = [&](int v, bool with_flags) -> Row {
     Row r;
     r.f = 0u;
     r.mk = make_uint4(0u, 0u, 0u, 0u);
     r.sz = make_uint2(0u, 0u);
+    r.res = 0u;
+    r.fr = make_int4(0, 0, 0, 0);
     if (v < v_hi) {
       if (with_flags) r.f = __ldcg(f1 + v);
       if (v * 4 + 4 <= C) {
         r.mk = ldg_nc_v4(reinterpret_cast<const uint4*>(replica_mask + v * 4));
-        if (!unit) r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));   // no size table needed for unit loads
-      } else {
+        if (need_sz) r.sz = __ldg(reinterpret_cast<const uint2*>(cluster_size + v * 4));
+        if (kCached && cache_vec) {
+          r.res = *reinterpret_cast<const uint32_t*>(cache.resident + v * 4);
+          r.fr = *reinterpret_cast<const int4*>(cache.freq + v * 4);
+        }
+      }
+      if (v * 4 + 4 > C || (kCached && !cache_vec)) {
         uint32_t* mk = &r.mk.x;
         uint32_t* sz = &r.sz.x;
+        int* fr = &r.fr.x;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (v * 4 + j < C) {
-            mk[j] = replica_mask[v * 4 + j];
-            if (!unit) sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
+            if (v * 4 + 4 > C) {
+              mk[j] = replica_mask[v * 4 + j];
+              if (need_sz) sz[j >> 1] |= (uint32_t)cluster_size[v * 4 + j] << (16 * (j & 1));
+            }
+            if (kCached) {
+              r.res |= (cache.resident[v * 4 + j] != 0 ? 1u : 0u) << (8 * j);
+              fr[j] = cache.freq[v * 4 + j];
+            }
           }
         }
       }
@@ -185,27 +205,35 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   if (one_vec) {
     cnt = nonzero_bytes(keep.f);
     if (kCached) {                                         // activated but resident: not fetched (Eq. 8)
-      const int v = v_lo + lane;
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (((keep.f >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+        if (((keep.f >> (8 * j)) & 0xFFu) && ((keep.res >> (8 * j)) & 0xFFu)) --cnt;
     }
   } else {
     for (int v0 = v_lo; v0 < v_hi; v0 += 128) {            // four independent loads in flight per lane
-      uint32_t f[4];
+      uint32_t f[4], res[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + 32 * u + lane;
         f[u] = v < v_hi ? __ldcg(f1 + v) : 0u;
+        res[u] = 0u;
+        if (kCached && v < v_hi) {                         // the resident bytes travel with the flags
+          if (cache_vec && v * 4 + 4 <= C) {
+            res[u] = *reinterpret_cast<const uint32_t*>(cache.resident + v * 4);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (v * 4 + j < C) res[u] |= (cache.resident[v * 4 + j] != 0 ? 1u : 0u) << (8 * j);
+          }
+        }
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         cnt += nonzero_bytes(f[u]);
         if (kCached) {
-          const int v = v0 + 32 * u + lane;
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            if (((f[u] >> (8 * j)) & 0xFFu) && cache.resident[v * 4 + j]) --cnt;
+            if (((f[u] >> (8 * j)) & 0xFFu) && ((res[u] >> (8 * j)) & 0xFFu)) --cnt;
         }
       }
     }
@@ -245,12 +273,12 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
         // cache bookkeeping of Sec. 5.2 for every cluster, activated or not
         const int c = v * 4 + j;
         if (v < v_hi && c < C) {
-          const bool res = cache.resident[c] != 0;
-          int fr = cache.freq[c];
+          const bool res = ((cur.res >> (8 * j)) & 0xFFu) != 0u;
+          int fr = (&cur.fr.x)[j];
           if (on) ++fr; else if (res) --fr;
           if (on || res) cache.freq[c] = fr;
           if (cache.score != nullptr) {
-            const float size_f = (float)cluster_size[c];
+            const float size_f = (float)(((&cur.sz.x)[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
             cache.score[c] = (float)fr * (cache.t_base + size_f * cache.t_transfer) / size_f;
           }
           if (on && res) { fetch = false; atomicAdd(&s_hits, 1); }
@@ -422,28 +450,54 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
     for (int i = tid; i < 33 * 32; i += kThreads) s_group[i] = 0;
     __syncthreads();                                       // also: every queue_of entry is written
     if (!order_keys_early) {
-      for (int i = tid; i < n; i += kThreads) {
-        const unsigned q = __ldcg(queue_of + i);
-        const unsigned cls = by_id ? 0u : (unsigned)__popc(replica_mask[__ldcg(uniq + i)]);
-        key_of[i] = q >= 32u ? 0xFFFFFFFFu : (cls * 32u + q);   // clusters with a bad replica mask are not submitted
-      }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      const unsigned lt = (1u << lane) - 1u;
-      for (int i0 = 0; i0 < n; i0 += 32) {
-        const int i = i0 + lane;
-        const uint32_t key = i < n ? key_of[i] : 0xFFFFFFFFu;
-        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
-        if (key != 0xFFFFFFFFu) {
-          rank_of[i] = (uint32_t)(s_group[key] + __popc(same & lt));
+      // from global memory: four clusters per thread and turn, so that the two dependent reads of each
+      // (its id, then that id's replica mask) overlap with the others'
+      for (int i0 = tid; i0 < n; i0 += 4 * kThreads) {
+        unsigned q[4], m[4];
+        int id[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kThreads;
+          q[u] = i < n ? __ldcg(queue_of + i) : 0xFFu;
+          id[u] = (i < n && !by_id) ? __ldcg(uniq + i) : -1;
         }
-        __syncwarp();
-        if (key != 0xFFFFFFFFu && (same & lt) == 0u) s_group[key] += __popc(same);   // the group's first lane
-        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) m[u] = id[u] >= 0 ? replica_mask[id[u]] : 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kThreads;
+          // clusters with a bad replica mask are not submitted
+          if (i < n) key_of[i] = q[u] >= 32u ? 0xFFFFFFFFu : ((unsigned)__popc(m[u]) * 32u + q[u]);
+        }
       }
     }
     __syncthreads();
+    // The walk is one warp's; its keys come from shared memory.  When the keys live in global memory (more
+    // clusters than the item stage holds, which then is free) they are brought in by all threads, a stage at a time.
+    uint32_t* s_keys = reinterpret_cast<uint32_t*>(s_items);
+    const int walk_cap = staged ? max(n, 1) : (int)(kResolveSmemBytes / 4);
+    for (int c0 = 0; c0 < n; c0 += walk_cap) {
+      const int m_keys = min(walk_cap, n - c0);
+      if (!staged) {
+        for (int i = tid; i < m_keys; i += kThreads) s_keys[i] = key_of[c0 + i];
+        __syncthreads();
+      }
+      if (warp == 0) {
+        const unsigned lt = (1u << lane) - 1u;
+        for (int i0 = c0; i0 < c0 + m_keys; i0 += 32) {
+          const int i = i0 + lane;
+          const uint32_t key = i >= c0 + m_keys ? 0xFFFFFFFFu : (staged ? key_of[i] : s_keys[i - c0]);
+          const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+          if (key != 0xFFFFFFFFu) {
+            rank_of[i] = (uint32_t)(s_group[key] + __popc(same & lt));
+          }
+          __syncwarp();
+          if (key != 0xFFFFFFFFu && (same & lt) == 0u) s_group[key] += __popc(same);   // the group's first lane
+          __syncwarp();
+        }
+      }
+      __syncthreads();
+    }
     if (tid < 32) {                                        // bucket sizes; group counts -> group starts
       int run = 0;
       for (int c = 0; c <= 32; ++c) {
@@ -459,14 +513,24 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
       submitted += s_bucket[q];
       rounds = max(rounds, s_bucket[q]);
     }
-    for (int i = tid; i < n; i += kThreads) {
-      const uint32_t key = key_of[i];
-      if (key == 0xFFFFFFFFu) continue;
-      const int q = (int)(key & 31u);
-      const int depth = s_group[key] + (int)rank_of[i];    // position inside bucket q
-      int pos = 0;
-      for (int q2 = 0; q2 < geo.D; ++q2) pos += min(s_bucket[q2], depth) + ((q2 < q && s_bucket[q2] > depth) ? 1 : 0);
-      r.submit_order[pos] = i;
+    for (int i0 = tid; i0 < n; i0 += 4 * kThreads) {       // four per turn: the reads of key and rank overlap
+      uint32_t key4[4], rank4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * kThreads;
+        key4[u] = i < n ? key_of[i] : 0xFFFFFFFFu;
+        rank4[u] = i < n ? rank_of[i] : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t key = key4[u];
+        if (key == 0xFFFFFFFFu) continue;
+        const int q = (int)(key & 31u);
+        const int depth = s_group[key] + (int)rank4[u];    // position inside bucket q
+        int pos = 0;
+        for (int q2 = 0; q2 < geo.D; ++q2) pos += min(s_bucket[q2], depth) + ((q2 < q && s_bucket[q2] > depth) ? 1 : 0);
+        r.submit_order[pos] = i0 + u * kThreads;
+      }
     }
     if (tid == 0 && r.submit_info != nullptr) {
       r.submit_info[0] = rounds;
