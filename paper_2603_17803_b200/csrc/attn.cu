@@ -446,19 +446,21 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 
   // ---- merge the warps of the CTA (the ring is idle now and is reused as scratch) ------------------
   __syncthreads();
-  float* s_acc = reinterpret_cast<float*>(ring);        // [warp][head 8][128]
-  float* s_m = s_acc + kAttnWarps * 8 * kHeadDim;       // [warp][8]
+  // rows of 128 + 4 floats: the four lanes of a quad store to heads 2*tq, whose rows then start 8 banks apart
+  constexpr int kAccRow = kHeadDim + 4;
+  float* s_acc = reinterpret_cast<float*>(ring);        // [warp][head 8][kAccRow]
+  float* s_m = s_acc + kAttnWarps * 8 * kAccRow;        // [warp][8]
   float* s_l = s_m + kAttnWarps * 8;                    // [warp][8]
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
   if (tq == 0) { s_m[warp * 8 + quad] = m_run; s_l[warp * 8 + quad] = l_run; }
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
-    float* base = s_acc + (warp * 8 + 2 * tq) * kHeadDim + 16 * mt + quad;
+    float* base = s_acc + (warp * 8 + 2 * tq) * kAccRow + 16 * mt + quad;
     base[0] = acc[mt][0];
-    base[kHeadDim] = acc[mt][1];
+    base[kAccRow] = acc[mt][1];
     base[8] = acc[mt][2];
-    base[kHeadDim + 8] = acc[mt][3];
+    base[kAccRow + 8] = acc[mt][3];
   }
   __syncthreads();
   const int t = threadIdx.x;                            // threads 0..127: one output coordinate each
@@ -474,7 +476,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       for (int w = 0; w < kAttnWarps; ++w) {
         const float sc = exp2_or_zero(s_m[w * 8 + hh], M[hh]);
         L[hh] += s_l[w * 8 + hh] * sc;
-        o[hh] += s_acc[(w * 8 + hh) * kHeadDim + t] * sc;
+        o[hh] += s_acc[(w * 8 + hh) * kAccRow + t] * sc;
       }
     }
   }
