@@ -405,7 +405,7 @@ def cpu_baseline(w, budget_s: float):
         fn()
         n += 1
         el = time.perf_counter() - t0
-        if el >= budget_s or n >= 50:
+        if el >= budget_s or n >= 1000:
             break
     return {"value": n / el, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} whole steps of {w.cfg.name} (all {w.cfg.batch * w.cfg.n_q_heads} heads), "
