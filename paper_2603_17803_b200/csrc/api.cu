@@ -383,7 +383,8 @@ int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const 
   a.out = out;
   a.lse = lse;
   a.n_splits = pick_splits(ctx, false);
-  SWARM_TRY(launch_attention(ctx->geo, a, ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream)));
+  SWARM_TRY(launch_attention(ctx->geo, a, ws_ptr<uint32_t>(ctx, ctx->lay.status), static_cast<cudaStream_t>(stream),
+                             /*overlap=*/true));
   return SWARM_OK;
 }
 
@@ -416,7 +417,8 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const in
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (sel != nullptr)   // otherwise: the page bitmaps of this ctx's last swarm_select / swarm_step are reused
     SWARM_TRY(launch_selmap_from_sel(ctx->geo, sel, n_sel, ws_ptr<uint8_t>(ctx, ctx->lay.selmap), st));
-  SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, out, lse), ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
+  SWARM_TRY(launch_attention(ctx->geo, paged_args(ctx, in, out, lse), ws_ptr<uint32_t>(ctx, ctx->lay.status), st,
+                             /*overlap=*/true));
   return SWARM_OK;
 }
 

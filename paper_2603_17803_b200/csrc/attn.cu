@@ -175,6 +175,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   __syncwarp();
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 2);
+  // Stand-alone, the next kernel in the stream may set itself up meanwhile.  Inside the fused step the attention
+  // CTAs release their dependents by exiting: with this trigger the step was measured 1.5 us slower.
+  if (kFused == 0) pdl_launch_dependents();
   pdl_wait();                                           // the selection comes from the previous kernel
   SWARM_STAMP(status, 1);
 
