@@ -244,15 +244,18 @@ def medoid_rows(ksum, page_base, cluster_base, medoid_page):
     return rows
 
 
-def expand_clusters(sel_c, n_sel_c, cluster_base, cluster_page_ptr, cluster_pages):
-    """Pages of the selected clusters of every (request, head): ascending page id, -1 padded, and their number."""
+def expand_clusters(sel_c, n_sel_c, cluster_base, cluster_page_ptr, cluster_pages, ctx_len=None, S=None, window=0):
+    """Pages of the selected clusters of every (request, head): ascending page id, -1 padded, and their number.
+    With ``window`` > 0 the last ``window`` pages of the request (Sec. 4.2, Tier 1 (2): the local window) belong
+    to every head's set as well; ``ctx_len`` and the page size ``S`` then give each request's page count."""
     sel_c, n_sel_c = np.asarray(sel_c), np.asarray(n_sel_c)
     B, Hq, _ = sel_c.shape
     lists = [[None] * Hq for _ in range(B)]
     width = 1
     for b in range(B):
+        P_b = -(-int(ctx_len[b]) // int(S)) if window > 0 else 0
         for h in range(Hq):
-            pages = set()
+            pages = set(range(max(0, P_b - int(window)), P_b))
             for j in range(int(n_sel_c[b, h])):
                 c = int(cluster_base[b]) + int(sel_c[b, h, j])
                 pages.update(int(p) for p in cluster_pages[int(cluster_page_ptr[c]):int(cluster_page_ptr[c + 1])])
@@ -285,7 +288,7 @@ class MedoidStepResult:
 
 def medoid_step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base, replica_mask, cluster_size,
                 cluster_page_ptr, cluster_pages, medoid_page, *, Hkv, S, k_c, D, flags=0,
-                sel_override=None) -> MedoidStepResult:
+                sel_override=None, window=0) -> MedoidStepResult:
     """The step with the medoid index: each cluster is scored by the page upper bound of its medoid page, the k_c
     best clusters of every head are retrieved whole, and the head attends to all of their pages.  The index is a
     context of its own whose "pages" are the clusters, so stages 1-2 are the page routines run on it."""
@@ -297,7 +300,7 @@ def medoid_step(q, ksum, kv_pool, page_base, ctx_len, page2cluster, cluster_base
     s64, s32, cond = scores(q, rows, cluster_base, len_c, Hkv, S, int(max(1, n_c.max())))
     sel_c, n_sel_c = topk(s32, len_c, S, k_c)
     use_c, use_n = (sel_c, n_sel_c) if sel_override is None else sel_override
-    sel_p, n_sel_p = expand_clusters(use_c, use_n, cluster_base, cluster_page_ptr, cluster_pages)
+    sel_p, n_sel_p = expand_clusters(use_c, use_n, cluster_base, cluster_page_ptr, cluster_pages, ctx_len, S, window)
     uniq, queue_of, load = resolve(sel_p, n_sel_p, page_base, page2cluster, cluster_base, replica_mask, cluster_size,
                                    D, flags)
     k_g, v_g, n_tok = gather(kv_pool, sel_p, n_sel_p, page_base, ctx_len, Hkv, d, S)

@@ -610,6 +610,45 @@ def test_medoid_step_scores_medoids_and_attends_whole_clusters():
     assert np.allclose(r.out[b, h], (pr / pr.sum()) @ V, rtol=1e-9, atol=1e-9)
 
 
+def test_medoid_step_local_window_joins_every_head_and_covers_the_context_at_full_width():
+    """Sec. 4.2, Tier 1 (2): the last W pages are attended whatever the index selects.  Pins: each head's set is the
+    union of its clusters' members and the window; W = 0 changes nothing; with W >= P every head attends the whole
+    context, i.e. plain dense attention (Eq. 1 over all tokens), and every cluster of the request is scheduled."""
+    from paper_2603_17803_b200 import workloads as W
+    cfg = W.scaled(W.CONFIGS["c5_skewed"], batch=2, ctx_range=(200, 700), top_k=8, n_topics=5)
+    w = W.generate(cfg, seed=11)
+    ptr, members, medoid = (t.numpy() for t in W.cluster_members(w))
+    u = W.bits_u16
+    pb, cl, cb = w.page_base.numpy(), w.ctx_len.numpy(), w.cluster_base.numpy()
+    p2c = w.page2cluster.numpy()
+    mask = w.cluster_replica_mask.numpy().view(np.uint32)
+    size = w.cluster_size.numpy().view(np.uint16)
+    S, Hq, g = cfg.page_size, cfg.n_q_heads, cfg.n_q_heads // cfg.n_kv_heads
+    ksum = oracle.build_summaries(u(w.kv_pool), pb, cl, cfg.n_kv_heads, cfg.head_dim, S)
+    run = lambda window: oracle.medoid_step(u(w.q), ksum, u(w.kv_pool), pb, cl, p2c, cb, mask, size, ptr, members, medoid,
+                                            Hkv=cfg.n_kv_heads, S=S, k_c=2, D=cfg.n_queues, window=window)
+    r0, r3, rall = run(0), run(3), run(10_000)
+    assert np.array_equal(r0.sel_clusters, r3.sel_clusters)            # the window does not touch the index
+    f = lambda bits: (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    pool = u(w.kv_pool)
+    for b in range(cfg.batch):
+        P = -(-int(cl[b]) // S)
+        for h in range(Hq):
+            base = set(r0.sel_pages[b, h, :r0.n_sel_pages[b, h]].tolist())
+            assert set(r3.sel_pages[b, h, :r3.n_sel_pages[b, h]].tolist()) == base | set(range(max(0, P - 3), P))
+            assert list(rall.sel_pages[b, h, :rall.n_sel_pages[b, h]]) == list(range(P))
+            K = f(pool[pb[b]:pb[b] + P, h // g, 0]).reshape(P * S, -1)[: int(cl[b])]
+            V = f(pool[pb[b]:pb[b] + P, h // g, 1]).reshape(P * S, -1)[: int(cl[b])]
+            logits = K @ f(u(w.q)[b, h]) / np.sqrt(cfg.head_dim)
+            pr = np.exp(logits - logits.max())
+            assert np.allclose(rall.out[b, h], (pr / pr.sum()) @ V, rtol=1e-9, atol=1e-9)
+    assert list(rall.uniq) == list(range(int(cb[-1])))                  # everything is fetched
+    window_clusters = {int(cb[b]) + int(p2c[pb[b] + p]) for b in range(cfg.batch)
+                       for p in range(max(0, -(-int(cl[b]) // S) - 3), -(-int(cl[b]) // S))}
+    assert set(r3.uniq.tolist()) == set(r0.uniq.tolist()) | window_clusters
+    replay_check(r3.uniq, r3.queue_of, r3.load, mask, size, cfg.n_queues, 0)
+
+
 # --------------------------------------------------------------------------------- batched submission order
 
 def test_submit_order_hand_case():
