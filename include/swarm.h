@@ -281,12 +281,14 @@ int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* inputs, con
  * inputs and the cache state are not used by the scheduling, and the ctx must have been created with
  * max_clusters_total >= n_pool_pages (SWARM_ERR_INVALID_ARG otherwise; uniq and queue_of sized accordingly).
  * A member page outside the request sets SWARM_DEV_BAD_PAGE and is skipped.  The local window of the shape
- * is not applied.  Page bitmaps longer than 160 KiB per head (1.3 M pages) are SWARM_ERR_UNSUPPORTED. */
+ * (Sec. 4.2, Tier 1 (2)) applies: the last local_window_pages pages of every request join every head's set of
+ * attended pages and are scheduled like the members of the selected clusters (through page2cluster, or as
+ * pages under entry-level scheduling); the window does not take places from the top_k_clusters clusters.  Page bitmaps longer than 160 KiB per head (1.3 M pages) are SWARM_ERR_UNSUPPORTED. */
 int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_medoid_index* index,
                           const swarm_outputs* outputs, void* stream);
 
-/* Which clusters the fast tier holds (no ctx; Sec. 4.2 Tier 1 (3): "clusters are cached in descending order of
- * this score" under a fixed capacity; Sec. 5.2: the cached set follows the updated scores).  Clusters are taken in
+/* Which clusters the fast tier holds (no ctx; Sec. 4.2 Tier 1 (3): the fast tier is filled with the clusters of
+ * highest Eq. 6 score under a fixed capacity; Sec. 5.2: the cached set follows the updated scores).  Clusters are taken in
  * descending score (the Eq. 6 values swarm_set_cache maintains; ties to the lower id) while their sizes
  * (cluster_size, pages) still fit into capacity_pages; the first cluster that does not fit ends the admission.
  * Writes resident[c] = 1 or 0 for every cluster -- the table swarm_set_cache reads -- and, if info is not NULL,

@@ -591,7 +591,7 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
                                    idx->cluster_page_ptr, idx->cluster_pages, in->ctx_len,
                                    ws_ptr<uint8_t>(ctx, ctx->lay.selmap), ws_ptr<uint8_t>(ctx, ctx->lay.flags), status, st,
                                    true, idx->entry_replica_mask != nullptr ? in->page_base : nullptr,
-                                   idx->n_member_entries));
+                                   idx->n_member_entries, in->page_base, in->page2cluster));
   AttnArgs a = paged_args(ctx, in, o->out, o->lse);
   a.n_splits = pick_splits(ctx, true, /*fused=*/true);
   ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);

@@ -7,8 +7,8 @@
 // exactly like cluster_base.  What this file adds is the glue around them:
 //   medoid_rows_kernel     index build: copy the summary rows of the medoid pages into the index
 //   cluster_len_kernel     pseudo context lengths (clusters of the request x page size) for the page kernels
-//   expand_clusters_kernel selected clusters -> per-head bitmap of their member pages (what the attention
-//                          kernel reads) and the cluster flags (what the resolve kernel reads)
+//   expand_clusters_kernel selected clusters -> per-head bitmap of their member pages plus the local window (what
+//                          the attention kernel reads) and the cluster flags (what the resolve kernel reads)
 #include "swarm_internal.cuh"
 
 namespace swarm {
@@ -55,7 +55,8 @@ expand_clusters_kernel(Geometry geo, int k_c, int pitch, const int32_t* __restri
                        const int32_t* __restrict__ n_sel_c, const int64_t* __restrict__ cluster_base,
                        const int64_t* __restrict__ cluster_page_ptr, const int32_t* __restrict__ cluster_pages,
                        const int32_t* __restrict__ ctx_len, uint8_t* __restrict__ selmap, uint8_t* __restrict__ flags,
-                       uint32_t* __restrict__ status, const int64_t* __restrict__ entry_base, long long n_member_entries) {
+                       uint32_t* __restrict__ status, const int64_t* __restrict__ entry_base, long long n_member_entries,
+                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ page2cluster) {
   extern __shared__ uint32_t s_row[];
   const int bh = blockIdx.x, b = bh / geo.Hq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -87,6 +88,20 @@ expand_clusters_kernel(Geometry geo, int k_c, int pitch, const int32_t* __restri
       }
     }
   }
+  // the local window (Sec. 4.2, Tier 1 (2)): the last W pages of the request join every head's set and are
+  // scheduled like the members of the selected clusters
+  for (int p = max(0, P - geo.W) + tid; p < P && p < pitch * 8; p += blockDim.x) {
+    atomicOr(&s_row[p >> 5], 1u << (p & 31));
+    if (entry_base != nullptr) {
+      const long long unit = entry_base[b] + p;
+      if (unit < geo.Cmax) flags[unit] = 1;
+      else err |= SWARM_DEV_BAD_CLUSTER;
+    } else {
+      const int c = page2cluster[page_base[b] + p];
+      if (c < 0 || c >= cn - cb || cb + c >= geo.Cmax) err |= SWARM_DEV_BAD_CLUSTER;
+      else flags[cb + c] = 1;
+    }
+  }
   if (err) atomicOr(status, err);
   __syncthreads();
   uint32_t* row = reinterpret_cast<uint32_t*>(selmap + (long long)bh * pitch);
@@ -116,11 +131,11 @@ cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* 
                                    const int64_t* cluster_base, const int64_t* cluster_page_ptr,
                                    const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
                                    uint32_t* status, cudaStream_t st, bool overlap, const int64_t* entry_base,
-                                   long long n_member_entries) {
+                                   long long n_member_entries, const int64_t* page_base, const int32_t* page2cluster) {
   const int pitch = selmap_pitch_bytes(geo.Pmax);
   return launch_pdl(expand_clusters_kernel, dim3((unsigned)(geo.B * geo.Hq)), dim3(256), (size_t)pitch, st, overlap, geo,
                     k_c, pitch, sel_c, n_sel_c, cluster_base, cluster_page_ptr, cluster_pages, ctx_len, selmap, flags,
-                    status, entry_base, n_member_entries);
+                    status, entry_base, n_member_entries, page_base, page2cluster);
 }
 
 }  // namespace swarm

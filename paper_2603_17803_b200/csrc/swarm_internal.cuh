@@ -153,7 +153,7 @@ cudaError_t launch_expand_clusters(const Geometry& geo, int k_c, const int32_t* 
                                    const int64_t* cluster_base, const int64_t* cluster_page_ptr,
                                    const int32_t* cluster_pages, const int32_t* ctx_len, uint8_t* selmap, uint8_t* flags,
                                    uint32_t* status, cudaStream_t st, bool overlap, const int64_t* entry_base,
-                                   long long n_member_entries);
+                                   long long n_member_entries, const int64_t* page_base, const int32_t* page2cluster);
 
 // Algorithm 1 (offline co-activation clustering): see cluster.cu.
 long long build_clusters_workspace_bytes(int n);

@@ -501,7 +501,7 @@ def test_selection_at_every_list_length(pages, window):
 
 
 # ---- medoid index (Sec. 4.2 Tier 1 (1)): clusters are scored by their medoid page and retrieved whole -------
-def check_medoid_step(w, sess, k_c, flags=0):
+def check_medoid_step(w, sess, k_c, flags=0, window=0):
     torch.cuda.synchronize()
     assert sess.status() == 0
     cfg = w.cfg
@@ -515,7 +515,7 @@ def check_medoid_step(w, sess, k_c, flags=0):
     r = oracle.medoid_step(W.bits_u16(w.q), ksum, W.bits_u16(w.kv_pool), tabs["page_base"], tabs["ctx_len"],
                            tabs["page2cluster"], tabs["cluster_base"], tabs["replica_mask"], tabs["cluster_size"],
                            ptr, members, medoid, Hkv=cfg.n_kv_heads, S=cfg.page_size, k_c=k_c, D=cfg.n_queues,
-                           flags=flags, sel_override=(sel_c, n_sel_c))
+                           flags=flags, sel_override=(sel_c, n_sel_c), window=window)
     cb = tabs["cluster_base"]
     exact = 0
     for b in range(cfg.batch):
@@ -775,6 +775,64 @@ def test_algorithm1_clusters_drive_the_medoid_step():
     assert np.array_equal(o.queue_load.cpu().numpy()[: cfg.n_queues], load) and int(load.sum()) == n
     want_order, rounds = oracle.submit_order(queue_of, entry_masks[uniq], cfg.n_queues)
     assert np.array_equal(sess.submit_order.cpu().numpy()[:n], want_order)
+    parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
+    sess.close()
+
+
+@pytest.mark.parametrize("name,k_c,window", [("c2_small", 12, 3), ("c5_small", 4, 2), ("k_exceeds_pages", 7, 5),
+                                             ("c4_small", 9, 64), ("c3_small", 1, 40)])
+def test_medoid_step_with_local_window(name, k_c, window):
+    """The paper's whole Tier-1 step: clusters chosen through the medoid index, attended whole, plus the local
+    window (requests shorter than the window are attended densely)."""
+    cfg = CASES[name]
+    window = min(window, cfg.top_k)                         # the shape allows 0 <= W <= top_k
+    w = W.generate(cfg, seed=83, device=DEV)
+    sess = Session(w, local_window_pages=window)
+    sess.enable_medoid_index(k_c, keep_scores=True)
+    sess.step_medoid()
+    check_medoid_step(w, sess, k_c, window=window)
+    sess.step()                                             # the page step with the same window still works
+    parity.check_step(w, sess)
+    sess.step_medoid()
+    check_medoid_step(w, sess, k_c, window=window)
+    sess.close()
+
+
+def test_medoid_step_entry_level_with_local_window():
+    """Entry-level scheduling: the window's pages are units of their own, like the members of the selected clusters."""
+    cfg = small("c2_128k", ctx_len=16 * 300 + 7, top_k=32, n_topics=6)
+    window = 5
+    w = W.generate(cfg, seed=89, device=DEV)
+    P = cfg.max_pages()
+    ptr, members, medoid = W.cluster_members(w)
+    entry_masks = oracle.entry_replica_masks(ptr.cpu().numpy(), members.cpu().numpy(), P, cfg.n_queues)
+    # give every third page a second copy so that the scheduling has something to decide
+    entry_masks = entry_masks.copy()
+    entry_masks[::3] |= np.uint32(1) << ((np.arange(P)[::3] // 3) % cfg.n_queues).astype(np.uint32)
+    sess = Session(w, local_window_pages=window, max_clusters_total=P)
+    sess.enable_medoid_index(4)
+    masks_dev = torch.from_numpy(entry_masks.view(np.int32)).to(DEV)
+    index = B.make_medoid_index(medoid_ksum=sess.medoid_ksum, cluster_page_ptr=sess.cluster_page_ptr,
+                                cluster_pages=sess.cluster_pages, cluster_ctx_len=sess.cluster_ctx_len, top_k_clusters=4,
+                                max_clusters_per_req=sess.max_clusters_per_req, entry_replica_mask=masks_dev)
+    B.swarm_step_medoid(sess.ctx, sess.inputs, index, sess.medoid_outputs)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    tabs = parity.host_tables(w)
+    sel_c, n_sel_c = sess.sel_clusters.cpu().numpy(), sess.n_sel_clusters.cpu().numpy()
+    sel_p, n_sel_p = oracle.expand_clusters(sel_c, n_sel_c, tabs["cluster_base"], ptr.cpu().numpy(), members.cpu().numpy(),
+                                            tabs["ctx_len"], cfg.page_size, window)
+    assert all(set(range(P - window, P)) <= set(sel_p[0, h, : n_sel_p[0, h]].tolist()) for h in range(cfg.n_q_heads))
+    uniq, queue_of, load = oracle.resolve(sel_p, n_sel_p, tabs["page_base"], np.arange(P, dtype=np.int32), tabs["page_base"],
+                                          entry_masks, np.ones(P, dtype=np.uint16), cfg.n_queues, oracle.UNIT_LOAD)
+    o = sess.o
+    n = int(o.n_uniq.cpu().numpy()[0])
+    assert n == len(uniq) and np.array_equal(o.uniq.cpu().numpy()[:n], uniq)
+    assert np.array_equal(o.queue_of.cpu().numpy()[:n], queue_of)
+    assert np.array_equal(o.queue_load.cpu().numpy()[: cfg.n_queues], load)
+    k_g, v_g, n_tok = oracle.gather(W.bits_u16(w.kv_pool), sel_p, n_sel_p, tabs["page_base"], tabs["ctx_len"],
+                                    cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
+    out, lse = oracle.attention(W.bits_u16(w.q), k_g, v_g, n_tok)
     parity.check_attention(o.out.cpu().numpy(), o.lse.cpu().numpy(), out, lse)
     sess.close()
 
