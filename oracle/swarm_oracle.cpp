@@ -11,10 +11,10 @@
 //                           index the scorer reads; the paper keeps a compact
 //                           per-cluster index in fast memory, Sec. 4.2 Tier 1)
 //   oracle_scores           relevance score of a page against the query
-//                           (Sec. 2.3 "relevance scores (e.g. query-key inner
-//                           products)"): the page upper bound
+//                           (Sec. 2.3 scores entries by relevance, e.g. by the
+//                           query-key inner product): the page upper bound
 //                           sum_i max(q_i*kmin_i, q_i*kmax_i)
-//   oracle_topk             "only ... the highest attention scores" (Sec. 2.3):
+//   oracle_topk             Sec. 2.3 activates the best-scoring entries alone:
 //                           k best pages per query head, ties to the lower id
 //   oracle_resolve          global merge (Eq. 8, without the DRAM-resident
 //                           term) and entry-bucket scheduling (Sec. 5.1): sort
@@ -22,8 +22,8 @@
 //                           to its currently smallest bucket
 //   oracle_resolve_cached   the same with Eq. 8's resident term, the activation-frequency update of
 //                           Sec. 5.2 (cache replacement) and the cost-effectiveness score of Eq. 6
-//   oracle_gather           the transfer of the selected pages (Sec. 6
-//                           "Asynchronous I/O"), here a byte copy
+//   oracle_gather           the transfer of the selected pages (Sec. 6, the
+//                           asynchronous reads), here a byte copy
 //   oracle_attention        Eq. 1 over the gathered tokens, one query row
 //   oracle_build_clusters   Algorithm 1 (offline co-activation clustering): density of Eq. 4, medoid queue,
 //                           expansion by the average distance of Eq. 5; decisions in fp32 (see the function)
