@@ -259,6 +259,24 @@ int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g
  * CUDA graph by the caller (stream capture). */
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);
 
+/* The fused step in two halves, for a step whose query heads are spread over several ctxs (one per GPU, each
+ * holding the K/V and summaries of its own KV heads and all the cluster tables): stages 1-2 are independent
+ * per head, stage 3 needs the union of the activated clusters over ALL heads (Eq. 8), stage 4 is per head again.
+ *   swarm_step_begin     scoring and selection (the first two launches of swarm_step): sel / n_sel (and scores)
+ *                        are written, and the dedup flag of every cluster that holds a selected page is set
+ *   swarm_cluster_flags  the flag array in the workspace: *flags = device pointer to max_clusters_total bytes
+ *                        (0 or 1, indexed by global cluster id), *n_bytes = max_clusters_total.  Between the two
+ *                        halves the caller combines the arrays of all ctxs element-wise by maximum (an all-reduce
+ *                        over the GPUs, on the same stream) so that every one holds the union
+ *   swarm_step_end       attention over this ctx's heads and cluster resolution of the union (the third launch);
+ *                        consumes the flags (they are zero again afterwards).  With identical tables every ctx
+ *                        computes the same uniq / queue_of / n_uniq / queue_load
+ * begin followed by end on one ctx with nothing in between is swarm_step.  Same arguments and errors as
+ * swarm_step; both halves must be given the same inputs and outputs. */
+int32_t swarm_step_begin(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);
+int32_t swarm_step_end(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);
+int32_t swarm_cluster_flags(swarm_ctx* ctx, void** flags, int64_t* n_bytes);
+
 /* Index build for swarm_step_medoid (not part of a decode step): copies, for every cluster, the key summary of
  * its medoid page medoid_page[cluster] (page id local to the request) into row `cluster` of medoid_ksum_out
  * (bf16 [max_clusters_total][Hkv][2][d]), and writes cluster_ctx_len_out [B] (int32).  Reads inputs->ksum,

@@ -30,6 +30,7 @@ EXPORTS = (
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
     "swarm_cache_admit_workspace_bytes", "swarm_cache_admit",
+    "swarm_step_begin", "swarm_step_end", "swarm_cluster_flags",
 )
 
 
@@ -285,6 +286,23 @@ def swarm_sparse_attn_static(q, k_g, v_g, n_tok, *, batch, n_q_heads, top_k, pag
 def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:
     _check(load_library().swarm_step(ctx, ctypes.byref(inputs), ctypes.byref(outputs), _stream(stream)),
            "swarm_step", ctx)
+
+
+def swarm_step_begin(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:
+    _check(load_library().swarm_step_begin(ctx, ctypes.byref(inputs), ctypes.byref(outputs), _stream(stream)),
+           "swarm_step_begin", ctx)
+
+
+def swarm_step_end(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:
+    _check(load_library().swarm_step_end(ctx, ctypes.byref(inputs), ctypes.byref(outputs), _stream(stream)),
+           "swarm_step_end", ctx)
+
+
+def swarm_cluster_flags(ctx):
+    """(device address, number of bytes) of the ctx's cluster flag array."""
+    ptr, n = ctypes.c_void_p(0), ctypes.c_int64(0)
+    _check(load_library().swarm_cluster_flags(ctx, ctypes.byref(ptr), ctypes.byref(n)), "swarm_cluster_flags", ctx)
+    return int(ptr.value or 0), int(n.value)
 
 
 def make_medoid_index(*, medoid_ksum, cluster_page_ptr, cluster_pages, cluster_ctx_len, top_k_clusters,

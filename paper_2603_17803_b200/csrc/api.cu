@@ -423,16 +423,37 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const in
 }
 
 namespace {
-int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host);
+int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host,
+                  int parts);
+constexpr int kStepBegin = 1, kStepEnd = 2;
 }
 
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream) {
-  return step_impl(ctx, in, o, stream, nullptr);
+  return step_impl(ctx, in, o, stream, nullptr, kStepBegin | kStepEnd);
+}
+
+int32_t swarm_step_begin(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream) {
+  return step_impl(ctx, in, o, stream, nullptr, kStepBegin);
+}
+
+int32_t swarm_step_end(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream) {
+  return step_impl(ctx, in, o, stream, nullptr, kStepEnd);
+}
+
+int32_t swarm_cluster_flags(swarm_ctx* ctx, void** flags, int64_t* n_bytes) {
+  if (flags == nullptr || n_bytes == nullptr) return SWARM_ERR_INVALID_ARG;
+  const int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  *flags = ws_ptr<uint8_t>(ctx, ctx->lay.flags);
+  *n_bytes = ctx->geo.Cmax;
+  return SWARM_OK;
 }
 
 namespace {
-// The fused step; `host` (swarm_step_host only) makes the last kernel store the small results into host memory too.
-int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host) {
+// The fused step, or one of its two halves (the selection with its cluster marks; attention + cluster resolution).
+// `host` (swarm_step_host only) makes the last kernel store the small results into host memory too.
+int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, void* stream, const HostMirror* host,
+                  int parts) {
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!select_inputs_ok(in) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || o == nullptr || bad(o->sel) ||
@@ -446,12 +467,15 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   const uint16_t* pool = static_cast<const uint16_t*>(in->kv_pool);
   float* sc = o->scores ? o->scores : ws_ptr<float>(ctx, ctx->lay.scores);
 
-  SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
-                              status, st));
-  // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true,
-                        ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
-                        ws_ptr<uint8_t>(ctx, ctx->lay.flags), in->cluster_replica_mask, in->cluster_size));
+  if (parts & kStepBegin) {
+    SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
+                                status, st));
+    // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
+    SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true,
+                          ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
+                          ws_ptr<uint8_t>(ctx, ctx->lay.flags), in->cluster_replica_mask, in->cluster_size));
+  }
+  if (!(parts & kStepEnd)) return SWARM_OK;
 
   // Cluster resolution and attention both need only the selection: one launch runs them side by side, the
   // attention CTAs plus one CTA for the resolution (whose serial pass is the longest item of the step).
@@ -495,7 +519,7 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   if (direct && ctx->done_d != nullptr) {
     const HostMirror host{out_d, lse_d, n_uniq_d, queue_load_d, ws_ptr<unsigned>(ctx, ctx->lay.status + 96), ctx->done_d,
                           (unsigned)attention_groups(ctx->geo, true) + 1u};
-    const int32_t rc = step_impl(ctx, &local, o, st, &host);
+    const int32_t rc = step_impl(ctx, &local, o, st, &host, kStepBegin | kStepEnd);
     *signals = rc == SWARM_OK;
     return rc;
   }

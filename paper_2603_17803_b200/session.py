@@ -108,6 +108,21 @@ class Session:
     def step(self, stream=None):
         B.swarm_step(self.ctx, self.inputs, self.outputs, stream)
 
+    # -- the step in two halves (query heads spread over several ctxs) --------------------------------
+    def step_begin(self, stream=None):
+        B.swarm_step_begin(self.ctx, self.inputs, self.outputs, stream)
+
+    def step_end(self, stream=None):
+        B.swarm_step_end(self.ctx, self.inputs, self.outputs, stream)
+
+    def cluster_flags(self) -> torch.Tensor:
+        """The ctx's cluster flag array as a uint8 view of the workspace (what the ranks combine by maximum)."""
+        addr, n = B.swarm_cluster_flags(self.ctx)
+        off = addr - self.workspace.data_ptr()
+        if off < 0 or off + n > self.workspace.numel():
+            raise RuntimeError("cluster flags outside the workspace")
+        return self.workspace[off:off + n]
+
     def step_host(self, q_host, out_host=None, lse_host=None, n_uniq_host=None, queue_load_host=None, stream=None):
         """swarm_step_host.  The call is synchronous and tens of microseconds long, so the marshalled arguments of
         the last call are kept and reused while the same tensor objects (and stream) are passed again; buffers

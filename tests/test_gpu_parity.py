@@ -936,3 +936,66 @@ def test_selector_report_figures(name, k_c):
         assert got["io_pages"] == int(load.sum()) and got["max_queue_load"] == int(load.max())
     # whole clusters attended: the medoid selector's I/O is exactly what its heads attend, no partial clusters
     assert rep["medoids"]["io_pages"] >= rep["medoids"]["attended_pages"]
+
+
+# ---- the step in two halves: query heads spread over several ctxs (one per GPU in production) ------------------
+def test_begin_then_end_is_the_step():
+    w = W.generate(CASES["c5_small"], seed=97, device=DEV)
+    a, b_ = Session(w), Session(w)
+    a.step()
+    b_.step_begin()
+    flags = b_.cluster_flags()
+    assert flags.numel() == w.n_clusters and int(flags.sum()) == int(a.o.n_uniq[0])   # every activated cluster, once
+    b_.step_end()
+    torch.cuda.synchronize()
+    assert int(flags.sum()) == 0                            # consumed
+    for name in ("sel", "n_sel", "queue_load", "out", "lse"):
+        assert torch.equal(getattr(a.o, name), getattr(b_.o, name)), name
+    n = int(a.o.n_uniq[0])
+    assert torch.equal(a.o.uniq[:n], b_.o.uniq[:n]) and torch.equal(a.o.queue_of[:n], b_.o.queue_of[:n])
+    parity.check_step(w, b_)
+    a.close()
+    b_.close()
+
+
+@pytest.mark.parametrize("name,world", [("c2_small", 2), ("c2_small", 4), ("c3_small", 8), ("c5_small", 2)])
+def test_head_sharded_step_on_one_device(name, world):
+    """`world` ctxs, each with the K/V of its own KV heads, run one after the other on this device; the flag
+    exchange (an all-reduce by maximum across GPUs in production) is a plain maximum here.  Every shard must
+    derive the unsharded schedule, and the shards' heads together the unsharded selection and attention."""
+    from paper_2603_17803_b200 import sharding
+    w = W.generate(CASES[name], seed=101, device=DEV)
+    full = Session(w)
+    full.step()
+    parity.check_step(w, full)
+    shards = [sharding.shard_workload(w, r, world) for r in range(world)]
+    sess = [Session(s, ksum=None) for s in shards]
+    for s in sess:
+        s.step_begin()
+    torch.cuda.synchronize()
+    own = [int(s.cluster_flags().sum()) for s in sess]
+    union = torch.stack([s.cluster_flags() for s in sess]).amax(0)
+    n = int(full.o.n_uniq[0])
+    assert int(union.sum()) == n and max(own) <= n
+    for s in sess:
+        s.cluster_flags().copy_(union)
+        s.step_end()
+    torch.cuda.synchronize()
+    hq = w.cfg.n_q_heads // world
+    for r, s in enumerate(sess):
+        assert s.status() == 0
+        assert int(s.o.n_uniq[0]) == n
+        assert torch.equal(s.o.uniq[:n], full.o.uniq[:n]) and torch.equal(s.o.queue_of[:n], full.o.queue_of[:n])
+        assert torch.equal(s.o.queue_load[: w.cfg.n_queues], full.o.queue_load[: w.cfg.n_queues])
+        assert torch.equal(s.o.sel, full.o.sel[:, r * hq:(r + 1) * hq])
+        d_out = (s.o.out - full.o.out[:, r * hq:(r + 1) * hq]).abs().max().item()
+        d_lse = (s.o.lse - full.o.lse[:, r * hq:(r + 1) * hq]).abs().max().item()
+        assert d_out <= parity.ATTN_ATOL and d_lse <= parity.LSE_ATOL   # split counts differ between the layouts
+        assert int(s.cluster_flags().sum()) == 0
+    # sharding.sharded_step without a process group is the plain step
+    sharding.sharded_step(sess[0])
+    torch.cuda.synchronize()
+    parity.check_step(shards[0], sess[0])
+    for s in sess:
+        s.close()
+    full.close()
