@@ -687,8 +687,10 @@ int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outp
     }
   }
   bool signals = false;
+  if (ctx->done_h != nullptr) *static_cast<volatile unsigned*>(ctx->done_h) = 0u;
   rc = enqueue_host_step(ctx, in, o, q_host, out_host, lse_host, n_uniq_host, queue_load_host, st, &signals);
   if (rc != SWARM_OK) return rc;
+  if (signals && cap == cudaStreamCaptureStatusNone && wait_done_word(ctx)) return SWARM_OK;
   SWARM_TRY(cudaStreamSynchronize(st));
   return SWARM_OK;
 }
