@@ -241,6 +241,9 @@ def test_invalid_arguments_are_rejected_on_the_host():
     with pytest.raises(B.SwarmError) as e:
         B.swarm_set_workspace(ctx, torch.empty(16, dtype=torch.uint8, device=DEV))
     assert e.value.code == B.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(B.SwarmError) as e:                # the flag array lives in the workspace
+        B.swarm_cluster_flags(ctx)
+    assert e.value.code == B.ERR_WORKSPACE_TOO_SMALL
     ws = torch.empty(B.swarm_workspace_bytes(shape), dtype=torch.uint8, device=DEV)
     B.swarm_set_workspace(ctx, ws)
     with pytest.raises(B.SwarmError) as e:                # null input
@@ -249,6 +252,12 @@ def test_invalid_arguments_are_rejected_on_the_host():
     with pytest.raises(B.SwarmError) as e:                # misaligned pointer
         B.swarm_select(ctx, B.make_inputs(q=t[1:], ksum=t, page_base=t, ctx_len=t), None, t, t)
     assert e.value.code == B.ERR_INVALID_ARG
+    addr, n = B.swarm_cluster_flags(ctx)
+    assert n == 4 and ws.data_ptr() <= addr and addr + n <= ws.data_ptr() + ws.numel()
+    for half in (B.swarm_step_begin, B.swarm_step_end):    # the halves validate like the whole step
+        with pytest.raises(B.SwarmError) as e:
+            half(ctx, B.make_inputs(q=t, ksum=t, page_base=t, ctx_len=t), B.make_outputs(sel=t, n_sel=t))
+        assert e.value.code == B.ERR_INVALID_ARG
     B.swarm_destroy(ctx)
 
 
