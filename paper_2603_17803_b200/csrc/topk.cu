@@ -204,29 +204,14 @@ __device__ __forceinline__ void finish_by_ranking(SelectState& st, int tid, int 
 }
 
 // ---- register-resident variant -------------------------------------------------------------------
-template <int THREADS, int ITEMS>
-__global__ void __launch_bounds__(THREADS)
-topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
-                 int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
-  __shared__ SelectState st;
+// The selection of one list with ITEMS consecutive pages per thread (the kernel was launched for lists of up to
+// THREADS * MAX_ITEMS pages; rows of the page bitmap are that long).
+template <int THREADS, int ITEMS, int MAX_ITEMS>
+__device__ __forceinline__ void topk_regs_body(SelectState& st, const Geometry& geo, const TopkExtras& x,
+                                               const RequestBases& rb, const float* __restrict__ s,
+                                               int32_t* __restrict__ out, int32_t* __restrict__ n_sel,
+                                               uint32_t* __restrict__ status, int bh, int P, int Pw, int k_eff, int k_sel) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int bh = blockIdx.x, b = bh / geo.Hq;
-  pdl_launch_dependents();
-  SWARM_STAMP(status, 0);
-  SWARM_KERNEL_BEGIN(status, 1);
-  for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
-  prefetch_tables(geo, x);
-  const RequestBases rb = load_bases(x, b);
-  const int len_b = ctx_len[b];
-  pdl_wait();                                               // the scores come from the previous kernel
-  SWARM_STAMP(status, 1);
-  const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
-  const int k_eff = min(geo.k, P);
-  const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
-  const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
-  const float* s = scores + (long long)bh * geo.Pmax;
-  int32_t* out = sel + (long long)bh * geo.k;
-
   // thread t owns pages [t*ITEMS, (t+1)*ITEMS); keys of pages that do not exist are never used
   uint32_t key[ITEMS];
   const int p0 = tid * ITEMS;
@@ -372,7 +357,42 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   }
   for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
+  if (ITEMS < MAX_ITEMS && x.selmap != nullptr) {          // the part of the bitmap row these threads do not reach
+    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
+    for (int o = THREADS * ITEMS / 8 + tid * 4; o + 4 <= x.selmap_pitch; o += THREADS * 4)
+      *reinterpret_cast<uint32_t*>(row + o) = 0u;
+  }
   SWARM_STAMP(status, 13);
+}
+
+template <int THREADS, int ITEMS>
+__global__ void __launch_bounds__(THREADS)
+topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
+                 int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
+  __shared__ SelectState st;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int bh = blockIdx.x, b = bh / geo.Hq;
+  pdl_launch_dependents();
+  SWARM_STAMP(status, 0);
+  SWARM_KERNEL_BEGIN(status, 1);
+  for (int i = tid; i < kBins; i += THREADS) st.hist[i] = 0;
+  prefetch_tables(geo, x);
+  const RequestBases rb = load_bases(x, b);
+  const int len_b = ctx_len[b];
+  pdl_wait();                                               // the scores come from the previous kernel
+  SWARM_STAMP(status, 1);
+  const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
+  const int k_eff = min(geo.k, P);
+  const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
+  const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
+  const float* s = scores + (long long)bh * geo.Pmax;
+  int32_t* out = sel + (long long)bh * geo.k;
+  // A list half as long as the kernel's capacity is handled with half the pages per thread: the work of every
+  // phase is per page held, and the lists of one launch differ in length (ragged batches).
+  if (ITEMS == 16 && P <= THREADS * 8)
+    topk_regs_body<THREADS, 8, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
+  else
+    topk_regs_body<THREADS, ITEMS, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
   SWARM_KERNEL_END(status, 1);
 }
 
