@@ -11,7 +11,8 @@
 // (k - #greater) pages with key == T, placed by a block-wide scan of per-thread counts.  That order
 // gives "ties go to the lower page id" and the ascending-id output at once.
 //
-// topk_regs keeps ITEMS consecutive pages per thread in registers (lists of up to 16384 pages);
+// topk_regs keeps ITEMS consecutive pages per thread in registers (lists of up to 16384 pages; in the
+// largest instance a list of at most half that length is handled with half the pages per thread);
 // topk_generic walks lists of any length in shared or global memory with the same algorithm.
 #include "swarm_internal.cuh"
 
