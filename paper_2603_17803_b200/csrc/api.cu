@@ -526,8 +526,7 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
   const int32_t rc = swarm_step(ctx, &local, o, st);
   if (rc != SWARM_OK) return rc;
   if (direct) {
-    SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d,
-                             ws_ptr<unsigned>(ctx, ctx->lay.status + 96), nullptr, st));
+    SWARM_TRY(launch_publish(ctx->geo, o->out, o->lse, o->n_uniq, o->queue_load, out_d, lse_d, n_uniq_d, queue_load_d, st));
     return SWARM_OK;
   }
   if (out_host) SWARM_TRY(cudaMemcpyAsync(out_host, o->out, bh * kHeadDim * 4, cudaMemcpyDeviceToHost, st));

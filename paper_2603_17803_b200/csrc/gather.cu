@@ -120,9 +120,8 @@ cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool,
 // addressing) instead of by copy operations: a copy node between kernels costs several microseconds of
 // engine hand-over, a load or store over the bus does not.
 //   fetch_kernel    the step's queries, host -> workspace (volatile loads: the host rewrites the buffer between calls)
-//   publish_kernel  the step's small results, device -> host; 16-byte vectors for out, words for the rest.  The
-//                   last CTA to finish then raises `done` (a word in host memory) after a system-wide fence, so
-//                   the caller can wait on that word instead of on the stream.
+//   publish_kernel  the step's small results, device -> host; 16-byte vectors for out, words for the rest (used
+//                   when the step's last kernel cannot store them itself, see HostMirror)
 namespace {
 __global__ void __launch_bounds__(256)
 fetch_kernel(const uint4* src_h, uint4* __restrict__ dst, int n16) {
@@ -137,7 +136,7 @@ fetch_kernel(const uint4* src_h, uint4* __restrict__ dst, int n16) {
 __global__ void __launch_bounds__(256)
 publish_kernel(const float* __restrict__ out, const float* __restrict__ lse, const int32_t* __restrict__ n_uniq,
                const int32_t* __restrict__ queue_load, float* out_h, float* lse_h, int32_t* n_uniq_h,
-               int32_t* queue_load_h, int n_out4, int n_lse, int n_queues, unsigned* ticket, unsigned* done_h) {
+               int32_t* queue_load_h, int n_out4, int n_lse, int n_queues) {
   pdl_wait();                                               // the results come from the previous kernel
   const int t = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
   if (out_h != nullptr)
@@ -148,18 +147,6 @@ publish_kernel(const float* __restrict__ out, const float* __restrict__ lse, con
   if (queue_load_h != nullptr)
     for (int i = t; i < n_queues; i += stride) queue_load_h[i] = __ldcg(queue_load + i);
   if (n_uniq_h != nullptr && t == 0) *n_uniq_h = __ldcg(n_uniq);
-  if (done_h != nullptr) {
-    __threadfence_system();                                 // this thread's stores are visible to the host ...
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      const unsigned arrived = atomicAdd(ticket, 1u);       // ... before the CTA is counted
-      if (arrived == gridDim.x - 1) {
-        *ticket = 0u;                                       // ready for the next call
-        __threadfence_system();
-        *reinterpret_cast<volatile unsigned*>(done_h) = 1u;
-      }
-    }
-  }
 }
 }  // namespace
 
@@ -172,11 +159,11 @@ cudaError_t launch_fetch(const void* src_h, void* dst, long long bytes, cudaStre
 
 cudaError_t launch_publish(const Geometry& geo, const float* out, const float* lse, const int32_t* n_uniq,
                            const int32_t* queue_load, float* out_h, float* lse_h, int32_t* n_uniq_h,
-                           int32_t* queue_load_h, unsigned* ticket, unsigned* done_h, cudaStream_t st) {
+                           int32_t* queue_load_h, cudaStream_t st) {
   const int n_out4 = geo.B * geo.Hq * kHeadDim / 4;
   const int grid = max(1, min(32, (n_out4 + 255) / 256));
   return launch_pdl(publish_kernel, dim3(grid), dim3(256), 0, st, true, out, lse, n_uniq, queue_load, out_h, lse_h,
-                    n_uniq_h, queue_load_h, n_out4, geo.B * geo.Hq, geo.D, ticket, done_h);
+                    n_uniq_h, queue_load_h, n_out4, geo.B * geo.Hq, geo.D);
 }
 
 }  // namespace swarm

@@ -108,11 +108,10 @@ cudaError_t launch_resolve(const ResolveArgs& r, cudaStream_t st, bool overlap);
 cudaError_t launch_gather(const Geometry& geo, const uint16_t* kv_pool, const int32_t* sel, const int32_t* n_sel,
                           const int64_t* page_base, const int32_t* ctx_len, uint16_t* k_out, uint16_t* v_out,
                           int32_t* n_tok, uint32_t* status, cudaStream_t st);
-// The step's small results written by a kernel into device-addressable host memory (any *_h may be null); the
-// last CTA then sets *done_h (host memory, may be null) using the zero-initialised counter `ticket`.
+// The step's small results written by a kernel into device-addressable host memory (any *_h may be null).
 cudaError_t launch_publish(const Geometry& geo, const float* out, const float* lse, const int32_t* n_uniq,
                            const int32_t* queue_load, float* out_h, float* lse_h, int32_t* n_uniq_h,
-                           int32_t* queue_load_h, unsigned* ticket, unsigned* done_h, cudaStream_t st);
+                           int32_t* queue_load_h, cudaStream_t st);
 // `bytes` (a multiple of 16) from device-addressable host memory into device memory, by a kernel.
 cudaError_t launch_fetch(const void* src_h, void* dst, long long bytes, cudaStream_t st);
 // Attention over contiguous gathered buffers (pool == nullptr) or straight from the pool (k_g == nullptr).
