@@ -47,6 +47,9 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="call the library directly instead of replaying graphs")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--attn-splits", type=int, default=0, help="key-range splits of the attention kernel (0: chosen from the shape)")
+    ap.add_argument("--shard", default="none", choices=["none", "heads"],
+                    help="heads: ONE step stream whose KV heads are spread over the ranks (strong scaling; the ranks "
+                         "exchange the cluster flags once per step); default: independent replicas")
     return ap.parse_args()
 
 
@@ -412,6 +415,64 @@ def cpu_baseline(w, budget_s: float):
                       f"OpenMP over (request, head) units, {el:.1f} s"}
 
 
+def run_sharded(args):
+    """--shard heads: every rank holds the K/V of its own KV heads of the SAME workload; a step is selection,
+    all-reduce(max) of the cluster flags, attention + resolution (paper_2603_17803_b200.sharding).  Plain launches,
+    no graph (the collective sits between the two halves)."""
+    import torch
+    from paper_2603_17803_b200 import replicas, sharding
+    from paper_2603_17803_b200 import workloads as W
+    from paper_2603_17803_b200.session import Session
+
+    world, rank, local_rank = replicas.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    replicas.init("nccl", dev)
+    K = args.steps if args.steps is not None else 5000
+    Wm = max(3, args.warmup if args.warmup is not None else 50)
+    cfg = W.CONFIGS[args.workload]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    sessions = []
+    for r in range(args.n_rot):                             # the same data sets on every rank, each keeps its heads
+        w = W.generate(cfg, seed=r, device=dev, step=r)
+        sessions.append(Session(sharding.shard_workload(w, rank, world)))
+        del w
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(Wm):
+            sharding.sharded_step(sessions[i % args.n_rot], stream)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_a = time.perf_counter()
+        e0.record(stream)
+        for i in range(K):
+            sharding.sharded_step(sessions[i % args.n_rot], stream)
+        e1.record(stream)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        t_b = time.perf_counter()
+        ms = e0.elapsed_time(e1)
+    sampler.stop()
+    ms, = replicas.max_over_ranks([ms], device=dev)
+    status = max(s.status() for s in sessions)
+    n_flags = int(sessions[0].cluster_flags().numel())
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "parallelism": f"kv-head shards x{world}: one all-reduce(max) of {n_flags} "
+                                                             "cluster-flag bytes per step, every rank schedules the union",
+                       "l2_policy": f"rotating {args.n_rot} independent data sets", "launch": "plain launches, no graph"},
+            "gpu_launches": K * 3, "device_status": status, "clocks": sampler.summary([(t_a, t_b)])}))
+    replicas.shutdown()
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on the host cores, same config / metric / unit."""
     rank = int(os.environ.get("RANK", "0"))
@@ -467,5 +528,7 @@ if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.shard == "heads":
+        run_sharded(a)
     else:
         run_swarm(a)
