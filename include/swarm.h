@@ -171,6 +171,16 @@ int32_t swarm_set_submit_order(swarm_ctx* ctx, int32_t* submit_order, int32_t* s
  * from the shape).  Results do not depend on it beyond floating-point rounding. */
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits);
 
+/* Which kernel scores the pages (stage 1).  The result is the same sum either way, within fp32 rounding.
+ *   SWARM_SCORER_AUTO    the streaming tensor-core kernel whenever the shape allows it (batch <= 1024 and fewer
+ *                        than 2^31 pool pages), else the fp32-pipe kernel
+ *   SWARM_SCORER_TENSOR  the streaming tensor-core kernel; SWARM_ERR_UNSUPPORTED if the shape does not allow it
+ *   SWARM_SCORER_FP32    the fp32-pipe kernel (16-byte row loads, sign-split weights in registers) */
+#define SWARM_SCORER_AUTO 0
+#define SWARM_SCORER_TENSOR 1
+#define SWARM_SCORER_FP32 2
+int32_t swarm_set_scorer(swarm_ctx* ctx, int32_t kind);
+
 /* Index build (not part of a decode step): per page and KV head, element-wise min and max of
  * the valid tokens' keys -- the compact index the scorer reads instead of the keys themselves
  * (the role the in-memory cluster index plays in Sec. 4.2, Tier 1).
@@ -200,14 +210,18 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* inputs, const
 
 /* Stage 4a: copy the selected pages' K and V blocks, in `sel` order, into contiguous per-head
  * buffers (the transfer the paper performs across storage tiers, Sec. 6; here within HBM).
- * Rows beyond the valid tokens are zero.  n_tok may be NULL. */
+ * Rows beyond the valid tokens are zero.  n_tok may be NULL.
+ * `sel` as swarm_select writes it: ascending page ids.  What matters is that a partial last page of a request,
+ * if selected, is the LAST entry of its head (swarm_sparse_attn masks only the end of the buffer); a selection
+ * that places it elsewhere sets SWARM_DEV_BAD_PAGE and that page is skipped (its slot is zero-filled). */
 int32_t swarm_gather(swarm_ctx* ctx, const swarm_inputs* inputs, const int32_t* sel, const int32_t* n_sel,
                      void* k_out, void* v_out, int32_t* n_tok, void* stream);
 
 /* Stage 4b: Eq. 1 for one query row per head over its own gathered tokens,
  *   out[b][h] = softmax_t(q . K_t / sqrt(d)) V_t  over t < n_tok[b][h],  lse = log sum exp,
  * computed as split-K partials (fp32) merged by their log-sum-exp.  k_g / v_g are
- * bf16 [B][Hq][k*S][d].  n_tok[b][h] must be >= 1. */
+ * bf16 [B][Hq][k*S][d].  n_tok[b][h] must be in [1, k*S]: a value outside [0, k*S] sets SWARM_DEV_BAD_LENGTH
+ * and is clamped to that range. */
 int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
                           float* out, float* lse, void* stream);
 
@@ -244,12 +258,18 @@ int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* inputs, cons
  * The per-head arrival counters must be zero when a call starts: they are zero when the library is
  * loaded and the kernel sets each one back to zero after using it, so nothing has to be cleared
  * between calls.  Two calls whose kernels overlap on the GPU (different streams, or graph
- * branches) race on the array; serialise them. */
+ * branches) race on the array; serialise them.
+ * Device-side faults: the kernel reports them like the other entry points (n_tok outside [0, top_k * page_size]
+ * sets SWARM_DEV_BAD_LENGTH and is clamped; a bounded wait that runs out sets SWARM_DEV_TIMEOUT and leaves
+ * out / lse of that head undefined), in a status word inside the same array.
+ * swarm_sparse_attn_static_status copies that word to *bits and clears it; it SYNCHRONISES `stream` and, like
+ * the entry point itself, allocates nothing. */
 #define SWARM_STATIC_MAX_HEADS 2048
 #define SWARM_STATIC_SCRATCH_BYTES (256 + 4096 * (128 + 2) * 4 + SWARM_STATIC_MAX_HEADS * 4)
 int32_t swarm_sparse_attn_static(const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
                                  int32_t batch, int32_t n_q_heads, int32_t top_k, int32_t page_size, float* out,
                                  float* lse, void* stream);
+int32_t swarm_sparse_attn_static_status(void* stream, uint32_t* bits);
 
 /* The fused step: stages 1-4 enqueued back to back with no host round trip.  Attention reads the
  * selected pages straight from the pool; the gathered copies are written only when k_out / v_out

@@ -355,6 +355,75 @@ def build_clusters(dist, tau, members_cap=None):
     return rho, ptr[:C + 1].copy(), members[:int(ptr[C])].copy(), medoid[:C].copy()
 
 
+def build_clusters_plain(dist, tau, members_cap=None, near_rtol=1e-5):
+    """Algorithm 1 with Step 4's test as Eq. 5 prints it: the average distance to the current members, recomputed
+    from scratch in double for every candidate.  Returns (rho, ptr, members, medoid, n_near) where n_near counts
+    the join decisions within near_rtol * tau of the radius."""
+    dist = np.ascontiguousarray(dist, dtype=np.float32)
+    n = dist.shape[0]
+    assert dist.shape == (n, n)
+    cap = int(members_cap if members_cap is not None else max(1, n) * 64)
+    rho = np.zeros(n, dtype=np.int32)
+    ptr = np.zeros(n + 1, dtype=np.int32)
+    members = np.zeros(cap, dtype=np.int32)
+    medoid = np.zeros(n, dtype=np.int32)
+    n_c = np.zeros(1, dtype=np.int32)
+    n_near = np.zeros(1, dtype=np.int64)
+    _check(_load().oracle_build_clusters_plain(_p(dist), ctypes.c_int32(n), ctypes.c_float(tau),
+                                               ctypes.c_double(near_rtol), _p(rho), _p(ptr), _p(members),
+                                               ctypes.c_int64(cap), _p(medoid), _p(n_c), _p(n_near)),
+           "build_clusters_plain")
+    C = int(n_c[0])
+    return rho, ptr[:C + 1].copy(), members[:int(ptr[C])].copy(), medoid[:C].copy(), int(n_near[0])
+
+
+def replay_clusters(dist, tau, ptr, members, medoid, near_rtol=1e-5):
+    """Band rule for a clustering someone else computed (Algorithm 1; Eq. 4, Eq. 5).  Walks the given clusters in
+    order and checks every step against the plain statement: the medoid is the first uncovered entry of the queue
+    (density descending, index ascending), the candidates are visited by (distance to the medoid, index), and a
+    candidate joined exactly when the average of its distances to the members so far -- recomputed in double -- is
+    <= tau, EXCEPT that a decision whose margin |average - tau| is at most near_rtol * tau may go either way (the
+    replay then follows the given clustering).  Returns the number of such near decisions; raises AssertionError
+    on the first step that is wrong outside the band."""
+    d32 = np.ascontiguousarray(dist, dtype=np.float32)
+    n = d32.shape[0]
+    d64 = d32.astype(np.float64)
+    tau32, tau64 = np.float32(tau), float(np.float32(tau))
+    within = d32 <= tau32
+    rho = within.sum(axis=1) - within.diagonal().astype(np.int64)
+    queue = sorted(range(n), key=lambda i: (-int(rho[i]), i))
+    covered = np.zeros(n, dtype=bool)
+    qi, near = 0, 0
+    ptr, members, medoid = np.asarray(ptr), np.asarray(members), np.asarray(medoid)
+    for c in range(len(medoid)):
+        assert not covered.all(), "a cluster was created after every entry was covered"
+        while covered[queue[qi]]:
+            qi += 1
+        m = queue[qi]
+        assert int(medoid[c]) == m, f"cluster {c}: medoid {int(medoid[c])}, expected {m}"
+        given = members[ptr[c]:ptr[c + 1]].tolist()
+        assert given and given[0] == m, f"cluster {c} does not start with its medoid"
+        idx = np.flatnonzero(within[m])
+        idx = idx[idx != m]
+        cand = idx[np.lexsort((idx, d32[m, idx]))].tolist()     # by (distance to the medoid, index)
+        mem, gi = [m], 1
+        for e in cand:
+            avg = float(d64[mem, e].sum() / len(mem))
+            joined = gi < len(given) and given[gi] == e
+            if abs(avg - tau64) <= near_rtol * tau64:
+                near += 1
+            else:
+                assert joined == (avg <= tau64), \
+                    f"cluster {c}, candidate {e}: average {avg!r} vs tau {tau64!r}, joined={joined}"
+            if joined:
+                mem.append(e)
+                gi += 1
+        assert gi == len(given), f"cluster {c} holds entries that are not candidates, or out of order"
+        covered[mem] = True
+    assert covered.all(), "entries left uncovered"
+    return near
+
+
 # ---- placement of the clusters' entries across the SSDs (Eq. 7) and entry-level scheduling --------------------
 def entry_replica_masks(cluster_ptr, cluster_members, n_entries, D):
     """Round-robin placement of Eq. 7: clusters are laid out one after another, a global pointer advances by one

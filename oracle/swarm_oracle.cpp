@@ -427,4 +427,57 @@ int oracle_build_clusters(const float* D, int32_t n, float tau, int32_t* rho, in
   return ORACLE_OK;
 }
 
+// Algorithm 1 again, with Step 4's test written as Eq. 5 states it: for every candidate the AVERAGE of its
+// distances to the current members, recomputed from scratch in double over the members in joining order and
+// compared with tau in double.  No running sums, nothing in fp32 beyond the matrix entries themselves.  Same
+// density, medoid queue, candidate order and outputs as oracle_build_clusters.  *n_near counts the join
+// decisions whose margin |average - tau| is at most near_rtol * tau: those are the decisions a different
+// summation order or precision may legitimately take the other way.
+int oracle_build_clusters_plain(const float* D, int32_t n, float tau, double near_rtol, int32_t* rho, int32_t* ptr,
+                                int32_t* members, int64_t members_cap, int32_t* medoid, int32_t* n_clusters,
+                                int64_t* n_near) {
+  if (!D || !rho || !ptr || !members || !medoid || !n_clusters || !n_near || n < 1) return ORACLE_BAD_ARG;
+  const double tau_d = static_cast<double>(tau);
+  for (int32_t i = 0; i < n; ++i) {
+    int32_t c = 0;
+    for (int32_t j = 0; j < n; ++j)
+      if (j != i && D[static_cast<int64_t>(i) * n + j] <= tau) ++c;
+    rho[i] = c;
+  }
+  std::vector<int32_t> queue(static_cast<size_t>(n));
+  for (int32_t i = 0; i < n; ++i) queue[static_cast<size_t>(i)] = i;
+  std::stable_sort(queue.begin(), queue.end(), [rho](int32_t a, int32_t b) { return rho[a] > rho[b]; });
+  std::vector<char> covered(static_cast<size_t>(n), 0);
+  int32_t n_cov = 0, nc = 0;
+  int64_t fill = 0, near = 0;
+  ptr[0] = 0;
+  for (int32_t qi = 0; qi < n && n_cov < n; ++qi) {
+    const int32_t m = queue[static_cast<size_t>(qi)];
+    if (covered[static_cast<size_t>(m)]) continue;
+    const float* row_m = D + static_cast<int64_t>(m) * n;
+    std::vector<int32_t> cand;
+    for (int32_t e = 0; e < n; ++e)
+      if (e != m && row_m[e] <= tau) cand.push_back(e);
+    std::stable_sort(cand.begin(), cand.end(), [row_m](int32_t a, int32_t b) { return row_m[a] < row_m[b]; });
+    std::vector<int32_t> mem{m};
+    for (int32_t e : cand) {
+      double total = 0.0;
+      for (int32_t c : mem) total += static_cast<double>(D[static_cast<int64_t>(c) * n + e]);
+      const double avg = total / static_cast<double>(mem.size());
+      if (std::fabs(avg - tau_d) <= near_rtol * tau_d) ++near;
+      if (avg <= tau_d) mem.push_back(e);
+    }
+    if (fill + static_cast<int64_t>(mem.size()) > members_cap) return ORACLE_BAD_ARG;
+    for (int32_t e : mem) {
+      members[fill++] = e;
+      if (!covered[static_cast<size_t>(e)]) { covered[static_cast<size_t>(e)] = 1; ++n_cov; }
+    }
+    medoid[nc] = m;
+    ptr[++nc] = static_cast<int32_t>(fill);
+  }
+  *n_clusters = nc;
+  *n_near = near;
+  return ORACLE_OK;
+}
+
 }  // extern "C"

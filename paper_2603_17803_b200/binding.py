@@ -20,13 +20,14 @@ ERR_STATIC_SCRATCH_TOO_SMALL = 5
 STATIC_MAX_HEADS = 2048
 DEV_BAD_PAGE, DEV_BAD_CLUSTER, DEV_BAD_REPLICA, DEV_BAD_LENGTH, DEV_TIMEOUT = 1, 2, 4, 8, 16
 ORDER_BY_ID, UNIT_LOAD = 1, 2
+SCORER_AUTO, SCORER_TENSOR, SCORER_FP32 = 0, 1, 2
 _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA",
               5: "STATIC_SCRATCH_TOO_SMALL"}
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
-    "swarm_set_attn_splits", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
-    "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
+    "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_sparse_attn_static_status", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
     "swarm_cache_admit_workspace_bytes", "swarm_cache_admit",
@@ -167,6 +168,10 @@ def swarm_set_attn_splits(ctx, n_splits: int) -> None:
     _check(load_library().swarm_set_attn_splits(ctx, ctypes.c_int32(n_splits)), "swarm_set_attn_splits", ctx)
 
 
+def swarm_set_scorer(ctx, kind: int) -> None:
+    _check(load_library().swarm_set_scorer(ctx, ctypes.c_int32(kind)), "swarm_set_scorer", ctx)
+
+
 def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_base=0.0, t_transfer=0.0) -> None:
     """Attach cache state (uint8 resident, int32 freq, optional float32 score, optional int32 n_hit), or detach it
     when ``resident`` is None.  The caller keeps the tensors alive while they are attached."""
@@ -281,6 +286,14 @@ def swarm_sparse_attn_static(q, k_g, v_g, n_tok, *, batch, n_q_heads, top_k, pag
                                                    ctypes.c_int32(n_q_heads), ctypes.c_int32(top_k),
                                                    ctypes.c_int32(page_size), _ptr(out, "out"), _ptr(lse, "lse"),
                                                    _stream(stream)), "swarm_sparse_attn_static")
+
+
+def swarm_sparse_attn_static_status(stream=None) -> int:
+    """Reads and clears the device status word of swarm_sparse_attn_static (synchronises the stream)."""
+    bits = ctypes.c_uint32(0)
+    _check(load_library().swarm_sparse_attn_static_status(_stream(stream), ctypes.byref(bits)),
+           "swarm_sparse_attn_static_status")
+    return int(bits.value)
 
 
 def swarm_step(ctx, inputs: swarm_inputs, outputs: swarm_outputs, stream=None) -> None:

@@ -179,6 +179,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   g.S = shape->page_size; g.k = shape->top_k; g.D = shape->n_queues; g.Pmax = shape->max_pages_per_req;
   g.Cmax = shape->max_clusters_total; g.flags = shape->flags; g.n_pool_pages = shape->n_pool_pages;
   g.W = shape->local_window_pages;
+  g.scorer = SWARM_SCORER_AUTO;
   ctx->lay = make_layout(*shape);
   ctx->ws = nullptr;
   ctx->ws_bytes = 0;
@@ -244,6 +245,14 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits) {
   if (ctx == nullptr || n_splits < 0 || n_splits > kMaxSplits) return SWARM_ERR_INVALID_ARG;
   ctx->user_splits = n_splits;
+  return SWARM_OK;
+}
+
+int32_t swarm_set_scorer(swarm_ctx* ctx, int32_t kind) {
+  if (ctx == nullptr || kind < SWARM_SCORER_AUTO || kind > SWARM_SCORER_FP32) return SWARM_ERR_INVALID_ARG;
+  if (kind == SWARM_SCORER_TENSOR && !score_streams(ctx->geo)) return SWARM_ERR_UNSUPPORTED;
+  ctx->geo.scorer = kind;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
   return SWARM_OK;
 }
 

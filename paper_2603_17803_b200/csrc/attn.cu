@@ -28,6 +28,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "swarm_internal.cuh"
 #include "resolve_body.cuh"
 
@@ -233,6 +235,10 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     for (int w2 = 0; w2 < kAttnWarps; ++w2) n_items += s_wcnt[w2];
   } else {
     total_tok = a.n_tok[bh0];
+    if (total_tok < 0 || total_tok > geo.k * S) {          // more tokens than the head's buffer holds: attend what it holds
+      if (threadIdx.x == 0 && split == 0) atomicOr(status, SWARM_DEV_BAD_LENGTH);
+      total_tok = max(0, min(total_tok, geo.k * S));
+    }
     n_items = (total_tok + S - 1) / S;
   }
   const int it_begin = (int)((long long)n_items * split / a.n_splits);
@@ -716,7 +722,8 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
 // ---------------------------------------------------------------------------------------------
 // Allocation-free variant of swarm_sparse_attn (see swarm.h).  The split-K partials live in a
 // file-scope device array instead of a caller-provided workspace.  Layout of the array:
-//   [0, 256)                       status word (unused by the contiguous-buffer kernel) + padding
+//   [0, 256)                       device status word (bits SWARM_DEV_*; read and cleared by
+//                                  swarm_sparse_attn_static_status) + padding
 //   [256, 256 + kSlots*128*4)      partial accumulators, one 128-float row per (head, split) slot
 //   [.., .. + kSlots*2*4)          partial (max, sum) pairs
 //   [.., .. + kMaxHeads*4)         per-head arrival counters; zero at load (static storage) and set
@@ -730,20 +737,30 @@ static_assert(SWARM_STATIC_SCRATCH_BYTES == 256 + kStaticSlots * (swarm::kHeadDi
 static __device__ __align__(256) unsigned char g_static_scratch[SWARM_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+struct StaticDevice {
+  unsigned char* scratch;   // device address of the array on this device; null until the set-up has run
+  int sms;
+};
+StaticDevice g_static_dev[kMaxDevices] = {};
 
-cudaError_t static_scratch_address(unsigned char** out) {
+// Set-up for the current device, on the first call there (idempotent if two threads race): the array's
+// address, the SM count, the kernels' shared-memory attribute.  Allocates nothing.
+cudaError_t static_device(const StaticDevice** out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (g_static_ptr[dev] == nullptr) {   // set-up for this device (idempotent if two threads race here)
+  if (g_static_dev[dev].scratch == nullptr) {
     void* p = nullptr;
+    int sms = 0;
     e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = swarm::configure_attention();
     if (e != cudaSuccess) return e;
-    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    g_static_dev[dev].sms = sms > 0 ? sms : 1;
+    g_static_dev[dev].scratch = static_cast<unsigned char*>(p);
   }
-  *out = g_static_ptr[dev];
+  *out = &g_static_dev[dev];
   return cudaSuccess;
 }
 }  // namespace
@@ -759,16 +776,16 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   const long long bh = (long long)batch * n_q_heads;
   if (bh > SWARM_STATIC_MAX_HEADS) return SWARM_ERR_STATIC_SCRATCH_TOO_SMALL;
   if (bh * top_k >= (1LL << 31)) return SWARM_ERR_UNSUPPORTED;
-  // same split heuristic as the ctx path (about 2 CTAs per SM, >= 4 pages per split), capped by the array
-  long long n = 148 / bh;
-  n = n < (top_k / 4 > 1 ? top_k / 4 : 1) ? n : (top_k / 4 > 1 ? top_k / 4 : 1);
-  n = n < kMaxSplits ? n : kMaxSplits;
-  n = n < kStaticSlots / bh ? n : kStaticSlots / bh;
-  n = n < 1 ? 1 : n;
+  const StaticDevice* dev = nullptr;
+  if (static_device(&dev) != cudaSuccess) return SWARM_ERR_CUDA;
+  // same split heuristic as the ctx path (one wave of CTAs, at least 4 pages per split); the array holds
+  // kStaticSlots >= 2 * SWARM_STATIC_MAX_HEADS (head, split) slots, and the last bound keeps any SM count inside it
+  long long n = std::max<long long>(1, dev->sms / bh);
+  n = std::min<long long>(n, std::max(1, top_k / 4));
+  n = std::min<long long>(n, kMaxSplits);
+  n = std::min<long long>(n, kStaticSlots / bh);
 
-  unsigned char* base = nullptr;
-  if (static_scratch_address(&base) != cudaSuccess) return SWARM_ERR_CUDA;
-  if (configure_attention() != cudaSuccess) return SWARM_ERR_CUDA;   // raises a kernel attribute; allocates nothing
+  unsigned char* base = dev->scratch;
   Geometry geo{};
   geo.B = batch; geo.Hq = n_q_heads; geo.Hkv = n_q_heads; geo.g = 1; geo.S = page_size; geo.k = top_k; geo.D = 1;
   geo.Pmax = top_k; geo.Cmax = 1; geo.flags = 0; geo.n_pool_pages = 0; geo.W = 0;
@@ -785,4 +802,15 @@ extern "C" int32_t swarm_sparse_attn_static(const void* q, const void* k_g, cons
   a.n_splits = (int)n;
   return launch_attention(geo, a, reinterpret_cast<uint32_t*>(base), static_cast<cudaStream_t>(stream)) == cudaSuccess
              ? SWARM_OK : SWARM_ERR_CUDA;
+}
+
+extern "C" int32_t swarm_sparse_attn_static_status(void* stream, uint32_t* bits) {
+  if (bits == nullptr) return SWARM_ERR_INVALID_ARG;
+  const StaticDevice* dev = nullptr;
+  if (static_device(&dev) != cudaSuccess) return SWARM_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(bits, dev->scratch, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(dev->scratch, 0, sizeof(uint32_t), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return SWARM_ERR_CUDA;
+  return SWARM_OK;
 }

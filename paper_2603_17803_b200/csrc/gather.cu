@@ -28,6 +28,13 @@ gather_kernel(Geometry geo, const uint16_t* __restrict__ kv_pool, const int32_t*
     if (threadIdx.x == 0) atomicOr(status, SWARM_DEV_BAD_PAGE);
     p = -1;
   }
+  // The attention over gathered buffers masks only the end of the last slot: a partial page anywhere else would
+  // put its padding rows among the valid tokens.  The library's own selections are ascending, so this can only
+  // happen with a selection the caller wrote.
+  if (p == P - 1 && tail != S && j != ns - 1) {
+    if (threadIdx.x == 0) atomicOr(status, SWARM_DEV_BAD_PAGE);
+    p = -1;
+  }
   const int valid = p < 0 ? 0 : (p == P - 1 ? tail : S);
   const uint4 zero = make_uint4(0, 0, 0, 0);
   const uint16_t* src = kv_pool + (((page_base[b] + max(p, 0)) * geo.Hkv + h / geo.g) * 2) * blk;

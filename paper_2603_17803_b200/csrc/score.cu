@@ -432,12 +432,14 @@ cudaError_t configure_score() {
   return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaSmemBytes);
 }
 
+bool score_streams(const Geometry& geo) { return geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31); }
+
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st) {
   // Streaming tensor-core variant whenever the batch fits its prefix table and the pool fits 32-bit TMA
   // coordinates; otherwise the register-resident grid kernel on the fp32 pipes.
-  if (geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31))
+  if (geo.scorer != SWARM_SCORER_FP32 && score_streams(geo))
     return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, st);
   // Heads of a KV group are processed G at a time, G the largest of 8/4/2/1 dividing the group size.
   if (geo.g % 8 == 0) return launch_one<8, 4, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);

@@ -35,6 +35,7 @@ struct Geometry {   // plain copy of the shape in kernel-friendly form
   int W;                // local window in pages: the last W pages of a request are always selected
   unsigned flags;
   long long n_pool_pages;
+  int scorer;           // SWARM_SCORER_*: which kernel scores the pages
 };
 
 // ---- one-time per-device kernel attribute set-up (dynamic shared-memory limits) ---------------
@@ -48,6 +49,7 @@ cudaError_t configure_medoid();
 // ---- kernel launchers (each returns cudaGetLastError() after the launch) ----------------------
 cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool, const int64_t* page_base,
                                    const int32_t* ctx_len, uint16_t* ksum, uint32_t* status, cudaStream_t st);
+bool score_streams(const Geometry& geo);   // the shape allows the streaming tensor-core scorer
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st);

@@ -34,7 +34,7 @@ class Session:
 
     def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
                  ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0,
-                 max_clusters_total: Optional[int] = None):
+                 max_clusters_total: Optional[int] = None, scorer: int = B.SCORER_AUTO):
         cfg = workload.cfg
         self.cfg = cfg
         self.w = workload
@@ -51,6 +51,8 @@ class Session:
         self.ctx = B.swarm_create(self.shape)
         self.workspace = torch.empty(B.swarm_workspace_bytes(self.shape), dtype=torch.uint8, device=dev)
         B.swarm_set_workspace(self.ctx, self.workspace)
+        if scorer != B.SCORER_AUTO:
+            B.swarm_set_scorer(self.ctx, scorer)
         self.ksum = ksum if ksum is not None else torch.empty(
             (workload.n_pool_pages, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
         self.inputs = self._inputs(workload.q)

@@ -72,6 +72,36 @@ def test_fused_step_equals_composition(name):
         s.close()
 
 
+@pytest.mark.parametrize("hq,hkv", [(16, 2), (8, 2), (6, 3), (5, 5), (6, 2)])
+def test_fp32_pipe_scorer_matches_oracle(hq, hkv):
+    """The scorer on the fp32 pipes (what shapes beyond the streaming kernel's limits fall back to), forced by
+    swarm_set_scorer: groups of 8, 4, 2 and 1 query heads per KV head (its four instantiations; a group of 3 runs
+    the single-head one three times), ragged tails, requests of unequal length, then the whole step on top."""
+    cfg = small("c5_skewed", batch=3, n_q_heads=hq, n_kv_heads=hkv, ctx_range=(16 * 9, 16 * 333), top_k=24, n_topics=5)
+    w = W.generate(cfg, seed=31, device=DEV)
+    ref = Session(w, keep_scores=True, keep_gathered=True)
+    ref.step()
+    sess = Session(w, keep_scores=True, keep_gathered=True, scorer=B.SCORER_FP32, ksum=ref.ksum)
+    run_separate_calls(sess)
+    info = parity.check_step(w, sess)
+    assert info["heads"] == cfg.batch * hq
+    sess.step()
+    parity.check_step(w, sess)
+    # the two scorers agree far inside the tolerance of the score rule
+    torch.cuda.synchronize()
+    a, b = ref.o.scores, sess.o.scores
+    live = torch.isfinite(a)
+    assert torch.equal(live, torch.isfinite(b))
+    assert ((a[live] - b[live]).abs() <= 1e-5 * a[live].abs() + 1e-4).all()
+    with pytest.raises(B.SwarmError):
+        B.swarm_set_scorer(sess.ctx, 3)
+    B.swarm_set_scorer(sess.ctx, B.SCORER_TENSOR)
+    sess.step()
+    parity.check_step(w, sess)
+    ref.close()
+    sess.close()
+
+
 @pytest.mark.parametrize("name", ["c1_tiny", "c2_128k"])
 def test_full_size_configs_match_oracle(name):
     """The two configurations the oracle handles whole, at full size, through the fused step."""
@@ -104,6 +134,45 @@ def test_c5_full_size_sampled():
     sess.enable_submit_order()
     sess.step()
     assert check_submit_order(w, sess) > 20000
+    sess.close()
+
+
+def test_caller_supplied_selection_and_misplaced_partial_page():
+    """swarm_gather / swarm_sparse_attn on a selection the caller wrote (ascending, a subset of the pages, the
+    partial last page included): parity with the oracle; the same pages with the partial page NOT last are
+    refused for that page (status bit, slot zero-filled) instead of attending its padding rows."""
+    cfg = small("c2_128k", ctx_len=16 * 300 + 5, top_k=20, n_topics=4)
+    w = W.generate(cfg, seed=17, device=DEV)
+    sess = Session(w, keep_gathered=True)
+    P = cfg.max_pages()
+    rng = np.random.default_rng(2)
+    sel = np.full((1, cfg.n_q_heads, cfg.top_k), -1, dtype=np.int32)
+    n_sel = np.zeros((1, cfg.n_q_heads), dtype=np.int32)
+    for h in range(cfg.n_q_heads):
+        n = int(rng.integers(1, cfg.top_k + 1))
+        pages = np.sort(rng.choice(P - 1, size=n - 1, replace=False)) if n > 1 else np.zeros(0, np.int64)
+        sel[0, h, :n] = np.concatenate([pages, [P - 1]])     # the partial page, last
+        n_sel[0, h] = n
+    sel_t, n_sel_t = torch.from_numpy(sel).to(DEV), torch.from_numpy(n_sel).to(DEV)
+    sess.gather(sel_t, n_sel_t)
+    sess.sparse_attn()
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    tabs = parity.host_tables(w)
+    pool = parity.bits_u16(w.kv_pool)
+    kg, vg, n_tok = oracle.gather(pool, sel, n_sel, tabs["page_base"], tabs["ctx_len"], cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
+    assert np.array_equal(parity.bits_u16(sess.o.k_out), kg) and np.array_equal(parity.bits_u16(sess.o.v_out), vg)
+    assert np.array_equal(sess.o.n_tok.cpu().numpy(), n_tok)
+    out_ref, lse_ref = oracle.attention(parity.bits_u16(w.q), kg, vg, n_tok)
+    parity.check_attention(sess.o.out.cpu().numpy(), sess.o.lse.cpu().numpy(), out_ref, lse_ref)
+    # the partial page first: flagged and skipped
+    h = int(np.argmax(n_sel[0] >= 2))
+    n = int(n_sel[0, h])
+    sel[0, h, :n] = np.concatenate([[P - 1], sel[0, h, :n - 1]])
+    sess.gather(torch.from_numpy(sel).to(DEV), n_sel_t)
+    torch.cuda.synchronize()
+    assert sess.status() == B.DEV_BAD_PAGE
+    assert not sess.o.k_out[0, h, : cfg.page_size].any()
     sess.close()
 
 
@@ -654,7 +723,17 @@ def test_submit_order_full_size_and_bad_masks():
 def check_clusters(dist, tau, cap=None):
     density, ptr, members, medoid = B.swarm_build_clusters(dist, tau, members_cap=cap)
     torch.cuda.synchronize()
-    rho, ptr_ref, members_ref, medoid_ref = oracle.build_clusters(dist.cpu().numpy(), tau, members_cap=cap)
+    d_host = dist.cpu().numpy()
+    # the rule: every step agrees with Eq. 5's plain average (double, from scratch) outside a band of 1e-5 * tau
+    # around the radius; where no decision falls inside the band the clustering is the plain oracle's exactly
+    near = oracle.replay_clusters(d_host, tau, ptr.cpu().numpy(), members.cpu().numpy(), medoid.cpu().numpy(), near_rtol=1e-5)
+    rho_p, ptr_p, members_p, medoid_p, near_p = oracle.build_clusters_plain(d_host, tau, members_cap=cap, near_rtol=1e-5)
+    assert np.array_equal(density.cpu().numpy(), rho_p)
+    if near == 0 and near_p == 0:
+        assert np.array_equal(ptr.cpu().numpy(), ptr_p) and np.array_equal(members.cpu().numpy(), members_p)
+        assert np.array_equal(medoid.cpu().numpy(), medoid_p)
+    # and, beyond the rule, the fp32 reading of the oracle (running sum in joining order) bit for bit
+    rho, ptr_ref, members_ref, medoid_ref = oracle.build_clusters(d_host, tau, members_cap=cap)
     assert np.array_equal(density.cpu().numpy(), rho)
     assert np.array_equal(medoid.cpu().numpy(), medoid_ref)
     assert np.array_equal(ptr.cpu().numpy(), ptr_ref)

@@ -772,6 +772,58 @@ def test_algorithm1_replay_in_exact_arithmetic():
         assert any(members.tolist().count(e) > 1 for e in range(n))         # and some sit in several clusters
 
 
+def test_algorithm1_fp32_reading_agrees_with_the_plain_average_outside_the_band():
+    """General (non-grid) distances.  The oracle the GPU is compared with bit for bit decides on an fp32 running
+    sum; Eq. 5 is a plain average.  The two must take the same decision whenever |average - tau| > 1e-5 * tau:
+    the fp32 clustering is replayed against averages recomputed in double, and where no decision falls inside
+    that band the two clusterings are identical."""
+    rng = np.random.default_rng(47)
+    near_total, exact_cases = 0, 0
+    for n, topics, tau in [(40, 3, 0.45), (150, 6, 0.4), (400, 10, 0.38), (257, 5, 0.5), (300, 4, 0.62)]:
+        topic = rng.integers(0, topics, size=n)
+        base = np.where(topic[:, None] == topic[None, :], 0.22, 0.8)
+        d = (base + rng.uniform(-0.2, 0.2, size=(n, n))).astype(np.float32)
+        d = np.minimum(d, d.T)
+        np.fill_diagonal(d, 0.0)
+        rho, ptr, members, medoid = oracle.build_clusters(d, tau)
+        near = oracle.replay_clusters(d, tau, ptr, members, medoid, near_rtol=1e-5)
+        rho_p, ptr_p, members_p, medoid_p, near_p = oracle.build_clusters_plain(d, tau, near_rtol=1e-5)
+        assert np.array_equal(rho, rho_p)
+        assert oracle.replay_clusters(d, tau, ptr_p, members_p, medoid_p, near_rtol=1e-5) == near_p
+        if near == 0 and near_p == 0:
+            assert np.array_equal(ptr, ptr_p) and np.array_equal(members, members_p) and np.array_equal(medoid, medoid_p)
+            exact_cases += 1
+        near_total += near
+    assert exact_cases >= 3, "random distances should rarely come within 1e-5 of the radius"
+    print(f"decisions within the band: {near_total}")
+
+
+def test_algorithm1_replay_rejects_wrong_clusterings():
+    """The band replay is itself a checker: a dropped member, a wrong medoid, a swapped order must all fail it."""
+    d = sym(5, 0.9, {(0, 1): 0.1, (0, 2): 0.2, (1, 2): 0.3, (3, 4): 0.1, (2, 3): 0.4, (2, 4): 0.5})
+    rho, ptr, members, medoid = oracle.build_clusters(d, 0.5)
+    assert oracle.replay_clusters(d, 0.5, ptr, members, medoid) == 0
+    bad = [
+        (np.array([0, 2, 5]), np.array([2, 0, 3, 4, 2]), medoid),            # entry 1 dropped from the first cluster
+        (ptr, np.array([2, 1, 0, 3, 4, 2]), medoid),                         # joining order swapped
+        (ptr, np.array([0, 2, 1, 3, 4, 2]), np.array([0, 3])),               # wrong medoid
+        (np.array([0, 3]), np.array([2, 0, 1]), np.array([2])),              # entries 3 and 4 left uncovered
+    ]
+    for p_, m_, med_ in bad:
+        with pytest.raises(AssertionError):
+            oracle.replay_clusters(d, 0.5, p_, m_, med_)
+    # a decision exactly on the radius may go either way inside the band, and only there
+    d2 = sym(3, 0.9, {(0, 1): 0.2, (0, 2): 0.4, (1, 2): 0.6000000238418579})
+    r = oracle.build_clusters_plain(d2, 0.5, near_rtol=1e-5)
+    assert r[4] >= 1
+    # entry 2's average distance to {0, 1} is 0.5 + 1.2e-8: it joins (one cluster) or not (then it founds [2, 0])
+    both = [(np.array([0, 3]), np.array([0, 1, 2]), np.array([0])), (np.array([0, 2, 4]), np.array([0, 1, 2, 0]), np.array([0, 2]))]
+    for p_, m_, med_ in both:
+        assert oracle.replay_clusters(d2, 0.5, p_, m_, med_, near_rtol=1e-5) >= 1
+    with pytest.raises(AssertionError):
+        oracle.replay_clusters(d2, 0.5, both[0][0], both[0][1], both[0][2], near_rtol=0.0)   # strictly, it does not join
+
+
 # ------------------------------------------------------------------------------- Eq. 7 placement of entries
 
 def test_entry_placement_hand_case_and_round_robin():
