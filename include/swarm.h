@@ -171,6 +171,30 @@ int32_t swarm_set_submit_order(swarm_ctx* ctx, int32_t* submit_order, int32_t* s
  * from the shape).  Results do not depend on it beyond floating-point rounding. */
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits);
 
+/* Overlapped tail of swarm_step (off by default).  Cluster resolution ends in a serial pass (the greedy queue
+ * assignment of Sec. 5.1) whose result feeds the I/O side, not the next layer's computation.  With a tail
+ * stream attached (another cudaStream_t of the same device; NULL detaches), swarm_step enqueues the
+ * resolution there, ordered behind the step's selection, and `stream` itself carries only scoring, selection
+ * and attention: the next swarm_step on `stream` starts as soon as this step's attention has finished, while
+ * the resolution of this step may still run.  uniq / queue_of / n_uniq / queue_load (and the cache state and
+ * submission order, when attached) are then complete once the TAIL stream has run the resolution:
+ *   swarm_tail_join(ctx, s)   makes stream s wait for the last resolution enqueued by this ctx (no host
+ *                             synchronisation).  Required before s reads those outputs, and before a stream
+ *                             capture that recorded steps of this ctx is ended (a capture must join the
+ *                             streams it forked).
+ * sel, n_sel, out, lse, scores are complete in `stream` order as always.  The resolutions of consecutive steps
+ * never overlap each other (they follow one another on the tail stream), and the step keeps two sets of dedup
+ * flags so that the next step's selection may mark clusters while this step's resolution still reads its own.
+ * swarm_step_begin / swarm_step_end / swarm_step_host are not affected.  Attach or detach while no step of the
+ * ctx is in flight. */
+int32_t swarm_set_tail_stream(swarm_ctx* ctx, void* tail_stream);
+int32_t swarm_tail_join(swarm_ctx* ctx, void* stream);
+
+/* SMs the scoring kernel leaves free for the selection kernel, whose CTAs are resident beside it and start on
+ * a head as soon as its scores are complete (-1 restores the default chosen from the shape).  Tuning only:
+ * results do not depend on it. */
+int32_t swarm_set_select_sms(swarm_ctx* ctx, int32_t n_sms);
+
 /* Which kernel scores the pages (stage 1).  The result is the same sum either way, within fp32 rounding.
  *   SWARM_SCORER_AUTO    the streaming tensor-core kernel whenever the shape allows it (batch <= 1024 and fewer
  *                        than 2^31 pool pages), else the fp32-pipe kernel
@@ -274,7 +298,10 @@ int32_t swarm_sparse_attn_static_status(void* stream, uint32_t* bits);
 /* The fused step: stages 1-4 enqueued back to back with no host round trip.  Attention reads the
  * selected pages straight from the pool; the gathered copies are written only when k_out / v_out
  * are given.  Three launches on `stream`: scoring, selection, and one kernel in which cluster resolution
- * runs as one extra CTA beside the attention CTAs.  Integer outputs equal those of the
+ * runs as one extra CTA beside the attention CTAs (with swarm_set_tail_stream the resolution is a kernel of its own on the
+ * tail stream).  The kernels are chained by programmatic dependent launch and hand their data over head by
+ * head: the selection of a KV-head pair starts when that pair's scores are stored, the attention of a KV head
+ * when its heads are selected.  Integer outputs equal those of the
  * four separate calls exactly; out / lse agree within rounding.  The call can be captured into a
  * CUDA graph by the caller (stream capture). */
 int32_t swarm_step(swarm_ctx* ctx, const swarm_inputs* inputs, const swarm_outputs* outputs, void* stream);

@@ -26,7 +26,7 @@ _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
-    "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_tail_stream", "swarm_tail_join", "swarm_set_select_sms", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_sparse_attn_static_status", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
@@ -166,6 +166,20 @@ def swarm_set_workspace(ctx, workspace: torch.Tensor, stream=None) -> None:
 
 def swarm_set_attn_splits(ctx, n_splits: int) -> None:
     _check(load_library().swarm_set_attn_splits(ctx, ctypes.c_int32(n_splits)), "swarm_set_attn_splits", ctx)
+
+
+def swarm_set_tail_stream(ctx, tail_stream) -> None:
+    """Attach a torch.cuda.Stream on which swarm_step enqueues cluster resolution (None detaches)."""
+    ptr = ctypes.c_void_p(tail_stream.cuda_stream) if tail_stream is not None else None
+    _check(load_library().swarm_set_tail_stream(ctx, ptr), "swarm_set_tail_stream", ctx)
+
+
+def swarm_tail_join(ctx, stream=None) -> None:
+    _check(load_library().swarm_tail_join(ctx, _stream(stream)), "swarm_tail_join", ctx)
+
+
+def swarm_set_select_sms(ctx, n_sms: int) -> None:
+    _check(load_library().swarm_set_select_sms(ctx, ctypes.c_int32(n_sms)), "swarm_set_select_sms", ctx)
 
 
 def swarm_set_scorer(ctx, kind: int) -> None:

@@ -1,6 +1,7 @@
 // C-ABI layer of libswarm: argument validation, workspace carving and kernel sequencing.
 // No device memory is allocated here; every scratch byte comes from the caller's workspace.  (swarm_create
 // allocates one 64-byte word of pinned host memory, the completion word of swarm_step_host.)
+#include <algorithm>
 #include <atomic>
 #include <chrono>
 #include <cstdlib>
@@ -18,6 +19,11 @@ struct swarm_ctx {
   uint8_t* ws;
   int64_t ws_bytes;
   int user_splits;            // 0 = chosen from the shape
+  int select_sms;             // SMs the scorer leaves to the selection CTAs; < 0 = chosen from the shape
+  cudaStream_t tail_stream;   // swarm_set_tail_stream: where swarm_step enqueues cluster resolution (null: inside the step)
+  cudaEvent_t ev_selected;    // recorded on the step's stream behind the selection; the tail stream waits for it
+  cudaEvent_t ev_resolved;    // recorded on the tail stream behind the resolution; swarm_tail_join waits for it
+  bool tail_pending;          // a resolution has been enqueued on the tail stream since the last join
   cudaError_t last_err;
   cudaGraphExec_t host_graph;  // swarm_step_host: the recorded step, valid for the arguments in host_key
   unsigned char host_key[256];
@@ -60,12 +66,17 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.scores = off;   off = align256(off + bh * s.max_pages_per_req * 4);
   l.n_tok = off;    off = align256(off + bh * 4);
   l.q_stage = off;  off = align256(off + bh * kHeadDim * 2);
-  l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);
+  l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);   // two arrays: alternate steps of the
+  l.flags_alt = off - l.flags;                                                  // overlapped tail mark alternate ones
+  off = align256(off + (int64_t)s.max_clusters_total + 16);
   l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
   l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
   l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 16);
   l.selmap = off;   off = align256(off + bh * selmap_pitch_bytes(s.max_pages_per_req));
   l.tickets = off;  off = align256(off + bh * 4);
+  l.ctl = off;      off = align256(off + 64 * 4);
+  l.ready = off;    off = align256(off + (int64_t)s.batch * head_pairs(s.n_kv_heads) * 4);
+  l.sel_ready = off; off = align256(off + (int64_t)s.batch * s.n_kv_heads * 4);
   l.total = off;
   return l;
 }
@@ -94,6 +105,31 @@ int pick_splits(const swarm_ctx* ctx, bool paged, bool fused = false) {
   }
   n = std::min<int64_t>(n, kMaxSplits);
   return (int)std::max<int64_t>(n, 1);
+}
+
+// The hand-off counters of a step (see StepTickets).  The scorer's tickets exist only when the streaming scorer
+// runs; `with_attention`: the selection also announces its heads to an attention kernel launched by the same call.
+StepTickets step_tickets(const swarm_ctx* ctx, const Geometry& g, bool with_attention) {
+  StepTickets t;
+  t.ctl = reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ctl);
+  t.ready = score_raises_tickets(g) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ready) : nullptr;
+  t.sel_ready = (with_attention && t.ready != nullptr) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.sel_ready) : nullptr;
+  return t;
+}
+
+// SMs the scorer leaves free so that the selection CTAs are resident while it runs (they wait for its
+// tickets); inside a step with an overlapped tail one more for the resolution CTA of the previous step.
+int reserved_sms(const swarm_ctx* ctx, const Geometry& g, bool tail) {
+  if (!score_raises_tickets(g)) return 0;
+  int n = ctx->select_sms;
+  if (n < 0) {
+    const int threads = topk_threads(g.Pmax);
+    const int per_sm = std::max(1, std::min(2048 / threads, 65536 / (64 * threads)));
+    const long long lists = (long long)g.B * g.Hq;
+    n = (int)std::min<long long>((lists + per_sm - 1) / per_sm, sm_count() / 4);
+  }
+  n += tail ? 1 : 0;
+  return std::min(n, sm_count() - 8);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -184,6 +220,11 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->ws = nullptr;
   ctx->ws_bytes = 0;
   ctx->user_splits = 0;
+  ctx->select_sms = -1;
+  ctx->tail_stream = nullptr;
+  ctx->ev_selected = nullptr;
+  ctx->ev_resolved = nullptr;
+  ctx->tail_pending = false;
   ctx->last_err = cudaSuccess;
   ctx->host_graph = nullptr;
   ctx->host_graph_ok = true;
@@ -224,6 +265,8 @@ int32_t swarm_destroy(swarm_ctx* ctx) {
   if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
   if (ctx->host_graph != nullptr) cudaGraphExecDestroy(ctx->host_graph);
   if (ctx->done_h != nullptr) cudaFreeHost(ctx->done_h);
+  if (ctx->ev_selected != nullptr) cudaEventDestroy(ctx->ev_selected);
+  if (ctx->ev_resolved != nullptr) cudaEventDestroy(ctx->ev_resolved);
   delete ctx;
   return SWARM_OK;
 }
@@ -238,13 +281,40 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 256, st));
   SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.flags, 0, ctx->lay.part_acc - ctx->lay.flags, st));
-  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.tickets, 0, ctx->lay.total - ctx->lay.tickets, st));
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.tickets, 0, ctx->lay.total - ctx->lay.tickets, st));   // and the hand-off counters
   return SWARM_OK;
 }
 
 int32_t swarm_set_attn_splits(swarm_ctx* ctx, int32_t n_splits) {
   if (ctx == nullptr || n_splits < 0 || n_splits > kMaxSplits) return SWARM_ERR_INVALID_ARG;
   ctx->user_splits = n_splits;
+  return SWARM_OK;
+}
+
+int32_t swarm_set_tail_stream(swarm_ctx* ctx, void* tail_stream) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (tail_stream != nullptr && ctx->ev_selected == nullptr) {
+    SWARM_TRY(cudaEventCreateWithFlags(&ctx->ev_selected, cudaEventDisableTiming));
+    SWARM_TRY(cudaEventCreateWithFlags(&ctx->ev_resolved, cudaEventDisableTiming));
+  }
+  ctx->tail_stream = static_cast<cudaStream_t>(tail_stream);
+  ctx->tail_pending = false;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
+  return SWARM_OK;
+}
+
+int32_t swarm_tail_join(swarm_ctx* ctx, void* stream) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  if (ctx->tail_stream == nullptr || !ctx->tail_pending) return SWARM_OK;
+  SWARM_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), ctx->ev_resolved, 0));
+  ctx->tail_pending = false;
+  return SWARM_OK;
+}
+
+int32_t swarm_set_select_sms(swarm_ctx* ctx, int32_t n_sms) {
+  if (ctx == nullptr || n_sms < -1 || n_sms > 1024) return SWARM_ERR_INVALID_ARG;
+  ctx->select_sms = n_sms;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
   return SWARM_OK;
 }
 
@@ -345,9 +415,13 @@ int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int3
   if (!select_inputs_ok(in) || bad(sel) || bad(n_sel) || (scores && !aligned16(scores))) return SWARM_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* sc = scores ? scores : ws_ptr<float>(ctx, ctx->lay.scores);
+  TopkLinks links;
+  links.tk = step_tickets(ctx, ctx->geo, false);
+  links.req_base = in->page_base;
   SWARM_TRY(launch_page_score(ctx->geo, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(in->ksum),
-                              in->page_base, in->ctx_len, sc, ws_ptr<uint32_t>(ctx, ctx->lay.status), st));
-  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, true,
+                              in->page_base, in->ctx_len, sc, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, links.tk.ready,
+                              reserved_sms(ctx, ctx->geo, false)));
+  SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, sel, n_sel, ws_ptr<uint32_t>(ctx, ctx->lay.status), st, true, links,
                         ws_ptr<uint8_t>(ctx, ctx->lay.selmap)));
   return SWARM_OK;
 }
@@ -476,28 +550,55 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   const uint16_t* pool = static_cast<const uint16_t*>(in->kv_pool);
   float* sc = o->scores ? o->scores : ws_ptr<float>(ctx, ctx->lay.scores);
 
+  // Overlapped tail only for a whole step (the halves exchange the flag array between them).
+  const bool whole = parts == (kStepBegin | kStepEnd);
+  const bool tail = ctx->tail_stream != nullptr && whole && host == nullptr;   // (a host step waits for everything anyway)
+  // the attention CTAs wait per KV head for the selection -- unless a gather sits between the two kernels,
+  // which waits for all of the selection anyway
+  const bool attn_tickets = whole && o->k_out == nullptr;
+  TopkLinks links;
+  links.tk = step_tickets(ctx, ctx->geo, attn_tickets);
+  links.req_base = in->page_base;
+  links.flags_alt = tail ? ctx->lay.flags_alt : 0;
   if (parts & kStepBegin) {
     SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
-                                status, st));
+                                status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail)));
     // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
-    SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true,
+    SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true, links,
                           ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
                           ws_ptr<uint8_t>(ctx, ctx->lay.flags), in->cluster_replica_mask, in->cluster_size));
   }
   if (!(parts & kStepEnd)) return SWARM_OK;
 
-  // Cluster resolution and attention both need only the selection: one launch runs them side by side, the
-  // attention CTAs plus one CTA for the resolution (whose serial pass is the longest item of the step).
   if (o->k_out != nullptr)
     SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
                             static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
   AttnArgs a = paged_args(ctx, in, o->out, o->lse);
-  a.n_splits = pick_splits(ctx, true, /*fused=*/true);
   ResolveArgs rs = step_resolve_args(ctx, in, nullptr, o->n_sel, o->uniq, o->queue_of, o->n_uniq, o->queue_load);
   if (host != nullptr) {
     a.host = *host;
     rs.host = *host;
   }
+  if (attn_tickets) a.tk = links.tk;
+  if (tail) {
+    // Cluster resolution as a kernel of its own on the tail stream, forked behind the selection: nothing on the
+    // step's stream waits for it, so its serial pass runs beside this step's attention and the next step's
+    // scoring and selection.  (On the step's own stream it would not: a kernel launched behind another, even
+    // one that never waits for it, was measured to complete only after it.)
+    rs.tail_ctl = links.tk.ctl;
+    rs.flags_alt = ctx->lay.flags_alt;
+    SWARM_TRY(cudaEventRecord(ctx->ev_selected, st));
+    SWARM_TRY(cudaStreamWaitEvent(ctx->tail_stream, ctx->ev_selected, 0));
+    SWARM_TRY(launch_resolve(rs, ctx->tail_stream, /*overlap=*/false));
+    SWARM_TRY(cudaEventRecord(ctx->ev_resolved, ctx->tail_stream));
+    ctx->tail_pending = true;
+    a.n_splits = pick_splits(ctx, true, /*fused=*/false);
+    SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, nullptr));
+    return SWARM_OK;
+  }
+  // Otherwise one launch runs them side by side: the attention CTAs plus one CTA for the resolution (whose
+  // serial pass is the longest item of the step).
+  a.n_splits = pick_splits(ctx, true, /*fused=*/true);
   SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, &rs));
   return SWARM_OK;
 }
@@ -615,9 +716,12 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
   gc.k = idx->top_k_clusters;
   gc.W = 0;
   gc.n_pool_pages = ctx->geo.Cmax;
+  TopkLinks links;
+  links.tk = step_tickets(ctx, gc, false);
+  links.req_base = in->cluster_base;
   SWARM_TRY(launch_page_score(gc, static_cast<const uint16_t*>(in->q), static_cast<const uint16_t*>(idx->medoid_ksum),
-                              in->cluster_base, len_c, sc, status, st));
-  SWARM_TRY(launch_topk(gc, sc, len_c, o->sel, o->n_sel, status, st, true));
+                              in->cluster_base, len_c, sc, status, st, links.tk.ready, reserved_sms(ctx, gc, false)));
+  SWARM_TRY(launch_topk(gc, sc, len_c, o->sel, o->n_sel, status, st, true, links));
   // selected clusters -> page bitmaps per head (for attention) and cluster flags (for the resolve kernel)
   SWARM_TRY(launch_expand_clusters(ctx->geo, idx->top_k_clusters, o->sel, o->n_sel, in->cluster_base,
                                    idx->cluster_page_ptr, idx->cluster_pages, in->ctx_len,

@@ -177,10 +177,31 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   __syncwarp();
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 2);
-  // Stand-alone, the next kernel in the stream may set itself up meanwhile.  Inside the fused step the attention
+  // Stand-alone, the next kernel in the stream may set itself up meanwhile.  Inside a step the attention
   // CTAs release their dependents by exiting: with this trigger the step was measured 1.5 us slower.
-  if (kFused == 0) pdl_launch_dependents();
-  pdl_wait();                                           // the selection comes from the previous kernel
+  const bool ticketed = kPaged && a.tk.sel_ready != nullptr;
+  if (kFused == 0 && !ticketed) pdl_launch_dependents();
+  if (ticketed) {
+    // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The last CTA
+    // of the grid to get past its wait sets the tickets back to zero for the next step -- after the selection
+    // kernel's own last CTA has finished its bookkeeping, so that the next step cannot start before it.
+    if (threadIdx.x == 0) {
+      bool ok = wait_at_least(a.tk.sel_ready + (long long)b * geo.Hkv + kvh, (unsigned)geo.g);
+      const unsigned n_ctas = gridDim.x - (kFused != 0 ? 1u : 0u);
+      const bool last = atomicAdd(a.tk.ctl + kCtlAttnPast, 1u) == n_ctas - 1u;
+      if (last) ok = wait_zero(a.tk.ctl + kCtlTopkDone) && ok;
+      if (!ok) atomicOr(status, SWARM_DEV_TIMEOUT);
+      s_last = last;
+    }
+    __syncthreads();
+    if (s_last) {
+      for (int i = threadIdx.x; i < geo.B * geo.Hkv; i += kAttnWarps * 32) a.tk.sel_ready[i] = 0u;
+      __syncthreads();
+      if (threadIdx.x == 0) st_release(a.tk.ctl + kCtlAttnPast, 0u);
+    }
+  } else {
+    pdl_wait();                                         // the selection comes from the previous kernel
+  }
   SWARM_STAMP(status, 1);
 
   int P = 0, tail = S, total_tok = 0, n_items;          // items: pages of the union (paged) or page slots (gathered)

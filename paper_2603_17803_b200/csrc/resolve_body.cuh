@@ -53,7 +53,7 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   const int64_t* __restrict__ cluster_base = r.cluster_base;
   const uint32_t* __restrict__ replica_mask = r.replica_mask;
   const uint16_t* __restrict__ cluster_size = r.cluster_size;
-  uint8_t* __restrict__ flags = r.flags;
+  uint8_t* __restrict__ flags = r.flags;                 // (the overlapped tail picks one of two arrays below)
   unsigned* __restrict__ ticket = r.ticket;
   uint4* __restrict__ items = r.items;
   int32_t* __restrict__ uniq = r.uniq;
@@ -79,6 +79,17 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   pdl_wait();                                            // the flags / the selection come from the previous kernel
   const int C = (int)min((long long)geo.Cmax, c_all);
   unsigned err = (c_all > geo.Cmax) ? SWARM_DEV_BAD_CLUSTER : 0u;
+  // Overlapped tail: nothing after this kernel in the step waits for it, so it runs beside the next step's
+  // scoring and selection.  That selection marks the other one of two flag arrays (the selection kernel counts
+  // the steps it has marked; step n uses array (n - 1) & 1), and this kernel first lets the resolution of the
+  // step before finish, which shares its outputs and scratch.
+  unsigned step_no = 0u;
+  if (r.tail_ctl != nullptr) {
+    step_no = *reinterpret_cast<volatile unsigned*>(r.tail_ctl + kCtlMarked);
+    flags += ((step_no - 1u) & 1u) * r.flags_alt;
+    if (tid == 0 && !wait_at_least(r.tail_ctl + kCtlResolved, step_no - 1u)) err |= SWARM_DEV_TIMEOUT;
+    __syncthreads();
+  }
 
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 3);
@@ -540,6 +551,10 @@ __device__ __forceinline__ void resolve_body(const ResolveArgs& r, int cta, int 
   if (r.host.done_h != nullptr) {                          // host step: the resolution's results are in host memory
     __syncthreads();
     if (tid == 0) host_arrive(r.host);
+  }
+  if (r.tail_ctl != nullptr) {                             // overlapped tail: this step's resolution has finished
+    __syncthreads();
+    if (tid == 0) st_release(r.tail_ctl + kCtlResolved, step_no);
   }
 }
 

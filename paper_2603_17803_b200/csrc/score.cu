@@ -156,18 +156,33 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 // the memory bandwidth; as m16n8k16 MMAs (16 pages x up to 8 heads per tile, fp32 accumulation) it costs
 // ~3, and the kernel runs at the speed of the bulk copies.
 //
-// One persistent CTA per SM.  A block is 16 consecutive pages of one request for a group of up to 8 KV
-// heads: per KV head four TMA boxes of 16 pages x 64 coordinates (128-byte swizzle) = 8 KiB, so a block of
-// 8 KV heads is 64 KiB.  A producer warp keeps a 3-slot ring full; consumer warp j scores KV head j of the
-// block that has landed with ldmatrix + mma and stores the tile of scores.  Waits are bounded.
-constexpr int kMmaConsumers = 8;                           // = KV heads per block
-constexpr int kMmaThreads = (kMmaConsumers + 1) * 32;
+// Persistent CTAs, one per SM, on all SMs but the ones left to the selection kernel (see launch_mma).  A block
+// is 64 consecutive pages of one request for one PAIR of KV heads: 16 TMA boxes of 16 pages x 2 heads x 64
+// coordinates (128-byte swizzle) = 64 KiB.  Blocks are numbered request by request, inside a request pair by
+// pair, and dealt to the CTAs round-robin, so that at any moment all CTAs work on the same (request, pair) and
+// the pairs of a request are finished one after the other: the selection of a pair's heads starts while the
+// later pairs are still being scored (StepTickets::ready).  Reading one pair at a time touches 1 KiB of every
+// 4 KiB summary row; measured, that streams at the same rate as whole rows.  A producer warp keeps a 3-slot
+// ring full; consumer warp w scores (tile w / 2, head w % 2) of the block that has landed with ldmatrix + mma,
+// stores the tile of scores and counts it on the pair's ticket.  Waits are bounded.
+constexpr int kMmaConsumers = 8;
+constexpr int kMmaThreads = (kMmaConsumers + 2) * 32;      // consumers, the producer warp, the ticket warp
 constexpr int kMmaStages = 3;
-constexpr int kMmaPages = 16;                              // pages per block = M of the MMA tile
-constexpr int kMmaHeadBytes = 4 * kMmaPages * 128;         // 4 boxes of 16 pages x 128 B
+constexpr int kMmaPages = 16;                              // pages per tile = M of the MMA tile
+constexpr int kMmaHeadBytes = 4 * kMmaPages * 128;         // one KV head of one tile: 4 boxes' share, 8 KiB
 constexpr int kBoxHeads = 2;                               // KV heads per TMA box (rows of a box: page-major, head-minor)
-constexpr int kMmaStageBytes = kMmaConsumers * kMmaHeadBytes;
-constexpr int kMmaSmemBytes = 1024 + kMmaStages * kMmaStageBytes;
+constexpr int kBlkTiles = kMmaConsumers / kBoxHeads;       // 16-page tiles per block
+constexpr int kBlkPages = kBlkTiles * kMmaPages;           // 64
+constexpr int kTileBytes = kBoxHeads * kMmaHeadBytes;      // one tile of a pair: 4 boxes of 4 KiB
+constexpr int kMmaStageBytes = kBlkTiles * kTileBytes;
+// Sign-split weights of the current request's query heads, bf16 [head][minima part 128 | maxima part 128], kept in
+// shared memory: in pair-by-pair order nearly every block of a CTA belongs to another KV pair, and fetching a
+// pair's weights from global memory per block cost more than the block's arithmetic.  Rows are padded by 16
+// bytes so that the 8 heads a warp reads side by side fall into different banks.
+constexpr int kWeightRowBytes = 512 + 16;
+constexpr int kWeightRows = 56;                            // query heads that fit; heads beyond them are fetched from global memory
+constexpr int kWeightBytes = kWeightRows * kWeightRowBytes;
+constexpr int kMmaSmemBytes = 1024 + kMmaStages * kMmaStageBytes + kWeightBytes;
 constexpr int kStreamMaxBatch = 1024;                      // requests whose block counts fit the shared prefix table
 constexpr unsigned kStreamWaitLimit = 1u << 22;
 
@@ -184,20 +199,37 @@ __device__ __forceinline__ bool sm_try_wait(uint64_t* bar, unsigned parity) {
   return ok != 0;
 }
 
+// What block `blk` of the launch covers; s_cum[b] = blocks before request b.
+struct ScoreBlock {
+  int b, hp, page0, n_tiles, P;   // request, KV-head pair, first page (request-local), tiles that exist, pages of the request
+};
+__device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const int* s_cum, const int32_t* __restrict__ ctx_len, int S) {
+  while (s_cum[cur_b + 1] <= blk) ++cur_b;
+  ScoreBlock k;
+  k.b = cur_b;
+  k.P = pages_of(ctx_len[cur_b], S);
+  const int per_pair = (k.P + kBlkPages - 1) / kBlkPages;
+  const int c = blk - s_cum[cur_b];
+  k.hp = c / per_pair;
+  k.page0 = (c - k.hp * per_pair) * kBlkPages;
+  k.n_tiles = min(kBlkTiles, (k.P - k.page0 + kMmaPages - 1) / kMmaPages);
+  return k;
+}
+
 __global__ void __launch_bounds__(kMmaThreads, 1)
 page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
-                      float* __restrict__ scores, uint32_t* __restrict__ status) {
+                      float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready) {
   extern __shared__ unsigned char mma_smem_raw[];
   __shared__ __align__(8) uint64_t full[kMmaStages], empty[kMmaStages];
   __shared__ int s_cum[kStreamMaxBatch + 1];               // blocks before request b
   __shared__ int s_abort;
-  pdl_launch_dependents();
+  __shared__ unsigned s_scored[kMmaStages];                // consumer warps done with the blocks of a ring slot, ever growing
   SWARM_KERNEL_BEGIN(status, 0);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned char* ring = mma_smem_raw + ((1024u - (sm_addr(mma_smem_raw) & 1023u)) & 1023u);
 
-  const int kv_groups = (geo.Hkv + kMmaConsumers - 1) / kMmaConsumers;   // blocks per page tile
+  const int hpairs = head_pairs(geo.Hkv);
   if (tid == 0) {
     for (int sidx = 0; sidx < kMmaStages; ++sidx) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&full[sidx])), "r"(1));
@@ -206,12 +238,17 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_abort = 0;
     s_cum[0] = 0;
+    for (int sidx = 0; sidx < kMmaStages; ++sidx) s_scored[sidx] = 0u;
   }
   // Launched with programmatic serialization behind whatever precedes it in the stream -- inside a chain of
-  // steps the previous step's attention + resolution kernel -- so that this kernel's launch and set-up
-  // overlap that kernel's tail.  Nothing a predecessor may have written (q, lengths, tables, summaries) is
-  // read before this point.
+  // steps the previous step's attention kernel -- so that this kernel's launch and set-up overlap that kernel's
+  // tail.  Nothing a predecessor may have written (q, lengths, tables, summaries) is read before this point.
+  SWARM_STAMP(status, 0);
   pdl_wait();
+  SWARM_STAMP(status, 1);
+  // Only now may the selection kernel be scheduled: its CTAs poll the tickets this kernel raises, and tickets
+  // of the previous step are guaranteed to be cleared only once everything before this kernel has finished.
+  pdl_launch_dependents();
   if (warp == 1) {                                         // blocks per request, prefix by one warp
     int running = 0;
     for (int b0 = 0; b0 < geo.B; b0 += 32) {
@@ -221,7 +258,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
         const int len = ctx_len[b];
         const int P = pages_of(len, geo.S);
         if (len < 1 || P > page_base[b + 1] - page_base[b] || P > geo.Pmax) atomicOr(status, SWARM_DEV_BAD_LENGTH);
-        else nb = ((P + kMmaPages - 1) / kMmaPages) * kv_groups;
+        else nb = ((P + kBlkPages - 1) / kBlkPages) * hpairs;
       }
       int incl = nb;
 #pragma unroll
@@ -234,15 +271,10 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     }
   }
   __syncthreads();
-  // The CTAs share the work in units of one KV head of one block (8 KiB), so that their byte counts differ by
-  // one unit at most; a CTA's first and last block may therefore cover only some of the block's KV heads.
-  const long long total_units = (long long)s_cum[geo.B] * kMmaConsumers;
-  const long long u_lo = total_units * blockIdx.x / gridDim.x, u_hi = total_units * (blockIdx.x + 1) / gridDim.x;
-  const int blk_lo = (int)(u_lo / kMmaConsumers);
-  const int blk_hi = u_hi > u_lo ? (int)((u_hi - 1) / kMmaConsumers) + 1 : blk_lo;
-  const int n_blk = blk_hi - blk_lo;
-  const int first_head = (int)(u_lo % kMmaConsumers);                    // of block blk_lo
-  const int last_heads = u_hi > u_lo ? (int)((u_hi - 1) % kMmaConsumers) + 1 : 0;   // heads of block blk_hi - 1
+  SWARM_STAMP(status, 2);
+  const int total = s_cum[geo.B];
+  const int blk_first = (int)blockIdx.x, blk_step = (int)gridDim.x;
+  const int n_blk = blk_first < total ? (total - blk_first + blk_step - 1) / blk_step : 0;
 
   if (warp == kMmaConsumers) {
     // ---- producer ----
@@ -260,26 +292,20 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           while (!sm_try_wait(&empty[stage], parity) && ++polls < kStreamWaitLimit && !s_abort) {}
           if (polls >= kStreamWaitLimit || s_abort) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; break; }
         }
-        const int blk = blk_lo + k;
-        while (s_cum[fb + 1] <= blk) ++fb;
-        const int c = blk - s_cum[fb];
-        const int tile = c / kv_groups, kvg = c % kv_groups;
-        const int j_lo = k == 0 ? first_head : 0;
-        const int j_hi = min(k == n_blk - 1 ? last_heads : kMmaConsumers, geo.Hkv - kvg * kMmaConsumers);
-        const int page0 = (int)(page_base[fb] + (long long)tile * kMmaPages);
-        // one box carries kBoxHeads KV heads: the copy engine's rate per box, not the memory, bounds small boxes
-        const int p_lo = j_lo / kBoxHeads, p_hi = j_hi > j_lo ? (j_hi + kBoxHeads - 1) / kBoxHeads : p_lo;
+        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+        const int page0 = (int)(page_base[blk.b] + blk.page0);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])),
-                     "r"((unsigned)((p_hi - p_lo) * kBoxHeads * kMmaHeadBytes))
+                     "r"((unsigned)(blk.n_tiles * kTileBytes))
                      : "memory");
-        for (int pj = p_lo; pj < p_hi; ++pj) {
+        // a box carries both heads of the pair (the copy engine's rate per box, not the memory, bounds smaller
+        // boxes); the second head of an odd last pair lies outside the tensor and arrives as zeros
+        for (int pt = 0; pt < blk.n_tiles; ++pt) {
 #pragma unroll
           for (int bx = 0; bx < 4; ++bx) {
-            const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + pj * (kBoxHeads * kMmaHeadBytes) +
-                                         bx * (kBoxHeads * kMmaPages * 128));
+            const uint32_t dst = sm_addr(ring + (size_t)stage * kMmaStageBytes + pt * kTileBytes + bx * (kTileBytes / 4));
             asm volatile(
                 "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
-                "l"(&map), "r"(bx * 64), "r"(kvg * kMmaConsumers + pj * kBoxHeads), "r"(page0), "r"(sm_addr(&full[stage])), "l"(stream_policy)
+                "l"(&map), "r"(bx * 64), "r"(blk.hp * kBoxHeads), "r"(page0 + pt * kMmaPages), "r"(sm_addr(&full[stage])), "l"(stream_policy)
                 : "memory");
           }
         }
@@ -288,58 +314,122 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     return;
   }
 
-  // ---- consumers: warp j <-> KV head j of the block ----
+  if (warp == kMmaConsumers + 1) {
+    // ---- ticket warp ----
+    // Raising a ticket needs a GPU-wide release behind the consumers' score stores, which waits for those stores
+    // to be acknowledged: about a microsecond per block.  In the consumers' loop that wait held back the ring
+    // (measured: +4 us per launch); here one otherwise idle thread pays it.  The consumers count themselves on
+    // a per-slot counter in shared memory (release at CTA scope); a slot is refilled only after all of them
+    // have arrived on its `empty` barrier, so block k is complete exactly when its slot's counter has reached
+    // 8 * (k / slots + 1).
+    if (lane == 0 && ready != nullptr) {
+      int fb = 0;
+      for (int k = 0; k < n_blk; ++k) {
+        const int stage = k % kMmaStages;
+        const unsigned want = (unsigned)kMmaConsumers * (unsigned)(k / kMmaStages + 1);
+        unsigned polls = 0, seen = 0;
+        do {
+          asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(seen) : "r"(sm_addr(&s_scored[stage])) : "memory");
+          if (seen >= want) break;
+          __nanosleep(64);
+        } while (++polls < kStreamWaitLimit && !s_abort);
+        if (seen < want) break;                             // the consumers gave up (they have set the status bit)
+        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+        const unsigned units = (unsigned)blk.n_tiles * (unsigned)min(kBoxHeads, geo.Hkv - blk.hp * kBoxHeads);
+        red_release_add(ready + (long long)blk.b * hpairs + blk.hp, units);
+      }
+    }
+    return;
+  }
+
+  // ---- consumers: warp w <-> (tile w / 2, head w % 2) of the block ----
   const int quad = lane >> 2, tq = lane & 3;
+  const int pt = warp / kBoxHeads, hl = warp % kBoxHeads;
   const int tiles = (geo.g + 7) / 8;                        // head tiles of 8 per KV head (N of the MMA)
   uint32_t wb[16][2];                                       // B operand: weights of head `quad`, 16 k-steps
   long long w_key = -1;
-  int cur_b = 0;
+  int cur_b = 0, cached_b = -1;
+  unsigned char* wcache = ring + kMmaStages * kMmaStageBytes;
+  const int n_cached = min(geo.Hq, kWeightRows);
+  // weights of head h0 + quad of request b: min(q,0) against the minima (k < 128), max(q,0) against the maxima
+  auto load_weights = [&](int b, int h0, int nh) {
+    w_key = (long long)b * geo.Hq + h0;
+    if (h0 + nh <= n_cached) {                              // from the request's rows in shared memory
+      const unsigned char* row = wcache + (size_t)(h0 + (quad < nh ? quad : 0)) * kWeightRowBytes + tq * 4;
+#pragma unroll
+      for (int ks = 0; ks < 16; ++ks) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t v = *reinterpret_cast<const uint32_t*>(row + (ks * 16 + half * 8) * 2);
+          wb[ks][half] = quad < nh ? v : 0u;
+        }
+      }
+      return;
+    }
+    const uint16_t* qrow = q + (w_key + (quad < nh ? quad : 0)) * kHeadDim;
+#pragma unroll
+    for (int ks = 0; ks < 16; ++ks) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int col = ks * 16 + half * 8 + tq * 2;                // 0..255
+        uint32_t pr = *reinterpret_cast<const uint32_t*>(qrow + (col & 127));
+        // clamp each bf16 by its sign bit: keep negatives for the minima part, positives for the maxima part
+        const bool want_neg = col < 128;
+        uint32_t lo = pr & 0xFFFFu, hi = pr >> 16;
+        if (((lo >> 15) != 0u) != want_neg) lo = 0u;
+        if (((hi >> 15) != 0u) != want_neg) hi = 0u;
+        wb[ks][half] = quad < nh ? (lo | (hi << 16)) : 0u;
+      }
+    }
+  };
+  // All consumer warps walk the same blocks, so they reach a new request together: they rewrite the rows behind
+  // a barrier of their own (the producer warp takes no part).
+  auto cache_request = [&](int b) {
+    asm volatile("bar.sync 1, %0;" ::"n"(kMmaConsumers * 32) : "memory");   // nobody still reads the previous request's rows
+    for (int i = tid; i < n_cached * 64; i += kMmaConsumers * 32) {
+      const int h = i >> 6, c2 = (i & 63) * 2;              // two coordinates per thread
+      const uint32_t pr = *reinterpret_cast<const uint32_t*>(q + ((long long)b * geo.Hq + h) * kHeadDim + c2);
+      const uint32_t lo = pr & 0xFFFFu, hi = pr >> 16;
+      const uint32_t neg = ((lo >> 15) ? lo : 0u) | (((hi >> 15) ? hi : 0u) << 16);
+      const uint32_t pos = ((lo >> 15) ? 0u : lo) | (((hi >> 15) ? 0u : hi) << 16);
+      unsigned char* row = wcache + (size_t)h * kWeightRowBytes;
+      *reinterpret_cast<uint32_t*>(row + c2 * 2) = neg;
+      *reinterpret_cast<uint32_t*>(row + 256 + c2 * 2) = pos;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMmaConsumers * 32) : "memory");
+    cached_b = b;
+    w_key = -1;
+  };
+  bool dead = false;                                        // a wait ran out: keep only the consumers' barriers
   for (int k = 0; k < n_blk; ++k) {
-    const int blk = blk_lo + k, stage = k % kMmaStages;
-    while (s_cum[cur_b + 1] <= blk) ++cur_b;
-    const int b = cur_b;
-    const int c = blk - s_cum[b];
-    const int tile_p = c / kv_groups, kvg = c % kv_groups;
-    const int kvh = kvg * kMmaConsumers + warp;
-    const bool active = kvh < geo.Hkv && warp >= (k == 0 ? first_head : 0) &&
-                        warp < (k == n_blk - 1 ? last_heads : kMmaConsumers);
-    const int P = pages_of(ctx_len[b], geo.S);
-    const int p0 = tile_p * kMmaPages;
-    {
+    const int stage = k % kMmaStages;
+    const ScoreBlock blk = locate_block(blk_first + k * blk_step, cur_b, s_cum, ctx_len, geo.S);
+    const int b = blk.b, P = blk.P;
+    const int kvh = blk.hp * kBoxHeads + hl;
+    const bool active = !dead && kvh < geo.Hkv && pt < blk.n_tiles;
+    const int p0 = blk.page0 + pt * kMmaPages;
+    if (b != cached_b) cache_request(b);
+    // the weights of the block's first head tile are fetched before the block has landed
+    if (active && (long long)b * geo.Hq + kvh * geo.g != w_key) load_weights(b, kvh * geo.g, min(8, geo.g));
+    if (!dead) {
       const unsigned parity = (k / kMmaStages) & 1u;
       unsigned polls = 0;
       while (!sm_try_wait(&full[stage], parity) && ++polls < kStreamWaitLimit) __nanosleep(32);
       if (__any_sync(0xFFFFFFFFu, polls >= kStreamWaitLimit || s_abort != 0)) {
         if (lane == 0) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; }
-        break;
+        dead = true;
+        continue;
       }
+    } else {
+      continue;
     }
+    SWARM_STAMP(status, 3 + 2 * min(k, 4));
     if (active) {
       // rows of a box: (page, head of the box) pairs, page-major; 128-byte swizzle over the row index
-      const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + (warp / kBoxHeads) * (kBoxHeads * kMmaHeadBytes));
-      const int hl = warp % kBoxHeads;
+      const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + pt * kTileBytes);
       for (int ht = 0; ht < tiles; ++ht) {
         const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
-        const long long key = ((long long)b * geo.Hq + h0);
-        if (key != w_key) {
-          // weights of head h0 + quad: min(q,0) against the minima (k < 128), max(q,0) against the maxima
-          w_key = key;
-          const uint16_t* qrow = q + (key + (quad < nh ? quad : 0)) * kHeadDim;
-#pragma unroll
-          for (int ks = 0; ks < 16; ++ks) {
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const int col = ks * 16 + half * 8 + tq * 2;                // 0..255
-              uint32_t pr = *reinterpret_cast<const uint32_t*>(qrow + (col & 127));
-              // clamp each bf16 by its sign bit: keep negatives for the minima part, positives for the maxima part
-              const bool want_neg = col < 128;
-              uint32_t lo = pr & 0xFFFFu, hi = pr >> 16;
-              if (((lo >> 15) != 0u) != want_neg) lo = 0u;
-              if (((hi >> 15) != 0u) != want_neg) hi = 0u;
-              wb[ks][half] = quad < nh ? (lo | (hi << 16)) : 0u;
-            }
-          }
-        }
+        if ((long long)b * geo.Hq + h0 != w_key) load_weights(b, h0, nh);
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < 16; ++ks) {
@@ -348,7 +438,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           uint32_t a[4];
           asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                        : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
-                       : "r"(base + (uint32_t)((cc >> 3) * (kBoxHeads * kMmaPages * 128) + (r * kBoxHeads + hl) * 128 +
+                       : "r"(base + (uint32_t)((cc >> 3) * (kTileBytes / 4) + (r * kBoxHeads + hl) * 128 +
                                                (((cc & 7) ^ ((r * kBoxHeads + hl) & 7)) << 4))));
           asm volatile(
               "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -364,8 +454,14 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       }
     }
     __syncwarp();
-    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sm_addr(&empty[stage])) : "memory");
+    SWARM_STAMP(status, 4 + 2 * min(k, 4));
+    if (lane == 0) {
+      // the warp's stores are ordered before this release by the barrier above; the ticket warp takes it from there
+      asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(sm_addr(&s_scored[stage])) : "memory");
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sm_addr(&empty[stage])) : "memory");
+    }
   }
+  SWARM_STAMP(status, 13);
   SWARM_KERNEL_END(status, 0);
 }
 
@@ -385,7 +481,7 @@ EncodeTiledFn summary_encode_fn() {
   return fn;
 }
 
-// summaries as a 3-D bf16 tensor [page][kv head][256]; boxes of 16 pages x 1 KV head x 64 coordinates
+// summaries as a 3-D bf16 tensor [page][kv head][256]; boxes of 16 pages x 2 KV heads x 64 coordinates
 cudaError_t make_summary_map(CUtensorMap* map, const void* ksum, int Hkv, long long n_pool_pages) {
   EncodeTiledFn fn = summary_encode_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
@@ -409,15 +505,16 @@ cudaError_t launch_one(const Geometry& geo, const uint16_t* q, const uint16_t* k
 }
 
 cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
-                       const int32_t* ctx_len, float* scores, uint32_t* status, cudaStream_t st) {
+                       const int32_t* ctx_len, float* scores, uint32_t* status, unsigned* ready, int reserve_sms,
+                       cudaStream_t st) {
   CUtensorMap map;
   cudaError_t e = make_summary_map(&map, ksum, geo.Hkv, geo.n_pool_pages);
   if (e != cudaSuccess) return e;
-  const int kv_groups = (geo.Hkv + kMmaConsumers - 1) / kMmaConsumers;
-  const long long max_blocks = (long long)geo.B * ((geo.Pmax + kMmaPages - 1) / kMmaPages) * kv_groups;
-  const int grid = (int)std::min<long long>(g_sm_count, std::max<long long>(1, max_blocks));
+  const long long max_blocks = (long long)geo.B * ((geo.Pmax + kBlkPages - 1) / kBlkPages) * head_pairs(geo.Hkv);
+  const int sms = std::max(1, g_sm_count - reserve_sms);
+  const int grid = (int)std::min<long long>(sms, std::max<long long>(1, max_blocks));
   return launch_pdl(page_score_mma_kernel, dim3(grid), dim3(kMmaThreads), kMmaSmemBytes, st, true, map, geo, q, page_base,
-                    ctx_len, scores, status);
+                    ctx_len, scores, status, ready);
 }
 
 }  // namespace
@@ -433,14 +530,14 @@ cudaError_t configure_score() {
 }
 
 bool score_streams(const Geometry& geo) { return geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31); }
+bool score_raises_tickets(const Geometry& geo) { return geo.scorer != SWARM_SCORER_FP32 && score_streams(geo); }
 
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
-                              cudaStream_t st) {
+                              cudaStream_t st, unsigned* ready, int reserve_sms) {
   // Streaming tensor-core variant whenever the batch fits its prefix table and the pool fits 32-bit TMA
   // coordinates; otherwise the register-resident grid kernel on the fp32 pipes.
-  if (geo.scorer != SWARM_SCORER_FP32 && score_streams(geo))
-    return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, st);
+  if (score_raises_tickets(geo)) return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, ready, reserve_sms, st);
   // Heads of a KV group are processed G at a time, G the largest of 8/4/2/1 dividing the group size.
   if (geo.g % 8 == 0) return launch_one<8, 4, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);
   if (geo.g % 4 == 0) return launch_one<4, 8, 2>(geo, q, ksum, page_base, ctx_len, scores, status, st);

@@ -16,14 +16,74 @@ struct WorkspaceLayout {
   int64_t scores;        // f32 [B][Hq][Pmax]          (used when the caller passes no scores buffer)
   int64_t n_tok;         // i32 [B][Hq]                (used when the caller passes no n_tok buffer)
   int64_t q_stage;       // bf16 [B][Hq][d]            (swarm_step_host)
-  int64_t flags;         // u8  [max_clusters_total]   cluster dedup flags (zero between calls)
+  int64_t flags;         // u8  2 x [max_clusters_total] cluster dedup flags (zero between calls); the second array
+  int64_t flags_alt;     //     starts flags_alt bytes after the first and is used by the overlapped tail only
   int64_t part_acc;      // f32 [B*Hq][max_splits][d]  split-K partial outputs
   int64_t part_ml;       // f32 [B*Hq][max_splits][2]  split-K partial (max, sum)
   int64_t items;         // uint4 [max_clusters_total]  (replica mask, weight, output slot, -) of the serial pass
   int64_t selmap;        // u8  [B*Hq][pitch]           per-head bitmap of the selected pages
   int64_t tickets;       // u32 [B*Hq]                 arrival counters of the split merge (zero between calls)
+  int64_t ctl;           // u32 [64]                   control words of the step's hand-offs, see StepTickets (zero at set-up)
+  int64_t ready;         // u32 [B][head pairs]        score units complete (scorer -> selection; zero between steps)
+  int64_t sel_ready;     // u32 [B][Hkv]               heads selected (selection -> attention; zero between steps)
   int64_t total;
 };
+
+// Hand-offs between the kernels of a step.  The kernels are chained by programmatic dependent launch, so a
+// kernel is resident before its predecessor has finished; instead of waiting for the whole predecessor it
+// waits (bounded) for the counter of exactly the data it reads:
+//   ready[b][hp]      the scorer adds 1 for every (16-page tile, KV head) of request b and KV-head pair hp whose
+//                     scores are stored; the selection of a head starts when its pair has all of them
+//   sel_ready[b][kv]  a selection CTA adds 1 when its head's page bitmap and cluster marks are stored; the
+//                     attention CTAs of (b, kv) start when all g heads have arrived
+// Every wait is on a kernel launched earlier in the same stream whose CTAs are all resident (that is the
+// condition for the dependent launch), so no waiter can hold a resource the producer needs.  The counters are
+// set back to zero by the last CTA that needs them (ctl words count those).  A null pointer switches a
+// hand-off off: the consumer then waits for its whole predecessor (griddepcontrol.wait).
+struct StepTickets {
+  unsigned* ready;
+  unsigned* sel_ready;
+  unsigned* ctl;   // [0] selection CTAs finished; [1] attention CTAs past their wait; [2] steps whose cluster marks
+                   // are complete; [3] steps whose cluster resolution has finished ([2], [3]: overlapped tail only)
+};
+constexpr int kCtlTopkDone = 0, kCtlAttnPast = 1, kCtlMarked = 2, kCtlResolved = 3;
+constexpr unsigned kTicketWaitLimit = 1u << 22;            // polls, ~100 ns apart
+__host__ __device__ inline int head_pairs(int Hkv) { return (Hkv + 1) / 2; }
+
+// Bounded wait until the counter *p has reached `target` (acquire; the difference is taken modulo 2^32, so
+// counters that only ever grow may wrap); false when the limit ran out.
+__device__ __forceinline__ bool wait_at_least(const unsigned* p, unsigned target) {
+  for (unsigned polls = 0; polls < kTicketWaitLimit; ++polls) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if ((int)(v - target) >= 0) return true;
+    __nanosleep(64);
+  }
+  return false;
+}
+// Release / acquire-release updates of a counter at GPU scope.  Called by one thread after a warp- or CTA-wide
+// barrier: the barrier orders the other threads' stores before this thread's release, which is cumulative over
+// them.  (A plain __threadfence() is the sequentially consistent fence, which costs far more.)
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned atom_acq_rel_add(unsigned* p, unsigned v) {
+  unsigned prev;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(p), "r"(v) : "memory");
+  return prev;
+}
+__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool wait_zero(const unsigned* p) {
+  for (unsigned polls = 0; polls < kTicketWaitLimit; ++polls) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if (v == 0u) return true;
+    __nanosleep(64);
+  }
+  return false;
+}
 
 constexpr int kMaxSplits = 64;
 
@@ -42,6 +102,7 @@ struct Geometry {   // plain copy of the shape in kernel-friendly form
 cudaError_t configure_score();
 int sm_count();         // SMs of the device current at configure_score() (148 on B200)
 cudaError_t configure_topk();
+int topk_threads(int Pmax);   // threads of the selection CTA launched for lists of up to Pmax pages
 cudaError_t configure_resolve();
 cudaError_t configure_attention();
 cudaError_t configure_medoid();
@@ -49,18 +110,29 @@ cudaError_t configure_medoid();
 // ---- kernel launchers (each returns cudaGetLastError() after the launch) ----------------------
 cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool, const int64_t* page_base,
                                    const int32_t* ctx_len, uint16_t* ksum, uint32_t* status, cudaStream_t st);
-bool score_streams(const Geometry& geo);   // the shape allows the streaming tensor-core scorer
+bool score_streams(const Geometry& geo);          // the shape allows the streaming tensor-core scorer
+bool score_raises_tickets(const Geometry& geo);   // ... and it is the one that will run: it counts its progress on `ready`
+// `ready` (StepTickets::ready, may be null) is raised by the streaming scorer only; `reserve_sms` SMs are left
+// free for the selection CTAs that wait on it.
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
-                              cudaStream_t st);
+                              cudaStream_t st, unsigned* ready = nullptr, int reserve_sms = 0);
 // `overlap`: launch with programmatic dependent launch after the previous kernel of the stream.
 // `selmap` (optional): per (request, head) bitmap of the selected pages, rows of selmap_pitch_bytes(Pmax).
 // `flags` with the three tables (optional): also mark the selected pages' clusters (see launch_resolve).
+// `links`: how the kernel is tied to its neighbours (all zero: it waits for the whole previous kernel and
+// announces nothing).  tk.ready needs req_base (what the scorer was given as page_base).
+struct TopkLinks {
+  StepTickets tk{nullptr, nullptr, nullptr};
+  const int64_t* req_base = nullptr;
+  long long flags_alt = 0;      // bytes between the two cluster-flag arrays of the overlapped tail, else 0
+};
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap = nullptr,
-                        const int64_t* page_base = nullptr, const int32_t* page2cluster = nullptr,
-                        const int64_t* cluster_base = nullptr, uint8_t* flags = nullptr,
-                        const uint32_t* replica_mask = nullptr, const uint16_t* cluster_size = nullptr);
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, const TopkLinks& links,
+                        uint8_t* selmap = nullptr, const int64_t* page_base = nullptr,
+                        const int32_t* page2cluster = nullptr, const int64_t* cluster_base = nullptr,
+                        uint8_t* flags = nullptr, const uint32_t* replica_mask = nullptr,
+                        const uint16_t* cluster_size = nullptr);
 // Everything the cluster-resolution body needs (see resolve_body.cuh).  sel == nullptr: the flags are already
 // set (by the selection or the expansion kernel) and a single CTA runs the tail.
 // Host-step extension of the fused attention + resolution kernel: the step's small results are also stored
@@ -99,6 +171,10 @@ struct ResolveArgs {
   int32_t* submit_order;   // optional: submission order (indices into uniq), see resolve_body.cuh
   int32_t* submit_info;    // optional: [0] batches, [1] clusters submitted
   HostMirror host{};
+  // Overlapped tail (the kernel runs beside the NEXT step's scoring and selection): the control words of
+  // StepTickets, and the distance between the two flag arrays that alternate steps mark.  Null / 0 otherwise.
+  unsigned* tail_ctl = nullptr;
+  long long flags_alt = 0;
 };
 ResolveArgs make_resolve_args(const Geometry& geo, const int32_t* sel, const int32_t* n_sel, const int64_t* page_base,
                               const int32_t* page2cluster, const int64_t* cluster_base, const uint32_t* replica_mask,
@@ -134,6 +210,7 @@ struct AttnArgs {
   float* lse;
   int n_splits;
   HostMirror host{};
+  StepTickets tk{nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
 };
 // `fused_resolve` (paged mode only): one extra CTA of the grid runs cluster resolution with these arguments.
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,

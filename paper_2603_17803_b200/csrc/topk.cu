@@ -45,7 +45,76 @@ struct TopkExtras {
   const uint32_t* replica_mask;
   const uint16_t* cluster_size;
   long long n_pool_pages;
+  // hand-offs (see StepTickets): wait for the scorer's tickets instead of the whole scorer; announce each head
+  const int64_t* req_base;        // [B+1] pages (or, for the medoid index, clusters) each request owns
+  StepTickets tk;
+  long long flags_alt;            // > 0: two flag arrays this many bytes apart, used by alternate steps (overlapped tail)
 };
+
+// What a selection CTA does before it reads its head's scores.  With tickets: one thread waits (bounded) until
+// the scorer has stored every tile of the head's KV pair; a request whose length the scorer refuses never gets
+// tickets and is not waited for.  Without: the whole previous kernel.  Returns false when the head has no
+// usable scores (refused length, or the wait ran out): the CTA then writes an empty selection.
+__device__ __forceinline__ bool scores_ready(const Geometry& geo, const TopkExtras& x, int b, int kvh, int len_b, bool* s_flag) {
+  // (Overlapped tail: the flag array this step marks was last read by the resolution of the step before the
+  // previous one, which has finished by now in any schedule that keeps up; make sure of it.)
+  if (threadIdx.x == 0 && x.flags_alt > 0) {
+    const unsigned marked = x.tk.ctl[kCtlMarked];
+    if (marked >= 1u && !wait_at_least(x.tk.ctl + kCtlResolved, marked - 1u)) atomicOr(x.status, SWARM_DEV_TIMEOUT);
+  }
+  if (x.tk.ready == nullptr) {
+    pdl_wait();
+    return true;
+  }
+  if (threadIdx.x == 0) {
+    const int P = pages_of(len_b, geo.S);
+    bool ok = len_b >= 1 && P <= geo.Pmax && (long long)P <= x.req_base[b + 1] - x.req_base[b];
+    if (ok) {
+      const int hp = kvh / 2;
+      const unsigned target = (unsigned)((P + 15) / 16) * (unsigned)min(2, geo.Hkv - 2 * hp);
+      ok = wait_at_least(x.tk.ready + (long long)b * head_pairs(geo.Hkv) + hp, target);
+      if (!ok) atomicOr(x.status, SWARM_DEV_TIMEOUT);
+    }
+    *s_flag = ok;
+  }
+  __syncthreads();
+  return *s_flag;
+}
+
+// An empty selection for head bh (no usable scores).
+__device__ __forceinline__ void write_empty_selection(const Geometry& geo, const TopkExtras& x, int bh, int32_t* out,
+                                                      int32_t* n_sel, int threads) {
+  for (int j = threadIdx.x; j < geo.k; j += threads) out[j] = -1;
+  if (threadIdx.x == 0) n_sel[bh] = 0;
+  if (x.selmap != nullptr) {
+    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
+    for (int o = threadIdx.x * 4; o + 4 <= x.selmap_pitch; o += threads * 4) *reinterpret_cast<uint32_t*>(row + o) = 0u;
+  }
+}
+
+// What a selection CTA does last, after a barrier behind its stores: announce the head to the attention CTAs of
+// its KV head, and count itself; the last CTA of the launch clears the scorer's tickets for the next step.
+__device__ __forceinline__ void selection_done(const Geometry& geo, const TopkExtras& x, int b, int kvh, bool* s_flag) {
+  if (x.tk.ctl == nullptr) return;
+  __syncthreads();                                          // every thread's stores are issued
+  if (threadIdx.x == 0) {                                   // releases, cumulative over them
+    if (x.tk.sel_ready != nullptr) red_release_add(x.tk.sel_ready + (long long)b * geo.Hkv + kvh, 1u);
+    const unsigned prev = atom_acq_rel_add(x.tk.ctl + kCtlTopkDone, 1u);
+    *s_flag = prev == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (*s_flag) {                                            // every other CTA has finished: nobody reads the tickets any more
+    if (x.tk.ready != nullptr)
+      for (int i = threadIdx.x; i < geo.B * head_pairs(geo.Hkv); i += blockDim.x) x.tk.ready[i] = 0u;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      if (x.flags_alt > 0) x.tk.ctl[kCtlMarked] += 1u;      // the cluster marks of one more step are complete
+      // last of all: whoever reads 0 here (the attention kernel, before it lets the next step start) also sees
+      // the cleared tickets
+      st_release(x.tk.ctl + kCtlTopkDone, 0u);
+    }
+  }
+}
 
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
@@ -220,12 +289,12 @@ __device__ __forceinline__ void topk_regs_body(SelectState& st, const Geometry& 
   if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
 #pragma unroll
     for (int j = 0; j < ITEMS; j += 4) {
-      const float4 v = *reinterpret_cast<const float4*>(s + p0 + j);
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(s + p0 + j));   // written by a kernel that may still run: not through L1
       key[j] = score_key(v.x); key[j + 1] = score_key(v.y); key[j + 2] = score_key(v.z); key[j + 3] = score_key(v.w);
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < ITEMS; ++j) key[j] = p0 + j < P ? score_key(s[p0 + j]) : 0u;
+    for (int j = 0; j < ITEMS; ++j) key[j] = p0 + j < P ? score_key(__ldcg(s + p0 + j)) : 0u;
   }
   if (tid == 0) st.remaining = k_sel;
   SWARM_STAMP(status, 2);
@@ -371,8 +440,9 @@ __global__ void __launch_bounds__(THREADS)
 topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
                  int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
   __shared__ SelectState st;
+  __shared__ bool s_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int bh = blockIdx.x, b = bh / geo.Hq;
+  const int bh = blockIdx.x, b = bh / geo.Hq, kvh = (bh - b * geo.Hq) / geo.g;
   pdl_launch_dependents();
   SWARM_STAMP(status, 0);
   SWARM_KERNEL_BEGIN(status, 1);
@@ -380,20 +450,26 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   prefetch_tables(geo, x);
   const RequestBases rb = load_bases(x, b);
   const int len_b = ctx_len[b];
-  pdl_wait();                                               // the scores come from the previous kernel
+  const float* s = scores + (long long)bh * geo.Pmax;
+  int32_t* out = sel + (long long)bh * geo.k;
+  if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;   // stable: the previous step's selection has finished
+  if (!scores_ready(geo, x, b, kvh, len_b, &s_flag)) {     // the scores come from the previous kernel
+    write_empty_selection(geo, x, bh, out, n_sel, THREADS);
+    selection_done(geo, x, b, kvh, &s_flag);
+    return;
+  }
   SWARM_STAMP(status, 1);
   const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
   const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
-  const float* s = scores + (long long)bh * geo.Pmax;
-  int32_t* out = sel + (long long)bh * geo.k;
   // A list half as long as the kernel's capacity is handled with half the pages per thread: the work of every
   // phase is per page held, and the lists of one launch differ in length (ragged batches).
   if (ITEMS == 16 && P <= THREADS * 8)
     topk_regs_body<THREADS, 8, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
   else
     topk_regs_body<THREADS, ITEMS, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
+  selection_done(geo, x, b, kvh, &s_flag);
   SWARM_KERNEL_END(status, 1);
 }
 
@@ -407,25 +483,31 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   extern __shared__ uint32_t skeys[];
   __shared__ SelectState st;
   __shared__ int warp_gt[32], warp_eq[32];
+  __shared__ bool s_flag;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int bh = blockIdx.x, b = bh / geo.Hq;
+  const int bh = blockIdx.x, b = bh / geo.Hq, kvh = (bh - b * geo.Hq) / geo.g;
   pdl_launch_dependents();
   for (int i = tid; i < kBins; i += kGenericThreads) st.hist[i] = 0;
   prefetch_tables(geo, x);
   const RequestBases rb = load_bases(x, b);
   const int len_b = ctx_len[b];
-  pdl_wait();
+  const float* s = scores + (long long)bh * geo.Pmax;
+  int32_t* out = sel + (long long)bh * geo.k;
+  if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;
+  if (!scores_ready(geo, x, b, kvh, len_b, &s_flag)) {
+    write_empty_selection(geo, x, bh, out, n_sel, kGenericThreads);
+    selection_done(geo, x, b, kvh, &s_flag);
+    return;
+  }
   const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // see topk_regs_kernel
   const int k_sel = k_eff - (P - Pw);
-  const float* s = scores + (long long)bh * geo.Pmax;
-  int32_t* out = sel + (long long)bh * geo.k;
-  auto key_at = [&](int i) -> uint32_t { return kKeysInSmem ? skeys[i] : score_key(s[i]); };
+  auto key_at = [&](int i) -> uint32_t { return kKeysInSmem ? skeys[i] : score_key(__ldcg(s + i)); };
 
   uint32_t lo = 0xFFFFFFFFu, hi = 0u;
   for (int i = tid; i < P; i += kGenericThreads) {
-    const uint32_t key = score_key(s[i]);
+    const uint32_t key = score_key(__ldcg(s + i));
     if (kKeysInSmem) skeys[i] = key;
     if (i < Pw) {
       lo = min(lo, key);
@@ -499,11 +581,14 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   }
   for (int j = k_eff + tid; j < geo.k; j += kGenericThreads) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
+  selection_done(geo, x, b, kvh, &s_flag);
 }
 
 constexpr size_t kSmemKeyBytes = 160 * 1024;
 
 }  // namespace
+
+int topk_threads(int Pmax) { return Pmax <= 1024 ? 128 : Pmax <= 2048 ? 256 : Pmax <= 4096 ? 512 : 1024; }
 
 cudaError_t configure_topk() {
   return cudaFuncSetAttribute(topk_generic_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -511,9 +596,10 @@ cudaError_t configure_topk() {
 }
 
 cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t* ctx_len, int32_t* sel,
-                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, uint8_t* selmap,
-                        const int64_t* page_base, const int32_t* page2cluster, const int64_t* cluster_base,
-                        uint8_t* flags, const uint32_t* replica_mask, const uint16_t* cluster_size) {
+                        int32_t* n_sel, uint32_t* status, cudaStream_t st, bool overlap, const TopkLinks& links,
+                        uint8_t* selmap, const int64_t* page_base, const int32_t* page2cluster,
+                        const int64_t* cluster_base, uint8_t* flags, const uint32_t* replica_mask,
+                        const uint16_t* cluster_size) {
   TopkExtras x;
   x.selmap = selmap;
   x.selmap_pitch = selmap_pitch_bytes(geo.Pmax);
@@ -525,6 +611,10 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   x.replica_mask = replica_mask;
   x.cluster_size = cluster_size;
   x.n_pool_pages = geo.n_pool_pages;
+  x.req_base = links.req_base;
+  x.tk = links.tk;
+  x.flags_alt = flags != nullptr ? links.flags_alt : 0;
+  if (x.req_base == nullptr) x.tk.ready = nullptr;         // the validity test of a request needs its page count
   const dim3 grid(geo.B * geo.Hq);
 #define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                    \
   return launch_pdl(topk_regs_kernel<THREADS, ITEMS>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \

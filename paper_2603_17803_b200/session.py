@@ -34,7 +34,7 @@ class Session:
 
     def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
                  ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0,
-                 max_clusters_total: Optional[int] = None, scorer: int = B.SCORER_AUTO):
+                 max_clusters_total: Optional[int] = None, scorer: int = B.SCORER_AUTO, tail_stream=None):
         cfg = workload.cfg
         self.cfg = cfg
         self.w = workload
@@ -53,6 +53,9 @@ class Session:
         B.swarm_set_workspace(self.ctx, self.workspace)
         if scorer != B.SCORER_AUTO:
             B.swarm_set_scorer(self.ctx, scorer)
+        self.tail_stream = tail_stream
+        if tail_stream is not None:
+            B.swarm_set_tail_stream(self.ctx, tail_stream)
         self.ksum = ksum if ksum is not None else torch.empty(
             (workload.n_pool_pages, cfg.n_kv_heads, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
         self.inputs = self._inputs(workload.q)
@@ -109,6 +112,10 @@ class Session:
 
     def step(self, stream=None):
         B.swarm_step(self.ctx, self.inputs, self.outputs, stream)
+
+    def tail_join(self, stream=None):
+        """Make `stream` wait for the cluster resolution of the last step (only needed with a tail stream)."""
+        B.swarm_tail_join(self.ctx, stream)
 
     # -- the step in two halves (query heads spread over several ctxs) --------------------------------
     def step_begin(self, stream=None):

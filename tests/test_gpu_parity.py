@@ -72,6 +72,61 @@ def test_fused_step_equals_composition(name):
         s.close()
 
 
+@pytest.mark.parametrize("name", ["c2_small", "c3_small", "c5_small", "k_exceeds_pages"])
+def test_overlapped_tail_gives_the_same_step(name):
+    """Cluster resolution on a tail stream (swarm_set_tail_stream): consecutive steps with changing queries are
+    enqueued without waiting in between, so a step's resolution runs beside the next step's scoring and
+    selection; every step's outputs must equal those of the plain step bit for bit (integers) / within rounding
+    (attention), and the last one must match the oracle."""
+    w = W.generate(CASES[name], seed=14, device=DEV)
+    plain = Session(w)
+    tail_stream, stream = torch.cuda.Stream(), torch.cuda.Stream()
+    tail = Session(w, ksum=plain.ksum, tail_stream=tail_stream)
+    qs = [w.q, (w.q.float() * -1.0).to(torch.bfloat16), (w.q.float() * 0.5 + 0.125).to(torch.bfloat16), w.q]
+    want = []
+    for q in qs:
+        plain.set_query(q)
+        plain.step()
+        torch.cuda.synchronize()
+        n = int(plain.o.n_uniq[0])
+        want.append(dict(sel=plain.o.sel.clone(), uniq=plain.o.uniq[:n].clone(), queue_of=plain.o.queue_of[:n].clone(),
+                         load=plain.o.queue_load.clone(), out=plain.o.out.clone(), lse=plain.o.lse.clone()))
+    # the tail session needs one set of outputs per step in flight: give every step its own
+    outs = []
+    with torch.cuda.stream(stream):
+        for q in qs:
+            o = type(tail.o)(**{f: (getattr(tail.o, f).clone() if getattr(tail.o, f) is not None else None)
+                                for f in tail.o.__dataclass_fields__})
+            outs.append(o)
+            tail.o = o
+            tail.outputs = B.make_outputs(**{k_: getattr(o, k_) for k_ in o.__dataclass_fields__})
+            tail.set_query(q)
+            tail.step(stream=stream)
+        tail.tail_join(stream)
+        stream.synchronize()
+    assert tail.status() == 0
+    for o, ref in zip(outs, want):
+        n = len(ref["uniq"])
+        assert int(o.n_uniq[0]) == n
+        assert torch.equal(o.sel, ref["sel"]) and torch.equal(o.uniq[:n], ref["uniq"])
+        assert torch.equal(o.queue_of[:n], ref["queue_of"]) and torch.equal(o.queue_load, ref["load"])
+        assert (o.out - ref["out"]).abs().max().item() <= 1e-4 and (o.lse - ref["lse"]).abs().max().item() <= 1e-4
+    parity.check_step(w, tail)
+    # the same chain recorded into a CUDA graph (the capture has to join the tail stream) and replayed twice
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(3):
+                tail.step(stream=stream)
+            tail.tail_join(stream)
+        g.replay()
+        g.replay()
+        stream.synchronize()
+    parity.check_step(w, tail)
+    plain.close()
+    tail.close()
+
+
 @pytest.mark.parametrize("hq,hkv", [(16, 2), (8, 2), (6, 3), (5, 5), (6, 2)])
 def test_fp32_pipe_scorer_matches_oracle(hq, hkv):
     """The scorer on the fp32 pipes (what shapes beyond the streaming kernel's limits fall back to), forced by
