@@ -196,7 +196,7 @@ int32_t swarm_tail_join(swarm_ctx* ctx, void* stream);
 int32_t swarm_set_select_sms(swarm_ctx* ctx, int32_t n_sms);
 
 /* Which kernel scores the pages (stage 1).  The result is the same sum either way, within fp32 rounding.
- *   SWARM_SCORER_AUTO    the streaming tensor-core kernel whenever the shape allows it (batch <= 1024 and fewer
+ *   SWARM_SCORER_AUTO    the streaming tensor-core kernel whenever the shape allows it (batch <= 512 and fewer
  *                        than 2^31 pool pages), else the fp32-pipe kernel
  *   SWARM_SCORER_TENSOR  the streaming tensor-core kernel; SWARM_ERR_UNSUPPORTED if the shape does not allow it
  *   SWARM_SCORER_FP32    the fp32-pipe kernel (16-byte row loads, sign-split weights in registers) */

@@ -123,10 +123,13 @@ int reserved_sms(const swarm_ctx* ctx, const Geometry& g, bool tail) {
   if (!score_raises_tickets(g)) return 0;
   int n = ctx->select_sms;
   if (n < 0) {
+    // Selection CTAs of up to 256 threads fit on an SM beside a scorer CTA (registers and shared memory were
+    // sized for it): nothing to reserve.  Larger ones need an SM of their own: one per list, at most a
+    // quarter of the device (measured at 64 requests of up to 16384 pages: 37 reserved SMs beat both 0 and 54).
     const int threads = topk_threads(g.Pmax);
-    const int per_sm = std::max(1, std::min(2048 / threads, 65536 / (64 * threads)));
     const long long lists = (long long)g.B * g.Hq;
-    n = (int)std::min<long long>((lists + per_sm - 1) / per_sm, sm_count() / 4);
+    const int per_sm = std::max(1, 1024 / threads);
+    n = threads <= 256 ? 0 : (int)std::min<long long>((lists + per_sm - 1) / per_sm, sm_count() / 4);
   }
   n += tail ? 1 : 0;
   return std::min(n, sm_count() - 8);
@@ -628,7 +631,7 @@ int32_t enqueue_host_step(swarm_ctx* ctx, const swarm_inputs* in, const swarm_ou
                       (n_uniq_host == nullptr || n_uniq_d) && (queue_load_host == nullptr || queue_load_d);
   if (direct && ctx->done_d != nullptr) {
     const HostMirror host{out_d, lse_d, n_uniq_d, queue_load_d, ws_ptr<unsigned>(ctx, ctx->lay.status + 96), ctx->done_d,
-                          (unsigned)attention_groups(ctx->geo, true) + 1u};
+                          (unsigned)bh + 1u};                // one arrival per head, one for the resolution
     const int32_t rc = step_impl(ctx, &local, o, st, &host, kStepBegin | kStepEnd);
     *signals = rc == SWARM_OK;
     return rc;

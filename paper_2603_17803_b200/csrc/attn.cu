@@ -142,7 +142,6 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   constexpr int kVOff = kWide ? kBoxBytes : 2 * kBoxBytes;   // V tile relative to the K tile
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
-  __shared__ __align__(8) uint64_t bar_merge;
   __shared__ int s_wcnt[kAttnWarps];
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -171,7 +170,6 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   if (lane == 0) {
 #pragma unroll
     for (int sidx = 0; sidx < kStages; ++sidx) mbar_init(&bars[warp][sidx], 1);
-    if (warp == 0) mbar_init(&bar_merge, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
@@ -181,7 +179,29 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   // CTAs release their dependents by exiting: with this trigger the step was measured 1.5 us slower.
   const bool ticketed = kPaged && a.tk.sel_ready != nullptr;
   if (kFused == 0 && !ticketed) pdl_launch_dependents();
+  // What the CTA needs besides the selection: the request's length and first pool page, and Q as the A operand of
+  // S^T = Q K^T (row = head (quad), 8 k-steps of 16 coordinates).  Inside a step these are inputs of the whole
+  // step, stable since its first kernel started, and are fetched while the CTA waits for the selection;
+  // stand-alone they may come from the previous kernel and are fetched after it.
+  uint32_t qa[8][2];
+  int len = 0;
+  long long pool_row0 = 0;
+  auto load_inputs = [&]() {
+    if (kPaged) {
+      len = a.ctx_len[b];
+      pool_row0 = a.page_base[b];
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&mapK) : "memory");
+    }
+    const bool row_ok = quad < G;
+    const uint16_t* qrow = a.q + (long long)(bh0 + (row_ok ? quad : 0)) * kHeadDim;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + tq * 2) : 0u;
+      qa[ks][1] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + tq * 2) : 0u;
+    }
+  };
   if (ticketed) {
+    load_inputs();
     // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The last CTA
     // of the grid to get past its wait sets the tickets back to zero for the next step -- after the selection
     // kernel's own last CTA has finished its bookkeeping, so that the next step cannot start before it.
@@ -201,11 +221,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     }
   } else {
     pdl_wait();                                         // the selection comes from the previous kernel
+    load_inputs();
   }
   SWARM_STAMP(status, 1);
 
   int P = 0, tail = S, total_tok = 0, n_items;          // items: pages of the union (paged) or page slots (gathered)
-  long long pool_row0 = 0;
   int n_words = 0;
 
   // one bitmap word (32 pages) of every head of the group; the row pitch bounds the loads, so they do not
@@ -235,9 +255,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 
   if (kPaged) {
     // number of pages in the union of the group's selections: the splits share them evenly by rank
-    HeadWords hw = load_raw((int)threadIdx.x);          // in flight together with the two loads below
-    const int len = a.ctx_len[b];
-    pool_row0 = a.page_base[b];
+    HeadWords hw = load_raw((int)threadIdx.x);
     P = pages_of(len, S);
     tail = len - S * (P - 1);
     n_words = min((P + 31) / 32, pitch_words);
@@ -265,17 +283,6 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   const int it_begin = (int)((long long)n_items * split / a.n_splits);
   const int it_end = (int)((long long)n_items * (split + 1) / a.n_splits);
 
-  // ---- Q as the A operand of S^T = Q K^T: row = head (quad), 8 k-steps of 16 coordinates -----------
-  uint32_t qa[8][2];
-  {
-    const bool row_ok = quad < G;
-    const uint16_t* qrow = a.q + (long long)(bh0 + (row_ok ? quad : 0)) * kHeadDim;
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      qa[ks][0] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + tq * 2) : 0u;
-      qa[ks][1] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + tq * 2) : 0u;
-    }
-  }
   const float scale = kLog2e * rsqrtf((float)kHeadDim);
 
   float m_run = -INFINITY, l_run = 0.f;                 // of head `quad`, over this lane's token columns
@@ -475,6 +482,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   SWARM_STAMP_ANY_CTA(status, 7);
 
   // ---- merge the warps of the CTA (the ring is idle now and is reused as scratch) ------------------
+  // Three short phases, each warp-parallel: (1) every warp posts its (max, sum) per head; (2) every lane scales
+  // its own accumulators to the CTA-wide maximum of its heads and posts them; (3) warp h sums head h over the
+  // warps, four coordinates per lane, and is the one that publishes (or finishes) that head.
   __syncthreads();
   // rows of 128 + 4 floats: the four lanes of a quad store to heads 2*tq, whose rows then start 8 banks apart
   constexpr int kAccRow = kHeadDim + 4;
@@ -483,139 +493,105 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   float* s_l = s_m + kAttnWarps * 8;                    // [warp][8]
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-  if (tq == 0) { s_m[warp * 8 + quad] = m_run; s_l[warp * 8 + quad] = l_run; }
+  if (tq == 0) s_m[warp * 8 + quad] = m_run;
+  __syncthreads();
+  {
+    float sc[2];
 #pragma unroll
-  for (int mt = 0; mt < 8; ++mt) {
-    float* base = s_acc + (warp * 8 + 2 * tq) * kAccRow + 16 * mt + quad;
-    base[0] = acc[mt][0];
-    base[kAccRow] = acc[mt][1];
-    base[8] = acc[mt][2];
-    base[kAccRow + 8] = acc[mt][3];
+    for (int j = 0; j < 2; ++j) {
+      const int hh = 2 * tq + j;
+      float Mh = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kAttnWarps; ++w) Mh = fmaxf(Mh, s_m[w * 8 + hh]);
+      sc[j] = exp2_or_zero(s_m[warp * 8 + hh], Mh);
+    }
+    if (tq == 0) {                                      // this warp's sum of head `quad`, on the common scale
+      float Mq = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kAttnWarps; ++w) Mq = fmaxf(Mq, s_m[w * 8 + quad]);
+      s_l[warp * 8 + quad] = l_run * exp2_or_zero(m_run, Mq);
+    }
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      float* base = s_acc + (warp * 8 + 2 * tq) * kAccRow + 16 * mt + quad;
+      base[0] = acc[mt][0] * sc[0];
+      base[kAccRow] = acc[mt][1] * sc[1];
+      base[8] = acc[mt][2] * sc[0];
+      base[kAccRow + 8] = acc[mt][3] * sc[1];
+    }
   }
   __syncthreads();
-  const int t = threadIdx.x;                            // threads 0..127: one output coordinate each
-  const bool has_dim = t < kHeadDim;
-  float M[8], L[8], o[8];
+  SWARM_STAMP(status, 5);
+  if (warp < G) {
+    const int hh = warp;                                // this warp's head; lane: coordinates 4 * lane .. + 3
+    float M = -INFINITY, L = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-  for (int hh = 0; hh < 8; ++hh) {
-    M[hh] = -INFINITY; L[hh] = 0.f; o[hh] = 0.f;
-    if (hh < G && has_dim) {
-#pragma unroll
-      for (int w = 0; w < kAttnWarps; ++w) M[hh] = fmaxf(M[hh], s_m[w * 8 + hh]);
-#pragma unroll
-      for (int w = 0; w < kAttnWarps; ++w) {
-        const float sc = exp2_or_zero(s_m[w * 8 + hh], M[hh]);
-        L[hh] += s_l[w * 8 + hh] * sc;
-        o[hh] += s_acc[(w * 8 + hh) * kAccRow + t] * sc;
-      }
+    for (int w = 0; w < kAttnWarps; ++w) {
+      M = fmaxf(M, s_m[w * 8 + hh]);
+      L += s_l[w * 8 + hh];
+      const float4 v = *reinterpret_cast<const float4*>(s_acc + (w * 8 + hh) * kAccRow + 4 * lane);
+      o.x += v.x; o.y += v.y; o.z += v.z; o.w += v.w;
     }
-  }
-  if (a.n_splits > 1) {
-    // publish this split's partials, then let the last split of the group merge all of them
+    const long long bh = bh0 + hh;
+    bool finish = true;                                 // this warp writes the head's final result
+    if (a.n_splits > 1) {
+      // publish this split's partial of the head; the warp that arrives last at the head's ticket (whichever
+      // CTA it sits in) merges the head's partials.  The heads of a group are thus merged side by side, and
+      // nothing waits for a CTA-wide barrier or a staging copy.
+      const long long slot = bh * a.n_splits + split;
+      __stcg(reinterpret_cast<float4*>(a.part_acc + slot * kHeadDim) + lane, o);
+      if (lane == 0) __stcg(reinterpret_cast<float2*>(a.part_ml + slot * 2), make_float2(M, L));
+      __syncwarp();                                     // the lanes' stores are ordered before lane 0's release
+      unsigned prev = 0u;
+      if (lane == 0) prev = atom_acq_rel_add(a.tickets + bh, 1u);
+      prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
+      __syncwarp();                                     // lane 0's acquire is ordered before the other lanes' loads
+      finish = prev == (unsigned)a.n_splits - 1u;
+      if (finish) {
+        // (max, sum) of split `lane` and `lane + 32`; then every lane sums its 4 coordinates over the splits
+        const float2 ml0 = lane < a.n_splits ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * a.n_splits + lane) * 2))
+                                             : make_float2(-INFINITY, 0.f);
+        const float2 ml1 = lane + 32 < a.n_splits
+                               ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * a.n_splits + lane + 32) * 2))
+                               : make_float2(-INFINITY, 0.f);
+        M = fmaxf(ml0.x, ml1.x);
 #pragma unroll
-    for (int hh = 0; hh < 8; ++hh) {
-      if (hh < G && has_dim) {
-        const long long slot = (long long)(bh0 + hh) * a.n_splits + split;
-        __stcg(&a.part_acc[slot * kHeadDim + t], o[hh]);
-        if (t == 0) { __stcg(&a.part_ml[slot * 2], M[hh]); __stcg(&a.part_ml[slot * 2 + 1], L[hh]); }
-      }
-    }
-    __syncthreads();                                    // all of the CTA's partial stores are issued ...
-    if (t == 0) {                                       // ... and published by one release-acquire ticket
-      unsigned prev;
-      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.tickets + grp) : "memory");
-      s_last = (prev == (unsigned)a.n_splits - 1u);
-    }
-    __syncthreads();
-    SWARM_STAMP(status, 5);
-    SWARM_STAMP_ANY_CTA(status, 8);
-    if (!s_last) { SWARM_KERNEL_END(status, 2); return; }
-    // Fetch the group's partial outputs ([head][split][128] floats, contiguous) with one bulk copy per
-    // batch of heads into the idle ring while the (max, sum) pairs are loaded directly; then reduce from
-    // shared memory.  One memory round trip instead of a chain of dependent loads.
-    float* s_part = reinterpret_cast<float*>(ring);
-    float* s_pm = reinterpret_cast<float*>(list_page);  // [head][kMaxSplits]  (the page list is no longer needed)
-    float* s_pl = s_pm + 8 * kMaxSplits;
-    const int row_bytes = a.n_splits * kHeadDim * 4;
-    const int heads_per_batch = max(1, kRingBytes / row_bytes);
-    unsigned phase = 0;
-    for (int hb = 0; hb < G; hb += heads_per_batch) {
-      const int nb = min(heads_per_batch, G - hb);
-      __syncthreads();                                  // everyone is done with the ring and the scratch
-      if (t == 0) {
-        asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy traffic (shared scratch, the partials) first
-        mbar_expect_tx(&bar_merge, (unsigned)(nb * row_bytes));
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                         smem_addr(s_part)),
-                     "l"(a.part_acc + (long long)(bh0 + hb) * a.n_splits * kHeadDim), "r"((unsigned)(nb * row_bytes)),
-                     "r"(smem_addr(&bar_merge))
-                     : "memory");
-      }
-      for (int idx = t; idx < nb * a.n_splits; idx += kAttnWarps * 32) {
-        const int hh = idx / a.n_splits, sp = idx - hh * a.n_splits;
-        const float2 ml =
-            __ldcg(reinterpret_cast<const float2*>(a.part_ml + ((long long)(bh0 + hb + hh) * a.n_splits + sp) * 2));
-        s_pm[hh * kMaxSplits + sp] = ml.x;
-        s_pl[hh * kMaxSplits + sp] = ml.y;
-      }
-      __syncthreads();
-      unsigned polls = 0;
-      while (!mbar_try_wait(&bar_merge, phase) && ++polls < kWaitLimit) {}
-      if (polls >= kWaitLimit) { if (t == 0) atomicOr(status, SWARM_DEV_TIMEOUT); }
-      phase ^= 1u;
-      SWARM_STAMP_ANY_CTA(status, 9);
-      // warp w reduces heads w, w + 4, ...: lanes first turn the (max, sum) pairs into weights, then each
-      // lane sums 4 coordinates over the splits
-      float* s_w = s_pl + 8 * kMaxSplits;               // [kMaxSplits] per warp
-      for (int hh = warp; hh < nb; hh += kAttnWarps) {
-        const float m0 = lane < a.n_splits ? s_pm[hh * kMaxSplits + lane] : -INFINITY;
-        const float m1 = lane + 32 < a.n_splits ? s_pm[hh * kMaxSplits + lane + 32] : -INFINITY;
-        float Mx = fmaxf(m0, m1);
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, o2));
+        const float w0 = exp2_or_zero(ml0.x, M), w1 = exp2_or_zero(ml1.x, M);
+        L = ml0.y * w0 + ml1.y * w1;
 #pragma unroll
-        for (int o2 = 16; o2 >= 1; o2 >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xFFFFFFFFu, Mx, o2));
-        const float w0 = exp2_or_zero(m0, Mx), w1 = exp2_or_zero(m1, Mx);
-        float Ls = (lane < a.n_splits ? s_pl[hh * kMaxSplits + lane] * w0 : 0.f) +
-                   (lane + 32 < a.n_splits ? s_pl[hh * kMaxSplits + lane + 32] * w1 : 0.f);
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) L += __shfl_xor_sync(0xFFFFFFFFu, L, o2);
+        const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * a.n_splits * kHeadDim) + lane;
+        o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp0 = 0; sp0 < a.n_splits; sp0 += 8) {
+          float4 v[8];
 #pragma unroll
-        for (int o2 = 16; o2 >= 1; o2 >>= 1) Ls += __shfl_xor_sync(0xFFFFFFFFu, Ls, o2);
-        s_w[warp * kMaxSplits + lane] = w0;
-        s_w[warp * kMaxSplits + lane + 32] = w1;
-        __syncwarp();
-        const float4* rows = reinterpret_cast<const float4*>(s_part + (long long)hh * a.n_splits * kHeadDim) + lane;
-        float4 os = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-        for (int sp = 0; sp < a.n_splits; ++sp) {
-          const float sc = s_w[warp * kMaxSplits + sp];
-          const float4 v = rows[sp * (kHeadDim / 4)];
-          os.x = fmaf(v.x, sc, os.x); os.y = fmaf(v.y, sc, os.y); os.z = fmaf(v.z, sc, os.z); os.w = fmaf(v.w, sc, os.w);
+          for (int u = 0; u < 8; ++u)                   // eight rows in flight together
+            v[u] = sp0 + u < a.n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int sp = sp0 + u;
+            const float ws = __shfl_sync(0xFFFFFFFFu, sp < 32 ? w0 : w1, sp & 31);
+            o.x = fmaf(v[u].x, ws, o.x); o.y = fmaf(v[u].y, ws, o.y); o.z = fmaf(v[u].z, ws, o.z); o.w = fmaf(v[u].w, ws, o.w);
+          }
         }
-        const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
-        const float4 res = make_float4(os.x * inv, os.y * inv, os.z * inv, os.w * inv);
-        const float lse_h = Ls > 0.f ? (Mx + log2f(Ls)) * kLn2 : -INFINITY;
-        reinterpret_cast<float4*>(a.out + (long long)(bh0 + hb + hh) * kHeadDim)[lane] = res;
-        if (lane == 0) a.lse[bh0 + hb + hh] = lse_h;
-        if (a.host.out_h != nullptr) reinterpret_cast<float4*>(a.host.out_h + (long long)(bh0 + hb + hh) * kHeadDim)[lane] = res;
-        if (a.host.lse_h != nullptr && lane == 0) a.host.lse_h[bh0 + hb + hh] = lse_h;
+        if (lane == 0) a.tickets[bh] = 0u;              // ready for the next launch
+      }
+    }
+    if (finish) {
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+      const float4 res = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+      const float lse_h = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+      reinterpret_cast<float4*>(a.out + bh * kHeadDim)[lane] = res;
+      if (lane == 0) a.lse[bh] = lse_h;
+      if (a.host.out_h != nullptr) reinterpret_cast<float4*>(a.host.out_h + bh * kHeadDim)[lane] = res;
+      if (a.host.lse_h != nullptr && lane == 0) a.host.lse_h[bh] = lse_h;
+      if (a.host.done_h != nullptr) {                   // host step: this head's results are in host memory
         __syncwarp();
+        if (lane == 0) host_arrive(a.host);
       }
     }
-    if (t == 0) a.tickets[grp] = 0u;                    // ready for the next launch
-  } else {
-#pragma unroll
-    for (int hh = 0; hh < 8; ++hh) {
-      if (hh < G && has_dim) {
-        const float res = L[hh] > 0.f ? o[hh] / L[hh] : 0.f;
-        const float lse_h = L[hh] > 0.f ? (M[hh] + log2f(L[hh])) * kLn2 : -INFINITY;
-        a.out[(long long)(bh0 + hh) * kHeadDim + t] = res;
-        if (t == 0) a.lse[bh0 + hh] = lse_h;
-        if (a.host.out_h != nullptr) a.host.out_h[(long long)(bh0 + hh) * kHeadDim + t] = res;
-        if (a.host.lse_h != nullptr && t == 0) a.host.lse_h[bh0 + hh] = lse_h;
-      }
-    }
-  }
-  if (a.host.done_h != nullptr) {                         // host step: this group's results are in host memory
-    __syncthreads();
-    if (t == 0) host_arrive(a.host);
   }
   SWARM_STAMP_ANY_CTA(status, 6);
   SWARM_KERNEL_END(status, 2);

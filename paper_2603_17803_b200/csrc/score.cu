@@ -166,7 +166,7 @@ page_score_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 // ring full; consumer warp w scores (tile w / 2, head w % 2) of the block that has landed with ldmatrix + mma,
 // stores the tile of scores and counts it on the pair's ticket.  Waits are bounded.
 constexpr int kMmaConsumers = 8;
-constexpr int kMmaThreads = (kMmaConsumers + 2) * 32;      // consumers, the producer warp, the ticket warp
+constexpr int kMmaThreads = (kMmaConsumers + 3) * 32;      // consumers, the producer warp, the ticket warp, the weight warp
 constexpr int kMmaStages = 3;
 constexpr int kMmaPages = 16;                              // pages per tile = M of the MMA tile
 constexpr int kMmaHeadBytes = 4 * kMmaPages * 128;         // one KV head of one tile: 4 boxes' share, 8 KiB
@@ -175,15 +175,21 @@ constexpr int kBlkTiles = kMmaConsumers / kBoxHeads;       // 16-page tiles per 
 constexpr int kBlkPages = kBlkTiles * kMmaPages;           // 64
 constexpr int kTileBytes = kBoxHeads * kMmaHeadBytes;      // one tile of a pair: 4 boxes of 4 KiB
 constexpr int kMmaStageBytes = kBlkTiles * kTileBytes;
-// Sign-split weights of the current request's query heads, bf16 [head][minima part 128 | maxima part 128], kept in
-// shared memory: in pair-by-pair order nearly every block of a CTA belongs to another KV pair, and fetching a
-// pair's weights from global memory per block cost more than the block's arithmetic.  Rows are padded by 16
-// bytes so that the 8 heads a warp reads side by side fall into different banks.
+// Sign-split weights (min(q,0) | max(q,0), bf16) of the query heads of a block's KV pair travel with the block:
+// the producer warp writes them into the ring slot's own weight rows after it has issued the slot's copies, and
+// the slot's `full` barrier counts them as a second arrival.  In pair-by-pair order nearly every block of a CTA
+// belongs to another pair (and, with several requests, to another request); fetching the weights from global
+// memory inside the consumers' loop cost more than the block's arithmetic.  Rows are padded by 16 bytes so that
+// the 8 heads a warp reads side by side fall into different banks.  Pairs with more query heads than fit
+// (groups of more than 8 heads) are fetched by the consumers from global memory.
 constexpr int kWeightRowBytes = 512 + 16;
-constexpr int kWeightRows = 56;                            // query heads that fit; heads beyond them are fetched from global memory
-constexpr int kWeightBytes = kWeightRows * kWeightRowBytes;
-constexpr int kMmaSmemBytes = 1024 + kMmaStages * kMmaStageBytes + kWeightBytes;
-constexpr int kStreamMaxBatch = 1024;                      // requests whose block counts fit the shared prefix table
+constexpr int kWeightRowsMax = 16;                         // 2 KV heads x up to 8 query heads
+__host__ __device__ constexpr int weight_rows(int g) { return 2 * g <= kWeightRowsMax ? 2 * g : 0; }
+__host__ __device__ constexpr int mma_smem_bytes(int g) {
+  return 1024 + kMmaStages * (kMmaStageBytes + weight_rows(g) * kWeightRowBytes);
+}
+constexpr int kStreamMaxBatch = 512;                       // requests whose block counts fit the shared prefix table (2 KiB:
+                                                           // the kernel's shared memory leaves room for a selection CTA beside it)
 constexpr unsigned kStreamWaitLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t sm_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -216,7 +222,8 @@ __device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const in
   return k;
 }
 
-__global__ void __launch_bounds__(kMmaThreads, 1)
+// 128 registers: with 11 warps that leaves room on the SM for a 256-thread selection CTA beside this one.
+__global__ void __maxnreg__(128)
 page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
                       float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready) {
@@ -232,7 +239,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   const int hpairs = head_pairs(geo.Hkv);
   if (tid == 0) {
     for (int sidx = 0; sidx < kMmaStages; ++sidx) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&full[sidx])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&full[sidx])), "r"(2));   // the copies, the weights
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_addr(&empty[sidx])), "r"(kMmaConsumers));
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -276,6 +283,8 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   const int blk_first = (int)blockIdx.x, blk_step = (int)gridDim.x;
   const int n_blk = blk_first < total ? (total - blk_first + blk_step - 1) / blk_step : 0;
 
+  const int w_rows = weight_rows(geo.g);                  // weight rows per ring slot (0: consumers fetch their own)
+  unsigned char* wring = ring + kMmaStages * kMmaStageBytes;
   if (warp == kMmaConsumers) {
     // ---- producer ----
     if (lane == 0) {
@@ -310,6 +319,55 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           }
         }
       }
+    }
+    return;
+  }
+  if (warp == kMmaConsumers + 2) {
+    // ---- weight warp: the second arrival on every slot's `full` barrier ----
+    // weights of the pair's query heads: row r <-> head (first head of the pair) + r; 16 chunks of 8 coordinates.
+    // The rows are fetched into registers before the warp waits for the slot, so the fetch of one block runs
+    // beside the consumers' work on the earlier ones.
+    int fb = 0;
+    for (int k = 0; k < n_blk; ++k) {
+      const int stage = k % kMmaStages;
+      const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+      const int n_chunks = w_rows > 0 ? min(kBoxHeads, geo.Hkv - blk.hp * kBoxHeads) * geo.g * 16 : 0;
+      const uint16_t* qpair = q + ((long long)blk.b * geo.Hq + (long long)blk.hp * kBoxHeads * geo.g) * kHeadDim;
+      uint4 v[kWeightRowsMax * 16 / 32];
+#pragma unroll
+      for (int j = 0; j < kWeightRowsMax * 16 / 32; ++j) {
+        const int i = lane + 32 * j;
+        v[j] = i < n_chunks ? *reinterpret_cast<const uint4*>(qpair + (long long)(i >> 4) * kHeadDim + (i & 15) * 8)
+                            : make_uint4(0u, 0u, 0u, 0u);
+      }
+      int go = 1;
+      if (lane == 0 && k >= kMmaStages) {
+        const unsigned parity = ((k / kMmaStages) - 1) & 1u;
+        unsigned polls = 0;
+        while (!sm_try_wait(&empty[stage], parity) && ++polls < kStreamWaitLimit && !s_abort) {}
+        if (polls >= kStreamWaitLimit || s_abort) go = 0;   // (the producer reports it)
+      }
+      if (!__shfl_sync(0xFFFFFFFFu, go, 0)) break;
+      unsigned char* wst = wring + (size_t)stage * w_rows * kWeightRowBytes;
+#pragma unroll
+      for (int j = 0; j < kWeightRowsMax * 16 / 32; ++j) {
+        const int i = lane + 32 * j;
+        if (i < n_chunks) {
+          const uint32_t in[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+          uint32_t neg[4], pos[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {                     // clamp each bf16 by its sign bit
+            const uint32_t lo = in[e] & 0xFFFFu, hi = in[e] >> 16;
+            neg[e] = ((lo >> 15) ? lo : 0u) | (((hi >> 15) ? hi : 0u) << 16);
+            pos[e] = ((lo >> 15) ? 0u : lo) | (((hi >> 15) ? 0u : hi) << 16);
+          }
+          unsigned char* row = wst + (size_t)(i >> 4) * kWeightRowBytes + (i & 15) * 16;
+          *reinterpret_cast<uint4*>(row) = make_uint4(neg[0], neg[1], neg[2], neg[3]);
+          *reinterpret_cast<uint4*>(row + 256) = make_uint4(pos[0], pos[1], pos[2], pos[3]);
+        }
+      }
+      __syncwarp();                                         // the lanes' rows are ordered before lane 0's arrival
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sm_addr(&full[stage])) : "memory");
     }
     return;
   }
@@ -348,24 +406,10 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   const int tiles = (geo.g + 7) / 8;                        // head tiles of 8 per KV head (N of the MMA)
   uint32_t wb[16][2];                                       // B operand: weights of head `quad`, 16 k-steps
   long long w_key = -1;
-  int cur_b = 0, cached_b = -1;
-  unsigned char* wcache = ring + kMmaStages * kMmaStageBytes;
-  const int n_cached = min(geo.Hq, kWeightRows);
+  int cur_b = 0;
   // weights of head h0 + quad of request b: min(q,0) against the minima (k < 128), max(q,0) against the maxima
-  auto load_weights = [&](int b, int h0, int nh) {
+  auto load_weights_global = [&](int b, int h0, int nh) {
     w_key = (long long)b * geo.Hq + h0;
-    if (h0 + nh <= n_cached) {                              // from the request's rows in shared memory
-      const unsigned char* row = wcache + (size_t)(h0 + (quad < nh ? quad : 0)) * kWeightRowBytes + tq * 4;
-#pragma unroll
-      for (int ks = 0; ks < 16; ++ks) {
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t v = *reinterpret_cast<const uint32_t*>(row + (ks * 16 + half * 8) * 2);
-          wb[ks][half] = quad < nh ? v : 0u;
-        }
-      }
-      return;
-    }
     const uint16_t* qrow = q + (w_key + (quad < nh ? quad : 0)) * kHeadDim;
 #pragma unroll
     for (int ks = 0; ks < 16; ++ks) {
@@ -382,46 +426,35 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       }
     }
   };
-  // All consumer warps walk the same blocks, so they reach a new request together: they rewrite the rows behind
-  // a barrier of their own (the producer warp takes no part).
-  auto cache_request = [&](int b) {
-    asm volatile("bar.sync 1, %0;" ::"n"(kMmaConsumers * 32) : "memory");   // nobody still reads the previous request's rows
-    for (int i = tid; i < n_cached * 64; i += kMmaConsumers * 32) {
-      const int h = i >> 6, c2 = (i & 63) * 2;              // two coordinates per thread
-      const uint32_t pr = *reinterpret_cast<const uint32_t*>(q + ((long long)b * geo.Hq + h) * kHeadDim + c2);
-      const uint32_t lo = pr & 0xFFFFu, hi = pr >> 16;
-      const uint32_t neg = ((lo >> 15) ? lo : 0u) | (((hi >> 15) ? hi : 0u) << 16);
-      const uint32_t pos = ((lo >> 15) ? 0u : lo) | (((hi >> 15) ? 0u : hi) << 16);
-      unsigned char* row = wcache + (size_t)h * kWeightRowBytes;
-      *reinterpret_cast<uint32_t*>(row + c2 * 2) = neg;
-      *reinterpret_cast<uint32_t*>(row + 256 + c2 * 2) = pos;
+  // the same from the ring slot's weight rows (the block's pair; this warp's KV head is row block hl)
+  auto load_weights_slot = [&](int stage, int nh) {
+    const unsigned char* row = wring + ((size_t)stage * w_rows + hl * geo.g + (quad < nh ? quad : 0)) * kWeightRowBytes + tq * 4;
+#pragma unroll
+    for (int ks = 0; ks < 16; ++ks) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(row + (ks * 16 + half * 8) * 2);
+        wb[ks][half] = quad < nh ? v : 0u;
+      }
     }
-    asm volatile("bar.sync 1, %0;" ::"n"(kMmaConsumers * 32) : "memory");
-    cached_b = b;
-    w_key = -1;
   };
-  bool dead = false;                                        // a wait ran out: keep only the consumers' barriers
   for (int k = 0; k < n_blk; ++k) {
     const int stage = k % kMmaStages;
     const ScoreBlock blk = locate_block(blk_first + k * blk_step, cur_b, s_cum, ctx_len, geo.S);
     const int b = blk.b, P = blk.P;
     const int kvh = blk.hp * kBoxHeads + hl;
-    const bool active = !dead && kvh < geo.Hkv && pt < blk.n_tiles;
+    const bool active = kvh < geo.Hkv && pt < blk.n_tiles;
     const int p0 = blk.page0 + pt * kMmaPages;
-    if (b != cached_b) cache_request(b);
-    // the weights of the block's first head tile are fetched before the block has landed
-    if (active && (long long)b * geo.Hq + kvh * geo.g != w_key) load_weights(b, kvh * geo.g, min(8, geo.g));
-    if (!dead) {
+    // without weight rows in the slot: the weights of the block's first head tile are fetched before the block has landed
+    if (w_rows == 0 && active && (long long)b * geo.Hq + kvh * geo.g != w_key) load_weights_global(b, kvh * geo.g, min(8, geo.g));
+    {
       const unsigned parity = (k / kMmaStages) & 1u;
       unsigned polls = 0;
       while (!sm_try_wait(&full[stage], parity) && ++polls < kStreamWaitLimit) __nanosleep(32);
       if (__any_sync(0xFFFFFFFFu, polls >= kStreamWaitLimit || s_abort != 0)) {
         if (lane == 0) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; }
-        dead = true;
-        continue;
+        break;                                              // (the ticket warp stops at the first block left incomplete)
       }
-    } else {
-      continue;
     }
     SWARM_STAMP(status, 3 + 2 * min(k, 4));
     if (active) {
@@ -429,22 +462,35 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + pt * kTileBytes);
       for (int ht = 0; ht < tiles; ++ht) {
         const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
-        if ((long long)b * geo.Hq + h0 != w_key) load_weights(b, h0, nh);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        if (w_rows > 0) load_weights_slot(stage, nh);
+        else if ((long long)b * geo.Hq + h0 != w_key) load_weights_global(b, h0, nh);
+        // A tiles: 16 pages x 16 coordinates per k-step; matrices (rows 0-7 | 8-15) x (chunk 2ks | 2ks+1).  Eight
+        // tiles are fetched before the MMAs that use them, and the MMAs alternate between two accumulators: issued
+        // one by one, every MMA waited for its own ldmatrix and for the MMA before it (~0.5 us per block).
+        float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        const int m = lane >> 3, r = (m & 1) * 8 + (lane & 7);
+        const uint32_t row_base = base + (uint32_t)((r * kBoxHeads + hl) * 128);
+        const int row_sw = (r * kBoxHeads + hl) & 7;
 #pragma unroll
-        for (int ks = 0; ks < 16; ++ks) {
-          // A tile: 16 pages x 16 coordinates; matrices (rows 0-7 | 8-15) x (chunk 2ks | 2ks+1)
-          const int m = lane >> 3, r = (m & 1) * 8 + (lane & 7), cc = 2 * ks + (m >> 1);
-          uint32_t a[4];
-          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
-                       : "r"(base + (uint32_t)((cc >> 3) * (kTileBytes / 4) + (r * kBoxHeads + hl) * 128 +
-                                               (((cc & 7) ^ ((r * kBoxHeads + hl) & 7)) << 4))));
-          asm volatile(
-              "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-              : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
-              : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(wb[ks][0]), "r"(wb[ks][1]));
+        for (int kh = 0; kh < 2; ++kh) {
+          uint32_t a[8][4];
+#pragma unroll
+          for (int k8 = 0; k8 < 8; ++k8) {
+            const int cc = 2 * (kh * 8 + k8) + (m >> 1);
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(a[k8][0]), "=r"(a[k8][1]), "=r"(a[k8][2]), "=r"(a[k8][3])
+                         : "r"(row_base + (uint32_t)((cc >> 3) * (kTileBytes / 4) + (((cc & 7) ^ row_sw) << 4))));
+          }
+#pragma unroll
+          for (int k8 = 0; k8 < 8; ++k8) {
+            float* c = acc2[k8 & 1];
+            asm volatile(
+                "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                : "r"(a[k8][0]), "r"(a[k8][1]), "r"(a[k8][2]), "r"(a[k8][3]), "r"(wb[kh * 8 + k8][0]), "r"(wb[kh * 8 + k8][1]));
+          }
         }
+        const float acc[4] = {acc2[0][0] + acc2[1][0], acc2[0][1] + acc2[1][1], acc2[0][2] + acc2[1][2], acc2[0][3] + acc2[1][3]};
         // C: (page p0 + quad, heads 2tq, 2tq+1), (page p0 + quad + 8, same heads)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -513,7 +559,7 @@ cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* k
   const long long max_blocks = (long long)geo.B * ((geo.Pmax + kBlkPages - 1) / kBlkPages) * head_pairs(geo.Hkv);
   const int sms = std::max(1, g_sm_count - reserve_sms);
   const int grid = (int)std::min<long long>(sms, std::max<long long>(1, max_blocks));
-  return launch_pdl(page_score_mma_kernel, dim3(grid), dim3(kMmaThreads), kMmaSmemBytes, st, true, map, geo, q, page_base,
+  return launch_pdl(page_score_mma_kernel, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q, page_base,
                     ctx_len, scores, status, ready);
 }
 
@@ -526,7 +572,7 @@ cudaError_t configure_score() {
   if (e != cudaSuccess) return e;
   g_sm_count = sms > 0 ? sms : 148;
   if (summary_encode_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
-  return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaSmemBytes);
+  return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
 }
 
 bool score_streams(const Geometry& geo) { return geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31); }

@@ -136,7 +136,7 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
 // Everything the cluster-resolution body needs (see resolve_body.cuh).  sel == nullptr: the flags are already
 // set (by the selection or the expansion kernel) and a single CTA runs the tail.
 // Host-step extension of the fused attention + resolution kernel: the step's small results are also stored
-// into host memory the device can address, and the last of `arrivals` finishing parts (one per attention group,
+// into host memory the device can address, and the last of `arrivals` finishing parts (one per query head,
 // one for the resolution CTA) raises *done_h after a system-wide fence.  All null / zero when unused.
 struct HostMirror {
   float* out_h;
@@ -303,9 +303,12 @@ __device__ __forceinline__ unsigned long long trace_now() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+#ifndef SWARM_TRACE_CTA
+#define SWARM_TRACE_CTA 0
+#endif
 #define SWARM_STAMP_RAW(status, i, any_cta)                                                          \
   do {                                                                                               \
-    if (threadIdx.x == 0 && ((any_cta) || (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)))  \
+    if (threadIdx.x == 0 && ((any_cta) || (blockIdx.x == (SWARM_TRACE_CTA) && blockIdx.y == 0 && blockIdx.z == 0)))  \
       reinterpret_cast<unsigned long long*>(status)[16 + (i)] = trace_now();                         \
   } while (0)
 #endif
