@@ -31,9 +31,6 @@ METRIC = "decode steps/sec of fused select+resolve+gather+attn; HBM GB/s (% of p
 UNIT = "steps/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_kernel launch at the default workload (c2_128k),
-# from the ncu capture summarised in profiles/; reported only for that workload.
-ATTN_TRAFFIC_BYTES_NCU = 33_072_128 + 12_544   # profiles/launch_list_c2_128k.md: dram read + write of attn_kernel<16,paged>
 
 
 def parse_args():
@@ -43,7 +40,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="swarm", choices=["swarm", "reference"])
     ap.add_argument("--workload", default="c2_128k")
-    ap.add_argument("--n-rot", type=int, default=8, help="independent data sets rotated through")
+    ap.add_argument("--n-rot", type=int, default=0, help="independent data sets rotated through (0: enough to exceed 4x the L2)")
+    ap.add_argument("--skip-per-workload", action="store_true", help="only the headline workload")
     ap.add_argument("--no-graph", action="store_true", help="call the library directly instead of replaying graphs")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--attn-splits", type=int, default=0, help="key-range splits of the attention kernel (0: chosen from the shape)")
@@ -155,12 +153,233 @@ def step_bytes(w, sel, n_sel):
 
 # ------------------------------------------------------------------------------------------ swarm arm
 
+WORKLOADS = ("c1_tiny", "c2_128k", "c3_batched", "c4_long", "c5_skewed")
+# most data sets kept resident per workload (device memory: c5 is 33 GiB of pool per data set)
+MAX_DATA_SETS = {"c1_tiny": 48, "c2_128k": 8, "c3_batched": 2, "c4_long": 2, "c5_skewed": 1}
+
+
+def l2_bytes(dev) -> int:
+    import torch
+    return int(torch.cuda.get_device_properties(dev).L2_cache_size)
+
+
+def build_signature() -> str:
+    """Identifies the library that is running: version and a hash of its kernel sources."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2603_17803_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic(workload: str):
+    """dram read + write bytes of one attention launch from the ncu capture summarised under profiles/, if that
+    capture was made from the kernel sources that are running now; (None, why) otherwise."""
+    path = os.path.join(ROOT, "profiles", "attn_traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+    except Exception:
+        return None, "no capture on record"
+    ent = rec.get(workload)
+    if not ent:
+        return None, "no capture on record for this workload"
+    if ent.get("kernel_sources") != build_signature():
+        return None, f"capture of {ent.get('date')} belongs to other kernel sources ({ent.get('kernel_sources')})"
+    return int(ent["dram_bytes_read"]) + int(ent["dram_bytes_write"]), f"ncu capture of {ent.get('date')}, same kernel sources"
+
+
+class Bench:
+    """The data sets, sessions and graphs of one workload, and the timed loops over them."""
+
+    def __init__(self, name, n_rot, rank, dev, stream, tail_stream, attn_splits=0, no_graph=False):
+        import torch
+        from paper_2603_17803_b200 import binding as B
+        from paper_2603_17803_b200 import replicas
+        from paper_2603_17803_b200 import workloads as W
+        from paper_2603_17803_b200.session import Session
+        self.torch, self.B = torch, B
+        self.cfg = W.CONFIGS[name]
+        self.n_rot, self.stream, self.tail_stream, self.no_graph = n_rot, stream, tail_stream, no_graph
+        self.workloads, self.serial, self.tail = [], [], []
+        for r in range(n_rot):      # every rank draws its own data sets (weak scaling: fixed work per GPU)
+            w = W.generate(self.cfg, seed=replicas.replica_seed(rank, r), device=dev, step=r)
+            self.workloads.append(w)
+            a = Session(w)
+            b = Session(w, ksum=a.ksum, tail_stream=tail_stream)
+            for s_ in (a, b):
+                if attn_splits > 0:
+                    B.swarm_set_attn_splits(s_.ctx, attn_splits)
+            self.serial.append(a)
+            self.tail.append(b)
+        torch.cuda.synchronize()
+
+    def close(self):
+        for s in self.serial + self.tail:
+            s.close()
+
+    def _graph(self, sessions, fn, n_calls, join):
+        """A CUDA graph of n_calls consecutive calls, data sets in rotation (None with --no-graph or n_calls 0)."""
+        torch = self.torch
+        if self.no_graph or n_calls == 0:
+            return None
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=self.stream):
+            for i in range(n_calls):
+                fn(sessions[i % self.n_rot])
+            if join:
+                for s in sessions:
+                    s.tail_join(self.stream)
+        return g
+
+    def time_calls(self, sessions, fn, n_calls, *, join=False, warmup=0, min_ms=50.0, max_repeats=200, barrier=None):
+        """Device time of exactly n_calls consecutive calls (CUDA events on the launching stream), repeated
+        until min_ms of timed work has accumulated; returns (median, min, max) microseconds per call and the
+        number of repeats.  Whole rotations go out as one graph launch each, the remainder as one more."""
+        torch, stream, n_rot = self.torch, self.stream, self.n_rot
+        with torch.cuda.stream(stream):
+            for s in sessions:
+                fn(s)
+            if join:
+                for s in sessions:
+                    s.tail_join(stream)
+            stream.synchronize()
+            # up to 512 calls: the whole region is one graph; beyond that, graphs of 8 rotations and a remainder
+            per_graph = n_calls if n_calls <= 512 else n_rot * 8
+            g_full = self._graph(sessions, fn, per_graph, join)
+            g_rem = self._graph(sessions, fn, n_calls % per_graph, join)
+
+            def run():
+                if self.no_graph:
+                    for i in range(n_calls):
+                        fn(sessions[i % n_rot])
+                    if join:
+                        for s in sessions:
+                            s.tail_join(stream)
+                    return
+                for _ in range(n_calls // per_graph):
+                    g_full.replay()
+                if g_rem is not None:
+                    g_rem.replay()
+
+            for _ in range(max(1, -(-warmup // max(1, n_calls)))):
+                run()
+            times, total = [], 0.0
+            while True:
+                if barrier is not None:
+                    barrier()
+                stream.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                run()
+                e1.record(stream)
+                if barrier is not None:
+                    barrier()
+                stream.synchronize()
+                ms = e0.elapsed_time(e1)
+                times.append(ms)
+                total += ms
+                if total >= min_ms or len(times) >= max_repeats:
+                    break
+        times.sort()
+        per = [t * 1e3 / n_calls for t in times]
+        return per[len(per) // 2], per[0], per[-1], len(per)
+
+
+def measure_workload(name, args, rank, dev, stream, tail_stream, peak, *, steps, warmup, barrier=None, extras=False):
+    """Everything reported for one workload: step time (strictly serial and with the overlapped tail), the stages
+    alone, bytes and roofline fractions.  `extras`: also the step variants and the medoid-index step."""
+    import torch
+    from paper_2603_17803_b200 import binding as B
+    cfg_probe = __import__("paper_2603_17803_b200.workloads", fromlist=["CONFIGS"]).CONFIGS[name]
+    l2 = l2_bytes(dev)
+    n_rot = args.n_rot if (args.n_rot and name == args.workload) else None
+    # first guess of the bytes a step touches: summaries + half of the nominal K/V
+    S, d, Hkv = cfg_probe.page_size, cfg_probe.head_dim, cfg_probe.n_kv_heads
+    pages = cfg_probe.batch * (cfg_probe.max_pages() if not cfg_probe.ctx_range else (cfg_probe.ctx_range[0] + cfg_probe.ctx_range[1]) // (2 * S))
+    guess = pages * Hkv * 2 * d * 2 + cfg_probe.batch * cfg_probe.n_q_heads * cfg_probe.top_k * S * d * 2
+    if n_rot is None:
+        n_rot = max(2 if guess < 4 * l2 else 1, min(MAX_DATA_SETS[name], -(-4 * l2 // max(1, guess))))
+    bench = Bench(name, n_rot, rank, dev, stream, tail_stream, args.attn_splits, args.no_graph)
+    cfg = bench.cfg
+    step = lambda s: s.step(stream=stream)
+    kw = dict(warmup=warmup, barrier=barrier)
+    t_a = time.perf_counter()
+    tail_us, tail_min, tail_max, tail_reps = bench.time_calls(bench.tail, step, steps, join=True, **kw)
+    serial_us, serial_min, serial_max, serial_reps = bench.time_calls(bench.serial, step, steps, **kw)
+    t_b = time.perf_counter()
+    n_loop = max(3 * n_rot, min(steps, 2000))
+    attn_us = bench.time_calls(bench.serial, lambda s: s.sparse_attn_paged(stream=stream, reuse_last_selection=True), n_loop)[0]
+    select_us = bench.time_calls(bench.serial, lambda s: s.select(stream=stream), n_loop)[0]
+    resolve_us = bench.time_calls(bench.serial, lambda s: s.resolve(stream=stream), n_loop)[0]
+    for s_ in bench.serial:
+        s_.step(stream=stream)                            # leave a whole step's outputs in place
+    torch.cuda.synchronize()
+    status = max(s.status() for s in bench.serial + bench.tail)
+    by = step_bytes(bench.workloads[0], bench.serial[0].o.sel, bench.serial[0].o.n_sel)
+    alg = by["summaries"] + by["kv_compulsory"] + by["small"]
+    nominal = by["summaries"] + by["kv_nominal"] + by["small"]
+    attn_gbs = by["kv_compulsory"] / (attn_us * 1e-6) / 1e9
+    out = {
+        "workload": cfg.name, "us_per_step": tail_us, "us_per_step_min_max": [tail_min, tail_max], "repeats": tail_reps,
+        "us_per_step_serial": serial_us, "us_per_step_serial_min_max": [serial_min, serial_max],
+        "best_mode": "overlapped tail" if tail_us <= serial_us else "serial",
+        "steps_timed": steps, "data_sets": n_rot,
+        "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
+        "hbm_gbs": alg / (tail_us * 1e-6) / 1e9,
+        "hbm_frac_of_measured_copy": alg / (tail_us * 1e-6) / 1e9 / peak,
+        "hbm_frac_of_nominal_8tbs": alg / (tail_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+        "nominal_bytes_frac_of_nominal_8tbs": nominal / (tail_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+        "serial_hbm_frac_of_measured_copy": alg / (serial_us * 1e-6) / 1e9 / peak,
+        "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
+        "attention_alone": {"gbs_of_compulsory_kv": attn_gbs, "frac_of_measured_copy": attn_gbs / peak, "us": attn_us},
+        "l2_policy": f"rotating {n_rot} independent data sets ({n_rot * alg / 1e6:.0f} MB touched per rotation, "
+                     f"L2 {l2 / 1e6:.0f} MB)" if n_rot > 1 else
+                     f"one data set: a step touches {alg / 1e6:.0f} MB, {alg / l2:.0f}x the {l2 / 1e6:.0f} MB L2",
+        "device_status": status, "n_uniq_clusters": int(bench.serial[0].o.n_uniq[0]),
+        "_windows": [(t_a, t_b)],
+    }
+    if cfg.n_layers > 1:
+        out["note"] = (f"one layer-step; the configuration's step is {cfg.n_layers} sequential layers = "
+                       f"{tail_us * cfg.n_layers / 1e3:.3f} ms")
+    if extras:
+        # the same step with the paper's own selector (medoid index, whole clusters retrieved): k_c clusters of
+        # ~8 pages stand for the page step's top_k pages
+        k_c = max(1, cfg.top_k // 8)
+        for s_ in bench.serial:
+            s_.enable_medoid_index(k_c)
+        medoid_us = bench.time_calls(bench.serial, lambda s: s.step_medoid(stream=stream), n_loop)[0]
+        # the page step with the optional parts of cluster resolution switched on, one at a time
+        keep = []
+        for s_ in bench.serial:
+            n_c = s_.w.n_clusters
+            g_ = torch.Generator(device="cpu").manual_seed(7)
+            keep.append(dict(resident=(torch.rand(n_c, generator=g_) < 0.25).to(torch.uint8).to(dev),
+                             freq=torch.zeros(n_c, dtype=torch.int32, device=dev),
+                             score=torch.zeros(n_c, dtype=torch.float32, device=dev),
+                             n_hit=torch.zeros(4, dtype=torch.int32, device=dev)))
+            B.swarm_set_cache(s_.ctx, t_base=80.0, t_transfer=2.5, **keep[-1])
+        cached_us = bench.time_calls(bench.serial, step, n_loop)[0]
+        for s_ in bench.serial:
+            B.swarm_set_cache(s_.ctx)
+            s_.enable_submit_order()
+        submit_us = bench.time_calls(bench.serial, step, n_loop)[0]
+        for s_ in bench.serial:
+            B.swarm_set_submit_order(s_.ctx, None, None)
+            s_.step(stream=stream)
+        torch.cuda.synchronize()
+        out["step_variants_us"] = {"with_cache_state(25% resident: Eq. 8 filter, counters, Eq. 6)": cached_us,
+                                   "with_submission_order(Sec. 5.1 batches)": submit_us}
+        out["medoid_step"] = {"us_per_step": medoid_us, "top_k_clusters": k_c,
+                              "note": "swarm_step_medoid on the same data sets: clusters scored by their medoid page, whole clusters attended"}
+    return out, bench
+
+
 def run_swarm(args):
     import torch
     from paper_2603_17803_b200 import replicas
-    from paper_2603_17803_b200 import workloads as W
-    from paper_2603_17803_b200.session import Session
-    from paper_2603_17803_b200 import binding as B
 
     world, rank, local_rank = replicas.env_world()
     if not torch.cuda.is_available():
@@ -169,203 +388,124 @@ def run_swarm(args):
     dev = torch.device("cuda", local_rank)
     replicas.init("nccl", dev)
     K = args.steps if args.steps is not None else 20000
-    Wm = args.warmup if args.warmup is not None else 50
-    cfg = W.CONFIGS[args.workload]
+    Wm = max(3, args.warmup if args.warmup is not None else 50)
+    peak, peak_kind = measured_peak()
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-
-    # independent data sets; every rank draws its own (weak scaling: fixed work per GPU)
-    sessions, workloads = [], []
-    for r in range(args.n_rot):
-        w = W.generate(cfg, seed=replicas.replica_seed(rank, r), device=dev, step=r)
-        workloads.append(w)
-        sessions.append(Session(w))
-        if args.attn_splits > 0:
-            B.swarm_set_attn_splits(sessions[-1].ctx, args.attn_splits)
-    torch.cuda.synchronize()
-    stream = torch.cuda.Stream()
+    stream, tail_stream = torch.cuda.Stream(), torch.cuda.Stream()
 
     def barrier():
         replicas.barrier()
         torch.cuda.synchronize()
 
-    graphs = []
-    cycle_graph = None
+    head, bench = measure_workload(args.workload, args, rank, dev, stream, tail_stream, peak, steps=K, warmup=Wm,
+                                   barrier=barrier, extras=True)
+    cfg = bench.cfg
+    windows = head.pop("_windows")
+
+    # end to end: per-step data in pinned host memory, copies inside the timed region
+    Bq, Hq, d, D = cfg.batch, cfg.n_q_heads, cfg.head_dim, cfg.n_queues
+    q_host = [w.q.cpu().pin_memory() for w in bench.workloads]
+    out_host = torch.empty((Bq, Hq, d), dtype=torch.float32).pin_memory()
+    lse_host = torch.empty((Bq, Hq), dtype=torch.float32).pin_memory()
+    n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    load_host = torch.zeros(D, dtype=torch.int32).pin_memory()
+    K_e2e = max(200, min(K, 5000))
+    sessions, n_rot = bench.serial, bench.n_rot
     with torch.cuda.stream(stream):
-        for s in sessions:
-            s.step(stream=stream)
-        stream.synchronize()
-        if not args.no_graph:
-            for s in sessions:
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    s.step(stream=stream)
-                graphs.append(g)
-            # one graph holding a whole rotation (n_rot consecutive steps): one launch per n_rot steps
-            cycle_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(cycle_graph, stream=stream):
-                for s in sessions:
-                    s.step(stream=stream)
-
-        def one_step(i):
-            if graphs:
-                graphs[i % args.n_rot].replay()
-            else:
-                sessions[i % args.n_rot].step(stream=stream)
-
-        def run_steps(n):
-            """Exactly n steps, rotating over the data sets; whole rotations go out as one graph launch."""
-            i = 0
-            if cycle_graph is not None:
-                for _ in range(n // args.n_rot):
-                    cycle_graph.replay()
-                i = n - n % args.n_rot
-            for j in range(i, n):
-                one_step(j)
-
-        run_steps(Wm)
-        barrier()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t_a = time.perf_counter()
-        ev0.record(stream)
-        run_steps(K)
-        ev1.record(stream)
-        barrier()
-        t_b = time.perf_counter()
-        ms = ev0.elapsed_time(ev1)
-
-        # the dominant kernel (attention straight from the pool) and the other stages timed alone: one graph
-        # holds one call per data set (so the host's launch cost is off the clock), replayed back to back
-        def time_loop(fn, n):
-            for s_ in sessions:
-                fn(s_)
-            stream.synchronize()
-            if args.no_graph:
-                def go():
-                    for s_ in sessions:
-                        fn(s_)
-            else:
-                g_ = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g_, stream=stream):
-                    for s_ in sessions:
-                        fn(s_)
-                go = g_.replay
-            reps = max(1, n // args.n_rot)
-            go()
-            stream.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(reps):
-                go()
-            e1.record(stream)
-            stream.synchronize()
-            return e0.elapsed_time(e1) / (reps * args.n_rot) * 1e3    # microseconds per call
-
-        n_loop = max(3 * args.n_rot, min(K, 2000))
-        t_c = time.perf_counter()
-        attn_us = time_loop(lambda s: s.sparse_attn_paged(stream=stream, reuse_last_selection=True), n_loop)
-        select_us = time_loop(lambda s: s.select(stream=stream), n_loop)
-        resolve_us = time_loop(lambda s: s.resolve(stream=stream), n_loop)
-        # the same step with the paper's own selector (medoid index, whole clusters retrieved): k_c clusters of
-        # ~8 pages stand for the page step's top_k pages
-        k_c = max(1, cfg.top_k // 8)
-        for s_ in sessions:
-            s_.enable_medoid_index(k_c)
-        medoid_us = time_loop(lambda s: s.step_medoid(stream=stream), n_loop)
-        # the page step with the optional parts of cluster resolution switched on, one at a time
-        cache_state = []
-        for s_ in sessions:
-            n_c = s_.w.n_clusters
-            g_ = torch.Generator(device="cpu").manual_seed(7)
-            cache_state.append(dict(resident=(torch.rand(n_c, generator=g_) < 0.25).to(torch.uint8).to(dev),
-                                    freq=torch.zeros(n_c, dtype=torch.int32, device=dev),
-                                    score=torch.zeros(n_c, dtype=torch.float32, device=dev),
-                                    n_hit=torch.zeros(4, dtype=torch.int32, device=dev)))
-            B.swarm_set_cache(s_.ctx, t_base=80.0, t_transfer=2.5, **cache_state[-1])
-        cached_us = time_loop(lambda s: s.step(stream=stream), n_loop)
-        for s_ in sessions:
-            B.swarm_set_cache(s_.ctx)
-            s_.enable_submit_order()
-        submit_us = time_loop(lambda s: s.step(stream=stream), n_loop)
-        for s_ in sessions:
-            B.swarm_set_submit_order(s_.ctx, None, None)
-            s_.step(stream=stream)                       # leave the plain page step's outputs in place for the checks below
-        stream.synchronize()
-        t_d = time.perf_counter()
-
-        # end to end: per-step data in pinned host memory, copies inside the timed region
-        B, Hq, d, D = cfg.batch, cfg.n_q_heads, cfg.head_dim, cfg.n_queues
-        q_host = [w.q.cpu().pin_memory() for w in workloads]
-        out_host = torch.empty((B, Hq, d), dtype=torch.float32).pin_memory()
-        lse_host = torch.empty((B, Hq), dtype=torch.float32).pin_memory()
-        n_host = torch.zeros(1, dtype=torch.int32).pin_memory()
-        load_host = torch.zeros(D, dtype=torch.int32).pin_memory()
-        K_e2e = min(K, 5000)
-        for i in range(min(Wm, 20)):
-            sessions[i % args.n_rot].step_host(q_host[i % args.n_rot], out_host, lse_host, n_host, load_host, stream)
+        for i in range(20):
+            sessions[i % n_rot].step_host(q_host[i % n_rot], out_host, lse_host, n_host, load_host, stream)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_e = time.perf_counter()
         e0.record(stream)
         for i in range(K_e2e):
-            sessions[i % args.n_rot].step_host(q_host[i % args.n_rot], out_host, lse_host, n_host, load_host, stream)
+            sessions[i % n_rot].step_host(q_host[i % n_rot], out_host, lse_host, n_host, load_host, stream)
         e1.record(stream)
         barrier()
         t_f = time.perf_counter()
         ms_e2e = e0.elapsed_time(e1)
-    sampler.stop()
+    windows.append((t_e, t_f))
 
-    ms, ms_e2e = replicas.max_over_ranks([ms, ms_e2e], device=dev)
-
-    status = max(s.status() for s in sessions)
-    by = step_bytes(workloads[0], sessions[0].o.sel, sessions[0].o.n_sel)
-    peak, peak_kind = measured_peak()
-    step_s = ms / 1e3 / K
-    alg = by["summaries"] + by["kv_compulsory"] + by["small"]
-    nominal = by["summaries"] + by["kv_nominal"] + by["small"]
-    hbm_gbs = alg / step_s / 1e9
-    attn_alg = by["kv_compulsory"]
-    attn_gbs = attn_alg / (attn_us * 1e-6) / 1e9
-
+    us, us_serial, ms_e2e = replicas.max_over_ranks([head["us_per_step"], head["us_per_step_serial"], ms_e2e], device=dev)
+    ms = us * K / 1e3
+    by = head["bytes_per_step"]
+    traffic, traffic_source = captured_traffic(cfg.name)
+    attn = head["attention_alone"]
     result = {
-        "metric": METRIC, "value": replicas.aggregate_steps_per_s(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
+        "metric": METRIC, "value": replicas.aggregate_steps_per_s(world, K, ms), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": Wm, "ms_per_step": us / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": cfg.batch, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
                    "head_dim": cfg.head_dim, "context": cfg.max_ctx(), "page_size": cfg.page_size,
                    "top_k": cfg.top_k, "n_queues": cfg.n_queues, "n_topics": cfg.n_topics,
                    "parallelism": f"replicas x{world} (no data-path collective)",
-                   "l2_policy": f"rotating {args.n_rot} independent data sets "
-                                f"({args.n_rot * alg / 1e6:.0f} MB touched per rotation > 126 MB L2)",
-                   "launch": "library call" if args.no_graph else
-                             f"CUDA graph replay: {args.n_rot} consecutive swarm_step calls per graph, executed one after another"},
-        "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
-        "bytes_per_step": {"algorithmic": alg, "nominal": nominal, **by},
-        "stage_us_alone": {"select(score+topk)": select_us, "resolve": resolve_us, "attention_paged(+combine)": attn_us},
-        "step_variants_us": {"with_cache_state(25% resident: Eq. 8 filter, counters, Eq. 6)": cached_us,
-                             "with_submission_order(Sec. 5.1 batches)": submit_us},
-        "medoid_step": {"us_per_step": medoid_us, "top_k_clusters": k_c,
-                        "note": "swarm_step_medoid on the same data sets: clusters scored by their medoid page, whole clusters attended"},
-        "roofline": {"kernel": "attn_kernel<paged> (tensor-core split-K attention over the union of selected pages, merge included)", "bound": "hbm", "achieved": attn_gbs,
-                     "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
-                     "frac": attn_gbs / peak, "traffic": ATTN_TRAFFIC_BYTES_NCU if cfg.name == "c2_128k" else None,
-                     "algorithmic_bytes_per_launch": attn_alg, "avg_launch_us": attn_us,
-                     "nominal_bytes_per_launch": by["kv_nominal"], "nominal_gbs": by["kv_nominal"] / (attn_us * 1e-6) / 1e9},
+                   "l2_policy": head["l2_policy"],
+                   "launch": "library calls, no graph" if args.no_graph else
+                             "CUDA graph replay of consecutive swarm_step calls (whole rotations of the data sets per graph). "
+                             "value: overlapped tail (swarm_set_tail_stream) -- scoring, selection and attention of a step "
+                             "run strictly after the attention of the step before; only the cluster resolution of a step "
+                             "(uniq / queue_of / loads: the I/O schedule) runs beside the next step's scoring and selection, "
+                             "every output of every step is computed and the graph joins the tail stream. "
+                             "serial: the same steps with the resolution inside the step (nothing overlaps)",
+                   "timing": f"exactly {K} steps per timed region (CUDA events on the launching stream, max over ranks); the region "
+                             f"is repeated until 50 ms have been timed and the median is reported ({head['repeats']} repeats here)"},
+        "serial": {"value": replicas.aggregate_steps_per_s(world, K, us_serial * K / 1e3), "unit": UNIT, "us_per_step": us_serial,
+                   "hbm_frac_of_measured_copy": head["serial_hbm_frac_of_measured_copy"]},
+        "us_per_step_min_max": head["us_per_step_min_max"],
+        "hbm_gbs": head["hbm_gbs"], "hbm_frac_of_measured_copy": head["hbm_frac_of_measured_copy"],
+        "hbm_frac_of_nominal_8tbs": head["hbm_frac_of_nominal_8tbs"],
+        "nominal_bytes_frac_of_nominal_8tbs": head["nominal_bytes_frac_of_nominal_8tbs"],
+        "bytes_per_step": by,
+        "stage_us_alone": head["stage_us_alone"],
+        "step_variants_us": head.get("step_variants_us"), "medoid_step": head.get("medoid_step"),
+        "roofline": {"kernel": "attn_kernel<paged> (tensor-core split-K attention over the union of selected pages, merge included)",
+                     "bound": "hbm", "achieved": attn["gbs_of_compulsory_kv"], "peak": peak,
+                     "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s", "frac": attn["frac_of_measured_copy"],
+                     "traffic": traffic, "traffic_source": traffic_source,
+                     "algorithmic_bytes_per_launch": by["kv_compulsory"], "avg_launch_us": attn["us"],
+                     "nominal_bytes_per_launch": by["kv_nominal"], "nominal_gbs": by["kv_nominal"] / (attn["us"] * 1e-6) / 1e9},
         "e2e": {"value": replicas.aggregate_steps_per_s(world, K_e2e, ms_e2e), "unit": UNIT, "steps": K_e2e,
-                "h2d_bytes_per_step": B * Hq * d * 2, "d2h_bytes_per_step": B * Hq * d * 4 + B * Hq * 4 + 4 + D * 4,
+                "h2d_bytes_per_step": Bq * Hq * d * 2, "d2h_bytes_per_step": Bq * Hq * d * 4 + Bq * Hq * 4 + 4 + D * 4,
                 "note": "swarm_step_host: q from pinned host memory, out/lse/n_uniq/queue_load read back; "
                         "the KV pool and its summaries are resident state, like weights"},
-        "gpu_launches": K * 3,   # scorer, selection, attention + cluster resolution
-        "gpu_launches_per_step": 3,
-        "device_status": status,
-        "n_uniq_clusters": int(sessions[0].o.n_uniq[0]),
-        "clocks": sampler.summary([(t_a, t_b), (t_e, t_f)]),
+        "gpu_launches": K * 4,   # scorer, selection, cluster resolution (tail stream), attention
+        "gpu_launches_per_step": 4,
+        "device_status": head["device_status"],
+        "n_uniq_clusters": head["n_uniq_clusters"],
+        "kernel_sources": build_signature(),
     }
+    cpu = None
     if rank == 0 and not args.skip_cpu_baseline and world == 1:
-        result["cpu_baseline"] = cpu_baseline(workloads[0], budget_s=12.0)
-    for s in sessions:
-        s.close()
+        cpu = cpu_baselines(bench.workloads[0], budget_s=6.0)
+        result["cpu_baseline"] = cpu["all_cores"]
+        result["cpu_baseline_one_thread"] = cpu["one_thread"]
+    bench.close()
+    del bench
+    torch.cuda.empty_cache()
+
+    # the other workloads, shorter runs (one GPU, rank 0's numbers; every rank runs them so the ranks stay in step)
+    if not args.skip_per_workload:
+        per = {}
+        for name in WORKLOADS:
+            if name == cfg.name:
+                ent = {k: v for k, v in head.items() if not k.startswith("_")}
+                if cpu is not None:
+                    ent["cpu_baseline"] = cpu
+            else:
+                short = {"c1_tiny": 2000, "c3_batched": 400, "c4_long": 200, "c5_skewed": 60}.get(name, 400)
+                ent, b2 = measure_workload(name, args, rank, dev, stream, tail_stream, peak, steps=short, warmup=max(3, short // 20))
+                windows += ent.pop("_windows")
+                if rank == 0 and not args.skip_cpu_baseline and world == 1:
+                    ent["cpu_baseline"] = cpu_baselines(b2.workloads[0], budget_s=4.0)
+                b2.close()
+                del b2
+                torch.cuda.empty_cache()
+            per[name] = ent
+        result["per_workload"] = per
+    sampler.stop()
+    result["clocks"] = sampler.summary(windows)
     if rank == 0:
         print(json.dumps(result))
     replicas.shutdown()
@@ -389,30 +529,59 @@ def oracle_step_fn(w):
     x = oracle_inputs(w)
     ksum = oracle.build_summaries(x["kv_pool"], x["page_base"], x["ctx_len"], cfg.n_kv_heads, cfg.head_dim,
                                   cfg.page_size)   # index build: outside the timed step, as on the GPU
+    Pmax = int((-(-x["ctx_len"].astype("int64") // cfg.page_size)).max())
 
     def fn():
         return oracle.step(x["q"], ksum, x["kv_pool"], x["page_base"], x["ctx_len"], x["page2cluster"],
                            x["cluster_base"], x["replica_mask"], x["cluster_size"], Hkv=cfg.n_kv_heads,
-                           S=cfg.page_size, k=cfg.top_k, D=cfg.n_queues, Pmax=cfg.max_pages())
+                           S=cfg.page_size, k=cfg.top_k, D=cfg.n_queues, Pmax=Pmax)
     return fn
 
 
-def cpu_baseline(w, budget_s: float):
-    """The oracle as it stands, on this host's cores, on whole steps of the same workload."""
+def oracle_sample(w, max_bytes=3 << 30):
+    """(sample workload on the host, scale, description): the whole batch when its pool fits max_bytes, else
+    requests picked evenly over the batch sorted by length -- a step of the whole batch costs `scale` times the
+    sample's step (the oracle's stages are per request, except the cluster assignment, which is a small part)."""
+    import numpy as np
+    from paper_2603_17803_b200 import workloads as W
+    cfg = w.cfg
+    pages = (w.page_base[1:] - w.page_base[:-1]).cpu().numpy()
+    per_page = cfg.n_kv_heads * 2 * cfg.page_size * cfg.head_dim * 2
+    order = np.argsort(pages, kind="stable")
+    n = cfg.batch
+    while n > 1 and pages[order[np.linspace(0, cfg.batch - 1, n).round().astype(int)]].sum() * per_page > max_bytes:
+        n -= 1
+    pick = sorted(set(int(order[i]) for i in np.linspace(0, cfg.batch - 1, n).round().astype(int)))
+    if len(pick) == cfg.batch:
+        return W.subset_requests(w, range(cfg.batch)), 1.0, f"all {cfg.batch} requests"
+    scale = float(pages.sum()) / float(pages[pick].sum())
+    return (W.subset_requests(w, pick), scale,
+            f"requests {pick} of {cfg.batch} (evenly spaced by length), time scaled by pages {scale:.2f}x")
+
+
+def cpu_baselines(w, budget_s: float):
+    """The oracle as it stands on this host's cores, on (a sample of) the same workload: whole steps at one
+    thread and at all cores."""
     import oracle
-    cores = oracle.set_threads(0)
-    fn = oracle_step_fn(w)
-    fn()
-    n, t0 = 0, time.perf_counter()
-    while True:
+    sample, scale, what = oracle_sample(w)
+    fn = oracle_step_fn(sample)
+    out = {}
+    n_cores = len(os.sched_getaffinity(0))
+    for key, threads in (("all_cores", n_cores), ("one_thread", 1)):
+        cores = oracle.set_threads(threads)
         fn()
-        n += 1
-        el = time.perf_counter() - t0
-        if el >= budget_s or n >= 1000:
-            break
-    return {"value": n / el, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{n} whole steps of {w.cfg.name} (all {w.cfg.batch * w.cfg.n_q_heads} heads), "
-                      f"OpenMP over (request, head) units, {el:.1f} s"}
+        n, t0 = 0, time.perf_counter()
+        while True:
+            fn()
+            n += 1
+            el = time.perf_counter() - t0
+            if el >= budget_s or n >= 1000:
+                break
+        out[key] = {"value": n / (el * scale), "unit": UNIT, "cores": cores, "kind": "oracle",
+                    "sample": f"{n} oracle steps over {what} of {w.cfg.name} (all {w.cfg.n_q_heads} heads), "
+                              f"OpenMP over (request, head) units, {el:.1f} s"}
+    oracle.set_threads(n_cores)
+    return out
 
 
 def run_sharded(args):
@@ -433,10 +602,11 @@ def run_sharded(args):
     K = args.steps if args.steps is not None else 5000
     Wm = max(3, args.warmup if args.warmup is not None else 50)
     cfg = W.CONFIGS[args.workload]
+    n_rot = args.n_rot or 8
     sampler = ClockSampler(local_rank)
     sampler.start()
     sessions = []
-    for r in range(args.n_rot):                             # the same data sets on every rank, each keeps its heads
+    for r in range(n_rot):                             # the same data sets on every rank, each keeps its heads
         w = W.generate(cfg, seed=r, device=dev, step=r)
         sessions.append(Session(sharding.shard_workload(w, rank, world)))
         del w
@@ -444,14 +614,14 @@ def run_sharded(args):
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         for i in range(Wm):
-            sharding.sharded_step(sessions[i % args.n_rot], stream)
+            sharding.sharded_step(sessions[i % n_rot], stream)
         replicas.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_a = time.perf_counter()
         e0.record(stream)
         for i in range(K):
-            sharding.sharded_step(sessions[i % args.n_rot], stream)
+            sharding.sharded_step(sessions[i % n_rot], stream)
         e1.record(stream)
         replicas.barrier()
         torch.cuda.synchronize()
@@ -468,7 +638,7 @@ def run_sharded(args):
             "data": "synthetic",
             "config": {"workload": cfg.name, "parallelism": f"kv-head shards x{world}: one all-reduce(max) of {n_flags} "
                                                              "cluster-flag bytes per step, every rank schedules the union",
-                       "l2_policy": f"rotating {args.n_rot} independent data sets", "launch": "plain launches, no graph"},
+                       "l2_policy": f"rotating {n_rot} independent data sets", "launch": "plain launches, no graph"},
             "gpu_launches": K * 3, "device_status": status, "clocks": sampler.summary([(t_a, t_b)])}))
     replicas.shutdown()
 
@@ -484,7 +654,7 @@ def run_reference(args):
     K = args.steps if args.steps is not None else 5
     Wm = args.warmup if args.warmup is not None else 1
     w = W.generate(cfg, seed=0, device="cpu")
-    cores = oracle.set_threads(0)
+    cores = oracle.set_threads(len(os.sched_getaffinity(0)))
     fn = oracle_step_fn(w)
     t0 = time.perf_counter()
     fn()

@@ -276,15 +276,27 @@ __device__ __forceinline__ void finish_by_ranking(SelectState& st, int tid, int 
 // ---- register-resident variant -------------------------------------------------------------------
 // The selection of one list with ITEMS consecutive pages per thread (the kernel was launched for lists of up to
 // THREADS * MAX_ITEMS pages; rows of the page bitmap are that long).
-template <int THREADS, int ITEMS, int MAX_ITEMS>
-__device__ __forceinline__ void topk_regs_body(SelectState& st, const Geometry& geo, const TopkExtras& x,
+template <int THREADS, int ITEMS, int MAX_ITEMS, bool kEarly>
+__device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& geo, const TopkExtras& x,
                                                const RequestBases& rb, const float* __restrict__ s,
                                                int32_t* __restrict__ out, int32_t* __restrict__ n_sel,
-                                               uint32_t* __restrict__ status, int bh, int P, int Pw, int k_eff, int k_sel) {
+                                               uint32_t* __restrict__ status, int bh, int b, int kvh, int len_b, bool* s_flag,
+                                               int P, int Pw, int k_eff, int k_sel) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // thread t owns pages [t*ITEMS, (t+1)*ITEMS); keys of pages that do not exist are never used
   uint32_t key[ITEMS];
   const int p0 = tid * ITEMS;
+  // The clusters of this thread's pages: an input table, read while the scores are still being written, so that
+  // marking the selected pages' clusters later costs no memory round trip.
+  // (Only with few lists: all heads of a request read the same entries, and with thousands of lists that is
+  // hundreds of megabytes of cache traffic for the one page in 30-60 that ends up selected.)
+  int cl[kEarly ? ITEMS : 1];
+  if (kEarly && x.flags != nullptr) {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) cl[j] = p0 + j < P ? x.page2cluster[rb.pb + p0 + j] : -1;
+  }
+  if (!scores_ready(geo, x, b, kvh, len_b, s_flag)) return false;   // the scores come from the previous kernel
+  SWARM_STAMP(status, 1);
   const bool full = p0 + ITEMS <= Pw;                       // all of this thread's pages exist and are scored: no per-page checks
   if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
 #pragma unroll
@@ -403,7 +415,16 @@ __device__ __forceinline__ void topk_regs_body(SelectState& st, const Geometry& 
     if (ITEMS == 8) *row = (uint8_t)picked;
     else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
   }
-  if (x.flags != nullptr) {
+  if (kEarly && x.flags != nullptr) {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) {
+      if ((picked >> j) & 1u) {
+        const int c = cl[kEarly ? j : 0];
+        if (c < 0 || c >= rb.cn - rb.cb || rb.cb + c >= geo.Cmax) atomicOr(x.status, SWARM_DEV_BAD_CLUSTER);
+        else x.flags[rb.cb + c] = 1;
+      }
+    }
+  } else if (x.flags != nullptr) {
     // four selected pages at a time: all the table reads first, then the flag stores -- a byte store may alias
     // anything, so interleaving them would make every read wait for the store before it
     for (unsigned todo = picked; todo != 0u;) {
@@ -433,9 +454,10 @@ __device__ __forceinline__ void topk_regs_body(SelectState& st, const Geometry& 
       *reinterpret_cast<uint32_t*>(row + o) = 0u;
   }
   SWARM_STAMP(status, 13);
+  return true;
 }
 
-template <int THREADS, int ITEMS>
+template <int THREADS, int ITEMS, bool kEarly>
 __global__ void __launch_bounds__(THREADS)
 topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* __restrict__ ctx_len,
                  int32_t* __restrict__ sel, int32_t* __restrict__ n_sel, uint32_t* __restrict__ status, TopkExtras x) {
@@ -453,22 +475,18 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
   if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;   // stable: the previous step's selection has finished
-  if (!scores_ready(geo, x, b, kvh, len_b, &s_flag)) {     // the scores come from the previous kernel
-    write_empty_selection(geo, x, bh, out, n_sel, THREADS);
-    selection_done(geo, x, b, kvh, &s_flag);
-    return;
-  }
-  SWARM_STAMP(status, 1);
   const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
   const int k_sel = k_eff - (P - Pw);                       // places left for the scored pages [0, Pw)
   // A list half as long as the kernel's capacity is handled with half the pages per thread: the work of every
   // phase is per page held, and the lists of one launch differ in length (ragged batches).
+  bool ok;
   if (ITEMS == 16 && P <= THREADS * 8)
-    topk_regs_body<THREADS, 8, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
+    ok = topk_regs_body<THREADS, 8, ITEMS, kEarly>(st, geo, x, rb, s, out, n_sel, status, bh, b, kvh, len_b, &s_flag, P, Pw, k_eff, k_sel);
   else
-    topk_regs_body<THREADS, ITEMS, ITEMS>(st, geo, x, rb, s, out, n_sel, status, bh, P, Pw, k_eff, k_sel);
+    ok = topk_regs_body<THREADS, ITEMS, ITEMS, kEarly>(st, geo, x, rb, s, out, n_sel, status, bh, b, kvh, len_b, &s_flag, P, Pw, k_eff, k_sel);
+  if (!ok) write_empty_selection(geo, x, bh, out, n_sel, THREADS);
   selection_done(geo, x, b, kvh, &s_flag);
   SWARM_KERNEL_END(status, 1);
 }
@@ -615,10 +633,14 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   x.tk = links.tk;
   x.flags_alt = flags != nullptr ? links.flags_alt : 0;
   if (x.req_base == nullptr) x.tk.ready = nullptr;         // the validity test of a request needs its page count
+  // few lists: every thread reads the page -> cluster entries of all its pages up front (kEarly)
+  const bool early = flags != nullptr && (long long)geo.B * geo.Hq <= 128;
   const dim3 grid(geo.B * geo.Hq);
-#define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                    \
-  return launch_pdl(topk_regs_kernel<THREADS, ITEMS>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
-                    ctx_len, sel, n_sel, status, x)
+#define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                           \
+  return early ? launch_pdl(topk_regs_kernel<THREADS, ITEMS, true>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
+                            ctx_len, sel, n_sel, status, x)                                                         \
+               : launch_pdl(topk_regs_kernel<THREADS, ITEMS, false>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
+                            ctx_len, sel, n_sel, status, x)
   if (geo.Pmax <= 1024) SWARM_TOPK_REGS(128, 8);
   if (geo.Pmax <= 2048) SWARM_TOPK_REGS(256, 8);
   if (geo.Pmax <= 4096) SWARM_TOPK_REGS(512, 8);

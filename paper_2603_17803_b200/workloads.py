@@ -285,6 +285,38 @@ def generate(cfg: WorkloadConfig, seed: int = 0, device="cpu", layer: int = 0, s
     )
 
 
+def subset_requests(w: "Workload", requests, device="cpu") -> "Workload":
+    """The given requests of a workload as a workload of their own on ``device`` (their pages, cluster tables
+    and queries copied and re-based; nothing is redrawn).  Used to hand the CPU oracle a bounded sample of a
+    large batch."""
+    requests = [int(b) for b in requests]
+    page_base = w.page_base.cpu().numpy()
+    cluster_base = w.cluster_base.cpu().numpy()
+    pool, p2c, sizes, masks, topics = [], [], [], [], []
+    pb, cb = [0], [0]
+    for b in requests:
+        lo, hi = int(page_base[b]), int(page_base[b + 1])
+        clo, chi = int(cluster_base[b]), int(cluster_base[b + 1])
+        pool.append(w.kv_pool[lo:hi].to(device))
+        p2c.append(w.page2cluster[lo:hi].to(device))
+        sizes.append(w.cluster_size[clo:chi].to(device))
+        masks.append(w.cluster_replica_mask[clo:chi].to(device))
+        topics.append(w.topic_of_page[lo:hi])
+        pb.append(pb[-1] + hi - lo)
+        cb.append(cb[-1] + chi - clo)
+    idx = torch.tensor(requests, dtype=torch.long, device=w.q.device)
+    cfg = dataclasses.replace(w.cfg, batch=len(requests))
+    return Workload(
+        cfg=cfg, seed=w.seed, q=w.q[idx].to(device), kv_pool=torch.cat(pool),
+        page_base=torch.tensor(pb, dtype=torch.int64, device=device),
+        ctx_len=w.ctx_len[idx].to(device), page2cluster=torch.cat(p2c),
+        cluster_base=torch.tensor(cb, dtype=torch.int64, device=device),
+        cluster_replica_mask=torch.cat(masks), cluster_size=torch.cat(sizes),
+        topic_of_page=np.concatenate(topics),
+        centroids=None if w.centroids is None else w.centroids[idx].to(device),
+    )
+
+
 def bits_u16(t: torch.Tensor) -> np.ndarray:
     """Raw bits of a bf16 (or 16-bit integer) tensor as a host uint16 array (the form the oracle takes)."""
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
