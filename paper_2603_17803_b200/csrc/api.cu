@@ -62,7 +62,7 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   WorkspaceLayout l;
   const int64_t bh = (int64_t)s.batch * s.n_q_heads;
   int64_t off = 0;
-  l.status = off;   off = align256(off + 4);
+  l.status = off;   off = align256(off + 256 + 1024);
   l.scores = off;   off = align256(off + bh * s.max_pages_per_req * 4);
   l.n_tok = off;    off = align256(off + bh * 4);
   l.q_stage = off;  off = align256(off + bh * kHeadDim * 2);

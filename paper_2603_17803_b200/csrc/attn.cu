@@ -30,6 +30,7 @@
 
 #include <algorithm>
 
+#define SWARM_TRACE_FILE 2
 #include "swarm_internal.cuh"
 #include "resolve_body.cuh"
 
@@ -148,7 +149,8 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
 
   // ---- which (request, heads, page range) --------------------------------------------------------
-  const int split = cta % a.n_splits, grp = cta / a.n_splits;
+  const int n_splits = a.n_splits, slot_stride = a.n_splits;
+  const int split = cta % n_splits, grp = cta / n_splits;
   int b, kvh = 0, bh0, G;
   if (kPaged) {
     const int tiles = (geo.g + 7) / 8;
@@ -202,23 +204,13 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   };
   if (ticketed) {
     load_inputs();
-    // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The last CTA
-    // of the grid to get past its wait sets the tickets back to zero for the next step -- after the selection
-    // kernel's own last CTA has finished its bookkeeping, so that the next step cannot start before it.
+    // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The CTA then
+    // counts itself as past its wait (no result comes back: an atomic with one held the CTA's next barrier).
     if (threadIdx.x == 0) {
-      bool ok = wait_at_least(a.tk.sel_ready + (long long)b * geo.Hkv + kvh, (unsigned)geo.g);
-      const unsigned n_ctas = gridDim.x - (kFused != 0 ? 1u : 0u);
-      const bool last = atomicAdd(a.tk.ctl + kCtlAttnPast, 1u) == n_ctas - 1u;
-      if (last) ok = wait_zero(a.tk.ctl + kCtlTopkDone) && ok;
-      if (!ok) atomicOr(status, SWARM_DEV_TIMEOUT);
-      s_last = last;
+      if (!wait_at_least(a.tk.sel_ready + (long long)b * geo.Hkv + kvh, (unsigned)geo.g)) atomicOr(status, SWARM_DEV_TIMEOUT);
+      red_relaxed_add(a.tk.ctl + kCtlAttnPast, 1u);
     }
     __syncthreads();
-    if (s_last) {
-      for (int i = threadIdx.x; i < geo.B * geo.Hkv; i += kAttnWarps * 32) a.tk.sel_ready[i] = 0u;
-      __syncthreads();
-      if (threadIdx.x == 0) st_release(a.tk.ctl + kCtlAttnPast, 0u);
-    }
   } else {
     pdl_wait();                                         // the selection comes from the previous kernel
     load_inputs();
@@ -280,8 +272,8 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     }
     n_items = (total_tok + S - 1) / S;
   }
-  const int it_begin = (int)((long long)n_items * split / a.n_splits);
-  const int it_end = (int)((long long)n_items * (split + 1) / a.n_splits);
+  const int it_begin = (int)((long long)n_items * split / n_splits);
+  const int it_end = (int)((long long)n_items * (split + 1) / n_splits);
 
   const float scale = kLog2e * rsqrtf((float)kHeadDim);
 
@@ -535,11 +527,11 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     }
     const long long bh = bh0 + hh;
     bool finish = true;                                 // this warp writes the head's final result
-    if (a.n_splits > 1) {
+    if (n_splits > 1) {
       // publish this split's partial of the head; the warp that arrives last at the head's ticket (whichever
       // CTA it sits in) merges the head's partials.  The heads of a group are thus merged side by side, and
       // nothing waits for a CTA-wide barrier or a staging copy.
-      const long long slot = bh * a.n_splits + split;
+      const long long slot = bh * slot_stride + split;
       __stcg(reinterpret_cast<float4*>(a.part_acc + slot * kHeadDim) + lane, o);
       if (lane == 0) __stcg(reinterpret_cast<float2*>(a.part_ml + slot * 2), make_float2(M, L));
       __syncwarp();                                     // the lanes' stores are ordered before lane 0's release
@@ -547,13 +539,13 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       if (lane == 0) prev = atom_acq_rel_add(a.tickets + bh, 1u);
       prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
       __syncwarp();                                     // lane 0's acquire is ordered before the other lanes' loads
-      finish = prev == (unsigned)a.n_splits - 1u;
+      finish = prev == (unsigned)n_splits - 1u;
       if (finish) {
         // (max, sum) of split `lane` and `lane + 32`; then every lane sums its 4 coordinates over the splits
-        const float2 ml0 = lane < a.n_splits ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * a.n_splits + lane) * 2))
+        const float2 ml0 = lane < n_splits ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * slot_stride + lane) * 2))
                                              : make_float2(-INFINITY, 0.f);
-        const float2 ml1 = lane + 32 < a.n_splits
-                               ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * a.n_splits + lane + 32) * 2))
+        const float2 ml1 = lane + 32 < n_splits
+                               ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * slot_stride + lane + 32) * 2))
                                : make_float2(-INFINITY, 0.f);
         M = fmaxf(ml0.x, ml1.x);
 #pragma unroll
@@ -562,13 +554,13 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         L = ml0.y * w0 + ml1.y * w1;
 #pragma unroll
         for (int o2 = 16; o2 >= 1; o2 >>= 1) L += __shfl_xor_sync(0xFFFFFFFFu, L, o2);
-        const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * a.n_splits * kHeadDim) + lane;
+        const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * slot_stride * kHeadDim) + lane;
         o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp0 = 0; sp0 < a.n_splits; sp0 += 8) {
+        for (int sp0 = 0; sp0 < n_splits; sp0 += 8) {
           float4 v[8];
 #pragma unroll
           for (int u = 0; u < 8; ++u)                   // eight rows in flight together
-            v[u] = sp0 + u < a.n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[u] = sp0 + u < n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int sp = sp0 + u;
@@ -592,6 +584,16 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         if (lane == 0) host_arrive(a.host);
       }
     }
+  }
+  if (ticketed && threadIdx.x == 0 && blockIdx.x == gridDim.x - 1) {
+    // The last CTA of the grid (its KV head is selected last, so it tends to finish last) tidies up: once every
+    // CTA is past its wait nobody reads the selection's tickets any more, and they go back to zero for the next
+    // step -- after the selection kernel has finished its own bookkeeping, so that the next step (which starts
+    // after this kernel) finds all of it done.
+    const unsigned n_ctas = gridDim.x - (kFused != 0 ? 1u : 0u);
+    if (!wait_at_least(a.tk.ctl + kCtlAttnPast, n_ctas) || !wait_zero(a.tk.ctl + kCtlTopkDone)) atomicOr(status, SWARM_DEV_TIMEOUT);
+    for (int i = 0; i < geo.B * geo.Hkv; ++i) a.tk.sel_ready[i] = 0u;
+    st_release(a.tk.ctl + kCtlAttnPast, 0u);
   }
   SWARM_STAMP_ANY_CTA(status, 6);
   SWARM_KERNEL_END(status, 2);

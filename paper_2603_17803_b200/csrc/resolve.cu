@@ -1,4 +1,5 @@
 // Stage 3 as a kernel of its own (swarm_resolve_clusters); the algorithm is in resolve_body.cuh.
+#define SWARM_TRACE_FILE 3
 #include "resolve_body.cuh"
 
 namespace swarm {

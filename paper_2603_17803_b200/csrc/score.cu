@@ -23,6 +23,7 @@
 
 #include <algorithm>
 
+#define SWARM_TRACE_FILE 0
 #include "swarm_internal.cuh"
 
 namespace swarm {

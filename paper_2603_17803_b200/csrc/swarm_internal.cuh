@@ -12,7 +12,8 @@ constexpr int kHeadDim = 128;
 
 // Where each scratch region sits inside the caller-provided workspace (byte offsets, 256-aligned).
 struct WorkspaceLayout {
-  int64_t status;        // uint32 status word; +64: ticket counter of the resolve kernel; +96: of the publish kernel (all start at 0)
+  int64_t status;        // uint32 status word; +64: ticket counter of the resolve kernel; +96: of the publish kernel (all start at 0);
+                         // +256: 1 KiB of time stamps in development builds
   int64_t scores;        // f32 [B][Hq][Pmax]          (used when the caller passes no scores buffer)
   int64_t n_tok;         // i32 [B][Hq]                (used when the caller passes no n_tok buffer)
   int64_t q_stage;       // bf16 [B][Hq][d]            (swarm_step_host)
@@ -66,6 +67,9 @@ __device__ __forceinline__ bool wait_at_least(const unsigned* p, unsigned target
 // them.  (A plain __threadfence() is the sequentially consistent fence, which costs far more.)
 __device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_relaxed_add(unsigned* p, unsigned v) {   // no result: nothing waits for it
+  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ unsigned atom_acq_rel_add(unsigned* p, unsigned v) {
   unsigned prev;
@@ -294,22 +298,33 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Development-only time stamps (compiled in with -DSWARM_TRACE): thread 0 of CTA 0 records %globaltimer (ns)
-// at up to 16 numbered points of a kernel into bytes [128, 256) of the workspace's status block, where
-// a developer reads them back from the workspace tensor.  Absent from normal builds.
+// Development-only time stamps (compiled in with -DSWARM_TRACE): thread 0 of one CTA records %globaltimer (ns)
+// at up to 16 numbered points of a kernel into the workspace's trace block (1 KiB behind the status block:
+// 16 slots per source file, SWARM_TRACE_FILE selects the group), where a developer reads them back from the
+// workspace tensor.  Absent from normal builds.
 #ifdef SWARM_TRACE
 __device__ __forceinline__ unsigned long long trace_now() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+#ifndef SWARM_TRACE_FILE
+#define SWARM_TRACE_FILE 0
+#endif
+#if SWARM_TRACE_FILE == 0 && defined(SWARM_TRACE_CTA_F0)
+#define SWARM_TRACE_CTA SWARM_TRACE_CTA_F0
+#elif SWARM_TRACE_FILE == 1 && defined(SWARM_TRACE_CTA_F1)
+#define SWARM_TRACE_CTA SWARM_TRACE_CTA_F1
+#elif SWARM_TRACE_FILE == 2 && defined(SWARM_TRACE_CTA_F2)
+#define SWARM_TRACE_CTA SWARM_TRACE_CTA_F2
+#endif
 #ifndef SWARM_TRACE_CTA
 #define SWARM_TRACE_CTA 0
 #endif
 #define SWARM_STAMP_RAW(status, i, any_cta)                                                          \
   do {                                                                                               \
     if (threadIdx.x == 0 && ((any_cta) || (blockIdx.x == (SWARM_TRACE_CTA) && blockIdx.y == 0 && blockIdx.z == 0)))  \
-      reinterpret_cast<unsigned long long*>(status)[16 + (i)] = trace_now();                         \
+      reinterpret_cast<unsigned long long*>(status)[32 + 16 * (SWARM_TRACE_FILE) + (i)] = trace_now(); \
   } while (0)
 #endif
 #if defined(SWARM_TRACE) && SWARM_TRACE == 1      // phases inside one kernel

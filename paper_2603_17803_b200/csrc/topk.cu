@@ -14,6 +14,7 @@
 // topk_regs keeps ITEMS consecutive pages per thread in registers (lists of up to 16384 pages; in the
 // largest instance a list of at most half that length is handled with half the pages per thread);
 // topk_generic walks lists of any length in shared or global memory with the same algorithm.
+#define SWARM_TRACE_FILE 1
 #include "swarm_internal.cuh"
 
 namespace swarm {
@@ -64,6 +65,7 @@ __device__ __forceinline__ bool scores_ready(const Geometry& geo, const TopkExtr
   }
   if (x.tk.ready == nullptr) {
     pdl_wait();
+    if (threadIdx.x == 0 && x.tk.ctl != nullptr) red_relaxed_add(x.tk.ctl + kCtlTopkDone, 1u);
     return true;
   }
   if (threadIdx.x == 0) {
@@ -75,6 +77,8 @@ __device__ __forceinline__ bool scores_ready(const Geometry& geo, const TopkExtr
       ok = wait_at_least(x.tk.ready + (long long)b * head_pairs(geo.Hkv) + hp, target);
       if (!ok) atomicOr(x.status, SWARM_DEV_TIMEOUT);
     }
+    // this CTA is past its wait (no result comes back: an atomic with one held the CTA's next barrier)
+    red_relaxed_add(x.tk.ctl + kCtlTopkDone, 1u);
     *s_flag = ok;
   }
   __syncthreads();
@@ -92,27 +96,27 @@ __device__ __forceinline__ void write_empty_selection(const Geometry& geo, const
   }
 }
 
-// What a selection CTA does last, after a barrier behind its stores: announce the head to the attention CTAs of
-// its KV head, and count itself; the last CTA of the launch clears the scorer's tickets for the next step.
-__device__ __forceinline__ void selection_done(const Geometry& geo, const TopkExtras& x, int b, int kvh, bool* s_flag) {
-  if (x.tk.ctl == nullptr) return;
-  __syncthreads();                                          // every thread's stores are issued
-  if (threadIdx.x == 0) {                                   // releases, cumulative over them
-    if (x.tk.sel_ready != nullptr) red_release_add(x.tk.sel_ready + (long long)b * geo.Hkv + kvh, 1u);
-    const unsigned prev = atom_acq_rel_add(x.tk.ctl + kCtlTopkDone, 1u);
-    *s_flag = prev == gridDim.x - 1u;
-  }
+// The head's page bitmap is stored: announce it to the attention CTAs of its KV head (a barrier, then one
+// release that is cumulative over the CTA's stores so far).
+__device__ __forceinline__ void selection_announce(const Geometry& geo, const TopkExtras& x, int b, int kvh) {
+  if (x.tk.sel_ready == nullptr) return;
   __syncthreads();
-  if (*s_flag) {                                            // every other CTA has finished: nobody reads the tickets any more
+  if (threadIdx.x == 0) red_release_add(x.tk.sel_ready + (long long)b * geo.Hkv + kvh, 1u);
+}
+
+// What a selection CTA does last.  The last CTA of the grid (its scores arrive last, so it tends to finish last)
+// tidies up: once every CTA is past its wait for the scorer nobody reads the scorer's tickets any more, and they
+// go back to zero.
+__device__ __forceinline__ void selection_done(const Geometry& geo, const TopkExtras& x) {
+  if (x.tk.ctl == nullptr) return;
+  if (threadIdx.x == 0 && blockIdx.x == gridDim.x - 1) {
+    if (!wait_at_least(x.tk.ctl + kCtlTopkDone, gridDim.x)) atomicOr(x.status, SWARM_DEV_TIMEOUT);
     if (x.tk.ready != nullptr)
-      for (int i = threadIdx.x; i < geo.B * head_pairs(geo.Hkv); i += blockDim.x) x.tk.ready[i] = 0u;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      if (x.flags_alt > 0) x.tk.ctl[kCtlMarked] += 1u;      // the cluster marks of one more step are complete
-      // last of all: whoever reads 0 here (the attention kernel, before it lets the next step start) also sees
-      // the cleared tickets
-      st_release(x.tk.ctl + kCtlTopkDone, 0u);
-    }
+      for (int i = 0; i < geo.B * head_pairs(geo.Hkv); ++i) x.tk.ready[i] = 0u;
+    if (x.flags_alt > 0) x.tk.ctl[kCtlMarked] += 1u;        // one more step has its cluster marks (complete when this kernel is)
+    // last of all: whoever reads 0 here (the attention kernel, before it lets the next step start) also sees
+    // the cleared tickets
+    st_release(x.tk.ctl + kCtlTopkDone, 0u);
   }
 }
 
@@ -401,19 +405,29 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
   __syncthreads();
   const int before = incl - cnt + totals_before<THREADS>(st.warp_tot, warp, lane);
   const int gt_before = before & 0xFFFF, eq_before = before >> 16;
+  // The page bitmap goes out first and the head is announced to the attention CTAs right behind it: a release
+  // waits for every store issued before it to be acknowledged, so the selection list, the cluster marks and the
+  // rest (which the attention does not read) are stored after the announcement, not before.
   unsigned picked = 0u;                                     // bit j: page p0 + j is selected
   for (unsigned todo = gt_mask | eq_mask; todo != 0u; todo &= todo - 1u) {
-    const unsigned bit = todo & (0u - todo), below = bit - 1u;
-    const int eq_b = eq_before + __popc(eq_mask & below);
-    if ((gt_mask & bit) || eq_b < need_eq) {
-      out[gt_before + __popc(gt_mask & below) + min(eq_b, need_eq)] = p0 + (__ffs(bit) - 1);
-      picked |= bit;
-    }
+    const unsigned bit = todo & (0u - todo);
+    if ((gt_mask & bit) || eq_before + __popc(eq_mask & (bit - 1u)) < need_eq) picked |= bit;
   }
   if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
     uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch + p0 / 8;
     if (ITEMS == 8) *row = (uint8_t)picked;
     else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
+  }
+  if (ITEMS < MAX_ITEMS && x.selmap != nullptr) {          // the part of the bitmap row these threads do not reach
+    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
+    for (int o = THREADS * ITEMS / 8 + tid * 4; o + 4 <= x.selmap_pitch; o += THREADS * 4)
+      *reinterpret_cast<uint32_t*>(row + o) = 0u;
+  }
+  selection_announce(geo, x, b, kvh);
+  for (unsigned todo = picked; todo != 0u; todo &= todo - 1u) {
+    const unsigned bit = todo & (0u - todo), below = bit - 1u;
+    const int eq_b = eq_before + __popc(eq_mask & below);
+    out[gt_before + __popc(gt_mask & below) + min(eq_b, need_eq)] = p0 + (__ffs(bit) - 1);
   }
   if (kEarly && x.flags != nullptr) {
 #pragma unroll
@@ -448,11 +462,6 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
   }
   for (int j = k_eff + tid; j < geo.k; j += THREADS) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
-  if (ITEMS < MAX_ITEMS && x.selmap != nullptr) {          // the part of the bitmap row these threads do not reach
-    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
-    for (int o = THREADS * ITEMS / 8 + tid * 4; o + 4 <= x.selmap_pitch; o += THREADS * 4)
-      *reinterpret_cast<uint32_t*>(row + o) = 0u;
-  }
   SWARM_STAMP(status, 13);
   return true;
 }
@@ -486,8 +495,11 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
     ok = topk_regs_body<THREADS, 8, ITEMS, kEarly>(st, geo, x, rb, s, out, n_sel, status, bh, b, kvh, len_b, &s_flag, P, Pw, k_eff, k_sel);
   else
     ok = topk_regs_body<THREADS, ITEMS, ITEMS, kEarly>(st, geo, x, rb, s, out, n_sel, status, bh, b, kvh, len_b, &s_flag, P, Pw, k_eff, k_sel);
-  if (!ok) write_empty_selection(geo, x, bh, out, n_sel, THREADS);
-  selection_done(geo, x, b, kvh, &s_flag);
+  if (!ok) {
+    write_empty_selection(geo, x, bh, out, n_sel, THREADS);
+    selection_announce(geo, x, b, kvh);
+  }
+  selection_done(geo, x);
   SWARM_KERNEL_END(status, 1);
 }
 
@@ -514,7 +526,8 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;
   if (!scores_ready(geo, x, b, kvh, len_b, &s_flag)) {
     write_empty_selection(geo, x, bh, out, n_sel, kGenericThreads);
-    selection_done(geo, x, b, kvh, &s_flag);
+    selection_announce(geo, x, b, kvh);
+    selection_done(geo, x);
     return;
   }
   const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));
@@ -599,7 +612,8 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   }
   for (int j = k_eff + tid; j < geo.k; j += kGenericThreads) out[j] = -1;
   if (tid == 0) n_sel[bh] = k_eff;
-  selection_done(geo, x, b, kvh, &s_flag);
+  selection_announce(geo, x, b, kvh);
+  selection_done(geo, x);
 }
 
 constexpr size_t kSmemKeyBytes = 160 * 1024;
