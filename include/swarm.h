@@ -148,6 +148,12 @@ int32_t swarm_destroy(swarm_ctx* ctx);
 int64_t swarm_workspace_bytes(const swarm_shape* shape);
 int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, void* stream);
 
+/* Debugging aid: the workspace regions are separated by 256 canary bytes each (one in front of every region,
+ * one behind the last), written by swarm_set_workspace.  Copies them back and sets bit i of *damaged for every
+ * canary i (in workspace order) that no longer holds its pattern, i.e. some kernel wrote outside its region.
+ * SYNCHRONISES `stream`.  Stands in for a memory checker where none can be run. */
+int32_t swarm_check_workspace(swarm_ctx* ctx, void* stream, uint32_t* damaged);
+
 /* Attaches (or, with NULL, detaches) cache state to the ctx; the struct is copied.  While attached,
  * swarm_resolve_clusters and swarm_step compute the full Eq. 8: the clusters to fetch are the activated
  * ones minus the resident ones (only those appear in uniq / queue_of / queue_load), and the bookkeeping of

@@ -26,7 +26,7 @@ _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
-    "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_tail_stream", "swarm_tail_join", "swarm_set_select_sms", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_check_workspace", "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_tail_stream", "swarm_tail_join", "swarm_set_select_sms", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_sparse_attn_static_status", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
@@ -162,6 +162,13 @@ def swarm_set_workspace(ctx, workspace: torch.Tensor, stream=None) -> None:
     _check(load_library().swarm_set_workspace(ctx, _ptr(workspace, "workspace"),
                                               ctypes.c_int64(workspace.numel() * workspace.element_size()),
                                               _stream(stream)), "swarm_set_workspace", ctx)
+
+
+def swarm_check_workspace(ctx, stream=None) -> int:
+    """Bit mask of the workspace canaries that were overwritten (0 = intact); synchronises the stream."""
+    bits = ctypes.c_uint32(0)
+    _check(load_library().swarm_check_workspace(ctx, _stream(stream), ctypes.byref(bits)), "swarm_check_workspace", ctx)
+    return int(bits.value)
 
 
 def swarm_set_attn_splits(ctx, n_splits: int) -> None:

@@ -10,6 +10,19 @@
 
 #include "swarm_internal.cuh"
 
+// Stage ranges for timeline tools (Nsight Systems and the like): compiled in with -DSWARM_NVTX, absent otherwise.
+// A range covers the enqueueing of a stage on the host; the tools attach the kernels launched inside it.
+#ifdef SWARM_NVTX
+#include <nvtx3/nvToolsExt.h>
+struct StageRange {
+  explicit StageRange(const char* name) { nvtxRangePushA(name); }
+  ~StageRange() { nvtxRangePop(); }
+};
+#define SWARM_RANGE(name) StageRange swarm_range_(name)
+#else
+#define SWARM_RANGE(name) do { } while (0)
+#endif
+
 using namespace swarm;
 
 struct swarm_ctx {
@@ -62,22 +75,29 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   WorkspaceLayout l;
   const int64_t bh = (int64_t)s.batch * s.n_q_heads;
   int64_t off = 0;
-  l.status = off;   off = align256(off + 256 + 1024);
-  l.scores = off;   off = align256(off + bh * s.max_pages_per_req * 4);
-  l.n_tok = off;    off = align256(off + bh * 4);
-  l.q_stage = off;  off = align256(off + bh * kHeadDim * 2);
-  l.flags = off;    off = align256(off + (int64_t)s.max_clusters_total + 16);   // two arrays: alternate steps of the
-  l.flags_alt = off - l.flags;                                                  // overlapped tail mark alternate ones
-  off = align256(off + (int64_t)s.max_clusters_total + 16);
-  l.part_acc = off; off = align256(off + bh * kMaxSplits * kHeadDim * 4);
-  l.part_ml = off;  off = align256(off + bh * kMaxSplits * 2 * 4);
-  l.items = off;    off = align256(off + (int64_t)s.max_clusters_total * 16);
-  l.selmap = off;   off = align256(off + bh * selmap_pitch_bytes(s.max_pages_per_req));
-  l.tickets = off;  off = align256(off + bh * 4);
-  l.ctl = off;      off = align256(off + 64 * 4);
-  l.ready = off;    off = align256(off + (int64_t)s.batch * head_pairs(s.n_kv_heads) * 4);
-  l.sel_ready = off; off = align256(off + (int64_t)s.batch * s.n_kv_heads * 4);
-  l.total = off;
+  l.n_guard = 0;
+  auto place = [&](int64_t bytes) -> int64_t {               // a guard, then the region
+    l.guard[l.n_guard++] = off;
+    const int64_t at = off + kGuardBytes;
+    off = align256(at + bytes);
+    return at;
+  };
+  l.status = place(256 + 1024);
+  l.scores = place(bh * s.max_pages_per_req * 4);
+  l.n_tok = place(bh * 4);
+  l.q_stage = place(bh * kHeadDim * 2);
+  l.flags_alt = align256((int64_t)s.max_clusters_total + 16);          // two arrays: alternate steps of the overlapped
+  l.flags = place(2 * l.flags_alt);                                    // tail mark alternate ones
+  l.part_acc = place(bh * kMaxSplits * kHeadDim * 4);
+  l.part_ml = place(bh * kMaxSplits * 2 * 4);
+  l.items = place((int64_t)s.max_clusters_total * 16);
+  l.selmap = place(bh * selmap_pitch_bytes(s.max_pages_per_req));
+  l.tickets = place(bh * 4);
+  l.ctl = place(64 * 4);
+  l.ready = place((int64_t)s.batch * head_pairs(s.n_kv_heads) * 4);
+  l.sel_ready = place((int64_t)s.batch * s.n_kv_heads * 4);
+  l.guard[l.n_guard++] = off;
+  l.total = off + kGuardBytes;
   return l;
 }
 
@@ -283,8 +303,28 @@ int32_t swarm_set_workspace(swarm_ctx* ctx, void* device_mem, int64_t bytes, voi
   // regions that must hold zeros between calls: status word, ticket counters, dedup flags
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 256, st));
-  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.flags, 0, ctx->lay.part_acc - ctx->lay.flags, st));
+  SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.flags, 0, 2 * ctx->lay.flags_alt, st));
   SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.tickets, 0, ctx->lay.total - ctx->lay.tickets, st));   // and the hand-off counters
+  for (int i = 0; i < ctx->lay.n_guard; ++i)               // canaries last: the spans above run over some of them
+    SWARM_TRY(cudaMemsetAsync(ctx->ws + ctx->lay.guard[i], kCanaryByte, kGuardBytes, st));
+  return SWARM_OK;
+}
+
+int32_t swarm_check_workspace(swarm_ctx* ctx, void* stream, uint32_t* damaged) {
+  int32_t rc = need_ws(ctx);
+  if (rc != SWARM_OK) return rc;
+  if (damaged == nullptr) return SWARM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  static_assert(sizeof(ctx->lay.guard) / sizeof(ctx->lay.guard[0]) <= 32, "one bit per guard");
+  unsigned char host[20 * kGuardBytes];
+  for (int i = 0; i < ctx->lay.n_guard; ++i)
+    SWARM_TRY(cudaMemcpyAsync(host + i * kGuardBytes, ctx->ws + ctx->lay.guard[i], kGuardBytes, cudaMemcpyDeviceToHost, st));
+  SWARM_TRY(cudaStreamSynchronize(st));
+  uint32_t bits = 0u;
+  for (int i = 0; i < ctx->lay.n_guard; ++i)
+    for (int j = 0; j < kGuardBytes; ++j)
+      if (host[i * kGuardBytes + j] != (unsigned char)kCanaryByte) { bits |= 1u << i; break; }
+  *damaged = bits;
   return SWARM_OK;
 }
 
@@ -413,6 +453,7 @@ int32_t swarm_build_summaries(swarm_ctx* ctx, const swarm_inputs* in, void* ksum
 
 int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int32_t* sel, int32_t* n_sel,
                      void* stream) {
+  SWARM_RANGE("swarm_select");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!select_inputs_ok(in) || bad(sel) || bad(n_sel) || (scores && !aligned16(scores))) return SWARM_ERR_INVALID_ARG;
@@ -432,6 +473,7 @@ int32_t swarm_select(swarm_ctx* ctx, const swarm_inputs* in, float* scores, int3
 int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
                                int32_t* uniq, uint8_t* queue_of, int32_t* n_uniq, int32_t* queue_load,
                                void* stream) {
+  SWARM_RANGE("swarm_resolve_clusters");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!resolve_inputs_ok(in) || bad(sel) || bad(n_sel) || bad(uniq) || bad(queue_of) || bad(n_uniq) ||
@@ -443,6 +485,7 @@ int32_t swarm_resolve_clusters(swarm_ctx* ctx, const swarm_inputs* in, const int
 
 int32_t swarm_gather(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel, void* k_out,
                      void* v_out, int32_t* n_tok, void* stream) {
+  SWARM_RANGE("swarm_gather");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!pool_inputs_ok(in) || bad(sel) || bad(n_sel) || bad(k_out) || bad(v_out) || (n_tok && !aligned16(n_tok)))
@@ -455,6 +498,7 @@ int32_t swarm_gather(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel,
 
 int32_t swarm_sparse_attn(swarm_ctx* ctx, const void* q, const void* k_g, const void* v_g, const int32_t* n_tok,
                           float* out, float* lse, void* stream) {
+  SWARM_RANGE("swarm_sparse_attn");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (bad(q) || bad(k_g) || bad(v_g) || bad(n_tok) || bad(out) || bad(lse)) return SWARM_ERR_INVALID_ARG;
@@ -495,6 +539,7 @@ AttnArgs paged_args(const swarm_ctx* ctx, const swarm_inputs* in, float* out, fl
 
 int32_t swarm_sparse_attn_paged(swarm_ctx* ctx, const swarm_inputs* in, const int32_t* sel, const int32_t* n_sel,
                                 float* out, float* lse, void* stream) {
+  SWARM_RANGE("swarm_sparse_attn_paged");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (!pool_inputs_ok(in) || bad(in->q) || bad(out) || bad(lse) || ((sel == nullptr) != (n_sel == nullptr)) ||
@@ -564,6 +609,7 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   links.req_base = in->page_base;
   links.flags_alt = tail ? ctx->lay.flags_alt : 0;
   if (parts & kStepBegin) {
+    SWARM_RANGE("swarm: score + select");
     SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
                                 status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail)));
     // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
@@ -573,6 +619,7 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   }
   if (!(parts & kStepEnd)) return SWARM_OK;
 
+  SWARM_RANGE("swarm: resolve + gather + attention");
   if (o->k_out != nullptr)
     SWARM_TRY(launch_gather(ctx->geo, pool, o->sel, o->n_sel, in->page_base, in->ctx_len,
                             static_cast<uint16_t*>(o->k_out), static_cast<uint16_t*>(o->v_out), o->n_tok, status, st));
@@ -694,6 +741,7 @@ int32_t swarm_build_medoid_index(swarm_ctx* ctx, const swarm_inputs* in, const i
 
 int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_medoid_index* idx,
                           const swarm_outputs* o, void* stream) {
+  SWARM_RANGE("swarm_step_medoid");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (in == nullptr || bad(in->q) || !resolve_inputs_ok(in) || !pool_inputs_ok(in) || idx == nullptr ||
@@ -749,6 +797,7 @@ int32_t swarm_step_medoid(swarm_ctx* ctx, const swarm_inputs* in, const swarm_me
 int32_t swarm_step_host(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o, const void* q_host,
                         float* out_host, float* lse_host, int32_t* n_uniq_host, int32_t* queue_load_host,
                         void* stream) {
+  SWARM_RANGE("swarm_step_host");
   int32_t rc = need_ws(ctx);
   if (rc != SWARM_OK) return rc;
   if (in == nullptr || o == nullptr || q_host == nullptr) return SWARM_ERR_INVALID_ARG;

@@ -28,7 +28,13 @@ struct WorkspaceLayout {
   int64_t ready;         // u32 [B][head pairs]        score units complete (scorer -> selection; zero between steps)
   int64_t sel_ready;     // u32 [B][Hkv]               heads selected (selection -> attention; zero between steps)
   int64_t total;
+  // 256 canary bytes sit in front of every region and behind the last one (kCanaryByte, written by
+  // swarm_set_workspace; swarm_check_workspace reports the ones that no longer hold it)
+  int64_t guard[20];
+  int n_guard;
 };
+constexpr int kGuardBytes = 256;
+constexpr int kCanaryByte = 0xA5;
 
 // Hand-offs between the kernels of a step.  The kernels are chained by programmatic dependent launch, so a
 // kernel is resident before its predecessor has finished; instead of waiting for the whole predecessor it

@@ -189,10 +189,15 @@ class Session:
         return B.swarm_device_status(self.ctx)
 
     def close(self):
+        """Destroys the ctx.  Before that, checks the canaries between the workspace regions: a kernel that wrote
+        outside its region is reported here (every test closes its sessions)."""
         if self.ctx is not None:
             torch.cuda.synchronize(self.device)
+            damaged = B.swarm_check_workspace(self.ctx)
             B.swarm_destroy(self.ctx)
             self.ctx = None
+            if damaged:
+                raise RuntimeError(f"workspace canaries overwritten: mask {damaged:#x}")
 
     def __del__(self):
         try:

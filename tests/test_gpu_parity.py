@@ -72,6 +72,23 @@ def test_fused_step_equals_composition(name):
         s.close()
 
 
+def test_workspace_canaries_catch_a_stray_write():
+    """Every Session.close() checks the canaries between the workspace regions (the stand-in for a memory checker
+    on this path).  Here one canary byte is overwritten from the host side -- a torch fill, no kernel of the
+    library involved -- to show that the check fires, and where."""
+    w = W.generate(CASES["c1_small"], seed=3, device=DEV)
+    sess = Session(w)
+    sess.step()
+    assert B.swarm_check_workspace(sess.ctx) == 0
+    sess.workspace[7] = 0                                   # inside the canary in front of the first region
+    assert B.swarm_check_workspace(sess.ctx) == 1
+    sess.workspace[-3] = 1                                  # and inside the one behind the last region
+    damaged = B.swarm_check_workspace(sess.ctx)
+    assert damaged & 1 and damaged >> 1 and (damaged >> 1) & ((damaged >> 1) - 1) == 0
+    with pytest.raises(RuntimeError, match="canaries"):
+        sess.close()
+
+
 @pytest.mark.parametrize("name", ["c2_small", "c3_small", "c5_small", "k_exceeds_pages"])
 def test_overlapped_tail_gives_the_same_step(name):
     """Cluster resolution on a tail stream (swarm_set_tail_stream): consecutive steps with changing queries are
