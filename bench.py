@@ -175,20 +175,20 @@ def build_signature() -> str:
 
 
 def captured_traffic(workload: str):
-    """dram read + write bytes of one attention launch from the ncu capture summarised under profiles/, if that
-    capture was made from the kernel sources that are running now; (None, why) otherwise."""
-    path = os.path.join(ROOT, "profiles", "attn_traffic.json")
+    """dram read + write bytes of one attention launch from the ncu capture summarised under profiles/ (a text
+    file of `key: value` lines), if that capture was made from the kernel sources that are running now;
+    (None, why) otherwise."""
+    path = os.path.join(ROOT, "profiles", f"attn_kernel_{workload}_traffic.txt")
     try:
         with open(path) as f:
-            rec = json.load(f)
+            ent = dict(line.split(":", 1) for line in f if ":" in line and not line.startswith("#"))
+        ent = {k.strip(): v.strip() for k, v in ent.items()}
+        total = int(ent["dram_bytes_read"]) + int(ent["dram_bytes_write"])
     except Exception:
-        return None, "no capture on record"
-    ent = rec.get(workload)
-    if not ent:
         return None, "no capture on record for this workload"
     if ent.get("kernel_sources") != build_signature():
-        return None, f"capture of {ent.get('date')} belongs to other kernel sources ({ent.get('kernel_sources')})"
-    return int(ent["dram_bytes_read"]) + int(ent["dram_bytes_write"]), f"ncu capture of {ent.get('date')}, same kernel sources"
+        return None, f"the capture of {ent.get('date')} belongs to other kernel sources ({ent.get('kernel_sources')})"
+    return total, f"ncu capture of {ent.get('date')}, same kernel sources"
 
 
 class Bench:
