@@ -102,7 +102,7 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
 }
 
 int pick_splits(const swarm_ctx* ctx, bool paged, bool fused = false) {
-  // One CTA of 8 warps fits per SM (the shared-memory rings).  Two regimes, both measured:
+  // One CTA fits per SM (the shared-memory rings).  Two regimes, both measured:
   //  - one wave: as many splits as keep every CTA resident at once (inside the fused step one SM is left for
   //    the resolution CTA); right when a group's pages do not give many CTAs enough to do;
   //  - several waves: about 2.6 CTAs per SM in total.  The hardware then hands the next CTA to whichever SM

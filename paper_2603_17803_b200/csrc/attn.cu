@@ -53,9 +53,11 @@ __global__ void __launch_bounds__(kAttnWarps * 32, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Geometry geo,
             AttnArgs a, uint32_t* __restrict__ status, const __grid_constant__ ResolveArgs rs) {
   static_assert(kFused == 0 || kPaged, "cluster resolution rides with the paged kernel only");
-  static_assert(resolve_detail::kThreads == kAttnWarps * 32, "the resolution body runs in a CTA of this kernel");
+  static_assert(resolve_detail::kThreads <= kAttnWarps * 32, "the resolution body runs in a CTA of this kernel");
   if (kFused != 0 && blockIdx.x == 0) {
-    resolve_detail::resolve_body<kFused == 2>(rs, 0, 1);
+    // (the body is written for kThreads threads; the CTA's other warps leave, and a CTA-wide barrier counts the
+    // threads that have not left)
+    if (threadIdx.x < resolve_detail::kThreads) resolve_detail::resolve_body<kFused == 2>(rs, 0, 1);
     return;
   }
   const int cta = (int)blockIdx.x - (kFused != 0 ? 1 : 0);
