@@ -124,6 +124,9 @@ int pick_splits(const swarm_ctx* ctx, bool paged, bool fused = false) {
     n = std::min<int64_t>(n, std::max(1, g.k / 4));
   }
   n = std::min<int64_t>(n, kMaxSplits);
+  // The CTA that merges a head reads the splits' partials sixteen at a time: a few splits past a multiple of 16
+  // cost it another trip to L2 (128K tokens, 8 groups: 16 splits 29.9 us per step, 18 splits 30.2).
+  if (n > 16 && (n % 16) * 4 <= n) n -= n % 16;
   return (int)std::max<int64_t>(n, 1);
 }
 

@@ -171,6 +171,22 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     return uni;
   };
   constexpr int kChunkWords = kAttnWarps * 32;          // bitmap words one pass of the CTA covers
+  // (page, head mask) entries of the union pages in `bits` (word w, first rank `rank`) that rank in [lo, hi)
+  auto emit_entries = [&](int w, const HeadWords& hw, uint32_t bits, int rank, int lo, int hi) {
+    while (bits) {
+      const int bit = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (rank >= lo && rank < hi) {
+        uint32_t hm = 0u;
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) hm |= ((hw.v[hh] >> bit) & 1u) << hh;
+        list_page[rank - lo] = (uint32_t)(w * 32 + bit);
+        list_mask[rank - lo] = (uint8_t)hm;
+      }
+      ++rank;
+    }
+  };
+  bool first_list_built = false;                        // the first round's list is written already
 
   if (kPaged) {
     // number of pages in the union of the group's selections: the splits share them evenly by rank
@@ -178,19 +194,45 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     P = pages_of(len, S);
     tail = len - S * (P - 1);
     n_words = min((P + 31) / 32, pitch_words);
-    int total = 0;
-    for (int base = 0; base < n_words; base += kChunkWords) {
-      const int w = base + (int)threadIdx.x;
-      if (base > 0) hw = load_raw(w);
-      total += __popc(union_of(w, hw));
+    if (n_words <= kChunkWords) {
+      // The whole bitmap is one word per thread: one CTA-wide scan gives the size of the union and every
+      // thread's first rank, and the first round's list is written from the words already in registers.
+      const uint32_t bits = union_of((int)threadIdx.x, hw);
+      const int cnt = __popc(bits);
+      int incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (lane == 31) s_wcnt[warp] = incl;
+      __syncthreads();
+      int rank = incl - cnt;
+      n_items = 0;
+#pragma unroll
+      for (int w2 = 0; w2 < kAttnWarps; ++w2) {
+        if (w2 < warp) rank += s_wcnt[w2];
+        n_items += s_wcnt[w2];
+      }
+      const int lo = (int)((long long)n_items * split / n_splits);
+      const int hi = min((int)((long long)n_items * (split + 1) / n_splits), lo + kListCap);
+      if (rank + cnt > lo && rank < hi) emit_entries((int)threadIdx.x, hw, bits, rank, lo, hi);
+      first_list_built = true;
+    } else {
+      int total = 0;
+      for (int base = 0; base < n_words; base += kChunkWords) {
+        const int w = base + (int)threadIdx.x;
+        if (base > 0) hw = load_raw(w);
+        total += __popc(union_of(w, hw));
+      }
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+      if (lane == 0) s_wcnt[warp] = total;
+      __syncthreads();
+      n_items = 0;
+#pragma unroll
+      for (int w2 = 0; w2 < kAttnWarps; ++w2) n_items += s_wcnt[w2];
     }
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-    if (lane == 0) s_wcnt[warp] = total;
-    __syncthreads();
-    n_items = 0;
-#pragma unroll
-    for (int w2 = 0; w2 < kAttnWarps; ++w2) n_items += s_wcnt[w2];
   } else {
     total_tok = a.n_tok[bh0];
     if (total_tok < 0 || total_tok > geo.k * S) {          // more tokens than the head's buffer holds: attend what it holds
@@ -225,7 +267,8 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       // thread ranks the pages of its own word with a CTA-wide scan of the per-thread counts
       const int round_end = min(it_end, round0 + kListCap);
       int rank0 = 0;                                    // union pages before the current chunk of words
-      for (int base = 0; base < n_words && rank0 < round_end; base += kChunkWords) {
+      const bool have_list = first_list_built && round0 == it_begin;
+      for (int base = 0; !have_list && base < n_words && rank0 < round_end; base += kChunkWords) {
         const int w = base + (int)threadIdx.x;
         const HeadWords hw = load_raw(w);
         uint32_t bits = union_of(w, hw);
@@ -245,20 +288,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
           if (w2 < warp) rank += s_wcnt[w2];
           rank0 += s_wcnt[w2];
         }
-        if (rank + cnt > round0 && rank < round_end) {
-          while (bits) {
-            const int bit = __ffs(bits) - 1;
-            bits &= bits - 1;
-            if (rank >= round0 && rank < round_end) {
-              uint32_t hm = 0u;
-#pragma unroll
-              for (int hh = 0; hh < 8; ++hh) hm |= ((hw.v[hh] >> bit) & 1u) << hh;
-              list_page[rank - round0] = (uint32_t)(w * 32 + bit);
-              list_mask[rank - round0] = (uint8_t)hm;
-            }
-            ++rank;
-          }
-        }
+        if (rank + cnt > round0 && rank < round_end) emit_entries(w, hw, bits, rank, round0, round_end);
       }
       __syncthreads();
       n_list = round_end - round0;

@@ -204,13 +204,13 @@ __device__ __forceinline__ void finish_head(const AttnArgs& a, long long bh, int
       for (int o2 = 16; o2 >= 1; o2 >>= 1) L += __shfl_xor_sync(0xFFFFFFFFu, L, o2);
       const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * slot_stride * kHeadDim) + lane;
       o = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int sp0 = 0; sp0 < n_splits; sp0 += 8) {
-        float4 v[8];
+      for (int sp0 = 0; sp0 < n_splits; sp0 += 16) {
+        float4 v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)                     // eight rows in flight together
+        for (int u = 0; u < 16; ++u)                    // sixteen rows in flight together
           v[u] = sp0 + u < n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 16; ++u) {
           const int sp = sp0 + u;
           const float ws = __shfl_sync(0xFFFFFFFFu, sp < 32 ? w0 : w1, sp & 31);
           o.x = fmaf(v[u].x, ws, o.x); o.y = fmaf(v[u].y, ws, o.y); o.z = fmaf(v[u].z, ws, o.z); o.w = fmaf(v[u].w, ws, o.w);
