@@ -40,9 +40,8 @@ namespace {
 using namespace attn_detail;
 
 constexpr int kListCap = 1024;                                     // pages per round = 32 bitmap words
-constexpr int kScratchBytes = 8192;   // page list (5 KiB) during the main loop; (max, sum, weight) tables (6 KiB) in the merge
+constexpr int kScratchBytes = kListCap * 5;                        // the page list: ids (u32) and head masks (u8)
 constexpr int kAttnSmemBytes = 1024 /*alignment slack*/ + kRingBytes + kScratchBytes;
-static_assert(kListCap * 5 <= kScratchBytes && (16 + kAttnWarps) * kMaxSplits * 4 <= kScratchBytes, "scratch too small");
 
 // kFused != 0 (fused step only): CTA 0 of the grid does not attend; it runs cluster resolution (stage 3) beside
 // the attention CTAs -- 1: plain, 2: with cache state.  As a kernel of its own on a second stream the serial
@@ -71,7 +70,6 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
   __shared__ int s_wcnt[kAttnWarps];
-  __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
 
@@ -366,57 +364,52 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   SWARM_STAMP(status, 4);
   SWARM_STAMP_ANY_CTA(status, 7);
 
-  // ---- merge the warps of the CTA (the ring is idle now and is reused as scratch) ------------------
-  // Three short phases, each warp-parallel: (1) every warp posts its (max, sum) per head; (2) every lane scales
-  // its own accumulators to the CTA-wide maximum of its heads and posts them; (3) warp h sums head h over the
-  // warps, four coordinates per lane, and is the one that publishes (or finishes) that head.
-  __syncthreads();
-  // rows of 128 + 4 floats: the four lanes of a quad store to heads 2*tq, whose rows then start 8 banks apart
+  // ---- merge the warps of the CTA ---------------------------------------------------------------------
+  // Every warp posts its (max, sum) per head and its raw accumulators into its own ring (idle now: all its copies
+  // have been consumed), so nobody waits for anybody before posting; after the one barrier warp h sums head h
+  // over the warps on their common scale, four coordinates per lane, and is the one that publishes (or
+  // finishes) that head.
+  // rows of 128 + 4 floats: the four lanes of a quad store to heads 2*tq, whose rows then start 8 banks apart;
+  // the row's spare floats hold the head's (max, sum)
   constexpr int kAccRow = kHeadDim + 4;
-  float* s_acc = reinterpret_cast<float*>(ring);        // [warp][head 8][kAccRow]
-  float* s_m = s_acc + kAttnWarps * 8 * kAccRow;        // [warp][8]
-  float* s_l = s_m + kAttnWarps * 8;                    // [warp][8]
-  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
-  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-  if (tq == 0) s_m[warp * 8 + quad] = m_run;
-  __syncthreads();
+  constexpr int kPostStride = kStages * kSlotBytes / 4; // floats between two warps' posts
+  static_assert(8 * kAccRow * 4 <= kStages * kSlotBytes, "a warp's post fits its ring");
   {
-    float sc[2];
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int hh = 2 * tq + j;
-      float Mh = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < kAttnWarps; ++w) Mh = fmaxf(Mh, s_m[w * 8 + hh]);
-      sc[j] = exp2_or_zero(s_m[warp * 8 + hh], Mh);
-    }
-    if (tq == 0) {                                      // this warp's sum of head `quad`, on the common scale
-      float Mq = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < kAttnWarps; ++w) Mq = fmaxf(Mq, s_m[w * 8 + quad]);
-      s_l[warp * 8 + quad] = l_run * exp2_or_zero(m_run, Mq);
+    float* mine = reinterpret_cast<float*>(my_ring);    // [head 8][kAccRow]
+    l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+    l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+    if (tq == 0) {
+      mine[quad * kAccRow + kHeadDim] = m_run;
+      mine[quad * kAccRow + kHeadDim + 1] = l_run;
     }
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
-      float* base = s_acc + (warp * 8 + 2 * tq) * kAccRow + 16 * mt + quad;
-      base[0] = acc[mt][0] * sc[0];
-      base[kAccRow] = acc[mt][1] * sc[1];
-      base[8] = acc[mt][2] * sc[0];
-      base[kAccRow + 8] = acc[mt][3] * sc[1];
+      float* base = mine + 2 * tq * kAccRow + 16 * mt + quad;
+      base[0] = acc[mt][0];
+      base[kAccRow] = acc[mt][1];
+      base[8] = acc[mt][2];
+      base[kAccRow + 8] = acc[mt][3];
     }
   }
   __syncthreads();
   SWARM_STAMP(status, 5);
   if (warp < G) {
     const int hh = warp;                                // this warp's head; lane: coordinates 4 * lane .. + 3
+    const float* posts = reinterpret_cast<const float*>(ring) + hh * kAccRow;
+    float mw[kAttnWarps];
     float M = -INFINITY, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) {
+      mw[w] = posts[w * kPostStride + kHeadDim];
+      M = fmaxf(M, mw[w]);
+    }
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int w = 0; w < kAttnWarps; ++w) {
-      M = fmaxf(M, s_m[w * 8 + hh]);
-      L += s_l[w * 8 + hh];
-      const float4 v = *reinterpret_cast<const float4*>(s_acc + (w * 8 + hh) * kAccRow + 4 * lane);
-      o.x += v.x; o.y += v.y; o.z += v.z; o.w += v.w;
+      const float sc = exp2_or_zero(mw[w], M);
+      const float4 v = *reinterpret_cast<const float4*>(posts + w * kPostStride + 4 * lane);
+      L = fmaf(posts[w * kPostStride + kHeadDim + 1], sc, L);
+      o.x = fmaf(v.x, sc, o.x); o.y = fmaf(v.y, sc, o.y); o.z = fmaf(v.z, sc, o.z); o.w = fmaf(v.w, sc, o.w);
     }
     finish_head(a, bh0 + hh, split, n_splits, lane, M, L, o);
   }

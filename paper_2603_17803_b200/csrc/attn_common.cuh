@@ -189,7 +189,13 @@ __device__ __forceinline__ void finish_head(const AttnArgs& a, long long bh, int
     __syncwarp();                                       // lane 0's acquire is ordered before the other lanes' loads
     finish = prev == (unsigned)n_splits - 1u;
     if (finish) {
-      // (max, sum) of split `lane` and `lane + 32`; then every lane sums its 4 coordinates over the splits
+      // every lane sums its 4 coordinates over the splits, weighted to their common scale: (max, sum) of split
+      // `lane` and `lane + 32` give the weights.  The first sixteen rows are asked for together with them, so that
+      // the merge of up to 16 splits is one trip to L2.
+      const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * slot_stride * kHeadDim) + lane;
+      float4 v[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) v[u] = u < n_splits ? __ldcg(rows + u * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
       const float2 ml0 = lane < n_splits ? __ldcg(reinterpret_cast<const float2*>(a.part_ml + (bh * slot_stride + lane) * 2))
                                            : make_float2(-INFINITY, 0.f);
       const float2 ml1 = lane + 32 < n_splits
@@ -202,13 +208,13 @@ __device__ __forceinline__ void finish_head(const AttnArgs& a, long long bh, int
       L = ml0.y * w0 + ml1.y * w1;
 #pragma unroll
       for (int o2 = 16; o2 >= 1; o2 >>= 1) L += __shfl_xor_sync(0xFFFFFFFFu, L, o2);
-      const float4* rows = reinterpret_cast<const float4*>(a.part_acc + bh * slot_stride * kHeadDim) + lane;
       o = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int sp0 = 0; sp0 < n_splits; sp0 += 16) {
-        float4 v[16];
+        if (sp0 > 0) {
 #pragma unroll
-        for (int u = 0; u < 16; ++u)                    // sixteen rows in flight together
-          v[u] = sp0 + u < n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int u = 0; u < 16; ++u)                  // sixteen rows in flight together
+            v[u] = sp0 + u < n_splits ? __ldcg(rows + (sp0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
           const int sp = sp0 + u;
