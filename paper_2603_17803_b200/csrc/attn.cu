@@ -252,6 +252,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
 
   const uint64_t stream_policy = evict_first_policy();
+  // token row of page (or page slot) p of this CTA's tensor: row_base + p * row_stride
+  const int row_stride = kPaged ? geo.Hkv * 2 * S : S;
+  const int row_base = kPaged ? (int)((pool_row0 * geo.Hkv + kvh) * 2 * S) : (int)((long long)bh0 * geo.k * S);
   unsigned char* my_ring = ring + (size_t)warp * kStages * kSlotBytes;
   unsigned fills = 0, drains = 0;                       // units issued / consumed so far (slot = count % kStages)
   bool timed_out = false;
@@ -305,25 +308,17 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     auto issue = [&](int u) {
       if (lane == 0) {
         const int pg = entry_page(u / SB), sb = u % SB;
-        long long rowK, rowV;
-        if (kPaged) {
-          rowK = ((pool_row0 + pg) * geo.Hkv + kvh) * 2 * S + sb * kUnitTokens;
-          rowV = rowK + S;
-        } else {
-          rowK = rowV = ((long long)bh0 * geo.k + pg) * S + sb * kUnitTokens;
-        }
+        // token row of the unit's K rows (the row count fits 31 bits: checked at launch)
+        const int rowK = row_base + pg * row_stride + sb * kUnitTokens;
         const unsigned slot = fills % kStages;
         const uint32_t dst = smem_addr(my_ring + slot * kSlotBytes);
         uint64_t* bar = &bars[warp][slot];
         mbar_expect_tx(bar, kSlotBytes);
         if (kWide) {                                   // mapK's box is 32 rows here: K then V
-          tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
-          tma_load_2d(dst + kHalf, &mapK, 64, (int)rowK, bar, stream_policy);
+          tma_load_rows(dst, &mapK, rowK, bar, stream_policy);
         } else {
-          tma_load_2d(dst, &mapK, 0, (int)rowK, bar, stream_policy);
-          tma_load_2d(dst + kBoxBytes, &mapK, 64, (int)rowK, bar, stream_policy);
-          tma_load_2d(dst + 2 * kBoxBytes, &mapV, 0, (int)rowV, bar, stream_policy);
-          tma_load_2d(dst + 3 * kBoxBytes, &mapV, 64, (int)rowV, bar, stream_policy);
+          tma_load_rows(dst, &mapK, rowK, bar, stream_policy);
+          tma_load_rows(dst + 2 * kBoxBytes, &mapV, kPaged ? rowK + S : rowK, bar, stream_policy);
         }
       }
       ++fills;
@@ -459,16 +454,16 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 tensor of `rows` token rows x 128 coordinates at `base`; boxes of `box_rows` rows x 64 coordinates,
-// 128-byte swizzle
+// bf16 tensor of `rows` token rows x 128 coordinates at `base`, seen as (64 coordinates, row, half of the
+// coordinates); boxes of 64 coordinates x `box_rows` rows x both halves, 128-byte swizzle (see tma_load_rows)
 cudaError_t make_row_map(CUtensorMap* map, const void* base, long long rows, int box_rows = kUnitTokens) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return cudaErrorNotSupported;
-  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const cuuint64_t dims[3] = {64, (cuuint64_t)rows, 2};
+  const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;

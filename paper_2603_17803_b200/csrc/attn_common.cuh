@@ -44,14 +44,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-// 2-D tiled TMA load: box (64 coordinates, 16 rows) at (x, row) of the tensor behind `map`.  The pages are
-// read once per step: `policy` (evict-first) keeps them from pushing the small tables, the workspace and the
+// Tiled TMA load of token rows.  The tensor of rows x 128 coordinates is described as (64 coordinates, row, half):
+// the two halves of the 128 coordinates are a third dimension 128 bytes apart, so one copy brings a box of both
+// -- in shared memory half 0 of all the box's rows, then half 1, each 128-byte line swizzled by its row.  The pages
+// are read once per step: `policy` (evict-first) keeps them from pushing the small tables, the workspace and the
 // kernels' own instructions out of L2.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int row, uint64_t* bar,
-                                            uint64_t policy) {
+__device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* map, int row, uint64_t* bar, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
-      "l"(map), "r"(x), "r"(row), "r"(smem_addr(bar)), "l"(policy)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+      "l"(map), "r"(0), "r"(row), "r"(0), "r"(smem_addr(bar)), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ uint64_t evict_first_policy() {
