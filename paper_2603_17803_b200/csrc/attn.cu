@@ -74,8 +74,22 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
 
   // ---- which (request, heads, page range) --------------------------------------------------------
-  const int n_splits = a.n_splits;
-  const int split = cta % n_splits, grp = cta / n_splits;
+  // The groups are cut into a.n_splits page ranges each, the last a.n_more of them into one more: the host picks
+  // n_more so that the grid is a whole number of waves (the smaller CTAs come last).
+  const int n_groups = kPaged ? geo.B * geo.Hkv * ((geo.g + 7) / 8) : geo.B * geo.Hq;
+  const int slot_stride = a.n_splits + (a.n_more > 0 ? 1 : 0);
+  const int base_ctas = (n_groups - a.n_more) * a.n_splits;
+  int n_splits, split, grp;
+  if (cta < base_ctas) {
+    n_splits = a.n_splits;
+    grp = cta / n_splits;
+    split = cta - grp * n_splits;
+  } else {
+    n_splits = a.n_splits + 1;
+    const int c = cta - base_ctas;
+    grp = n_groups - a.n_more + c / n_splits;
+    split = c % n_splits;
+  }
   int b, kvh = 0, bh0, G;
   if (kPaged) {
     const int tiles = (geo.g + 7) / 8;
@@ -406,7 +420,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       L = fmaf(posts[w * kPostStride + kHeadDim + 1], sc, L);
       o.x = fmaf(v.x, sc, o.x); o.y = fmaf(v.y, sc, o.y); o.z = fmaf(v.z, sc, o.z); o.w = fmaf(v.w, sc, o.w);
     }
-    finish_head(a, bh0 + hh, split, n_splits, lane, M, L, o);
+    finish_head(a, bh0 + hh, split, n_splits, slot_stride, lane, M, L, o);
   }
   if (ticketed && threadIdx.x == 0 && blockIdx.x == gridDim.x - 1) {
     // The last CTA of the grid (its KV head is selected last, so it tends to finish last) tidies up: once every
@@ -531,7 +545,7 @@ cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* s
     if (e == cudaSuccess) e = make_row_map(&mv, a.v_g, rows);
   }
   if (e != cudaSuccess) return e;
-  const unsigned grid = (unsigned)attention_groups(geo, paged) * a.n_splits;
+  const unsigned grid = (unsigned)attention_groups(geo, paged) * a.n_splits + (unsigned)a.n_more;
   if (geo.S == 16)
     return paged ? launch_variant<16, true>(mk, mv, geo, a, status, grid, st, overlap, fused_resolve)
                  : launch_variant<16, false>(mk, mv, geo, a, status, grid, st, overlap, nullptr);

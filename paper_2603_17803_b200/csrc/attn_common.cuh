@@ -175,11 +175,11 @@ __device__ __forceinline__ void attend_unit(unsigned char* slot, int v16, bool h
 // warp that arrives last at the head's ticket (whichever CTA it sits in) merges the head's partials -- the heads
 // of a group are thus merged side by side, and nothing waits for a CTA-wide barrier or a staging copy.  The
 // finishing warp writes out / lse (and their host mirrors, counting the head as arrived there).
-__device__ __forceinline__ void finish_head(const AttnArgs& a, long long bh, int split, int n_splits, int lane, float M,
-                                            float L, float4 o) {
+// `n_splits`: page ranges of this head's group; `slot_stride`: partial slots per head (the launch's largest count).
+__device__ __forceinline__ void finish_head(const AttnArgs& a, long long bh, int split, int n_splits, int slot_stride,
+                                            int lane, float M, float L, float4 o) {
   bool finish = true;                                   // this warp writes the head's final result
   if (n_splits > 1) {
-    const int slot_stride = n_splits;
     const long long slot = bh * slot_stride + split;
     __stcg(reinterpret_cast<float4*>(a.part_acc + slot * kHeadDim) + lane, o);
     if (lane == 0) __stcg(reinterpret_cast<float2*>(a.part_ml + slot * 2), make_float2(M, L));

@@ -219,6 +219,7 @@ struct AttnArgs {
   float* out;
   float* lse;
   int n_splits;
+  int n_more;          // the last n_more groups are cut into n_splits + 1 ranges (a grid of whole waves), the others into n_splits
   HostMirror host{};
   StepTickets tk{nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
 };

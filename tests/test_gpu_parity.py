@@ -571,6 +571,9 @@ EDGE_SHAPES = {
     "k1_d1": small("c3_batched", batch=3, ctx_len=16 * 150 + 1, top_k=1, n_topics=4, n_queues=1, replication="one"),
     # group of 12 heads: a full head tile of 8 plus a partial one of 4
     "g12": small("c2_128k", batch=1, n_q_heads=24, n_kv_heads=2, ctx_len=16 * 400, top_k=40, n_topics=6),
+    # more (request, KV head) groups than fit one wave of attention CTAs with short page ranges: two waves, the
+    # last groups cut into one range more than the others
+    "two_waves": small("c3_batched", batch=12, ctx_len=16 * 300 + 7, top_k=128, n_topics=8),
 }
 
 
