@@ -96,6 +96,7 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.ctl = place(64 * 4);
   l.ready = place((int64_t)s.batch * head_pairs(s.n_kv_heads) * 4);
   l.sel_ready = place((int64_t)s.batch * s.n_kv_heads * 4);
+  l.selmap_ll = place(bh * selmap_pitch_bytes(s.max_pages_per_req) * 2);
   l.guard[l.n_guard++] = off;
   l.total = off + kGuardBytes;
   return l;
@@ -153,11 +154,17 @@ int pick_more(const swarm_ctx* ctx, bool paged, int n_splits, bool fused = false
 
 // The hand-off counters of a step (see StepTickets).  The scorer's tickets exist only when the streaming scorer
 // runs; `with_attention`: the selection also announces its heads to an attention kernel launched by the same call.
-StepTickets step_tickets(const swarm_ctx* ctx, const Geometry& g, bool with_attention) {
+// `bitmaps_by_word`: the page bitmaps go to the attention kernel as self-validating words instead of behind a
+// ticket per KV head -- for attention grids of one wave, where the step is a chain of latencies and the hand-off
+// is on it (128K tokens: 29.15 -> 28.64 us per step, 32K tokens: 18.1 -> 17.1); with several waves the CTAs
+// that wait would all be polling while the scorer and the selection still need the memory system (4 x 512K
+// tokens: 224.5 -> 226.5 us).
+StepTickets step_tickets(const swarm_ctx* ctx, const Geometry& g, bool with_attention, bool bitmaps_by_word = false) {
   StepTickets t;
   t.ctl = reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ctl);
   t.ready = score_raises_tickets(g) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ready) : nullptr;
   t.sel_ready = (with_attention && t.ready != nullptr) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.sel_ready) : nullptr;
+  t.selmap_ll = (t.sel_ready != nullptr && bitmaps_by_word) ? reinterpret_cast<uint2*>(ctx->ws + ctx->lay.selmap_ll) : nullptr;
   return t;
 }
 
@@ -630,7 +637,8 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   // which waits for all of the selection anyway
   const bool attn_tickets = whole && o->k_out == nullptr;
   TopkLinks links;
-  links.tk = step_tickets(ctx, ctx->geo, attn_tickets);
+  const bool one_wave = (long long)attention_groups(ctx->geo, true) * pick_splits(ctx, true, !tail) + (tail ? 0 : 1) <= sm_count();
+  links.tk = step_tickets(ctx, ctx->geo, attn_tickets, one_wave);
   links.req_base = in->page_base;
   links.flags_alt = tail ? ctx->lay.flags_alt : 0;
   if (parts & kStepBegin) {

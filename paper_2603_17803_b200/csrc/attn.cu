@@ -70,6 +70,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[kAttnWarps][kStages];
   __shared__ int s_wcnt[kAttnWarps];
+  __shared__ unsigned s_epoch;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int quad = lane >> 2, tq = lane & 3;            // MMA fragment coordinates of this lane
 
@@ -141,13 +142,22 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       qa[ks][1] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + tq * 2) : 0u;
     }
   };
+  const bool lines = ticketed && a.tk.selmap_ll != nullptr;   // the bitmaps arrive as self-validating words
   if (ticketed) {
     load_inputs();
     // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The CTA then
     // counts itself as past its wait (no result comes back: an atomic with one held the CTA's next barrier).
+    // With self-validating bitmaps there is no wait here: the threads look for their own words below, and what
+    // the count says is that the CTA has read the step's epoch (which it is made to wait for).
     if (threadIdx.x == 0) {
-      if (!wait_at_least(a.tk.sel_ready + (long long)b * geo.Hkv + kvh, (unsigned)geo.g)) atomicOr(status, SWARM_DEV_TIMEOUT);
-      red_relaxed_add(a.tk.ctl + kCtlAttnPast, 1u);
+      unsigned epoch = 0u;
+      if (lines) {
+        epoch = *reinterpret_cast<const volatile unsigned*>(a.tk.ctl + kCtlEpoch);
+        s_epoch = epoch + 1u;
+      } else if (!wait_at_least(a.tk.sel_ready + (long long)b * geo.Hkv + kvh, (unsigned)geo.g)) {
+        atomicOr(status, SWARM_DEV_TIMEOUT);
+      }
+      red_relaxed_add(a.tk.ctl + kCtlAttnPast, 1u + zero_after(epoch));
     }
     __syncthreads();
   } else {
@@ -165,6 +175,27 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   struct HeadWords { uint32_t v[8]; };
   auto load_raw = [&](int w) -> HeadWords {
     HeadWords hw;
+    if (lines) {
+      // {word, epoch} pairs written by selection CTAs that may still be running: all heads' pairs are asked for
+      // together and asked for again until every one carries this step's flag (bounded)
+      const unsigned flag = s_epoch;
+      const uint2* base = a.tk.selmap_ll + (long long)bh0 * pitch_words + w;
+      unsigned bad = 0u, polls = 0u;
+      do {
+        bad = 0u;
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          hw.v[hh] = 0u;
+          if (hh < G && w < pitch_words) {
+            const uint2 v = ll_word_load(base + (long long)hh * pitch_words);
+            hw.v[hh] = v.x;
+            bad |= v.y ^ flag;
+          }
+        }
+      } while (bad != 0u && ++polls < kLlWaitLimit);
+      if (bad != 0u) atomicOr(status, SWARM_DEV_TIMEOUT);
+      return hw;
+    }
 #pragma unroll
     for (int hh = 0; hh < 8; ++hh) {
       hw.v[hh] = 0u;
@@ -430,6 +461,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     const unsigned n_ctas = gridDim.x - (kFused != 0 ? 1u : 0u);
     if (!wait_at_least(a.tk.ctl + kCtlAttnPast, n_ctas) || !wait_zero(a.tk.ctl + kCtlTopkDone)) atomicOr(status, SWARM_DEV_TIMEOUT);
     for (int i = 0; i < geo.B * geo.Hkv; ++i) a.tk.sel_ready[i] = 0u;
+    if (lines) a.tk.ctl[kCtlEpoch] = s_epoch;            // one more step finished: its bitmap words no longer validate
     st_release(a.tk.ctl + kCtlAttnPast, 0u);
   }
   SWARM_STAMP_ANY_CTA(status, 6);

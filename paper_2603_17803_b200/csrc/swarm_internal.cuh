@@ -27,6 +27,7 @@ struct WorkspaceLayout {
   int64_t ctl;           // u32 [64]                   control words of the step's hand-offs, see StepTickets (zero at set-up)
   int64_t ready;         // u32 [B][head pairs]        score units complete (scorer -> selection; zero between steps)
   int64_t sel_ready;     // u32 [B][Hkv]               heads selected (selection -> attention; zero between steps)
+  int64_t selmap_ll;     // uint2 [B*Hq][pitch/4]      the page bitmaps as self-validating {word, epoch} pairs (zero at set-up)
   int64_t total;
   // 256 canary bytes sit in front of every region and behind the last one (kCanaryByte, written by
   // swarm_set_workspace; swarm_check_workspace reports the ones that no longer hold it)
@@ -41,8 +42,9 @@ constexpr int kCanaryByte = 0xA5;
 // waits (bounded) for the counter of exactly the data it reads:
 //   ready[b][hp]      the scorer adds 1 for every (16-page tile, KV head) of request b and KV-head pair hp whose
 //                     scores are stored; the selection of a head starts when its pair has all of them
-//   sel_ready[b][kv]  a selection CTA adds 1 when its head's page bitmap and cluster marks are stored; the
-//                     attention CTAs of (b, kv) start when all g heads have arrived
+//   sel_ready[b][kv]  a selection CTA adds 1 when its head's page bitmap is stored; the attention CTAs of (b, kv)
+//                     start when all g heads have arrived.  For attention grids of one wave the bitmaps travel
+//                     as self-validating words instead (selmap_ll, see ll_word_store) and this ticket is unused
 // Every wait is on a kernel launched earlier in the same stream whose CTAs are all resident (that is the
 // condition for the dependent launch), so no waiter can hold a resource the producer needs.  The counters are
 // set back to zero by the last CTA that needs them (ctl words count those).  A null pointer switches a
@@ -51,9 +53,11 @@ struct StepTickets {
   unsigned* ready;
   unsigned* sel_ready;
   unsigned* ctl;   // [0] selection CTAs finished; [1] attention CTAs past their wait; [2] steps whose cluster marks
-                   // are complete; [3] steps whose cluster resolution has finished ([2], [3]: overlapped tail only)
+                   // are complete; [3] steps whose cluster resolution has finished ([2], [3]: overlapped tail only);
+                   // [4] steps whose attention kernel has finished: the epoch of the self-validating bitmaps
+  uint2* selmap_ll;  // with sel_ready: the bitmaps travel as {word, epoch + 1} pairs instead (see ll_word_store)
 };
-constexpr int kCtlTopkDone = 0, kCtlAttnPast = 1, kCtlMarked = 2, kCtlResolved = 3;
+constexpr int kCtlTopkDone = 0, kCtlAttnPast = 1, kCtlMarked = 2, kCtlResolved = 3, kCtlEpoch = 4;
 constexpr unsigned kTicketWaitLimit = 1u << 22;            // polls, ~100 ns apart
 __host__ __device__ inline int head_pairs(int Hkv) { return (Hkv + 1) / 2; }
 
@@ -97,6 +101,30 @@ __device__ __forceinline__ bool wait_zero(const unsigned* p) {
 
 constexpr int kMaxSplits = 64;
 
+// Self-validating words.  Where a CTA that is already waiting is handed a few hundred bytes, a release / acquire
+// pair costs two more trips to L2 than the data: the release waits for the stores to be acknowledged, the
+// consumer polls the flag and only then fetches what it covers.  Instead every 32-bit word travels with its own
+// evidence in one 8-byte store (single-copy atomic): {word, flag}, the flag being the count of finished steps + 1
+// (never the 0 of fresh memory, never a value an earlier step wrote).  The consumer reads the pair with a volatile
+// load until the flag matches; no ordering between words is needed.  (Not ld.global.cg: on this part a repeated
+// .cg load of a line was served the first, stale answer about a million times in a row.)
+__device__ __forceinline__ void ll_word_store(uint2* p, uint32_t word, uint32_t flag) {
+  asm volatile("st.global.cg.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(word), "r"(flag) : "memory");
+}
+__device__ __forceinline__ uint2 ll_word_load(const uint2* p) {
+  uint2 v;
+  asm volatile("ld.volatile.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  return v;
+}
+constexpr unsigned kLlWaitLimit = 1u << 20;                // re-reads, each a trip to L2 (~0.7 us)
+// 0 that the compiler cannot tell from a value depending on x: added to an operand, it makes that instruction
+// wait for the load that produced x.
+__device__ __forceinline__ unsigned zero_after(unsigned x) {
+  unsigned z;
+  asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"(x));
+  return z;
+}
+
 // Row pitch of the per-head selection bitmap: one bit per page, rounded up to 16 bytes.
 __host__ __device__ inline int selmap_pitch_bytes(int Pmax) { return ((Pmax + 7) / 8 + 15) & ~15; }
 
@@ -133,7 +161,7 @@ cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint
 // `links`: how the kernel is tied to its neighbours (all zero: it waits for the whole previous kernel and
 // announces nothing).  tk.ready needs req_base (what the scorer was given as page_base).
 struct TopkLinks {
-  StepTickets tk{nullptr, nullptr, nullptr};
+  StepTickets tk{nullptr, nullptr, nullptr, nullptr};
   const int64_t* req_base = nullptr;
   long long flags_alt = 0;      // bytes between the two cluster-flag arrays of the overlapped tail, else 0
 };
@@ -210,6 +238,7 @@ struct AttnArgs {
   const int32_t* n_tok;
   const uint16_t* kv_pool;
   const uint8_t* selmap;   // paged mode: per (request, head) bitmap of selected pages, rows of selmap_pitch bytes
+                           // (with tk.selmap_ll: the same words as {word, epoch} pairs there instead)
   int selmap_pitch;
   const int64_t* page_base;
   const int32_t* ctx_len;
@@ -221,7 +250,7 @@ struct AttnArgs {
   int n_splits;
   int n_more;          // the last n_more groups are cut into n_splits + 1 ranges (a grid of whole waves), the others into n_splits
   HostMirror host{};
-  StepTickets tk{nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
+  StepTickets tk{nullptr, nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
 };
 // `fused_resolve` (paged mode only): one extra CTA of the grid runs cluster resolution with these arguments.
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,

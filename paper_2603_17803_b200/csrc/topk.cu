@@ -50,6 +50,7 @@ struct TopkExtras {
   const int64_t* req_base;        // [B+1] pages (or, for the medoid index, clusters) each request owns
   StepTickets tk;
   long long flags_alt;            // > 0: two flag arrays this many bytes apart, used by alternate steps (overlapped tail)
+  uint32_t ll_flag;               // with tk.selmap_ll: the flag this step's bitmap words carry (set by the kernel)
 };
 
 // What a selection CTA does before it reads its head's scores.  With tickets: one thread waits (bounded) until
@@ -77,8 +78,9 @@ __device__ __forceinline__ bool scores_ready(const Geometry& geo, const TopkExtr
       ok = wait_at_least(x.tk.ready + (long long)b * head_pairs(geo.Hkv) + hp, target);
       if (!ok) atomicOr(x.status, SWARM_DEV_TIMEOUT);
     }
-    // this CTA is past its wait (no result comes back: an atomic with one held the CTA's next barrier)
-    red_relaxed_add(x.tk.ctl + kCtlTopkDone, 1u);
+    // this CTA is past its wait (no result comes back: an atomic with one held the CTA's next barrier); the count
+    // also says that the CTA has read the step's epoch, which it is made to wait for
+    red_relaxed_add(x.tk.ctl + kCtlTopkDone, 1u + zero_after(x.ll_flag));
     *s_flag = ok;
   }
   __syncthreads();
@@ -90,7 +92,10 @@ __device__ __forceinline__ void write_empty_selection(const Geometry& geo, const
                                                       int32_t* n_sel, int threads) {
   for (int j = threadIdx.x; j < geo.k; j += threads) out[j] = -1;
   if (threadIdx.x == 0) n_sel[bh] = 0;
-  if (x.selmap != nullptr) {
+  if (x.tk.selmap_ll != nullptr) {
+    uint2* row = x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4);
+    for (int w = threadIdx.x; w < x.selmap_pitch / 4; w += threads) ll_word_store(row + w, 0u, x.ll_flag);
+  } else if (x.selmap != nullptr) {
     uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
     for (int o = threadIdx.x * 4; o + 4 <= x.selmap_pitch; o += threads * 4) *reinterpret_cast<uint32_t*>(row + o) = 0u;
   }
@@ -99,7 +104,7 @@ __device__ __forceinline__ void write_empty_selection(const Geometry& geo, const
 // The head's page bitmap is stored: announce it to the attention CTAs of its KV head (a barrier, then one
 // release that is cumulative over the CTA's stores so far).
 __device__ __forceinline__ void selection_announce(const Geometry& geo, const TopkExtras& x, int b, int kvh) {
-  if (x.tk.sel_ready == nullptr) return;
+  if (x.tk.sel_ready == nullptr || x.tk.selmap_ll != nullptr) return;   // (self-validating bitmaps announce themselves)
   __syncthreads();
   if (threadIdx.x == 0) red_release_add(x.tk.sel_ready + (long long)b * geo.Hkv + kvh, 1u);
 }
@@ -413,15 +418,32 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
     const unsigned bit = todo & (0u - todo);
     if ((gt_mask & bit) || eq_before + __popc(eq_mask & (bit - 1u)) < need_eq) picked |= bit;
   }
-  if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
-    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch + p0 / 8;
-    if (ITEMS == 8) *row = (uint8_t)picked;
-    else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
-  }
-  if (ITEMS < MAX_ITEMS && x.selmap != nullptr) {          // the part of the bitmap row these threads do not reach
-    uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
-    for (int o = THREADS * ITEMS / 8 + tid * 4; o + 4 <= x.selmap_pitch; o += THREADS * 4)
-      *reinterpret_cast<uint32_t*>(row + o) = 0u;
+  if (x.tk.selmap_ll != nullptr) {
+    // as {word, epoch} pairs: neighbouring lanes put their bytes together, the first of each group stores
+    uint2* row = x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4);
+    unsigned word = picked;
+    if (ITEMS == 8) {
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 8;
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 2) << 16;
+    } else {
+      word |= __shfl_down_sync(0xFFFFFFFFu, word, 1) << 16;
+    }
+    constexpr int kLanesPerWord = 32 / ITEMS;
+    const int w = tid / kLanesPerWord;
+    if (tid % kLanesPerWord == 0 && w < x.selmap_pitch / 4) ll_word_store(row + w, word, x.ll_flag);
+    if (ITEMS < MAX_ITEMS)                                 // the part of the bitmap row these threads do not reach
+      for (int w2 = THREADS * ITEMS / 32 + tid; w2 < x.selmap_pitch / 4; w2 += THREADS) ll_word_store(row + w2, 0u, x.ll_flag);
+  } else {
+    if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
+      uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch + p0 / 8;
+      if (ITEMS == 8) *row = (uint8_t)picked;
+      else *reinterpret_cast<uint16_t*>(row) = (uint16_t)picked;
+    }
+    if (ITEMS < MAX_ITEMS && x.selmap != nullptr) {        // the part of the bitmap row these threads do not reach
+      uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
+      for (int o = THREADS * ITEMS / 8 + tid * 4; o + 4 <= x.selmap_pitch; o += THREADS * 4)
+        *reinterpret_cast<uint32_t*>(row + o) = 0u;
+    }
   }
   selection_announce(geo, x, b, kvh);
   for (unsigned todo = picked; todo != 0u; todo &= todo - 1u) {
@@ -484,6 +506,8 @@ topk_regs_kernel(Geometry geo, const float* __restrict__ scores, const int32_t* 
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
   if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;   // stable: the previous step's selection has finished
+  // the step's epoch (stable too: the previous step's attention kernel, which raises it, has finished)
+  x.ll_flag = x.tk.selmap_ll != nullptr ? *reinterpret_cast<const volatile unsigned*>(x.tk.ctl + kCtlEpoch) + 1u : 0u;
   const int P = max(0, min(pages_of(len_b, geo.S), geo.Pmax));   // invalid lengths are reported by the scorer
   const int k_eff = min(geo.k, P);
   const int Pw = P - min(geo.W, P);                         // pages [Pw, P) are the local window: always kept
@@ -524,6 +548,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   const float* s = scores + (long long)bh * geo.Pmax;
   int32_t* out = sel + (long long)bh * geo.k;
   if (x.flags_alt > 0) x.flags += (x.tk.ctl[kCtlMarked] & 1u) * x.flags_alt;
+  x.ll_flag = x.tk.selmap_ll != nullptr ? *reinterpret_cast<const volatile unsigned*>(x.tk.ctl + kCtlEpoch) + 1u : 0u;
   if (!scores_ready(geo, x, b, kvh, len_b, &s_flag)) {
     write_empty_selection(geo, x, bh, out, n_sel, kGenericThreads);
     selection_announce(geo, x, b, kvh);
@@ -600,12 +625,17 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
       if (x.flags != nullptr) mark_cluster(geo, x, rb, i);
     }
     const unsigned word = __ballot_sync(0xFFFFFFFFu, take);
-    if (x.selmap != nullptr && lane == 0 && i0 / 8 + 4 <= x.selmap_pitch)
-      *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + i0 / 8) = word;
+    if (lane == 0 && i0 / 8 + 4 <= x.selmap_pitch) {
+      if (x.tk.selmap_ll != nullptr) ll_word_store(x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4) + i0 / 32, word, x.ll_flag);
+      else if (x.selmap != nullptr) *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + i0 / 8) = word;
+    }
     gt_before += __popc(bg);
     eq_before += __popc(be);
   }
-  if (x.selmap != nullptr) {                                // words past the last page of the request
+  if (x.tk.selmap_ll != nullptr) {                          // words past the last page of the request
+    for (int w = (P + 31) / 32 + tid; w < x.selmap_pitch / 4; w += kGenericThreads)
+      ll_word_store(x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4) + w, 0u, x.ll_flag);
+  } else if (x.selmap != nullptr) {
     const int first = ((P + 31) / 32) * 4;
     for (int o = first + tid * 4; o + 4 <= x.selmap_pitch; o += kGenericThreads * 4)
       *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + o) = 0u;
@@ -647,6 +677,8 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   x.tk = links.tk;
   x.flags_alt = flags != nullptr ? links.flags_alt : 0;
   if (x.req_base == nullptr) x.tk.ready = nullptr;         // the validity test of a request needs its page count
+  if (x.tk.ready == nullptr) x.tk.selmap_ll = nullptr;     // (the epoch is counted with the scorer's tickets)
+  x.ll_flag = 0u;
   // few lists: every thread reads the page -> cluster entries of all its pages up front (kEarly)
   const bool early = flags != nullptr && (long long)geo.B * geo.Hq <= 128;
   const dim3 grid(geo.B * geo.Hq);
