@@ -97,6 +97,7 @@ WorkspaceLayout make_layout(const swarm_shape& s) {
   l.ready = place((int64_t)s.batch * head_pairs(s.n_kv_heads) * 4);
   l.sel_ready = place((int64_t)s.batch * s.n_kv_heads * 4);
   l.selmap_ll = place(bh * selmap_pitch_bytes(s.max_pages_per_req) * 2);
+  l.scores_ll = place(bh <= kLlScoreLists ? bh * s.max_pages_per_req * 8 : 0);
   l.guard[l.n_guard++] = off;
   l.total = off + kGuardBytes;
   return l;
@@ -164,7 +165,11 @@ StepTickets step_tickets(const swarm_ctx* ctx, const Geometry& g, bool with_atte
   t.ctl = reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ctl);
   t.ready = score_raises_tickets(g) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.ready) : nullptr;
   t.sel_ready = (with_attention && t.ready != nullptr) ? reinterpret_cast<unsigned*>(ctx->ws + ctx->lay.sel_ready) : nullptr;
-  t.selmap_ll = (t.sel_ready != nullptr && bitmaps_by_word) ? reinterpret_cast<uint2*>(ctx->ws + ctx->lay.selmap_ll) : nullptr;
+  // (few lists: the instances of the selection kernel that carry the code for it, see launch_topk)
+  const bool few = (long long)g.B * g.Hq <= kLlScoreLists && g.Pmax <= 16384;
+  t.selmap_ll = (t.sel_ready != nullptr && bitmaps_by_word && few) ? reinterpret_cast<uint2*>(ctx->ws + ctx->lay.selmap_ll) : nullptr;
+  // ... and with an even row length (16-byte loads of two pairs) so do the scores
+  t.scores_ll = (t.selmap_ll != nullptr && g.Pmax % 2 == 0) ? reinterpret_cast<uint2*>(ctx->ws + ctx->lay.scores_ll) : nullptr;
   return t;
 }
 
@@ -644,7 +649,7 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   if (parts & kStepBegin) {
     SWARM_RANGE("swarm: score + select");
     SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
-                                status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail)));
+                                status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail), links.tk.scores_ll, links.tk.ctl));
     // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
     SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true, links,
                           ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,

@@ -224,10 +224,15 @@ __device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const in
 }
 
 // 128 registers: with 11 warps that leaves room on the SM for a 256-thread selection CTA beside this one.
+// kPairs: every score is also stored as a self-validating {score, epoch + 1} pair (few lists in a one-wave step:
+// the selection then reads those, waiting for no ticket); an instance of its own, so that the other one keeps the
+// register count that lets a selection CTA sit beside it.
+template <bool kPairs>
 __global__ void __maxnreg__(128)
 page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
-                      float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready) {
+                      float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready,
+                      uint2* __restrict__ scores_ll, const unsigned* __restrict__ ctl) {
   extern __shared__ unsigned char mma_smem_raw[];
   __shared__ __align__(8) uint64_t full[kMmaStages], empty[kMmaStages];
   __shared__ int s_cum[kStreamMaxBatch + 1];               // blocks before request b
@@ -402,6 +407,8 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   }
 
   // ---- consumers: warp w <-> (tile w / 2, head w % 2) of the block ----
+  // the flag of this step's self-validating scores (the epoch is stable: the previous step has finished)
+  const unsigned ll_flag = kPairs ? *reinterpret_cast<const volatile unsigned*>(ctl + kCtlEpoch) + 1u : 0u;
   const int quad = lane >> 2, tq = lane & 3;
   const int pt = warp / kBoxHeads, hl = warp % kBoxHeads;
   const int tiles = (geo.g + 7) / 8;                        // head tiles of 8 per KV head (N of the MMA)
@@ -496,7 +503,11 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int hh = 2 * tq + (e & 1), p = p0 + quad + (e >> 1) * 8;
-          if (hh < nh && p < P) scores[((long long)b * geo.Hq + h0 + hh) * geo.Pmax + p] = acc[e];
+          if (hh < nh && p < P) {
+            const long long at = ((long long)b * geo.Hq + h0 + hh) * geo.Pmax + p;
+            scores[at] = acc[e];
+            if (kPairs) ll_word_store(scores_ll + at, __float_as_uint(acc[e]), ll_flag);
+          }
         }
       }
     }
@@ -553,15 +564,18 @@ cudaError_t launch_one(const Geometry& geo, const uint16_t* q, const uint16_t* k
 
 cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
                        const int32_t* ctx_len, float* scores, uint32_t* status, unsigned* ready, int reserve_sms,
-                       cudaStream_t st) {
+                       uint2* scores_ll, const unsigned* ctl, cudaStream_t st) {
   CUtensorMap map;
   cudaError_t e = make_summary_map(&map, ksum, geo.Hkv, geo.n_pool_pages);
   if (e != cudaSuccess) return e;
   const long long max_blocks = (long long)geo.B * ((geo.Pmax + kBlkPages - 1) / kBlkPages) * head_pairs(geo.Hkv);
   const int sms = std::max(1, g_sm_count - reserve_sms);
   const int grid = (int)std::min<long long>(sms, std::max<long long>(1, max_blocks));
-  return launch_pdl(page_score_mma_kernel, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q, page_base,
-                    ctx_len, scores, status, ready);
+  if (scores_ll != nullptr && ctl != nullptr)
+    return launch_pdl(page_score_mma_kernel<true>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
+                      page_base, ctx_len, scores, status, ready, scores_ll, ctl);
+  return launch_pdl(page_score_mma_kernel<false>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
+                    page_base, ctx_len, scores, status, ready, static_cast<uint2*>(nullptr), static_cast<const unsigned*>(nullptr));
 }
 
 }  // namespace
@@ -573,7 +587,9 @@ cudaError_t configure_score() {
   if (e != cudaSuccess) return e;
   g_sm_count = sms > 0 ? sms : 148;
   if (summary_encode_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
-  return cudaFuncSetAttribute(page_score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
+  cudaError_t e2 = cudaFuncSetAttribute(page_score_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
+  if (e2 != cudaSuccess) return e2;
+  return cudaFuncSetAttribute(page_score_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
 }
 
 bool score_streams(const Geometry& geo) { return geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31); }
@@ -581,10 +597,10 @@ bool score_raises_tickets(const Geometry& geo) { return geo.scorer != SWARM_SCOR
 
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
-                              cudaStream_t st, unsigned* ready, int reserve_sms) {
+                              cudaStream_t st, unsigned* ready, int reserve_sms, uint2* scores_ll, const unsigned* ctl) {
   // Streaming tensor-core variant whenever the batch fits its prefix table and the pool fits 32-bit TMA
   // coordinates; otherwise the register-resident grid kernel on the fp32 pipes.
-  if (score_raises_tickets(geo)) return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, ready, reserve_sms, st);
+  if (score_raises_tickets(geo)) return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, ready, reserve_sms, scores_ll, ctl, st);
   // Heads of a KV group are processed G at a time, G the largest of 8/4/2/1 dividing the group size.
   if (geo.g % 8 == 0) return launch_one<8, 4, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);
   if (geo.g % 4 == 0) return launch_one<4, 8, 2>(geo, q, ksum, page_base, ctx_len, scores, status, st);

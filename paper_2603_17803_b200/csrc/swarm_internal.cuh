@@ -28,6 +28,8 @@ struct WorkspaceLayout {
   int64_t ready;         // u32 [B][head pairs]        score units complete (scorer -> selection; zero between steps)
   int64_t sel_ready;     // u32 [B][Hkv]               heads selected (selection -> attention; zero between steps)
   int64_t selmap_ll;     // uint2 [B*Hq][pitch/4]      the page bitmaps as self-validating {word, epoch} pairs (zero at set-up)
+  int64_t scores_ll;     // uint2 [B*Hq][Pmax]         the scores as {score, epoch} pairs (zero at set-up); only for shapes of
+                         //                            at most kLlScoreLists lists, else empty
   int64_t total;
   // 256 canary bytes sit in front of every region and behind the last one (kCanaryByte, written by
   // swarm_set_workspace; swarm_check_workspace reports the ones that no longer hold it)
@@ -56,7 +58,9 @@ struct StepTickets {
                    // are complete; [3] steps whose cluster resolution has finished ([2], [3]: overlapped tail only);
                    // [4] steps whose attention kernel has finished: the epoch of the self-validating bitmaps
   uint2* selmap_ll;  // with sel_ready: the bitmaps travel as {word, epoch + 1} pairs instead (see ll_word_store)
+  uint2* scores_ll;  // with selmap_ll: so do the scores, [B*Hq][Pmax] pairs; the selection then waits for no ticket
 };
+constexpr int kLlScoreLists = 128;                          // shapes with more lists keep the scorer's tickets
 constexpr int kCtlTopkDone = 0, kCtlAttnPast = 1, kCtlMarked = 2, kCtlResolved = 3, kCtlEpoch = 4;
 constexpr unsigned kTicketWaitLimit = 1u << 22;            // polls, ~100 ns apart
 __host__ __device__ inline int head_pairs(int Hkv) { return (Hkv + 1) / 2; }
@@ -151,17 +155,19 @@ cudaError_t launch_build_summaries(const Geometry& geo, const uint16_t* kv_pool,
 bool score_streams(const Geometry& geo);          // the shape allows the streaming tensor-core scorer
 bool score_raises_tickets(const Geometry& geo);   // ... and it is the one that will run: it counts its progress on `ready`
 // `ready` (StepTickets::ready, may be null) is raised by the streaming scorer only; `reserve_sms` SMs are left
-// free for the selection CTAs that wait on it.
+// free for the selection CTAs that wait on it.  `scores_ll` with `ctl` (StepTickets, may be null): the streaming
+// scorer also stores every score as a {score, epoch + 1} pair there.
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
-                              cudaStream_t st, unsigned* ready = nullptr, int reserve_sms = 0);
+                              cudaStream_t st, unsigned* ready = nullptr, int reserve_sms = 0, uint2* scores_ll = nullptr,
+                              const unsigned* ctl = nullptr);
 // `overlap`: launch with programmatic dependent launch after the previous kernel of the stream.
 // `selmap` (optional): per (request, head) bitmap of the selected pages, rows of selmap_pitch_bytes(Pmax).
 // `flags` with the three tables (optional): also mark the selected pages' clusters (see launch_resolve).
 // `links`: how the kernel is tied to its neighbours (all zero: it waits for the whole previous kernel and
 // announces nothing).  tk.ready needs req_base (what the scorer was given as page_base).
 struct TopkLinks {
-  StepTickets tk{nullptr, nullptr, nullptr, nullptr};
+  StepTickets tk{nullptr, nullptr, nullptr, nullptr, nullptr};
   const int64_t* req_base = nullptr;
   long long flags_alt = 0;      // bytes between the two cluster-flag arrays of the overlapped tail, else 0
 };
@@ -250,7 +256,7 @@ struct AttnArgs {
   int n_splits;
   int n_more;          // the last n_more groups are cut into n_splits + 1 ranges (a grid of whole waves), the others into n_splits
   HostMirror host{};
-  StepTickets tk{nullptr, nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
+  StepTickets tk{nullptr, nullptr, nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
 };
 // `fused_resolve` (paged mode only): one extra CTA of the grid runs cluster resolution with these arguments.
 cudaError_t launch_attention(const Geometry& geo, const AttnArgs& a, uint32_t* status, cudaStream_t st,

@@ -72,7 +72,7 @@ __device__ __forceinline__ bool scores_ready(const Geometry& geo, const TopkExtr
   if (threadIdx.x == 0) {
     const int P = pages_of(len_b, geo.S);
     bool ok = len_b >= 1 && P <= geo.Pmax && (long long)P <= x.req_base[b + 1] - x.req_base[b];
-    if (ok) {
+    if (ok && x.tk.scores_ll == nullptr) {                 // (self-validating scores are waited for one by one, by their readers)
       const int hp = kvh / 2;
       const unsigned target = (unsigned)((P + 15) / 16) * (unsigned)min(2, geo.Hkv - 2 * hp);
       ok = wait_at_least(x.tk.ready + (long long)b * head_pairs(geo.Hkv) + hp, target);
@@ -307,7 +307,31 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
   if (!scores_ready(geo, x, b, kvh, len_b, s_flag)) return false;   // the scores come from the previous kernel
   SWARM_STAMP(status, 1);
   const bool full = p0 + ITEMS <= Pw;                       // all of this thread's pages exist and are scored: no per-page checks
-  if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
+  if (kEarly && x.tk.scores_ll != nullptr) {             // (few lists only, like kEarly: see launch_topk)
+    // {score, epoch} pairs that the scorer may still be writing: all of this thread's pairs are asked for together
+    // (two per 16-byte load: the row length is even) and asked for again until every existing page's carries this
+    // step's flag (bounded)
+    const uint2* pairs = x.tk.scores_ll + (long long)bh * geo.Pmax + p0;
+    unsigned bad = 0u, polls = 0u;
+    do {
+      bad = 0u;
+#pragma unroll
+      for (int j = 0; j < ITEMS; j += 2) {
+        key[j] = key[j + 1] = 0u;
+        if (p0 + j < P) {
+          uint4 v;
+          asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(pairs + j) : "memory");
+          key[j] = score_key(__uint_as_float(v.x));
+          bad |= v.y ^ x.ll_flag;
+          if (p0 + j + 1 < P) {
+            key[j + 1] = score_key(__uint_as_float(v.z));
+            bad |= v.w ^ x.ll_flag;
+          }
+        }
+      }
+    } while (bad != 0u && ++polls < kLlWaitLimit);
+    if (bad != 0u) atomicOr(x.status, SWARM_DEV_TIMEOUT);
+  } else if (p0 + ITEMS <= P && (geo.Pmax & 3) == 0) {
 #pragma unroll
     for (int j = 0; j < ITEMS; j += 4) {
       const float4 v = __ldcg(reinterpret_cast<const float4*>(s + p0 + j));   // written by a kernel that may still run: not through L1
@@ -418,7 +442,7 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
     const unsigned bit = todo & (0u - todo);
     if ((gt_mask & bit) || eq_before + __popc(eq_mask & (bit - 1u)) < need_eq) picked |= bit;
   }
-  if (x.tk.selmap_ll != nullptr) {
+  if (kEarly && x.tk.selmap_ll != nullptr) {              // (few lists only, like kEarly: see launch_topk)
     // as {word, epoch} pairs: neighbouring lanes put their bytes together, the first of each group stores
     uint2* row = x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4);
     unsigned word = picked;
@@ -677,10 +701,14 @@ cudaError_t launch_topk(const Geometry& geo, const float* scores, const int32_t*
   x.tk = links.tk;
   x.flags_alt = flags != nullptr ? links.flags_alt : 0;
   if (x.req_base == nullptr) x.tk.ready = nullptr;         // the validity test of a request needs its page count
-  if (x.tk.ready == nullptr) x.tk.selmap_ll = nullptr;     // (the epoch is counted with the scorer's tickets)
+  if (x.tk.ready == nullptr) x.tk.selmap_ll = x.tk.scores_ll = nullptr;     // (the epoch is counted with the scorer's tickets)
   x.ll_flag = 0u;
   // few lists: every thread reads the page -> cluster entries of all its pages up front (kEarly)
   const bool early = flags != nullptr && (long long)geo.B * geo.Hq <= 128;
+  // Only the few-lists instances of the register-resident kernel carry the code for self-validating words (the
+  // others keep the register count that lets a 256-thread CTA sit beside a scorer CTA); callers ask for them only
+  // where these instances run (step_tickets).
+  if ((x.tk.selmap_ll != nullptr || x.tk.scores_ll != nullptr) && (!early || geo.Pmax > 16384)) return cudaErrorInvalidValue;
   const dim3 grid(geo.B * geo.Hq);
 #define SWARM_TOPK_REGS(THREADS, ITEMS)                                                                           \
   return early ? launch_pdl(topk_regs_kernel<THREADS, ITEMS, true>, grid, dim3(THREADS), 0, st, overlap, geo, scores, \
