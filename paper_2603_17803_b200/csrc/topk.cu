@@ -95,7 +95,8 @@ __device__ __forceinline__ void write_empty_selection(const Geometry& geo, const
   if (x.tk.selmap_ll != nullptr) {
     uint2* row = x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4);
     for (int w = threadIdx.x; w < x.selmap_pitch / 4; w += threads) ll_word_store(row + w, 0u, x.ll_flag);
-  } else if (x.selmap != nullptr) {
+  }
+  if (x.selmap != nullptr) {
     uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch;
     for (int o = threadIdx.x * 4; o + 4 <= x.selmap_pitch; o += threads * 4) *reinterpret_cast<uint32_t*>(row + o) = 0u;
   }
@@ -457,7 +458,8 @@ __device__ __forceinline__ bool topk_regs_body(SelectState& st, const Geometry& 
     if (tid % kLanesPerWord == 0 && w < x.selmap_pitch / 4) ll_word_store(row + w, word, x.ll_flag);
     if (ITEMS < MAX_ITEMS)                                 // the part of the bitmap row these threads do not reach
       for (int w2 = THREADS * ITEMS / 32 + tid; w2 < x.selmap_pitch / 4; w2 += THREADS) ll_word_store(row + w2, 0u, x.ll_flag);
-  } else {
+  }
+  {                                                        // the plain bitmap (behind the pairs, if any: later calls read it)
     if (x.selmap != nullptr && p0 < x.selmap_pitch * 8) {
       uint8_t* row = x.selmap + (long long)bh * x.selmap_pitch + p0 / 8;
       if (ITEMS == 8) *row = (uint8_t)picked;
@@ -651,7 +653,7 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
     const unsigned word = __ballot_sync(0xFFFFFFFFu, take);
     if (lane == 0 && i0 / 8 + 4 <= x.selmap_pitch) {
       if (x.tk.selmap_ll != nullptr) ll_word_store(x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4) + i0 / 32, word, x.ll_flag);
-      else if (x.selmap != nullptr) *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + i0 / 8) = word;
+      if (x.selmap != nullptr) *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + i0 / 8) = word;
     }
     gt_before += __popc(bg);
     eq_before += __popc(be);
@@ -659,7 +661,8 @@ topk_generic_kernel(Geometry geo, const float* __restrict__ scores, const int32_
   if (x.tk.selmap_ll != nullptr) {                          // words past the last page of the request
     for (int w = (P + 31) / 32 + tid; w < x.selmap_pitch / 4; w += kGenericThreads)
       ll_word_store(x.tk.selmap_ll + (long long)bh * (x.selmap_pitch / 4) + w, 0u, x.ll_flag);
-  } else if (x.selmap != nullptr) {
+  }
+  if (x.selmap != nullptr) {
     const int first = ((P + 31) / 32) * 4;
     for (int o = first + tid * 4; o + 4 <= x.selmap_pitch; o += kGenericThreads * 4)
       *reinterpret_cast<uint32_t*>(x.selmap + (long long)bh * x.selmap_pitch + o) = 0u;

@@ -517,6 +517,26 @@ def test_paged_attention_alone_matches_gathered_attention():
     sess.close()
 
 
+@pytest.mark.parametrize("name", ["c1_small", "c2_small", "c3_small", "c5_small"])
+def test_paged_attention_reuses_the_bitmaps_a_step_left(name):
+    """A fused step hands its page bitmaps to its own attention kernel in whichever form is fastest; whatever
+    that is, a later swarm_sparse_attn_paged without a selection finds them in the workspace."""
+    w = W.generate(CASES[name], seed=16, device=DEV)
+    sess = Session(w)
+    sess.step()
+    sess.step()
+    torch.cuda.synchronize()
+    out, lse = sess.o.out.clone(), sess.o.lse.clone()
+    sess.o.out.zero_()
+    sess.o.lse.zero_()
+    sess.sparse_attn_paged(reuse_last_selection=True)
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    assert (sess.o.out - out).abs().max().item() <= 1e-5 and (sess.o.lse - lse).abs().max().item() <= 1e-5
+    parity.check_step(w, sess)
+    sess.close()
+
+
 @pytest.mark.parametrize("name", ["c3_small", "c5_small"])
 def test_resident_filter_and_cache_counters(name):
     """Eq. 8 with the resident term, activation frequencies and Eq. 6 scores, against the oracle on the GPU's
