@@ -47,11 +47,16 @@ constexpr int kAttnSmemBytes = 1024 /*alignment slack*/ + kRingBytes + kScratchB
 // the attention CTAs -- 1: plain, 2: with cache state.  As a kernel of its own on a second stream the serial
 // pass stalled for about 2 us each time the attention kernel started or retired; as one more CTA of the same
 // grid it does not, and the step needs neither the second stream nor its two events.
-template <int S, bool kPaged, int kFused>
+// kMode = kFused + 4 * kLines.  kLines (inside a step with a one-wave grid and few lists only): the page bitmaps
+// arrive as self-validating words (StepTickets::selmap_ll); instances of their own, because the kernel sits at its
+// register limit and the other instances must not pay for the polling code.
+template <int S, bool kPaged, int kMode>
 __global__ void __launch_bounds__(kAttnWarps * 32, 1)
 attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Geometry geo,
             AttnArgs a, uint32_t* __restrict__ status, const __grid_constant__ ResolveArgs rs) {
-  static_assert(kFused == 0 || kPaged, "cluster resolution rides with the paged kernel only");
+  constexpr int kFused = kMode & 3;
+  constexpr bool kLines = (kMode & 4) != 0;
+  static_assert(kMode == 0 || kPaged, "cluster resolution and word-wise bitmaps ride with the paged kernel only");
   static_assert(resolve_detail::kThreads <= kAttnWarps * 32, "the resolution body runs in a CTA of this kernel");
   if (kFused != 0 && blockIdx.x == 0) {
     // (the body is written for kThreads threads; the CTA's other warps leave, and a CTA-wide barrier counts the
@@ -142,7 +147,7 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
       qa[ks][1] = row_ok ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + tq * 2) : 0u;
     }
   };
-  const bool lines = ticketed && a.tk.selmap_ll != nullptr;   // the bitmaps arrive as self-validating words
+  const bool lines = kLines;                            // the bitmaps arrive as self-validating words (then `ticketed` holds)
   if (ticketed) {
     load_inputs();
     // The selection kernel may still be running: wait for the heads of this CTA's KV head only.  The CTA then
@@ -520,10 +525,15 @@ cudaError_t launch_variant(const CUtensorMap& mk, const CUtensorMap& mv, const G
                            uint32_t* status, unsigned grid, cudaStream_t st, bool overlap, const ResolveArgs* rs) {
   const dim3 block(kAttnWarps * 32);
   if constexpr (kPaged) {
+    const bool lines = a.tk.sel_ready != nullptr && a.tk.selmap_ll != nullptr;
     if (rs != nullptr && rs->has_cache)
-      return launch_pdl(attn_kernel<S, true, 2>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
+      return lines ? launch_pdl(attn_kernel<S, true, 6>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs)
+                   : launch_pdl(attn_kernel<S, true, 2>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
     if (rs != nullptr)
-      return launch_pdl(attn_kernel<S, true, 1>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
+      return lines ? launch_pdl(attn_kernel<S, true, 5>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs)
+                   : launch_pdl(attn_kernel<S, true, 1>, dim3(grid + 1), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, *rs);
+    if (lines)
+      return launch_pdl(attn_kernel<S, true, 4>, dim3(grid), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status, ResolveArgs{});
   }
   return launch_pdl(attn_kernel<S, kPaged, 0>, dim3(grid), block, kAttnSmemBytes, st, overlap, mk, mv, geo, a, status,
                     ResolveArgs{});
@@ -542,6 +552,12 @@ cudaError_t configure_attention() {
   cudaError_t e = allow_smem(attn_kernel<16, true, 0>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 1>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 2>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 4>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 5>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<16, true, 6>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 4>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 5>);
+  if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 6>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<16, false, 0>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 0>);
   if (e == cudaSuccess) e = allow_smem(attn_kernel<32, true, 1>);
