@@ -47,7 +47,7 @@ extern "C" {
 #define SWARM_DEV_BAD_CLUSTER 2u        /* page2cluster entry outside the request's cluster range  */
 #define SWARM_DEV_BAD_REPLICA 4u        /* replica mask is 0 or names a queue >= n_queues          */
 #define SWARM_DEV_BAD_LENGTH 8u         /* ctx_len < 1 or more pages than the request owns         */
-#define SWARM_DEV_TIMEOUT 16u           /* a bounded wait on an asynchronous copy expired          */
+#define SWARM_DEV_TIMEOUT 16u           /* a bounded wait expired (a copy, or a hand-off between kernels) */
 
 /* ---- flags in swarm_shape.flags --------------------------------------------------------- */
 #define SWARM_ORDER_BY_ID 1u            /* schedule clusters by id only (default: by number of
