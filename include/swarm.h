@@ -211,6 +211,18 @@ int32_t swarm_set_select_sms(swarm_ctx* ctx, int32_t n_sms);
 #define SWARM_SCORER_FP32 2
 int32_t swarm_set_scorer(swarm_ctx* ctx, int32_t kind);
 
+/* Index prefetch (off by default).  The page index (inputs->ksum, located through ctx_len and page_base) does not
+ * depend on the queries (Sec. 4.2, Tier 1: it is built when pages are written).  With `on` != 0 the scoring kernel
+ * of swarm_step / swarm_step_begin asks for its first blocks of it as soon as its CTAs are resident, before it
+ * waits for the work that precedes the step in the stream -- in a chain of steps: while the previous step's
+ * attention kernel merges its partial results -- and the attention kernel of a step lets the next kernel's CTAs
+ * become resident as soon as its own have read all their pages.  Everything that reads q (scoring itself,
+ * selection, attention) still starts after the preceding work has completed.
+ * The caller vouches that the operation enqueued directly before the step in its stream writes none of ksum,
+ * ctx_len and page_base (an index update for newly written pages goes at least one operation earlier, or the
+ * switch stays off).  Results do not depend on it. */
+int32_t swarm_set_index_prefetch(swarm_ctx* ctx, int32_t on);
+
 /* Index build (not part of a decode step): per page and KV head, element-wise min and max of
  * the valid tokens' keys -- the compact index the scorer reads instead of the keys themselves
  * (the role the in-memory cluster index plays in Sec. 4.2, Tier 1).

@@ -26,7 +26,7 @@ _ERR_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "
 
 EXPORTS = (
     "swarm_version", "swarm_create", "swarm_destroy", "swarm_workspace_bytes", "swarm_set_workspace",
-    "swarm_check_workspace", "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_tail_stream", "swarm_tail_join", "swarm_set_select_sms", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
+    "swarm_check_workspace", "swarm_set_attn_splits", "swarm_set_scorer", "swarm_set_index_prefetch", "swarm_set_tail_stream", "swarm_tail_join", "swarm_set_select_sms", "swarm_set_cache", "swarm_build_summaries", "swarm_select", "swarm_resolve_clusters", "swarm_gather",
     "swarm_sparse_attn", "swarm_sparse_attn_paged", "swarm_sparse_attn_static", "swarm_sparse_attn_static_status", "swarm_step", "swarm_step_host", "swarm_device_status", "swarm_last_cuda_error",
     "swarm_build_medoid_index", "swarm_step_medoid", "swarm_set_submit_order",
     "swarm_build_clusters_workspace_bytes", "swarm_build_clusters",
@@ -191,6 +191,10 @@ def swarm_set_select_sms(ctx, n_sms: int) -> None:
 
 def swarm_set_scorer(ctx, kind: int) -> None:
     _check(load_library().swarm_set_scorer(ctx, ctypes.c_int32(kind)), "swarm_set_scorer", ctx)
+
+
+def swarm_set_index_prefetch(ctx, on: bool) -> None:
+    _check(load_library().swarm_set_index_prefetch(ctx, ctypes.c_int32(1 if on else 0)), "swarm_set_index_prefetch", ctx)
 
 
 def swarm_set_cache(ctx, *, resident=None, freq=None, score=None, n_hit=None, t_base=0.0, t_transfer=0.0) -> None:

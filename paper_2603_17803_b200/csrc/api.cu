@@ -33,6 +33,7 @@ struct swarm_ctx {
   int64_t ws_bytes;
   int user_splits;            // 0 = chosen from the shape
   int select_sms;             // SMs the scorer leaves to the selection CTAs; < 0 = chosen from the shape
+  bool index_prefetch;        // swarm_set_index_prefetch
   cudaStream_t tail_stream;   // swarm_set_tail_stream: where swarm_step enqueues cluster resolution (null: inside the step)
   cudaEvent_t ev_selected;    // recorded on the step's stream behind the selection; the tail stream waits for it
   cudaEvent_t ev_resolved;    // recorded on the tail stream behind the resolution; swarm_tail_join waits for it
@@ -280,6 +281,7 @@ int32_t swarm_create(const swarm_shape* shape, swarm_ctx** out_ctx) {
   ctx->ws_bytes = 0;
   ctx->user_splits = 0;
   ctx->select_sms = -1;
+  ctx->index_prefetch = false;
   ctx->tail_stream = nullptr;
   ctx->ev_selected = nullptr;
   ctx->ev_resolved = nullptr;
@@ -401,6 +403,13 @@ int32_t swarm_set_scorer(swarm_ctx* ctx, int32_t kind) {
   if (ctx == nullptr || kind < SWARM_SCORER_AUTO || kind > SWARM_SCORER_FP32) return SWARM_ERR_INVALID_ARG;
   if (kind == SWARM_SCORER_TENSOR && !score_streams(ctx->geo)) return SWARM_ERR_UNSUPPORTED;
   ctx->geo.scorer = kind;
+  if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
+  return SWARM_OK;
+}
+
+int32_t swarm_set_index_prefetch(swarm_ctx* ctx, int32_t on) {
+  if (ctx == nullptr) return SWARM_ERR_INVALID_ARG;
+  ctx->index_prefetch = on != 0;
   if (ctx->host_graph != nullptr) { cudaGraphExecDestroy(ctx->host_graph); ctx->host_graph = nullptr; }
   return SWARM_OK;
 }
@@ -649,7 +658,8 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
   if (parts & kStepBegin) {
     SWARM_RANGE("swarm: score + select");
     SWARM_TRY(launch_page_score(ctx->geo, q, static_cast<const uint16_t*>(in->ksum), in->page_base, in->ctx_len, sc,
-                                status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail), links.tk.scores_ll, links.tk.ctl));
+                                status, st, links.tk.ready, reserved_sms(ctx, ctx->geo, tail), links.tk.scores_ll, links.tk.ctl,
+                                ctx->index_prefetch));
     // the selection kernel also marks the selected pages' clusters and writes the per-head page bitmaps
     SWARM_TRY(launch_topk(ctx->geo, sc, in->ctx_len, o->sel, o->n_sel, status, st, true, links,
                           ws_ptr<uint8_t>(ctx, ctx->lay.selmap), in->page_base, in->page2cluster, in->cluster_base,
@@ -682,6 +692,10 @@ int32_t step_impl(swarm_ctx* ctx, const swarm_inputs* in, const swarm_outputs* o
     ctx->tail_pending = true;
     a.n_splits = pick_splits(ctx, true, /*fused=*/false);
     a.n_more = pick_more(ctx, true, a.n_splits, /*fused=*/false);
+    // With the index prefetch the SMs the attention CTAs leave are worth something to the next step's scorer
+    // (its CTAs fetch their first blocks there): they are released as soon as the CTAs have read all their pages.
+    // (Without it the early release was measured 1.5 us slower: the scorer's CTAs only sat there.)
+    a.release_early = ctx->index_prefetch && attn_tickets;
     SWARM_TRY(launch_attention(ctx->geo, a, status, st, /*overlap=*/true, nullptr));
     return SWARM_OK;
   }

@@ -408,6 +408,9 @@ attn_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
   }
   SWARM_STAMP(status, 4);
   SWARM_STAMP_ANY_CTA(status, 7);
+  // All pages read.  Inside a chain of steps the next kernel's CTAs may now take the SMs that CTAs of this kernel
+  // leave: they wait for this kernel's completion before they touch anything that depends on it.
+  if (kFused == 0 && ticketed && a.release_early) pdl_launch_dependents();
 
   // ---- merge the warps of the CTA ---------------------------------------------------------------------
   // Every warp posts its (max, sum) per head and its raw accumulators into its own ring (idle now: all its copies

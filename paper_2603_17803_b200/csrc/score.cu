@@ -232,7 +232,7 @@ __global__ void __maxnreg__(128)
 page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
                       float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready,
-                      uint2* __restrict__ scores_ll, const unsigned* __restrict__ ctl) {
+                      uint2* __restrict__ scores_ll, const unsigned* __restrict__ ctl, int index_early) {
   extern __shared__ unsigned char mma_smem_raw[];
   __shared__ __align__(8) uint64_t full[kMmaStages], empty[kMmaStages];
   __shared__ int s_cum[kStreamMaxBatch + 1];               // blocks before request b
@@ -255,13 +255,18 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   }
   // Launched with programmatic serialization behind whatever precedes it in the stream -- inside a chain of
   // steps the previous step's attention kernel -- so that this kernel's launch and set-up overlap that kernel's
-  // tail.  Nothing a predecessor may have written (q, lengths, tables, summaries) is read before this point.
+  // tail.  Nothing a predecessor may have written is read before the wait.  With `index_early` the caller vouches
+  // that the predecessor writes neither the lengths, nor the page bases, nor the summaries: the CTA then lays out
+  // its blocks and its producer asks for the first ones before the wait -- they do not depend on the queries --
+  // and everything that touches q, the scores or the tickets still comes after it.
   SWARM_STAMP(status, 0);
-  pdl_wait();
-  SWARM_STAMP(status, 1);
-  // Only now may the selection kernel be scheduled: its CTAs poll the tickets this kernel raises, and tickets
-  // of the previous step are guaranteed to be cleared only once everything before this kernel has finished.
-  pdl_launch_dependents();
+  if (!index_early) {
+    pdl_wait();
+    SWARM_STAMP(status, 1);
+    // Only now may the selection kernel be scheduled: its CTAs poll the tickets this kernel raises, and tickets
+    // of the previous step are guaranteed to be cleared only once everything before this kernel has finished.
+    pdl_launch_dependents();
+  }
   if (warp == 1) {                                         // blocks per request, prefix by one warp
     int running = 0;
     for (int b0 = 0; b0 < geo.B; b0 += 32) {
@@ -327,6 +332,11 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       }
     }
     return;
+  }
+  if (index_early) {                                       // (the producer above reads nothing that depends on a predecessor)
+    pdl_wait();
+    SWARM_STAMP(status, 1);
+    pdl_launch_dependents();
   }
   if (warp == kMmaConsumers + 2) {
     // ---- weight warp: the second arrival on every slot's `full` barrier ----
@@ -470,8 +480,15 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + pt * kTileBytes);
       for (int ht = 0; ht < tiles; ++ht) {
         const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
-        if (w_rows > 0) load_weights_slot(stage, nh);
-        else if ((long long)b * geo.Hq + h0 != w_key) load_weights_global(b, h0, nh);
+        // (consecutive blocks of a CTA mostly belong to the same request and pair: the operand registers are kept)
+        if (w_rows > 0) {
+          if ((long long)b * geo.Hq + h0 != w_key) {
+            load_weights_slot(stage, nh);
+            w_key = (long long)b * geo.Hq + h0;
+          }
+        } else if ((long long)b * geo.Hq + h0 != w_key) {
+          load_weights_global(b, h0, nh);
+        }
         // A tiles: 16 pages x 16 coordinates per k-step; matrices (rows 0-7 | 8-15) x (chunk 2ks | 2ks+1).  Eight
         // tiles are fetched before the MMAs that use them, and the MMAs alternate between two accumulators: issued
         // one by one, every MMA waited for its own ldmatrix and for the MMA before it (~0.5 us per block).
@@ -564,7 +581,7 @@ cudaError_t launch_one(const Geometry& geo, const uint16_t* q, const uint16_t* k
 
 cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* ksum, const int64_t* page_base,
                        const int32_t* ctx_len, float* scores, uint32_t* status, unsigned* ready, int reserve_sms,
-                       uint2* scores_ll, const unsigned* ctl, cudaStream_t st) {
+                       uint2* scores_ll, const unsigned* ctl, bool early, cudaStream_t st) {
   CUtensorMap map;
   cudaError_t e = make_summary_map(&map, ksum, geo.Hkv, geo.n_pool_pages);
   if (e != cudaSuccess) return e;
@@ -573,9 +590,9 @@ cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* k
   const int grid = (int)std::min<long long>(sms, std::max<long long>(1, max_blocks));
   if (scores_ll != nullptr && ctl != nullptr)
     return launch_pdl(page_score_mma_kernel<true>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
-                      page_base, ctx_len, scores, status, ready, scores_ll, ctl);
+                      page_base, ctx_len, scores, status, ready, scores_ll, ctl, early ? 1 : 0);
   return launch_pdl(page_score_mma_kernel<false>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
-                    page_base, ctx_len, scores, status, ready, static_cast<uint2*>(nullptr), static_cast<const unsigned*>(nullptr));
+                    page_base, ctx_len, scores, status, ready, static_cast<uint2*>(nullptr), static_cast<const unsigned*>(nullptr), early ? 1 : 0);
 }
 
 }  // namespace
@@ -597,10 +614,11 @@ bool score_raises_tickets(const Geometry& geo) { return geo.scorer != SWARM_SCOR
 
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
-                              cudaStream_t st, unsigned* ready, int reserve_sms, uint2* scores_ll, const unsigned* ctl) {
+                              cudaStream_t st, unsigned* ready, int reserve_sms, uint2* scores_ll, const unsigned* ctl,
+                              bool index_early) {
   // Streaming tensor-core variant whenever the batch fits its prefix table and the pool fits 32-bit TMA
   // coordinates; otherwise the register-resident grid kernel on the fp32 pipes.
-  if (score_raises_tickets(geo)) return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, ready, reserve_sms, scores_ll, ctl, st);
+  if (score_raises_tickets(geo)) return launch_mma(geo, q, ksum, page_base, ctx_len, scores, status, ready, reserve_sms, scores_ll, ctl, index_early, st);
   // Heads of a KV group are processed G at a time, G the largest of 8/4/2/1 dividing the group size.
   if (geo.g % 8 == 0) return launch_one<8, 4, 4>(geo, q, ksum, page_base, ctx_len, scores, status, st);
   if (geo.g % 4 == 0) return launch_one<4, 8, 2>(geo, q, ksum, page_base, ctx_len, scores, status, st);

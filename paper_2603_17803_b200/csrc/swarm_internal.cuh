@@ -156,11 +156,13 @@ bool score_streams(const Geometry& geo);          // the shape allows the stream
 bool score_raises_tickets(const Geometry& geo);   // ... and it is the one that will run: it counts its progress on `ready`
 // `ready` (StepTickets::ready, may be null) is raised by the streaming scorer only; `reserve_sms` SMs are left
 // free for the selection CTAs that wait on it.  `scores_ll` with `ctl` (StepTickets, may be null): the streaming
-// scorer also stores every score as a {score, epoch + 1} pair there.
+// scorer also stores every score as a {score, epoch + 1} pair there.  `index_early`: the streaming scorer's CTAs ask
+// for their first blocks of `ksum` -- located through ctx_len and page_base -- before they wait for what precedes
+// the kernel in the stream (the caller vouches that it writes none of the three).
 cudaError_t launch_page_score(const Geometry& geo, const uint16_t* q, const uint16_t* ksum,
                               const int64_t* page_base, const int32_t* ctx_len, float* scores, uint32_t* status,
                               cudaStream_t st, unsigned* ready = nullptr, int reserve_sms = 0, uint2* scores_ll = nullptr,
-                              const unsigned* ctl = nullptr);
+                              const unsigned* ctl = nullptr, bool index_early = false);
 // `overlap`: launch with programmatic dependent launch after the previous kernel of the stream.
 // `selmap` (optional): per (request, head) bitmap of the selected pages, rows of selmap_pitch_bytes(Pmax).
 // `flags` with the three tables (optional): also mark the selected pages' clusters (see launch_resolve).
@@ -255,6 +257,7 @@ struct AttnArgs {
   float* lse;
   int n_splits;
   int n_more;          // the last n_more groups are cut into n_splits + 1 ranges (a grid of whole waves), the others into n_splits
+  bool release_early = false;   // inside a step: the CTAs let the next kernel's CTAs become resident once they have read all their pages
   HostMirror host{};
   StepTickets tk{nullptr, nullptr, nullptr, nullptr, nullptr};   // paged mode inside a step: wait per KV head for the selection (sel_ready, ctl)
 };

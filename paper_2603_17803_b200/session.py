@@ -34,7 +34,8 @@ class Session:
 
     def __init__(self, workload, *, flags: int = 0, keep_scores: bool = False, keep_gathered: bool = False,
                  ksum: Optional[torch.Tensor] = None, local_window_pages: int = 0,
-                 max_clusters_total: Optional[int] = None, scorer: int = B.SCORER_AUTO, tail_stream=None):
+                 max_clusters_total: Optional[int] = None, scorer: int = B.SCORER_AUTO, tail_stream=None,
+                 index_prefetch: bool = False):
         cfg = workload.cfg
         self.cfg = cfg
         self.w = workload
@@ -53,6 +54,8 @@ class Session:
         B.swarm_set_workspace(self.ctx, self.workspace)
         if scorer != B.SCORER_AUTO:
             B.swarm_set_scorer(self.ctx, scorer)
+        if index_prefetch:                       # the workload's index and lengths are written once, before any step
+            B.swarm_set_index_prefetch(self.ctx, True)
         self.tail_stream = tail_stream
         if tail_stream is not None:
             B.swarm_set_tail_stream(self.ctx, tail_stream)

@@ -537,6 +537,42 @@ def test_paged_attention_reuses_the_bitmaps_a_step_left(name):
     sess.close()
 
 
+@pytest.mark.parametrize("name", ["c1_small", "c2_small", "c3_small", "c4_small", "c5_small"])
+@pytest.mark.parametrize("tail", [False, True])
+def test_index_prefetch_changes_no_result(name, tail):
+    """swarm_set_index_prefetch: the scorer asks for its first index blocks before it waits for the previous
+    step's attention kernel (which releases its SMs early for it).  Back-to-back steps with the switch on give the
+    results of the switch off, bit for bit, and match the oracle."""
+    w = W.generate(CASES[name], seed=17, device=DEV)
+    tstream = torch.cuda.Stream() if tail else None
+    ref = Session(w, tail_stream=tstream)
+    for _ in range(2):
+        ref.step()
+    if tail:
+        ref.tail_join()
+    torch.cuda.synchronize()
+    sess = Session(w, ksum=ref.ksum, tail_stream=tstream, index_prefetch=True)
+    for _ in range(4):                                     # each step's scorer is launched behind the previous step's attention
+        sess.step()
+    if tail:
+        sess.tail_join()
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    for key in ("sel", "n_sel", "out", "lse"):
+        assert torch.equal(getattr(ref.o, key), getattr(sess.o, key)), key
+    n_q = w.cfg.n_queues
+    assert int(ref.o.n_uniq[0]) == int(sess.o.n_uniq[0]) and torch.equal(ref.o.queue_load[:n_q], sess.o.queue_load[:n_q])
+    parity.check_step(w, sess)
+    B.swarm_set_index_prefetch(sess.ctx, False)            # and off again
+    sess.step()
+    if tail:
+        sess.tail_join()
+    torch.cuda.synchronize()
+    assert sess.status() == 0 and torch.equal(ref.o.out, sess.o.out)
+    sess.close()
+    ref.close()
+
+
 @pytest.mark.parametrize("name", ["c3_small", "c5_small"])
 def test_resident_filter_and_cache_counters(name):
     """Eq. 8 with the resident term, activation frequencies and Eq. 6 scores, against the oracle on the GPU's
