@@ -227,12 +227,12 @@ __device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const in
 // kPairs: every score is also stored as a self-validating {score, epoch + 1} pair (few lists in a one-wave step:
 // the selection then reads those, waiting for no ticket); an instance of its own, so that the other one keeps the
 // register count that lets a selection CTA sit beside it.
-template <bool kPairs>
+template <bool kPairs, bool kEarly>
 __global__ void __maxnreg__(128)
 page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, const uint16_t* __restrict__ q,
                       const int64_t* __restrict__ page_base, const int32_t* __restrict__ ctx_len,
                       float* __restrict__ scores, uint32_t* __restrict__ status, unsigned* __restrict__ ready,
-                      uint2* __restrict__ scores_ll, const unsigned* __restrict__ ctl, int index_early) {
+                      uint2* __restrict__ scores_ll, const unsigned* __restrict__ ctl) {
   extern __shared__ unsigned char mma_smem_raw[];
   __shared__ __align__(8) uint64_t full[kMmaStages], empty[kMmaStages];
   __shared__ int s_cum[kStreamMaxBatch + 1];               // blocks before request b
@@ -255,12 +255,12 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   }
   // Launched with programmatic serialization behind whatever precedes it in the stream -- inside a chain of
   // steps the previous step's attention kernel -- so that this kernel's launch and set-up overlap that kernel's
-  // tail.  Nothing a predecessor may have written is read before the wait.  With `index_early` the caller vouches
+  // tail.  Nothing a predecessor may have written is read before the wait.  In the kEarly instances the caller vouches
   // that the predecessor writes neither the lengths, nor the page bases, nor the summaries: the CTA then lays out
   // its blocks and its producer asks for the first ones before the wait -- they do not depend on the queries --
   // and everything that touches q, the scores or the tickets still comes after it.
   SWARM_STAMP(status, 0);
-  if (!index_early) {
+  if (!kEarly) {
     pdl_wait();
     SWARM_STAMP(status, 1);
     // Only now may the selection kernel be scheduled: its CTAs poll the tickets this kernel raises, and tickets
@@ -333,7 +333,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     }
     return;
   }
-  if (index_early) {                                       // (the producer above reads nothing that depends on a predecessor)
+  if (kEarly) {                                            // (the producer above reads nothing that depends on a predecessor)
     pdl_wait();
     SWARM_STAMP(status, 1);
     pdl_launch_dependents();
@@ -480,15 +480,8 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
       const uint32_t base = sm_addr(ring + (size_t)stage * kMmaStageBytes + pt * kTileBytes);
       for (int ht = 0; ht < tiles; ++ht) {
         const int h0 = kvh * geo.g + ht * 8, nh = min(8, geo.g - ht * 8);
-        // (consecutive blocks of a CTA mostly belong to the same request and pair: the operand registers are kept)
-        if (w_rows > 0) {
-          if ((long long)b * geo.Hq + h0 != w_key) {
-            load_weights_slot(stage, nh);
-            w_key = (long long)b * geo.Hq + h0;
-          }
-        } else if ((long long)b * geo.Hq + h0 != w_key) {
-          load_weights_global(b, h0, nh);
-        }
+        if (w_rows > 0) load_weights_slot(stage, nh);
+        else if ((long long)b * geo.Hq + h0 != w_key) load_weights_global(b, h0, nh);
         // A tiles: 16 pages x 16 coordinates per k-step; matrices (rows 0-7 | 8-15) x (chunk 2ks | 2ks+1).  Eight
         // tiles are fetched before the MMAs that use them, and the MMAs alternate between two accumulators: issued
         // one by one, every MMA waited for its own ldmatrix and for the MMA before it (~0.5 us per block).
@@ -588,11 +581,15 @@ cudaError_t launch_mma(const Geometry& geo, const uint16_t* q, const uint16_t* k
   const long long max_blocks = (long long)geo.B * ((geo.Pmax + kBlkPages - 1) / kBlkPages) * head_pairs(geo.Hkv);
   const int sms = std::max(1, g_sm_count - reserve_sms);
   const int grid = (int)std::min<long long>(sms, std::max<long long>(1, max_blocks));
+  const dim3 g(grid), b(kMmaThreads);
+  const size_t smem = mma_smem_bytes(geo.g);
+  uint2* no_pairs = nullptr;
+  const unsigned* no_ctl = nullptr;
   if (scores_ll != nullptr && ctl != nullptr)
-    return launch_pdl(page_score_mma_kernel<true>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
-                      page_base, ctx_len, scores, status, ready, scores_ll, ctl, early ? 1 : 0);
-  return launch_pdl(page_score_mma_kernel<false>, dim3(grid), dim3(kMmaThreads), mma_smem_bytes(geo.g), st, true, map, geo, q,
-                    page_base, ctx_len, scores, status, ready, static_cast<uint2*>(nullptr), static_cast<const unsigned*>(nullptr), early ? 1 : 0);
+    return early ? launch_pdl(page_score_mma_kernel<true, true>, g, b, smem, st, true, map, geo, q, page_base, ctx_len, scores, status, ready, scores_ll, ctl)
+                 : launch_pdl(page_score_mma_kernel<true, false>, g, b, smem, st, true, map, geo, q, page_base, ctx_len, scores, status, ready, scores_ll, ctl);
+  return early ? launch_pdl(page_score_mma_kernel<false, true>, g, b, smem, st, true, map, geo, q, page_base, ctx_len, scores, status, ready, no_pairs, no_ctl)
+               : launch_pdl(page_score_mma_kernel<false, false>, g, b, smem, st, true, map, geo, q, page_base, ctx_len, scores, status, ready, no_pairs, no_ctl);
 }
 
 }  // namespace
@@ -604,9 +601,12 @@ cudaError_t configure_score() {
   if (e != cudaSuccess) return e;
   g_sm_count = sms > 0 ? sms : 148;
   if (summary_encode_fn() == nullptr) return cudaErrorNotSupported;   // resolved here, not inside a stream capture
-  cudaError_t e2 = cudaFuncSetAttribute(page_score_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
-  if (e2 != cudaSuccess) return e2;
-  return cudaFuncSetAttribute(page_score_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(kWeightRowsMax / 2));
+  const int smem = mma_smem_bytes(kWeightRowsMax / 2);
+  cudaError_t e2 = cudaFuncSetAttribute(page_score_mma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(page_score_mma_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(page_score_mma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(page_score_mma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  return e2;
 }
 
 bool score_streams(const Geometry& geo) { return geo.B <= kStreamMaxBatch && geo.n_pool_pages < (1LL << 31); }
