@@ -210,16 +210,25 @@ __device__ __forceinline__ bool sm_try_wait(uint64_t* bar, unsigned parity) {
 struct ScoreBlock {
   int b, hp, page0, n_tiles, P;   // request, KV-head pair, first page (request-local), tiles that exist, pages of the request
 };
-__device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const int* s_cum, const int32_t* __restrict__ ctx_len, int S) {
+__device__ __forceinline__ ScoreBlock locate_block(int blk, int& cur_b, const int* s_cum, const int32_t* __restrict__ ctx_len, int S,
+                                                   int hpairs) {
   while (s_cum[cur_b + 1] <= blk) ++cur_b;
   ScoreBlock k;
   k.b = cur_b;
-  k.P = pages_of(ctx_len[cur_b], S);
-  const int per_pair = (k.P + kBlkPages - 1) / kBlkPages;
+  // blocks per pair from the table; the request's length is fetched only for the last block of a pair (the only
+  // one that can be partial): a fetch per block sat at the top of every warp's loop
+  const int per_pair = (s_cum[cur_b + 1] - s_cum[cur_b]) / hpairs;
   const int c = blk - s_cum[cur_b];
   k.hp = c / per_pair;
-  k.page0 = (c - k.hp * per_pair) * kBlkPages;
-  k.n_tiles = min(kBlkTiles, (k.P - k.page0 + kMmaPages - 1) / kMmaPages);
+  const int j = c - k.hp * per_pair;
+  k.page0 = j * kBlkPages;
+  if (j + 1 < per_pair) {
+    k.P = per_pair * kBlkPages;                              // (an upper bound does: every page of this block exists)
+    k.n_tiles = kBlkTiles;
+  } else {
+    k.P = pages_of(ctx_len[cur_b], S);
+    k.n_tiles = min(kBlkTiles, (k.P - k.page0 + kMmaPages - 1) / kMmaPages);
+  }
   return k;
 }
 
@@ -312,7 +321,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           while (!sm_try_wait(&empty[stage], parity) && ++polls < kStreamWaitLimit && !s_abort) {}
           if (polls >= kStreamWaitLimit || s_abort) { atomicOr(status, SWARM_DEV_TIMEOUT); s_abort = 1; break; }
         }
-        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S, hpairs);
         const int page0 = (int)(page_base[blk.b] + blk.page0);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&full[stage])),
                      "r"((unsigned)(blk.n_tiles * kTileBytes))
@@ -346,7 +355,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
     int fb = 0;
     for (int k = 0; k < n_blk; ++k) {
       const int stage = k % kMmaStages;
-      const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+      const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S, hpairs);
       const int n_chunks = w_rows > 0 ? min(kBoxHeads, geo.Hkv - blk.hp * kBoxHeads) * geo.g * 16 : 0;
       const uint16_t* qpair = q + ((long long)blk.b * geo.Hq + (long long)blk.hp * kBoxHeads * geo.g) * kHeadDim;
       uint4 v[kWeightRowsMax * 16 / 32];
@@ -408,7 +417,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
           __nanosleep(64);
         } while (++polls < kStreamWaitLimit && !s_abort);
         if (seen < want) break;                             // the consumers gave up (they have set the status bit)
-        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S);
+        const ScoreBlock blk = locate_block(blk_first + k * blk_step, fb, s_cum, ctx_len, geo.S, hpairs);
         const unsigned units = (unsigned)blk.n_tiles * (unsigned)min(kBoxHeads, geo.Hkv - blk.hp * kBoxHeads);
         red_release_add(ready + (long long)blk.b * hpairs + blk.hp, units);
       }
@@ -458,7 +467,7 @@ page_score_mma_kernel(const __grid_constant__ CUtensorMap map, Geometry geo, con
   };
   for (int k = 0; k < n_blk; ++k) {
     const int stage = k % kMmaStages;
-    const ScoreBlock blk = locate_block(blk_first + k * blk_step, cur_b, s_cum, ctx_len, geo.S);
+    const ScoreBlock blk = locate_block(blk_first + k * blk_step, cur_b, s_cum, ctx_len, geo.S, hpairs);
     const int b = blk.b, P = blk.P;
     const int kvh = blk.hp * kBoxHeads + hl;
     const bool active = kvh < geo.Hkv && pt < blk.n_tiles;
