@@ -55,6 +55,15 @@ def test_shape_validation_runs_without_a_gpu(lib_path):
     assert e.value.code == B.ERR_INVALID_ARG
 
 
+def test_switches_reject_a_null_ctx_without_a_gpu(lib_path):
+    """The ctx switches validate their arguments on the host (no CUDA call is made for a null ctx)."""
+    lib = ctypes.CDLL(lib_path)
+    for name in ("swarm_set_index_prefetch", "swarm_set_scorer", "swarm_set_select_sms", "swarm_set_attn_splits"):
+        fn = getattr(lib, name)
+        fn.restype = ctypes.c_int32
+        assert fn(None, ctypes.c_int32(1)) == 1, name      # SWARM_ERR_INVALID_ARG
+
+
 def test_struct_layouts_match_the_header():
     from paper_2603_17803_b200 import binding as B
     assert ctypes.sizeof(B.swarm_shape) == 56          # 9 x int32 + uint32 + int64 + 2 x int32
